@@ -1,0 +1,179 @@
+"""SpQt CPU oracle (ctypes front end of ``spqt_oracle.c``) -- TEST INFRASTRUCTURE.
+
+Only ``tests/``, ``__graft_entry__.smoke()`` and the ``cpu_baseline`` /
+``--impl reference`` legs of ``bench.py`` may import this package.  It shares
+nothing with the CUDA library: the layout and the quantizer are restated in
+``spqt_oracle.c`` from the paper (Sec. 2, Sec. 4.1.2, Sec. 4.2.3), not included
+from it.  Arrays are numpy; fp16 values travel as ``numpy.float16``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "spqt_oracle.c")
+_LIB = os.path.join(_HERE, "libspqt_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (fp contraction off, so every quantizer step
+    is one IEEE fp32 operation).  Returns the path of the shared object."""
+    stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+    if force or stale:
+        tmp = _LIB + ".%d.tmp" % os.getpid()
+        cmd = ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-fopenmp",
+               "-shared", "-fPIC", "-o", tmp, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    with _lock:
+        if _lib is None:
+            lib = ctypes.CDLL(build())
+            lib.spqt_oracle_block_bytes.restype = ctypes.c_size_t
+            lib.spqt_oracle_threads.restype = ctypes.c_int
+            _lib = lib
+    return _lib
+
+
+def _p(a):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _check(rc, what):
+    if rc != 0:
+        raise ValueError("oracle %s rejected its arguments (code %d)" % (what, rc))
+
+
+def _u16(a):
+    a = np.ascontiguousarray(a)
+    assert a.dtype == np.float16, a.dtype
+    return a.view(np.uint16)
+
+
+def block_bytes(bits: int, group: int) -> int:
+    return int(_load().spqt_oracle_block_bytes(int(bits), int(group)))
+
+
+def half_to_float(h_bits: np.ndarray) -> np.ndarray:
+    h = np.ascontiguousarray(h_bits, dtype=np.uint16)
+    out = np.empty(h.shape, np.float32)
+    _load().spqt_oracle_half_to_float(_p(h), _p(out), ctypes.c_size_t(h.size))
+    return out
+
+
+def float_to_half(f: np.ndarray) -> np.ndarray:
+    f = np.ascontiguousarray(f, dtype=np.float32)
+    out = np.empty(f.shape, np.uint16)
+    _load().spqt_oracle_float_to_half(_p(f), _p(out), ctypes.c_size_t(f.size))
+    return out
+
+
+def quantize(W: np.ndarray, bits: int = 4, group: int = 128):
+    """fp16 W[m][n] -> (q uint8[m][n] natural order, scales fp16[R][n], zeros fp16[R][n])."""
+    Wb = _u16(W)
+    m, n = Wb.shape
+    R = m // group if group else 0
+    q = np.empty((m, n), np.uint8)
+    s = np.empty((max(R, 0), n), np.uint16)
+    z = np.empty((max(R, 0), n), np.uint16)
+    _check(_load().spqt_oracle_quantize(_p(Wb), m, n, n, bits, group, _p(q), _p(s), _p(z)), "quantize")
+    return q, s.view(np.float16), z.view(np.float16)
+
+
+def pack_codes(q: np.ndarray, bits: int = 4, group: int = 128) -> np.ndarray:
+    q = np.ascontiguousarray(q, dtype=np.uint8)
+    m, n = q.shape
+    codes = np.empty((m // group) * n * block_bytes(bits, group), np.uint8)
+    _check(_load().spqt_oracle_pack_codes(_p(q), m, n, bits, group, _p(codes)), "pack_codes")
+    return codes
+
+
+def unpack_codes(codes: np.ndarray, m: int, n: int, bits: int = 4, group: int = 128) -> np.ndarray:
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    assert codes.size == (m // group) * n * block_bytes(bits, group)
+    q = np.empty((m, n), np.uint8)
+    _check(_load().spqt_oracle_unpack_codes(_p(codes), m, n, bits, group, _p(q)), "unpack_codes")
+    return q
+
+
+def pack(W: np.ndarray, bits: int = 4, group: int = 128):
+    """fp16 W[m][n] -> (codes uint8[R*n*B] zigzag, scales fp16[R][n], zeros fp16[R][n])."""
+    q, s, z = quantize(W, bits, group)
+    return pack_codes(q, bits, group), s, z
+
+
+def dequantize(codes, scales, zeros, m, n, bits=4, group=128) -> np.ndarray:
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    out = np.empty((m, n), np.float64)
+    _check(_load().spqt_oracle_dequantize(_p(codes), _p(_u16(scales)), _p(_u16(zeros)),
+                                          m, n, bits, group, _p(out)), "dequantize")
+    return out
+
+
+def sparsify(x: np.ndarray, t: float):
+    """fp16 x[n], threshold t -> (idx int32[count] ascending, count)."""
+    xb = _u16(x)
+    n = xb.size
+    idx = np.empty(max(n, 1), np.int32)
+    cnt = np.zeros(1, np.int32)
+    _check(_load().spqt_oracle_sparsify(_p(xb), n, ctypes.c_float(t), _p(idx), _p(cnt)), "sparsify")
+    c = int(cnt[0])
+    return idx[:c].copy(), c
+
+
+def _rows_arg(rows, m):
+    if rows is None:
+        return None, 0, m
+    rows = np.ascontiguousarray(rows, dtype=np.int32)
+    return rows, rows.size, rows.size
+
+
+def sparse_gemv(codes, scales, zeros, m, n, x, idx, bits=4, group=128, rows=None):
+    """-> (y float64[rows], bound float64[rows]); bound = sum |What||x| over the listed columns."""
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    rows_a, n_rows, out_n = _rows_arg(rows, m)
+    y = np.empty(out_n, np.float64)
+    b = np.empty(out_n, np.float64)
+    rc = _load().spqt_oracle_sparse_gemv(
+        _p(codes), _p(_u16(scales)), _p(_u16(zeros)), m, n, bits, group, _p(_u16(x)),
+        _p(idx), int(idx.size), _p(rows_a) if rows_a is not None else None, n_rows, _p(y), _p(b))
+    _check(rc, "sparse_gemv")
+    return y, b
+
+
+def dense_gemv(codes, scales, zeros, m, n, x, bits=4, group=128, rows=None):
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    rows_a, n_rows, out_n = _rows_arg(rows, m)
+    y = np.empty(out_n, np.float64)
+    b = np.empty(out_n, np.float64)
+    rc = _load().spqt_oracle_dense_gemv(
+        _p(codes), _p(_u16(scales)), _p(_u16(zeros)), m, n, bits, group, _p(_u16(x)),
+        _p(rows_a) if rows_a is not None else None, n_rows, _p(y), _p(b))
+    _check(rc, "dense_gemv")
+    return y, b
+
+
+def partition(count: int, S: int) -> np.ndarray:
+    out = np.empty(S + 1, np.int32)
+    _check(_load().spqt_oracle_partition(int(count), int(S), _p(out)), "partition")
+    return out
+
+
+def threads() -> int:
+    return int(_load().spqt_oracle_threads())
+
+
+def set_threads(t: int) -> None:
+    _load().spqt_oracle_set_threads(int(t))

@@ -1,0 +1,349 @@
+"""Pins for the CPU oracle: every check here compares the oracle with something
+other than itself -- a hand-worked example, a closed form, a library routine,
+exact integer/rational arithmetic, or an invariant the mathematics fixes."""
+import math
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+import oracle
+from conftest import read_golden
+from paper_2511_04477_b200 import inputs
+
+
+# ------------------------------------------------------------------ fp16 conversions
+
+def test_half_to_float_matches_numpy_exhaustively():
+    bits = np.arange(65536, dtype=np.uint16)
+    mine = oracle.half_to_float(bits)
+    ref = bits.view(np.float16).astype(np.float32)
+    nan = np.isnan(ref)
+    assert np.array_equal(np.isnan(mine), nan)
+    assert np.array_equal(mine[~nan].view(np.uint32), ref[~nan].view(np.uint32))
+
+
+def test_float_to_half_matches_numpy():
+    g = np.random.Generator(np.random.PCG64(7))
+    # random bit patterns cover every exponent; add the rounding boundaries explicitly
+    f = g.integers(0, 2**32, size=2_000_000, dtype=np.uint64).astype(np.uint32).view(np.float32)
+    h = np.arange(65536, dtype=np.uint16).view(np.float16).astype(np.float32)
+    h = h[np.isfinite(h)]
+    up = np.nextafter(h, np.float32(np.inf))
+    mid = ((h.astype(np.float64) + np.roll(h, -1).astype(np.float64)) / 2).astype(np.float32)
+    edge = np.array([65504, 65519.996, 65520, 65536, 1e-8, 2.0**-25, 2.0**-24, 3 * 2.0**-25,
+                     2.0**-14, 2.0**-14 - 2.0**-25, 0.0, -0.0, np.inf, -np.inf], dtype=np.float32)
+    allf = np.concatenate([f, h, up, mid, -mid, edge])
+    allf = allf[~np.isnan(allf)]
+    with np.errstate(over="ignore"):
+        ref = allf.astype(np.float16).view(np.uint16)
+    assert np.array_equal(oracle.float_to_half(allf), ref)
+
+
+# ------------------------------------------------------------------ hand-worked example
+
+def test_hand_example_quantizer_and_layout(hand_example):
+    e = hand_example
+    q, s, z = oracle.quantize(e["W"], e["bits"], e["group"])
+    assert np.array_equal(q, e["q"])
+    assert np.array_equal(s.astype(np.float64), e["scales"])
+    assert np.array_equal(z.astype(np.float64), e["zeros"])
+    assert s[0, 2].view(np.uint16) == 0x3266
+    codes = oracle.pack_codes(q, e["bits"], e["group"])
+    assert codes.tolist() == e["codes"].tolist()
+    assert np.array_equal(oracle.unpack_codes(e["codes"], e["m"], e["n"], e["bits"], e["group"]), e["q"])
+
+
+def test_hand_example_sparse_and_dense_gemv(hand_example):
+    e = hand_example
+    codes, s, z = oracle.pack(e["W"], e["bits"], e["group"])
+    idx, count = oracle.sparsify(e["x"], e["t"])
+    assert count == 2 and idx.tolist() == e["idx"].tolist()
+    y, bound = oracle.sparse_gemv(codes, s, z, e["m"], e["n"], e["x"], idx, e["bits"], e["group"])
+    assert np.array_equal(y, e["y_sparse"])            # exact, not approximate
+    yd, _ = oracle.dense_gemv(codes, s, z, e["m"], e["n"], e["x"], e["bits"], e["group"])
+    assert np.array_equal(yd, e["y_dense"])
+    # bound of row 0: |0|*1 + |2|*2 = 4 ; row 7: |0.875|*1 + |-1.5|*2 = 3.875
+    assert bound[0] == 4.0 and bound[7] == 3.875
+
+
+def test_int3_block_bytes_match_hand_packing():
+    g = read_golden("int3_block.txt")
+    G, bits = int(g["group"][0][0]), int(g["bits"][0][0])
+    col = np.array([[float(v)] for v in g["column"][0]], dtype=np.float16)
+    q, s, z = oracle.quantize(col, bits, G)
+    assert q[:, 0].tolist() == list(range(8))
+    assert float(s[0, 0]) == float(g["scale"][0][0]) and float(z[0, 0]) == float(g["zero"][0][0])
+    codes = oracle.pack_codes(q, bits, G)
+    assert codes.tolist() == [int(v, 16) for v in g["codes"][0]]
+    assert oracle.block_bytes(3, 128) == 48 and oracle.block_bytes(3, 64) == 24
+    assert oracle.block_bytes(4, 128) == 64 and oracle.block_bytes(4, 64) == 32
+
+
+# ------------------------------------------------------------------ layout structure
+
+@pytest.mark.parametrize("bits,group", [(4, 128), (4, 64), (3, 128), (3, 64), (4, 6), (3, 16)])
+def test_pack_unpack_round_trip_bit_exact(bits, group):
+    g = np.random.Generator(np.random.PCG64(bits * 1000 + group))
+    m, n = 3 * group, 37
+    q = g.integers(0, 1 << bits, size=(m, n), dtype=np.uint8)
+    codes = oracle.pack_codes(q, bits, group)
+    assert codes.size == 3 * n * group * bits // 8
+    assert np.array_equal(oracle.unpack_codes(codes, m, n, bits, group), q)
+
+
+@pytest.mark.parametrize("bits,group", [(4, 128), (3, 64)])
+def test_block_of_row_j_column_k_lives_at_r_times_n_plus_k(bits, group):
+    """Zigzag order: changing one weight's code touches only bytes of block (j//G, k),
+    and block index is r*n + k (row-major over (block-row, column))."""
+    m, n = 2 * group, 9
+    B = oracle.block_bytes(bits, group)
+    base = oracle.pack_codes(np.zeros((m, n), np.uint8), bits, group)
+    assert not base.any()
+    for (j, k) in [(0, 0), (5, 3), (group - 1, 8), (group, 0), (group + 17, 4), (2 * group - 1, 8)]:
+        q = np.zeros((m, n), np.uint8)
+        q[j, k] = (1 << bits) - 1
+        changed = np.nonzero(oracle.pack_codes(q, bits, group))[0]
+        blk = (j // group) * n + k
+        assert changed.size > 0
+        assert changed.min() >= blk * B and changed.max() < (blk + 1) * B
+    # int4: byte i of a block = row i in the low nibble, row i + G/2 in the high nibble
+    if bits == 4:
+        q = np.zeros((m, n), np.uint8)
+        q[3, 2] = 0x9
+        q[3 + group // 2, 2] = 0x6
+        c = oracle.pack_codes(q, bits, group)
+        assert c[(0 * n + 2) * B + 3] == 0x69
+
+
+# ------------------------------------------------------------------ quantizer invariants
+
+@pytest.mark.parametrize("bits,group", [(4, 128), (4, 64), (3, 128), (3, 64)])
+def test_quantizer_invariants(bits, group):
+    qmax = (1 << bits) - 1
+    W = inputs.weights(2 * group, 96, seed=11 + bits + group)
+    W[:group, 5] = np.float16(0.03125)                     # a constant group
+    q, s, z = oracle.quantize(W, bits, group)
+    Wf = W.astype(np.float64)
+    for r in range(2):
+        blk = Wf[r * group:(r + 1) * group]
+        assert np.array_equal(z[r].astype(np.float64), blk.min(axis=0))          # offset = group min
+        qb = q[r * group:(r + 1) * group]
+        amin, amax = blk.argmin(axis=0), blk.argmax(axis=0)
+        cols = np.arange(W.shape[1])
+        sf = s[r].astype(np.float64)
+        assert np.all(qb[amin, cols] == 0)                                       # min -> code 0
+        assert np.all((qb[amax, cols] == qmax) | (sf == 0))                      # max -> qmax
+        deq = sf[None, :] * qb + z[r].astype(np.float64)[None, :]
+        assert np.all(np.abs(deq - blk) <= sf[None, :] / 2 * (1 + 2.0**-10) + 1e-300)
+        # scale is the fp16 rounding of range/qmax computed in fp32
+        rng32 = (blk.max(axis=0).astype(np.float32) - blk.min(axis=0).astype(np.float32))
+        assert np.array_equal(s[r], (rng32 / np.float32(qmax)).astype(np.float16))
+    assert s[0, 5] == 0 and not q[:group, 5].any() and float(z[0, 5]) == 0.03125
+    assert q.max() <= qmax
+    # power-of-two scaling leaves the codes alone and scales s and z
+    q2, s2, z2 = oracle.quantize((W.astype(np.float32) * 4).astype(np.float16), bits, group)
+    assert np.array_equal(q2, q)
+    assert np.array_equal(s2.astype(np.float32), s.astype(np.float32) * 4)
+    assert np.array_equal(z2.astype(np.float32), z.astype(np.float32) * 4)
+
+
+def test_quantizer_codes_match_numpy_single_precision_steps():
+    """Same steps taken with numpy's IEEE float32 ufuncs (a different engine)."""
+    bits, group, qmax = 4, 128, 15
+    W = inputs.weights(256, 64, seed=3)
+    q, s, z = oracle.quantize(W, bits, group)
+    w32 = W.astype(np.float32).reshape(2, group, 64)
+    lo = w32.min(axis=1, keepdims=True)
+    sf = s.astype(np.float32)[:, None, :]
+    with np.errstate(divide="ignore", invalid="ignore"):
+        ref = np.clip(np.rint((w32 - lo) / sf), 0, qmax)
+    ref = np.where(sf == 0, 0, ref).astype(np.uint8).reshape(256, 64)
+    assert np.array_equal(q, ref)
+
+
+def test_lossless_family_is_reproduced_exactly():
+    W = inputs.lossless_weights(256, 40)
+    codes, s, z = oracle.pack(W, 4, 128)
+    assert np.all(s.astype(np.float64) == 1 / 16) and not z.any()
+    assert np.array_equal(oracle.dequantize(codes, s, z, 256, 40, 4, 128), W.astype(np.float64))
+
+
+def test_expected_scale_for_gaussian_weights():
+    """W ~ N(0, 0.02^2), G = 128: E[range] = 2*E[max of 128 normals]*sigma ~ 5.2 sigma,
+    so the mean scale is about 5.2*0.02/15 ~ 0.0069."""
+    _, s, _ = oracle.quantize(inputs.weights(128 * 8, 512, seed=0), 4, 128)
+    assert abs(float(s.astype(np.float64).mean()) - 0.0069) < 3e-4
+
+
+# ------------------------------------------------------------------ dequantize / GEMV definitions
+
+def _setup(m, n, bits, group, seed, dist="laplace", **kw):
+    W = inputs.weights(m, n, seed)
+    x = inputs.activations(n, seed + 100, dist, **kw)
+    q, s, z = oracle.quantize(W, bits, group)
+    codes = oracle.pack_codes(q, bits, group)
+    return W, x, q, s, z, codes
+
+
+@pytest.mark.parametrize("bits,group", [(4, 128), (3, 64), (4, 64), (3, 128)])
+def test_dequantize_is_scale_times_code_plus_offset(bits, group):
+    m, n = 2 * group, 33
+    _, _, q, s, z, codes = _setup(m, n, bits, group, seed=5)
+    What = oracle.dequantize(codes, s, z, m, n, bits, group)
+    ref = (np.repeat(s.astype(np.float64), group, axis=0) * q.astype(np.float64)
+           + np.repeat(z.astype(np.float64), group, axis=0))
+    assert np.array_equal(What, ref)
+
+
+@pytest.mark.parametrize("bits,group", [(4, 128), (3, 64)])
+def test_threshold_at_or_below_zero_equals_dense_matrix_product(bits, group):
+    m, n = 2 * group, 200
+    _, x, q, s, z, codes = _setup(m, n, bits, group, seed=9)
+    x[[3, 50]] = np.float16(0.0)
+    x[7] = np.float16(-0.0)
+    What = (np.repeat(s.astype(np.float64), group, axis=0) * q
+            + np.repeat(z.astype(np.float64), group, axis=0))
+    ref = What @ x.astype(np.float64)                       # library matmul on the m x n matrix
+    for t in (0.0, -1.0):
+        idx, cnt = oracle.sparsify(x, t)
+        assert cnt == (n - 3 if t == 0.0 else n)            # +-0 is not above 0
+        y, b = oracle.sparse_gemv(codes, s, z, m, n, x, idx, bits, group)
+        assert np.allclose(y, ref, rtol=0, atol=1e-12 * np.abs(What).sum(axis=1).max() * 10)
+    yd, bd = oracle.dense_gemv(codes, s, z, m, n, x, bits, group)
+    assert np.allclose(yd, ref, rtol=0, atol=1e-11)
+    assert np.allclose(bd, np.abs(What) @ np.abs(x.astype(np.float64)), rtol=1e-13)
+
+
+def test_tiny_matrix_brute_force_in_exact_rationals():
+    bits, group, m, n = 4, 4, 8, 5
+    g = np.random.Generator(np.random.PCG64(42))
+    W = (g.integers(-40, 40, size=(m, n)) / 16.0).astype(np.float16)
+    x = (g.integers(-6, 7, size=n) / 4.0).astype(np.float16)
+    t = 0.5
+    q, s, z = oracle.quantize(W, bits, group)
+    codes = oracle.pack_codes(q, bits, group)
+    idx, cnt = oracle.sparsify(x, t)
+    y, bound = oracle.sparse_gemv(codes, s, z, m, n, x, idx, bits, group)
+    active = [k for k in range(n) if abs(Fraction(float(x[k]))) > Fraction(t)]
+    assert idx.tolist() == active and cnt == len(active)
+    for j in range(m):
+        r = j // group
+        acc = sum((Fraction(float(s[r, k])) * int(q[j, k]) + Fraction(float(z[r, k]))) * Fraction(float(x[k]))
+                  for k in active)
+        bnd = sum(abs(Fraction(float(s[r, k])) * int(q[j, k]) + Fraction(float(z[r, k]))) * abs(Fraction(float(x[k])))
+                  for k in active)
+        assert abs(Fraction(y[j]) - acc) <= Fraction(1, 10**12) * (bnd + 1)
+        assert abs(Fraction(bound[j]) - bnd) <= Fraction(1, 10**12) * (bnd + 1)
+
+
+def test_one_hot_probe_returns_the_column():
+    bits, group, m, n = 4, 128, 256, 130
+    _, _, q, s, z, codes = _setup(m, n, bits, group, seed=21)
+    for k in (0, 1, 64, 129):
+        x = np.zeros(n, np.float16)
+        x[k] = np.float16(-1.5)
+        idx, cnt = oracle.sparsify(x, 0.25)
+        assert idx.tolist() == [k]
+        y, b = oracle.sparse_gemv(codes, s, z, m, n, x, idx, bits, group)
+        col = (np.repeat(s[:, k].astype(np.float64), group) * q[:, k] + np.repeat(z[:, k].astype(np.float64), group))
+        assert np.array_equal(y, -1.5 * col)
+        assert np.array_equal(b, 1.5 * np.abs(col))
+
+
+def test_lossless_family_gemv_equals_integer_arithmetic():
+    m, n = 256, 300
+    W = inputs.lossless_weights(m, n)
+    x = inputs.small_rational_activations(n, seed=4)
+    codes, s, z = oracle.pack(W, 4, 128)
+    t = 0.75                                               # drops the +-0.5 entries
+    idx, cnt = oracle.sparsify(x, t)
+    keep = np.abs(x.astype(np.float64)) > t
+    assert np.array_equal(idx, np.nonzero(keep)[0])
+    j = np.arange(m)[:, None]
+    k = np.arange(n)[None, :]
+    num = ((5 * j + 3 * k) % 16).astype(np.int64)          # 16 * W, integers
+    x2 = np.rint(x.astype(np.float64) * 2).astype(np.int64)  # 2 * x, integers
+    ref = (num[:, keep] @ x2[keep]) / 32.0                 # exact
+    y, _ = oracle.sparse_gemv(codes, s, z, m, n, x, idx, 4, 128)
+    assert np.array_equal(y, ref)
+
+
+def test_order_invariance_superposition_and_row_subset():
+    bits, group, m, n = 4, 128, 256, 257
+    _, x, q, s, z, codes = _setup(m, n, bits, group, seed=33)
+    idx, cnt = oracle.sparsify(x, 0.6)
+    y, b = oracle.sparse_gemv(codes, s, z, m, n, x, idx, bits, group)
+    perm = np.random.Generator(np.random.PCG64(1)).permutation(cnt)
+    yp, bp = oracle.sparse_gemv(codes, s, z, m, n, x, idx[perm], bits, group)
+    assert np.allclose(yp, y, rtol=0, atol=1e-13 * b.max())
+    half = cnt // 2
+    y1, _ = oracle.sparse_gemv(codes, s, z, m, n, x, idx[:half], bits, group)
+    y2, _ = oracle.sparse_gemv(codes, s, z, m, n, x, idx[half:], bits, group)
+    assert np.allclose(y1 + y2, y, rtol=0, atol=1e-13 * b.max())
+    rows = np.array([0, 5, 127, 128, 255], np.int32)
+    yr, br = oracle.sparse_gemv(codes, s, z, m, n, x, idx, bits, group, rows=rows)
+    assert np.array_equal(yr, y[rows]) and np.array_equal(br, b[rows])
+    yd, _ = oracle.dense_gemv(codes, s, z, m, n, x, bits, group)
+    ydr, _ = oracle.dense_gemv(codes, s, z, m, n, x, bits, group, rows=rows)
+    assert np.array_equal(ydr, yd[rows])
+
+
+# ------------------------------------------------------------------ index collection
+
+@pytest.mark.parametrize("n", [1, 31, 32, 33, 1000, 4096])
+def test_index_list_matches_a_brute_force_scan(n):
+    x = inputs.activations(n, seed=n, dist="laplace")
+    if n > 40:
+        x[5] = np.float16(np.nan)
+        x[6] = np.float16(np.inf)
+        x[7] = np.float16(-np.inf)
+    for t in (-1.0, 0.0, 0.3, float(np.abs(x.astype(np.float32))[0]), 2.0, float("inf")):
+        idx, cnt = oracle.sparsify(x, t)
+        ref = [k for k in range(n) if abs(float(x[k])) > t]          # NaN compares false
+        assert idx.tolist() == ref and cnt == len(ref)
+        with np.errstate(invalid="ignore"):
+            dropped = np.count_nonzero(np.abs(x.astype(np.float64)) <= t) + np.count_nonzero(np.isnan(x))
+        assert cnt == n - dropped
+    assert oracle.sparsify(x, float("inf"))[1] == 0
+    assert oracle.sparsify(x, -1.0)[1] == n - int(np.isnan(x).sum())
+
+
+def test_tie_at_the_threshold_is_dropped():
+    x = np.array([0.5, -0.5, 0.5004883, 0.25, -0.75], dtype=np.float16)
+    idx, cnt = oracle.sparsify(x, 0.5)
+    assert idx.tolist() == [2, 4]
+
+
+def test_partition_is_even_and_matches_the_papers_example():
+    assert oracle.partition(9, 3).tolist() == [0, 3, 6, 9]       # 9 active entries, 3 workers
+    for count, S in [(0, 4), (1, 4), (10, 4), (2048, 9), (7168, 37)]:
+        b = oracle.partition(count, S)
+        sizes = np.diff(b)
+        assert b[0] == 0 and b[-1] == count and sizes.min() >= 0
+        assert sizes.max() - sizes.min() <= 1
+
+
+# ------------------------------------------------------------------ input generator closed forms
+
+def test_laplace_and_gaussian_thresholds_match_closed_forms():
+    xl = inputs.activations(200_000, seed=0, dist="laplace")
+    xg = inputs.activations(200_000, seed=1, dist="gauss")
+    # |Laplace(0,1)| ~ Exp(1): quantile -ln(1-p); |N(0,1)|: Phi^-1((1+p)/2)
+    for p, ql, qg in [(0.25, 0.2877, 0.3186), (0.40, 0.5108, 0.5244), (0.50, math.log(2), 0.6745), (0.90, 2.3026, 1.6449)]:
+        assert abs(inputs.threshold_for_sparsity(xl, p) - ql) < 0.02
+        assert abs(inputs.threshold_for_sparsity(xg, p) - qg) < 0.02
+    x = inputs.activations(4096, seed=0)
+    t = inputs.threshold_for_sparsity(x, 0.5)
+    idx, cnt = oracle.sparsify(x, t)
+    assert cnt <= 2048 and cnt >= 2048 - 8                 # ties at t only ever drop more
+    assert abs(inputs.realised_sparsity(x, t) - (1 - cnt / 4096)) < 1e-12
+    assert inputs.threshold_for_sparsity(x, 0.0) == -1.0
+
+
+def test_outlier_recipe():
+    x0 = inputs.activations(8192, seed=2)
+    x1 = inputs.activations(8192, seed=2, outlier_frac=0.01, outlier_scale=20.0)
+    changed = np.nonzero(x0 != x1)[0]
+    assert 70 <= changed.size <= 82
+    assert np.allclose(x1[changed].astype(np.float32), 20 * x0[changed].astype(np.float32), rtol=2e-3)
