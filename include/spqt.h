@@ -1,0 +1,159 @@
+/*
+ * spqt.h -- C ABI of the SpQt hot path for NVIDIA B200 (sm_100a).
+ *
+ * SpQt ("Enabling Dynamic Sparsity in Quantized LLM Inference") runs every
+ * decode-time linear layer y = W x as: (1) collect the indices of the hidden
+ * state entries whose magnitude exceeds a calibrated threshold, (2) multiply
+ * only the matching columns of the group-quantized W, which is stored in the
+ * "zigzag" layout so that a skipped column is a run of whole quantization
+ * blocks.  This library is that path and nothing else.
+ *
+ * Conventions
+ *   W is m x n: m output features (rows), n input features (columns), y = W x
+ *   (paper Sec. 4.2.1).  G = group size, b = bits per code, R = m / G
+ *   block-rows, B = G*b/8 bytes of codes per block.
+ *   Every pointer is a DEVICE pointer unless its name ends in _host.
+ *   `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *   stream).  All calls are asynchronous on that stream and never synchronise
+ *   the device, except the *_host entry point, which says so.
+ *   The caller owns every buffer; the library allocates nothing, frees nothing
+ *   and keeps no pointer after a call returns.
+ *
+ * Data layout (paper Sec. 4.1.2: column-aligned grouping, row-major block storage)
+ *   A block (r,k) is the G codes of rows r*G .. r*G+G-1 of column k.
+ *   codes : R*n blocks of B bytes; block (r,k) starts at byte (r*n + k)*B.
+ *           4-bit block: byte i (i < G/2) = code[i] | code[i + G/2] << 4.
+ *           3-bit block: G/4 bytes of a 2-bit plane, byte j = sum_{u<4}
+ *           (code[j + u*G/4] & 3) << 2u, then G/8 bytes of a 1-bit plane,
+ *           byte j = sum_{u<8} (code[j + u*G/8] >> 2) << u.
+ *   scales, zeros : fp16 arrays of R*n entries, entry (r,k) at index r*n + k.
+ *           A weight is What[r*G+i][k] = scales[r,k] * code_i + zeros[r,k]
+ *           ("zero" is the additive offset of the block, its minimum).
+ *
+ * Errors
+ *   Every entry point returns a spqt_status.  Arguments that can be checked on
+ *   the host are checked before anything is launched; a failed check launches
+ *   nothing.  The contents of idx/count are trusted (indices in [0,n), no
+ *   duplicates, count <= n).
+ */
+#ifndef SPQT_H
+#define SPQT_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SPQT_OK = 0,
+    SPQT_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, ldw < n                 */
+    SPQT_ERR_UNSUPPORTED = 2, /* bits not in {3,4}, group not in {64,128}, m % group != 0 */
+    SPQT_ERR_ALIGNMENT = 3,   /* a pointer is not aligned as documented                   */
+    SPQT_ERR_WORKSPACE = 4,   /* workspace smaller than spqt_packed_sizes reports         */
+    SPQT_ERR_CUDA = 5         /* the CUDA runtime reported an error (launch, copy, query) */
+} spqt_status;
+
+/* Human-readable name of a status code; never NULL. */
+const char* spqt_status_string(int status);
+
+/* Library version, major*1000 + minor. */
+int spqt_version(void);
+
+/*
+ * Sizes in bytes of the buffers a problem needs.  Any out-pointer may be NULL.
+ * Needs no GPU.  gemv_workspace_bytes covers both GEMV entry points.
+ */
+spqt_status spqt_packed_sizes(int m, int n, int bits, int group,
+                              size_t* codes_bytes, size_t* scales_bytes, size_t* zeros_bytes,
+                              size_t* gemv_workspace_bytes);
+
+/*
+ * Offline conversion: quantize W group by group and write it in zigzag order
+ * (paper Sec. 3.2 "first quantized into the zigzag weight layout", Sec. 4.1.2).
+ * Per block: zero = min of the G weights; scale = fp16((max - zero) / (2^b - 1)),
+ * the subtraction and division each one IEEE fp32 operation; code_i =
+ * clamp(rint((w_i - zero) / scale), 0, 2^b - 1) with ties to even, all zero when
+ * scale == 0.  Results are bit-reproducible.
+ *   W      : fp16, row-major [m][ldw], ldw >= n, 2-byte aligned.
+ *   codes  : R*n*B bytes, 16-byte aligned.   scales, zeros : R*n fp16, 16-byte aligned.
+ */
+spqt_status spqt_pack(const void* W, int m, int n, int ldw, int bits, int group,
+                      void* codes, void* scales, void* zeros, void* stream);
+
+/*
+ * Inverse of the layout step of spqt_pack (a checking aid): natural-order codes,
+ * one byte each, q_u8[j*n + k] = code of row j, column k.
+ */
+spqt_status spqt_unpack(const void* codes, int m, int n, int bits, int group,
+                        void* q_u8, void* stream);
+
+/*
+ * Sparse index collection (paper Sec. 4.2.3, "Sparse index collecting kernel"):
+ * idx[0:*count] = every k with |x_k| > t, in ascending order; *count = how many.
+ * The comparison is strict and exact (fp16 widened); NaN entries are never
+ * active.  idx must hold n entries.  x: fp16[n], 2-byte aligned.  idx, count:
+ * int32, 4-byte aligned.  n == 0 is allowed and writes *count = 0.
+ */
+spqt_status spqt_sparsify(const void* x, int n, float t,
+                          int32_t* idx, int32_t* count, void* stream);
+
+/*
+ * Load-balanced sparse GEMV over the zigzag layout (paper Sec. 4.2.2 and 4.2.3):
+ *   y[j] = sum_{i < *count} What[j][idx[i]] * x[idx[i]],  j in [0,m), y fp16.
+ * For every block-row the index list -- not the matrix columns -- is split
+ * evenly over the workers of that block-row; partial sums are accumulated in
+ * fp32 and combined in a fixed order, so a call is bit-reproducible.  idx may be
+ * in any order.  *count == 0 gives y = 0.
+ *   codes/scales/zeros : as written by spqt_pack, 16-byte aligned.
+ *   x : fp16[n].  idx : int32[>= *count].  count : int32 on the device.
+ *   y : fp16[m], 2-byte aligned.
+ *   workspace : gemv_workspace_bytes of device memory, 16-byte aligned, zeroed
+ *       ONCE by the caller before its first use; every call leaves it ready for
+ *       the next.  Two calls that may overlap on the GPU need two workspaces.
+ * Supported: bits 4 with group 64 or 128; bits 3 with group 64 or 128.
+ */
+spqt_status spqt_sparse_gemv(const void* codes, const void* scales, const void* zeros,
+                             int m, int n, int bits, int group,
+                             const void* x, const int32_t* idx, const int32_t* count,
+                             void* y, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The same kernel over all n columns with no index list: the dense GEMV on the
+ * zigzag layout (paper Sec. 4.2.2), the sparsity-free comparison.
+ */
+spqt_status spqt_dense_gemv(const void* codes, const void* scales, const void* zeros,
+                            int m, int n, int bits, int group, const void* x,
+                            void* y, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * One decode-time linear layer from HOST activations (paper Sec. 3.2: hidden
+ * state -> index collection with the layer's threshold -> sparse GEMV):
+ * copies x_host (fp16[n]) to x_dev, runs spqt_sparsify and spqt_sparse_gemv,
+ * copies y (fp16[m]) to y_host and waits for the stream.  x_host / y_host
+ * should be pinned for the copies to be asynchronous; x_dev (fp16[n]), idx_dev
+ * (int32[n]), count_dev (int32[1]) and y_dev (fp16[m]) are caller-provided
+ * device staging buffers.  This is the only entry point that synchronises.
+ */
+spqt_status spqt_sparse_linear_host(const void* codes, const void* scales, const void* zeros,
+                                    int m, int n, int bits, int group,
+                                    const void* x_host, float t, void* y_host,
+                                    void* x_dev, int32_t* idx_dev, int32_t* count_dev, void* y_dev,
+                                    void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Tuning aid: override the number of workers (column splits) per block-row and
+ * the resident-CTA target used to size the grid; 0 restores the built-in rule.
+ * Not needed for correctness.  Process-wide, not thread-safe.
+ */
+spqt_status spqt_set_tuning(int splits_per_block_row, int ctas_per_sm);
+
+/* Number of kernels the library has launched in this process (a counter for
+ * benchmarks; not synchronised with the device). */
+unsigned long long spqt_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPQT_H */

@@ -1,0 +1,223 @@
+"""Thin Python binding of the C ABI in ``include/spqt.h``.
+
+Argument marshalling only: every function takes torch CUDA tensors (device
+memory and streams are PyTorch's job), checks dtypes, passes raw pointers to the
+entry point of the same name and raises :class:`SpqtError` on a non-zero status.
+No arithmetic of the method happens in Python and there is no CPU fallback: if
+``libspqt.so`` has not been built, the first call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libspqt.so")
+
+EXPORTS = (
+    "spqt_status_string", "spqt_version", "spqt_packed_sizes", "spqt_pack", "spqt_unpack",
+    "spqt_sparsify", "spqt_sparse_gemv", "spqt_dense_gemv", "spqt_sparse_linear_host",
+    "spqt_set_tuning", "spqt_launch_count",
+)
+
+_lib = None
+
+
+class SpqtError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = int(status)
+        super().__init__("%s failed: %s (%d)" % (where, status_string(status), status))
+
+
+def lib() -> ctypes.CDLL:
+    """Load the shared library (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                "libspqt.so is missing: build it with `python -m paper_2511_04477_b200.build` "
+                "(there is no CPU fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+        L.spqt_status_string.restype = ctypes.c_char_p
+        L.spqt_status_string.argtypes = [i32]
+        L.spqt_version.restype = i32
+        L.spqt_packed_sizes.argtypes = [i32, i32, i32, i32] + [ctypes.POINTER(sz)] * 4
+        L.spqt_pack.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp]
+        L.spqt_unpack.argtypes = [vp, i32, i32, i32, i32, vp, vp]
+        L.spqt_sparsify.argtypes = [vp, i32, ctypes.c_float, vp, vp, vp]
+        L.spqt_sparse_gemv.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
+        L.spqt_dense_gemv.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, sz, vp]
+        L.spqt_sparse_linear_host.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, vp,
+                                              vp, vp, vp, vp, vp, sz, vp]
+        L.spqt_set_tuning.argtypes = [i32, i32]
+        L.spqt_launch_count.restype = ctypes.c_ulonglong
+        for name in ("spqt_packed_sizes", "spqt_pack", "spqt_unpack", "spqt_sparsify",
+                     "spqt_sparse_gemv", "spqt_dense_gemv", "spqt_sparse_linear_host", "spqt_set_tuning"):
+            getattr(L, name).restype = i32
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().spqt_status_string(int(status)).decode()
+
+
+def _ok(status: int, where: str) -> None:
+    if status != 0:
+        raise SpqtError(status, where)
+
+
+def _stream(stream) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(s.cuda_stream)
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> int:
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError("%s must be a CUDA tensor" % name)
+    if t.dtype != dtype:
+        raise TypeError("%s must be %s, got %s" % (name, dtype, t.dtype))
+    if not t.is_contiguous():
+        raise ValueError("%s must be contiguous" % name)
+    return t.data_ptr()
+
+
+@dataclass
+class PackedSizes:
+    codes_bytes: int
+    scales_bytes: int
+    zeros_bytes: int
+    gemv_workspace_bytes: int
+
+
+def spqt_packed_sizes(m: int, n: int, bits: int = 4, group: int = 128) -> PackedSizes:
+    out = [ctypes.c_size_t(0) for _ in range(4)]
+    _ok(lib().spqt_packed_sizes(m, n, bits, group, *[ctypes.byref(o) for o in out]), "spqt_packed_sizes")
+    return PackedSizes(*[int(o.value) for o in out])
+
+
+@dataclass
+class Packed:
+    """Device buffers written by :func:`spqt_pack` (zigzag layout)."""
+    codes: torch.Tensor    # uint8[R*n*B]
+    scales: torch.Tensor   # float16[R*n]
+    zeros: torch.Tensor    # float16[R*n]
+    m: int
+    n: int
+    bits: int
+    group: int
+
+    @property
+    def nbytes(self) -> int:
+        return self.codes.numel() + 2 * self.scales.numel() + 2 * self.zeros.numel()
+
+
+def new_workspace(m: int, n: int, bits: int = 4, group: int = 128, device=None) -> torch.Tensor:
+    """Zeroed GEMV workspace (zeroed once; every call leaves it ready for the next)."""
+    sz = spqt_packed_sizes(m, n, bits, group).gemv_workspace_bytes
+    return torch.zeros(sz, dtype=torch.uint8, device=device or "cuda")
+
+
+def spqt_pack(W: torch.Tensor, bits: int = 4, group: int = 128, stream=None) -> Packed:
+    if W.dim() != 2 or W.stride(1) != 1:
+        raise ValueError("W must be 2-D with unit column stride")
+    if not W.is_cuda or W.dtype != torch.float16:
+        raise TypeError("W must be a CUDA float16 tensor")
+    m, n = W.shape
+    sz = spqt_packed_sizes(m, n, bits, group)
+    codes = torch.empty(sz.codes_bytes, dtype=torch.uint8, device=W.device)
+    scales = torch.empty(sz.scales_bytes // 2, dtype=torch.float16, device=W.device)
+    zeros = torch.empty(sz.zeros_bytes // 2, dtype=torch.float16, device=W.device)
+    _ok(lib().spqt_pack(W.data_ptr(), m, n, W.stride(0), bits, group, codes.data_ptr(),
+                        scales.data_ptr(), zeros.data_ptr(), _stream(stream)), "spqt_pack")
+    return Packed(codes, scales, zeros, m, n, bits, group)
+
+
+def spqt_unpack(p: Packed, stream=None) -> torch.Tensor:
+    q = torch.empty((p.m, p.n), dtype=torch.uint8, device=p.codes.device)
+    _ok(lib().spqt_unpack(_dev(p.codes, torch.uint8, "codes"), p.m, p.n, p.bits, p.group,
+                          q.data_ptr(), _stream(stream)), "spqt_unpack")
+    return q
+
+
+def spqt_sparsify(x: torch.Tensor, t: float, idx: torch.Tensor = None, count: torch.Tensor = None,
+                  stream=None):
+    """-> (idx int32[n] of which the first count[0] entries are valid, count int32[1]), both on the device."""
+    n = x.numel()
+    if idx is None:
+        idx = torch.empty(max(n, 1), dtype=torch.int32, device=x.device)
+    if count is None:
+        count = torch.empty(1, dtype=torch.int32, device=x.device)
+    if idx.numel() < n:
+        raise ValueError("idx must hold n entries")
+    _ok(lib().spqt_sparsify(_dev(x, torch.float16, "x"), n, float(t), _dev(idx, torch.int32, "idx"),
+                            _dev(count, torch.int32, "count"), _stream(stream)), "spqt_sparsify")
+    return idx, count
+
+
+def spqt_sparse_gemv(p: Packed, x: torch.Tensor, idx: torch.Tensor, count: torch.Tensor,
+                     workspace: torch.Tensor, y: torch.Tensor = None, stream=None) -> torch.Tensor:
+    if y is None:
+        y = torch.empty(p.m, dtype=torch.float16, device=x.device)
+    if x.numel() != p.n or y.numel() != p.m:
+        raise ValueError("x must have n entries and y m entries")
+    _ok(lib().spqt_sparse_gemv(
+        _dev(p.codes, torch.uint8, "codes"), _dev(p.scales, torch.float16, "scales"),
+        _dev(p.zeros, torch.float16, "zeros"), p.m, p.n, p.bits, p.group,
+        _dev(x, torch.float16, "x"), _dev(idx, torch.int32, "idx"), _dev(count, torch.int32, "count"),
+        _dev(y, torch.float16, "y"), _dev(workspace, torch.uint8, "workspace"), workspace.numel(),
+        _stream(stream)), "spqt_sparse_gemv")
+    return y
+
+
+def spqt_dense_gemv(p: Packed, x: torch.Tensor, workspace: torch.Tensor, y: torch.Tensor = None,
+                    stream=None) -> torch.Tensor:
+    if y is None:
+        y = torch.empty(p.m, dtype=torch.float16, device=x.device)
+    if x.numel() != p.n or y.numel() != p.m:
+        raise ValueError("x must have n entries and y m entries")
+    _ok(lib().spqt_dense_gemv(
+        _dev(p.codes, torch.uint8, "codes"), _dev(p.scales, torch.float16, "scales"),
+        _dev(p.zeros, torch.float16, "zeros"), p.m, p.n, p.bits, p.group,
+        _dev(x, torch.float16, "x"), _dev(y, torch.float16, "y"),
+        _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)), "spqt_dense_gemv")
+    return y
+
+
+class HostLinear:
+    """Staging buffers for :func:`spqt_sparse_linear_host`: pinned host x / y and
+    device x, idx, count, y for one packed matrix."""
+
+    def __init__(self, p: Packed, workspace: torch.Tensor = None):
+        dev = p.codes.device
+        self.p = p
+        self.x_host = torch.empty(p.n, dtype=torch.float16).pin_memory()
+        self.y_host = torch.empty(p.m, dtype=torch.float16).pin_memory()
+        self.x_dev = torch.empty(p.n, dtype=torch.float16, device=dev)
+        self.idx = torch.empty(p.n, dtype=torch.int32, device=dev)
+        self.count = torch.zeros(1, dtype=torch.int32, device=dev)
+        self.y_dev = torch.empty(p.m, dtype=torch.float16, device=dev)
+        self.workspace = workspace if workspace is not None else new_workspace(p.m, p.n, p.bits, p.group, dev)
+
+
+def spqt_sparse_linear_host(h: HostLinear, t: float, stream=None) -> torch.Tensor:
+    """x in ``h.x_host`` -> y in ``h.y_host`` (copies, index collection, sparse GEMV, sync)."""
+    p = h.p
+    _ok(lib().spqt_sparse_linear_host(
+        p.codes.data_ptr(), p.scales.data_ptr(), p.zeros.data_ptr(), p.m, p.n, p.bits, p.group,
+        h.x_host.data_ptr(), float(t), h.y_host.data_ptr(), h.x_dev.data_ptr(), h.idx.data_ptr(),
+        h.count.data_ptr(), h.y_dev.data_ptr(), h.workspace.data_ptr(), h.workspace.numel(),
+        _stream(stream)), "spqt_sparse_linear_host")
+    return h.y_host
+
+
+def spqt_set_tuning(splits_per_block_row: int = 0, ctas_per_sm: int = 0) -> None:
+    _ok(lib().spqt_set_tuning(int(splits_per_block_row), int(ctas_per_sm)), "spqt_set_tuning")
+
+
+def spqt_launch_count() -> int:
+    return int(lib().spqt_launch_count())

@@ -1,0 +1,63 @@
+// Shared host-side helpers of the SpQt CUDA library (argument checks, geometry,
+// device properties).  No kernel code lives here.
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/spqt.h"
+
+namespace spqt {
+
+struct Format {
+    int m, n, bits, group;
+    int R;          // block-rows
+    int B;          // bytes of codes per block
+    size_t blocks;  // R * n
+};
+
+// Validates the format and fills the derived sizes.
+inline spqt_status make_format(int m, int n, int bits, int group, Format* f)
+{
+    if (m <= 0 || n <= 0) return SPQT_ERR_INVALID_ARG;
+    if (bits != 3 && bits != 4) return SPQT_ERR_UNSUPPORTED;
+    if (group != 64 && group != 128) return SPQT_ERR_UNSUPPORTED;
+    if (m % group != 0) return SPQT_ERR_UNSUPPORTED;
+    f->m = m; f->n = n; f->bits = bits; f->group = group;
+    f->R = m / group;
+    f->B = group * bits / 8;
+    f->blocks = (size_t)f->R * (size_t)n;
+    return SPQT_OK;
+}
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// Upper bound on the number of workers per block-row that any tuning may pick;
+// the workspace is sized for it (independent of the device, so sizes can be
+// computed without a GPU).
+constexpr int kMaxCtaSlots = 148 * 8;
+constexpr int kMaxSplits = 128;
+
+inline int max_splits(int R)
+{
+    int s = (kMaxCtaSlots + R - 1) / R;
+    if (s < 1) s = 1;
+    if (s > kMaxSplits) s = kMaxSplits;
+    return s;
+}
+
+// Workspace layout: [R] int32 arrival counters (kept zero between calls),
+// padded to 256 B, then fp32 partials [R][S][G] and [R][S] offset-term partials.
+inline size_t counters_bytes(int R) { return (((size_t)R * 4 + 255) / 256) * 256; }
+
+inline size_t workspace_bytes(const Format& f)
+{
+    size_t S = (size_t)max_splits(f.R);
+    return counters_bytes(f.R) + S * (size_t)f.R * (size_t)(f.group + 4) * sizeof(float);
+}
+
+int sm_count();               // SMs of the current device (cached per device); <= 0 on error
+void count_launch(int k = 1); // bump the process-wide launch counter
+
+}  // namespace spqt

@@ -1,0 +1,177 @@
+// Offline conversion: group-wise min/max quantization of fp16 weights and the
+// zigzag block layout (groups run down G rows of one column; blocks stored
+// row-major over (block-row, column)), plus the inverse of the layout step.
+#include "spqt_common.cuh"
+
+namespace spqt {
+
+constexpr int kPackCols = 32;     // columns of one block-row handled by a CTA
+constexpr int kPackThreads = 256; // 8 warps, 4 columns each
+
+// One CTA stages a G x 32 tile of W in shared memory with row-contiguous
+// (coalesced) reads, then each warp quantizes four columns.  Lane l of a warp
+// owns rows l, l+32, ... of the column.
+template <int G, int BITS>
+__global__ void __launch_bounds__(kPackThreads)
+pack_kernel(const __half* __restrict__ W, int n, int ldw,
+            uint8_t* __restrict__ codes, __half* __restrict__ scales, __half* __restrict__ zeros)
+{
+    constexpr int B = G * BITS / 8;
+    constexpr int QMAX = (1 << BITS) - 1;
+    constexpr int PER_LANE = G / 32;
+    __shared__ __half tile[G][kPackCols + 2];
+    __shared__ uint8_t q_sm[kPackThreads / 32][G];
+
+    const int r = blockIdx.y;
+    const int k0 = blockIdx.x * kPackCols;
+    const int tid = threadIdx.x;
+
+    for (int e = tid; e < G * kPackCols; e += kPackThreads) {
+        int i = e / kPackCols, c = e % kPackCols;
+        int k = k0 + c;
+        tile[i][c] = (k < n) ? W[(size_t)(r * G + i) * ldw + k] : __float2half(0.0f);
+    }
+    __syncthreads();
+
+    const int warp = tid / 32, lane = tid % 32;
+    for (int cc = 0; cc < kPackCols / (kPackThreads / 32); ++cc) {
+        const int c = warp * (kPackCols / (kPackThreads / 32)) + cc;
+        const int k = k0 + c;
+        if (k >= n) break;  // uniform across the warp
+        float w[PER_LANE];
+        float lo = INFINITY, hi = -INFINITY;
+#pragma unroll
+        for (int u = 0; u < PER_LANE; ++u) {
+            w[u] = __half2float(tile[lane + 32 * u][c]);
+            lo = fminf(lo, w[u]);
+            hi = fmaxf(hi, w[u]);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+            hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+        }
+        // scale = fp16((max - min) / qmax): one IEEE subtract, one IEEE divide, RN-even
+        const float s32 = __fdiv_rn(__fsub_rn(hi, lo), (float)QMAX);
+        const __half sh = __float2half_rn(s32);
+        const float sf = __half2float(sh);
+#pragma unroll
+        for (int u = 0; u < PER_LANE; ++u) {
+            int code = 0;
+            if (sf != 0.0f) {
+                float t = rintf(__fdiv_rn(__fsub_rn(w[u], lo), sf));  // ties to even
+                t = fminf(fmaxf(t, 0.0f), (float)QMAX);
+                code = (int)t;
+            }
+            q_sm[warp][lane + 32 * u] = (uint8_t)code;
+        }
+        __syncwarp();
+        const size_t blk = (size_t)r * n + k;
+        uint8_t* out = codes + blk * B;
+        for (int b = lane; b < B; b += 32) {
+            unsigned v = 0;
+            if (BITS == 4) {
+                v = q_sm[warp][b] | (q_sm[warp][b + G / 2] << 4);
+            } else {
+                if (b < G / 4) {
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) v |= (q_sm[warp][b + u * (G / 4)] & 3u) << (2 * u);
+                } else {
+                    const int j = b - G / 4;
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) v |= ((q_sm[warp][j + u * (G / 8)] >> 2) & 1u) << u;
+                }
+            }
+            out[b] = (uint8_t)v;
+        }
+        if (lane == 0) {
+            scales[blk] = sh;
+            zeros[blk] = __float2half_rn(lo);  // exact: lo is an fp16 value
+        }
+        __syncwarp();
+    }
+}
+
+// One thread per weight: read its code out of the zigzag buffer.
+template <int G, int BITS>
+__global__ void unpack_kernel(const uint8_t* __restrict__ codes, int m, int n, uint8_t* __restrict__ q)
+{
+    constexpr int B = G * BITS / 8;
+    const size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= (size_t)m * n) return;
+    const int j = (int)(e / n), k = (int)(e % n);
+    const int r = j / G, i = j % G;
+    const uint8_t* blk = codes + ((size_t)r * n + k) * B;
+    int code;
+    if (BITS == 4) {
+        code = (i < G / 2) ? (blk[i] & 15) : (blk[i - G / 2] >> 4);
+    } else {
+        const int low2 = (blk[i % (G / 4)] >> (2 * (i / (G / 4)))) & 3;
+        const int top1 = (blk[G / 4 + i % (G / 8)] >> (i / (G / 8))) & 1;
+        code = low2 | (top1 << 2);
+    }
+    q[e] = (uint8_t)code;
+}
+
+template <int G, int BITS>
+static spqt_status launch_pack(const Format& f, const void* W, int ldw, void* codes, void* scales,
+                               void* zeros, cudaStream_t s)
+{
+    dim3 grid((f.n + kPackCols - 1) / kPackCols, f.R);
+    pack_kernel<G, BITS><<<grid, kPackThreads, 0, s>>>(
+        static_cast<const __half*>(W), f.n, ldw, static_cast<uint8_t*>(codes),
+        static_cast<__half*>(scales), static_cast<__half*>(zeros));
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? SPQT_OK : SPQT_ERR_CUDA;
+}
+
+template <int G, int BITS>
+static spqt_status launch_unpack(const Format& f, const void* codes, void* q, cudaStream_t s)
+{
+    const size_t total = (size_t)f.m * f.n;
+    const unsigned blocks = (unsigned)((total + 255) / 256);
+    unpack_kernel<G, BITS><<<blocks, 256, 0, s>>>(static_cast<const uint8_t*>(codes), f.m, f.n,
+                                                  static_cast<uint8_t*>(q));
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? SPQT_OK : SPQT_ERR_CUDA;
+}
+
+}  // namespace spqt
+
+extern "C" {
+
+spqt_status spqt_pack(const void* W, int m, int n, int ldw, int bits, int group,
+                      void* codes, void* scales, void* zeros, void* stream)
+{
+    using namespace spqt;
+    if (!W || !codes || !scales || !zeros) return SPQT_ERR_INVALID_ARG;
+    Format f;
+    spqt_status st = make_format(m, n, bits, group, &f);
+    if (st != SPQT_OK) return st;
+    if (ldw < n) return SPQT_ERR_INVALID_ARG;
+    if (f.R > 65535) return SPQT_ERR_UNSUPPORTED;
+    if (!aligned(W, 2) || !aligned(codes, 16) || !aligned(scales, 16) || !aligned(zeros, 16))
+        return SPQT_ERR_ALIGNMENT;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (bits == 4 && group == 128) return launch_pack<128, 4>(f, W, ldw, codes, scales, zeros, s);
+    if (bits == 4 && group == 64) return launch_pack<64, 4>(f, W, ldw, codes, scales, zeros, s);
+    if (bits == 3 && group == 128) return launch_pack<128, 3>(f, W, ldw, codes, scales, zeros, s);
+    return launch_pack<64, 3>(f, W, ldw, codes, scales, zeros, s);
+}
+
+spqt_status spqt_unpack(const void* codes, int m, int n, int bits, int group, void* q_u8, void* stream)
+{
+    using namespace spqt;
+    if (!codes || !q_u8) return SPQT_ERR_INVALID_ARG;
+    Format f;
+    spqt_status st = make_format(m, n, bits, group, &f);
+    if (st != SPQT_OK) return st;
+    if (((size_t)m * n + 255) / 256 > 0x7fffffffu) return SPQT_ERR_UNSUPPORTED;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (bits == 4 && group == 128) return launch_unpack<128, 4>(f, codes, q_u8, s);
+    if (bits == 4 && group == 64) return launch_unpack<64, 4>(f, codes, q_u8, s);
+    if (bits == 3 && group == 128) return launch_unpack<128, 3>(f, codes, q_u8, s);
+    return launch_unpack<64, 3>(f, codes, q_u8, s);
+}
+
+}  // extern "C"

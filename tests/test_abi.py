@@ -1,0 +1,87 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports every
+symbol the header declares, sizes are right, and bad arguments are refused before
+anything is launched."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from conftest import ROOT
+from paper_2511_04477_b200 import binding, build
+
+
+@pytest.fixture(scope="module")
+def L():
+    build.build()
+    return binding.lib()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "spqt.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(spqt_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(L):
+    names = declared_functions()
+    assert "spqt_pack" in names and "spqt_sparsify" in names and "spqt_sparse_gemv" in names
+    for name in names:
+        assert hasattr(L, name), name
+    assert set(names) == set(binding.EXPORTS)
+
+
+def test_status_strings(L):
+    assert binding.status_string(0) == "SPQT_OK"
+    assert binding.status_string(2) == "SPQT_ERR_UNSUPPORTED"
+    assert binding.status_string(99) == "SPQT_ERR_UNKNOWN"
+    assert L.spqt_version() >= 1000
+
+
+@pytest.mark.parametrize("m,n,bits,group,B", [(4096, 4096, 4, 128, 64), (14336, 4096, 4, 64, 32),
+                                              (8192, 28672, 3, 128, 48), (128, 1, 3, 64, 24)])
+def test_packed_sizes(L, m, n, bits, group, B):
+    s = binding.spqt_packed_sizes(m, n, bits, group)
+    R = m // group
+    assert s.codes_bytes == R * n * B
+    assert s.scales_bytes == R * n * 2 and s.zeros_bytes == R * n * 2
+    assert s.gemv_workspace_bytes >= R * 4 + 4 * (m + R)      # counters + one worker's partials
+    assert s.gemv_workspace_bytes < 64 << 20
+
+
+def test_unsupported_formats_are_refused(L):
+    for args in [(4096, 4096, 5, 128), (4096, 4096, 4, 32), (4000, 4096, 4, 128), (4096, 4096, 2, 64)]:
+        with pytest.raises(binding.SpqtError) as e:
+            binding.spqt_packed_sizes(*args)
+        assert e.value.status == 2
+    with pytest.raises(binding.SpqtError) as e:
+        binding.spqt_packed_sizes(0, 4096, 4, 128)
+    assert e.value.status == 1
+
+
+def test_bad_arguments_launch_nothing(L):
+    before = binding.spqt_launch_count()
+    buf = ctypes.create_string_buffer(4096)
+    base = ctypes.addressof(buf)
+    a16 = (base + 15) // 16 * 16            # 16-byte aligned fake "device" address; never dereferenced
+    ws = binding.spqt_packed_sizes(128, 8, 4, 128).gemv_workspace_bytes
+    # null pointers
+    assert L.spqt_pack(None, 128, 8, 8, 4, 128, a16, a16, a16, None) == 1
+    assert L.spqt_sparsify(None, 8, 0.5, a16, a16, None) == 1
+    assert L.spqt_sparse_gemv(a16, a16, a16, 128, 8, 4, 128, a16, None, a16, a16, a16, ws, None) == 1
+    assert L.spqt_dense_gemv(a16, a16, None, 128, 8, 4, 128, a16, a16, a16, ws, None) == 1
+    # ldw < n, negative n
+    assert L.spqt_pack(a16, 128, 8, 4, 4, 128, a16, a16, a16, None) == 1
+    assert L.spqt_sparsify(a16, -1, 0.5, a16, a16, None) == 1
+    # unsupported format
+    assert L.spqt_pack(a16, 100, 8, 8, 4, 128, a16, a16, a16, None) == 2
+    assert L.spqt_sparse_gemv(a16, a16, a16, 128, 8, 8, 128, a16, a16, a16, a16, a16, ws, None) == 2
+    # misaligned
+    assert L.spqt_pack(a16, 128, 8, 8, 4, 128, a16 + 4, a16, a16, None) == 3
+    assert L.spqt_sparse_gemv(a16 + 8, a16, a16, 128, 8, 4, 128, a16, a16, a16, a16, a16, ws, None) == 3
+    assert L.spqt_sparsify(a16 + 1, 8, 0.5, a16, a16, None) == 3
+    # workspace too small
+    assert L.spqt_sparse_gemv(a16, a16, a16, 128, 8, 4, 128, a16, a16, a16, a16, a16, ws - 1, None) == 4
+    assert L.spqt_dense_gemv(a16, a16, a16, 128, 8, 4, 128, a16, a16, a16, 16, None) == 4
+    assert L.spqt_set_tuning(-1, 0) == 1
+    assert binding.spqt_launch_count() == before

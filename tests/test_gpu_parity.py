@@ -1,0 +1,294 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle.
+
+Bit-exact for packed bytes, indices and counts; y within
+2e-3 * sum_k |What_jk||x_k| per row (exact where the arithmetic is exact)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2511_04477_b200 import binding, inputs
+from gpu_util import TOL, check_y, dev, pack_on_gpu, packed_to_host, run_sparse
+
+pytestmark = pytest.mark.gpu
+
+FORMATS = [(4, 128), (4, 64), (3, 128), (3, 64)]
+GEMV_FORMATS = [(4, 128), (4, 64)]
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _need_gpu():
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    binding.lib()
+
+
+# ------------------------------------------------------------------ a1: quantize + zigzag pack
+
+@pytest.mark.parametrize("bits,group", FORMATS)
+@pytest.mark.parametrize("m_blocks,n", [(1, 1), (2, 37), (3, 300), (8, 1030)])
+def test_pack_is_byte_identical_to_the_oracle(bits, group, m_blocks, n):
+    m = m_blocks * group
+    W = inputs.weights(m, n, seed=bits * 100 + group + n)
+    if n > 30:
+        W[:group, 5] = np.float16(0.0123)          # constant group -> scale 0
+        W[:, 7] = (W[:, 7].astype(np.float32) * 2.0**-12).astype(np.float16)   # fp16-subnormal scale
+        W[3, 9] = np.float16(60000.0)              # huge range
+    codes, s, z = oracle.pack(W, bits, group)
+    p = pack_on_gpu(W, bits, group)
+    gc, gs, gz = packed_to_host(p)
+    assert np.array_equal(gs.view(np.uint16), s.view(np.uint16))
+    assert np.array_equal(gz.view(np.uint16), z.view(np.uint16))
+    assert np.array_equal(gc, codes)
+    q = binding.spqt_unpack(p)
+    torch.cuda.synchronize()
+    assert np.array_equal(q.cpu().numpy(), oracle.unpack_codes(codes, m, n, bits, group))
+
+
+def test_pack_honours_the_leading_dimension():
+    m, n, ldw = 256, 100, 164
+    big = inputs.weights(m, ldw, seed=77)
+    Wd = dev(big)[:, :n]
+    p = binding.spqt_pack(Wd, 4, 128)
+    codes, s, z = oracle.pack(np.ascontiguousarray(big[:, :n]), 4, 128)
+    gc, gs, gz = packed_to_host(p)
+    assert np.array_equal(gc, codes) and np.array_equal(gs, s) and np.array_equal(gz, z)
+
+
+def test_group_sizes_outside_64_and_128_are_refused(hand_example):
+    # the library supports G in {64,128} only; the hand example (G=4) pins the oracle
+    with pytest.raises(binding.SpqtError):
+        binding.spqt_pack(dev(hand_example["W"]), 4, 4)
+
+
+# ------------------------------------------------------------------ a2: index collection
+
+@pytest.mark.parametrize("n", [1, 2, 31, 32, 33, 1023, 1024, 1025, 4096, 8192, 14336, 28672, 40000])
+def test_index_list_is_bit_exact(n):
+    x = inputs.activations(n, seed=1000 + n, dist="laplace" if n % 2 == 0 else "gauss")
+    if n > 100:
+        x[17] = np.float16(np.nan)
+        x[18] = np.float16(np.inf)
+        x[19] = np.float16(-np.inf)
+        x[20] = np.float16(-0.0)
+    ts = [-1.0, 0.0, inputs.threshold_for_sparsity(x, 0.25), inputs.threshold_for_sparsity(x, 0.5),
+          inputs.threshold_for_sparsity(x, 0.9), 1e9, float("inf")]
+    xd = dev(x)
+    for t in ts:
+        idx = torch.full((n,), -7, dtype=torch.int32, device="cuda")
+        cnt = torch.full((1,), -7, dtype=torch.int32, device="cuda")
+        binding.spqt_sparsify(xd, t, idx, cnt)
+        torch.cuda.synchronize()
+        ref_idx, ref_cnt = oracle.sparsify(x, t)
+        assert int(cnt.item()) == ref_cnt
+        assert np.array_equal(idx.cpu().numpy()[:ref_cnt], ref_idx)
+        assert np.all(idx.cpu().numpy()[ref_cnt:] == -7)       # nothing written past count
+
+
+def test_empty_input_gives_count_zero():
+    x = torch.empty(0, dtype=torch.float16, device="cuda")
+    idx = torch.empty(1, dtype=torch.int32, device="cuda")
+    cnt = torch.full((1,), 5, dtype=torch.int32, device="cuda")
+    binding.spqt_sparsify(x, 0.5, idx, cnt)
+    torch.cuda.synchronize()
+    assert int(cnt.item()) == 0
+
+
+# ------------------------------------------------------------------ a3-a5: sparse GEMV
+
+@pytest.mark.parametrize("bits,group", GEMV_FORMATS)
+@pytest.mark.parametrize("m_blocks,n,dist", [(2, 300, "laplace"), (8, 4096, "laplace"), (3, 1111, "gauss")])
+def test_sparse_gemv_matches_oracle_across_sparsities(bits, group, m_blocks, n, dist):
+    m = m_blocks * group
+    W = inputs.weights(m, n, seed=m + n + bits)
+    x = inputs.activations(n, seed=5 + n, dist=dist)
+    p = pack_on_gpu(W, bits, group)
+    codes, s, z = packed_to_host(p)
+    ws = binding.new_workspace(m, n, bits, group)
+    for sp in (0.0, 0.25, 0.5, 0.9, 0.999):
+        t = inputs.threshold_for_sparsity(x, sp)
+        y, idx, cnt = run_sparse(p, x, t, ws)
+        ref_idx, ref_cnt = oracle.sparsify(x, t)
+        assert cnt == ref_cnt and np.array_equal(idx, ref_idx)
+        y_ref, bound = oracle.sparse_gemv(codes, s, z, m, n, x, ref_idx, bits, group)
+        check_y(y, y_ref, bound, "sparsity %.3f" % sp)
+    assert not ws[: 4 * (m // group)].any()                    # arrival counters back to zero
+
+
+@pytest.mark.parametrize("bits,group", GEMV_FORMATS)
+def test_degenerate_counts(bits, group):
+    m, n = 2 * group, 500
+    W = inputs.weights(m, n, seed=3)
+    x = inputs.activations(n, seed=4)
+    p = pack_on_gpu(W, bits, group)
+    codes, s, z = packed_to_host(p)
+    ws = binding.new_workspace(m, n, bits, group)
+    # nothing active -> exactly zero
+    y, idx, cnt = run_sparse(p, x, float("inf"), ws)
+    assert cnt == 0 and not y.any()
+    # exactly one active entry (the largest magnitude)
+    a = np.abs(x.astype(np.float32))
+    t = float(np.sort(a)[-2])
+    y, idx, cnt = run_sparse(p, x, t, ws)
+    assert cnt == 1 and idx[0] == int(a.argmax())
+    y_ref, bound = oracle.sparse_gemv(codes, s, z, m, n, x, idx, bits, group)
+    check_y(y, y_ref, bound, "one active column")
+
+
+@pytest.mark.parametrize("bits,group", GEMV_FORMATS)
+def test_one_hot_probes_return_the_dequantized_column(bits, group):
+    """x = c e_k: y = c * What[:,k]; one product per row, so the result is the fp16
+    rounding of the exact value (catches any layout / row-permutation slip)."""
+    m, n = 3 * group, 140
+    W = inputs.weights(m, n, seed=8)
+    p = pack_on_gpu(W, bits, group)
+    codes, s, z = packed_to_host(p)
+    ws = binding.new_workspace(m, n, bits, group)
+    for k in (0, 1, 7, 8, 31, 32, 33, 139):
+        x = np.zeros(n, np.float16)
+        x[k] = np.float16(-1.5)
+        y, idx, cnt = run_sparse(p, x, 0.5, ws)
+        assert cnt == 1 and idx[0] == k
+        y_ref, bound = oracle.sparse_gemv(codes, s, z, m, n, x, idx, bits, group)
+        check_y(y, y_ref, bound, "one-hot k=%d" % k)
+        # stronger: a single product per row, so y is within half an fp16 ulp (plus fp32 dust)
+        assert np.all(np.abs(y.astype(np.float64) - y_ref) <= (2.0**-11 + 2.0**-20) * np.abs(y_ref) + 2.0**-25)
+
+
+@pytest.mark.parametrize("group", [64, 128])
+def test_lossless_family_is_bit_exact(group):
+    m, n = 4 * group, 700
+    W = inputs.lossless_weights(m, n)
+    x = inputs.small_rational_activations(n, seed=12)
+    p = pack_on_gpu(W, 4, group)
+    codes, s, z = packed_to_host(p)
+    ws = binding.new_workspace(m, n, 4, group)
+    for t in (0.25, 0.75, 1.5):
+        y, idx, cnt = run_sparse(p, x, t, ws)
+        y_ref, _ = oracle.sparse_gemv(codes, s, z, m, n, x, idx, 4, group)
+        assert np.array_equal(y.astype(np.float64), y_ref.astype(np.float16).astype(np.float64))
+        y2, _, _ = run_sparse(p, x, t, ws, shuffle_seed=3)       # any index order
+        assert np.array_equal(y2, y)
+
+
+def test_index_order_does_not_matter_beyond_rounding_and_calls_are_reproducible():
+    m, n, bits, group = 1024, 4096, 4, 128
+    W = inputs.weights(m, n, seed=1)
+    x = inputs.activations(n, seed=2)
+    p = pack_on_gpu(W, bits, group)
+    codes, s, z = packed_to_host(p)
+    ws = binding.new_workspace(m, n, bits, group)
+    t = inputs.threshold_for_sparsity(x, 0.5)
+    y1, idx, cnt = run_sparse(p, x, t, ws)
+    y2, _, _ = run_sparse(p, x, t, ws)
+    assert np.array_equal(y1.view(np.uint16), y2.view(np.uint16))  # fixed combination order
+    y3, idx3, _ = run_sparse(p, x, t, ws, shuffle_seed=9)
+    assert sorted(idx3.tolist()) == idx.tolist()
+    y_ref, bound = oracle.sparse_gemv(codes, s, z, m, n, x, idx, bits, group)
+    check_y(y3, y_ref, bound, "shuffled idx")
+
+
+@pytest.mark.parametrize("splits", [1, 2, 3, 7, 16, 33])
+def test_any_number_of_workers_per_block_row(splits):
+    m, n, bits, group = 512, 1500, 4, 128
+    W = inputs.weights(m, n, seed=31)
+    x = inputs.activations(n, seed=32)
+    p = pack_on_gpu(W, bits, group)
+    codes, s, z = packed_to_host(p)
+    ws = binding.new_workspace(m, n, bits, group)
+    t = inputs.threshold_for_sparsity(x, 0.4)
+    try:
+        binding.spqt_set_tuning(splits, 0)
+        y, idx, cnt = run_sparse(p, x, t, ws)
+    finally:
+        binding.spqt_set_tuning(0, 0)
+    y_ref, bound = oracle.sparse_gemv(codes, s, z, m, n, x, idx, bits, group)
+    check_y(y, y_ref, bound, "S=%d" % splits)
+
+
+def test_heavy_tailed_outliers():
+    m, n, bits, group = 1024, 8192, 4, 128
+    W = inputs.weights(m, n, seed=51)
+    x = inputs.activations(n, seed=52, outlier_frac=0.01, outlier_scale=20.0)
+    p = pack_on_gpu(W, bits, group)
+    codes, s, z = packed_to_host(p)
+    ws = binding.new_workspace(m, n, bits, group)
+    t = inputs.threshold_for_sparsity(x, 0.5)
+    y, idx, cnt = run_sparse(p, x, t, ws)
+    y_ref, bound = oracle.sparse_gemv(codes, s, z, m, n, x, idx, bits, group)
+    check_y(y, y_ref, bound, "outliers")
+
+
+# ------------------------------------------------------------------ a6: dense GEMV
+
+@pytest.mark.parametrize("bits,group", GEMV_FORMATS)
+@pytest.mark.parametrize("m_blocks,n", [(2, 300), (8, 4096), (1, 1)])
+def test_dense_gemv_matches_oracle_and_the_sparse_path_at_threshold_below_zero(bits, group, m_blocks, n):
+    m = m_blocks * group
+    W = inputs.weights(m, n, seed=61 + n)
+    x = inputs.activations(n, seed=62 + n)
+    p = pack_on_gpu(W, bits, group)
+    codes, s, z = packed_to_host(p)
+    ws = binding.new_workspace(m, n, bits, group)
+    yd = binding.spqt_dense_gemv(p, dev(x), ws)
+    torch.cuda.synchronize()
+    y_ref, bound = oracle.dense_gemv(codes, s, z, m, n, x, bits, group)
+    check_y(yd.cpu().numpy(), y_ref, bound, "dense")
+    ys, idx, cnt = run_sparse(p, x, -1.0, ws)
+    assert cnt == n
+    check_y(ys, y_ref, bound, "sparse at t<0")
+
+
+# ------------------------------------------------------------------ full-size shapes, sampled rows
+
+@pytest.mark.parametrize("name,m,n,dist", [l for l in inputs.LLAMA3_8B_LINEARS if l[0] in ("q", "k", "gate", "down")])
+def test_llama3_8b_shapes_on_sampled_rows(name, m, n, dist):
+    bits, group = 4, 128
+    W = inputs.weights(m, n, seed=hash(name) % 1000)
+    x = inputs.activations(n, seed=7, dist=dist)
+    p = pack_on_gpu(W, bits, group)
+    codes, s, z = packed_to_host(p)
+    ws = binding.new_workspace(m, n, bits, group)
+    rows = np.unique(np.concatenate([
+        np.random.Generator(np.random.PCG64(5)).integers(0, m, size=192),
+        [0, 63, 64, 127, 128, m - 129, m - 128, m - 1]])).astype(np.int32)
+    for sp in (0.25, 0.4, 0.5):
+        t = inputs.threshold_for_sparsity(x, sp)
+        y, idx, cnt = run_sparse(p, x, t, ws)
+        ref_idx, ref_cnt = oracle.sparsify(x, t)
+        assert cnt == ref_cnt and np.array_equal(idx, ref_idx)
+        y_ref, bound = oracle.sparse_gemv(codes, s, z, m, n, x, ref_idx, bits, group, rows=rows)
+        check_y(y[rows], y_ref, bound, "%s at %.2f" % (name, sp))
+    yd = binding.spqt_dense_gemv(p, dev(x), ws)
+    torch.cuda.synchronize()
+    y_ref, bound = oracle.dense_gemv(codes, s, z, m, n, x, bits, group, rows=rows)
+    check_y(yd.cpu().numpy()[rows], y_ref, bound, "%s dense" % name)
+    # spot-check the packed bytes of a few blocks against the oracle's pack of those rows
+    r = (m // group) - 1
+    sub = np.ascontiguousarray(W[r * group:(r + 1) * group])
+    c_ref, s_ref, z_ref = oracle.pack(sub, bits, group)
+    B = oracle.block_bytes(bits, group)
+    assert np.array_equal(codes[r * n * B:(r + 1) * n * B], c_ref)
+    assert np.array_equal(s[r], s_ref[0]) and np.array_equal(z[r], z_ref[0])
+
+
+# ------------------------------------------------------------------ host-buffer entry point
+
+def test_host_entry_point_matches_the_device_path():
+    m, n, bits, group = 1024, 4096, 4, 128
+    W = inputs.weights(m, n, seed=71)
+    x = inputs.activations(n, seed=72)
+    p = pack_on_gpu(W, bits, group)
+    h = binding.HostLinear(p)
+    t = inputs.threshold_for_sparsity(x, 0.5)
+    h.x_host.copy_(torch.from_numpy(x))
+    y_host = binding.spqt_sparse_linear_host(h, t).numpy().copy()
+    y_dev, idx, cnt = run_sparse(p, x, t, binding.new_workspace(m, n, bits, group))
+    assert np.array_equal(y_host.view(np.uint16), y_dev.view(np.uint16))
+    assert int(h.count.item()) == cnt
+
+
+def test_kernels_are_counted():
+    before = binding.spqt_launch_count()
+    x = dev(inputs.activations(256, seed=1))
+    binding.spqt_sparsify(x, 0.5)
+    assert binding.spqt_launch_count() == before + 1
