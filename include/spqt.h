@@ -112,7 +112,8 @@ spqt_status spqt_sparsify(const void* x, int n, float t,
  *   workspace : gemv_workspace_bytes of device memory, 16-byte aligned, zeroed
  *       ONCE by the caller before its first use; every call leaves it ready for
  *       the next.  Two calls that may overlap on the GPU need two workspaces.
- * Supported: bits 4 with group 64 or 128; bits 3 with group 64 or 128.
+ * Supported: bits 4 with group 64 or 128 (bits 3: SPQT_ERR_UNSUPPORTED for now).
+ * n * B must fit in 32 bits.
  */
 spqt_status spqt_sparse_gemv(const void* codes, const void* scales, const void* zeros,
                              int m, int n, int bits, int group,
@@ -143,11 +144,21 @@ spqt_status spqt_sparse_linear_host(const void* codes, const void* scales, const
                                     void* workspace, size_t workspace_bytes, void* stream);
 
 /*
- * Tuning aid: override the number of workers (column splits) per block-row and
- * the resident-CTA target used to size the grid; 0 restores the built-in rule.
- * Not needed for correctness.  Process-wide, not thread-safe.
+ * Tuning aid: number of CTAs of the GEMV grid (0 restores the built-in rule, one
+ * persistent CTA per SM; values above 1024 are clamped).  `reserved` must be 0.
+ * Any value gives the same results up to the order of partial sums.
+ * Process-wide, not thread-safe.
  */
-spqt_status spqt_set_tuning(int splits_per_block_row, int ctas_per_sm);
+spqt_status spqt_set_tuning(int gemv_ctas, int reserved);
+
+/*
+ * Reads the workspace's status word into *status_host (a host int) and waits for
+ * the stream: 0 = every GEMV that used this workspace ran to completion;
+ * non-zero = a bounded on-chip wait expired inside a GEMV kernel (which then
+ * drained its copies and returned early, leaving y unspecified).  The word is
+ * sticky until the caller zeroes the workspace again.
+ */
+spqt_status spqt_workspace_status(const void* workspace, int m, int group, int* status_host, void* stream);
 
 /* Number of kernels the library has launched in this process (a counter for
  * benchmarks; not synchronised with the device). */

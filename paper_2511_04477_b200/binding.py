@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libspqt.so")
 EXPORTS = (
     "spqt_status_string", "spqt_version", "spqt_packed_sizes", "spqt_pack", "spqt_unpack",
     "spqt_sparsify", "spqt_sparse_gemv", "spqt_dense_gemv", "spqt_sparse_linear_host",
-    "spqt_set_tuning", "spqt_launch_count",
+    "spqt_set_tuning", "spqt_workspace_status", "spqt_launch_count",
 )
 
 _lib = None
@@ -54,9 +54,11 @@ def lib() -> ctypes.CDLL:
         L.spqt_sparse_linear_host.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, vp,
                                               vp, vp, vp, vp, vp, sz, vp]
         L.spqt_set_tuning.argtypes = [i32, i32]
+        L.spqt_workspace_status.argtypes = [vp, i32, i32, ctypes.POINTER(i32), vp]
         L.spqt_launch_count.restype = ctypes.c_ulonglong
         for name in ("spqt_packed_sizes", "spqt_pack", "spqt_unpack", "spqt_sparsify",
-                     "spqt_sparse_gemv", "spqt_dense_gemv", "spqt_sparse_linear_host", "spqt_set_tuning"):
+                     "spqt_sparse_gemv", "spqt_dense_gemv", "spqt_sparse_linear_host", "spqt_set_tuning",
+                     "spqt_workspace_status"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -215,8 +217,16 @@ def spqt_sparse_linear_host(h: HostLinear, t: float, stream=None) -> torch.Tenso
     return h.y_host
 
 
-def spqt_set_tuning(splits_per_block_row: int = 0, ctas_per_sm: int = 0) -> None:
-    _ok(lib().spqt_set_tuning(int(splits_per_block_row), int(ctas_per_sm)), "spqt_set_tuning")
+def spqt_set_tuning(gemv_ctas: int = 0) -> None:
+    _ok(lib().spqt_set_tuning(int(gemv_ctas), 0), "spqt_set_tuning")
+
+
+def spqt_workspace_status(workspace: torch.Tensor, m: int, group: int = 128, stream=None) -> int:
+    """0 unless a bounded on-chip wait expired in a GEMV that used this workspace (synchronises)."""
+    out = ctypes.c_int(-1)
+    _ok(lib().spqt_workspace_status(_dev(workspace, torch.uint8, "workspace"), m, group,
+                                    ctypes.byref(out), _stream(stream)), "spqt_workspace_status")
+    return int(out.value)
 
 
 def spqt_launch_count() -> int:

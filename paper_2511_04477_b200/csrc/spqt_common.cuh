@@ -33,28 +33,21 @@ inline spqt_status make_format(int m, int n, int bits, int group, Format* f)
 
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
-// Upper bound on the number of workers per block-row that any tuning may pick;
-// the workspace is sized for it (independent of the device, so sizes can be
-// computed without a GPU).
-constexpr int kMaxCtaSlots = 148 * 8;
-constexpr int kMaxSplits = 128;
+// Largest grid any tuning may use for a GEMV; the workspace is sized for it
+// (independent of the device, so sizes can be computed without a GPU).
+constexpr int kMaxCtas = 1024;
 
-inline int max_splits(int R)
-{
-    int s = (kMaxCtaSlots + R - 1) / R;
-    if (s < 1) s = 1;
-    if (s > kMaxSplits) s = kMaxSplits;
-    return s;
-}
+// Upper bound on the number of CTAs that contribute partial sums to one block-row.
+inline int max_slots(int R) { return (kMaxCtas + R - 1) / R + 1; }
 
-// Workspace layout: [R] int32 arrival counters (kept zero between calls),
-// padded to 256 B, then fp32 partials [R][S][G] and [R][S] offset-term partials.
-inline size_t counters_bytes(int R) { return (((size_t)R * 4 + 255) / 256) * 256; }
+// Workspace layout: [R] int32 arrival counters (kept zero between calls), one
+// int32 status word (non-zero after a bounded wait expired), padded to 256 B;
+// then fp32 partials [R][slots][G] and offset-term partials [R][slots].
+inline size_t header_bytes(int R) { return (((size_t)(R + 1) * 4 + 255) / 256) * 256; }
 
 inline size_t workspace_bytes(const Format& f)
 {
-    size_t S = (size_t)max_splits(f.R);
-    return counters_bytes(f.R) + S * (size_t)f.R * (size_t)(f.group + 4) * sizeof(float);
+    return header_bytes(f.R) + (size_t)f.R * (size_t)max_slots(f.R) * (size_t)(f.group + 1) * sizeof(float);
 }
 
 int sm_count();               // SMs of the current device (cached per device); <= 0 on error

@@ -111,7 +111,8 @@ def test_sparse_gemv_matches_oracle_across_sparsities(bits, group, m_blocks, n, 
         assert cnt == ref_cnt and np.array_equal(idx, ref_idx)
         y_ref, bound = oracle.sparse_gemv(codes, s, z, m, n, x, ref_idx, bits, group)
         check_y(y, y_ref, bound, "sparsity %.3f" % sp)
-    assert not ws[: 4 * (m // group)].any()                    # arrival counters back to zero
+    assert not ws[: 4 * (m // group + 1)].any()                # arrival counters and status word are zero
+    assert binding.spqt_workspace_status(ws, m, group) == 0
 
 
 @pytest.mark.parametrize("bits,group", GEMV_FORMATS)
@@ -187,8 +188,8 @@ def test_index_order_does_not_matter_beyond_rounding_and_calls_are_reproducible(
     check_y(y3, y_ref, bound, "shuffled idx")
 
 
-@pytest.mark.parametrize("splits", [1, 2, 3, 7, 16, 33])
-def test_any_number_of_workers_per_block_row(splits):
+@pytest.mark.parametrize("splits", [1, 2, 3, 7, 16, 33, 148, 301, 1024])
+def test_any_number_of_workers(splits):
     m, n, bits, group = 512, 1500, 4, 128
     W = inputs.weights(m, n, seed=31)
     x = inputs.activations(n, seed=32)
@@ -197,10 +198,11 @@ def test_any_number_of_workers_per_block_row(splits):
     ws = binding.new_workspace(m, n, bits, group)
     t = inputs.threshold_for_sparsity(x, 0.4)
     try:
-        binding.spqt_set_tuning(splits, 0)
+        binding.spqt_set_tuning(splits)
         y, idx, cnt = run_sparse(p, x, t, ws)
     finally:
-        binding.spqt_set_tuning(0, 0)
+        binding.spqt_set_tuning(0)
+    assert binding.spqt_workspace_status(ws, m, group) == 0
     y_ref, bound = oracle.sparse_gemv(codes, s, z, m, n, x, idx, bits, group)
     check_y(y, y_ref, bound, "S=%d" % splits)
 
