@@ -1,0 +1,417 @@
+#!/usr/bin/env python
+"""Benchmark of the SpQt hot path on B200: one line of JSON on stdout.
+
+Workload (the configuration the metric is quoted on): the seven linear layers of
+one Llama-3-8B-shaped decoder layer at batch 1 -- q, k, v, o (4096->4096,
+4096->1024 x2, 4096->4096), gate/up (4096->14336), down (14336->4096) -- INT4
+codes, group 128, fp16 scale and zero, zigzag layout, 50 % activation sparsity.
+A *step* is one pass over those seven matrices: four index collections
+(attention input shared by q,k,v; attention output for o; MLP input shared by
+gate,up; MLP hidden for down) and seven sparse GEMVs.  Eight distinct layer
+copies (about 0.93 GB of packed weights, far larger than the 126 MB L2) are
+visited round-robin so that weights really come from HBM.
+
+value  = effective GB/s over the bytes the method needs
+         (sum over GEMVs of count*R*(B+4) + 2n + 4count + 4 + 2m, plus 2n + 4count + 4
+         per index collection), whole job, inputs resident in HBM.
+e2e    = the same metric through spqt_sparse_linear_host: x from pinned host memory,
+         y back to pinned host memory, copies and the final wait inside the timed region.
+roofline.achieved = algorithmic bytes per sparse-GEMV launch / its mean duration
+         (device events over a region that launches only the GEMVs of the same steps).
+
+`--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+BITS, GROUP = 4, 128
+SPARSITY = 0.5
+LAYER_COPIES = 8
+X_POOL = 4            # distinct hidden states per site, rotated
+FALLBACK_HBM_GBS = 6650.0
+METRIC = "sparse int4 GEMV effective HBM GB/s at 50% sparsity (Llama-3-8B-shaped decode-layer linears, batch 1)"
+
+# ncu dram__bytes_read.sum + dram__bytes_write.sum per sparse-GEMV launch, by shape, from the
+# capture summarised in profiles/ (see profiles/README.md); None until measured.
+NCU_TRAFFIC_BYTES = {}
+
+
+def needed_bytes_gemv(m, n, count, bits=BITS, group=GROUP):
+    R, B = m // group, group * bits // 8
+    return count * R * (B + 4) + 2 * n + 4 * count + 4 + 2 * m
+
+
+def needed_bytes_sparsify(n, count):
+    return 2 * n + 4 * count + 4
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc is not None:
+            time.sleep(0.15)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+                for nm, v in zip(names, r[2:6]):
+                    if v.lower().startswith("active"):
+                        reasons.add(nm)
+            except Exception:
+                pass
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------- reference arm (CPU oracle)
+
+def oracle_sample(steps, warmup, threads=None):
+    """Time the oracle (index collection + fp64 sparse GEMV) on a bounded sample of the
+    workload: ONE layer copy (all seven linears), a few steps."""
+    import oracle
+    from paper_2511_04477_b200 import inputs
+    if threads:
+        oracle.set_threads(threads)
+    sample = inputs.LLAMA3_8B_LINEARS
+    packed = []
+    for i, (name, m, n, dist) in enumerate(sample):
+        W = inputs.weights(m, n, seed=i)
+        x = inputs.activations(n, seed=100 + i, dist=dist)
+        t = inputs.threshold_for_sparsity(x, SPARSITY)
+        packed.append((m, n, x, t) + oracle.pack(W, BITS, GROUP))
+
+    def one_step():
+        nbytes = 0
+        for (m, n, x, t, codes, s, z) in packed:
+            idx, cnt = oracle.sparsify(x, t)
+            oracle.sparse_gemv(codes, s, z, m, n, x, idx, BITS, GROUP)
+            nbytes += needed_bytes_gemv(m, n, cnt) + needed_bytes_sparsify(n, cnt)
+        return nbytes
+
+    for _ in range(warmup):
+        one_step()
+    t0 = time.perf_counter()
+    total = 0
+    for _ in range(steps):
+        total += one_step()
+    dt = time.perf_counter() - t0
+    return {"value": total / dt / 1e9, "ms_per_step": dt / steps * 1e3, "cores": oracle.threads(),
+            "sample": "one layer copy (q,k,v,o,gate,up,down), int4 g128, 50%% sparsity, index collection + fp64 "
+                      "sparse GEMV per linear, %d timed steps after %d warm-up" % (steps, warmup)}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    steps = max(1, min(args.steps, 10))
+    r = oracle_sample(steps, min(args.warmup, 1))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": r["value"], "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": steps, "warmup": min(args.warmup, 1), "ms_per_step": r["ms_per_step"], "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "llama3-8b decode-layer linears, int4 g128, 50% sparsity (one layer copy, bounded number of steps; see cpu_baseline.sample)"},
+        "cpu_baseline": {"value": r["value"], "unit": "GB/s", "cores": r["cores"], "kind": "oracle", "sample": r["sample"]},
+        "e2e": {"value": r["value"], "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------- our arm
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2511_04477_b200 import binding, inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    binding.lib()
+
+    linears = inputs.LLAMA3_8B_LINEARS
+    sites = {"attn_in": ("laplace", 4096, ["q", "k", "v"]), "attn_out": ("laplace", 4096, ["o"]),
+             "mlp_in": ("laplace", 4096, ["gate", "up"]), "mlp_mid": ("gauss", 14336, ["down"])}
+    shape = {name: (m, n) for name, m, n, _ in linears}
+    order = ["q", "k", "v", "o", "gate", "up", "down"]
+    site_of = {nm: s for s, (_, _, names) in sites.items() for nm in names}
+
+    # ---- weights: LAYER_COPIES x 7 matrices, random-init on the device, packed by spqt_pack
+    layers = []
+    g = torch.Generator(device=dev)
+    for L in range(LAYER_COPIES):
+        packs = {}
+        for i, name in enumerate(order):
+            m, n = shape[name]
+            g.manual_seed(1000 * rank + L * 7 + i)
+            W = torch.empty((m, n), dtype=torch.float32, device=dev).normal_(0.0, 0.02, generator=g).half()
+            packs[name] = binding.spqt_pack(W, BITS, GROUP)
+            del W
+        layers.append(packs)
+    torch.cuda.synchronize()
+    weight_bytes = sum(p.nbytes for L in layers for p in L.values())
+
+    # ---- activations: X_POOL hidden states per site (host, seeded), thresholds by nearest rank
+    xs, ts = {}, {}
+    for si, (s, (dname, n, _)) in enumerate(sites.items()):
+        xs[s] = [inputs.activations(n, seed=10_000 + 97 * si + j, dist=dname) for j in range(X_POOL)]
+        ts[s] = [inputs.threshold_for_sparsity(x, SPARSITY) for x in xs[s]]
+    xd = {s: [torch.from_numpy(x).to(dev) for x in xs[s]] for s in sites}
+    idx = {s: torch.empty(sites[s][1], dtype=torch.int32, device=dev) for s in sites}
+    cnt = {s: torch.zeros(1, dtype=torch.int32, device=dev) for s in sites}
+    ys = {nm: torch.empty(shape[nm][0], dtype=torch.float16, device=dev) for nm in order}
+    ws = {nm: binding.new_workspace(shape[nm][0], shape[nm][1], BITS, GROUP, dev) for nm in order}
+
+    stream = torch.cuda.Stream(device=dev)
+
+    def step(i, with_sparsify=True, gemv=True, dense=False):
+        L = layers[i % LAYER_COPIES]
+        j = i % X_POOL if with_sparsify else 0   # kernel-only regions keep the index lists of pool entry 0
+        for s in sites:
+            if with_sparsify:
+                binding.spqt_sparsify(xd[s][j], ts[s][j], idx[s], cnt[s], stream=stream)
+            if gemv:
+                for nm in sites[s][2]:
+                    if dense:
+                        binding.spqt_dense_gemv(L[nm], xd[s][j], ws[nm], ys[nm], stream=stream)
+                    else:
+                        binding.spqt_sparse_gemv(L[nm], xd[s][j], idx[s], cnt[s], ws[nm], ys[nm], stream=stream)
+
+    def counts_for(j):
+        out = {}
+        for s in sites:
+            a = np.abs(xs[s][j].astype(np.float32))
+            out[s] = int(np.count_nonzero(a > np.float32(ts[s][j])))
+        return out
+
+    counts = [counts_for(j) for j in range(X_POOL)]
+
+    def step_bytes(i):
+        c = counts[i % X_POOL]
+        b = 0
+        for s in sites:
+            b += needed_bytes_sparsify(sites[s][1], c[s])
+            for nm in sites[s][2]:
+                b += needed_bytes_gemv(shape[nm][0], shape[nm][1], c[s])
+        return b
+
+    def gemv_bytes(i, dense=False):
+        c = counts[0]
+        return sum(needed_bytes_gemv(shape[nm][0], shape[nm][1], shape[nm][1] if dense else c[site_of[nm]])
+                   for nm in order)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, K, W):
+        """W warm-up steps, then K steps between two events on the launching stream; max over ranks (ms)."""
+        with torch.cuda.stream(stream):
+            for i in range(W):
+                fn(i)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            e0.record(stream)
+            for i in range(W, W + K):
+                fn(i)
+            e1.record(stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    K, W = args.steps, max(args.warmup, 3)
+
+    # ---- main timed region (whole hot path), with clocks sampled during it
+    l0 = binding.spqt_launch_count()
+    with ClockSampler(local) as clk:
+        ms = timed(lambda i: step(i), K, W)
+    launches = binding.spqt_launch_count() - l0
+    launches_timed = launches * K // (K + W)
+    total_bytes = sum(step_bytes(i) for i in range(W, W + K))
+    value = world * total_bytes / (ms * 1e-3) / 1e9
+
+    # ---- kernel-only regions for the roofline and the dense comparison (index lists of pool entry 0)
+    with torch.cuda.stream(stream):
+        for s in sites:
+            binding.spqt_sparsify(xd[s][0], ts[s][0], idx[s], cnt[s], stream=stream)
+    ms_gemv = timed(lambda i: step(i, with_sparsify=False), K, W)
+    ms_dense = timed(lambda i: step(i, with_sparsify=False, dense=True), K, W)
+    ms_sparsify = timed(lambda i: step(i, gemv=False), K, W)
+    with torch.cuda.stream(stream):
+        for s in sites:
+            binding.spqt_sparsify(xd[s][0], ts[s][0], idx[s], cnt[s], stream=stream)
+    gb = sum(gemv_bytes(i) for i in range(W, W + K))
+    gb_dense = sum(gemv_bytes(i, dense=True) for i in range(W, W + K))
+    n_gemv = 7 * K
+    achieved = gb / (ms_gemv * 1e-3) / 1e9
+    peak, peak_kind = measured_peak()
+
+    # per-shape device time, rotating the same layer copies (gemv only)
+    per_shape = {}
+    for nm in order:
+        s = site_of[nm]
+
+        reps = 4 * LAYER_COPIES
+        t_sp = timed(lambda i, nm=nm, s=s: binding.spqt_sparse_gemv(
+            layers[i % LAYER_COPIES][nm], xd[s][0], idx[s], cnt[s], ws[nm], ys[nm], stream=stream), reps, 3)
+        t_de = timed(lambda i, nm=nm, s=s: binding.spqt_dense_gemv(
+            layers[i % LAYER_COPIES][nm], xd[s][0], ws[nm], ys[nm], stream=stream), reps, 3)
+        m, n = shape[nm]
+        c0 = counts[0][s]
+        per_shape[nm] = {"m": m, "n": n, "count": c0,
+                         "sparse_us": t_sp * 1e3 / reps, "dense_us": t_de * 1e3 / reps,
+                         "sparse_gbs": needed_bytes_gemv(m, n, c0) / (t_sp * 1e-3 / reps) / 1e9,
+                         "dense_gbs": needed_bytes_gemv(m, n, n) / (t_de * 1e-3 / reps) / 1e9,
+                         "speedup_vs_dense": t_de / t_sp}
+
+    # ---- end to end from host buffers through the C ABI (copies + sync inside the timed region)
+    hosts = [{nm: binding.HostLinear(layers[L][nm], ws[nm]) for nm in order} for L in range(LAYER_COPIES)]
+    for L in range(LAYER_COPIES):
+        for nm in order:
+            hosts[L][nm].x_host.copy_(torch.from_numpy(xs[site_of[nm]][0]))
+
+    def e2e_step(i):
+        for nm in order:
+            binding.spqt_sparse_linear_host(hosts[i % LAYER_COPIES][nm], ts[site_of[nm]][0], stream=stream)
+
+    for i in range(3):
+        e2e_step(i)
+    barrier()
+    t0 = time.perf_counter()
+    e2e_K = K
+    for i in range(3, 3 + e2e_K):
+        e2e_step(i)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    if world > 1:
+        t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e_bytes = e2e_K * sum(needed_bytes_gemv(shape[nm][0], shape[nm][1], counts[0][site_of[nm]])
+                            + needed_bytes_sparsify(shape[nm][1], counts[0][site_of[nm]]) for nm in order)
+    h2d = sum(shape[nm][1] * 2 for nm in order)
+    d2h = sum(shape[nm][0] * 2 for nm in order)
+
+    status = max(binding.spqt_workspace_status(ws[nm], shape[nm][0], GROUP) for nm in order)
+
+    if rank == 0:
+        cpu = oracle_sample(3, 1) if world >= 1 else None
+        avg_launch_bytes = gb / n_gemv
+        traffic = None
+        if NCU_TRAFFIC_BYTES:
+            traffic = float(np.mean([NCU_TRAFFIC_BYTES[nm] for nm in order if nm in NCU_TRAFFIC_BYTES]))
+        line = {
+            "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int4 codes, f32 accumulate, f16 in/out", "data": "synthetic",
+            "config": {"workload": "llama3-8b decode-layer linears q,k,v,o,gate,up,down; int4 g128 zigzag; batch 1; "
+                                   "50% sparsity; 4 index collections + 7 sparse GEMVs per step",
+                       "l2_defeat": "%d distinct layer copies rotated, %.2f GB of packed weights (> 126 MB L2)" % (
+                           LAYER_COPIES, weight_bytes / 1e9),
+                       "parallelism": "replicas only" if world > 1 else "single GPU"},
+            "us_per_gemv": ms_gemv * 1e3 / n_gemv,
+            "us_per_step": {"hot_path": ms * 1e3 / K, "gemv_only": ms_gemv * 1e3 / K,
+                            "dense_gemv_only": ms_dense * 1e3 / K, "sparsify_only": ms_sparsify * 1e3 / K},
+            "speedup_vs_dense_same_layout": ms_dense / ms_gemv,
+            "dense_gbs": gb_dense / (ms_dense * 1e-3) / 1e9,
+            "pct_of_peak": {"of_measured_%.0f" % peak: 100 * achieved / peak, "of_nominal_8000": 100 * achieved / 8000},
+            "per_shape": per_shape,
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": traffic, "peak_kind": "of " + peak_kind,
+                         "kernel": "gemv_int4_kernel<128,sparse>", "algorithmic_bytes_per_launch": avg_launch_bytes,
+                         "avg_launch_us": ms_gemv * 1e3 / n_gemv},
+            "cpu_baseline": {"value": cpu["value"], "unit": "GB/s", "cores": cpu["cores"], "kind": "oracle",
+                             "sample": cpu["sample"]},
+            "e2e": {"value": world * e2e_bytes / e2e_s / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s / e2e_K * 1e3},
+            "gpu_launches": launches_timed,
+            "clocks": clk.summary(),
+            "device_status": status,
+            "paper_context": "paper reports up to 1.55x end-to-end decode speedup and up to 1.78x sparse-GEMV "
+                             "speedup at 50% sparsity on Apple GPUs (Q4_K); other hardware, context only",
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -107,7 +107,7 @@ spqt_status spqt_sparsify(const void* x, int n, float t,
  * fp32 and combined in a fixed order, so a call is bit-reproducible.  idx may be
  * in any order.  *count == 0 gives y = 0.
  *   codes/scales/zeros : as written by spqt_pack, 16-byte aligned.
- *   x : fp16[n].  idx : int32[>= *count].  count : int32 on the device.
+ *   x : fp16[n], 4-byte aligned.  idx : int32[>= *count].  count : int32 on the device.
  *   y : fp16[m], 2-byte aligned.
  *   workspace : gemv_workspace_bytes of device memory, 16-byte aligned, zeroed
  *       ONCE by the caller before its first use; every call leaves it ready for

@@ -3,29 +3,33 @@
 // Work decomposition (the paper's hybrid row/column parallelism, generalised):
 // the R block-rows are laid end to end and cut into P equal pieces, one per CTA,
 // P = one persistent CTA per SM.  A piece is a run of (fractions of) block-rows;
-// the fraction [u0,u1) of block-row r means the slice
-// [u0*count, u1*count) of the ACTIVE index list, so the load follows the active
-// entries, not the matrix columns, and every CTA streams the same number of
-// blocks whatever R is.  Each (CTA, block-row) segment yields G fp32 partial
-// sums; whichever CTA contributes last to a block-row (arrive-only counter:
-// nobody waits on another CTA) adds the partials in a fixed order, adds the
-// offset term and rounds to fp16.
+// the fraction [u0,u1) of block-row r means the slice [u0*count, u1*count) of
+// the ACTIVE index list, so the load follows the active entries, not the matrix
+// columns, and every CTA streams the same number of blocks whatever R is.  Each
+// (CTA, block-row) segment yields G fp32 partial sums; whichever CTA contributes
+// last to a block-row (arrive-only counter: nobody waits on another CTA) adds
+// the partials in a fixed order, adds the offset term and rounds to fp16.
 //
-// Inside a CTA the warps are specialised:
-//   * producer warps walk the segment in tiles of kTile list entries, gather
-//     idx, x, scale and zero for the tile and leave in shared memory the byte
-//     offset of every active block, its multiplier a = x_k*scale_rk (exact in
-//     fp32) and the tile's offset term sum x_k*zero_rk;
-//   * consumer warps stream the code blocks with 16-byte cp.async into a
-//     private ring of kStages x 512 B per warp (deep memory-level parallelism,
-//     no registers held, no barrier: a lane reads back what it copied) and do
-//     the dequantize-FMA work.
-//   * one writer warp takes the consumers' per-warp sums at the end of a
-//     segment, adds them, publishes the partial and, if its CTA is the last
-//     contributor of the block-row, produces y -- so the fence and the global
-//     round trip never stall the streaming warps.
-// Producers run a tile ahead; tiles are handed over with mbarriers whose waits
-// are bounded (on expiry an error word is set and the kernel drains and exits).
+// Inside a CTA, kWorkers warps each run their own copy pipeline over chunks of
+// 32 list entries (chunks are dealt round-robin to the warps); nothing is shared
+// between the warps until the end of a segment.  Per chunk, three stages, all
+// cp.async into the warp's private shared-memory ring, one commit group per
+// iteration:
+//   A  the chunk's 32 column numbers (one 4-byte copy per lane);
+//   B  once A has landed: the code blocks (16 bytes per lane, the lanes of a
+//      block adjacent so that every 32-byte sector crosses once, fetched with
+//      64-byte L2 granularity so that an inactive neighbour block is not dragged
+//      in) and the 4-byte words holding x_k, scale_rk and zero_rk of the lane's
+//      own entry;
+//   C  once B has landed: lane l turns its words into a = x_k*scale_rk (exact in
+//      fp32) and x_k*zero_rk, the multipliers are dealt out with shuffles, and
+//      the warp does the dequantize-FMA work.
+// A runs 2*kDepth chunks ahead of C and B kDepth chunks ahead, so kDepth chunks
+// (2 KB each) per warp are in flight.  One more warp, the writer, adds the
+// workers' sums at the end of a segment, publishes the partial and, if this CTA
+// is the last contributor of the block-row, produces y; its waits on shared-
+// memory barriers are bounded in wall time (on expiry the workspace's status
+// word is set and the kernel returns).
 //
 // Arithmetic:  y[j] = sum_k a_k * code_jk + sum_k x_k * zero_rk.  A 4-bit code
 // becomes an fp32 operand with no conversion: the nibble masked in place at bit
@@ -37,23 +41,17 @@
 
 namespace spqt {
 
-constexpr int kConsumerWarps = 13;
-constexpr int kProducerWarps = 2;
-constexpr int kWriterWarp = kConsumerWarps + kProducerWarps;  // one more warp combines and writes partial sums
-constexpr int kGemvThreads = (kConsumerWarps + kProducerWarps + 1) * 32;
-constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kProducerThreads = kProducerWarps * 32;
-constexpr int kSub = 2;                  // 512-byte warp loads per step (one commit / wait per step)
-constexpr int kStages = 8;               // ring depth per consumer warp, in steps (x kSub x 512 B)
-constexpr int kTile = 1024;              // list entries staged per tile
-constexpr int kTileBufs = 4;             // tiles in flight between producers and consumers
-constexpr int kTilePerThread = kTile / kProducerThreads;
+constexpr int kWorkers = 19;             // compute warps
+constexpr int kWriterWarp = kWorkers;
+constexpr int kGemvThreads = (kWorkers + 1) * 32;
+constexpr int kChunk = 32;               // list entries per chunk (one per lane)
+constexpr int kDepth = 3;                // chunks in flight per warp
 constexpr unsigned long long kWaitNs = 1000000000ull;  // bound on every mbarrier wait: one second
 
 static int g_tune_ctas = 0;  // 0 = one CTA per SM
 
 #ifdef SPQT_TRACE
-__device__ long long* g_trace;  // [role][event] time stamps of CTA 0 (debug builds only)
+__device__ long long* g_trace;  // time stamps of CTA 0 (debug builds only)
 #define SPQT_TRACE_EVENT(cond, slot) do { if ((cond) && blockIdx.x == 0 && g_trace && (slot) < 4096) g_trace[(slot)] = clock64(); } while (0)
 #else
 #define SPQT_TRACE_EVENT(cond, slot) do { } while (0)
@@ -108,24 +106,22 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity)
     }
 }
 
-// Non-blocking probe of the same condition.
-__device__ __forceinline__ bool mbar_test(uint64_t* bar, unsigned parity)
+__device__ __forceinline__ void cp_async_16(unsigned smem_dst, const void* gmem_src)
 {
-    unsigned done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return done != 0;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
 }
-
-__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gmem_src)
+// the same, asking L2 to fetch no more than the 64 bytes around the address
+__device__ __forceinline__ void cp_async_16_l2_64(unsigned smem_dst, const void* gmem_src)
 {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(smem_dst)), "l"(gmem_src)
-                 : "memory");
+    asm volatile("cp.async.cg.shared.global.L2::64B [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_4(unsigned smem_dst, const void* gmem_src)
+{
+    asm volatile("cp.async.ca.shared.global.L2::64B [%0], [%1], 4;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_4_ca(unsigned smem_dst, const void* gmem_src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
@@ -133,42 +129,45 @@ __device__ __forceinline__ void cp_async_wait()
 {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
-// Wait until at most `allow` of this thread's copy groups are still in flight
-// (rounded down to an encodable count, which only waits longer).
-__device__ __forceinline__ void cp_async_wait_at_most(int allow)
+
+// Two fp32 lanes in one 64-bit register, the operand form of the packed FMA.
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi)
 {
-    if (allow >= kStages - 1) cp_async_wait<kStages - 1>();
-    else if (allow >= 4) cp_async_wait<4>();
-    else if (allow >= 2) cp_async_wait<2>();
-    else if (allow >= 1) cp_async_wait<1>();
-    else cp_async_wait<0>();
+    unsigned long long r;
+    asm("mov.b64 %0, {%1,%2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(unsigned long long v, float& lo, float& hi)
+{
+    asm("mov.b64 {%0,%1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+// d = a * b + d on both lanes with one instruction
+__device__ __forceinline__ void ffma2(unsigned long long& d, unsigned long long a, unsigned long long b)
+{
+    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(d) : "l"(a), "l"(b));
 }
 
-__device__ __forceinline__ void named_barrier_sync(int id, int threads)
-{
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
-}
-
-// d = a * b + d on two fp32 lanes with one instruction
-__device__ __forceinline__ void ffma2(float& d0, float& d1, float a0, float a1, float b0, float b1)
-{
-    unsigned long long a, b, c;
-    asm("mov.b64 %0, {%1,%2};" : "=l"(a) : "f"(a0), "f"(a1));
-    asm("mov.b64 %0, {%1,%2};" : "=l"(b) : "f"(b0), "f"(b1));
-    asm("mov.b64 %0, {%1,%2};" : "=l"(c) : "f"(d0), "f"(d1));
-    asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(c) : "l"(a), "l"(b));
-    asm("mov.b64 {%0,%1}, %2;" : "=f"(d0), "=f"(d1) : "l"(c));
-}
-
-// acc[0..7] += the eight codes of one 32-bit word, each times a*2^-56;
-// mul[j] = a * 2^(93-4j), j = 0..4.
-__device__ __forceinline__ void fma_word(float* acc, unsigned w, const float* mul)
+// acc[0..3] (eight fp32 sums, two per register) += the eight codes of one 32-bit word, each
+// times a*2^-56; m01, m23, m40, m12 hold the multipliers a*2^(93-4j) paired as (0,1) (2,3) (4,0) (1,2).
+__device__ __forceinline__ void fma_word(unsigned long long* acc, unsigned w, unsigned long long m01,
+                                         unsigned long long m23, unsigned long long m40, unsigned long long m12)
 {
     const unsigned v = w >> 20;
-    ffma2(acc[0], acc[1], __uint_as_float(w & 0x0000000fu), __uint_as_float(w & 0x000000f0u), mul[0], mul[1]);
-    ffma2(acc[2], acc[3], __uint_as_float(w & 0x00000f00u), __uint_as_float(w & 0x0000f000u), mul[2], mul[3]);
-    ffma2(acc[4], acc[5], __uint_as_float(w & 0x000f0000u), __uint_as_float(v & 0x0000000fu), mul[4], mul[0]);
-    ffma2(acc[6], acc[7], __uint_as_float(v & 0x000000f0u), __uint_as_float(v & 0x00000f00u), mul[1], mul[2]);
+    ffma2(acc[0], pack2(__uint_as_float(w & 0x0000000fu), __uint_as_float(w & 0x000000f0u)), m01);
+    ffma2(acc[1], pack2(__uint_as_float(w & 0x00000f00u), __uint_as_float(w & 0x0000f000u)), m23);
+    ffma2(acc[2], pack2(__uint_as_float(w & 0x000f0000u), __uint_as_float(v & 0x0000000fu)), m40);
+    ffma2(acc[3], pack2(__uint_as_float(v & 0x000000f0u), __uint_as_float(v & 0x00000f00u)), m12);
+}
+
+// acc (32 fp32 sums in 16 registers) += the 32 codes of a lane's 16 bytes, each times a (scaled by 2^-56).
+__device__ __forceinline__ void fma_block16(unsigned long long* acc, const uint4& w, float a)
+{
+    const float m0 = a * 0x1p93f, m1 = a * 0x1p89f, m2 = a * 0x1p85f, m3 = a * 0x1p81f, m4 = a * 0x1p77f;
+    const unsigned long long m01 = pack2(m0, m1), m23 = pack2(m2, m3), m40 = pack2(m4, m0), m12 = pack2(m1, m2);
+    fma_word(acc + 0, w.x, m01, m23, m40, m12);
+    fma_word(acc + 4, w.y, m01, m23, m40, m12);
+    fma_word(acc + 8, w.z, m01, m23, m40, m12);
+    fma_word(acc + 12, w.w, m01, m23, m40, m12);
 }
 
 // One step of a butterfly reduce-scatter: lanes that differ in bit `bit` hold
@@ -188,17 +187,18 @@ __device__ __forceinline__ void halve(const float* in, float* out, int lane, int
 
 // ---------------------------------------------------------------- work map
 
-// Walks the tiles of one CTA's piece, segment by segment.  All members are
-// uniform across the CTA; producers and consumers each run their own copy and
-// see the same sequence.
-struct TileWalk {
-    int R, P, c, count;
-    int r, r_last;   // current / last block-row of the piece
-    int p1;          // end of the current segment's list slice
-    int t0, len;     // current tile: first list position, entries
-    int tg;          // running tile number (selects buffer and phase)
-    bool last_of_segment;
+// The piece of CTA c: block-rows r_first..r_last, and of each the slice of the
+// active list that belongs to this CTA.  Uniform across the CTA.
+struct Piece {
+    int R, P, c, count, r_first, r_last;
 
+    __device__ __forceinline__ void init(int R_, int P_, int c_, int count_)
+    {
+        R = R_; P = P_; c = c_; count = count_;
+        const long long lo = (long long)c * R, hi = lo + R;
+        r_first = (int)(lo / P);
+        r_last = (int)((hi - 1) / P);
+    }
     __device__ __forceinline__ void slice(int row, int* a, int* b) const
     {
         const long long lo = (long long)c * R, hi = lo + R, base = (long long)row * P;
@@ -207,39 +207,7 @@ struct TileWalk {
         *a = (int)((u0 * count) / P);
         *b = (int)((u1 * count) / P);
     }
-    __device__ __forceinline__ void set_tile(int start)
-    {
-        t0 = start;
-        len = min(kTile, p1 - t0);
-        last_of_segment = (t0 + len >= p1);
-    }
-    __device__ __forceinline__ void init(int R_, int P_, int c_, int count_)
-    {
-        R = R_; P = P_; c = c_; count = count_;
-        const long long lo = (long long)c * R, hi = lo + R;
-        r = (int)(lo / P);
-        r_last = (int)((hi - 1) / P);
-        tg = 0;
-        int p0;
-        slice(r, &p0, &p1);
-        set_tile(p0);
-    }
-    __device__ __forceinline__ bool valid() const { return r <= r_last; }
-    __device__ __forceinline__ void next()
-    {
-        ++tg;
-        if (!last_of_segment) {
-            set_tile(t0 + len);
-        } else {
-            ++r;
-            if (r <= r_last) {
-                int p0;
-                slice(r, &p0, &p1);
-                set_tile(p0);
-            }
-        }
-    }
-    // contributors to block-row `row`: CTAs first..last; this CTA's slot among them
+    // contributors to block-row `row`: CTAs first .. first+n-1
     __device__ __forceinline__ void contributors(int row, int* first, int* n) const
     {
         const int f = (int)(((long long)row * P) / R);
@@ -249,23 +217,54 @@ struct TileWalk {
     }
 };
 
+// A warp's position in its sequence of chunks: list position `pos` of the
+// chunk's first entry inside block-row r (whose slice ends at p1).
+struct Cursor {
+    int r, pos, p1;
+    __device__ __forceinline__ void settle(const Piece& pc, int warp)
+    {
+        while (r <= pc.r_last && pos >= p1) {
+            ++r;
+            if (r <= pc.r_last) {
+                int p0;
+                pc.slice(r, &p0, &p1);
+                pos = p0 + warp * kChunk;
+            }
+        }
+    }
+    __device__ __forceinline__ void init(const Piece& pc, int warp)
+    {
+        r = pc.r_first;
+        int p0;
+        pc.slice(r, &p0, &p1);
+        pos = p0 + warp * kChunk;
+        settle(pc, warp);
+    }
+    __device__ __forceinline__ bool valid(const Piece& pc) const { return r <= pc.r_last; }
+    __device__ __forceinline__ void advance(const Piece& pc, int warp)
+    {
+        pos += kWorkers * kChunk;
+        if (pos >= p1) settle(pc, warp);
+    }
+};
+
 // ---------------------------------------------------------------- kernel
 
 template <int G>
 struct GemvSmem {
     static constexpr int B = G / 2;
-    alignas(16) unsigned char ring[kConsumerWarps][kStages][kSub * 512];
-    alignas(16) unsigned off[kTileBufs][kTile];   // byte offset of the block inside its block-row
-    alignas(16) float a[kTileBufs][kTile];        // x_k * scale_rk
-    alignas(16) float red[2][kConsumerWarps][G];  // per-warp partial sums of a finished segment
-    float red_z[2];                               // its offset term
-    float zs_warp[kTileBufs][kProducerWarps];
-    float zs_tile[kTileBufs];
-    uint64_t full_off[kTileBufs], full_a[kTileBufs], empty[kTileBufs];
+    struct Stage {
+        alignas(16) unsigned char codes[kChunk * B];  // block e of the chunk at e*B
+        unsigned meta[3][kChunk];                     // words holding x_k, scale_rk, zero_rk of entry e
+    };
+    Stage stage[kWorkers][kDepth];
+    alignas(16) int cols[kWorkers][2 * kDepth][kChunk];  // column numbers of the chunks ahead
+    alignas(16) float red[2][kWorkers][G];               // per-warp partial sums of a finished segment
+    float red_z[2][kWorkers];                            // and their offset terms
     uint64_t red_full[2], red_empty[2];
 };
 
-template <int G, bool DENSE>
+template <int G, bool DENSE, bool ODD_N>
 __global__ void __launch_bounds__(kGemvThreads, 1)
 gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales,
                  const __half* __restrict__ zeros, int R, int n,
@@ -276,8 +275,10 @@ gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ s
 {
     constexpr int B = G / 2;
     constexpr int LPB = B / 16;       // lanes that share one block
-    constexpr int SLOTS = 32 / LPB;   // blocks per warp step
+    constexpr int SLOTS = 32 / LPB;   // blocks per 512-byte warp load
     constexpr int KEEP = 32 / SLOTS;  // values per lane after the in-warp reduce-scatter
+    constexpr int SUBS = kChunk / SLOTS;  // 512-byte loads per chunk
+    constexpr int D = kDepth;
 
     extern __shared__ __align__(16) unsigned char smem_raw[];
     GemvSmem<G>& sm = *reinterpret_cast<GemvSmem<G>*>(smem_raw);
@@ -286,123 +287,40 @@ gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ s
     const int P = gridDim.x, c = blockIdx.x;
 
     if (tid == 0) {
-        for (int b = 0; b < kTileBufs; ++b) {
-            mbar_init(&sm.full_off[b], kProducerThreads);
-            mbar_init(&sm.full_a[b], kProducerThreads);
-            mbar_init(&sm.empty[b], kConsumerWarps);
-        }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(&sm.red_full[b], kConsumerWarps);
+            mbar_init(&sm.red_full[b], kWorkers);
             mbar_init(&sm.red_empty[b], 1);
         }
     }
     __syncthreads();
 
     const int count = DENSE ? n : *count_ptr;
+    Piece pc;
+    pc.init(R, P, c, count);
     SPQT_TRACE_EVENT(tid == 0, 4000);
-
-    if (warp >= kConsumerWarps && warp < kWriterWarp) {
-        // ------------------------------------------------------------ producers
-        const int pt = tid - kConsumerThreads, pw = warp - kConsumerWarps;
-        const unsigned short* xb = reinterpret_cast<const unsigned short*>(x);
-        const unsigned short* sb = reinterpret_cast<const unsigned short*>(scales);
-        const unsigned short* zb = reinterpret_cast<const unsigned short*>(zeros);
-
-        // column of list entry i of a tile (entries past the tile's end repeat its last one,
-        // so that every load below is unconditional and in bounds)
-        auto load_cols = [&](const TileWalk& t, int* k) {
-            if (t.len > 0) {
-#pragma unroll
-                for (int u = 0; u < kTilePerThread; ++u) {
-                    const int i = min(pt + u * kProducerThreads, t.len - 1);
-                    k[u] = DENSE ? (t.t0 + i) : __ldg(idx + t.t0 + i);
-                }
-            } else {
-#pragma unroll
-                for (int u = 0; u < kTilePerThread; ++u) k[u] = 0;
-            }
-        };
-
-        TileWalk w;
-        w.init(R, P, c, count);
-        int k[kTilePerThread];
-        if (w.valid()) load_cols(w, k);
-        bool ok = true;
-        while (w.valid()) {
-            const int buf = w.tg % kTileBufs;
-            SPQT_TRACE_EVENT(pt == 0, w.tg * 4 + 0);
-            if (w.tg >= kTileBufs) ok = mbar_wait(&sm.empty[buf], ((w.tg / kTileBufs) - 1) & 1);
-            if (!ok) break;
-            SPQT_TRACE_EVENT(pt == 0, w.tg * 4 + 1);
-            const size_t row_base = (size_t)w.r * (size_t)n;
-#pragma unroll
-            for (int u = 0; u < kTilePerThread; ++u)
-                sm.off[buf][pt + u * kProducerThreads] = (unsigned)k[u] * (unsigned)B;
-            mbar_arrive(&sm.full_off[buf]);
-            SPQT_TRACE_EVENT(pt == 0, w.tg * 4 + 2);
-            // all gathers of this tile in flight at once, then the next tile's columns
-            unsigned short xr[kTilePerThread], sr[kTilePerThread], zr[kTilePerThread];
-#pragma unroll
-            for (int u = 0; u < kTilePerThread; ++u) {
-                xr[u] = __ldg(xb + k[u]);
-                sr[u] = __ldg(sb + row_base + k[u]);
-                zr[u] = __ldg(zb + row_base + k[u]);
-            }
-            TileWalk wn = w;
-            wn.next();
-            int kn[kTilePerThread];
-            if (wn.valid()) load_cols(wn, kn);
-            float zs = 0.0f;
-#pragma unroll
-            for (int u = 0; u < kTilePerThread; ++u) {
-                const bool in = pt + u * kProducerThreads < w.len;
-                const float xf = in ? __half2float(__ushort_as_half(xr[u])) : 0.0f;
-                sm.a[buf][pt + u * kProducerThreads] = xf * __half2float(__ushort_as_half(sr[u]));  // exact
-                zs = fmaf(xf, __half2float(__ushort_as_half(zr[u])), zs);
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) zs += __shfl_xor_sync(0xffffffffu, zs, o);
-            if (lane == 0) sm.zs_warp[buf][pw] = zs;
-            named_barrier_sync(2, kProducerThreads);
-            if (pt == 0) {
-                float t = 0.0f;
-#pragma unroll
-                for (int q = 0; q < kProducerWarps; ++q) t += sm.zs_warp[buf][q];
-                sm.zs_tile[buf] = t;
-            }
-            mbar_arrive(&sm.full_a[buf]);
-            SPQT_TRACE_EVENT(pt == 0, w.tg * 4 + 3);
-            w = wn;
-#pragma unroll
-            for (int u = 0; u < kTilePerThread; ++u) k[u] = kn[u];
-        }
-        if (!ok && pt == 0) atomicExch(status, 1);
-        return;
-    }
 
     if (warp == kWriterWarp) {
         // ------------------------------------------------------------ writer
         constexpr int RPL = G / 32;  // rows per lane
-        TileWalk w;
-        w.init(R, P, c, count);
-        const int r_first = w.r, r_last = w.r_last;
         bool ok = true;
-        for (int r = r_first, sg = 0; r <= r_last; ++r, ++sg) {
+        for (int r = pc.r_first, sg = 0; r <= pc.r_last; ++r, ++sg) {
             const int b = sg & 1;
             ok = mbar_wait(&sm.red_full[b], (sg >> 1) & 1);
             if (!ok) break;
             float v[RPL];
 #pragma unroll
             for (int i = 0; i < RPL; ++i) v[i] = 0.0f;
+            float zpart = 0.0f;
 #pragma unroll
-            for (int q = 0; q < kConsumerWarps; ++q)
+            for (int q = 0; q < kWorkers; ++q) {
 #pragma unroll
                 for (int i = 0; i < RPL; ++i) v[i] += sm.red[b][q][lane * RPL + i];
-            const float zpart = sm.red_z[b];
+                zpart += sm.red_z[b][q];
+            }
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.red_empty[b]);
             int first, nslots;
-            w.contributors(r, &first, &nslots);
+            pc.contributors(r, &first, &nslots);
             const size_t pslot = (size_t)r * max_slots + (c - first);
 #pragma unroll
             for (int i = 0; i < RPL; ++i) __stcg(partials + pslot * G + lane * RPL + i, v[i]);
@@ -434,203 +352,209 @@ gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ s
         return;
     }
 
-    // ---------------------------------------------------------------- consumers
+    // ---------------------------------------------------------------- workers
     const int slot = lane / LPB, h = lane % LPB;
-    constexpr unsigned kStepBytes = kSub * 512;
-    constexpr unsigned kRingBytes = kStages * kStepBytes;
-    constexpr int kStepCols = kSub * SLOTS;               // list entries per step
-    constexpr int kStride = kConsumerWarps * kStepCols;   // list entries between two steps of one warp
-    const unsigned ring_base = smem_u32(&sm.ring[warp][0][0]) + lane * 16;
+    const unsigned short* xb = reinterpret_cast<const unsigned short*>(x);
 
-    float acc[32];
-#pragma unroll
-    for (int i = 0; i < 32; ++i) acc[i] = 0.0f;
-    float zacc = 0.0f;  // meaningful in consumer thread 0 only
-    bool ok = true;
+    typename GemvSmem<G>::Stage* my_stage = &sm.stage[warp][0];
+    int (*my_cols)[kChunk] = sm.cols[warp];
 
-    // ---- issue side: runs up to kStages steps (and at most kTileBufs-1 tiles) ahead
-    TileWalk wi;
-    wi.init(R, P, c, count);
-    int ie = warp * kStepCols;        // first list entry (within the tile) of the next step to issue
-    bool i_open = false;              // current issue tile staged and has steps left for this warp
-    const unsigned* i_off = nullptr;  // &off[buf][slot]
-    const uint8_t* i_row = nullptr;   // codes of the tile's block-row, this lane's 16-byte part
-    unsigned ring_w = 0, ring_r = 0;
-    int in_flight = 0;
-    int consume_tg = 0;               // tile the consume side is in
+    Cursor ca, cb;  // stage A / stage B cursors (the consume side walks the segments itself)
+    ca.init(pc, warp);
+    cb = ca;
+    unsigned qa = 0, qb = 0, qc = 0;  // chunk sequence numbers of the three stages
 
-    // Move to the next tile in which this warp has a step, if producers have staged it.
-    // Only blocks when `must` (nothing in flight, so the consume side cannot go on otherwise).
-    auto open_issue_tile = [&](bool must) {
-        while (wi.valid() && ie >= wi.len) {
-            wi.next();
-            ie = warp * kStepCols;
+    // block-row constants of stage B, refreshed when its cursor enters a new block-row
+    int b_row = -1;
+    unsigned b_par = 0;                       // parity of r*n: which half of a word holds element (r,k)
+    const uint8_t* b_codes = nullptr;         // codes of the block-row, this lane's 16-byte part
+    const unsigned short* b_scales = nullptr; // scales / zeros of the block-row
+    const unsigned short* b_zeros = nullptr;
+
+    // stage A: column numbers of the warp's chunk number qa
+    auto issue_a = [&]() {
+        if (!DENSE && ca.valid(pc)) {
+            if (ca.pos + lane < ca.p1) cp_async_4(smem_u32(&my_cols[qa % (2 * D)][lane]), idx + ca.pos + lane);
+            ca.advance(pc, warp);
+            ++qa;
         }
-        if (!wi.valid() || wi.tg > consume_tg + (kTileBufs - 1)) return;
-        const int buf = wi.tg % kTileBufs;
-        const unsigned parity = (wi.tg / kTileBufs) & 1;
-        if (must) {
-            ok = mbar_wait(&sm.full_off[buf], parity);
-            if (!ok) return;
-        } else if (!mbar_test(&sm.full_off[buf], parity)) {
-            return;
-        }
-        i_off = &sm.off[buf][slot];
-        i_row = codes + (size_t)wi.r * (size_t)n * B + 16 * h;
-        i_open = true;
     };
-    auto top_up = [&]() {
-        while (in_flight < kStages) {
-            if (!i_open) {
-                open_issue_tile(in_flight == 0);
-                if (!i_open) return;
+    // stage B: code blocks and metadata words of chunk number qb (its columns have landed)
+    auto issue_b = [&]() {
+        if (cb.valid(pc)) {
+            if (cb.r != b_row) {
+                b_row = cb.r;
+                const size_t row_base = (size_t)b_row * (size_t)n;
+                b_par = (unsigned)(row_base & 1);
+                b_codes = codes + row_base * B + 16 * h;
+                b_scales = reinterpret_cast<const unsigned short*>(scales) + row_base;
+                b_zeros = reinterpret_cast<const unsigned short*>(zeros) + row_base;
             }
+            const int valid = cb.p1 - cb.pos;  // entries of this chunk (>= kChunk when full)
+            const int* cols = my_cols[qb % (2 * D)];
+            typename GemvSmem<G>::Stage& st = my_stage[qb % D];
+            const unsigned dst = smem_u32(&st.codes[0]) + lane * 16;
 #pragma unroll
-            for (int u = 0; u < kSub; ++u) {
-#ifdef SPQT_NO_COPY
-                if (false) {
-#else
-                if (ie + u * SLOTS + slot < wi.len) {
-#endif
-                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(ring_base + ring_w + u * 512),
-                                 "l"(i_row + i_off[ie + u * SLOTS])
-                                 : "memory");
+            for (int u = 0; u < SUBS; ++u) {
+                const int e = u * SLOTS + slot;
+                if (e < valid) {
+                    const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : (unsigned)cols[e];
+                    if (DENSE) cp_async_16(dst + u * 512, b_codes + (size_t)kk * B);
+                    else cp_async_16_l2_64(dst + u * 512, b_codes + (size_t)kk * B);
                 }
             }
-            cp_async_commit();
-            ring_w = (ring_w + kStepBytes) & (kRingBytes - 1);
-            ++in_flight;
-            ie += kStride;
-            if (ie >= wi.len) i_open = false;
-        }
-    };
-    // next step's codes and multipliers into registers (its copies have been in flight for kStages steps)
-    struct Step {
-        uint4 w[kSub];
-        float a[kSub];
-    };
-    auto fetch = [&](const float* a_ptr, int e, Step& st) {
-        top_up();
-        cp_async_wait_at_most(in_flight - 1);
-#pragma unroll
-        for (int u = 0; u < kSub; ++u) {
-            st.w[u] = *reinterpret_cast<const uint4*>(&sm.ring[warp][0][0] + lane * 16 + ring_r + u * 512);
-            st.a[u] = a_ptr[e + u * SLOTS];  // 0 past the tile's end: stale ring data is harmless
-        }
-        ring_r = (ring_r + kStepBytes) & (kRingBytes - 1);
-        --in_flight;
-    };
-    auto math = [&](const Step& st) {
-#ifdef SPQT_NO_MATH
-        acc[0] += __uint_as_float(st.w[0].x ^ st.w[1].y) * st.a[0] + st.a[1];
-        return;
-#endif
-#pragma unroll
-        for (int u = 0; u < kSub; ++u) {
-            float mul[5];
-            mul[0] = st.a[u] * 0x1p93f;
-            mul[1] = st.a[u] * 0x1p89f;
-            mul[2] = st.a[u] * 0x1p85f;
-            mul[3] = st.a[u] * 0x1p81f;
-            mul[4] = st.a[u] * 0x1p77f;
-            fma_word(acc + 0, st.w[u].x, mul);
-            fma_word(acc + 8, st.w[u].y, mul);
-            fma_word(acc + 16, st.w[u].z, mul);
-            fma_word(acc + 24, st.w[u].w, mul);
+            if (lane < valid) {
+                // the aligned 4-byte word that holds each fp16 value (index rounded down to even)
+                const unsigned kk = DENSE ? (unsigned)(cb.pos + lane) : (unsigned)cols[lane];
+                const unsigned mdst = smem_u32(&st.meta[0][lane]);
+                const int mo = (int)kk - (int)((kk ^ b_par) & 1u);  // may be -1 only when r*n is odd: still inside the array
+                if (!ODD_N || kk != (unsigned)(n - 1)) {
+                    cp_async_4_ca(mdst, xb + (kk & ~1u));
+                    cp_async_4(mdst + kChunk * 4, b_scales + mo);
+                    cp_async_4(mdst + 2 * kChunk * 4, b_zeros + mo);
+                } else {
+                    // n odd: the word of the last column may reach past the end of an array; fetch directly
+                    st.meta[0][lane] = (unsigned)__ldg(xb + kk) << ((kk & 1u) * 16);
+                    st.meta[1][lane] = (unsigned)__ldg(b_scales + kk) << (((kk ^ b_par) & 1u) * 16);
+                    st.meta[2][lane] = (unsigned)__ldg(b_zeros + kk) << (((kk ^ b_par) & 1u) * 16);
+                }
+            }
+            cb.advance(pc, warp);
+            ++qb;
         }
     };
 
-    // ---- consume side
-    TileWalk wc;
-    wc.init(R, P, c, count);
-    int sg = 0;  // segments finished by this CTA
-    for (; wc.valid() && ok; wc.next()) {
-        const int buf = wc.tg % kTileBufs;
-        consume_tg = wc.tg;
-        top_up();
-        if (!ok) break;
-        // every warp observes every tile's hand-over before releasing it
-        ok = mbar_wait(&sm.full_a[buf], (wc.tg / kTileBufs) & 1);
-        if (!ok) break;
-        if (tid == 0) zacc += sm.zs_tile[buf];
-        SPQT_TRACE_EVENT(tid == 0, 1024 + wc.tg * 4 + 0);
-        const float* a_ptr = &sm.a[buf][slot];
-        int e = warp * kStepCols;
-        if (e < wc.len) {
-            // two steps in registers: the next one is fetched before this one's arithmetic
-            Step s0, s1;
-            fetch(a_ptr, e, s0);
-            for (;;) {
-                e += kStride;
-                if (e >= wc.len) { math(s0); break; }
-                fetch(a_ptr, e, s1);
-                math(s0);
-                e += kStride;
-                if (e >= wc.len) { math(s1); break; }
-                fetch(a_ptr, e, s0);
-                math(s1);
-            }
-        }
-        if (!ok) break;
+    // fill the pipeline: D chunks of columns, then D chunks of blocks (each needs its columns)
+#pragma unroll 1
+    for (int s = 0; s < D; ++s) {
+        issue_a();
+        cp_async_commit();
+    }
+#pragma unroll 1
+    for (int s = 0; s < D; ++s) {
+        cp_async_wait<D - 1>();
         __syncwarp();
-        SPQT_TRACE_EVENT(tid == 0, 1024 + wc.tg * 4 + 1);
-        if (lane == 0) mbar_arrive(&sm.empty[buf]);
-        if (wc.last_of_segment) {
-            // ---- segment epilogue: in-warp reduce-scatter over the column slots,
-            // then hand the per-warp sums to the writer warp
-            const int b = sg & 1;
-            if (sg >= 2) {
-                ok = mbar_wait(&sm.red_empty[b], ((sg >> 1) - 1) & 1);
-                if (!ok) break;
-            }
-            float t16[16], t8[8], t4[4], keep[4];
-            halve<32>(acc, t16, lane, 16);
-            halve<16>(t16, t8, lane, 8);
-            halve<8>(t8, t4, lane, 4);
-            int a_base;
-            if (LPB == 4) {
+        issue_b();
+        issue_a();
+        cp_async_commit();
+    }
+
+    unsigned long long acc[16];  // 32 fp32 sums, two per register
 #pragma unroll
-                for (int i = 0; i < 4; ++i) keep[i] = t4[i];
-                a_base = lane & 0x1c;
-            } else {
-                float t2[2];
-                halve<4>(t4, t2, lane, 2);
-                keep[0] = t2[0];
-                keep[1] = t2[1];
-                a_base = lane & 0x1e;
-            }
-#pragma unroll
-            for (int i = 0; i < KEEP; ++i) {
-                const int ai = a_base + i;  // accumulator index = word*8 + nibble
-                const int cw = ai >> 3, e2 = ai & 7;
-                const int row = 16 * h + 4 * cw + (e2 >> 1) + (e2 & 1) * (G / 2);
-                sm.red[b][warp][row] = keep[i] * 0x1p56f;  // undo the 2^-56 of the subnormal trick
-            }
-#pragma unroll
-            for (int i = 0; i < 32; ++i) acc[i] = 0.0f;
-            if (tid == 0) {
-                sm.red_z[b] = zacc;
-                zacc = 0.0f;
-            }
+    for (int i = 0; i < 16; ++i) acc[i] = 0ull;
+    bool ok = true;
+#ifdef SPQT_TRACE
+    long long tr_wait = 0, tr_issue = 0, tr_math = 0, tr_n = 0;
+    SPQT_TRACE_EVENT(lane == 0, 3900 + warp);
+#endif
+
+    for (int r = pc.r_first, sg = 0; r <= pc.r_last; ++r, ++sg) {
+        int p0, p1;
+        pc.slice(r, &p0, &p1);
+        const unsigned c_par = (unsigned)(((size_t)r * (size_t)n) & 1);
+        float zl = 0.0f;  // this lane's share of sum x_k * zero_rk
+        for (int pos = p0 + warp * kChunk; pos < p1; pos += kWorkers * kChunk) {
+            // ---- stage C of chunk qc: everything it needs is in commit groups that wait<D-1> covers
+#ifdef SPQT_TRACE
+            const long long tc0 = clock64();
+#endif
+            cp_async_wait<D - 1>();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.red_full[b]);
-            ++sg;
+#ifdef SPQT_TRACE
+            const long long tc1 = clock64();
+#endif
+            const typename GemvSmem<G>::Stage& st = my_stage[qc % D];
+            const unsigned xw = st.meta[0][lane], sw = st.meta[1][lane], zw = st.meta[2][lane];
+            const unsigned kk = DENSE ? (unsigned)(pos + lane) : (unsigned)my_cols[qc % (2 * D)][lane];
+#ifdef SPQT_TRACE
+            const long long tc2 = clock64();
+#endif
+            float a = 0.0f;
+            if (pos + lane < p1) {
+                const unsigned xs = (kk & 1u) * 16, ms = ((kk ^ c_par) & 1u) * 16;
+                const float xf = __half2float(__ushort_as_half((unsigned short)(xw >> xs)));
+                const float sf = __half2float(__ushort_as_half((unsigned short)(sw >> ms)));
+                const float zf = __half2float(__ushort_as_half((unsigned short)(zw >> ms)));
+                a = xf * sf;  // exact; stays 0 past the end of the slice, where the code bytes are stale
+                zl = fmaf(xf, zf, zl);
+            }
+#pragma unroll
+            for (int u = 0; u < SUBS; ++u) {
+                const uint4 wv = *reinterpret_cast<const uint4*>(&st.codes[0] + lane * 16 + u * 512);
+                const float au = __shfl_sync(0xffffffffu, a, u * SLOTS + slot);
+                fma_block16(acc, wv, au);
+            }
+            __syncwarp();  // every lane has read its part of the slots that B and A now refill
+            issue_b();
+            issue_a();
+            cp_async_commit();
+            ++qc;
+#ifdef SPQT_TRACE
+            tr_wait += tc1 - tc0; tr_issue += 0; tr_math += clock64() - tc2; ++tr_n;
+#endif
         }
-        SPQT_TRACE_EVENT(tid == 0, 1024 + wc.tg * 4 + 2);
+
+        // ---- end of the segment: in-warp reduce-scatter over the column slots, then hand the
+        // per-warp sums to the writer warp
+        const int b = sg & 1;
+        if (sg >= 2) {
+            ok = mbar_wait(&sm.red_empty[b], ((sg >> 1) - 1) & 1);
+            if (!ok) break;
+        }
+        float accf[32];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            unpack2(acc[i], accf[2 * i], accf[2 * i + 1]);
+            acc[i] = 0ull;
+        }
+        float t16[16], t8[8], t4[4], keep[4];
+        halve<32>(accf, t16, lane, 16);
+        halve<16>(t16, t8, lane, 8);
+        halve<8>(t8, t4, lane, 4);
+        int a_base;
+        if (LPB == 4) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) keep[i] = t4[i];
+            a_base = lane & 0x1c;
+        } else {
+            float t2[2];
+            halve<4>(t4, t2, lane, 2);
+            keep[0] = t2[0];
+            keep[1] = t2[1];
+            a_base = lane & 0x1e;
+        }
+#pragma unroll
+        for (int i = 0; i < KEEP; ++i) {
+            const int ai = a_base + i;  // accumulator index = word*8 + nibble
+            const int cw = ai >> 3, e2 = ai & 7;
+            const int row = 16 * h + 4 * cw + (e2 >> 1) + (e2 & 1) * (G / 2);
+            sm.red[b][warp][row] = keep[i] * 0x1p56f;  // undo the 2^-56 of the subnormal trick
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) zl += __shfl_xor_sync(0xffffffffu, zl, o);
+        if (lane == 0) sm.red_z[b][warp] = zl;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.red_full[b]);
     }
     cp_async_wait<0>();
     SPQT_TRACE_EVENT(tid == 0, 4001);
+#ifdef SPQT_TRACE
+    if (blockIdx.x == 0 && lane == 0 && g_trace) {
+        g_trace[3000 + warp * 4 + 0] = tr_wait; g_trace[3000 + warp * 4 + 1] = tr_issue;
+        g_trace[3000 + warp * 4 + 2] = tr_math; g_trace[3000 + warp * 4 + 3] = tr_n;
+    }
+#endif
     if (!ok && lane == 0) atomicExch(status, 1);
 }
 
 // ---------------------------------------------------------------- host side
 
-template <int G, bool DENSE>
+template <int G, bool DENSE, bool ODD_N>
 static spqt_status launch_int4(const Format& f, const void* codes, const void* scales,
                                const void* zeros, const void* x, const int32_t* idx,
                                const int32_t* count, void* y, void* workspace, cudaStream_t s)
 {
-    auto kernel = gemv_int4_kernel<G, DENSE>;
+    auto kernel = gemv_int4_kernel<G, DENSE, ODD_N>;
     static bool configured[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPQT_ERR_CUDA;
@@ -672,16 +596,18 @@ static spqt_status gemv_entry(const void* codes, const void* scales, const void*
     Format f;
     spqt_status st = make_format(m, n, bits, group, &f);
     if (st != SPQT_OK) return st;
-    if ((size_t)n * (size_t)f.B > 0xffffffffull) return SPQT_ERR_UNSUPPORTED;  // 32-bit offsets inside a block-row
-    if (!aligned(codes, 16) || !aligned(scales, 16) || !aligned(zeros, 16) || !aligned(x, 2) ||
+    if (!aligned(codes, 16) || !aligned(scales, 16) || !aligned(zeros, 16) || !aligned(x, 4) ||
         !aligned(y, 2) || !aligned(workspace, 16) || (!DENSE && (!aligned(idx, 4) || !aligned(count, 4))))
         return SPQT_ERR_ALIGNMENT;
     if (ws_bytes < workspace_bytes(f)) return SPQT_ERR_WORKSPACE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const bool odd = (n & 1) != 0;
     if (bits == 4 && group == 128)
-        return launch_int4<128, DENSE>(f, codes, scales, zeros, x, idx, count, y, workspace, s);
+        return odd ? launch_int4<128, DENSE, true>(f, codes, scales, zeros, x, idx, count, y, workspace, s)
+                   : launch_int4<128, DENSE, false>(f, codes, scales, zeros, x, idx, count, y, workspace, s);
     if (bits == 4 && group == 64)
-        return launch_int4<64, DENSE>(f, codes, scales, zeros, x, idx, count, y, workspace, s);
+        return odd ? launch_int4<64, DENSE, true>(f, codes, scales, zeros, x, idx, count, y, workspace, s)
+                   : launch_int4<64, DENSE, false>(f, codes, scales, zeros, x, idx, count, y, workspace, s);
     return SPQT_ERR_UNSUPPORTED;
 }
 
