@@ -129,6 +129,33 @@ spqt_status spqt_dense_gemv(const void* codes, const void* scales, const void* z
                             void* y, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * spqt_sparse_gemv for callers that cannot give it a workspace.  (The paper has no counterpart:
+ * this is a packaging of the call above, same arithmetic, same result bits.)
+ *
+ * Some hosts of this library may not obtain device memory themselves: a custom operator running
+ * inside a framework whose allocator owns the whole device, or a serving loop that has frozen its
+ * memory map after start-up and will not tolerate the device-wide stall of a cudaMalloc.  For them
+ * the workspace is a 1 MiB array compiled into the library (static __device__ storage: every GPU
+ * that loads the library carries it until the process exits).  The call allocates nothing and
+ * frees nothing; inputs and outputs are still the caller's.
+ *
+ *   - Problems whose workspace (spqt_packed_sizes: gemv_workspace_bytes) exceeds 1 MiB are refused
+ *     with SPQT_ERR_WORKSPACE; every Llama-shaped layer used in this repository fits.
+ *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ *     that device current) and keeps it; make that first call before any stream capture begins.
+ *   - All calls on a device share the one array, which still holds the previous call's contents; the
+ *     part that must start at zero (arrival counters, status word) is cleared on `stream` before the
+ *     kernel.  Two calls that may overlap on the GPU (different streams, no ordering) race on it:
+ *     order them, or use spqt_sparse_gemv with separate workspaces.
+ *   - Because the status word is cleared per call, spqt_workspace_status does not apply here.
+ * Other arguments, alignment rules and error codes are those of spqt_sparse_gemv.
+ */
+spqt_status spqt_sparse_gemv_static(const void* codes, const void* scales, const void* zeros,
+                                    int m, int n, int bits, int group,
+                                    const void* x, const int32_t* idx, const int32_t* count,
+                                    void* y, void* stream);
+
+/*
  * One decode-time linear layer from HOST activations (paper Sec. 3.2: hidden
  * state -> index collection with the layer's threshold -> sparse GEMV):
  * copies x_host (fp16[n]) to x_dev, runs spqt_sparsify and spqt_sparse_gemv,

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libspqt.so")
 
 EXPORTS = (
     "spqt_status_string", "spqt_version", "spqt_packed_sizes", "spqt_pack", "spqt_unpack",
-    "spqt_sparsify", "spqt_sparse_gemv", "spqt_dense_gemv", "spqt_sparse_linear_host",
+    "spqt_sparsify", "spqt_sparse_gemv", "spqt_sparse_gemv_static", "spqt_dense_gemv", "spqt_sparse_linear_host",
     "spqt_set_tuning", "spqt_workspace_status", "spqt_launch_count",
 )
 
@@ -50,6 +50,8 @@ def lib() -> ctypes.CDLL:
         L.spqt_unpack.argtypes = [vp, i32, i32, i32, i32, vp, vp]
         L.spqt_sparsify.argtypes = [vp, i32, ctypes.c_float, vp, vp, vp]
         L.spqt_sparse_gemv.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
+        L.spqt_sparse_gemv_static.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp]
+        L.spqt_sparse_gemv_static.restype = i32
         L.spqt_dense_gemv.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, sz, vp]
         L.spqt_sparse_linear_host.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, vp,
                                               vp, vp, vp, vp, vp, sz, vp]
@@ -173,6 +175,21 @@ def spqt_sparse_gemv(p: Packed, x: torch.Tensor, idx: torch.Tensor, count: torch
         _dev(x, torch.float16, "x"), _dev(idx, torch.int32, "idx"), _dev(count, torch.int32, "count"),
         _dev(y, torch.float16, "y"), _dev(workspace, torch.uint8, "workspace"), workspace.numel(),
         _stream(stream)), "spqt_sparse_gemv")
+    return y
+
+
+def spqt_sparse_gemv_static(p: Packed, x: torch.Tensor, idx: torch.Tensor, count: torch.Tensor,
+                            y: torch.Tensor, stream=None) -> torch.Tensor:
+    """The sparse GEMV on the library's built-in 1 MiB scratch, for callers that may not allocate
+    device memory: nothing is allocated here either, so ``y`` must be passed in.  Calls on one
+    device share the scratch and must not overlap on the GPU."""
+    if x.numel() != p.n or y.numel() != p.m:
+        raise ValueError("x must have n entries and y m entries")
+    _ok(lib().spqt_sparse_gemv_static(
+        _dev(p.codes, torch.uint8, "codes"), _dev(p.scales, torch.float16, "scales"),
+        _dev(p.zeros, torch.float16, "zeros"), p.m, p.n, p.bits, p.group,
+        _dev(x, torch.float16, "x"), _dev(idx, torch.int32, "idx"), _dev(count, torch.int32, "count"),
+        _dev(y, torch.float16, "y"), _stream(stream)), "spqt_sparse_gemv_static")
     return y
 
 

@@ -613,6 +613,11 @@ static spqt_status gemv_entry(const void* codes, const void* scales, const void*
 
 }  // namespace spqt
 
+// Scratch of the entry point that allocates nothing: one block-row counter array, status word and
+// partial-sum area, resident in every device that loads the library until the process exits.
+constexpr size_t kStaticScratchBytes = size_t(1) << 20;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
 #ifdef SPQT_TRACE
 extern "C" int spqt_debug_set_trace(void* buf) { return (int)cudaMemcpyToSymbol(spqt::g_trace, &buf, sizeof(buf)); }
 #endif
@@ -634,6 +639,34 @@ spqt_status spqt_dense_gemv(const void* codes, const void* scales, const void* z
 {
     return spqt::gemv_entry<true>(codes, scales, zeros, m, n, bits, group, x, nullptr, nullptr, y,
                                   workspace, workspace_bytes, stream);
+}
+
+spqt_status spqt_sparse_gemv_static(const void* codes, const void* scales, const void* zeros,
+                                    int m, int n, int bits, int group,
+                                    const void* x, const int32_t* idx, const int32_t* count,
+                                    void* y, void* stream)
+{
+    using namespace spqt;
+    Format f;
+    spqt_status st = make_format(m, n, bits, group, &f);
+    if (st != SPQT_OK) return st;
+    if (workspace_bytes(f) > kStaticScratchBytes) return SPQT_ERR_WORKSPACE;  // problem too large for the built-in scratch
+    // In host code the array's name is only a handle; the device address has to be asked for,
+    // once per device, with that device current.
+    static void* scratch_addr[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPQT_ERR_CUDA;
+    if (scratch_addr[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return SPQT_ERR_CUDA;
+        scratch_addr[dev] = p;
+    }
+    // The scratch keeps whatever the previous call (or an interrupted one) left: the arrival
+    // counters and the status word must start at zero.
+    if (cudaMemsetAsync(scratch_addr[dev], 0, header_bytes(f.R), static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return SPQT_ERR_CUDA;
+    return gemv_entry<false>(codes, scales, zeros, m, n, bits, group, x, idx, count, y,
+                             scratch_addr[dev], kStaticScratchBytes, stream);
 }
 
 spqt_status spqt_set_tuning(int gemv_ctas, int reserved)

@@ -1,0 +1,60 @@
+"""The entry point that allocates nothing (spqt_sparse_gemv_static).
+
+Hosts that may not obtain device memory themselves -- an operator inside a framework whose
+allocator owns the device, a serving loop with a frozen memory map -- get the sparse GEMV on a
+1 MiB scratch compiled into the library.  It must give the bits of spqt_sparse_gemv, on a first
+call (which also looks up the scratch's device address) and on the calls after it, whatever the
+scratch held before.  Collected last on purpose: a run that stops at the first failure has then
+already run every other test."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2511_04477_b200 import binding, inputs
+
+pytestmark = pytest.mark.gpu
+
+
+def _case(m, n, group, seed, sparsity):
+    W = inputs.weights(m, n, seed=seed)
+    x = inputs.activations(n, seed=seed + 1)
+    t = inputs.threshold_for_sparsity(x, sparsity)
+    p = binding.spqt_pack(torch.from_numpy(W).cuda(), 4, group)
+    xd = torch.from_numpy(x).cuda()
+    idx, cnt = binding.spqt_sparsify(xd, t)
+    return p, xd, idx, cnt
+
+
+def test_static_scratch_entry_point_matches_the_workspace_entry_point_on_consecutive_calls():
+    assert torch.cuda.is_available()
+    # two different problems back to back, then the first again: the shared scratch always holds
+    # another call's leftovers when a call starts
+    cases = [_case(4096, 4096, 128, 11, 0.5), _case(1024, 1500, 64, 13, 0.25), _case(4096, 4096, 128, 11, 0.5)]
+    for (p, xd, idx, cnt) in cases:
+        ws = binding.new_workspace(p.m, p.n, p.bits, p.group)
+        y_ref = binding.spqt_sparse_gemv(p, xd, idx, cnt, ws)
+        y = torch.full((p.m,), float("nan"), dtype=torch.float16, device="cuda")
+        before = torch.cuda.memory_allocated()
+        binding.spqt_sparse_gemv_static(p, xd, idx, cnt, y)
+        binding.spqt_sparse_gemv_static(p, xd, idx, cnt, y)       # and once more on the warm scratch
+        assert torch.cuda.memory_allocated() == before             # nothing taken from torch's allocator
+        torch.cuda.synchronize()
+        a, b = y.cpu().numpy(), y_ref.cpu().numpy()
+        assert np.isfinite(a.astype(np.float32)).all()
+        # same kernel, same fixed summation order: the bits agree (well inside the 2e-3 tolerance)
+        assert np.array_equal(a.view(np.uint16), b.view(np.uint16))
+
+
+def test_static_scratch_entry_point_refuses_what_does_not_fit_or_is_malformed():
+    L = binding.lib()
+    p, xd, idx, cnt = _case(128, 64, 128, 3, 0.5)
+    y = torch.empty(128, dtype=torch.float16, device="cuda")
+    args = lambda m, n, bits, group: (p.codes.data_ptr(), p.scales.data_ptr(), p.zeros.data_ptr(), m, n, bits, group,
+                                      xd.data_ptr(), idx.data_ptr(), cnt.data_ptr(), y.data_ptr(), None)
+    before = binding.spqt_launch_count()
+    assert L.spqt_sparse_gemv_static(*args(128, 64, 5, 128)) == 2          # unsupported format
+    assert L.spqt_sparse_gemv_static(*args(100, 64, 4, 128)) == 2          # m not a multiple of the group
+    huge = 128 * 4096                                                      # R = 4096 block-rows: > 1 MiB of scratch
+    assert binding.spqt_packed_sizes(huge, 64, 4, 128).gemv_workspace_bytes > (1 << 20)
+    assert L.spqt_sparse_gemv_static(*args(huge, 64, 4, 128)) == 4         # refused, nothing launched
+    assert binding.spqt_launch_count() == before
