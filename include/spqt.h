@@ -121,6 +121,19 @@ spqt_status spqt_sparse_gemv(const void* codes, const void* scales, const void* 
                              void* y, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * spqt_sparsify followed by spqt_sparse_gemv in ONE launch (the paper runs the index collection as
+ * a kernel of its own before every GEMV, Sec. 4.2.3; on this GPU a separate launch plus the
+ * count -> idx -> blocks chain of dependent reads costs more than a small GEMV itself).  Results
+ * are identical to the two calls: idx[0:*count] ascending, *count, and the same y bits.  idx (n
+ * entries) and count are written; the other arguments are those of spqt_sparse_gemv.  For
+ * n > 32768 the two kernels are launched one after the other instead.
+ */
+spqt_status spqt_sparsify_gemv(const void* codes, const void* scales, const void* zeros,
+                               int m, int n, int bits, int group,
+                               const void* x, float t, int32_t* idx, int32_t* count,
+                               void* y, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * The same kernel over all n columns with no index list: the dense GEMV on the
  * zigzag layout (paper Sec. 4.2.2), the sparsity-free comparison.
  */

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libspqt.so")
 
 EXPORTS = (
     "spqt_status_string", "spqt_version", "spqt_packed_sizes", "spqt_pack", "spqt_unpack",
-    "spqt_sparsify", "spqt_sparse_gemv", "spqt_sparse_gemv_static", "spqt_dense_gemv", "spqt_sparse_linear_host",
+    "spqt_sparsify", "spqt_sparse_gemv", "spqt_sparse_gemv_static", "spqt_sparsify_gemv", "spqt_dense_gemv", "spqt_sparse_linear_host",
     "spqt_set_tuning", "spqt_workspace_status", "spqt_launch_count",
 )
 
@@ -52,6 +52,8 @@ def lib() -> ctypes.CDLL:
         L.spqt_sparse_gemv.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
         L.spqt_sparse_gemv_static.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp]
         L.spqt_sparse_gemv_static.restype = i32
+        L.spqt_sparsify_gemv.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, vp, vp, vp, vp, sz, vp]
+        L.spqt_sparsify_gemv.restype = i32
         L.spqt_dense_gemv.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, sz, vp]
         L.spqt_sparse_linear_host.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, vp,
                                               vp, vp, vp, vp, vp, sz, vp]
@@ -191,6 +193,26 @@ def spqt_sparse_gemv_static(p: Packed, x: torch.Tensor, idx: torch.Tensor, count
         _dev(x, torch.float16, "x"), _dev(idx, torch.int32, "idx"), _dev(count, torch.int32, "count"),
         _dev(y, torch.float16, "y"), _stream(stream)), "spqt_sparse_gemv_static")
     return y
+
+
+def spqt_sparsify_gemv(p: Packed, x: torch.Tensor, t: float, workspace: torch.Tensor,
+                       idx: torch.Tensor = None, count: torch.Tensor = None, y: torch.Tensor = None, stream=None):
+    """Index collection and sparse GEMV in one launch -> (y, idx, count)."""
+    if idx is None:
+        idx = torch.empty(p.n, dtype=torch.int32, device=x.device)
+    if count is None:
+        count = torch.empty(1, dtype=torch.int32, device=x.device)
+    if y is None:
+        y = torch.empty(p.m, dtype=torch.float16, device=x.device)
+    if x.numel() != p.n or y.numel() != p.m or idx.numel() < p.n:
+        raise ValueError("x and idx must have n entries and y m entries")
+    _ok(lib().spqt_sparsify_gemv(
+        _dev(p.codes, torch.uint8, "codes"), _dev(p.scales, torch.float16, "scales"),
+        _dev(p.zeros, torch.float16, "zeros"), p.m, p.n, p.bits, p.group,
+        _dev(x, torch.float16, "x"), float(t), _dev(idx, torch.int32, "idx"), _dev(count, torch.int32, "count"),
+        _dev(y, torch.float16, "y"), _dev(workspace, torch.uint8, "workspace"), workspace.numel(),
+        _stream(stream)), "spqt_sparsify_gemv")
+    return y, idx, count
 
 
 def spqt_dense_gemv(p: Packed, x: torch.Tensor, workspace: torch.Tensor, y: torch.Tensor = None,

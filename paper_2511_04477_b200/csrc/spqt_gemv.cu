@@ -47,6 +47,7 @@ constexpr int kGemvThreads = (kWorkers + 1) * 32;
 constexpr int kChunk = 32;               // list entries per chunk (one per lane)
 constexpr int kDepth = 3;                // chunks in flight per warp
 constexpr unsigned long long kWaitNs = 1000000000ull;  // bound on every mbarrier wait: one second
+constexpr int kMaxFusedN = 32768;        // largest n whose index collection can run inside the GEMV
 
 static int g_tune_ctas = 0;  // 0 = one CTA per SM
 
@@ -262,16 +263,25 @@ struct GemvSmem {
     alignas(16) float red[2][kWorkers][G];               // per-warp partial sums of a finished segment
     float red_z[2][kWorkers];                            // and their offset terms
     uint64_t red_full[2], red_empty[2];
+    // fused index collection only: activity mask and exclusive count of every 32 entries of x
+    unsigned act_mask[kMaxFusedN / 32];
+    int act_before[kMaxFusedN / 32 + 1];
 };
 
-template <int G, bool DENSE, bool ODD_N>
+// FUSED: the index collection runs in the kernel's prologue.  Every CTA scans x (ballot/popc per 32
+// entries, block counts scanned in shared memory), writes the part of the ascending index list that
+// its own slices cover to idx_out (the slices of all CTAs cover the whole list; overlapping parts
+// receive identical values), CTA 0 writes the count, and the pipeline then reads idx_out like a list
+// collected by a separate launch.
+template <int G, bool DENSE, bool ODD_N, bool FUSED>
 __global__ void __launch_bounds__(kGemvThreads, 1)
 gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales,
                  const __half* __restrict__ zeros, int R, int n,
-                 const __half* __restrict__ x, const int32_t* __restrict__ idx,
-                 const int32_t* __restrict__ count_ptr, __half* __restrict__ y,
+                 const __half* __restrict__ x, const int32_t* idx_in,
+                 const int32_t* count_ptr, __half* __restrict__ y,
                  int* __restrict__ counters, int* __restrict__ status,
-                 float* __restrict__ partials, float* __restrict__ zpartials, int max_slots)
+                 float* __restrict__ partials, float* __restrict__ zpartials, int max_slots,
+                 float thr, int32_t* idx_out, int32_t* count_out)
 {
     constexpr int B = G / 2;
     constexpr int LPB = B / 16;       // lanes that share one block
@@ -294,9 +304,67 @@ gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ s
     }
     __syncthreads();
 
-    const int count = DENSE ? n : *count_ptr;
+    int count;
     Piece pc;
-    pc.init(R, P, c, count);
+    const int32_t* idx = idx_in;
+    if (FUSED) {
+        const int nb = (n + 31) / 32;
+        for (int b = warp; b < nb; b += kGemvThreads / 32) {
+            const int k = b * 32 + lane;
+            // exact widening; NaN compares false and is never active
+            const bool p = (k < n) && (fabsf(__half2float(x[k])) > thr);
+            const unsigned m = __ballot_sync(0xffffffffu, p);
+            if (lane == 0) {
+                sm.act_mask[b] = m;
+                sm.act_before[b + 1] = __popc(m);
+            }
+        }
+        __syncthreads();
+        if (warp == 0) {
+            // exclusive scan of the block counts: each lane owns a run of consecutive blocks
+            const int per = (nb + 31) / 32, b0 = lane * per, b1 = min(b0 + per, nb);
+            int sum = 0;
+            for (int b = b0; b < b1; ++b) sum += sm.act_before[b + 1];
+            int incl = sum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int up = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += up;
+            }
+            int run = incl - sum;
+            if (lane == 0) sm.act_before[0] = 0;
+            for (int b = b0; b < b1; ++b) {
+                run += sm.act_before[b + 1];
+                sm.act_before[b + 1] = run;
+            }
+        }
+        __syncthreads();
+        count = sm.act_before[nb];
+        pc.init(R, P, c, count);
+        if (c == 0 && tid == 0) *count_out = count;
+        // list positions this CTA will read: the union of its slices
+        int need_lo = count, need_hi = 0;
+        for (int r = pc.r_first; r <= pc.r_last; ++r) {
+            int p0, p1;
+            pc.slice(r, &p0, &p1);
+            need_lo = min(need_lo, p0);
+            need_hi = max(need_hi, p1);
+        }
+        for (int b = warp; b < nb; b += kGemvThreads / 32) {
+            const int before = sm.act_before[b];
+            if (sm.act_before[b + 1] <= need_lo || before >= need_hi) continue;
+            const unsigned m = sm.act_mask[b];
+            if ((m >> lane) & 1u) {
+                const int pos = before + __popc(m & ((1u << lane) - 1u));
+                if (pos >= need_lo && pos < need_hi) idx_out[pos] = b * 32 + lane;
+            }
+        }
+        __syncthreads();  // the CTA's own global writes are visible to its later copies
+        idx = idx_out;
+    } else {
+        count = DENSE ? n : *count_ptr;
+        pc.init(R, P, c, count);
+    }
     SPQT_TRACE_EVENT(tid == 0, 4000);
 
     if (warp == kWriterWarp) {
@@ -321,6 +389,12 @@ gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ s
             if (lane == 0) mbar_arrive(&sm.red_empty[b]);
             int first, nslots;
             pc.contributors(r, &first, &nslots);
+            if (nslots == 1) {
+                // this CTA holds the whole block-row: no partial, no counter, no fence
+#pragma unroll
+                for (int i = 0; i < RPL; ++i) y[(size_t)r * G + lane * RPL + i] = __float2half_rn(v[i] + zpart);
+                continue;
+            }
             const size_t pslot = (size_t)r * max_slots + (c - first);
 #pragma unroll
             for (int i = 0; i < RPL; ++i) __stcg(partials + pslot * G + lane * RPL + i, v[i]);
@@ -549,12 +623,19 @@ gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ s
 
 // ---------------------------------------------------------------- host side
 
-template <int G, bool DENSE, bool ODD_N>
+struct FusedArgs {
+    float t;
+    int32_t* idx_out;
+    int32_t* count_out;
+};
+
+template <int G, bool DENSE, bool ODD_N, bool FUSED>
 static spqt_status launch_int4(const Format& f, const void* codes, const void* scales,
                                const void* zeros, const void* x, const int32_t* idx,
-                               const int32_t* count, void* y, void* workspace, cudaStream_t s)
+                               const int32_t* count, void* y, void* workspace, cudaStream_t s,
+                               FusedArgs fa)
 {
-    auto kernel = gemv_int4_kernel<G, DENSE, ODD_N>;
+    auto kernel = gemv_int4_kernel<G, DENSE, ODD_N, FUSED>;
     static bool configured[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPQT_ERR_CUDA;
@@ -580,19 +661,22 @@ static spqt_status launch_int4(const Format& f, const void* codes, const void* s
     kernel<<<P, kGemvThreads, smem, s>>>(
         static_cast<const uint8_t*>(codes), static_cast<const __half*>(scales),
         static_cast<const __half*>(zeros), f.R, f.n, static_cast<const __half*>(x), idx, count,
-        static_cast<__half*>(y), counters, status, partials, zpartials, slots);
+        static_cast<__half*>(y), counters, status, partials, zpartials, slots,
+        fa.t, fa.idx_out, fa.count_out);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? SPQT_OK : SPQT_ERR_CUDA;
 }
 
-template <bool DENSE>
+template <bool DENSE, bool FUSED = false>
 static spqt_status gemv_entry(const void* codes, const void* scales, const void* zeros,
                               int m, int n, int bits, int group, const void* x,
                               const int32_t* idx, const int32_t* count, void* y,
-                              void* workspace, size_t ws_bytes, void* stream)
+                              void* workspace, size_t ws_bytes, void* stream,
+                              FusedArgs fa = FusedArgs{0.0f, nullptr, nullptr})
 {
     if (!codes || !scales || !zeros || !x || !y || !workspace) return SPQT_ERR_INVALID_ARG;
     if (!DENSE && (!idx || !count)) return SPQT_ERR_INVALID_ARG;
+    if (FUSED && n > kMaxFusedN) return SPQT_ERR_UNSUPPORTED;
     Format f;
     spqt_status st = make_format(m, n, bits, group, &f);
     if (st != SPQT_OK) return st;
@@ -603,11 +687,11 @@ static spqt_status gemv_entry(const void* codes, const void* scales, const void*
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool odd = (n & 1) != 0;
     if (bits == 4 && group == 128)
-        return odd ? launch_int4<128, DENSE, true>(f, codes, scales, zeros, x, idx, count, y, workspace, s)
-                   : launch_int4<128, DENSE, false>(f, codes, scales, zeros, x, idx, count, y, workspace, s);
+        return odd ? launch_int4<128, DENSE, true, FUSED>(f, codes, scales, zeros, x, idx, count, y, workspace, s, fa)
+                   : launch_int4<128, DENSE, false, FUSED>(f, codes, scales, zeros, x, idx, count, y, workspace, s, fa);
     if (bits == 4 && group == 64)
-        return odd ? launch_int4<64, DENSE, true>(f, codes, scales, zeros, x, idx, count, y, workspace, s)
-                   : launch_int4<64, DENSE, false>(f, codes, scales, zeros, x, idx, count, y, workspace, s);
+        return odd ? launch_int4<64, DENSE, true, FUSED>(f, codes, scales, zeros, x, idx, count, y, workspace, s, fa)
+                   : launch_int4<64, DENSE, false, FUSED>(f, codes, scales, zeros, x, idx, count, y, workspace, s, fa);
     return SPQT_ERR_UNSUPPORTED;
 }
 
@@ -631,6 +715,23 @@ spqt_status spqt_sparse_gemv(const void* codes, const void* scales, const void* 
 {
     return spqt::gemv_entry<false>(codes, scales, zeros, m, n, bits, group, x, idx, count, y,
                                    workspace, workspace_bytes, stream);
+}
+
+spqt_status spqt_sparsify_gemv(const void* codes, const void* scales, const void* zeros,
+                               int m, int n, int bits, int group,
+                               const void* x, float t, int32_t* idx, int32_t* count,
+                               void* y, void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (n > spqt::kMaxFusedN) {
+        // too long for the in-kernel scan: the same result from the two separate launches
+        spqt_status st = spqt_sparsify(x, n, t, idx, count, stream);
+        if (st != SPQT_OK) return st;
+        return spqt_sparse_gemv(codes, scales, zeros, m, n, bits, group, x, idx, count, y, workspace,
+                                workspace_bytes, stream);
+    }
+    return spqt::gemv_entry<false, true>(codes, scales, zeros, m, n, bits, group, x, idx, count, y,
+                                         workspace, workspace_bytes, stream,
+                                         spqt::FusedArgs{t, idx, count});
 }
 
 spqt_status spqt_dense_gemv(const void* codes, const void* scales, const void* zeros,

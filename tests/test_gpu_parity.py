@@ -220,6 +220,38 @@ def test_heavy_tailed_outliers():
     check_y(y, y_ref, bound, "outliers")
 
 
+# ------------------------------------------------------------------ a2 + a3-a5 in one launch
+
+@pytest.mark.parametrize("bits,group", GEMV_FORMATS)
+@pytest.mark.parametrize("m_blocks,n", [(2, 300), (8, 4096), (3, 1111), (32, 4096), (1, 1), (2, 33000)])
+def test_fused_index_collection_and_gemv_equals_the_two_calls(bits, group, m_blocks, n):
+    m = m_blocks * group
+    W = inputs.weights(m, n, seed=m + n + 7)
+    x = inputs.activations(n, seed=9 + n)
+    if n > 100:
+        x[3] = np.float16(np.nan)
+        x[4] = np.float16(-np.inf)
+    p = pack_on_gpu(W, bits, group)
+    codes, s, z = packed_to_host(p)
+    ws = binding.new_workspace(m, n, bits, group)
+    xd = dev(x)
+    for sp in (0.0, 0.5, 0.97, None):
+        t = float("inf") if sp is None else inputs.threshold_for_sparsity(x, sp)
+        idx = torch.full((n,), -7, dtype=torch.int32, device="cuda")
+        cnt = torch.full((1,), -7, dtype=torch.int32, device="cuda")
+        y, _, _ = binding.spqt_sparsify_gemv(p, xd, t, ws, idx, cnt)
+        torch.cuda.synchronize()
+        ref_idx, ref_cnt = oracle.sparsify(x, t)
+        assert int(cnt.item()) == ref_cnt
+        got = idx.cpu().numpy()
+        assert np.array_equal(got[:ref_cnt], ref_idx) and np.all(got[ref_cnt:] == -7)
+        y_ref, bound = oracle.sparse_gemv(codes, s, z, m, n, x, ref_idx, bits, group)
+        check_y(y.cpu().numpy(), y_ref, bound, "fused, sparsity %r" % sp)
+        y2, _, _ = run_sparse(p, x, t, ws)
+        assert np.array_equal(y.cpu().numpy().view(np.uint16), y2.view(np.uint16))
+    assert binding.spqt_workspace_status(ws, m, group) == 0
+
+
 # ------------------------------------------------------------------ a6: dense GEMV
 
 @pytest.mark.parametrize("bits,group", GEMV_FORMATS)
