@@ -25,11 +25,11 @@
 //      fp32) and x_k*zero_rk, the multipliers are dealt out with shuffles, and
 //      the warp does the dequantize-FMA work.
 // A runs 2*kDepth chunks ahead of C and B kDepth chunks ahead, so kDepth chunks
-// (2 KB each) per warp are in flight.  One more warp, the writer, adds the
-// workers' sums at the end of a segment, publishes the partial and, if this CTA
-// is the last contributor of the block-row, produces y; its waits on shared-
-// memory barriers are bounded in wall time (on expiry the workspace's status
-// word is set and the kernel returns).
+// (2 KB each) per warp are in flight.  Two more warps, the writers (one per
+// hand-over buffer), add the workers' sums at the end of a segment, publish the
+// partial and, if this CTA is the last contributor of the block-row, produce y;
+// their waits on shared-memory barriers are bounded in wall time (on expiry the
+// workspace's status word is set and the kernel returns).
 //
 // Arithmetic:  y[j] = sum_k a_k * code_jk + sum_k x_k * zero_rk.  A 4-bit code
 // becomes an fp32 operand with no conversion: the nibble masked in place at bit
@@ -41,9 +41,9 @@
 
 namespace spqt {
 
-constexpr int kWorkers = 19;             // compute warps
-constexpr int kWriterWarp = kWorkers;
-constexpr int kGemvThreads = (kWorkers + 1) * 32;
+constexpr int kWorkers = 18;             // compute warps
+constexpr int kWriterWarp = kWorkers;      // first of two writer warps: segment sg goes to writer sg & 1
+constexpr int kGemvThreads = (kWorkers + 2) * 32;
 constexpr int kChunk = 32;               // list entries per chunk (one per lane)
 constexpr int kDepth = 3;                // chunks in flight per warp
 constexpr unsigned long long kWaitNs = 1000000000ull;  // bound on every mbarrier wait: one second
@@ -295,6 +295,10 @@ gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ s
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int P = gridDim.x, c = blockIdx.x;
+    SPQT_TRACE_EVENT(tid == 0, 3990);
+#ifdef SPQT_TRACE
+    if (tid == 0 && g_trace && c < 200) g_trace[2000 + c] = (long long)global_ns();
+#endif
 
     if (tid == 0) {
         for (int b = 0; b < 2; ++b) {
@@ -367,12 +371,14 @@ gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ s
     }
     SPQT_TRACE_EVENT(tid == 0, 4000);
 
-    if (warp == kWriterWarp) {
-        // ------------------------------------------------------------ writer
+    if (warp >= kWriterWarp) {
+        // ------------------------------------------------------------ writers
+        // Two warps, one per hand-over buffer, so that the chains of dependent L2 round trips
+        // (store, fence, counter, read back) of consecutive segments overlap.
         constexpr int RPL = G / 32;  // rows per lane
+        const int b = warp - kWriterWarp;
         bool ok = true;
-        for (int r = pc.r_first, sg = 0; r <= pc.r_last; ++r, ++sg) {
-            const int b = sg & 1;
+        for (int r = pc.r_first + b, sg = b; r <= pc.r_last; r += 2, sg += 2) {
             ok = mbar_wait(&sm.red_full[b], (sg >> 1) & 1);
             if (!ok) break;
             float v[RPL];
@@ -412,16 +418,32 @@ gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ s
                 for (int i = 0; i < RPL; ++i) v[i] = 0.0f;
                 const float* p = partials + (size_t)r * max_slots * G + lane * RPL;
                 const float* zp = zpartials + (size_t)r * max_slots;
-                for (int s2 = 0; s2 < nslots; ++s2) {
+                // eight slots' loads in flight at a time; the additions keep the slot order
+                for (int s0 = 0; s0 < nslots; s0 += 8) {
+                    float pv[8][RPL], pz[8];
 #pragma unroll
-                    for (int i = 0; i < RPL; ++i) v[i] += __ldcg(p + (size_t)s2 * G + i);
-                    zsum += __ldcg(zp + s2);
+                    for (int j = 0; j < 8; ++j) {
+                        const bool in = s0 + j < nslots;
+#pragma unroll
+                        for (int i = 0; i < RPL; ++i) pv[j][i] = in ? __ldcg(p + (size_t)(s0 + j) * G + i) : 0.0f;
+                        pz[j] = in ? __ldcg(zp + s0 + j) : 0.0f;
+                    }
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+#pragma unroll
+                        for (int i = 0; i < RPL; ++i) v[i] += pv[j][i];
+                        zsum += pz[j];
+                    }
                 }
 #pragma unroll
                 for (int i = 0; i < RPL; ++i) y[(size_t)r * G + lane * RPL + i] = __float2half_rn(v[i] + zsum);
                 if (lane == 0) counters[r] = 0;  // leave the workspace ready for the next call
             }
         }
+        SPQT_TRACE_EVENT(lane == 0, 4002);
+#ifdef SPQT_TRACE
+        if (lane == 0 && g_trace && c < 200) g_trace[2200 + c] = (long long)global_ns();
+#endif
         if (!ok && lane == 0) atomicExch(status, 1);
         return;
     }
@@ -608,6 +630,7 @@ gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ s
         for (int o = 16; o > 0; o >>= 1) zl += __shfl_xor_sync(0xffffffffu, zl, o);
         if (lane == 0) sm.red_z[b][warp] = zl;
         __syncwarp();
+        SPQT_TRACE_EVENT(tid == 0, 3950 + sg);
         if (lane == 0) mbar_arrive(&sm.red_full[b]);
     }
     cp_async_wait<0>();
@@ -648,6 +671,9 @@ static spqt_status launch_int4(const Format& f, const void* codes, const void* s
     const int sms = sm_count();
     if (sms <= 0) return SPQT_ERR_CUDA;
     int P = g_tune_ctas > 0 ? g_tune_ctas : sms;
+    // With few block-rows, a whole number of CTAs per block-row (if that keeps >= 85 % of the SMs
+    // busy) gives every CTA a single segment: no CTA then carries two aggregation chains.
+    if (g_tune_ctas == 0 && f.R <= P && (P / f.R) * f.R * 100 >= 85 * P) P = (P / f.R) * f.R;
     // no more CTAs than pieces of at least 64 columns of one block-row
     const long long pieces = (long long)f.R * ((f.n + 63) / 64);
     if (P > pieces) P = (int)pieces;
