@@ -48,6 +48,7 @@ constexpr int kChunk = 32;               // list entries per chunk (one per lane
 constexpr int kDepth = 3;                // chunks in flight per warp
 constexpr unsigned long long kWaitNs = 1000000000ull;  // bound on every mbarrier wait: one second
 constexpr int kMaxFusedN = 32768;        // largest n whose index collection can run inside the GEMV
+constexpr int kFusedCols = 8192;         // list entries a CTA keeps in shared memory in that case
 
 static int g_tune_ctas = 0;  // 0 = one CTA per SM
 
@@ -192,29 +193,34 @@ __device__ __forceinline__ void halve(const float* in, float* out, int lane, int
 // active list that belongs to this CTA.  Uniform across the CTA.
 struct Piece {
     int R, P, c, count, r_first, r_last;
+    unsigned qc, rc;  // count = qc * P + rc: keeps the slice arithmetic in 32 bits (the host checks R * P < 2^31)
 
     __device__ __forceinline__ void init(int R_, int P_, int c_, int count_)
     {
         R = R_; P = P_; c = c_; count = count_;
-        const long long lo = (long long)c * R, hi = lo + R;
-        r_first = (int)(lo / P);
-        r_last = (int)((hi - 1) / P);
+        const unsigned lo = (unsigned)c * (unsigned)R, hi = lo + (unsigned)R;
+        r_first = (int)(lo / (unsigned)P);
+        r_last = (int)((hi - 1u) / (unsigned)P);
+        qc = (unsigned)count / (unsigned)P;
+        rc = (unsigned)count - qc * (unsigned)P;
     }
+    // floor(u * count / P) for 0 <= u <= P
+    __device__ __forceinline__ int scaled(unsigned u) const { return (int)(u * qc + (u * rc) / (unsigned)P); }
     __device__ __forceinline__ void slice(int row, int* a, int* b) const
     {
-        const long long lo = (long long)c * R, hi = lo + R, base = (long long)row * P;
-        const long long u0 = (lo > base ? lo : base) - base;
-        const long long u1 = (hi < base + P ? hi : base + P) - base;
-        *a = (int)((u0 * count) / P);
-        *b = (int)((u1 * count) / P);
+        const unsigned lo = (unsigned)c * (unsigned)R, hi = lo + (unsigned)R, base = (unsigned)row * (unsigned)P;
+        const unsigned u0 = (lo > base ? lo : base) - base;
+        const unsigned u1 = (hi < base + (unsigned)P ? hi : base + (unsigned)P) - base;
+        *a = scaled(u0);
+        *b = scaled(u1);
     }
     // contributors to block-row `row`: CTAs first .. first+n-1
     __device__ __forceinline__ void contributors(int row, int* first, int* n) const
     {
-        const int f = (int)(((long long)row * P) / R);
-        const int l = (int)((((long long)row + 1) * P - 1) / R);
-        *first = f;
-        *n = l - f + 1;
+        const unsigned f = ((unsigned)row * (unsigned)P) / (unsigned)R;
+        const unsigned l = (((unsigned)row + 1u) * (unsigned)P - 1u) / (unsigned)R;
+        *first = (int)f;
+        *n = (int)(l - f + 1u);
     }
 };
 
@@ -266,6 +272,7 @@ struct GemvSmem {
     // fused index collection only: activity mask and exclusive count of every 32 entries of x
     unsigned act_mask[kMaxFusedN / 32];
     int act_before[kMaxFusedN / 32 + 1];
+    int fused_cols[kFusedCols];  // the part of the index list this CTA reads, when it fits
 };
 
 // FUSED: the index collection runs in the kernel's prologue.  Every CTA scans x (ballot/popc per 32
@@ -311,19 +318,64 @@ gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ s
     int count;
     Piece pc;
     const int32_t* idx = idx_in;
+    int need_lo = 0;          // FUSED: first list position held in sm.fused_cols
+    bool cols_local = false;  // FUSED: the pipeline reads its column numbers from sm.fused_cols
     if (FUSED) {
         const int nb = (n + 31) / 32;
-        for (int b = warp; b < nb; b += kGemvThreads / 32) {
-            const int k = b * 32 + lane;
-            // exact widening; NaN compares false and is never active
-            const bool p = (k < n) && (fabsf(__half2float(x[k])) > thr);
-            const unsigned m = __ballot_sync(0xffffffffu, p);
-            if (lane == 0) {
-                sm.act_mask[b] = m;
-                sm.act_before[b + 1] = __popc(m);
+        // All loads first (one memory round trip), then the ballots.  A warp load covers 256 entries:
+        // lane l holds entries 8l..8l+7, so every four lanes make one 32-entry block.
+        constexpr int kWarps = kGemvThreads / 32;
+        constexpr int kMaxLoads = (kMaxFusedN / 256 + kWarps - 1) / kWarps;
+        const int nv = (n + 255) / 256;
+        const bool vec_ok = (reinterpret_cast<uintptr_t>(x) & 15) == 0;
+        uint4 xv[kMaxLoads];
+#pragma unroll
+        for (int j = 0; j < kMaxLoads; ++j) {
+            const int li = warp + j * kWarps;
+            const int k0 = li * 256 + lane * 8;
+            xv[j] = make_uint4(0u, 0u, 0u, 0u);
+            if (li < nv) {
+                if (vec_ok && k0 + 8 <= n) {
+                    xv[j] = __ldg(reinterpret_cast<const uint4*>(x + k0));
+                } else {
+                    unsigned short hv[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        hv[e] = (k0 + e < n) ? __ldg(reinterpret_cast<const unsigned short*>(x) + k0 + e) : (unsigned short)0;
+                    xv[j].x = hv[0] | ((unsigned)hv[1] << 16);
+                    xv[j].y = hv[2] | ((unsigned)hv[3] << 16);
+                    xv[j].z = hv[4] | ((unsigned)hv[5] << 16);
+                    xv[j].w = hv[6] | ((unsigned)hv[7] << 16);
+                }
             }
         }
+#pragma unroll
+        for (int j = 0; j < kMaxLoads; ++j) {
+            const int li = warp + j * kWarps;
+            if (li < nv) {  // uniform across the warp
+                const int k0 = li * 256 + lane * 8;
+                const unsigned wds[4] = {xv[j].x, xv[j].y, xv[j].z, xv[j].w};
+                unsigned m8 = 0;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const unsigned short hb = (unsigned short)(wds[e >> 1] >> ((e & 1) * 16));
+                    // exact widening; NaN compares false and is never active
+                    const bool p = (k0 + e < n) && (fabsf(__half2float(__ushort_as_half(hb))) > thr);
+                    m8 |= (p ? 1u : 0u) << e;
+                }
+                unsigned m = m8 << ((lane & 3) * 8);
+                m |= __shfl_xor_sync(0xffffffffu, m, 1);
+                m |= __shfl_xor_sync(0xffffffffu, m, 2);
+                const int b = li * 8 + (lane >> 2);
+                if ((lane & 3) == 0 && b < nb) {
+                    sm.act_mask[b] = m;
+                    sm.act_before[b + 1] = __popc(m);
+                }
+            }
+        }
+        SPQT_TRACE_EVENT(tid == 0, 3991);
         __syncthreads();
+        SPQT_TRACE_EVENT(tid == 0, 3992);
         if (warp == 0) {
             // exclusive scan of the block counts: each lane owns a run of consecutive blocks
             const int per = (nb + 31) / 32, b0 = lane * per, b1 = min(b0 + per, nb);
@@ -343,27 +395,38 @@ gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ s
             }
         }
         __syncthreads();
+        SPQT_TRACE_EVENT(tid == 0, 3993);
         count = sm.act_before[nb];
         pc.init(R, P, c, count);
         if (c == 0 && tid == 0) *count_out = count;
-        // list positions this CTA will read: the union of its slices
-        int need_lo = count, need_hi = 0;
+        // list positions this CTA will read: the union of its slices.  If that part fits in shared
+        // memory the pipeline takes its column numbers from there (no round trip through global
+        // memory); idx_out is then written once, an even share of the list per CTA.
+        need_lo = count;
+        int need_hi = 0;
         for (int r = pc.r_first; r <= pc.r_last; ++r) {
             int p0, p1;
             pc.slice(r, &p0, &p1);
             need_lo = min(need_lo, p0);
             need_hi = max(need_hi, p1);
         }
+        cols_local = (need_hi - need_lo) <= kFusedCols;
+        SPQT_TRACE_EVENT(tid == 0, 3994);
+        const int out_lo = pc.scaled((unsigned)c), out_hi = pc.scaled((unsigned)c + 1u);
         for (int b = warp; b < nb; b += kGemvThreads / 32) {
-            const int before = sm.act_before[b];
-            if (sm.act_before[b + 1] <= need_lo || before >= need_hi) continue;
+            const int before = sm.act_before[b], after = sm.act_before[b + 1];
+            const bool mine = after > need_lo && before < need_hi, share = after > out_lo && before < out_hi;
+            if (!mine && !share) continue;
             const unsigned m = sm.act_mask[b];
             if ((m >> lane) & 1u) {
                 const int pos = before + __popc(m & ((1u << lane) - 1u));
-                if (pos >= need_lo && pos < need_hi) idx_out[pos] = b * 32 + lane;
+                const int col = b * 32 + lane;
+                const bool need = pos >= need_lo && pos < need_hi;
+                if (need && cols_local) sm.fused_cols[pos - need_lo] = col;
+                if ((need && !cols_local) || (pos >= out_lo && pos < out_hi)) idx_out[pos] = col;
             }
         }
-        __syncthreads();  // the CTA's own global writes are visible to its later copies
+        __syncthreads();  // the CTA's own writes (shared or global) are visible to its pipeline
         idx = idx_out;
     } else {
         count = DENSE ? n : *count_ptr;
@@ -469,7 +532,7 @@ gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ s
 
     // stage A: column numbers of the warp's chunk number qa
     auto issue_a = [&]() {
-        if (!DENSE && ca.valid(pc)) {
+        if (!DENSE && !(FUSED && cols_local) && ca.valid(pc)) {
             if (ca.pos + lane < ca.p1) cp_async_4(smem_u32(&my_cols[qa % (2 * D)][lane]), idx + ca.pos + lane);
             ca.advance(pc, warp);
             ++qa;
@@ -487,7 +550,7 @@ gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ s
                 b_zeros = reinterpret_cast<const unsigned short*>(zeros) + row_base;
             }
             const int valid = cb.p1 - cb.pos;  // entries of this chunk (>= kChunk when full)
-            const int* cols = my_cols[qb % (2 * D)];
+            const int* cols = (FUSED && cols_local) ? &sm.fused_cols[cb.pos - need_lo] : my_cols[qb % (2 * D)];
             typename GemvSmem<G>::Stage& st = my_stage[qb % D];
             const unsigned dst = smem_u32(&st.codes[0]) + lane * 16;
 #pragma unroll
@@ -561,7 +624,10 @@ gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ s
 #endif
             const typename GemvSmem<G>::Stage& st = my_stage[qc % D];
             const unsigned xw = st.meta[0][lane], sw = st.meta[1][lane], zw = st.meta[2][lane];
-            const unsigned kk = DENSE ? (unsigned)(pos + lane) : (unsigned)my_cols[qc % (2 * D)][lane];
+            unsigned kk;
+            if (DENSE) kk = (unsigned)(pos + lane);
+            else if (FUSED && cols_local) kk = (pos + lane < p1) ? (unsigned)sm.fused_cols[pos - need_lo + lane] : 0u;
+            else kk = (unsigned)my_cols[qc % (2 * D)][lane];
 #ifdef SPQT_TRACE
             const long long tc2 = clock64();
 #endif
@@ -710,6 +776,7 @@ static spqt_status gemv_entry(const void* codes, const void* scales, const void*
         !aligned(y, 2) || !aligned(workspace, 16) || (!DENSE && (!aligned(idx, 4) || !aligned(count, 4))))
         return SPQT_ERR_ALIGNMENT;
     if (ws_bytes < workspace_bytes(f)) return SPQT_ERR_WORKSPACE;
+    if ((long long)f.R * kMaxCtas >= (1ll << 31)) return SPQT_ERR_UNSUPPORTED;  // the work map is 32-bit
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool odd = (n & 1) != 0;
     if (bits == 4 && group == 128)
