@@ -399,7 +399,7 @@ def run_ours(args):
             "per_shape": per_shape,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": traffic, "peak_kind": "of " + peak_kind,
-                         "kernel": "gemv_int4_kernel<128,sparse>", "algorithmic_bytes_per_launch": avg_launch_bytes,
+                         "kernel": "gemv_kernel<128,sparse>", "algorithmic_bytes_per_launch": avg_launch_bytes,
                          "avg_launch_us": ms_gemv * 1e3 / n_gemv},
             "cpu_baseline": {"value": cpu["value"], "unit": "GB/s", "cores": cpu["cores"], "kind": "oracle",
                              "sample": cpu["sample"]},

@@ -112,8 +112,7 @@ spqt_status spqt_sparsify(const void* x, int n, float t,
  *   workspace : gemv_workspace_bytes of device memory, 16-byte aligned, zeroed
  *       ONCE by the caller before its first use; every call leaves it ready for
  *       the next.  Two calls that may overlap on the GPU need two workspaces.
- * Supported: bits 4 with group 64 or 128 (bits 3: SPQT_ERR_UNSUPPORTED for now).
- * n * B must fit in 32 bits.
+ * Supported: bits 4 or 3 with group 64 or 128.
  */
 spqt_status spqt_sparse_gemv(const void* codes, const void* scales, const void* zeros,
                              int m, int n, int bits, int group,

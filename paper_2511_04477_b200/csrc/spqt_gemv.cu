@@ -1,4 +1,4 @@
-// Activation-sparse GEMV over the zigzag layout, and its dense twin (4-bit codes).
+// Activation-sparse GEMV over the zigzag layout, and its dense twin (4-bit and 3-bit codes).
 //
 // Work decomposition (the paper's hybrid row/column parallelism, generalised):
 // the R block-rows are laid end to end and cut into P equal pieces, one per CTA,
@@ -117,6 +117,10 @@ __device__ __forceinline__ void cp_async_16_l2_64(unsigned smem_dst, const void*
 {
     asm volatile("cp.async.cg.shared.global.L2::64B [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
 }
+__device__ __forceinline__ void cp_async_8(unsigned smem_dst, const void* gmem_src)
+{
+    asm volatile("cp.async.ca.shared.global.L2::64B [%0], [%1], 8;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
+}
 __device__ __forceinline__ void cp_async_4(unsigned smem_dst, const void* gmem_src)
 {
     asm volatile("cp.async.ca.shared.global.L2::64B [%0], [%1], 4;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
@@ -170,6 +174,19 @@ __device__ __forceinline__ void fma_block16(unsigned long long* acc, const uint4
     fma_word(acc + 4, w.y, m01, m23, m40, m12);
     fma_word(acc + 8, w.z, m01, m23, m40, m12);
     fma_word(acc + 12, w.w, m01, m23, m40, m12);
+}
+
+// 3-bit codes: w2a, w2b are words of the 2-bit plane (byte i, field v = bits 2v..2v+1), w1 the word
+// of the 1-bit plane whose byte i, bit u carries the top bit of the code in w2a (u = 2v) or w2b
+// (u = 2v+1).  The fields are first widened to four words of eight 4-bit codes, then treated like
+// 4-bit codes: word 0/1 = w2a fields v = {0,2} / {1,3}, word 2/3 = the same of w2b (low nibble first).
+__device__ __forceinline__ void fma_block3(unsigned long long* acc, unsigned w2a, unsigned w2b, unsigned w1, float a)
+{
+    const unsigned c0 = (w2a & 0x33333333u) | ((w1 << 2) & 0x44444444u);
+    const unsigned c1 = ((w2a >> 2) & 0x33333333u) | (w1 & 0x44444444u);
+    const unsigned c2 = (w2b & 0x33333333u) | ((w1 << 1) & 0x44444444u);
+    const unsigned c3 = ((w2b >> 2) & 0x33333333u) | ((w1 >> 1) & 0x44444444u);
+    fma_block16(acc, make_uint4(c0, c1, c2, c3), a);
 }
 
 // One step of a butterfly reduce-scatter: lanes that differ in bit `bit` hold
@@ -257,9 +274,9 @@ struct Cursor {
 
 // ---------------------------------------------------------------- kernel
 
-template <int G>
+template <int G, int BITS>
 struct GemvSmem {
-    static constexpr int B = G / 2;
+    static constexpr int B = G * BITS / 8;
     struct Stage {
         alignas(16) unsigned char codes[kChunk * B];  // block e of the chunk at e*B
         unsigned meta[3][kChunk];                     // words holding x_k, scale_rk, zero_rk of entry e
@@ -280,9 +297,9 @@ struct GemvSmem {
 // its own slices cover to idx_out (the slices of all CTAs cover the whole list; overlapping parts
 // receive identical values), CTA 0 writes the count, and the pipeline then reads idx_out like a list
 // collected by a separate launch.
-template <int G, bool DENSE, bool ODD_N, bool FUSED>
+template <int G, int BITS, bool DENSE, bool ODD_N, bool FUSED>
 __global__ void __launch_bounds__(kGemvThreads, 1)
-gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales,
+gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales,
                  const __half* __restrict__ zeros, int R, int n,
                  const __half* __restrict__ x, const int32_t* idx_in,
                  const int32_t* count_ptr, __half* __restrict__ y,
@@ -290,15 +307,17 @@ gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ s
                  float* __restrict__ partials, float* __restrict__ zpartials, int max_slots,
                  float thr, int32_t* idx_out, int32_t* count_out)
 {
-    constexpr int B = G / 2;
-    constexpr int LPB = B / 16;       // lanes that share one block
+    constexpr int B = G * BITS / 8;
+    constexpr int LPB = G / 32;       // lanes that share one block (each owns 32 of its rows)
+    constexpr int CB = (B % 16 == 0) ? 16 : 8;   // bytes per copy: 3-bit blocks of 64 rows are only 8-byte aligned
+    static_assert(BITS == 3 || BITS == 4, "3- or 4-bit codes");
     constexpr int SLOTS = 32 / LPB;   // blocks per 512-byte warp load
     constexpr int KEEP = 32 / SLOTS;  // values per lane after the in-warp reduce-scatter
     constexpr int SUBS = kChunk / SLOTS;  // 512-byte loads per chunk
     constexpr int D = kDepth;
 
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    GemvSmem<G>& sm = *reinterpret_cast<GemvSmem<G>*>(smem_raw);
+    GemvSmem<G, BITS>& sm = *reinterpret_cast<GemvSmem<G, BITS>*>(smem_raw);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int P = gridDim.x, c = blockIdx.x;
@@ -515,7 +534,7 @@ gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ s
     const int slot = lane / LPB, h = lane % LPB;
     const unsigned short* xb = reinterpret_cast<const unsigned short*>(x);
 
-    typename GemvSmem<G>::Stage* my_stage = &sm.stage[warp][0];
+    typename GemvSmem<G, BITS>::Stage* my_stage = &sm.stage[warp][0];
     int (*my_cols)[kChunk] = sm.cols[warp];
 
     Cursor ca, cb;  // stage A / stage B cursors (the consume side walks the segments itself)
@@ -545,21 +564,42 @@ gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ s
                 b_row = cb.r;
                 const size_t row_base = (size_t)b_row * (size_t)n;
                 b_par = (unsigned)(row_base & 1);
-                b_codes = codes + row_base * B + 16 * h;
+                b_codes = codes + row_base * B + (BITS == 4 ? 16 * h : 0);
                 b_scales = reinterpret_cast<const unsigned short*>(scales) + row_base;
                 b_zeros = reinterpret_cast<const unsigned short*>(zeros) + row_base;
             }
             const int valid = cb.p1 - cb.pos;  // entries of this chunk (>= kChunk when full)
             const int* cols = (FUSED && cols_local) ? &sm.fused_cols[cb.pos - need_lo] : my_cols[qb % (2 * D)];
-            typename GemvSmem<G>::Stage& st = my_stage[qb % D];
+            typename GemvSmem<G, BITS>::Stage& st = my_stage[qb % D];
             const unsigned dst = smem_u32(&st.codes[0]) + lane * 16;
+            if (BITS == 4) {
 #pragma unroll
-            for (int u = 0; u < SUBS; ++u) {
-                const int e = u * SLOTS + slot;
-                if (e < valid) {
-                    const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : (unsigned)cols[e];
-                    if (DENSE) cp_async_16(dst + u * 512, b_codes + (size_t)kk * B);
-                    else cp_async_16_l2_64(dst + u * 512, b_codes + (size_t)kk * B);
+                for (int u = 0; u < SUBS; ++u) {
+                    const int e = u * SLOTS + slot;
+                    if (e < valid) {
+                        const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : (unsigned)cols[e];
+                        if (DENSE) cp_async_16(dst + u * 512, b_codes + (size_t)kk * B);
+                        else cp_async_16_l2_64(dst + u * 512, b_codes + (size_t)kk * B);
+                    }
+                }
+            } else {
+                // 3-bit blocks (48 or 24 bytes): the chunk's bytes in copies of CB bytes, lane after lane
+                constexpr int NC = kChunk * B / CB / 32;
+#pragma unroll
+                for (int q = 0; q < NC; ++q) {
+                    const int off = (q * 32 + lane) * CB;    // byte offset inside the chunk's stage
+                    const int e = off / B, part = off % B;
+                    if (e < valid) {
+                        const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : (unsigned)cols[e];
+                        const uint8_t* src = b_codes + (size_t)kk * B + part;
+                        const unsigned d = smem_u32(&st.codes[0]) + off;
+                        if (CB == 16) {
+                            if (DENSE) cp_async_16(d, src);
+                            else cp_async_16_l2_64(d, src);
+                        } else {
+                            cp_async_8(d, src);
+                        }
+                    }
                 }
             }
             if (lane < valid) {
@@ -622,7 +662,7 @@ gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ s
 #ifdef SPQT_TRACE
             const long long tc1 = clock64();
 #endif
-            const typename GemvSmem<G>::Stage& st = my_stage[qc % D];
+            const typename GemvSmem<G, BITS>::Stage& st = my_stage[qc % D];
             const unsigned xw = st.meta[0][lane], sw = st.meta[1][lane], zw = st.meta[2][lane];
             unsigned kk;
             if (DENSE) kk = (unsigned)(pos + lane);
@@ -642,9 +682,15 @@ gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ s
             }
 #pragma unroll
             for (int u = 0; u < SUBS; ++u) {
-                const uint4 wv = *reinterpret_cast<const uint4*>(&st.codes[0] + lane * 16 + u * 512);
                 const float au = __shfl_sync(0xffffffffu, a, u * SLOTS + slot);
-                fma_block16(acc, wv, au);
+                if (BITS == 4) {
+                    const uint4 wv = *reinterpret_cast<const uint4*>(&st.codes[0] + lane * 16 + u * 512);
+                    fma_block16(acc, wv, au);
+                } else {
+                    // lane h of a block: words h and h+LPB of the 2-bit plane, word h of the 1-bit plane
+                    const unsigned* blk = reinterpret_cast<const unsigned*>(&st.codes[0] + (u * SLOTS + slot) * B);
+                    fma_block3(acc, blk[h], blk[h + LPB], blk[2 * LPB + h], au);
+                }
             }
             __syncwarp();  // every lane has read its part of the slots that B and A now refill
             issue_b();
@@ -689,7 +735,9 @@ gemv_int4_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ s
         for (int i = 0; i < KEEP; ++i) {
             const int ai = a_base + i;  // accumulator index = word*8 + nibble
             const int cw = ai >> 3, e2 = ai & 7;
-            const int row = 16 * h + 4 * cw + (e2 >> 1) + (e2 & 1) * (G / 2);
+            const int row = (BITS == 4)
+                                ? 16 * h + 4 * cw + (e2 >> 1) + (e2 & 1) * (G / 2)
+                                : 4 * h + (e2 >> 1) + (G / 8) * (cw >> 1) + (G / 4) * ((cw & 1) + 2 * (e2 & 1));
             sm.red[b][warp][row] = keep[i] * 0x1p56f;  // undo the 2^-56 of the subnormal trick
         }
 #pragma unroll
@@ -718,17 +766,17 @@ struct FusedArgs {
     int32_t* count_out;
 };
 
-template <int G, bool DENSE, bool ODD_N, bool FUSED>
-static spqt_status launch_int4(const Format& f, const void* codes, const void* scales,
+template <int G, int BITS, bool DENSE, bool ODD_N, bool FUSED>
+static spqt_status launch_gemv(const Format& f, const void* codes, const void* scales,
                                const void* zeros, const void* x, const int32_t* idx,
                                const int32_t* count, void* y, void* workspace, cudaStream_t s,
                                FusedArgs fa)
 {
-    auto kernel = gemv_int4_kernel<G, DENSE, ODD_N, FUSED>;
+    auto kernel = gemv_kernel<G, BITS, DENSE, ODD_N, FUSED>;
     static bool configured[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPQT_ERR_CUDA;
-    const int smem = (int)sizeof(GemvSmem<G>);
+    const int smem = (int)sizeof(GemvSmem<G, BITS>);
     if (!configured[dev]) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
             return SPQT_ERR_CUDA;
@@ -779,12 +827,14 @@ static spqt_status gemv_entry(const void* codes, const void* scales, const void*
     if ((long long)f.R * kMaxCtas >= (1ll << 31)) return SPQT_ERR_UNSUPPORTED;  // the work map is 32-bit
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const bool odd = (n & 1) != 0;
-    if (bits == 4 && group == 128)
-        return odd ? launch_int4<128, DENSE, true, FUSED>(f, codes, scales, zeros, x, idx, count, y, workspace, s, fa)
-                   : launch_int4<128, DENSE, false, FUSED>(f, codes, scales, zeros, x, idx, count, y, workspace, s, fa);
-    if (bits == 4 && group == 64)
-        return odd ? launch_int4<64, DENSE, true, FUSED>(f, codes, scales, zeros, x, idx, count, y, workspace, s, fa)
-                   : launch_int4<64, DENSE, false, FUSED>(f, codes, scales, zeros, x, idx, count, y, workspace, s, fa);
+#define SPQT_DISPATCH(GG, BB)                                                                                      \
+    return odd ? launch_gemv<GG, BB, DENSE, true, FUSED>(f, codes, scales, zeros, x, idx, count, y, workspace, s, fa) \
+               : launch_gemv<GG, BB, DENSE, false, FUSED>(f, codes, scales, zeros, x, idx, count, y, workspace, s, fa)
+    if (bits == 4 && group == 128) { SPQT_DISPATCH(128, 4); }
+    if (bits == 4 && group == 64) { SPQT_DISPATCH(64, 4); }
+    if (bits == 3 && group == 128) { SPQT_DISPATCH(128, 3); }
+    if (bits == 3 && group == 64) { SPQT_DISPATCH(64, 3); }
+#undef SPQT_DISPATCH
     return SPQT_ERR_UNSUPPORTED;
 }
 

@@ -13,7 +13,7 @@ from gpu_util import TOL, check_y, dev, pack_on_gpu, packed_to_host, run_sparse
 pytestmark = pytest.mark.gpu
 
 FORMATS = [(4, 128), (4, 64), (3, 128), (3, 64)]
-GEMV_FORMATS = [(4, 128), (4, 64)]
+GEMV_FORMATS = FORMATS
 
 
 @pytest.fixture(scope="module", autouse=True)
@@ -157,6 +157,7 @@ def test_one_hot_probes_return_the_dequantized_column(bits, group):
 
 @pytest.mark.parametrize("group", [64, 128])
 def test_lossless_family_is_bit_exact(group):
+    # (4-bit only: the family needs 16 levels)
     m, n = 4 * group, 700
     W = inputs.lossless_weights(m, n)
     x = inputs.small_rational_activations(n, seed=12)
@@ -303,6 +304,29 @@ def test_llama3_8b_shapes_on_sampled_rows(name, m, n, dist):
     B = oracle.block_bytes(bits, group)
     assert np.array_equal(codes[r * n * B:(r + 1) * n * B], c_ref)
     assert np.array_equal(s[r], s_ref[0]) and np.array_equal(z[r], z_ref[0])
+
+
+@pytest.mark.parametrize("bits,group", FORMATS)
+def test_llama2_70b_attention_shape_with_heavy_tailed_outliers(bits, group):
+    """8192 -> 8192, every format, x ~ Laplace with 1 % of the entries multiplied by 20, 50 % sparsity."""
+    m = n = 8192
+    W = inputs.weights(m, n, seed=70 + bits + group)
+    x = inputs.activations(n, seed=71, outlier_frac=0.01, outlier_scale=20.0)
+    p = pack_on_gpu(W, bits, group)
+    codes, s, z = packed_to_host(p)
+    ws = binding.new_workspace(m, n, bits, group)
+    rows = np.unique(np.concatenate([np.random.Generator(np.random.PCG64(6)).integers(0, m, size=160),
+                                     [0, group - 1, group, m - group, m - 1]])).astype(np.int32)
+    t = inputs.threshold_for_sparsity(x, 0.5)
+    y, idx, cnt = run_sparse(p, x, t, ws)
+    ref_idx, ref_cnt = oracle.sparsify(x, t)
+    assert cnt == ref_cnt and np.array_equal(idx, ref_idx)
+    y_ref, bound = oracle.sparse_gemv(codes, s, z, m, n, x, ref_idx, bits, group, rows=rows)
+    check_y(y[rows], y_ref, bound, "70B attention shape")
+    yd = binding.spqt_dense_gemv(p, dev(x), ws)
+    torch.cuda.synchronize()
+    yd_ref, dbound = oracle.dense_gemv(codes, s, z, m, n, x, bits, group, rows=rows)
+    check_y(yd.cpu().numpy()[rows], yd_ref, dbound, "70B attention shape, dense")
 
 
 # ------------------------------------------------------------------ host-buffer entry point
