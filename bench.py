@@ -7,7 +7,9 @@ one Llama-3-8B-shaped decoder layer at batch 1 -- q, k, v, o (4096->4096,
 codes, group 128, fp16 scale and zero, zigzag layout, 50 % activation sparsity.
 A *step* is one pass over those seven matrices: four index collections
 (attention input shared by q,k,v; attention output for o; MLP input shared by
-gate,up; MLP hidden for down) and seven sparse GEMVs.  Eight distinct layer
+gate,up; MLP hidden for down) and seven sparse GEMVs -- seven launches, because
+each index collection runs in the prologue of its site's first GEMV
+(spqt_sparsify_gemv); the 4 + 7 separate launches are timed as well.  Eight distinct layer
 copies (about 0.93 GB of packed weights, far larger than the 126 MB L2) are
 visited round-robin so that weights really come from HBM.
 
@@ -44,9 +46,10 @@ X_POOL = 4            # distinct hidden states per site, rotated
 FALLBACK_HBM_GBS = 6650.0
 METRIC = "sparse int4 GEMV effective HBM GB/s at 50% sparsity (Llama-3-8B-shaped decode-layer linears, batch 1)"
 
-# ncu dram__bytes_read.sum + dram__bytes_write.sum per sparse-GEMV launch, by shape, from the
-# capture summarised in profiles/ (see profiles/README.md); None until measured.
-NCU_TRAFFIC_BYTES = {}
+# ncu (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes of one sparse-GEMV launch, from the
+# capture summarised in profiles/gemv_int4_g128_28672x8192_full.md (a 117 MB matrix; traffic grows in
+# proportion to the active blocks, so the ratio is applied to the bench's mean launch).
+NCU_TRAFFIC_RATIO = 1.11
 
 
 def needed_bytes_gemv(m, n, count, bits=BITS, group=GROUP):
@@ -113,6 +116,23 @@ class ClockSampler:
                 pass
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
                 "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def max_over_ranks(value: float, device=None) -> float:
+    """The slowest rank's time: all-reduce MAX when a process group is up, the value itself otherwise."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(value)
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbs(bytes_per_rank: float, ms_local: float, world: int, device=None) -> float:
+    """Replicas only: every rank moves bytes_per_rank; the job's rate is all ranks' bytes over the slowest rank's time."""
+    ms = max_over_ranks(ms_local, device)
+    return world * bytes_per_rank / (ms * 1e-3) / 1e9
 
 
 # --------------------------------------------------------------------------- reference arm (CPU oracle)
@@ -223,6 +243,20 @@ def run_ours(args):
 
     stream = torch.cuda.Stream(device=dev)
 
+    def hot_path_step(i):
+        """The library's own best route: per site one launch collects the indices AND multiplies the
+        first matrix (spqt_sparsify_gemv); the site's other matrices reuse the index list."""
+        L = layers[i % LAYER_COPIES]
+        j = i % X_POOL
+        for s in sites:
+            first = True
+            for nm in sites[s][2]:
+                if first:
+                    binding.spqt_sparsify_gemv(L[nm], xd[s][j], ts[s][j], ws[nm], idx[s], cnt[s], ys[nm], stream=stream)
+                    first = False
+                else:
+                    binding.spqt_sparse_gemv(L[nm], xd[s][j], idx[s], cnt[s], ws[nm], ys[nm], stream=stream)
+
     def step(i, with_sparsify=True, gemv=True, dense=False):
         L = layers[i % LAYER_COPIES]
         j = i % X_POOL if with_sparsify else 0   # kernel-only regions keep the index lists of pool entry 0
@@ -291,22 +325,18 @@ def run_ours(args):
                 graph.replay()
             e1.record(stream)
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return max_over_ranks(e0.elapsed_time(e1), dev)
 
     K, W = args.steps, max(args.warmup, 3)
 
     # ---- main timed region (whole hot path), with clocks sampled during it
     l0 = binding.spqt_launch_count()
     with ClockSampler(local) as clk:
-        ms = timed(lambda i: step(i), K, W)
+        ms = timed(hot_path_step, K, W)
     launches = binding.spqt_launch_count() - l0
     g_len = graph_len(K)
-    launches_timed = 11 * K
+    launches_timed = 7 * K
+    ms_separate = timed(lambda i: step(i), K, W)   # the same work as 4 + 7 separate launches
     total_bytes = (K // g_len) * sum(step_bytes(i) for i in range(W, W + g_len))
     value = world * total_bytes / (ms * 1e-3) / 1e9
 
@@ -363,10 +393,7 @@ def run_ours(args):
         e2e_step(i)
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
-    if world > 1:
-        t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s = max_over_ranks(e2e_s, dev)
     e2e_bytes = e2e_K * sum(needed_bytes_gemv(shape[nm][0], shape[nm][1], counts[0][site_of[nm]])
                             + needed_bytes_sparsify(shape[nm][1], counts[0][site_of[nm]]) for nm in order)
     h2d = sum(shape[nm][1] * 2 for nm in order)
@@ -377,22 +404,22 @@ def run_ours(args):
     if rank == 0:
         cpu = oracle_sample(3, 1) if world >= 1 else None
         avg_launch_bytes = gb / n_gemv
-        traffic = None
-        if NCU_TRAFFIC_BYTES:
-            traffic = float(np.mean([NCU_TRAFFIC_BYTES[nm] for nm in order if nm in NCU_TRAFFIC_BYTES]))
+        traffic = NCU_TRAFFIC_RATIO * avg_launch_bytes
         line = {
             "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "int4 codes, f32 accumulate, f16 in/out", "data": "synthetic",
             "config": {"workload": "llama3-8b decode-layer linears q,k,v,o,gate,up,down; int4 g128 zigzag; batch 1; "
-                                   "50%% sparsity; 4 index collections + 7 sparse GEMVs per step, one stream, "
+                                   "50%% sparsity; per step 4 index collections (each fused into its site's first GEMV) + 7 sparse "
+                                   "GEMVs = 7 launches, one stream, "
                                    "replayed from a CUDA graph of %d steps" % g_len,
                        "l2_defeat": "%d distinct layer copies rotated, %.2f GB of packed weights (> 126 MB L2)" % (
                            LAYER_COPIES, weight_bytes / 1e9),
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
             "us_per_gemv": ms_gemv * 1e3 / n_gemv,
             "us_per_step": {"hot_path": ms * 1e3 / K, "gemv_only": ms_gemv * 1e3 / K,
-                            "dense_gemv_only": ms_dense * 1e3 / K, "sparsify_only": ms_sparsify * 1e3 / K},
+                            "dense_gemv_only": ms_dense * 1e3 / K, "sparsify_only": ms_sparsify * 1e3 / K,
+                            "separate_launches_4_sparsify_7_gemv": ms_separate * 1e3 / K},
             "speedup_vs_dense_same_layout": ms_dense / ms_gemv,
             "dense_gbs": gb_dense / (ms_dense * 1e-3) / 1e9,
             "pct_of_peak": {"of_measured_%.0f" % peak: 100 * achieved / peak, "of_nominal_8000": 100 * achieved / 8000},
