@@ -256,8 +256,8 @@ def spqt_sparse_linear_host(h: HostLinear, t: float, stream=None) -> torch.Tenso
     return h.y_host
 
 
-def spqt_set_tuning(gemv_ctas: int = 0) -> None:
-    _ok(lib().spqt_set_tuning(int(gemv_ctas), 0), "spqt_set_tuning")
+def spqt_set_tuning(gemv_ctas: int = 0, no_overlap: int = 0) -> None:
+    _ok(lib().spqt_set_tuning(int(gemv_ctas), int(no_overlap)), "spqt_set_tuning")
 
 
 def spqt_workspace_status(workspace: torch.Tensor, m: int, group: int = 128, stream=None) -> int:

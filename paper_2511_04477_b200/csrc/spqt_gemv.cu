@@ -51,6 +51,7 @@ constexpr int kMaxFusedN = 32768;        // largest n whose index collection can
 constexpr int kFusedCols = 8192;         // list entries a CTA keeps in shared memory in that case
 
 static int g_tune_ctas = 0;  // 0 = one CTA per SM
+static int g_no_pdl = 0;     // 1 = plain stream-ordered launches
 
 #ifdef SPQT_TRACE
 __device__ long long* g_trace;  // time stamps of CTA 0 (debug builds only)
@@ -333,6 +334,12 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
         }
     }
     __syncthreads();
+
+    // Programmatic dependent launch: this grid may have been started while the previous kernel of
+    // the stream was still draining.  Nothing above touches global memory; everything below waits
+    // for that kernel to complete, and lets the next kernel of the stream start early in turn.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     int count;
     Piece pc;
@@ -798,13 +805,23 @@ static spqt_status launch_gemv(const Format& f, const void* codes, const void* s
     int* status = counters + f.R;
     float* partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + header_bytes(f.R));
     float* zpartials = partials + (size_t)f.R * slots * G;
-    kernel<<<P, kGemvThreads, smem, s>>>(
-        static_cast<const uint8_t*>(codes), static_cast<const __half*>(scales),
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(P);
+    cfg.blockDim = dim3(kGemvThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_no_pdl ? 0 : 1;
+    const cudaError_t err = cudaLaunchKernelEx(
+        &cfg, kernel, static_cast<const uint8_t*>(codes), static_cast<const __half*>(scales),
         static_cast<const __half*>(zeros), f.R, f.n, static_cast<const __half*>(x), idx, count,
         static_cast<__half*>(y), counters, status, partials, zpartials, slots,
         fa.t, fa.idx_out, fa.count_out);
     count_launch();
-    return cudaGetLastError() == cudaSuccess ? SPQT_OK : SPQT_ERR_CUDA;
+    return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SPQT_OK : SPQT_ERR_CUDA;
 }
 
 template <bool DENSE, bool FUSED = false>
@@ -915,8 +932,9 @@ spqt_status spqt_sparse_gemv_static(const void* codes, const void* scales, const
 
 spqt_status spqt_set_tuning(int gemv_ctas, int reserved)
 {
-    if (gemv_ctas < 0 || reserved < 0) return SPQT_ERR_INVALID_ARG;
+    if (gemv_ctas < 0 || reserved < 0 || reserved > 1) return SPQT_ERR_INVALID_ARG;
     spqt::g_tune_ctas = gemv_ctas;
+    spqt::g_no_pdl = reserved;
     return SPQT_OK;
 }
 
