@@ -209,28 +209,54 @@ __device__ __forceinline__ void halve(const float* in, float* out, int lane, int
 
 // The piece of CTA c: block-rows r_first..r_last, and of each the slice of the
 // active list that belongs to this CTA.  Uniform across the CTA.
+constexpr int kSegTable = 16;  // segments of a CTA whose slices are computed once and kept in shared memory
+
 struct Piece {
     int R, P, c, count, r_first, r_last;
     unsigned qc, rc;  // count = qc * P + rc: keeps the slice arithmetic in 32 bits (the host checks R * P < 2^31)
+    const int* tab;   // shared memory: [2 * kSegTable] slice begin / end of the first segments, or nullptr
 
-    __device__ __forceinline__ void init(int R_, int P_, int c_, int count_)
+    // the block-rows of the piece do not depend on the count: computed while the count is being fetched
+    __device__ __forceinline__ void init_rows(int R_, int P_, int c_)
     {
-        R = R_; P = P_; c = c_; count = count_;
+        R = R_; P = P_; c = c_;
         const unsigned lo = (unsigned)c * (unsigned)R, hi = lo + (unsigned)R;
         r_first = (int)(lo / (unsigned)P);
         r_last = (int)((hi - 1u) / (unsigned)P);
+        tab = nullptr;
+    }
+    __device__ __forceinline__ void set_count(int count_)
+    {
+        count = count_;
         qc = (unsigned)count / (unsigned)P;
         rc = (unsigned)count - qc * (unsigned)P;
     }
     // floor(u * count / P) for 0 <= u <= P
     __device__ __forceinline__ int scaled(unsigned u) const { return (int)(u * qc + (u * rc) / (unsigned)P); }
-    __device__ __forceinline__ void slice(int row, int* a, int* b) const
+    __device__ __forceinline__ void slice_compute(int row, int* a, int* b) const
     {
         const unsigned lo = (unsigned)c * (unsigned)R, hi = lo + (unsigned)R, base = (unsigned)row * (unsigned)P;
         const unsigned u0 = (lo > base ? lo : base) - base;
         const unsigned u1 = (hi < base + (unsigned)P ? hi : base + (unsigned)P) - base;
         *a = scaled(u0);
         *b = scaled(u1);
+    }
+    __device__ __forceinline__ void slice(int row, int* a, int* b) const
+    {
+        const int i = row - r_first;
+        if (tab != nullptr && i < kSegTable) {
+            *a = tab[2 * i];
+            *b = tab[2 * i + 1];
+        } else {
+            slice_compute(row, a, b);
+        }
+    }
+    // Fills the shared-memory table (threads 0..kSegTable-1 each take one segment, so the divisions
+    // run side by side) -- call with the whole CTA, followed by a CTA barrier.
+    __device__ __forceinline__ void fill_table(int* table, int tid)
+    {
+        if (tid < kSegTable && r_first + tid <= r_last) slice_compute(r_first + tid, &table[2 * tid], &table[2 * tid + 1]);
+        tab = table;
     }
     // contributors to block-row `row`: CTAs first .. first+n-1
     __device__ __forceinline__ void contributors(int row, int* first, int* n) const
@@ -287,17 +313,17 @@ struct GemvSmem {
     alignas(16) float red[2][kWorkers][G];               // per-warp partial sums of a finished segment
     float red_z[2][kWorkers];                            // and their offset terms
     uint64_t red_full[2], red_empty[2];
-    // fused index collection only: activity mask and exclusive count of every 32 entries of x
-    unsigned act_mask[kMaxFusedN / 32];
-    int act_before[kMaxFusedN / 32 + 1];
-    int fused_cols[kFusedCols];  // the part of the index list this CTA reads, when it fits
+    int seg_table[2 * kSegTable];                        // slices of the CTA's first segments
+    // fused index collection only
+    alignas(16) int load_tot[kMaxFusedN / 256];  // active entries of every 256 entries of x
+    int fused_cols[kFusedCols];                   // the part of the index list this CTA reads, when it fits
 };
 
-// FUSED: the index collection runs in the kernel's prologue.  Every CTA scans x (ballot/popc per 32
-// entries, block counts scanned in shared memory), writes the part of the ascending index list that
-// its own slices cover to idx_out (the slices of all CTAs cover the whole list; overlapping parts
-// receive identical values), CTA 0 writes the count, and the pipeline then reads idx_out like a list
-// collected by a separate launch.
+// FUSED: the index collection runs in the kernel's prologue.  Every CTA scans x (each lane tests 8
+// entries, popc and warp-shuffle prefix sums; only the totals of every 256 entries cross shared
+// memory), keeps the part of the ascending index list that its own slices cover in shared memory (or,
+// when that part is too long, writes it to idx_out and reads it back like a list collected by a
+// separate launch), and writes an even share of idx_out; CTA 0 writes the count.
 template <int G, int BITS, bool DENSE, bool ODD_N, bool FUSED>
 __global__ void __launch_bounds__(kGemvThreads, 1)
 gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales,
@@ -341,15 +367,17 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-    int count;
+    int count = 0;
+    if (!FUSED) count = DENSE ? n : *count_ptr;  // in flight while the row range is worked out
     Piece pc;
+    pc.init_rows(R, P, c);
     const int32_t* idx = idx_in;
     int need_lo = 0;          // FUSED: first list position held in sm.fused_cols
     bool cols_local = false;  // FUSED: the pipeline reads its column numbers from sm.fused_cols
     if (FUSED) {
-        const int nb = (n + 31) / 32;
-        // All loads first (one memory round trip), then the ballots.  A warp load covers 256 entries:
-        // lane l holds entries 8l..8l+7, so every four lanes make one 32-entry block.
+        // All loads first (one memory round trip).  A warp load covers 256 entries: lane l holds
+        // entries 8l..8l+7.  Masks and counts stay in registers; only the per-load totals go through
+        // shared memory, and every warp scans those totals for itself (no second barrier).
         constexpr int kWarps = kGemvThreads / 32;
         constexpr int kMaxLoads = (kMaxFusedN / 256 + kWarps - 1) / kWarps;
         const int nv = (n + 255) / 256;
@@ -375,55 +403,65 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
                 }
             }
         }
+        // the largest fp16 value not above t (any negative value if t < 0: everything but NaN is
+        // active; +inf if t is NaN or +inf: nothing is)
+        const __half thr_h = (thr != thr) ? __ushort_as_half((unsigned short)0x7c00)
+                                          : (thr < 0.0f ? __float2half_rn(-1.0f) : __float2half_rd(thr));
+        const __half2 thr_h2 = __half2half2(thr_h);
+        unsigned m8[kMaxLoads];   // activity of this lane's 8 entries of load j
+        int lane_excl[kMaxLoads]; // active entries of load j in the lanes below
 #pragma unroll
         for (int j = 0; j < kMaxLoads; ++j) {
             const int li = warp + j * kWarps;
+            m8[j] = 0;
+            lane_excl[j] = 0;
             if (li < nv) {  // uniform across the warp
                 const int k0 = li * 256 + lane * 8;
                 const unsigned wds[4] = {xv[j].x, xv[j].y, xv[j].z, xv[j].w};
-                unsigned m8 = 0;
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const unsigned short hb = (unsigned short)(wds[e >> 1] >> ((e & 1) * 16));
-                    // exact widening; NaN compares false and is never active
-                    const bool p = (k0 + e < n) && (fabsf(__half2float(__ushort_as_half(hb))) > thr);
-                    m8 |= (p ? 1u : 0u) << e;
+                for (int e2 = 0; e2 < 4; ++e2) {
+                    // |x| > t  <=>  |x| > (largest fp16 value <= t): two entries per compare, in fp16,
+                    // exact; the ordered compare is false for NaN
+                    const unsigned ab = wds[e2] & 0x7fff7fffu;
+                    const unsigned gt = __hgt2_mask(*reinterpret_cast<const __half2*>(&ab), thr_h2);
+                    m8[j] |= ((gt & 1u) | ((gt >> 15) & 2u)) << (2 * e2);
                 }
-                unsigned m = m8 << ((lane & 3) * 8);
-                m |= __shfl_xor_sync(0xffffffffu, m, 1);
-                m |= __shfl_xor_sync(0xffffffffu, m, 2);
-                const int b = li * 8 + (lane >> 2);
-                if ((lane & 3) == 0 && b < nb) {
-                    sm.act_mask[b] = m;
-                    sm.act_before[b + 1] = __popc(m);
+                const int left = n - k0;  // entries of this lane that exist
+                if (left < 8) m8[j] &= (left <= 0) ? 0u : ((1u << left) - 1u);
+                const int c8 = __popc(m8[j]);
+                int incl = c8;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int up = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += up;
                 }
+                lane_excl[j] = incl - c8;
+                if (lane == 31) sm.load_tot[li] = incl;
             }
         }
         SPQT_TRACE_EVENT(tid == 0, 3991);
         __syncthreads();
         SPQT_TRACE_EVENT(tid == 0, 3992);
-        if (warp == 0) {
-            // exclusive scan of the block counts: each lane owns a run of consecutive blocks
-            const int per = (nb + 31) / 32, b0 = lane * per, b1 = min(b0 + per, nb);
-            int sum = 0;
-            for (int b = b0; b < b1; ++b) sum += sm.act_before[b + 1];
-            int incl = sum;
+        // every warp: exclusive scan of the (at most 128) load totals, four per lane
+        int tot4[4], base4[4];
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int up = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += up;
-            }
-            int run = incl - sum;
-            if (lane == 0) sm.act_before[0] = 0;
-            for (int b = b0; b < b1; ++b) {
-                run += sm.act_before[b + 1];
-                sm.act_before[b + 1] = run;
-            }
+        for (int q = 0; q < 4; ++q) tot4[q] = (lane * 4 + q < nv) ? sm.load_tot[lane * 4 + q] : 0;
+        const int s4 = tot4[0] + tot4[1] + tot4[2] + tot4[3];
+        int incl4 = s4;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int up = __shfl_up_sync(0xffffffffu, incl4, o);
+            if (lane >= o) incl4 += up;
         }
-        __syncthreads();
+        base4[0] = incl4 - s4;
+        base4[1] = base4[0] + tot4[0];
+        base4[2] = base4[1] + tot4[1];
+        base4[3] = base4[2] + tot4[2];
+        count = __shfl_sync(0xffffffffu, incl4, 31);
         SPQT_TRACE_EVENT(tid == 0, 3993);
-        count = sm.act_before[nb];
-        pc.init(R, P, c, count);
+        pc.set_count(count);
+        pc.fill_table(sm.seg_table, tid);
+        __syncthreads();
         if (c == 0 && tid == 0) *count_out = count;
         // list positions this CTA will read: the union of its slices.  If that part fits in shared
         // memory the pipeline takes its column numbers from there (no round trip through global
@@ -439,24 +477,37 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
         cols_local = (need_hi - need_lo) <= kFusedCols;
         SPQT_TRACE_EVENT(tid == 0, 3994);
         const int out_lo = pc.scaled((unsigned)c), out_hi = pc.scaled((unsigned)c + 1u);
-        for (int b = warp; b < nb; b += kGemvThreads / 32) {
-            const int before = sm.act_before[b], after = sm.act_before[b + 1];
-            const bool mine = after > need_lo && before < need_hi, share = after > out_lo && before < out_hi;
-            if (!mine && !share) continue;
-            const unsigned m = sm.act_mask[b];
-            if ((m >> lane) & 1u) {
-                const int pos = before + __popc(m & ((1u << lane) - 1u));
-                const int col = b * 32 + lane;
-                const bool need = pos >= need_lo && pos < need_hi;
-                if (need && cols_local) sm.fused_cols[pos - need_lo] = col;
-                if ((need && !cols_local) || (pos >= out_lo && pos < out_hi)) idx_out[pos] = col;
+#pragma unroll
+        for (int j = 0; j < kMaxLoads; ++j) {
+            const int li = warp + j * kWarps;
+            if (li < nv) {
+                // first list position of load li: component li & 3 of lane li >> 2
+                const int b0 = __shfl_sync(0xffffffffu, base4[0], li >> 2), b1 = __shfl_sync(0xffffffffu, base4[1], li >> 2);
+                const int b2 = __shfl_sync(0xffffffffu, base4[2], li >> 2), b3 = __shfl_sync(0xffffffffu, base4[3], li >> 2);
+                const int q = li & 3;
+                const int first = (q == 0 ? b0 : q == 1 ? b1 : q == 2 ? b2 : b3) + lane_excl[j];
+                const int last = first + __popc(m8[j]);
+                const bool mine = last > need_lo && first < need_hi, share = last > out_lo && first < out_hi;
+                if (mine || share) {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        if ((m8[j] >> e) & 1u) {
+                            const int pos = first + __popc(m8[j] & ((1u << e) - 1u));
+                            const int col = li * 256 + lane * 8 + e;
+                            const bool need = pos >= need_lo && pos < need_hi;
+                            if (need && cols_local) sm.fused_cols[pos - need_lo] = col;
+                            if ((need && !cols_local) || (pos >= out_lo && pos < out_hi)) idx_out[pos] = col;
+                        }
+                    }
+                }
             }
         }
         __syncthreads();  // the CTA's own writes (shared or global) are visible to its pipeline
         idx = idx_out;
     } else {
-        count = DENSE ? n : *count_ptr;
-        pc.init(R, P, c, count);
+        pc.set_count(count);
+        pc.fill_table(sm.seg_table, tid);
+        __syncthreads();
     }
     SPQT_TRACE_EVENT(tid == 0, 4000);
 

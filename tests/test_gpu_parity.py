@@ -273,6 +273,35 @@ def test_dense_gemv_matches_oracle_and_the_sparse_path_at_threshold_below_zero(b
     check_y(ys, y_ref, bound, "sparse at t<0")
 
 
+def test_config_single_gemv_4096x4096_seed0_every_row():
+    """The single-GEMV configuration, every output row: W 4096x4096 ~ N(0, 0.02^2) int4 g128,
+    x ~ Laplace(0,1), threshold = nearest-rank median of |x|, seed 0."""
+    m = n = 4096
+    W = inputs.weights(m, n, seed=0)
+    x = inputs.activations(n, seed=0, dist="laplace")
+    t = inputs.threshold_for_sparsity(x, 0.5)
+    assert abs(t - 0.693) < 0.03                       # ln 2 for |Laplace|
+    p = pack_on_gpu(W, 4, 128)
+    codes, s, z = packed_to_host(p)
+    c_ref, s_ref, z_ref = oracle.pack(W, 4, 128)
+    assert np.array_equal(codes, c_ref) and np.array_equal(s, s_ref) and np.array_equal(z, z_ref)
+    ws = binding.new_workspace(m, n, 4, 128)
+    y, idx, cnt = run_sparse(p, x, t, ws)
+    ref_idx, ref_cnt = oracle.sparsify(x, t)
+    assert cnt == ref_cnt and np.array_equal(idx, ref_idx)
+    assert abs(inputs.realised_sparsity(x, t) - 0.5) < 2e-3
+    y_ref, bound = oracle.sparse_gemv(codes, s, z, m, n, x, ref_idx, 4, 128)
+    worst = check_y(y, y_ref, bound, "config 0")
+    assert worst < 5e-4                                # an order of magnitude inside the tolerance
+    yf, _, _ = binding.spqt_sparsify_gemv(p, dev(x), t, ws)
+    torch.cuda.synchronize()
+    assert np.array_equal(yf.cpu().numpy().view(np.uint16), y.view(np.uint16))
+    yd = binding.spqt_dense_gemv(p, dev(x), ws)
+    torch.cuda.synchronize()
+    yd_ref, dbound = oracle.dense_gemv(codes, s, z, m, n, x, 4, 128)
+    check_y(yd.cpu().numpy(), yd_ref, dbound, "config 0 dense")
+
+
 # ------------------------------------------------------------------ full-size shapes, sampled rows
 
 @pytest.mark.parametrize("name,m,n,dist", [l for l in inputs.LLAMA3_8B_LINEARS if l[0] in ("q", "k", "gate", "down")])
