@@ -49,8 +49,8 @@ METRIC = "sparse int4 GEMV effective HBM GB/s at 50% sparsity (Llama-3-8B-shaped
 
 # ncu (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes of one sparse-GEMV launch, from the
 # capture summarised in profiles/gemv_int4_g128_28672x8192_full.md (a 117 MB matrix; traffic grows in
-# proportion to the active blocks, so the ratio is applied to the bench's mean launch).
-NCU_TRAFFIC_RATIO = 1.11
+# proportion to the active blocks; 1.06 on the bench-sized 28672x4096 case, 1.12 on the 117 MB one).
+NCU_TRAFFIC_RATIO = 1.06
 
 
 def needed_bytes_gemv(m, n, count, bits=BITS, group=GROUP):
