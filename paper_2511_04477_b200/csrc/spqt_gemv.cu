@@ -598,7 +598,10 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
     Cursor ca, cb;  // stage A / stage B cursors (the consume side walks the segments itself)
     ca.init(pc, warp);
     cb = ca;
-    unsigned qa = 0, qb = 0, qc = 0;  // chunk sequence numbers of the three stages
+    // ring positions of the three stages: chunk number modulo the ring length, kept by wrap-around
+    // (the lengths are not powers of two)
+    unsigned qa2 = 0, qb1 = 0, qb2 = 0, qc1 = 0, qc2 = 0;  // ..1: modulo D (stages), ..2: modulo 2*D (columns)
+    auto wrap = [](unsigned& v, unsigned len) { v = (v + 1 == len) ? 0u : v + 1; };
 
     // block-row constants of stage B, refreshed when its cursor enters a new block-row
     int b_row = -1;
@@ -610,9 +613,9 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
     // stage A: column numbers of the warp's chunk number qa
     auto issue_a = [&]() {
         if (!DENSE && !(FUSED && cols_local) && ca.valid(pc)) {
-            if (ca.pos + lane < ca.p1) cp_async_4(smem_u32(&my_cols[qa % (2 * D)][lane]), idx + ca.pos + lane);
+            if (ca.pos + lane < ca.p1) cp_async_4(smem_u32(&my_cols[qa2][lane]), idx + ca.pos + lane);
             ca.advance(pc, warp);
-            ++qa;
+            wrap(qa2, 2 * D);
         }
     };
     // stage B: code blocks and metadata words of chunk number qb (its columns have landed)
@@ -627,8 +630,8 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
                 b_zeros = reinterpret_cast<const unsigned short*>(zeros) + row_base;
             }
             const int valid = cb.p1 - cb.pos;  // entries of this chunk (>= kChunk when full)
-            const int* cols = (FUSED && cols_local) ? &sm.fused_cols[cb.pos - need_lo] : my_cols[qb % (2 * D)];
-            typename GemvSmem<G, BITS>::Stage& st = my_stage[qb % D];
+            const int* cols = (FUSED && cols_local) ? &sm.fused_cols[cb.pos - need_lo] : my_cols[qb2];
+            typename GemvSmem<G, BITS>::Stage& st = my_stage[qb1];
             const unsigned dst = smem_u32(&st.codes[0]) + lane * 16;
             if (BITS == 4) {
 #pragma unroll
@@ -677,7 +680,8 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
                 }
             }
             cb.advance(pc, warp);
-            ++qb;
+            wrap(qb1, D);
+            wrap(qb2, 2 * D);
         }
     };
 
@@ -720,12 +724,12 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
 #ifdef SPQT_TRACE
             const long long tc1 = clock64();
 #endif
-            const typename GemvSmem<G, BITS>::Stage& st = my_stage[qc % D];
+            const typename GemvSmem<G, BITS>::Stage& st = my_stage[qc1];
             const unsigned xw = st.meta[0][lane], sw = st.meta[1][lane], zw = st.meta[2][lane];
             unsigned kk;
             if (DENSE) kk = (unsigned)(pos + lane);
             else if (FUSED && cols_local) kk = (pos + lane < p1) ? (unsigned)sm.fused_cols[pos - need_lo + lane] : 0u;
-            else kk = (unsigned)my_cols[qc % (2 * D)][lane];
+            else kk = (unsigned)my_cols[qc2][lane];
 #ifdef SPQT_TRACE
             const long long tc2 = clock64();
 #endif
@@ -754,7 +758,8 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
             issue_b();
             issue_a();
             cp_async_commit();
-            ++qc;
+            wrap(qc1, D);
+            wrap(qc2, 2 * D);
 #ifdef SPQT_TRACE
             tr_wait += tc1 - tc0; tr_issue += 0; tr_math += clock64() - tc2; ++tr_n;
 #endif
