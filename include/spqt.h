@@ -184,7 +184,7 @@ spqt_status spqt_sparse_linear_host(const void* codes, const void* scales, const
 
 /*
  * Tuning aid: number of CTAs of the GEMV grid (0 restores the built-in rule, one
- * persistent CTA per SM; values above 1024 are clamped).  `no_overlap` = 1 launches the GEMV
+ * persistent CTA per SM; values above 512 are clamped).  `no_overlap` = 1 launches the GEMV
  * kernels strictly stream-ordered instead of letting a GEMV start (and wait inside the kernel)
  * while the previous kernel of the stream drains; 0 is the default.
  * Any value gives the same results up to the order of partial sums.

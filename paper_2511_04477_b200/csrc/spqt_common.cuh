@@ -35,19 +35,34 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 
 // Largest grid any tuning may use for a GEMV; the workspace is sized for it
 // (independent of the device, so sizes can be computed without a GPU).
-constexpr int kMaxCtas = 1024;
+constexpr int kMaxCtas = 512;
 
 // Upper bound on the number of CTAs that contribute partial sums to one block-row.
 inline int max_slots(int R) { return (kMaxCtas + R - 1) / R + 1; }
 
+// Block-rows with at most kTagSlots contributing CTAs exchange their partial sums as tagged 64-bit
+// words, the others as plain fp32 values behind a fence.
+constexpr int kTagSlots = 4;
+
 // Workspace layout: [R] int32 arrival counters (kept zero between calls), one
 // int32 status word (non-zero after a bounded wait expired), padded to 256 B;
-// then fp32 partials [R][slots][G] and offset-term partials [R][slots].
+// then 64-bit words [R][kTagSlots][G + 2]: per contributing CTA the G partial sums
+// of the block-row, its offset-term partial and a word of padding, each an fp32
+// value with a tag in the high half (all zero between calls); then, only when a
+// block-row can have more than kTagSlots contributors, fp32 partials
+// [R][slots][G] and offset-term partials [R][slots] (contents irrelevant between calls).
 inline size_t header_bytes(int R) { return (((size_t)(R + 1) * 4 + 255) / 256) * 256; }
+
+inline size_t tagged_bytes(const Format& f)
+{
+    return (size_t)f.R * kTagSlots * (size_t)(f.group + 2) * sizeof(unsigned long long);
+}
 
 inline size_t workspace_bytes(const Format& f)
 {
-    return header_bytes(f.R) + (size_t)f.R * (size_t)max_slots(f.R) * (size_t)(f.group + 1) * sizeof(float);
+    const int slots = max_slots(f.R);
+    const size_t plain = slots > kTagSlots ? (size_t)f.R * (size_t)slots * (size_t)(f.group + 1) * sizeof(float) : 0;
+    return header_bytes(f.R) + tagged_bytes(f) + plain;
 }
 
 int sm_count();               // SMs of the current device (cached per device); <= 0 on error

@@ -6,9 +6,12 @@
 // the fraction [u0,u1) of block-row r means the slice [u0*count, u1*count) of
 // the ACTIVE index list, so the load follows the active entries, not the matrix
 // columns, and every CTA streams the same number of blocks whatever R is.  Each
-// (CTA, block-row) segment yields G fp32 partial sums; whichever CTA contributes
-// last to a block-row (arrive-only counter: nobody waits on another CTA) adds
-// the partials in a fixed order, adds the offset term and rounds to fp16.
+// (CTA, block-row) segment yields G fp32 partial sums, published as tagged 64-bit
+// words; whichever CTA contributes last to a block-row (arrive-only counter: no
+// CTA ever waits for another one to run, only for stores already issued to
+// become visible) adds the partials in slot order, adds the offset term and
+// rounds to fp16.  A CTA that finds all the other partials present before its own
+// sum is ready skips the counter and finishes the block-row directly.
 //
 // Inside a CTA, kWorkers warps each run their own copy pipeline over chunks of
 // 32 list entries (chunks are dealt round-robin to the warps); nothing is shared
@@ -37,6 +40,8 @@
 // multiplier a*2^(93-p) is an exact power-of-two rescale, so each product is
 // a*code*2^-56 up to the single rounding of the FMA.  One logic op and one FMA
 // per weight; two FMAs are issued as one packed fma.rn.f32x2.
+#include <cstddef>
+
 #include "spqt_common.cuh"
 
 namespace spqt {
@@ -55,7 +60,7 @@ static int g_no_pdl = 0;     // 1 = plain stream-ordered launches
 
 #ifdef SPQT_TRACE
 __device__ long long* g_trace;  // time stamps of CTA 0 (debug builds only)
-#define SPQT_TRACE_EVENT(cond, slot) do { if ((cond) && blockIdx.x == 0 && g_trace && (slot) < 4096) g_trace[(slot)] = clock64(); } while (0)
+#define SPQT_TRACE_EVENT(cond, slot) do { if ((cond) && blockIdx.x == 0 && spqt_tr && (slot) < 4096) spqt_tr[(slot)] = clock64(); } while (0)
 #else
 #define SPQT_TRACE_EVENT(cond, slot) do { } while (0)
 #endif
@@ -129,6 +134,30 @@ __device__ __forceinline__ void cp_async_4(unsigned smem_dst, const void* gmem_s
 __device__ __forceinline__ void cp_async_4_ca(unsigned smem_dst, const void* gmem_src)
 {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
+}
+// A partial sum travels between CTAs as one 64-bit word: the fp32 value in the low half, a non-zero
+// tag in the high half.  One aligned 64-bit access is indivisible, so a reader that sees the tag has
+// the value: no fence is needed between the two.
+constexpr unsigned long long kTagBit = 1ull << 32;
+__device__ __forceinline__ unsigned long long ld_word(const unsigned long long* p)
+{
+    unsigned long long v;
+    asm volatile("ld.relaxed.gpu.global.b64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_word(unsigned long long* p, unsigned long long v)
+{
+    asm volatile("st.relaxed.gpu.global.b64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+// stores under a predicate (never a branch)
+__device__ __forceinline__ void st_shared_if(unsigned cond, unsigned smem_dst, int v)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %0, 0;\n\t@p st.shared.u32 [%1], %2;\n\t}" ::"r"(cond), "r"(smem_dst), "r"(v) : "memory");
+}
+__device__ __forceinline__ void st_global_if(unsigned cond, int* dst, int v)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %0, 0;\n\t@p st.global.u32 [%1], %2;\n\t}" ::"r"(cond), "l"(dst), "r"(v) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
@@ -209,30 +238,40 @@ __device__ __forceinline__ void halve(const float* in, float* out, int lane, int
 
 // The piece of CTA c: block-rows r_first..r_last, and of each the slice of the
 // active list that belongs to this CTA.  Uniform across the CTA.
-constexpr int kSegTable = 16;  // segments of a CTA whose slices are computed once and kept in shared memory
+
+// floor(v / d) for any 32-bit v from the multiplier m = floor((2^32 - 1) / d): the high product is
+// the quotient or one less (the multiplier falls short of 2^32 / d by at most 1), one compare fixes it.
+__device__ __forceinline__ unsigned magic_of(unsigned d) { return 0xffffffffu / d; }
+__device__ __forceinline__ unsigned magic_div(unsigned v, unsigned d, unsigned m)
+{
+    const unsigned q = __umulhi(v, m);
+    return q + ((v - q * d >= d) ? 1u : 0u);
+}
 
 struct Piece {
     int R, P, c, count, r_first, r_last;
+    unsigned mP, mR;  // multipliers of magic_div for P and R: one real division each per thread,
+                      // issued while the first loads are in flight
     unsigned qc, rc;  // count = qc * P + rc: keeps the slice arithmetic in 32 bits (the host checks R * P < 2^31)
-    const int* tab;   // shared memory: [2 * kSegTable] slice begin / end of the first segments, or nullptr
 
     // the block-rows of the piece do not depend on the count: computed while the count is being fetched
     __device__ __forceinline__ void init_rows(int R_, int P_, int c_)
     {
         R = R_; P = P_; c = c_;
+        mP = magic_of((unsigned)P);
+        mR = magic_of((unsigned)R);
         const unsigned lo = (unsigned)c * (unsigned)R, hi = lo + (unsigned)R;
-        r_first = (int)(lo / (unsigned)P);
-        r_last = (int)((hi - 1u) / (unsigned)P);
-        tab = nullptr;
+        r_first = (int)magic_div(lo, (unsigned)P, mP);
+        r_last = (int)magic_div(hi - 1u, (unsigned)P, mP);
     }
     __device__ __forceinline__ void set_count(int count_)
     {
         count = count_;
-        qc = (unsigned)count / (unsigned)P;
+        qc = magic_div((unsigned)count, (unsigned)P, mP);
         rc = (unsigned)count - qc * (unsigned)P;
     }
     // floor(u * count / P) for 0 <= u <= P
-    __device__ __forceinline__ int scaled(unsigned u) const { return (int)(u * qc + (u * rc) / (unsigned)P); }
+    __device__ __forceinline__ int scaled(unsigned u) const { return (int)(u * qc + magic_div(u * rc, (unsigned)P, mP)); }
     __device__ __forceinline__ void slice_compute(int row, int* a, int* b) const
     {
         const unsigned lo = (unsigned)c * (unsigned)R, hi = lo + (unsigned)R, base = (unsigned)row * (unsigned)P;
@@ -241,28 +280,12 @@ struct Piece {
         *a = scaled(u0);
         *b = scaled(u1);
     }
-    __device__ __forceinline__ void slice(int row, int* a, int* b) const
-    {
-        const int i = row - r_first;
-        if (tab != nullptr && i < kSegTable) {
-            *a = tab[2 * i];
-            *b = tab[2 * i + 1];
-        } else {
-            slice_compute(row, a, b);
-        }
-    }
-    // Fills the shared-memory table (threads 0..kSegTable-1 each take one segment, so the divisions
-    // run side by side) -- call with the whole CTA, followed by a CTA barrier.
-    __device__ __forceinline__ void fill_table(int* table, int tid)
-    {
-        if (tid < kSegTable && r_first + tid <= r_last) slice_compute(r_first + tid, &table[2 * tid], &table[2 * tid + 1]);
-        tab = table;
-    }
+    __device__ __forceinline__ void slice(int row, int* a, int* b) const { slice_compute(row, a, b); }
     // contributors to block-row `row`: CTAs first .. first+n-1
     __device__ __forceinline__ void contributors(int row, int* first, int* n) const
     {
-        const unsigned f = ((unsigned)row * (unsigned)P) / (unsigned)R;
-        const unsigned l = (((unsigned)row + 1u) * (unsigned)P - 1u) / (unsigned)R;
+        const unsigned f = magic_div((unsigned)row * (unsigned)P, (unsigned)R, mR);
+        const unsigned l = magic_div(((unsigned)row + 1u) * (unsigned)P - 1u, (unsigned)R, mR);
         *first = (int)f;
         *n = (int)(l - f + 1u);
     }
@@ -313,17 +336,17 @@ struct GemvSmem {
     alignas(16) float red[2][kWorkers][G];               // per-warp partial sums of a finished segment
     float red_z[2][kWorkers];                            // and their offset terms
     uint64_t red_full[2], red_empty[2];
-    int seg_table[2 * kSegTable];                        // slices of the CTA's first segments
     // fused index collection only
     alignas(16) int load_tot[kMaxFusedN / 256];  // active entries of every 256 entries of x
     int fused_cols[kFusedCols];                   // the part of the index list this CTA reads, when it fits
 };
 
-// FUSED: the index collection runs in the kernel's prologue.  Every CTA scans x (each lane tests 8
-// entries, popc and warp-shuffle prefix sums; only the totals of every 256 entries cross shared
-// memory), keeps the part of the ascending index list that its own slices cover in shared memory (or,
-// when that part is too long, writes it to idx_out and reads it back like a list collected by a
-// separate launch), and writes an even share of idx_out; CTA 0 writes the count.
+// FUSED: the index collection runs in the kernel's prologue.  Every CTA copies x to shared memory and
+// scans it (each lane tests 8 entries in fp16; popc and warp reductions give the number of active
+// entries of every 256-entry piece), then expands only the pieces that overlap the list positions its
+// own slices cover: into shared memory, or, when that part is too long, into idx_out, from where it
+// reads them back like a list collected by a separate launch.  The CTAs that work on block-row 0
+// cover the whole list between them and write idx_out; CTA 0 writes the count.
 template <int G, int BITS, bool DENSE, bool ODD_N, bool FUSED>
 __global__ void __launch_bounds__(kGemvThreads, 1)
 gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales,
@@ -331,7 +354,8 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
                  const __half* __restrict__ x, const int32_t* idx_in,
                  const int32_t* count_ptr, __half* __restrict__ y,
                  int* __restrict__ counters, int* __restrict__ status,
-                 float* __restrict__ partials, float* __restrict__ zpartials, int max_slots,
+                 unsigned long long* __restrict__ words, float* __restrict__ partials,
+                 float* __restrict__ zpartials, int max_slots,
                  float thr, int32_t* idx_out, int32_t* count_out)
 {
     constexpr int B = G * BITS / 8;
@@ -348,6 +372,9 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int P = gridDim.x, c = blockIdx.x;
+#ifdef SPQT_TRACE
+    long long* const spqt_tr = g_trace;  // one load: an event is then a clock read and a store
+#endif
     SPQT_TRACE_EVENT(tid == 0, 3990);
 #ifdef SPQT_TRACE
     if (tid == 0 && g_trace && c < 200) g_trace[2000 + c] = (long long)global_ns();
@@ -372,100 +399,76 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
     Piece pc;
     pc.init_rows(R, P, c);
     const int32_t* idx = idx_in;
+    const unsigned short* xb0 = reinterpret_cast<const unsigned short*>(x);
     int need_lo = 0;          // FUSED: first list position held in sm.fused_cols
     bool cols_local = false;  // FUSED: the pipeline reads its column numbers from sm.fused_cols
     if (FUSED) {
-        // All loads first (one memory round trip).  A warp load covers 256 entries: lane l holds
-        // entries 8l..8l+7.  Masks and counts stay in registers; only the per-load totals go through
-        // shared memory, and every warp scans those totals for itself (no second barrier).
+        // Three short loops over the 256-entry pieces of x (piece li belongs to warp li % kWarps, lane l
+        // holds entries 8l..8l+7), with x and the per-lane results kept in shared memory that the
+        // pipeline only uses afterwards: (1) activity mask of the lane's entries and warp prefix sums,
+        // (2) every warp scans the piece totals for itself, (3) the pieces that overlap the list
+        // positions this CTA needs are expanded into column numbers.
         constexpr int kWarps = kGemvThreads / 32;
-        constexpr int kMaxLoads = (kMaxFusedN / 256 + kWarps - 1) / kWarps;
+        unsigned short* xs = reinterpret_cast<unsigned short*>(smem_raw);           // x, n entries
+        unsigned char* pm = reinterpret_cast<unsigned char*>(xs + kMaxFusedN);  // per (piece, lane): activity of its 8 entries
+        using Smem = GemvSmem<G, BITS>;
+        static_assert(offsetof(Smem, red_z) >= kMaxFusedN * 2 + kMaxFusedN / 8,
+                      "the prologue's scratch must fit in the part of shared memory it borrows");
         const int nv = (n + 255) / 256;
-        const bool vec_ok = (reinterpret_cast<uintptr_t>(x) & 15) == 0;
-        uint4 xv[kMaxLoads];
-#pragma unroll
-        for (int j = 0; j < kMaxLoads; ++j) {
-            const int li = warp + j * kWarps;
-            const int k0 = li * 256 + lane * 8;
-            xv[j] = make_uint4(0u, 0u, 0u, 0u);
-            if (li < nv) {
-                if (vec_ok && k0 + 8 <= n) {
-                    xv[j] = __ldg(reinterpret_cast<const uint4*>(x + k0));
-                } else {
-                    unsigned short hv[8];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e)
-                        hv[e] = (k0 + e < n) ? __ldg(reinterpret_cast<const unsigned short*>(x) + k0 + e) : (unsigned short)0;
-                    xv[j].x = hv[0] | ((unsigned)hv[1] << 16);
-                    xv[j].y = hv[2] | ((unsigned)hv[3] << 16);
-                    xv[j].z = hv[4] | ((unsigned)hv[5] << 16);
-                    xv[j].w = hv[6] | ((unsigned)hv[7] << 16);
-                }
-            }
+        for (int i = nv + tid; i < kMaxFusedN / 256; i += kGemvThreads) sm.load_tot[i] = 0;
+        if ((reinterpret_cast<uintptr_t>(x) & 15) == 0) {
+            const int n16 = n >> 3;
+            for (int i = tid; i < n16; i += kGemvThreads) cp_async_16(smem_u32(xs + 8 * i), x + 8 * i);
+            for (int k = 8 * n16 + tid; k < n; k += kGemvThreads) xs[k] = __ldg(xb0 + k);
+        } else {
+            for (int k = tid; k < n; k += kGemvThreads) xs[k] = __ldg(xb0 + k);
         }
+        cp_async_commit();
         // the largest fp16 value not above t (any negative value if t < 0: everything but NaN is
         // active; +inf if t is NaN or +inf: nothing is)
         const __half thr_h = (thr != thr) ? __ushort_as_half((unsigned short)0x7c00)
                                           : (thr < 0.0f ? __float2half_rn(-1.0f) : __float2half_rd(thr));
         const __half2 thr_h2 = __half2half2(thr_h);
-        unsigned m8[kMaxLoads];   // activity of this lane's 8 entries of load j
-        int lane_excl[kMaxLoads]; // active entries of load j in the lanes below
-#pragma unroll
-        for (int j = 0; j < kMaxLoads; ++j) {
-            const int li = warp + j * kWarps;
-            m8[j] = 0;
-            lane_excl[j] = 0;
-            if (li < nv) {  // uniform across the warp
-                const int k0 = li * 256 + lane * 8;
-                const unsigned wds[4] = {xv[j].x, xv[j].y, xv[j].z, xv[j].w};
-#pragma unroll
-                for (int e2 = 0; e2 < 4; ++e2) {
-                    // |x| > t  <=>  |x| > (largest fp16 value <= t): two entries per compare, in fp16,
-                    // exact; the ordered compare is false for NaN
-                    const unsigned ab = wds[e2] & 0x7fff7fffu;
-                    const unsigned gt = __hgt2_mask(*reinterpret_cast<const __half2*>(&ab), thr_h2);
-                    m8[j] |= ((gt & 1u) | ((gt >> 15) & 2u)) << (2 * e2);
-                }
-                const int left = n - k0;  // entries of this lane that exist
-                if (left < 8) m8[j] &= (left <= 0) ? 0u : ((1u << left) - 1u);
-                const int c8 = __popc(m8[j]);
-                int incl = c8;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const int up = __shfl_up_sync(0xffffffffu, incl, o);
-                    if (lane >= o) incl += up;
-                }
-                lane_excl[j] = incl - c8;
-                if (lane == 31) sm.load_tot[li] = incl;
-            }
-        }
+        cp_async_wait<0>();
+        __syncthreads();
         SPQT_TRACE_EVENT(tid == 0, 3991);
+        // (1) per piece: the mask of each lane's eight entries and the number of active entries
+#pragma unroll 1
+        for (int li = warp; li < nv; li += kWarps) {
+            const int k0 = li * 256 + lane * 8;
+            const uint4 xv = *reinterpret_cast<const uint4*>(xs + k0);
+            const unsigned wds[4] = {xv.x, xv.y, xv.z, xv.w};
+            unsigned m8 = 0;
+#pragma unroll
+            for (int e2 = 0; e2 < 4; ++e2) {
+                // |x| > t  <=>  |x| > (largest fp16 value <= t): two entries per compare, in fp16,
+                // exact; the ordered compare is false for NaN
+                const unsigned ab = wds[e2] & 0x7fff7fffu;
+                const unsigned gt = __hgt2_mask(*reinterpret_cast<const __half2*>(&ab), thr_h2);
+                m8 |= (gt & (1u << (2 * e2))) | (gt & (0x20000u << (2 * e2))) >> 16;
+            }
+            const int left = n - k0;  // entries of this lane that exist (shared memory past n is stale)
+            if (left < 8) m8 &= (left <= 0) ? 0u : ((1u << left) - 1u);
+            pm[li * 32 + lane] = (unsigned char)m8;
+            const unsigned tot = __reduce_add_sync(0xffffffffu, (unsigned)__popc(m8));
+            if (lane == 0) sm.load_tot[li] = (int)tot;
+        }
         __syncthreads();
         SPQT_TRACE_EVENT(tid == 0, 3992);
-        // every warp: exclusive scan of the (at most 128) load totals, four per lane
-        int tot4[4], base4[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) tot4[q] = (lane * 4 + q < nv) ? sm.load_tot[lane * 4 + q] : 0;
-        const int s4 = tot4[0] + tot4[1] + tot4[2] + tot4[3];
-        int incl4 = s4;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int up = __shfl_up_sync(0xffffffffu, incl4, o);
-            if (lane >= o) incl4 += up;
+        // (2) every warp for itself: lane l holds the totals of pieces 4l..4l+3; sums over the pieces
+        // below a given one come from one warp reduction each
+        int tot4[4];
+        {
+            const int4 t4 = *reinterpret_cast<const int4*>(&sm.load_tot[lane * 4]);  // zero past nv (cleared below)
+            tot4[0] = t4.x; tot4[1] = t4.y; tot4[2] = t4.z; tot4[3] = t4.w;
         }
-        base4[0] = incl4 - s4;
-        base4[1] = base4[0] + tot4[0];
-        base4[2] = base4[1] + tot4[1];
-        base4[3] = base4[2] + tot4[2];
-        count = __shfl_sync(0xffffffffu, incl4, 31);
+        count = (int)__reduce_add_sync(0xffffffffu, (unsigned)(tot4[0] + tot4[1] + tot4[2] + tot4[3]));
         SPQT_TRACE_EVENT(tid == 0, 3993);
         pc.set_count(count);
-        pc.fill_table(sm.seg_table, tid);
-        __syncthreads();
         if (c == 0 && tid == 0) *count_out = count;
         // list positions this CTA will read: the union of its slices.  If that part fits in shared
         // memory the pipeline takes its column numbers from there (no round trip through global
-        // memory); idx_out is then written once, an even share of the list per CTA.
+        // memory); otherwise they go to idx_out and come back like a list collected by a separate launch.
         need_lo = count;
         int need_hi = 0;
         for (int r = pc.r_first; r <= pc.r_last; ++r) {
@@ -475,39 +478,52 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
             need_hi = max(need_hi, p1);
         }
         cols_local = (need_hi - need_lo) <= kFusedCols;
+        const unsigned need_len = (unsigned)max(need_hi - need_lo, 0);
+        const unsigned fc0 = smem_u32(&sm.fused_cols[0]);
         SPQT_TRACE_EVENT(tid == 0, 3994);
-        const int out_lo = pc.scaled((unsigned)c), out_hi = pc.scaled((unsigned)c + 1u);
+        // (3) the pieces that overlap [need_lo, need_hi): prefix sums over the lanes, then one
+        // predicated store per entry (a divergent branch per entry would cost far more than the store)
+#pragma unroll 1
+        for (int li = warp; li < nv; li += kWarps) {
+            unsigned below = 0;  // active entries of this lane's pieces that come before piece li
 #pragma unroll
-        for (int j = 0; j < kMaxLoads; ++j) {
-            const int li = warp + j * kWarps;
-            if (li < nv) {
-                // first list position of load li: component li & 3 of lane li >> 2
-                const int b0 = __shfl_sync(0xffffffffu, base4[0], li >> 2), b1 = __shfl_sync(0xffffffffu, base4[1], li >> 2);
-                const int b2 = __shfl_sync(0xffffffffu, base4[2], li >> 2), b3 = __shfl_sync(0xffffffffu, base4[3], li >> 2);
-                const int q = li & 3;
-                const int first = (q == 0 ? b0 : q == 1 ? b1 : q == 2 ? b2 : b3) + lane_excl[j];
-                const int last = first + __popc(m8[j]);
-                const bool mine = last > need_lo && first < need_hi, share = last > out_lo && first < out_hi;
-                if (mine || share) {
+            for (int q = 0; q < 4; ++q) below += (lane * 4 + q < li) ? (unsigned)tot4[q] : 0u;
+            const int base = (int)__reduce_add_sync(0xffffffffu, below);
+            const int q = li & 3;
+            const int tsel = q == 0 ? tot4[0] : q == 1 ? tot4[1] : q == 2 ? tot4[2] : tot4[3];
+            const int end = base + __shfl_sync(0xffffffffu, tsel, li >> 2);
+            if (end <= need_lo || base >= need_hi) continue;  // uniform across the warp
+            const unsigned m8 = pm[li * 32 + lane];
+            const int c8 = __popc(m8);
+            int incl = c8;
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) {
-                        if ((m8[j] >> e) & 1u) {
-                            const int pos = first + __popc(m8[j] & ((1u << e) - 1u));
-                            const int col = li * 256 + lane * 8 + e;
-                            const bool need = pos >= need_lo && pos < need_hi;
-                            if (need && cols_local) sm.fused_cols[pos - need_lo] = col;
-                            if ((need && !cols_local) || (pos >= out_lo && pos < out_hi)) idx_out[pos] = col;
-                        }
-                    }
+            for (int o = 1; o < 32; o <<= 1) {
+                const int up = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += up;
+            }
+            int pos = base + incl - c8;
+            const int col0 = li * 256 + lane * 8;
+            if (cols_local) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const unsigned on = (m8 >> e) & 1u, d = (unsigned)(pos - need_lo);
+                    st_shared_if(on & (d < need_len ? 1u : 0u), fc0 + 4u * d, col0 + e);
+                    pos += (int)on;
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const unsigned on = (m8 >> e) & 1u, d = (unsigned)(pos - need_lo);
+                    st_global_if(on & (d < need_len ? 1u : 0u), idx_out + pos, col0 + e);
+                    pos += (int)on;
                 }
             }
         }
+        SPQT_TRACE_EVENT(lane == 0, 3960 + warp);
         __syncthreads();  // the CTA's own writes (shared or global) are visible to its pipeline
         idx = idx_out;
     } else {
         pc.set_count(count);
-        pc.fill_table(sm.seg_table, tid);
-        __syncthreads();
     }
     SPQT_TRACE_EVENT(tid == 0, 4000);
 
@@ -516,9 +532,46 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
         // Two warps, one per hand-over buffer, so that the chains of dependent L2 round trips
         // (store, fence, counter, read back) of consecutive segments overlap.
         constexpr int RPL = G / 32;  // rows per lane
+        constexpr int kStride = G + 2;  // words per contributing CTA: G sums, the offset term, one of padding
         const int b = warp - kWriterWarp;
         bool ok = true;
+        if (FUSED && cols_local && pc.r_first == 0) {
+            // this CTA's slice of block-row 0 is its part of the index list the call returns
+            int p0, p1;
+            pc.slice(0, &p0, &p1);
+            for (int i = p0 + b * 32 + lane; i < p1; i += 64) idx_out[i] = sm.fused_cols[i - need_lo];
+        }
         for (int r = pc.r_first + b, sg = b; r <= pc.r_last; r += 2, sg += 2) {
+            int first, nslots;
+            pc.contributors(r, &first, &nslots);
+            const int mine = c - first;
+            unsigned long long* const row_words = words + (size_t)r * kTagSlots * kStride;
+            // While the workers are still computing: if at most three other CTAs contribute to this
+            // block-row, fetch their words now.  If all of them are there already, this CTA is the one
+            // that finishes the block-row, and nothing remains to be done across CTAs after its own sum.
+            constexpr int kSpec = kTagSlots - 1;
+            float ov[kSpec][RPL], oz[kSpec];
+            bool spec = false;
+            if (nslots > 1 && nslots <= kSpec + 1) {
+                unsigned tags = 1u;
+#pragma unroll
+                for (int j = 0; j < kSpec; ++j) {
+                    const bool in = j < nslots - 1;
+                    const unsigned long long* src = row_words + (size_t)(j + (j >= mine ? 1 : 0)) * kStride;
+#pragma unroll
+                    for (int i = 0; i < RPL; ++i) {
+                        const unsigned long long wv = in ? ld_word(src + lane * RPL + i) : kTagBit;
+                        ov[j][i] = __uint_as_float((unsigned)wv);
+                        tags &= (unsigned)(wv >> 32);
+                    }
+                    const unsigned long long wz = (in && lane == 0) ? ld_word(src + G) : kTagBit;
+                    oz[j] = __uint_as_float((unsigned)wz);
+                    tags &= (unsigned)(wz >> 32);
+                }
+                spec = __all_sync(0xffffffffu, tags != 0u);
+#pragma unroll
+                for (int j = 0; j < kSpec; ++j) oz[j] = __shfl_sync(0xffffffffu, oz[j], 0);
+            }
             ok = mbar_wait(&sm.red_full[b], (sg >> 1) & 1);
             if (!ok) break;
             float v[RPL];
@@ -533,32 +586,93 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(&sm.red_empty[b]);
-            int first, nslots;
-            pc.contributors(r, &first, &nslots);
             if (nslots == 1) {
-                // this CTA holds the whole block-row: no partial, no counter, no fence
+                // this CTA holds the whole block-row: nothing to combine
 #pragma unroll
                 for (int i = 0; i < RPL; ++i) y[(size_t)r * G + lane * RPL + i] = __float2half_rn(v[i] + zpart);
                 continue;
             }
-            const size_t pslot = (size_t)r * max_slots + (c - first);
+            float t[RPL], zsum = 0.0f;  // the block-row's sums, always accumulated in slot order
 #pragma unroll
-            for (int i = 0; i < RPL; ++i) __stcg(partials + pslot * G + lane * RPL + i, v[i]);
-            if (lane == 0) __stcg(zpartials + pslot, zpart);
-            __threadfence();
-            __syncwarp();
-            int prev = 0;
-            if (lane == 0) prev = atomicAdd(counters + r, 1);
-            prev = __shfl_sync(0xffffffffu, prev, 0);
-            if (prev == nslots - 1) {
-                // last contributor of this block-row: combine in slot order
+            for (int i = 0; i < RPL; ++i) t[i] = 0.0f;
+            if (spec) {
+#pragma unroll
+                for (int s = 0; s < kSpec + 1; ++s) {
+                    if (s < nslots) {
+                        const int j = s - (s > mine ? 1 : 0);  // position among the other CTAs
+#pragma unroll
+                        for (int i = 0; i < RPL; ++i) {
+                            float pv = v[i];
+#pragma unroll
+                            for (int jj = 0; jj < kSpec; ++jj) pv = (s != mine && j == jj) ? ov[jj][i] : pv;
+                            t[i] += pv;
+                        }
+                        float pz = zpart;
+#pragma unroll
+                        for (int jj = 0; jj < kSpec; ++jj) pz = (s != mine && j == jj) ? oz[jj] : pz;
+                        zsum += pz;
+                    }
+                }
+            } else if (nslots <= kSpec + 1) {
+                // publish this CTA's words (value and tag travel together: no fence), then count arrivals
+                unsigned long long* dst = row_words + (size_t)mine * kStride;
+#pragma unroll
+                for (int i = 0; i < RPL; ++i) st_word(dst + lane * RPL + i, kTagBit | __float_as_uint(v[i]));
+                if (lane == 0) st_word(dst + G, kTagBit | __float_as_uint(zpart));
+                int prev = 0;
+                if (lane == 0) prev = atomicAdd(counters + r, 1);
+                prev = __shfl_sync(0xffffffffu, prev, 0);
+                if (prev != nslots - 1) continue;
+                // last to arrive: every other CTA has issued its stores; wait (bounded) until their
+                // words are visible
+                float pv[kSpec + 1][RPL], pz[kSpec + 1];
+                unsigned long long t0 = 0;
+                for (unsigned it = 0;; ++it) {
+                    unsigned tags = 1u;
+#pragma unroll
+                    for (int j = 0; j < kSpec + 1; ++j) {
+                        const bool in = j < nslots && j != mine;
+                        const unsigned long long* src = row_words + (size_t)j * kStride;
+#pragma unroll
+                        for (int i = 0; i < RPL; ++i) {
+                            const unsigned long long wv = in ? ld_word(src + lane * RPL + i) : kTagBit;
+                            pv[j][i] = __uint_as_float((unsigned)wv);
+                            tags &= (unsigned)(wv >> 32);
+                        }
+                        const unsigned long long wz = (in && lane == 0) ? ld_word(src + G) : kTagBit;
+                        pz[j] = __uint_as_float((unsigned)wz);
+                        tags &= (unsigned)(wz >> 32);
+                    }
+                    if (__all_sync(0xffffffffu, tags != 0u)) break;
+                    if (it == 4) t0 = global_ns();
+                    if (it > 4 && global_ns() - t0 > kWaitNs) { ok = false; break; }
+                }
+                if (!ok) break;
+#pragma unroll
+                for (int j = 0; j < kSpec + 1; ++j) {
+                    const float z0 = __shfl_sync(0xffffffffu, pz[j], 0);
+                    if (j < nslots) {
+#pragma unroll
+                        for (int i = 0; i < RPL; ++i) t[i] += (j == mine) ? v[i] : pv[j][i];
+                        zsum += (j == mine) ? zpart : z0;
+                    }
+                }
+            } else {
+                // many contributors: plain fp32 partials in a region of their own, a fence, and the
+                // counter; the last to arrive reads eight slots at a time
+                const size_t pslot = (size_t)r * max_slots + mine;
+#pragma unroll
+                for (int i = 0; i < RPL; ++i) __stcg(partials + pslot * G + lane * RPL + i, v[i]);
+                if (lane == 0) __stcg(zpartials + pslot, zpart);
                 __threadfence();
-                float zsum = 0.0f;
-#pragma unroll
-                for (int i = 0; i < RPL; ++i) v[i] = 0.0f;
+                __syncwarp();
+                int prev = 0;
+                if (lane == 0) prev = atomicAdd(counters + r, 1);
+                prev = __shfl_sync(0xffffffffu, prev, 0);
+                if (prev != nslots - 1) continue;
+                __threadfence();
                 const float* p = partials + (size_t)r * max_slots * G + lane * RPL;
                 const float* zp = zpartials + (size_t)r * max_slots;
-                // eight slots' loads in flight at a time; the additions keep the slot order
                 for (int s0 = 0; s0 < nslots; s0 += 8) {
                     float pv[8][RPL], pz[8];
 #pragma unroll
@@ -570,14 +684,31 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
                     }
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
+                        if (s0 + j < nslots) {
 #pragma unroll
-                        for (int i = 0; i < RPL; ++i) v[i] += pv[j][i];
-                        zsum += pz[j];
+                            for (int i = 0; i < RPL; ++i) t[i] += pv[j][i];
+                            zsum += pz[j];
+                        }
                     }
                 }
+            }
 #pragma unroll
-                for (int i = 0; i < RPL; ++i) y[(size_t)r * G + lane * RPL + i] = __float2half_rn(v[i] + zsum);
-                if (lane == 0) counters[r] = 0;  // leave the workspace ready for the next call
+            for (int i = 0; i < RPL; ++i) y[(size_t)r * G + lane * RPL + i] = __float2half_rn(t[i] + zsum);
+            // leave the workspace ready for the next call: no tag may stay set
+            if (nslots <= kSpec + 1) {
+                for (int s = 0; s < nslots; ++s) {
+                    unsigned long long* dst = row_words + (size_t)s * kStride;
+#pragma unroll
+                    for (int i = 0; i < RPL; ++i) st_word(dst + lane * RPL + i, 0ull);
+                    if (lane == 0) st_word(dst + G, 0ull);
+                }
+            }
+            // The counter: after the last arrival nobody else touches it, so it is simply cleared.  On the
+            // early path the other CTAs' increments may still be under way: a reduction that takes away
+            // exactly what they add leaves zero whatever the order (and none of them can see "last").
+            if (lane == 0) {
+                if (spec) atomicAdd(counters + r, -(nslots - 1));
+                else counters[r] = 0;
             }
         }
         SPQT_TRACE_EVENT(lane == 0, 4002);
@@ -859,7 +990,8 @@ static spqt_status launch_gemv(const Format& f, const void* codes, const void* s
     const int slots = max_slots(f.R);
     int* counters = static_cast<int*>(workspace);
     int* status = counters + f.R;
-    float* partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + header_bytes(f.R));
+    unsigned long long* words = reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) + header_bytes(f.R));
+    float* partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + header_bytes(f.R) + tagged_bytes(f));
     float* zpartials = partials + (size_t)f.R * slots * G;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(P);
@@ -874,7 +1006,7 @@ static spqt_status launch_gemv(const Format& f, const void* codes, const void* s
     const cudaError_t err = cudaLaunchKernelEx(
         &cfg, kernel, static_cast<const uint8_t*>(codes), static_cast<const __half*>(scales),
         static_cast<const __half*>(zeros), f.R, f.n, static_cast<const __half*>(x), idx, count,
-        static_cast<__half*>(y), counters, status, partials, zpartials, slots,
+        static_cast<__half*>(y), counters, status, words, partials, zpartials, slots,
         fa.t, fa.idx_out, fa.count_out);
     count_launch();
     return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SPQT_OK : SPQT_ERR_CUDA;
