@@ -156,8 +156,8 @@ spqt_status spqt_dense_gemv(const void* codes, const void* scales, const void* z
  *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
  *     that device current) and keeps it; make that first call before any stream capture begins.
  *   - All calls on a device share the one array, which still holds the previous call's contents; the
- *     part that must start at zero (arrival counters, status word) is cleared on `stream` before the
- *     kernel.  Two calls that may overlap on the GPU (different streams, no ordering) race on it:
+ *     part that must start at zero (arrival counters, status word, the tagged words that carry partial
+ *     sums between thread blocks: up to about 0.9 MiB) is cleared on `stream` before the kernel.  Two calls that may overlap on the GPU (different streams, no ordering) race on it:
  *     order them, or use spqt_sparse_gemv with separate workspaces.
  *   - Because the status word is cleared per call, spqt_workspace_status does not apply here.
  * Other arguments, alignment rules and error codes are those of spqt_sparse_gemv.

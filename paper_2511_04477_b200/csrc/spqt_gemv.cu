@@ -90,6 +90,20 @@ __device__ __forceinline__ unsigned long long global_ns()
     return t;
 }
 
+// One non-blocking look at the phase with the given parity.
+__device__ __forceinline__ bool mbar_test(uint64_t* bar, unsigned parity)
+{
+    unsigned done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return done != 0;
+}
+
 // Bounded wait for the phase with the given parity; false when the bound
 // (wall time, so that a logic error can never hold the GPU) expires.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity)
@@ -546,31 +560,48 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
             pc.contributors(r, &first, &nslots);
             const int mine = c - first;
             unsigned long long* const row_words = words + (size_t)r * kTagSlots * kStride;
-            // While the workers are still computing: if at most three other CTAs contribute to this
-            // block-row, fetch their words now.  If all of them are there already, this CTA is the one
-            // that finishes the block-row, and nothing remains to be done across CTAs after its own sum.
+            // A block-row that is not the CTA's first is shared with CTAs that work on it first and are
+            // done long before this one.  While the workers are still computing, watch for their words
+            // (one word per CTA as a cheap hint, at a low rate).  Once all of them are there, this CTA
+            // is the one that finishes the block-row, and nothing remains to be done across CTAs after
+            // its own sum.  (On a CTA's first block-row all contributors finish at about the same time
+            // and watching would only delay the counter path.)
             constexpr int kSpec = kTagSlots - 1;
             float ov[kSpec][RPL], oz[kSpec];
             bool spec = false;
-            if (nslots > 1 && nslots <= kSpec + 1) {
-                unsigned tags = 1u;
+            if (sg > 0 && nslots > 1 && nslots <= kSpec + 1) {
+                unsigned long long t0 = 0;
+                for (unsigned it = 0;; ++it) {
+                    const unsigned long long hint =
+                        lane < nslots - 1 ? ld_word(row_words + (size_t)(lane + (lane >= mine ? 1 : 0)) * kStride + G) : kTagBit;
+                    if (__all_sync(0xffffffffu, (hint >> 32) != 0ull)) {
+                        unsigned tags = 1u;
 #pragma unroll
-                for (int j = 0; j < kSpec; ++j) {
-                    const bool in = j < nslots - 1;
-                    const unsigned long long* src = row_words + (size_t)(j + (j >= mine ? 1 : 0)) * kStride;
+                        for (int j = 0; j < kSpec; ++j) {
+                            const bool in = j < nslots - 1;
+                            const unsigned long long* src = row_words + (size_t)(j + (j >= mine ? 1 : 0)) * kStride;
 #pragma unroll
-                    for (int i = 0; i < RPL; ++i) {
-                        const unsigned long long wv = in ? ld_word(src + lane * RPL + i) : kTagBit;
-                        ov[j][i] = __uint_as_float((unsigned)wv);
-                        tags &= (unsigned)(wv >> 32);
+                            for (int i = 0; i < RPL; ++i) {
+                                const unsigned long long wv = in ? ld_word(src + lane * RPL + i) : kTagBit;
+                                ov[j][i] = __uint_as_float((unsigned)wv);
+                                tags &= (unsigned)(wv >> 32);
+                            }
+                            const unsigned long long wz = (in && lane == 0) ? ld_word(src + G) : kTagBit;
+                            oz[j] = __uint_as_float((unsigned)wz);
+                            tags &= (unsigned)(wz >> 32);
+                        }
+                        spec = __all_sync(0xffffffffu, tags != 0u);
+                        if (spec) break;
                     }
-                    const unsigned long long wz = (in && lane == 0) ? ld_word(src + G) : kTagBit;
-                    oz[j] = __uint_as_float((unsigned)wz);
-                    tags &= (unsigned)(wz >> 32);
+                    if (mbar_test(&sm.red_full[b], (sg >> 1) & 1)) break;  // own sums are ready: stop watching
+                    if (it == 64) t0 = global_ns();
+                    if (it > 64 && global_ns() - t0 > kWaitNs) break;
+                    __nanosleep(100);
                 }
-                spec = __all_sync(0xffffffffu, tags != 0u);
+                if (spec) {
 #pragma unroll
-                for (int j = 0; j < kSpec; ++j) oz[j] = __shfl_sync(0xffffffffu, oz[j], 0);
+                    for (int j = 0; j < kSpec; ++j) oz[j] = __shfl_sync(0xffffffffu, oz[j], 0);
+                }
             }
             ok = mbar_wait(&sm.red_full[b], (sg >> 1) & 1);
             if (!ok) break;
@@ -1110,9 +1141,9 @@ spqt_status spqt_sparse_gemv_static(const void* codes, const void* scales, const
         if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return SPQT_ERR_CUDA;
         scratch_addr[dev] = p;
     }
-    // The scratch keeps whatever the previous call (or an interrupted one) left: the arrival
-    // counters and the status word must start at zero.
-    if (cudaMemsetAsync(scratch_addr[dev], 0, header_bytes(f.R), static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    // The scratch keeps whatever the previous call (or an interrupted one, or one of another shape)
+    // left: the arrival counters, the status word and the tagged words must start at zero.
+    if (cudaMemsetAsync(scratch_addr[dev], 0, header_bytes(f.R) + tagged_bytes(f), static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return SPQT_ERR_CUDA;
     return gemv_entry<false>(codes, scales, zeros, m, n, bits, group, x, idx, count, y,
                              scratch_addr[dev], kStaticScratchBytes, stream);
