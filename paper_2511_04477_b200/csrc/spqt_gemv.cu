@@ -198,26 +198,35 @@ __device__ __forceinline__ void ffma2(unsigned long long& d, unsigned long long 
 }
 
 // acc[0..3] (eight fp32 sums, two per register) += the eight codes of one 32-bit word, each
-// times a*2^-56; m01, m23, m40, m12 hold the multipliers a*2^(93-4j) paired as (0,1) (2,3) (4,0) (1,2).
+// times a*2^-56.  Codes 0..3 are masked in place, codes 4..7 after a shift by 16, so that both
+// halves use the same two multiplier pairs m01 = a*(2^93, 2^89) and m23 = a*(2^85, 2^81).
 __device__ __forceinline__ void fma_word(unsigned long long* acc, unsigned w, unsigned long long m01,
-                                         unsigned long long m23, unsigned long long m40, unsigned long long m12)
+                                         unsigned long long m23)
 {
-    const unsigned v = w >> 20;
+    const unsigned v = w >> 16;
     ffma2(acc[0], pack2(__uint_as_float(w & 0x0000000fu), __uint_as_float(w & 0x000000f0u)), m01);
     ffma2(acc[1], pack2(__uint_as_float(w & 0x00000f00u), __uint_as_float(w & 0x0000f000u)), m23);
-    ffma2(acc[2], pack2(__uint_as_float(w & 0x000f0000u), __uint_as_float(v & 0x0000000fu)), m40);
-    ffma2(acc[3], pack2(__uint_as_float(v & 0x000000f0u), __uint_as_float(v & 0x00000f00u)), m12);
+    ffma2(acc[2], pack2(__uint_as_float(v & 0x0000000fu), __uint_as_float(v & 0x000000f0u)), m01);
+    ffma2(acc[3], pack2(__uint_as_float(v & 0x00000f00u), __uint_as_float(v & 0x0000f000u)), m23);
+}
+
+// d = a * b on both lanes
+__device__ __forceinline__ unsigned long long fmul2(unsigned long long a, unsigned long long b)
+{
+    unsigned long long d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
 }
 
 // acc (32 fp32 sums in 16 registers) += the 32 codes of a lane's 16 bytes, each times a (scaled by 2^-56).
 __device__ __forceinline__ void fma_block16(unsigned long long* acc, const uint4& w, float a)
 {
-    const float m0 = a * 0x1p93f, m1 = a * 0x1p89f, m2 = a * 0x1p85f, m3 = a * 0x1p81f, m4 = a * 0x1p77f;
-    const unsigned long long m01 = pack2(m0, m1), m23 = pack2(m2, m3), m40 = pack2(m4, m0), m12 = pack2(m1, m2);
-    fma_word(acc + 0, w.x, m01, m23, m40, m12);
-    fma_word(acc + 4, w.y, m01, m23, m40, m12);
-    fma_word(acc + 8, w.z, m01, m23, m40, m12);
-    fma_word(acc + 12, w.w, m01, m23, m40, m12);
+    const unsigned long long aa = pack2(a, a);
+    const unsigned long long m01 = fmul2(aa, pack2(0x1p93f, 0x1p89f)), m23 = fmul2(aa, pack2(0x1p85f, 0x1p81f));
+    fma_word(acc + 0, w.x, m01, m23);
+    fma_word(acc + 4, w.y, m01, m23);
+    fma_word(acc + 8, w.z, m01, m23);
+    fma_word(acc + 12, w.w, m01, m23);
 }
 
 // 3-bit codes: w2a, w2b are words of the 2-bit plane (byte i, field v = bits 2v..2v+1), w1 the word
@@ -786,7 +795,7 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
             if (cb.r != b_row) {
                 b_row = cb.r;
                 const size_t row_base = (size_t)b_row * (size_t)n;
-                b_par = (unsigned)(row_base & 1);
+                b_par = ODD_N ? (unsigned)(row_base & 1) : 0u;  // n even: every block-row starts on a word
                 b_codes = codes + row_base * B + (BITS == 4 ? 16 * h : 0);
                 b_scales = reinterpret_cast<const unsigned short*>(scales) + row_base;
                 b_zeros = reinterpret_cast<const unsigned short*>(zeros) + row_base;
@@ -874,7 +883,7 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
     for (int r = pc.r_first, sg = 0; r <= pc.r_last; ++r, ++sg) {
         int p0, p1;
         pc.slice(r, &p0, &p1);
-        const unsigned c_par = (unsigned)(((size_t)r * (size_t)n) & 1);
+        const unsigned c_par = ODD_N ? (unsigned)(((size_t)r * (size_t)n) & 1) : 0u;
         float zl = 0.0f;  // this lane's share of sum x_k * zero_rk
         for (int pos = p0 + warp * kChunk; pos < p1; pos += kWorkers * kChunk) {
             // ---- stage C of chunk qc: everything it needs is in commit groups that wait<D-1> covers
