@@ -164,6 +164,24 @@ __device__ __forceinline__ void st_word(unsigned long long* p, unsigned long lon
     asm volatile("st.relaxed.gpu.global.b64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 
+// shared-memory accesses by 32-bit shared address
+__device__ __forceinline__ unsigned lds_u32(unsigned addr)
+{
+    unsigned v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint4 lds_v4(unsigned addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sts_u32(unsigned addr, unsigned v)
+{
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+
 // stores under a predicate (never a branch)
 __device__ __forceinline__ void st_shared_if(unsigned cond, unsigned smem_dst, int v)
 {
@@ -760,19 +778,30 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
     }
 
     // ---------------------------------------------------------------- workers
+    // Everything the loop touches in shared memory is addressed with 32-bit shared addresses kept in
+    // registers (ring positions are byte offsets that wrap), and entries past the end of a slice are
+    // handled by clamping the entry number (they re-read the slice's last entry and get weight 0)
+    // rather than by branches: the loop is bound by instruction issue.
+    using Stage = typename GemvSmem<G, BITS>::Stage;
+    constexpr unsigned kStageBytes = (unsigned)sizeof(Stage);
+    constexpr unsigned kMetaOff = (unsigned)(kChunk * B);     // offset of Stage::meta
+    constexpr unsigned kColsBytes = kChunk * 4;               // one chunk of column numbers
+    static_assert(offsetof(Stage, meta) == kMetaOff, "stage layout");
     const int slot = lane / LPB, h = lane % LPB;
     const unsigned short* xb = reinterpret_cast<const unsigned short*>(x);
-
-    typename GemvSmem<G, BITS>::Stage* my_stage = &sm.stage[warp][0];
-    int (*my_cols)[kChunk] = sm.cols[warp];
+    const unsigned stage_base = smem_u32(&sm.stage[warp][0]);
+    const unsigned cols_base = smem_u32(&sm.cols[warp][0][0]);
+    const unsigned fused_base = smem_u32(&sm.fused_cols[0]) - 4u * (unsigned)need_lo;  // + 4 * list position
+    const bool use_list = !DENSE && !(FUSED && cols_local);  // column numbers come through stage A
 
     Cursor ca, cb;  // stage A / stage B cursors (the consume side walks the segments itself)
     ca.init(pc, warp);
     cb = ca;
-    // ring positions of the three stages: chunk number modulo the ring length, kept by wrap-around
-    // (the lengths are not powers of two)
-    unsigned qa2 = 0, qb1 = 0, qb2 = 0, qc1 = 0, qc2 = 0;  // ..1: modulo D (stages), ..2: modulo 2*D (columns)
-    auto wrap = [](unsigned& v, unsigned len) { v = (v + 1 == len) ? 0u : v + 1; };
+    // Ring positions (byte offsets) of the chunk stage C works on: rc_s in the ring of D stages, rc_c
+    // in the ring of 2*D chunks of column numbers, rb_c = D chunks further in that ring.  Stage B
+    // refills the stage slot C has just read and takes its columns from rb_c; stage A refills rc_c.
+    unsigned rc_s = 0, rc_c = 0, rb_c = D * kColsBytes;
+    auto wrap = [](unsigned& v, unsigned step, unsigned len) { v = (v + step == len) ? 0u : v + step; };
 
     // block-row constants of stage B, refreshed when its cursor enters a new block-row
     int b_row = -1;
@@ -781,16 +810,15 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
     const unsigned short* b_scales = nullptr; // scales / zeros of the block-row
     const unsigned short* b_zeros = nullptr;
 
-    // stage A: column numbers of the warp's chunk number qa
-    auto issue_a = [&]() {
-        if (!DENSE && !(FUSED && cols_local) && ca.valid(pc)) {
-            if (ca.pos + lane < ca.p1) cp_async_4(smem_u32(&my_cols[qa2][lane]), idx + ca.pos + lane);
+    // stage A: column numbers of the warp's next chunk
+    auto issue_a = [&](unsigned ring_c) {
+        if (use_list && ca.valid(pc)) {
+            if (ca.pos + lane < ca.p1) cp_async_4(cols_base + ring_c + 4u * lane, idx + ca.pos + lane);
             ca.advance(pc, warp);
-            wrap(qa2, 2 * D);
         }
     };
-    // stage B: code blocks and metadata words of chunk number qb (its columns have landed)
-    auto issue_b = [&]() {
+    // stage B: code blocks and metadata words of the next chunk (its column numbers have landed)
+    auto issue_b = [&](unsigned ring_s, unsigned ring_c) {
         if (cb.valid(pc)) {
             if (cb.r != b_row) {
                 b_row = cb.r;
@@ -800,19 +828,17 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
                 b_scales = reinterpret_cast<const unsigned short*>(scales) + row_base;
                 b_zeros = reinterpret_cast<const unsigned short*>(zeros) + row_base;
             }
-            const int valid = cb.p1 - cb.pos;  // entries of this chunk (>= kChunk when full)
-            const int* cols = (FUSED && cols_local) ? &sm.fused_cols[cb.pos - need_lo] : my_cols[qb2];
-            typename GemvSmem<G, BITS>::Stage& st = my_stage[qb1];
-            const unsigned dst = smem_u32(&st.codes[0]) + lane * 16;
+            const int vm1 = min(cb.p1 - cb.pos, kChunk) - 1;  // last entry of this chunk that exists
+            // address of the chunk's first column number (unused when DENSE)
+            const unsigned cols_addr = use_list ? cols_base + ring_c : fused_base + 4u * (unsigned)cb.pos;
+            const unsigned st_addr = stage_base + ring_s;
             if (BITS == 4) {
 #pragma unroll
                 for (int u = 0; u < SUBS; ++u) {
-                    const int e = u * SLOTS + slot;
-                    if (e < valid) {
-                        const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : (unsigned)cols[e];
-                        if (DENSE) cp_async_16(dst + u * 512, b_codes + (size_t)kk * B);
-                        else cp_async_16_l2_64(dst + u * 512, b_codes + (size_t)kk * B);
-                    }
+                    const int e = min(u * SLOTS + slot, vm1);
+                    const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : lds_u32(cols_addr + 4u * e);
+                    if (DENSE) cp_async_16(st_addr + lane * 16 + u * 512, b_codes + (size_t)kk * B);
+                    else cp_async_16_l2_64(st_addr + lane * 16 + u * 512, b_codes + (size_t)kk * B);
                 }
             } else {
                 // 3-bit blocks (48 or 24 bytes): the chunk's bytes in copies of CB bytes, lane after lane
@@ -820,24 +846,22 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
 #pragma unroll
                 for (int q = 0; q < NC; ++q) {
                     const int off = (q * 32 + lane) * CB;    // byte offset inside the chunk's stage
-                    const int e = off / B, part = off % B;
-                    if (e < valid) {
-                        const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : (unsigned)cols[e];
-                        const uint8_t* src = b_codes + (size_t)kk * B + part;
-                        const unsigned d = smem_u32(&st.codes[0]) + off;
-                        if (CB == 16) {
-                            if (DENSE) cp_async_16(d, src);
-                            else cp_async_16_l2_64(d, src);
-                        } else {
-                            cp_async_8(d, src);
-                        }
+                    const int e = min(off / B, vm1), part = off % B;
+                    const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : lds_u32(cols_addr + 4u * e);
+                    const uint8_t* src = b_codes + (size_t)kk * B + part;
+                    if (CB == 16) {
+                        if (DENSE) cp_async_16(st_addr + off, src);
+                        else cp_async_16_l2_64(st_addr + off, src);
+                    } else {
+                        cp_async_8(st_addr + off, src);
                     }
                 }
             }
-            if (lane < valid) {
+            {
                 // the aligned 4-byte word that holds each fp16 value (index rounded down to even)
-                const unsigned kk = DENSE ? (unsigned)(cb.pos + lane) : (unsigned)cols[lane];
-                const unsigned mdst = smem_u32(&st.meta[0][lane]);
+                const int e = min(lane, vm1);
+                const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : lds_u32(cols_addr + 4u * e);
+                const unsigned mdst = st_addr + kMetaOff + 4u * lane;
                 const int mo = (int)kk - (int)((kk ^ b_par) & 1u);  // may be -1 only when r*n is odd: still inside the array
                 if (!ODD_N || kk != (unsigned)(n - 1)) {
                     cp_async_4_ca(mdst, xb + (kk & ~1u));
@@ -845,29 +869,27 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
                     cp_async_4(mdst + 2 * kChunk * 4, b_zeros + mo);
                 } else {
                     // n odd: the word of the last column may reach past the end of an array; fetch directly
-                    st.meta[0][lane] = (unsigned)__ldg(xb + kk) << ((kk & 1u) * 16);
-                    st.meta[1][lane] = (unsigned)__ldg(b_scales + kk) << (((kk ^ b_par) & 1u) * 16);
-                    st.meta[2][lane] = (unsigned)__ldg(b_zeros + kk) << (((kk ^ b_par) & 1u) * 16);
+                    sts_u32(mdst, (unsigned)__ldg(xb + kk) << ((kk & 1u) * 16));
+                    sts_u32(mdst + kChunk * 4, (unsigned)__ldg(b_scales + kk) << (((kk ^ b_par) & 1u) * 16));
+                    sts_u32(mdst + 2 * kChunk * 4, (unsigned)__ldg(b_zeros + kk) << (((kk ^ b_par) & 1u) * 16));
                 }
             }
             cb.advance(pc, warp);
-            wrap(qb1, D);
-            wrap(qb2, 2 * D);
         }
     };
 
     // fill the pipeline: D chunks of columns, then D chunks of blocks (each needs its columns)
 #pragma unroll 1
     for (int s = 0; s < D; ++s) {
-        issue_a();
+        issue_a(s * kColsBytes);
         cp_async_commit();
     }
 #pragma unroll 1
     for (int s = 0; s < D; ++s) {
         cp_async_wait<D - 1>();
         __syncwarp();
-        issue_b();
-        issue_a();
+        issue_b(s * kStageBytes, s * kColsBytes);
+        issue_a((D + s) * kColsBytes);
         cp_async_commit();
     }
 
@@ -886,7 +908,7 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
         const unsigned c_par = ODD_N ? (unsigned)(((size_t)r * (size_t)n) & 1) : 0u;
         float zl = 0.0f;  // this lane's share of sum x_k * zero_rk
         for (int pos = p0 + warp * kChunk; pos < p1; pos += kWorkers * kChunk) {
-            // ---- stage C of chunk qc: everything it needs is in commit groups that wait<D-1> covers
+            // ---- stage C of the oldest chunk: everything it needs is in commit groups that wait<D-1> covers
 #ifdef SPQT_TRACE
             const long long tc0 = clock64();
 #endif
@@ -895,42 +917,43 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
 #ifdef SPQT_TRACE
             const long long tc1 = clock64();
 #endif
-            const typename GemvSmem<G, BITS>::Stage& st = my_stage[qc1];
-            const unsigned xw = st.meta[0][lane], sw = st.meta[1][lane], zw = st.meta[2][lane];
+            const unsigned st_addr = stage_base + rc_s;
+            const unsigned xw = lds_u32(st_addr + kMetaOff + 4u * lane);
+            const unsigned sw = lds_u32(st_addr + kMetaOff + 4u * lane + kChunk * 4);
+            const unsigned zw = lds_u32(st_addr + kMetaOff + 4u * lane + 2 * kChunk * 4);
+            const int e = min(lane, p1 - pos - 1);  // the entry whose metadata this lane holds
             unsigned kk;
-            if (DENSE) kk = (unsigned)(pos + lane);
-            else if (FUSED && cols_local) kk = (pos + lane < p1) ? (unsigned)sm.fused_cols[pos - need_lo + lane] : 0u;
-            else kk = (unsigned)my_cols[qc2][lane];
+            if (DENSE) kk = (unsigned)(pos + e);
+            else kk = lds_u32((use_list ? cols_base + rc_c : fused_base + 4u * (unsigned)pos) + 4u * e);
 #ifdef SPQT_TRACE
             const long long tc2 = clock64();
 #endif
-            float a = 0.0f;
-            if (pos + lane < p1) {
-                const unsigned xs = (kk & 1u) * 16, ms = ((kk ^ c_par) & 1u) * 16;
-                const float xf = __half2float(__ushort_as_half((unsigned short)(xw >> xs)));
-                const float sf = __half2float(__ushort_as_half((unsigned short)(sw >> ms)));
-                const float zf = __half2float(__ushort_as_half((unsigned short)(zw >> ms)));
-                a = xf * sf;  // exact; stays 0 past the end of the slice, where the code bytes are stale
-                zl = fmaf(xf, zf, zl);
-            }
+            const unsigned xs = (kk & 1u) * 16, ms = ((kk ^ c_par) & 1u) * 16;
+            const float xf = __half2float(__ushort_as_half((unsigned short)(xw >> xs)));
+            const float sf = __half2float(__ushort_as_half((unsigned short)(sw >> ms)));
+            const float zf = __half2float(__ushort_as_half((unsigned short)(zw >> ms)));
+            const float xin = (e == lane) ? xf : 0.0f;  // 0 past the end of the slice
+            const float a = xin * sf;                   // exact
+            zl = fmaf(xin, zf, zl);
 #pragma unroll
             for (int u = 0; u < SUBS; ++u) {
                 const float au = __shfl_sync(0xffffffffu, a, u * SLOTS + slot);
                 if (BITS == 4) {
-                    const uint4 wv = *reinterpret_cast<const uint4*>(&st.codes[0] + lane * 16 + u * 512);
+                    const uint4 wv = lds_v4(st_addr + lane * 16 + u * 512);
                     fma_block16(acc, wv, au);
                 } else {
                     // lane h of a block: words h and h+LPB of the 2-bit plane, word h of the 1-bit plane
-                    const unsigned* blk = reinterpret_cast<const unsigned*>(&st.codes[0] + (u * SLOTS + slot) * B);
-                    fma_block3(acc, blk[h], blk[h + LPB], blk[2 * LPB + h], au);
+                    const unsigned blk = st_addr + (u * SLOTS + slot) * B + 4u * h;
+                    fma_block3(acc, lds_u32(blk), lds_u32(blk + 4u * LPB), lds_u32(blk + 8u * LPB), au);
                 }
             }
             __syncwarp();  // every lane has read its part of the slots that B and A now refill
-            issue_b();
-            issue_a();
+            issue_b(rc_s, rb_c);
+            issue_a(rc_c);
             cp_async_commit();
-            wrap(qc1, D);
-            wrap(qc2, 2 * D);
+            wrap(rc_s, kStageBytes, D * kStageBytes);
+            wrap(rc_c, kColsBytes, 2 * D * kColsBytes);
+            wrap(rb_c, kColsBytes, 2 * D * kColsBytes);
 #ifdef SPQT_TRACE
             tr_wait += tc1 - tc0; tr_issue += 0; tr_math += clock64() - tc2; ++tr_n;
 #endif

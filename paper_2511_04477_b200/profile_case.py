@@ -1,7 +1,9 @@
 """Run one sparse and one dense GEMV a few times on a single packed matrix, with L2 flushed
 before every call -- a small, self-terminating case for `ncu` captures.
 
-    python -m paper_2511_04477_b200.profile_case M N SPARSITY [GROUP] [REPEATS]
+    python -m paper_2511_04477_b200.profile_case M N SPARSITY [GROUP] [REPEATS] [fused]
+
+With `fused` the sparse call is the one that collects the indices in the same launch.
 
 Weights are random-init on the device (values do not affect timing); x and the threshold come
 from the seeded input module.  Prints the active count and the workspace status word.
@@ -19,6 +21,7 @@ def main(argv):
     m, n, sp = int(argv[0]), int(argv[1]), float(argv[2])
     group = int(argv[3]) if len(argv) > 3 else 128
     repeats = int(argv[4]) if len(argv) > 4 else 3
+    fused = len(argv) > 5 and argv[5] == "fused"
     torch.manual_seed(0)
     W = (torch.randn(m, n, device="cuda", dtype=torch.float32) * 0.02).half()
     p = binding.spqt_pack(W, 4, group)
@@ -31,7 +34,10 @@ def main(argv):
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")   # larger than the 126 MB L2
     for _ in range(repeats):
         flush.zero_()
-        binding.spqt_sparse_gemv(p, xd, idx, cnt, ws)
+        if fused:
+            binding.spqt_sparsify_gemv(p, xd, t, ws, idx, cnt)
+        else:
+            binding.spqt_sparse_gemv(p, xd, idx, cnt, ws)
         flush.zero_()
         binding.spqt_dense_gemv(p, xd, ws)
     torch.cuda.synchronize()
