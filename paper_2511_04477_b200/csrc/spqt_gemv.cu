@@ -53,7 +53,7 @@ constexpr int kChunk = 32;               // list entries per chunk (one per lane
 constexpr int kDepth = 3;                // chunks in flight per warp
 constexpr unsigned long long kWaitNs = 1000000000ull;  // bound on every mbarrier wait: one second
 constexpr int kMaxFusedN = 32768;        // largest n whose index collection can run inside the GEMV
-constexpr int kFusedCols = 8192;         // list entries a CTA keeps in shared memory in that case
+constexpr int kFusedCols = 16384;        // list entries (16-bit column numbers) a CTA keeps in shared memory in that case
 
 static int g_tune_ctas = 0;  // 0 = one CTA per SM
 static int g_no_pdl = 0;     // 1 = plain stream-ordered launches
@@ -171,6 +171,12 @@ __device__ __forceinline__ unsigned lds_u32(unsigned addr)
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
     return v;
 }
+__device__ __forceinline__ unsigned lds_u16(unsigned addr)
+{
+    unsigned short v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr) : "memory");
+    return v;
+}
 __device__ __forceinline__ uint4 lds_v4(unsigned addr)
 {
     uint4 v;
@@ -183,9 +189,9 @@ __device__ __forceinline__ void sts_u32(unsigned addr, unsigned v)
 }
 
 // stores under a predicate (never a branch)
-__device__ __forceinline__ void st_shared_if(unsigned cond, unsigned smem_dst, int v)
+__device__ __forceinline__ void st_shared_u16_if(unsigned cond, unsigned smem_dst, int v)
 {
-    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %0, 0;\n\t@p st.shared.u32 [%1], %2;\n\t}" ::"r"(cond), "r"(smem_dst), "r"(v) : "memory");
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %0, 0;\n\t@p st.shared.u16 [%1], %2;\n\t}" ::"r"(cond), "r"(smem_dst), "h"((unsigned short)v) : "memory");
 }
 __device__ __forceinline__ void st_global_if(unsigned cond, int* dst, int v)
 {
@@ -379,7 +385,7 @@ struct GemvSmem {
     uint64_t red_full[2], red_empty[2];
     // fused index collection only
     alignas(16) int load_tot[kMaxFusedN / 256];  // active entries of every 256 entries of x
-    int fused_cols[kFusedCols];                   // the part of the index list this CTA reads, when it fits
+    unsigned short fused_cols[kFusedCols];       // the part of the index list this CTA reads, when it fits (n <= 32768)
 };
 
 // FUSED: the index collection runs in the kernel's prologue.  Every CTA copies x to shared memory and
@@ -548,7 +554,7 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                     const unsigned on = (m8 >> e) & 1u, d = (unsigned)(pos - need_lo);
-                    st_shared_if(on & (d < need_len ? 1u : 0u), fc0 + 4u * d, col0 + e);
+                    st_shared_u16_if(on & (d < need_len ? 1u : 0u), fc0 + 2u * d, col0 + e);
                     pos += (int)on;
                 }
             } else {
@@ -791,8 +797,15 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
     const unsigned short* xb = reinterpret_cast<const unsigned short*>(x);
     const unsigned stage_base = smem_u32(&sm.stage[warp][0]);
     const unsigned cols_base = smem_u32(&sm.cols[warp][0][0]);
-    const unsigned fused_base = smem_u32(&sm.fused_cols[0]) - 4u * (unsigned)need_lo;  // + 4 * list position
+    const unsigned fused_base = smem_u32(&sm.fused_cols[0]) - 2u * (unsigned)need_lo;  // + 2 * list position
     const bool use_list = !DENSE && !(FUSED && cols_local);  // column numbers come through stage A
+
+    // column number of entry e of a chunk: 32-bit entries in the stage-A ring, 16-bit ones in the list
+    // the fused prologue keeps
+    auto col_at = [&](unsigned chunk_addr, int e) -> unsigned {
+        if (!FUSED || use_list) return lds_u32(chunk_addr + 4u * e);
+        return lds_u16(chunk_addr + 2u * e);
+    };
 
     Cursor ca, cb;  // stage A / stage B cursors (the consume side walks the segments itself)
     ca.init(pc, warp);
@@ -830,13 +843,13 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
             }
             const int vm1 = min(cb.p1 - cb.pos, kChunk) - 1;  // last entry of this chunk that exists
             // address of the chunk's first column number (unused when DENSE)
-            const unsigned cols_addr = use_list ? cols_base + ring_c : fused_base + 4u * (unsigned)cb.pos;
+            const unsigned cols_addr = use_list ? cols_base + ring_c : fused_base + 2u * (unsigned)cb.pos;
             const unsigned st_addr = stage_base + ring_s;
             if (BITS == 4) {
 #pragma unroll
                 for (int u = 0; u < SUBS; ++u) {
                     const int e = min(u * SLOTS + slot, vm1);
-                    const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : lds_u32(cols_addr + 4u * e);
+                    const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : col_at(cols_addr, e);
                     if (DENSE) cp_async_16(st_addr + lane * 16 + u * 512, b_codes + (size_t)kk * B);
                     else cp_async_16_l2_64(st_addr + lane * 16 + u * 512, b_codes + (size_t)kk * B);
                 }
@@ -847,7 +860,7 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
                 for (int q = 0; q < NC; ++q) {
                     const int off = (q * 32 + lane) * CB;    // byte offset inside the chunk's stage
                     const int e = min(off / B, vm1), part = off % B;
-                    const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : lds_u32(cols_addr + 4u * e);
+                    const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : col_at(cols_addr, e);
                     const uint8_t* src = b_codes + (size_t)kk * B + part;
                     if (CB == 16) {
                         if (DENSE) cp_async_16(st_addr + off, src);
@@ -860,7 +873,7 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
             {
                 // the aligned 4-byte word that holds each fp16 value (index rounded down to even)
                 const int e = min(lane, vm1);
-                const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : lds_u32(cols_addr + 4u * e);
+                const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : col_at(cols_addr, e);
                 const unsigned mdst = st_addr + kMetaOff + 4u * lane;
                 const int mo = (int)kk - (int)((kk ^ b_par) & 1u);  // may be -1 only when r*n is odd: still inside the array
                 if (!ODD_N || kk != (unsigned)(n - 1)) {
@@ -924,7 +937,7 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
             const int e = min(lane, p1 - pos - 1);  // the entry whose metadata this lane holds
             unsigned kk;
             if (DENSE) kk = (unsigned)(pos + e);
-            else kk = lds_u32((use_list ? cols_base + rc_c : fused_base + 4u * (unsigned)pos) + 4u * e);
+            else kk = col_at(use_list ? cols_base + rc_c : fused_base + 2u * (unsigned)pos, e);
 #ifdef SPQT_TRACE
             const long long tc2 = clock64();
 #endif
