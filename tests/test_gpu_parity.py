@@ -208,6 +208,36 @@ def test_any_number_of_workers(splits):
     check_y(y, y_ref, bound, "S=%d" % splits)
 
 
+def test_one_workspace_serves_changing_shapes_and_worker_counts():
+    """The workspace cleans itself: calls of different shapes, formats and CTA counts (so that block-rows
+    have one, two to four and many contributing CTAs in turn) share one workspace; every result stays
+    right, and the second round repeats the first bit for bit."""
+    cases = [(1024, 2048, 4, 128, 0), (4096, 1024, 4, 128, 0), (28672, 512, 4, 128, 0), (512, 3000, 3, 64, 7),
+             (1024, 2048, 4, 64, 0), (2048, 1024, 3, 128, 40), (1024, 2048, 4, 128, 300)]
+    nbytes = max(binding.new_workspace(m, n, b, g).numel() for (m, n, b, g, _) in cases)
+    ws = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+    prepared, first_round = [], []
+    for ci, (m, n, bits, group, ctas) in enumerate(cases):
+        p = pack_on_gpu(inputs.weights(m, n, seed=700 + ci), bits, group)
+        prepared.append((p, packed_to_host(p), inputs.activations(n, seed=800 + ci)))
+    for rep in range(2):
+        for ci, (m, n, bits, group, ctas) in enumerate(cases):
+            p, (codes, s, z), x = prepared[ci]
+            t = inputs.threshold_for_sparsity(x, 0.5)
+            try:
+                binding.spqt_set_tuning(ctas)
+                y, idx, cnt = run_sparse(p, x, t, ws)
+            finally:
+                binding.spqt_set_tuning(0)
+            assert binding.spqt_workspace_status(ws, m, group) == 0
+            if rep == 0:
+                y_ref, bound = oracle.sparse_gemv(codes, s, z, m, n, x, idx, bits, group)
+                check_y(y, y_ref, bound, "case %d" % ci)
+                first_round.append(y.copy())
+            else:
+                assert np.array_equal(y.view(np.uint16), first_round[ci].view(np.uint16)), "case %d changed" % ci
+
+
 def test_heavy_tailed_outliers():
     m, n, bits, group = 1024, 8192, 4, 128
     W = inputs.weights(m, n, seed=51)
