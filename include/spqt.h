@@ -193,11 +193,22 @@ spqt_status spqt_sparse_linear_host(const void* codes, const void* scales, const
 spqt_status spqt_set_tuning(int gemv_ctas, int no_overlap);
 
 /*
+ * Checked mode (off by default; paper Sec. 4.2.3 assumes a well-formed index list and so does the
+ * normal path).  With on != 0, spqt_sparse_gemv and spqt_sparse_gemv_static first check the list on
+ * the device: *count in [0, n], every index in [0, n), and, for n <= 1048576, no index twice.  A bad
+ * list sets the workspace's status word to 2 and the product is computed with a count of 0 (y = 0)
+ * instead of reading wherever the indices point.  Costs two small extra launches per call; the check
+ * keeps its state per device, so checked calls on one device must not overlap.  Process-wide, not
+ * thread-safe.
+ */
+spqt_status spqt_set_debug(int on);
+
+/*
  * Reads the workspace's status word into *status_host (a host int) and waits for
  * the stream: 0 = every GEMV that used this workspace ran to completion;
- * non-zero = a bounded on-chip wait expired inside a GEMV kernel (which then
- * drained its copies and returned early, leaving y unspecified).  The word is
- * sticky until the caller zeroes the workspace again.
+ * 1 = a bounded wait expired inside a GEMV kernel (which then drained its copies
+ * and returned early, leaving y unspecified); 2 = checked mode found a bad index
+ * list.  The word is sticky until the caller zeroes the workspace again.
  */
 spqt_status spqt_workspace_status(const void* workspace, int m, int group, int* status_host, void* stream);
 

@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libspqt.so")
 EXPORTS = (
     "spqt_status_string", "spqt_version", "spqt_packed_sizes", "spqt_pack", "spqt_unpack",
     "spqt_sparsify", "spqt_sparse_gemv", "spqt_sparse_gemv_static", "spqt_sparsify_gemv", "spqt_dense_gemv", "spqt_sparse_linear_host",
-    "spqt_set_tuning", "spqt_workspace_status", "spqt_launch_count",
+    "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_launch_count",
 )
 
 _lib = None
@@ -58,11 +58,12 @@ def lib() -> ctypes.CDLL:
         L.spqt_sparse_linear_host.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, vp,
                                               vp, vp, vp, vp, vp, sz, vp]
         L.spqt_set_tuning.argtypes = [i32, i32]
+        L.spqt_set_debug.argtypes = [i32]
         L.spqt_workspace_status.argtypes = [vp, i32, i32, ctypes.POINTER(i32), vp]
         L.spqt_launch_count.restype = ctypes.c_ulonglong
         for name in ("spqt_packed_sizes", "spqt_pack", "spqt_unpack", "spqt_sparsify",
                      "spqt_sparse_gemv", "spqt_dense_gemv", "spqt_sparse_linear_host", "spqt_set_tuning",
-                     "spqt_workspace_status"):
+                     "spqt_set_debug", "spqt_workspace_status"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -254,6 +255,11 @@ def spqt_sparse_linear_host(h: HostLinear, t: float, stream=None) -> torch.Tenso
         h.count.data_ptr(), h.y_dev.data_ptr(), h.workspace.data_ptr(), h.workspace.numel(),
         _stream(stream)), "spqt_sparse_linear_host")
     return h.y_host
+
+
+def spqt_set_debug(on: bool) -> None:
+    """Checked mode: validate idx/count on the device before every sparse GEMV (off by default)."""
+    _ok(lib().spqt_set_debug(1 if on else 0), "spqt_set_debug")
 
 
 def spqt_set_tuning(gemv_ctas: int = 0, no_overlap: int = 0) -> None:

@@ -1030,6 +1030,67 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
 
 // ---------------------------------------------------------------- host side
 
+// ---------------------------------------------------------------- checked mode
+// spqt_set_debug(1): before a sparse GEMV the index list is checked on the device (count in
+// [0, n], every index in [0, n), no index twice for n up to kDebugBits).  A bad list sets the
+// workspace's status word to 2 and the GEMV then runs with a count of 0 (y = 0) instead of reading
+// wherever the indices point.  Two small extra launches per call; state is per device, not per stream.
+constexpr int kDebugBits = 1 << 20;
+static __device__ unsigned g_debug_bitmap[kDebugBits / 32];  // all zero between calls
+static __device__ int g_debug_count;                         // the count the GEMV is given
+static int g_debug = 0;
+
+__global__ void debug_mark_kernel(const int32_t* __restrict__ idx, const int32_t* __restrict__ count, int n,
+                                  int* __restrict__ status)
+{
+    const int c = *count;
+    bool bad = (c < 0 || c > n) && blockIdx.x == 0 && threadIdx.x == 0;
+    const int lim = c < 0 ? 0 : (c > n ? n : c);  // idx holds n entries at most
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < lim; i += gridDim.x * blockDim.x) {
+        const int k = idx[i];
+        if (k < 0 || k >= n) {
+            bad = true;
+        } else if (n <= kDebugBits) {
+            const unsigned bit = 1u << (k & 31);
+            if (atomicOr(&g_debug_bitmap[k >> 5], bit) & bit) bad = true;  // seen before
+        }
+    }
+    if (bad) atomicExch(status, 2);
+}
+
+__global__ void debug_clear_kernel(const int32_t* __restrict__ idx, const int32_t* __restrict__ count, int n,
+                                   const int* __restrict__ status)
+{
+    const int c = *count;
+    const int lim = c < 0 ? 0 : (c > n ? n : c);
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < lim; i += gridDim.x * blockDim.x) {
+        const int k = idx[i];
+        if (k >= 0 && k < n && n <= kDebugBits) g_debug_bitmap[k >> 5] = 0u;
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) g_debug_count = (*status != 0) ? 0 : c;
+}
+
+// Launches the two kernels; returns the device address of the count the GEMV must use.
+static spqt_status debug_check(const int32_t* idx, const int32_t* count, int n, int* status, cudaStream_t s,
+                               const int32_t** checked_count)
+{
+    static int* count_addr[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPQT_ERR_CUDA;
+    if (count_addr[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_debug_count) != cudaSuccess || p == nullptr) return SPQT_ERR_CUDA;
+        count_addr[dev] = static_cast<int*>(p);
+    }
+    const int blocks = n < 256 * 64 ? (n + 255) / 256 : 64;
+    debug_mark_kernel<<<blocks, 256, 0, s>>>(idx, count, n, status);
+    debug_clear_kernel<<<blocks, 256, 0, s>>>(idx, count, n, status);
+    if (cudaGetLastError() != cudaSuccess) return SPQT_ERR_CUDA;
+    count_launch(2);
+    *checked_count = count_addr[dev];
+    return SPQT_OK;
+}
+
 struct FusedArgs {
     float t;
     int32_t* idx_out;
@@ -1107,6 +1168,10 @@ static spqt_status gemv_entry(const void* codes, const void* scales, const void*
     if (ws_bytes < workspace_bytes(f)) return SPQT_ERR_WORKSPACE;
     if ((long long)f.R * kMaxCtas >= (1ll << 31)) return SPQT_ERR_UNSUPPORTED;  // the work map is 32-bit
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (!DENSE && !FUSED && g_debug) {
+        st = debug_check(idx, count, n, static_cast<int*>(workspace) + f.R, s, &count);
+        if (st != SPQT_OK) return st;
+    }
     const bool odd = (n & 1) != 0;
 #define SPQT_DISPATCH(GG, BB)                                                                                      \
     return odd ? launch_gemv<GG, BB, DENSE, true, FUSED>(f, codes, scales, zeros, x, idx, count, y, workspace, s, fa) \
@@ -1192,6 +1257,12 @@ spqt_status spqt_sparse_gemv_static(const void* codes, const void* scales, const
         return SPQT_ERR_CUDA;
     return gemv_entry<false>(codes, scales, zeros, m, n, bits, group, x, idx, count, y,
                              scratch_addr[dev], kStaticScratchBytes, stream);
+}
+
+spqt_status spqt_set_debug(int on)
+{
+    spqt::g_debug = on ? 1 : 0;
+    return SPQT_OK;
 }
 
 spqt_status spqt_set_tuning(int gemv_ctas, int reserved)

@@ -238,6 +238,47 @@ def test_one_workspace_serves_changing_shapes_and_worker_counts():
                 assert np.array_equal(y.view(np.uint16), first_round[ci].view(np.uint16)), "case %d changed" % ci
 
 
+def test_checked_mode_refuses_bad_index_lists():
+    """Checked mode: a well-formed list gives the same bits as the normal path and status 0; a list with an
+    index out of range, a negative index, a repeated index or a count outside [0, n] gives status 2 and
+    y = 0, and nothing is read through the bad indices."""
+    m, n, bits, group = 256, 1000, 4, 128
+    p = pack_on_gpu(inputs.weights(m, n, seed=91), bits, group)
+    x = inputs.activations(n, seed=92)
+    xd = dev(x)
+    idx, cnt = binding.spqt_sparsify(xd, inputs.threshold_for_sparsity(x, 0.5))
+    torch.cuda.synchronize()
+    c = int(cnt.item())
+    y_plain = binding.spqt_sparse_gemv(p, xd, idx, cnt, binding.new_workspace(m, n, bits, group)).cpu().numpy()
+
+    def run_checked(idx_t, count_value):
+        ws = binding.new_workspace(m, n, bits, group)
+        cnt_t = torch.tensor([count_value], dtype=torch.int32, device="cuda")
+        try:
+            binding.spqt_set_debug(True)
+            y = binding.spqt_sparse_gemv(p, xd, idx_t, cnt_t, ws)
+        finally:
+            binding.spqt_set_debug(False)
+        return y.cpu().numpy(), binding.spqt_workspace_status(ws, m, group)
+
+    y, status = run_checked(idx, c)
+    assert status == 0 and np.array_equal(y.view(np.uint16), y_plain.view(np.uint16))
+    bad = {}
+    t = idx.clone(); t[3] = n; bad["index == n"] = (t, c)
+    t = idx.clone(); t[c - 1] = 2 ** 31 - 1; bad["huge index"] = (t, c)
+    t = idx.clone(); t[0] = -5; bad["negative index"] = (t, c)
+    t = idx.clone(); t[7] = t[8]; bad["repeated index"] = (t, c)
+    bad["count > n"] = (idx, n + 1)
+    bad["count < 0"] = (idx, -1)
+    for what, (idx_t, count_value) in bad.items():
+        y, status = run_checked(idx_t, count_value)
+        assert status == 2, what
+        assert not y.any(), what
+    # and the next well-formed call on a fresh workspace is untouched by all that
+    y, status = run_checked(idx, c)
+    assert status == 0 and np.array_equal(y.view(np.uint16), y_plain.view(np.uint16))
+
+
 def test_heavy_tailed_outliers():
     m, n, bits, group = 1024, 8192, 4, 128
     W = inputs.weights(m, n, seed=51)
