@@ -17,8 +17,9 @@ visited round-robin so that weights really come from HBM.
 value  = effective GB/s over the bytes the method needs
          (sum over GEMVs of count*R*(B+4) + 2n + 4count + 4 + 2m, plus 2n + 4count + 4
          per index collection), whole job, inputs resident in HBM.
-e2e    = the same metric through spqt_sparse_linear_host: x from pinned host memory,
-         y back to pinned host memory, copies and the final wait inside the timed region.
+e2e    = the same metric through spqt_sparse_linear_host: x copied from pinned host memory,
+         y written into pinned host memory by the kernel, the copy and the final wait of every
+         call inside the timed region.
 roofline.achieved = algorithmic bytes per sparse-GEMV launch / its mean duration
          (device events over a region that launches only the GEMVs of the same steps).
 

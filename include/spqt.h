@@ -170,9 +170,11 @@ spqt_status spqt_sparse_gemv_static(const void* codes, const void* scales, const
 /*
  * One decode-time linear layer from HOST activations (paper Sec. 3.2: hidden
  * state -> index collection with the layer's threshold -> sparse GEMV):
- * copies x_host (fp16[n]) to x_dev, runs spqt_sparsify and spqt_sparse_gemv,
- * copies y (fp16[m]) to y_host and waits for the stream.  x_host / y_host
- * should be pinned for the copies to be asynchronous; x_dev (fp16[n]), idx_dev
+ * copies x_host (fp16[n]) to x_dev, runs spqt_sparsify_gemv (same results as
+ * spqt_sparsify followed by spqt_sparse_gemv), copies y (fp16[m]) to y_host and
+ * waits for the stream.  x_host / y_host
+ * should be pinned for the copies to be asynchronous (the kernel then writes y
+ * straight into y_host and the copy back is skipped); x_dev (fp16[n]), idx_dev
  * (int32[n]), count_dev (int32[1]) and y_dev (fp16[m]) are caller-provided
  * device staging buffers.  This is the only entry point that synchronises.
  */

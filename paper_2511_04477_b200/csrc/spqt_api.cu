@@ -70,12 +70,21 @@ spqt_status spqt_sparse_linear_host(const void* codes, const void* scales, const
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (cudaMemcpyAsync(x_dev, x_host, (size_t)n * 2, cudaMemcpyHostToDevice, s) != cudaSuccess)
         return SPQT_ERR_CUDA;
-    st = spqt_sparsify(x_dev, n, t, idx_dev, count_dev, stream);
+    // If y_host is pinned memory the device can address, the kernel writes y there itself (posted
+    // writes over the bus) and the copy back, with its start-up latency, is not needed.
+    void* y_target = y_dev;
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, y_host) == cudaSuccess && attr.type == cudaMemoryTypeHost &&
+        attr.devicePointer != nullptr)
+        y_target = attr.devicePointer;
+    else
+        (void)cudaGetLastError();  // pageable memory is not an error here
+    // index collection and product in one launch (two for very long x: the call decides)
+    st = spqt_sparsify_gemv(codes, scales, zeros, m, n, bits, group, x_dev, t, idx_dev, count_dev,
+                            y_target, workspace, workspace_bytes, stream);
     if (st != SPQT_OK) return st;
-    st = spqt_sparse_gemv(codes, scales, zeros, m, n, bits, group, x_dev, idx_dev, count_dev,
-                          y_dev, workspace, workspace_bytes, stream);
-    if (st != SPQT_OK) return st;
-    if (cudaMemcpyAsync(y_host, y_dev, (size_t)m * 2, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+    if (y_target == y_dev &&
+        cudaMemcpyAsync(y_host, y_dev, (size_t)m * 2, cudaMemcpyDeviceToHost, s) != cudaSuccess)
         return SPQT_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return SPQT_ERR_CUDA;
     return SPQT_OK;
