@@ -288,7 +288,7 @@ __device__ __forceinline__ void halve(const float* in, float* out, int lane, int
 
 // floor(v / d) for any 32-bit v from the multiplier m = floor((2^32 - 1) / d): the high product is
 // the quotient or one less (the multiplier falls short of 2^32 / d by at most 1), one compare fixes it.
-__device__ __forceinline__ unsigned magic_of(unsigned d) { return 0xffffffffu / d; }
+__host__ __device__ __forceinline__ unsigned magic_of(unsigned d) { return 0xffffffffu / d; }
 __device__ __forceinline__ unsigned magic_div(unsigned v, unsigned d, unsigned m)
 {
     const unsigned q = __umulhi(v, m);
@@ -297,16 +297,15 @@ __device__ __forceinline__ unsigned magic_div(unsigned v, unsigned d, unsigned m
 
 struct Piece {
     int R, P, c, count, r_first, r_last;
-    unsigned mP, mR;  // multipliers of magic_div for P and R: one real division each per thread,
-                      // issued while the first loads are in flight
+    unsigned mP, mR;  // multipliers of magic_div for P and R, computed by the host
     unsigned qc, rc;  // count = qc * P + rc: keeps the slice arithmetic in 32 bits (the host checks R * P < 2^31)
 
     // the block-rows of the piece do not depend on the count: computed while the count is being fetched
-    __device__ __forceinline__ void init_rows(int R_, int P_, int c_)
+    __device__ __forceinline__ void init_rows(int R_, int P_, int c_, unsigned mP_, unsigned mR_)
     {
         R = R_; P = P_; c = c_;
-        mP = magic_of((unsigned)P);
-        mR = magic_of((unsigned)R);
+        mP = mP_;
+        mR = mR_;
         const unsigned lo = (unsigned)c * (unsigned)R, hi = lo + (unsigned)R;
         r_first = (int)magic_div(lo, (unsigned)P, mP);
         r_last = (int)magic_div(hi - 1u, (unsigned)P, mP);
@@ -402,7 +401,7 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
                  const int32_t* count_ptr, __half* __restrict__ y,
                  int* __restrict__ counters, int* __restrict__ status,
                  unsigned long long* __restrict__ words, float* __restrict__ partials,
-                 float* __restrict__ zpartials, int max_slots,
+                 float* __restrict__ zpartials, int max_slots, unsigned magic_p, unsigned magic_r,
                  float thr, int32_t* idx_out, int32_t* count_out)
 {
     constexpr int B = G * BITS / 8;
@@ -444,61 +443,75 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
     int count = 0;
     if (!FUSED) count = DENSE ? n : *count_ptr;  // in flight while the row range is worked out
     Piece pc;
-    pc.init_rows(R, P, c);
+    pc.init_rows(R, P, c, magic_p, magic_r);
     const int32_t* idx = idx_in;
     const unsigned short* xb0 = reinterpret_cast<const unsigned short*>(x);
     int need_lo = 0;          // FUSED: first list position held in sm.fused_cols
     bool cols_local = false;  // FUSED: the pipeline reads its column numbers from sm.fused_cols
     if (FUSED) {
         // Three short loops over the 256-entry pieces of x (piece li belongs to warp li % kWarps, lane l
-        // holds entries 8l..8l+7), with x and the per-lane results kept in shared memory that the
-        // pipeline only uses afterwards: (1) activity mask of the lane's entries and warp prefix sums,
-        // (2) every warp scans the piece totals for itself, (3) the pieces that overlap the list
-        // positions this CTA needs are expanded into column numbers.
+        // holds entries 8l..8l+7): (1) activity mask of the lane's entries and the piece totals, four
+        // pieces per warp and round so that their loads share one round trip, (2) every warp sums the
+        // totals below its own pieces, (3) the pieces that overlap the list positions this CTA needs are
+        // expanded into column numbers.  The per-lane masks wait in shared memory that the pipeline
+        // only uses afterwards.
         constexpr int kWarps = kGemvThreads / 32;
-        unsigned short* xs = reinterpret_cast<unsigned short*>(smem_raw);           // x, n entries
-        unsigned char* pm = reinterpret_cast<unsigned char*>(xs + kMaxFusedN);  // per (piece, lane): activity of its 8 entries
+        constexpr int kPiecesPerRound = 4;
+        unsigned char* pm = reinterpret_cast<unsigned char*>(smem_raw);  // per (piece, lane): activity of its 8 entries
         using Smem = GemvSmem<G, BITS>;
-        static_assert(offsetof(Smem, red_z) >= kMaxFusedN * 2 + kMaxFusedN / 8,
+        static_assert(offsetof(Smem, red_z) >= kMaxFusedN / 8,
                       "the prologue's scratch must fit in the part of shared memory it borrows");
         const int nv = (n + 255) / 256;
         for (int i = nv + tid; i < kMaxFusedN / 256; i += kGemvThreads) sm.load_tot[i] = 0;
-        if ((reinterpret_cast<uintptr_t>(x) & 15) == 0) {
-            const int n16 = n >> 3;
-            for (int i = tid; i < n16; i += kGemvThreads) cp_async_16(smem_u32(xs + 8 * i), x + 8 * i);
-            for (int k = 8 * n16 + tid; k < n; k += kGemvThreads) xs[k] = __ldg(xb0 + k);
-        } else {
-            for (int k = tid; k < n; k += kGemvThreads) xs[k] = __ldg(xb0 + k);
-        }
-        cp_async_commit();
+        const bool vec_ok = (reinterpret_cast<uintptr_t>(x) & 15) == 0;
         // the largest fp16 value not above t (any negative value if t < 0: everything but NaN is
         // active; +inf if t is NaN or +inf: nothing is)
         const __half thr_h = (thr != thr) ? __ushort_as_half((unsigned short)0x7c00)
                                           : (thr < 0.0f ? __float2half_rn(-1.0f) : __float2half_rd(thr));
         const __half2 thr_h2 = __half2half2(thr_h);
-        cp_async_wait<0>();
-        __syncthreads();
         SPQT_TRACE_EVENT(tid == 0, 3991);
-        // (1) per piece: the mask of each lane's eight entries and the number of active entries
 #pragma unroll 1
-        for (int li = warp; li < nv; li += kWarps) {
-            const int k0 = li * 256 + lane * 8;
-            const uint4 xv = *reinterpret_cast<const uint4*>(xs + k0);
-            const unsigned wds[4] = {xv.x, xv.y, xv.z, xv.w};
-            unsigned m8 = 0;
+        for (int l0 = warp; l0 < nv; l0 += kPiecesPerRound * kWarps) {
+            uint4 xv[kPiecesPerRound];
 #pragma unroll
-            for (int e2 = 0; e2 < 4; ++e2) {
-                // |x| > t  <=>  |x| > (largest fp16 value <= t): two entries per compare, in fp16,
-                // exact; the ordered compare is false for NaN
-                const unsigned ab = wds[e2] & 0x7fff7fffu;
-                const unsigned gt = __hgt2_mask(*reinterpret_cast<const __half2*>(&ab), thr_h2);
-                m8 |= (gt & (1u << (2 * e2))) | (gt & (0x20000u << (2 * e2))) >> 16;
+            for (int j = 0; j < kPiecesPerRound; ++j) {
+                const int li = l0 + j * kWarps, k0 = li * 256 + lane * 8;
+                xv[j] = make_uint4(0u, 0u, 0u, 0u);
+                if (li < nv) {  // uniform across the warp
+                    if (vec_ok && k0 + 8 <= n) {
+                        xv[j] = __ldg(reinterpret_cast<const uint4*>(x + k0));
+                    } else {
+                        unsigned short hv[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) hv[e] = (k0 + e < n) ? __ldg(xb0 + k0 + e) : (unsigned short)0;
+                        xv[j].x = hv[0] | ((unsigned)hv[1] << 16);
+                        xv[j].y = hv[2] | ((unsigned)hv[3] << 16);
+                        xv[j].z = hv[4] | ((unsigned)hv[5] << 16);
+                        xv[j].w = hv[6] | ((unsigned)hv[7] << 16);
+                    }
+                }
             }
-            const int left = n - k0;  // entries of this lane that exist (shared memory past n is stale)
-            if (left < 8) m8 &= (left <= 0) ? 0u : ((1u << left) - 1u);
-            pm[li * 32 + lane] = (unsigned char)m8;
-            const unsigned tot = __reduce_add_sync(0xffffffffu, (unsigned)__popc(m8));
-            if (lane == 0) sm.load_tot[li] = (int)tot;
+#pragma unroll
+            for (int j = 0; j < kPiecesPerRound; ++j) {
+                const int li = l0 + j * kWarps, k0 = li * 256 + lane * 8;
+                if (li < nv) {
+                    const unsigned wds[4] = {xv[j].x, xv[j].y, xv[j].z, xv[j].w};
+                    unsigned m8 = 0;
+#pragma unroll
+                    for (int e2 = 0; e2 < 4; ++e2) {
+                        // |x| > t  <=>  |x| > (largest fp16 value <= t): two entries per compare, in fp16,
+                        // exact; the ordered compare is false for NaN
+                        const unsigned ab = wds[e2] & 0x7fff7fffu;
+                        const unsigned gt = __hgt2_mask(*reinterpret_cast<const __half2*>(&ab), thr_h2);
+                        m8 |= (gt & (1u << (2 * e2))) | (gt & (0x20000u << (2 * e2))) >> 16;
+                    }
+                    const int left = n - k0;  // entries of this lane that exist
+                    if (left < 8) m8 &= (left <= 0) ? 0u : ((1u << left) - 1u);
+                    pm[li * 32 + lane] = (unsigned char)m8;
+                    const unsigned tot = __reduce_add_sync(0xffffffffu, (unsigned)__popc(m8));
+                    if (lane == 0) sm.load_tot[li] = (int)tot;
+                }
+            }
         }
         __syncthreads();
         SPQT_TRACE_EVENT(tid == 0, 3992);
@@ -516,14 +529,11 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
         // list positions this CTA will read: the union of its slices.  If that part fits in shared
         // memory the pipeline takes its column numbers from there (no round trip through global
         // memory); otherwise they go to idx_out and come back like a list collected by a separate launch.
-        need_lo = count;
-        int need_hi = 0;
-        for (int r = pc.r_first; r <= pc.r_last; ++r) {
-            int p0, p1;
-            pc.slice(r, &p0, &p1);
-            need_lo = min(need_lo, p0);
-            need_hi = max(need_hi, p1);
-        }
+        // (A piece that spans several block-rows ends the first one and begins the last one: its slices
+        // cover the whole list between them.)
+        need_lo = 0;
+        int need_hi = count;
+        if (pc.r_first == pc.r_last) pc.slice(pc.r_first, &need_lo, &need_hi);
         cols_local = (need_hi - need_lo) <= kFusedCols;
         const unsigned need_len = (unsigned)max(need_hi - need_lo, 0);
         const unsigned fc0 = smem_u32(&sm.fused_cols[0]);
@@ -1144,7 +1154,7 @@ static spqt_status launch_gemv(const Format& f, const void* codes, const void* s
         &cfg, kernel, static_cast<const uint8_t*>(codes), static_cast<const __half*>(scales),
         static_cast<const __half*>(zeros), f.R, f.n, static_cast<const __half*>(x), idx, count,
         static_cast<__half*>(y), counters, status, words, partials, zpartials, slots,
-        fa.t, fa.idx_out, fa.count_out);
+        magic_of((unsigned)P), magic_of((unsigned)f.R), fa.t, fa.idx_out, fa.count_out);
     count_launch();
     return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SPQT_OK : SPQT_ERR_CUDA;
 }
