@@ -186,9 +186,11 @@ spqt_status spqt_sparse_linear_host(const void* codes, const void* scales, const
 
 /*
  * Tuning aid: number of CTAs of the GEMV grid (0 restores the built-in rule, one
- * persistent CTA per SM; values above 512 are clamped).  `no_overlap` = 1 launches the GEMV
- * kernels strictly stream-ordered instead of letting a GEMV start (and wait inside the kernel)
- * while the previous kernel of the stream drains; 0 is the default.
+ * persistent CTA per SM; values above 512 are clamped).  `no_overlap` is a set of bits, 0 by
+ * default: bit 0 launches the GEMV kernels strictly stream-ordered instead of letting a GEMV start
+ * (and wait inside the kernel) while the previous kernel of the stream drains; bit 1 never launches
+ * thread-block clusters (otherwise the 2..8 CTAs that share a block-row combine their sums through
+ * shared memory when the device can hold all the clusters at once).
  * Any value gives the same results up to the order of partial sums.
  * Process-wide, not thread-safe.
  */

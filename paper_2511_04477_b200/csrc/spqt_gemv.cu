@@ -52,11 +52,13 @@ constexpr int kGemvThreads = (kWorkers + 2) * 32;
 constexpr int kChunk = 32;               // list entries per chunk (one per lane)
 constexpr int kDepth = 3;                // chunks in flight per warp
 constexpr unsigned long long kWaitNs = 1000000000ull;  // bound on every mbarrier wait: one second
+constexpr int kMaxCluster = 8;           // largest thread-block cluster (CTAs of one block-row) used
 constexpr int kMaxFusedN = 32768;        // largest n whose index collection can run inside the GEMV
 constexpr int kFusedCols = 16384;        // list entries (16-bit column numbers) a CTA keeps in shared memory in that case
 
 static int g_tune_ctas = 0;  // 0 = one CTA per SM
 static int g_no_pdl = 0;     // 1 = plain stream-ordered launches
+static int g_no_cluster = 0; // 1 = never launch thread-block clusters
 
 #ifdef SPQT_TRACE
 __device__ long long* g_trace;  // time stamps of CTA 0 (debug builds only)
@@ -186,6 +188,54 @@ __device__ __forceinline__ uint4 lds_v4(unsigned addr)
 __device__ __forceinline__ void sts_u32(unsigned addr, unsigned v)
 {
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+
+// ---- thread-block clusters: the CTAs of one block-row hand their sums to CTA rank 0 through its
+// shared memory
+__device__ __forceinline__ void cluster_arrive()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait()
+{
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory location in the CTA of the given rank
+__device__ __forceinline__ unsigned cluster_map(unsigned smem_addr, unsigned rank)
+{
+    unsigned r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_f32(unsigned addr, float v)
+{
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(unsigned remote_bar)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(remote_bar) : "memory");
+}
+// Bounded wait with cluster-scope acquire (the data were written by other CTAs of the cluster).
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, unsigned parity)
+{
+    const unsigned addr = smem_u32(bar);
+    unsigned long long t0 = 0;
+    for (unsigned it = 0;; ++it) {
+        unsigned done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(addr), "r"(parity)
+            : "memory");
+        if (done) return true;
+        if (it == 16) t0 = global_ns();
+        if (it > 16) {
+            __nanosleep(64);
+            if (global_ns() - t0 > kWaitNs) return false;
+        }
+    }
 }
 
 // stores under a predicate (never a branch)
@@ -382,6 +432,9 @@ struct GemvSmem {
     alignas(16) float red[2][kWorkers][G];               // per-warp partial sums of a finished segment
     float red_z[2][kWorkers];                            // and their offset terms
     uint64_t red_full[2], red_empty[2];
+    // thread-block clusters only: partial sums the other CTAs of the cluster store here (CTA rank 0)
+    alignas(16) float xred[kMaxCluster][G + 4];
+    uint64_t xbar;                                       // counts their arrivals
     // fused index collection only
     alignas(16) int load_tot[kMaxFusedN / 256];  // active entries of every 256 entries of x
     unsigned short fused_cols[kFusedCols];       // the part of the index list this CTA reads, when it fits (n <= 32768)
@@ -393,7 +446,7 @@ struct GemvSmem {
 // own slices cover: into shared memory, or, when that part is too long, into idx_out, from where it
 // reads them back like a list collected by a separate launch.  The CTAs that work on block-row 0
 // cover the whole list between them and write idx_out; CTA 0 writes the count.
-template <int G, int BITS, bool DENSE, bool ODD_N, bool FUSED>
+template <int G, int BITS, bool DENSE, bool ODD_N, bool FUSED, bool CLUSTER>
 __global__ void __launch_bounds__(kGemvThreads, 1)
 gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales,
                  const __half* __restrict__ zeros, int R, int n,
@@ -402,7 +455,7 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
                  int* __restrict__ counters, int* __restrict__ status,
                  unsigned long long* __restrict__ words, float* __restrict__ partials,
                  float* __restrict__ zpartials, int max_slots, unsigned magic_p, unsigned magic_r,
-                 float thr, int32_t* idx_out, int32_t* count_out)
+                 int cluster_k, float thr, int32_t* idx_out, int32_t* count_out)
 {
     constexpr int B = G * BITS / 8;
     constexpr int LPB = G / 32;       // lanes that share one block (each owns 32 of its rows)
@@ -431,8 +484,13 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
             mbar_init(&sm.red_full[b], kWorkers);
             mbar_init(&sm.red_empty[b], 1);
         }
+        if (CLUSTER) mbar_init(&sm.xbar, cluster_k - 1);
+        if (CLUSTER) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    // Cluster launch (cluster_k CTAs work on one block-row and CTA rank 0 collects their sums): nobody
+    // may touch another CTA's barrier before it is initialised.  Arrive now, wait much later.
+    if (CLUSTER) cluster_arrive();
 
     // Programmatic dependent launch: this grid may have been started while the previous kernel of
     // the stream was still draining.  Nothing above touches global memory; everything below waits
@@ -583,6 +641,7 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
         pc.set_count(count);
     }
     SPQT_TRACE_EVENT(tid == 0, 4000);
+    if (CLUSTER) cluster_wait();  // every CTA of the cluster has initialised its barriers by now
 
     if (warp >= kWriterWarp) {
         // ------------------------------------------------------------ writers
@@ -669,6 +728,33 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
             float t[RPL], zsum = 0.0f;  // the block-row's sums, always accumulated in slot order
 #pragma unroll
             for (int i = 0; i < RPL; ++i) t[i] = 0.0f;
+            if (CLUSTER) {
+                // The contributors of this block-row are the CTAs of this cluster, in rank order.  The
+                // others store their sums into rank 0's shared memory and arrive on its barrier; rank 0
+                // adds them in rank order.  Nothing goes through global memory.
+                if (mine != 0) {
+                    const unsigned dst = cluster_map(smem_u32(&sm.xred[mine][0]), 0u);
+#pragma unroll
+                    for (int i = 0; i < RPL; ++i) st_cluster_f32(dst + 4u * (lane * RPL + i), v[i]);
+                    if (lane == 0) st_cluster_f32(dst + 4u * G, zpart);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(cluster_map(smem_u32(&sm.xbar), 0u));
+                    continue;
+                }
+                ok = mbar_wait_cluster(&sm.xbar, 0);
+                if (!ok) break;
+#pragma unroll
+                for (int i = 0; i < RPL; ++i) t[i] += v[i];
+                zsum += zpart;
+                for (int s = 1; s < cluster_k; ++s) {
+#pragma unroll
+                    for (int i = 0; i < RPL; ++i) t[i] += sm.xred[s][lane * RPL + i];
+                    zsum += sm.xred[s][G];
+                }
+#pragma unroll
+                for (int i = 0; i < RPL; ++i) y[(size_t)r * G + lane * RPL + i] = __float2half_rn(t[i] + zsum);
+                continue;
+            }
             if (spec) {
 #pragma unroll
                 for (int s = 0; s < kSpec + 1; ++s) {
@@ -1113,13 +1199,15 @@ static spqt_status launch_gemv(const Format& f, const void* codes, const void* s
                                const int32_t* count, void* y, void* workspace, cudaStream_t s,
                                FusedArgs fa)
 {
-    auto kernel = gemv_kernel<G, BITS, DENSE, ODD_N, FUSED>;
+    auto kernel = gemv_kernel<G, BITS, DENSE, ODD_N, FUSED, false>;
+    auto kernel_c = gemv_kernel<G, BITS, DENSE, ODD_N, FUSED, true>;  // the thread-block-cluster variant
     static bool configured[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPQT_ERR_CUDA;
     const int smem = (int)sizeof(GemvSmem<G, BITS>);
     if (!configured[dev]) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess ||
+            cudaFuncSetAttribute(kernel_c, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
             return SPQT_ERR_CUDA;
         configured[dev] = true;
     }
@@ -1145,16 +1233,43 @@ static spqt_status launch_gemv(const Format& f, const void* codes, const void* s
     cfg.blockDim = dim3(kGemvThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int nattr = 0;
+    if (!g_no_pdl) {
+        attr[nattr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[nattr].val.programmaticStreamSerializationAllowed = 1;
+        ++nattr;
+    }
+    // A whole number (2..8) of CTAs per block-row: launch them as one thread-block cluster each, if the
+    // device can hold all the clusters at once (asked once per kernel, cluster size and device).
+    int cluster_k = 0;
+    if (!g_no_cluster && f.R <= P && P % f.R == 0 && P / f.R >= 2 && P / f.R <= kMaxCluster) {
+        const int k = P / f.R;
+        static signed char fits[64][kMaxCluster + 1][149] = {};  // [device][k][clusters]: 0 unknown, 1 yes, -1 no
+        const int nclusters = P / k;
+        if (nclusters <= 148) {
+            signed char& known = fits[dev][k][nclusters];
+            attr[nattr].id = cudaLaunchAttributeClusterDimension;
+            attr[nattr].val.clusterDim.x = k;
+            attr[nattr].val.clusterDim.y = 1;
+            attr[nattr].val.clusterDim.z = 1;
+            if (known == 0) {
+                cfg.attrs = attr;
+                cfg.numAttrs = nattr + 1;
+                int can = 0;
+                if (cudaOccupancyMaxActiveClusters(&can, kernel_c, &cfg) == cudaSuccess && can >= nclusters) known = 1;
+                else { known = -1; (void)cudaGetLastError(); }
+            }
+            if (known == 1) { cluster_k = k; ++nattr; }
+        }
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = g_no_pdl ? 0 : 1;
+    cfg.numAttrs = nattr;
     const cudaError_t err = cudaLaunchKernelEx(
-        &cfg, kernel, static_cast<const uint8_t*>(codes), static_cast<const __half*>(scales),
+        &cfg, cluster_k ? kernel_c : kernel, static_cast<const uint8_t*>(codes), static_cast<const __half*>(scales),
         static_cast<const __half*>(zeros), f.R, f.n, static_cast<const __half*>(x), idx, count,
         static_cast<__half*>(y), counters, status, words, partials, zpartials, slots,
-        magic_of((unsigned)P), magic_of((unsigned)f.R), fa.t, fa.idx_out, fa.count_out);
+        magic_of((unsigned)P), magic_of((unsigned)f.R), cluster_k, fa.t, fa.idx_out, fa.count_out);
     count_launch();
     return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SPQT_OK : SPQT_ERR_CUDA;
 }
@@ -1277,9 +1392,10 @@ spqt_status spqt_set_debug(int on)
 
 spqt_status spqt_set_tuning(int gemv_ctas, int reserved)
 {
-    if (gemv_ctas < 0 || reserved < 0 || reserved > 1) return SPQT_ERR_INVALID_ARG;
+    if (gemv_ctas < 0 || reserved < 0 || reserved > 3) return SPQT_ERR_INVALID_ARG;
     spqt::g_tune_ctas = gemv_ctas;
-    spqt::g_no_pdl = reserved;
+    spqt::g_no_pdl = reserved & 1;
+    spqt::g_no_cluster = (reserved >> 1) & 1;
     return SPQT_OK;
 }
 

@@ -279,6 +279,31 @@ def test_checked_mode_refuses_bad_index_lists():
     assert status == 0 and np.array_equal(y.view(np.uint16), y_plain.view(np.uint16))
 
 
+@pytest.mark.parametrize("m,group", [(4096, 128), (8192, 128), (2048, 64)])
+def test_cluster_and_global_memory_combination_give_the_same_bits(m, group):
+    """With 2 or 4 CTAs per block-row the partial sums are combined through a thread-block cluster's
+    shared memory when the device can hold all clusters; switched off, through global memory.  Both add
+    in the same order, so y must not change by a bit (and both must match the oracle)."""
+    n, bits = 2048, 4
+    p = pack_on_gpu(inputs.weights(m, n, seed=61), bits, group)
+    codes, s, z = packed_to_host(p)
+    x = inputs.activations(n, seed=62)
+    t = inputs.threshold_for_sparsity(x, 0.5)
+    ys = []
+    for flags in (0, 2):
+        ws = binding.new_workspace(m, n, bits, group)
+        try:
+            binding.spqt_set_tuning(0, flags)
+            y, idx, cnt = run_sparse(p, x, t, ws)
+        finally:
+            binding.spqt_set_tuning(0, 0)
+        assert binding.spqt_workspace_status(ws, m, group) == 0
+        ys.append(y)
+    y_ref, bound = oracle.sparse_gemv(codes, s, z, m, n, x, idx, bits, group)
+    check_y(ys[0], y_ref, bound, "cluster")
+    assert np.array_equal(ys[0].view(np.uint16), ys[1].view(np.uint16))
+
+
 def test_heavy_tailed_outliers():
     m, n, bits, group = 1024, 8192, 4, 128
     W = inputs.weights(m, n, seed=51)
