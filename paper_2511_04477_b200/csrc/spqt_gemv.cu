@@ -11,7 +11,10 @@
 // CTA ever waits for another one to run, only for stores already issued to
 // become visible) adds the partials in slot order, adds the offset term and
 // rounds to fp16.  A CTA that finds all the other partials present before its own
-// sum is ready skips the counter and finishes the block-row directly.
+// sum is ready skips the counter and finishes the block-row directly.  With 2 or 4
+// CTAs per block-row the grid is launched as thread-block clusters of that size
+// (when the device can hold all of them at once) and the partial sums go through
+// the shared memory of the cluster's first CTA instead of global memory.
 //
 // Inside a CTA, kWorkers warps each run their own copy pipeline over chunks of
 // 32 list entries (chunks are dealt round-robin to the warps); nothing is shared
