@@ -49,11 +49,19 @@
 
 namespace spqt {
 
-constexpr int kWorkers = 18;             // compute warps
+// 12 workers + 2 writers = 14 warps leave 128 registers per thread: measured faster than 18 + 2 at 96
+// registers (which spilled) on every shape, and than 10, 11, 13 or 14 workers.
+#ifndef SPQT_WORKERS
+#define SPQT_WORKERS 12
+#endif
+#ifndef SPQT_DEPTH
+#define SPQT_DEPTH 3
+#endif
+constexpr int kWorkers = SPQT_WORKERS;   // compute warps
 constexpr int kWriterWarp = kWorkers;      // first of two writer warps: segment sg goes to writer sg & 1
 constexpr int kGemvThreads = (kWorkers + 2) * 32;
 constexpr int kChunk = 32;               // list entries per chunk (one per lane)
-constexpr int kDepth = 3;                // chunks in flight per warp
+constexpr int kDepth = SPQT_DEPTH;       // chunks in flight per warp
 constexpr unsigned long long kWaitNs = 1000000000ull;  // bound on every mbarrier wait: one second
 constexpr int kMaxCluster = 8;           // largest thread-block cluster (CTAs of one block-row) used
 constexpr int kMaxFusedN = 32768;        // largest n whose index collection can run inside the GEMV
