@@ -205,7 +205,8 @@ __device__ __forceinline__ void sts_u32(unsigned addr, unsigned v)
 // shared memory
 __device__ __forceinline__ void cluster_arrive()
 {
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    // relaxed: the only thing the other CTAs must see, the barrier initialisation, has its own fence
+    asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void cluster_wait()
 {
