@@ -58,8 +58,12 @@ namespace spqt {
 #define SPQT_DEPTH 3
 #endif
 constexpr int kWorkers = SPQT_WORKERS;   // compute warps
-constexpr int kWriterWarp = kWorkers;      // first of two writer warps: segment sg goes to writer sg & 1
-constexpr int kGemvThreads = (kWorkers + 2) * 32;
+#ifndef SPQT_WRITERS
+#define SPQT_WRITERS 2
+#endif
+constexpr int kWriters = SPQT_WRITERS;     // 1 or 2 writer warps; segment sg goes to writer sg % kWriters
+constexpr int kWriterWarp = kWorkers;      // the first of them
+constexpr int kGemvThreads = (kWorkers + kWriters) * 32;
 constexpr int kChunk = 32;               // list entries per chunk (one per lane)
 constexpr int kDepth = SPQT_DEPTH;       // chunks in flight per warp
 constexpr unsigned long long kWaitNs = 1000000000ull;  // bound on every mbarrier wait: one second
@@ -661,15 +665,16 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
         // (store, fence, counter, read back) of consecutive segments overlap.
         constexpr int RPL = G / 32;  // rows per lane
         constexpr int kStride = G + 2;  // words per contributing CTA: G sums, the offset term, one of padding
-        const int b = warp - kWriterWarp;
+        const int wr = warp - kWriterWarp;
         bool ok = true;
         if (FUSED && cols_local && pc.r_first == 0) {
             // this CTA's slice of block-row 0 is its part of the index list the call returns
             int p0, p1;
             pc.slice(0, &p0, &p1);
-            for (int i = p0 + b * 32 + lane; i < p1; i += 64) idx_out[i] = sm.fused_cols[i - need_lo];
+            for (int i = p0 + wr * 32 + lane; i < p1; i += 32 * kWriters) idx_out[i] = sm.fused_cols[i - need_lo];
         }
-        for (int r = pc.r_first + b, sg = b; r <= pc.r_last; r += 2, sg += 2) {
+        for (int r = pc.r_first + wr, sg = wr; r <= pc.r_last; r += kWriters, sg += kWriters) {
+            const int b = sg & 1;  // hand-over buffer of this segment
             int first, nslots;
             pc.contributors(r, &first, &nslots);
             const int mine = c - first;
