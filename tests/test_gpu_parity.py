@@ -304,6 +304,45 @@ def test_cluster_and_global_memory_combination_give_the_same_bits(m, group):
     assert np.array_equal(ys[0].view(np.uint16), ys[1].view(np.uint16))
 
 
+def test_seeded_random_shapes_formats_worker_counts_and_launch_modes():
+    """Sixty seeded draws of (format, m, n, sparsity, number of CTAs, launch flags, fused or not): every
+    y row against the oracle, index lists bit-exact, status word clean."""
+    rng = np.random.Generator(np.random.PCG64(20251125))
+    for case in range(60):
+        bits, group = FORMATS[int(rng.integers(0, 4))]
+        m = group * int(rng.choice([1, 2, 3, 5, 8, 16, 24, 32, 48, 64]))
+        n = int(rng.choice([1, 2, 7, 33, 64, 255, 1000, 1024, 2049, 4096, 5000]))
+        sp = float(rng.choice([0.0, 0.3, 0.5, 0.9, 1.0]))
+        ctas = int(rng.choice([0, 0, 0, 1, 5, 37, 96, 148, 300]))
+        flags = int(rng.integers(0, 4))
+        fused = bool(rng.integers(0, 2))
+        W = inputs.weights(m, n, seed=1000 + case)
+        x = inputs.activations(n, seed=2000 + case, dist="laplace" if case % 2 else "gauss")
+        t = inputs.threshold_for_sparsity(x, sp) if sp < 1.0 else float("inf")
+        p = pack_on_gpu(W, bits, group)
+        codes, s, z = packed_to_host(p)
+        ws = binding.new_workspace(m, n, bits, group)
+        what = "case %d: int%d g%d %dx%d sp %.1f ctas %d flags %d fused %d" % (case, bits, group, m, n, sp, ctas, flags, fused)
+        try:
+            binding.spqt_set_tuning(ctas, flags)
+            if fused:
+                idx_t = torch.full((n,), -1, dtype=torch.int32, device="cuda")
+                cnt_t = torch.zeros(1, dtype=torch.int32, device="cuda")
+                y_t, _, _ = binding.spqt_sparsify_gemv(p, dev(x), t, ws, idx_t, cnt_t)
+                torch.cuda.synchronize()
+                cnt = int(cnt_t.item())
+                y, idx = y_t.cpu().numpy(), idx_t.cpu().numpy()[:cnt]
+            else:
+                y, idx, cnt = run_sparse(p, x, t, ws)
+        finally:
+            binding.spqt_set_tuning(0, 0)
+        assert binding.spqt_workspace_status(ws, m, group) == 0, what
+        ref_idx, ref_cnt = oracle.sparsify(x, t)
+        assert cnt == ref_cnt and np.array_equal(idx, ref_idx), what
+        y_ref, bound = oracle.sparse_gemv(codes, s, z, m, n, x, ref_idx, bits, group)
+        check_y(y, y_ref, bound, what)
+
+
 def test_heavy_tailed_outliers():
     m, n, bits, group = 1024, 8192, 4, 128
     W = inputs.weights(m, n, seed=51)
