@@ -65,6 +65,7 @@ inline size_t workspace_bytes(const Format& f)
     return header_bytes(f.R) + tagged_bytes(f) + plain;
 }
 
+extern int g_no_pdl;          // 1 = launch strictly stream-ordered (spqt_set_tuning)
 int sm_count();               // SMs of the current device (cached per device); <= 0 on error
 void count_launch(int k = 1); // bump the process-wide launch counter
 

@@ -72,7 +72,7 @@ constexpr int kMaxFusedN = 32768;        // largest n whose index collection can
 constexpr int kFusedCols = 16384;        // list entries (16-bit column numbers) a CTA keeps in shared memory in that case
 
 static int g_tune_ctas = 0;  // 0 = one CTA per SM
-static int g_no_pdl = 0;     // 1 = plain stream-ordered launches
+int g_no_pdl = 0;            // 1 = plain stream-ordered launches (also read by the index-collection launch)
 static int g_no_cluster = 0; // 1 = never launch thread-block clusters
 
 #ifdef SPQT_TRACE

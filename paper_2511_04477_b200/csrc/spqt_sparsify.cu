@@ -23,6 +23,10 @@ sparsify_kernel(const __half* __restrict__ x, int n, float t,
     __shared__ int warp_total[32];
     __shared__ int warp_base[32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // Programmatic dependent launch: the block may have been started while the previous kernel of the
+    // stream was still draining; nothing above touches global memory, everything below waits for it.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // segment of this warp: a multiple of 32 elements, contiguous, ascending with the warp id
     const int seg = ((n + 32 * 32 - 1) / (32 * 32)) * 32;
     const int begin = min(warp * seg, n), end = min(begin + seg, n);
@@ -64,8 +68,16 @@ extern "C" spqt_status spqt_sparsify(const void* x, int n, float t,
     using namespace spqt;
     if (n < 0 || !count || (n > 0 && (!x || !idx))) return SPQT_ERR_INVALID_ARG;
     if (!aligned(x, 2) || !aligned(idx, 4) || !aligned(count, 4)) return SPQT_ERR_ALIGNMENT;
-    sparsify_kernel<<<1, kSparsifyThreads, 0, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<const __half*>(x), n, t, idx, count);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(1);
+    cfg.blockDim = dim3(kSparsifyThreads);
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_no_pdl ? 0 : 1;
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, sparsify_kernel, static_cast<const __half*>(x), n, t, idx, count);
     count_launch();
-    return cudaGetLastError() == cudaSuccess ? SPQT_OK : SPQT_ERR_CUDA;
+    return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SPQT_OK : SPQT_ERR_CUDA;
 }
