@@ -944,7 +944,9 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
         }
     };
     // stage B: code blocks and metadata words of the next chunk (its column numbers have landed)
-    auto issue_b = [&](unsigned ring_s, unsigned ring_c) {
+    // (pre: column numbers of the copies and of the lane's metadata entry, read ahead of time by prep_b,
+    // or nullptr to read them here)
+    auto issue_b = [&](unsigned ring_s, unsigned ring_c, const unsigned* pre) {
         if (cb.valid(pc)) {
             if (cb.r != b_row) {
                 b_row = cb.r;
@@ -962,7 +964,7 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
 #pragma unroll
                 for (int u = 0; u < SUBS; ++u) {
                     const int e = min(u * SLOTS + slot, vm1);
-                    const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : col_at(cols_addr, e);
+                    const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : (pre ? pre[u] : col_at(cols_addr, e));
                     if (DENSE) cp_async_16(st_addr + lane * 16 + u * 512, b_codes + (size_t)kk * B);
                     else cp_async_16_l2_64(st_addr + lane * 16 + u * 512, b_codes + (size_t)kk * B);
                 }
@@ -986,7 +988,7 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
             {
                 // the aligned 4-byte word that holds each fp16 value (index rounded down to even)
                 const int e = min(lane, vm1);
-                const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : col_at(cols_addr, e);
+                const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : ((pre && BITS == 4) ? pre[SUBS] : col_at(cols_addr, e));
                 const unsigned mdst = st_addr + kMetaOff + 4u * lane;
                 const int mo = (int)kk - (int)((kk ^ b_par) & 1u);  // may be -1 only when r*n is odd: still inside the array
                 if (!ODD_N || kk != (unsigned)(n - 1)) {
@@ -1004,6 +1006,18 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
         }
     };
 
+    // The column numbers stage B will need at the end of this iteration, read before the arithmetic so
+    // that the shared-memory latency hides under it (4-bit sparse path only).
+    auto prep_b = [&](unsigned ring_c, unsigned* pre) {
+        if (!DENSE && BITS == 4 && cb.valid(pc)) {
+            const int vm1 = min(cb.p1 - cb.pos, kChunk) - 1;
+            const unsigned cols_addr = use_list ? cols_base + ring_c : fused_base + 2u * (unsigned)cb.pos;
+#pragma unroll
+            for (int u = 0; u < SUBS; ++u) pre[u] = col_at(cols_addr, min(u * SLOTS + slot, vm1));
+            pre[SUBS] = col_at(cols_addr, min(lane, vm1));
+        }
+    };
+
     // fill the pipeline: D chunks of columns, then D chunks of blocks (each needs its columns)
 #pragma unroll 1
     for (int s = 0; s < D; ++s) {
@@ -1014,7 +1028,7 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
     for (int s = 0; s < D; ++s) {
         cp_async_wait<D - 1>();
         __syncwarp();
-        issue_b(s * kStageBytes, s * kColsBytes);
+        issue_b(s * kStageBytes, s * kColsBytes, nullptr);
         issue_a((D + s) * kColsBytes);
         cp_async_commit();
     }
@@ -1043,6 +1057,8 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
 #ifdef SPQT_TRACE
             const long long tc1 = clock64();
 #endif
+            unsigned pre[SUBS + 1];
+            prep_b(rb_c, pre);
             const unsigned st_addr = stage_base + rc_s;
             const unsigned xw = lds_u32(st_addr + kMetaOff + 4u * lane);
             const unsigned sw = lds_u32(st_addr + kMetaOff + 4u * lane + kChunk * 4);
@@ -1074,7 +1090,7 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
                 }
             }
             __syncwarp();  // every lane has read its part of the slots that B and A now refill
-            issue_b(rc_s, rb_c);
+            issue_b(rc_s, rb_c, (!DENSE && BITS == 4) ? pre : nullptr);
             issue_a(rc_c);
             cp_async_commit();
             wrap(rc_s, kStageBytes, D * kStageBytes);
