@@ -2,6 +2,7 @@
 
     python -m paper_2511_04477_b200.sweep sparsity      # 0-90 % on 4096x14336 and 14336x4096, int4 g128
     python -m paper_2511_04477_b200.sweep formats       # Llama-2-70B-shaped linears x {int4,int3} x {g64,g128}, 50 %
+    python -m paper_2511_04477_b200.sweep stack         # 32-layer Llama-3-8B-shaped stack, thresholds calibrated for 40 %
 
 Each case packs several distinct weight copies (together well above the 126 MB L2), visits them
 round-robin inside one CUDA graph and times graph replays with CUDA events.  Printed per case: device
@@ -114,6 +115,86 @@ def copies_for(m, n, bits, group):
     return int(min(64, max(4, math.ceil(512e6 / size))))
 
 
+STACK_SITES = [  # (site, stacked matrix rows, n, distribution of the site's input)
+    ("attn_in", 6144, 4096, "laplace"),    # q | k | v share x and idx
+    ("attn_out", 4096, 4096, "laplace"),   # o
+    ("mlp_in", 28672, 4096, "laplace"),    # gate | up
+    ("mlp_mid", 4096, 14336, "gauss"),     # down
+]
+
+
+def build_stack(layers, tokens, sparsity=0.4, calib_vectors=64):
+    """Packed weights of `layers` decoder layers (random-init on the device, one seed per matrix), per-site
+    thresholds calibrated once on pooled calibration vectors, and `tokens` fresh inputs per site."""
+    g = torch.Generator(device="cuda")
+    packs, thr, xs = [], {}, {}
+    for L in range(layers):
+        row = {}
+        for i, (site, m, n, _) in enumerate(STACK_SITES):
+            g.manual_seed(L * 7 + i)
+            W = torch.empty((m, n), dtype=torch.float32, device="cuda").normal_(0.0, 0.02, generator=g).half()
+            row[site] = binding.spqt_pack(W, 4, 128)
+            del W
+        packs.append(row)
+    for i, (site, m, n, dist) in enumerate(STACK_SITES):
+        calib = [inputs.activations(n, seed=9000 + 100 * i + c, dist=dist) for c in range(calib_vectors)]
+        thr[site] = inputs.pooled_threshold(calib, sparsity)
+        host = np.stack([inputs.activations(n, seed=20000 + 1000 * i + t, dist=dist) for t in range(tokens)])
+        xs[site] = (host, torch.from_numpy(host).cuda())
+    return packs, thr, xs
+
+
+def run_stack(layers=32, tokens=100, peak=None):
+    """Per-token pass over the linear layers of the whole stack: 4 launches per layer (index collection
+    inside the GEMV), one CUDA graph per token, device-timed; tokens/s of the linear layers."""
+    packs, thr, xs = build_stack(layers, tokens)
+    ws = {site: binding.new_workspace(m, n, 4, 128) for (site, m, n, _) in STACK_SITES}
+    y = {site: torch.empty(m, dtype=torch.float16, device="cuda") for (site, m, n, _) in STACK_SITES}
+    idx = {site: torch.empty(n, dtype=torch.int32, device="cuda") for (site, m, n, _) in STACK_SITES}
+    cnt = {site: torch.zeros(1, dtype=torch.int32, device="cuda") for (site, m, n, _) in STACK_SITES}
+    s = torch.cuda.Stream()
+
+    def token_pass(t, stream):
+        for L in range(layers):
+            for (site, m, n, _) in STACK_SITES:
+                binding.spqt_sparsify_gemv(packs[L][site], xs[site][1][t], thr[site], ws[site], idx[site], cnt[site],
+                                           y[site], stream=stream)
+
+    with torch.cuda.stream(s):
+        token_pass(0, s)
+    torch.cuda.synchronize()
+    graphs = []
+    for t in range(tokens):
+        gph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gph, stream=s):
+            token_pass(t, s)
+        graphs.append(gph)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(s):
+        for gph in graphs[:3]:
+            gph.replay()
+        e0.record(s)
+        for gph in graphs:
+            gph.replay()
+        e1.record(s)
+        e1.synchronize()
+    ms_token = e0.elapsed_time(e1) / tokens
+    sp = {site: [inputs.realised_sparsity(xs[site][0][t], thr[site]) for t in range(tokens)] for (site, _, _, _) in STACK_SITES}
+    needed = 0
+    for (site, m, n, _) in STACK_SITES:
+        counts = [int(round((1.0 - v) * n)) for v in sp[site]]
+        needed += layers * float(np.mean([needed_bytes(m, n, c, 4, 128) + 2 * n + 4 * c + 4 for c in counts]))
+    status = max(binding.spqt_workspace_status(ws[site], m, 128) for (site, m, n, _) in STACK_SITES)
+    out = {"layers": layers, "tokens": tokens, "ms_per_token": ms_token, "tokens_per_s": 1e3 / ms_token,
+           "launches_per_token": 4 * layers, "needed_gb_per_token": needed * 1e-9,
+           "needed_gbs": needed / ms_token * 1e-6, "pct_of_measured_peak": 100 * needed / ms_token * 1e-6 / (peak or _peak()),
+           "thresholds": thr,
+           "realised_sparsity": {k: {"mean": float(np.mean(v)), "min": float(np.min(v)), "max": float(np.max(v))} for k, v in sp.items()},
+           "packed_gb": sum(p.codes.numel() + 2 * p.scales.numel() + 2 * p.zeros.numel() for row in packs for p in row.values()) * 1e-9,
+           "device_status": status}
+    return out
+
+
 def main(argv):
     which = argv[0] if argv else "sparsity"
     peak = _peak()
@@ -130,8 +211,17 @@ def main(argv):
             for bits in (4, 3):
                 for group in (128, 64):
                     out += run_case(m, n, bits, group, [0.5], x, copies_for(m, n, bits, group), peak)
+    elif which == "stack":
+        res = run_stack(peak=peak)
+        print("32-layer stack: %.3f ms per token over the linear layers, %.0f tokens/s, %d launches per token, "
+              "%.2f GB needed per token (%.0f GB/s, %.1f %% of the measured HBM peak); realised sparsity %s" % (
+                  res["ms_per_token"], res["tokens_per_s"], res["launches_per_token"], res["needed_gb_per_token"],
+                  res["needed_gbs"], res["pct_of_measured_peak"],
+                  {k: "%.3f (%.3f-%.3f)" % (v["mean"], v["min"], v["max"]) for k, v in res["realised_sparsity"].items()}))
+        print(json.dumps({"sweep": which, "hbm_peak_gbs": peak, "result": res}))
+        return
     else:
-        raise SystemExit("usage: python -m paper_2511_04477_b200.sweep [sparsity|formats]")
+        raise SystemExit("usage: python -m paper_2511_04477_b200.sweep [sparsity|formats|stack]")
     show(out)
     print(json.dumps({"sweep": which, "hbm_peak_gbs": peak, "rows": out}))
 

@@ -470,6 +470,33 @@ def test_llama3_8b_shapes_on_sampled_rows(name, m, n, dist):
     assert np.array_equal(s[r], s_ref[0]) and np.array_equal(z[r], z_ref[0])
 
 
+def test_32_layer_stack_token_pass_on_sampled_layers_sites_and_rows():
+    """The 32-layer Llama-3-8B-shaped stack as the sweep tool runs it (3.7 GB of packed weights, thresholds
+    calibrated once per site for 40 % on pooled vectors, fresh x per token, index collection inside the GEMV
+    launch): index lists bit-exact and y on sampled rows against the oracle, for three layers, all four
+    sites and two tokens."""
+    from paper_2511_04477_b200 import sweep
+    layers, tokens = 32, 3
+    packs, thr, xs = sweep.build_stack(layers, tokens)
+    rng = np.random.Generator(np.random.PCG64(77))
+    for L in (0, 17, 31):
+        for (site, m, n, _) in sweep.STACK_SITES:
+            p = packs[L][site]
+            codes, s, z = packed_to_host(p)
+            ws = binding.new_workspace(m, n, 4, 128)
+            rows = np.unique(np.concatenate([rng.integers(0, m, size=48), [0, 127, 128, m - 1]])).astype(np.int32)
+            for t in (0, tokens - 1):
+                x = xs[site][0][t]
+                y, idx, cnt = binding.spqt_sparsify_gemv(p, xs[site][1][t], thr[site], ws)
+                torch.cuda.synchronize()
+                ref_idx, ref_cnt = oracle.sparsify(x, thr[site])
+                assert int(cnt.item()) == ref_cnt and np.array_equal(idx.cpu().numpy()[:ref_cnt], ref_idx)
+                assert 0.3 < 1.0 - ref_cnt / n < 0.5   # calibrated for 40 %, fluctuates per token
+                y_ref, bound = oracle.sparse_gemv(codes, s, z, m, n, x, ref_idx, 4, 128, rows=rows)
+                check_y(y.cpu().numpy()[rows], y_ref, bound, "layer %d %s token %d" % (L, site, t))
+            assert binding.spqt_workspace_status(ws, m, 128) == 0
+
+
 @pytest.mark.parametrize("bits,group", FORMATS)
 def test_llama2_70b_attention_shape_with_heavy_tailed_outliers(bits, group):
     """8192 -> 8192, every format, x ~ Laplace with 1 % of the entries multiplied by 20, 50 % sparsity."""
