@@ -392,6 +392,26 @@ def run_ours(args):
                          "dense_gbs": needed_bytes_gemv(m, n, n) / (t_de * 1e-3 / reps) / 1e9,
                          "speedup_vs_dense": t_de / t_sp}
 
+    # ---- achievable read and gather rates of this GPU with the GEMV's copy instruction (rank 0 only)
+    probes = None
+    if rank == 0:
+        buf = torch.empty(2 << 30, dtype=torch.uint8, device=dev)   # 2 GB, far beyond L2
+        buf.fill_(1)
+        moved = torch.zeros(1, dtype=torch.int64, device=dev)
+        probes = {}
+        for pattern, key in ((0, "stream_read_gbs"), (1, "gather_64B_half_of_lines_gbs")):
+            best = 0.0
+            for _ in range(3):
+                moved.zero_()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                binding.spqt_probe_read(buf, pattern, moved)
+                e1.record()
+                e1.synchronize()
+                best = max(best, float(moved.item()) / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+            probes[key] = best
+        del buf
+
     # ---- end to end from host buffers through the C ABI (copies + sync inside the timed region)
     e2e_names = list(stacked.values())
     hosts = [{nm: binding.HostLinear(layers[L][nm], ws[nm]) for nm in e2e_names} for L in range(LAYER_COPIES)]
@@ -442,7 +462,9 @@ def run_ours(args):
                             "seven_matrices_4_sparsify_7_gemv_launches": ms_separate * 1e3 / K},
             "speedup_vs_dense_same_layout": ms_dense / ms_gemv,
             "dense_gbs": gb_dense / (ms_dense * 1e-3) / 1e9,
-            "pct_of_peak": {"of_measured_%.0f" % peak: 100 * achieved / peak, "of_nominal_8000": 100 * achieved / 8000},
+            "pct_of_peak": {"of_measured_%.0f" % peak: 100 * achieved / peak, "of_nominal_8000": 100 * achieved / 8000,
+                            "of_probed_gather": 100 * achieved / probes["gather_64B_half_of_lines_gbs"]},
+            "probed_rooflines": probes,
             "per_shape": per_shape,
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": traffic, "peak_kind": "of " + peak_kind,

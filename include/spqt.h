@@ -216,6 +216,17 @@ spqt_status spqt_set_debug(int on);
  */
 spqt_status spqt_workspace_status(const void* workspace, int m, int group, int* status_host, void* stream);
 
+/*
+ * Measurement aid, not part of the method (the paper has no counterpart): reads `bytes` of device
+ * memory at `buf` (128-byte aligned) into shared memory in 64-byte blocks with the copy instruction
+ * the GEMV uses, and adds the number of bytes it fetched to *moved (a device counter the caller
+ * zeroes).  pattern 0: every block (the achievable read rate); pattern 1: one randomly chosen half
+ * of every 128-byte line (the gather a sparse GEMV performs at 50 % block density).  Time it with
+ * events on `stream`; the buffer should be much larger than L2.
+ */
+spqt_status spqt_probe_read(const void* buf, size_t bytes, int pattern,
+                            unsigned long long* moved, void* stream);
+
 /* Number of kernels the library has launched in this process (a counter for
  * benchmarks; not synchronised with the device). */
 unsigned long long spqt_launch_count(void);

@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libspqt.so")
 EXPORTS = (
     "spqt_status_string", "spqt_version", "spqt_packed_sizes", "spqt_pack", "spqt_unpack",
     "spqt_sparsify", "spqt_sparse_gemv", "spqt_sparse_gemv_static", "spqt_sparsify_gemv", "spqt_dense_gemv", "spqt_sparse_linear_host",
-    "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_launch_count",
+    "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_launch_count",
 )
 
 _lib = None
@@ -59,11 +59,12 @@ def lib() -> ctypes.CDLL:
                                               vp, vp, vp, vp, vp, sz, vp]
         L.spqt_set_tuning.argtypes = [i32, i32]
         L.spqt_set_debug.argtypes = [i32]
+        L.spqt_probe_read.argtypes = [vp, sz, i32, vp, vp]
         L.spqt_workspace_status.argtypes = [vp, i32, i32, ctypes.POINTER(i32), vp]
         L.spqt_launch_count.restype = ctypes.c_ulonglong
         for name in ("spqt_packed_sizes", "spqt_pack", "spqt_unpack", "spqt_sparsify",
                      "spqt_sparse_gemv", "spqt_dense_gemv", "spqt_sparse_linear_host", "spqt_set_tuning",
-                     "spqt_set_debug", "spqt_workspace_status"):
+                     "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read"):
             getattr(L, name).restype = i32
         _lib = L
     return _lib
@@ -255,6 +256,13 @@ def spqt_sparse_linear_host(h: HostLinear, t: float, stream=None) -> torch.Tenso
         h.count.data_ptr(), h.y_dev.data_ptr(), h.workspace.data_ptr(), h.workspace.numel(),
         _stream(stream)), "spqt_sparse_linear_host")
     return h.y_host
+
+
+def spqt_probe_read(buf: torch.Tensor, pattern: int, moved: torch.Tensor, stream=None) -> None:
+    """Measurement aid: stream `buf` into shared memory in 64-byte blocks (pattern 0: all of them, 1: one random
+    half of every 128-byte line); adds the bytes fetched to `moved` (int64[1] on the device)."""
+    _ok(lib().spqt_probe_read(_dev(buf, torch.uint8, "buf"), buf.numel(), int(pattern),
+                              _dev(moved, torch.int64, "moved"), _stream(stream)), "spqt_probe_read")
 
 
 def spqt_set_debug(on: bool) -> None:

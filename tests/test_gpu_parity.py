@@ -536,6 +536,20 @@ def test_host_entry_point_matches_the_device_path():
     assert int(h.count.item()) == cnt
 
 
+def test_read_and_gather_probes_fetch_what_they_report():
+    """The roofline probes of the benchmark: every 64-byte block of the region, or half of them."""
+    buf = torch.ones(256 << 20, dtype=torch.uint8, device="cuda")
+    moved = torch.zeros(1, dtype=torch.int64, device="cuda")
+    binding.spqt_probe_read(buf, 0, moved)
+    torch.cuda.synchronize()
+    all_blocks = int(moved.item())
+    assert 0.98 * buf.numel() <= all_blocks <= buf.numel()
+    moved.zero_()
+    binding.spqt_probe_read(buf, 1, moved)
+    torch.cuda.synchronize()
+    assert abs(int(moved.item()) - all_blocks // 2) <= all_blocks // 100
+
+
 def test_kernels_are_counted():
     before = binding.spqt_launch_count()
     x = dev(inputs.activations(256, seed=1))
