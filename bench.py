@@ -442,6 +442,10 @@ def run_ours(args):
 
     if rank == 0:
         cpu = oracle_sample(3, 1) if world >= 1 else None
+        cpu_all = cpu["cores"]
+        cpu1 = oracle_sample(1, 0, threads=1)      # the same sample on one core
+        import oracle as _oracle
+        _oracle.set_threads(cpu_all)
         avg_launch_bytes = gb / n_gemv
         traffic = NCU_TRAFFIC_RATIO * avg_launch_bytes
         line = {
@@ -471,7 +475,7 @@ def run_ours(args):
                          "kernel": "gemv_kernel<128,sparse>", "algorithmic_bytes_per_launch": avg_launch_bytes,
                          "avg_launch_us": ms_gemv * 1e3 / n_gemv},
             "cpu_baseline": {"value": cpu["value"], "unit": "GB/s", "cores": cpu["cores"], "kind": "oracle",
-                             "sample": cpu["sample"]},
+                             "sample": cpu["sample"], "single_thread_value": cpu1["value"]},
             "e2e": {"value": world * e2e_bytes / e2e_s / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s / e2e_K * 1e3},
             "gpu_launches": launches_timed, "launches_counted_incl_warmup_and_capture": launches,
