@@ -64,7 +64,8 @@ constexpr int kWorkers = SPQT_WORKERS;   // compute warps
 constexpr int kWriters = SPQT_WRITERS;     // 1 or 2 writer warps; segment sg goes to writer sg % kWriters
 constexpr int kWriterWarp = kWorkers;      // the first of them
 constexpr int kGemvThreads = (kWorkers + kWriters) * 32;
-constexpr int kChunk = 32;               // list entries per chunk (one per lane)
+// list entries per chunk: 2 KB of 4-bit code blocks for either group size (32 blocks of 128 rows, 64 of 64)
+__host__ __device__ constexpr int chunk_entries(int group) { return 32 * (128 / group); }
 constexpr int kDepth = SPQT_DEPTH;       // chunks in flight per warp
 constexpr unsigned long long kWaitNs = 1000000000ull;  // bound on every mbarrier wait: one second
 constexpr int kMaxCluster = 8;           // largest thread-block cluster (CTAs of one block-row) used
@@ -94,12 +95,13 @@ namespace spqt {
 template <int G, int BITS>
 struct GemvSmem {
     static constexpr int B = G * BITS / 8;
+    static constexpr int CH = chunk_entries(G);
     struct Stage {
-        alignas(16) unsigned char codes[kChunk * B];  // block e of the chunk at e*B
-        unsigned meta[3][kChunk];                     // words holding x_k, scale_rk, zero_rk of entry e
+        alignas(16) unsigned char codes[CH * B];  // block e of the chunk at e*B
+        unsigned meta[3][CH];                     // words holding x_k, scale_rk, zero_rk of entry e
     };
     Stage stage[kWorkers][kDepth];
-    alignas(16) int cols[kWorkers][2 * kDepth][kChunk];  // column numbers of the chunks ahead
+    alignas(16) int cols[kWorkers][2 * kDepth][CH];  // column numbers of the chunks ahead
     alignas(16) float red[2][kWorkers][G];               // per-warp partial sums of a finished segment
     float red_z[2][kWorkers];                            // and their offset terms
     uint64_t red_full[2], red_empty[2];
@@ -134,7 +136,9 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
     static_assert(BITS == 3 || BITS == 4, "3- or 4-bit codes");
     constexpr int SLOTS = 32 / LPB;   // blocks per 512-byte warp load
     constexpr int KEEP = 32 / SLOTS;  // values per lane after the in-warp reduce-scatter
-    constexpr int SUBS = kChunk / SLOTS;  // 512-byte loads per chunk
+    constexpr int CH = chunk_entries(G);  // list entries per chunk
+    constexpr int EPL = CH / 32;          // entries whose metadata a lane holds
+    constexpr int SUBS = CH / SLOTS;      // 512-byte loads per chunk
     constexpr int D = kDepth;
 
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -558,8 +562,8 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
     // rather than by branches: the loop is bound by instruction issue.
     using Stage = typename GemvSmem<G, BITS>::Stage;
     constexpr unsigned kStageBytes = (unsigned)sizeof(Stage);
-    constexpr unsigned kMetaOff = (unsigned)(kChunk * B);     // offset of Stage::meta
-    constexpr unsigned kColsBytes = kChunk * 4;               // one chunk of column numbers
+    constexpr unsigned kMetaOff = (unsigned)(CH * B);     // offset of Stage::meta
+    constexpr unsigned kColsBytes = CH * 4;               // one chunk of column numbers
     static_assert(offsetof(Stage, meta) == kMetaOff, "stage layout");
     const int slot = lane / LPB, h = lane % LPB;
     const unsigned short* xb = reinterpret_cast<const unsigned short*>(x);
@@ -576,7 +580,7 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
     };
 
     Cursor ca, cb;  // stage A / stage B cursors (the consume side walks the segments itself)
-    ca.init(pc, warp);
+    ca.init(pc, warp, CH);
     cb = ca;
     // Ring positions (byte offsets) of the chunk stage C works on: rc_s in the ring of D stages, rc_c
     // in the ring of 2*D chunks of column numbers, rb_c = D chunks further in that ring.  Stage B
@@ -594,7 +598,11 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
     // stage A: column numbers of the warp's next chunk
     auto issue_a = [&](unsigned ring_c) {
         if (use_list && ca.valid(pc)) {
-            if (ca.pos + lane < ca.p1) cp_async_4(cols_base + ring_c + 4u * lane, idx + ca.pos + lane);
+#pragma unroll
+            for (int q = 0; q < EPL; ++q) {
+                const int e = lane + 32 * q;
+                if (ca.pos + e < ca.p1) cp_async_4(cols_base + ring_c + 4u * e, idx + ca.pos + e);
+            }
             ca.advance(pc, warp);
         }
     };
@@ -611,7 +619,7 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
                 b_scales = reinterpret_cast<const unsigned short*>(scales) + row_base;
                 b_zeros = reinterpret_cast<const unsigned short*>(zeros) + row_base;
             }
-            const int vm1 = min(cb.p1 - cb.pos, kChunk) - 1;  // last entry of this chunk that exists
+            const int vm1 = min(cb.p1 - cb.pos, CH) - 1;  // last entry of this chunk that exists
             // address of the chunk's first column number (unused when DENSE)
             const unsigned cols_addr = use_list ? cols_base + ring_c : fused_base + 2u * (unsigned)cb.pos;
             const unsigned st_addr = stage_base + ring_s;
@@ -625,7 +633,7 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
                 }
             } else {
                 // 3-bit blocks (48 or 24 bytes): the chunk's bytes in copies of CB bytes, lane after lane
-                constexpr int NC = kChunk * B / CB / 32;
+                constexpr int NC = CH * B / CB / 32;
 #pragma unroll
                 for (int q = 0; q < NC; ++q) {
                     const int off = (q * 32 + lane) * CB;    // byte offset inside the chunk's stage
@@ -640,21 +648,22 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
                     }
                 }
             }
-            {
+#pragma unroll
+            for (int q = 0; q < EPL; ++q) {
                 // the aligned 4-byte word that holds each fp16 value (index rounded down to even)
-                const int e = min(lane, vm1);
-                const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : ((pre && BITS == 4) ? pre[SUBS] : col_at(cols_addr, e));
-                const unsigned mdst = st_addr + kMetaOff + 4u * lane;
+                const int e = min(lane + 32 * q, vm1);
+                const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : ((pre && BITS == 4) ? pre[SUBS + q] : col_at(cols_addr, e));
+                const unsigned mdst = st_addr + kMetaOff + 4u * (lane + 32 * q);
                 const int mo = (int)kk - (int)((kk ^ b_par) & 1u);  // may be -1 only when r*n is odd: still inside the array
                 if (!ODD_N || kk != (unsigned)(n - 1)) {
                     cp_async_4_ca(mdst, xb + (kk & ~1u));
-                    cp_async_4(mdst + kChunk * 4, b_scales + mo);
-                    cp_async_4(mdst + 2 * kChunk * 4, b_zeros + mo);
+                    cp_async_4(mdst + CH * 4, b_scales + mo);
+                    cp_async_4(mdst + 2 * CH * 4, b_zeros + mo);
                 } else {
                     // n odd: the word of the last column may reach past the end of an array; fetch directly
                     sts_u32(mdst, (unsigned)__ldg(xb + kk) << ((kk & 1u) * 16));
-                    sts_u32(mdst + kChunk * 4, (unsigned)__ldg(b_scales + kk) << (((kk ^ b_par) & 1u) * 16));
-                    sts_u32(mdst + 2 * kChunk * 4, (unsigned)__ldg(b_zeros + kk) << (((kk ^ b_par) & 1u) * 16));
+                    sts_u32(mdst + CH * 4, (unsigned)__ldg(b_scales + kk) << (((kk ^ b_par) & 1u) * 16));
+                    sts_u32(mdst + 2 * CH * 4, (unsigned)__ldg(b_zeros + kk) << (((kk ^ b_par) & 1u) * 16));
                 }
             }
             cb.advance(pc, warp);
@@ -665,11 +674,12 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
     // that the shared-memory latency hides under it (4-bit sparse path only).
     auto prep_b = [&](unsigned ring_c, unsigned* pre) {
         if (!DENSE && BITS == 4 && cb.valid(pc)) {
-            const int vm1 = min(cb.p1 - cb.pos, kChunk) - 1;
+            const int vm1 = min(cb.p1 - cb.pos, CH) - 1;
             const unsigned cols_addr = use_list ? cols_base + ring_c : fused_base + 2u * (unsigned)cb.pos;
 #pragma unroll
             for (int u = 0; u < SUBS; ++u) pre[u] = col_at(cols_addr, min(u * SLOTS + slot, vm1));
-            pre[SUBS] = col_at(cols_addr, min(lane, vm1));
+#pragma unroll
+            for (int q = 0; q < EPL; ++q) pre[SUBS + q] = col_at(cols_addr, min(lane + 32 * q, vm1));
         }
     };
 
@@ -702,7 +712,7 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
         pc.slice(r, &p0, &p1);
         const unsigned c_par = ODD_N ? (unsigned)(((size_t)r * (size_t)n) & 1) : 0u;
         float zl = 0.0f;  // this lane's share of sum x_k * zero_rk
-        for (int pos = p0 + warp * kChunk; pos < p1; pos += kWorkers * kChunk) {
+        for (int pos = p0 + warp * CH; pos < p1; pos += kWorkers * CH) {
             // ---- stage C of the oldest chunk: everything it needs is in commit groups that wait<D-1> covers
 #ifdef SPQT_TRACE
             const long long tc0 = clock64();
@@ -712,29 +722,33 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
 #ifdef SPQT_TRACE
             const long long tc1 = clock64();
 #endif
-            unsigned pre[SUBS + 1];
+            unsigned pre[SUBS + EPL];
             prep_b(rb_c, pre);
             const unsigned st_addr = stage_base + rc_s;
-            const unsigned xw = lds_u32(st_addr + kMetaOff + 4u * lane);
-            const unsigned sw = lds_u32(st_addr + kMetaOff + 4u * lane + kChunk * 4);
-            const unsigned zw = lds_u32(st_addr + kMetaOff + 4u * lane + 2 * kChunk * 4);
-            const int e = min(lane, p1 - pos - 1);  // the entry whose metadata this lane holds
-            unsigned kk;
-            if (DENSE) kk = (unsigned)(pos + e);
-            else kk = col_at(use_list ? cols_base + rc_c : fused_base + 2u * (unsigned)pos, e);
 #ifdef SPQT_TRACE
             const long long tc2 = clock64();
 #endif
-            const unsigned xs = (kk & 1u) * 16, ms = ((kk ^ c_par) & 1u) * 16;
-            const float xf = __half2float(__ushort_as_half((unsigned short)(xw >> xs)));
-            const float sf = __half2float(__ushort_as_half((unsigned short)(sw >> ms)));
-            const float zf = __half2float(__ushort_as_half((unsigned short)(zw >> ms)));
-            const float xin = (e == lane) ? xf : 0.0f;  // 0 past the end of the slice
-            const float a = xin * sf;                   // exact
-            zl = fmaf(xin, zf, zl);
+            float a[EPL];  // x_k * scale_rk of the entries this lane holds (entry lane + 32 q)
+#pragma unroll
+            for (int q = 0; q < EPL; ++q) {
+                const unsigned xw = lds_u32(st_addr + kMetaOff + 4u * (lane + 32 * q));
+                const unsigned sw = lds_u32(st_addr + kMetaOff + 4u * (lane + 32 * q) + CH * 4);
+                const unsigned zw = lds_u32(st_addr + kMetaOff + 4u * (lane + 32 * q) + 2 * CH * 4);
+                const int e = min(lane + 32 * q, p1 - pos - 1);  // the entry whose metadata this lane holds
+                unsigned kk;
+                if (DENSE) kk = (unsigned)(pos + e);
+                else kk = col_at(use_list ? cols_base + rc_c : fused_base + 2u * (unsigned)pos, e);
+                const unsigned xs = (kk & 1u) * 16, ms = ((kk ^ c_par) & 1u) * 16;
+                const float xf = __half2float(__ushort_as_half((unsigned short)(xw >> xs)));
+                const float sf = __half2float(__ushort_as_half((unsigned short)(sw >> ms)));
+                const float zf = __half2float(__ushort_as_half((unsigned short)(zw >> ms)));
+                const float xin = (e == lane + 32 * q) ? xf : 0.0f;  // 0 past the end of the slice
+                a[q] = xin * sf;                                      // exact
+                zl = fmaf(xin, zf, zl);
+            }
 #pragma unroll
             for (int u = 0; u < SUBS; ++u) {
-                const float au = __shfl_sync(0xffffffffu, a, u * SLOTS + slot);
+                const float au = __shfl_sync(0xffffffffu, a[(u * SLOTS) / 32], (u * SLOTS + slot) & 31);
                 if (BITS == 4) {
                     const uint4 wv = lds_v4(st_addr + lane * 16 + u * 512);
                     fma_block16(acc, wv, au);

@@ -1,6 +1,6 @@
 // The work map of the GEMV kernel: which block-rows, and which slices of the active index list,
 // belong to which CTA and warp (32-bit arithmetic, divisions by multiply-high).  Included by
-// spqt_gemv.cu only, after its compile-time constants (kWorkers, kChunk).
+// spqt_gemv.cu only, after its compile-time constants (kWorkers).
 #pragma once
 
 namespace spqt {
@@ -65,6 +65,7 @@ struct Piece {
 // chunk's first entry inside block-row r (whose slice ends at p1).
 struct Cursor {
     int r, pos, p1;
+    int chunk;  // list entries per chunk (32 or 64, by format)
     __device__ __forceinline__ void settle(const Piece& pc, int warp)
     {
         while (r <= pc.r_last && pos >= p1) {
@@ -72,22 +73,23 @@ struct Cursor {
             if (r <= pc.r_last) {
                 int p0;
                 pc.slice(r, &p0, &p1);
-                pos = p0 + warp * kChunk;
+                pos = p0 + warp * chunk;
             }
         }
     }
-    __device__ __forceinline__ void init(const Piece& pc, int warp)
+    __device__ __forceinline__ void init(const Piece& pc, int warp, int chunk_)
     {
+        chunk = chunk_;
         r = pc.r_first;
         int p0;
         pc.slice(r, &p0, &p1);
-        pos = p0 + warp * kChunk;
+        pos = p0 + warp * chunk;
         settle(pc, warp);
     }
     __device__ __forceinline__ bool valid(const Piece& pc) const { return r <= pc.r_last; }
     __device__ __forceinline__ void advance(const Piece& pc, int warp)
     {
-        pos += kWorkers * kChunk;
+        pos += kWorkers * chunk;
         if (pos >= p1) settle(pc, warp);
     }
 };
