@@ -17,11 +17,12 @@
 // the shared memory of the cluster's first CTA instead of global memory.
 //
 // Inside a CTA, kWorkers warps each run their own copy pipeline over chunks of
-// 32 list entries (chunks are dealt round-robin to the warps); nothing is shared
+// 32 list entries (64 with groups of 64 rows: 2 KB of 4-bit codes either way;
+// chunks are dealt round-robin to the warps); nothing is shared
 // between the warps until the end of a segment.  Per chunk, three stages, all
 // cp.async into the warp's private shared-memory ring, one commit group per
 // iteration:
-//   A  the chunk's 32 column numbers (one 4-byte copy per lane);
+//   A  the chunk's column numbers (one 4-byte copy per lane and entry);
 //   B  once A has landed: the code blocks (16 bytes per lane, the lanes of a
 //      block adjacent so that every 32-byte sector crosses once, fetched with
 //      64-byte L2 granularity so that an inactive neighbour block is not dragged
