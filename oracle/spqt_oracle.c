@@ -105,7 +105,10 @@ size_t spqt_oracle_block_bytes(int bits, int group) { return block_bytes(bits, g
  * Asymmetric min/max round-to-nearest per superblock (group-wise scheme with a
  * scale and an additive offset per block, Sec. 2 / Sec. 4.1.1; any group-based
  * scheme and bit-width is admissible, Sec. 4.1.3).
- *   z  = min_i w_i                       (an fp16 value, kept exactly)
+ *   z  = min_i w_i                       (an fp16 value, kept exactly; a minimum or maximum
+ *                                         that is zero is taken as +0.0 whatever the signs of
+ *                                         the zeros in the group: the values are the same and
+ *                                         the stored bytes do not depend on the order of the rows)
  *   s  = fp16( (max_i w_i - z) / qmax )  (fp32 subtract, fp32 divide, RN-even)
  *   q_i = clamp( rint( (w_i - z) / s ), 0, qmax ),  all zero when s == 0
  * W: fp16 bits, row-major, leading dimension ldw.
@@ -125,6 +128,8 @@ int spqt_oracle_quantize(const uint16_t* W, int m, int n, int ldw, int bits, int
                 if (w < lo) lo = w;
                 if (w > hi) hi = w;
             }
+            if (lo == 0.0f) lo = 0.0f;                   /* a zero extreme of either sign is +0.0 */
+            if (hi == 0.0f) hi = 0.0f;
             volatile float range = hi - lo;              /* one fp32 subtract */
             volatile float s32 = range / (float)qmax;    /* one fp32 divide   */
             uint16_t sh = float_to_half(s32);

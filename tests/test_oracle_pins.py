@@ -148,6 +148,25 @@ def test_quantizer_invariants(bits, group):
     assert np.array_equal(z2.astype(np.float32), z.astype(np.float32) * 4)
 
 
+def test_zero_minimum_is_stored_as_plus_zero_whatever_the_signs_and_order():
+    """A group whose minimum is zero with both signs present (pruned weights): the offset is +0.0
+    (bits 0x0000) for every order of the rows, and the codes are those of the non-negative values
+    divided by the scale (the sign of a zero changes no quotient)."""
+    group, bits = 4, 4
+    pos = np.array([0.0, 0.5, 1.5, 0.0], np.float16)
+    for first_zero, other_zero in ((np.float16(-0.0), np.float16(0.0)), (np.float16(0.0), np.float16(-0.0))):
+        col = pos.copy()
+        col[0], col[3] = first_zero, other_zero
+        assert np.signbit(col[0]) != np.signbit(col[3])
+        q, s, z = oracle.quantize(col.reshape(group, 1), bits, group)
+        assert z.view(np.uint16)[0, 0] == 0x0000
+        assert float(s[0, 0]) == 0.0999755859375            # fp16(1.5 / 15)
+        assert q[:, 0].tolist() == [0, 5, 15, 0]
+    # all zeros of either sign: constant group, scale 0, offset +0.0
+    q, s, z = oracle.quantize(np.array([[-0.0], [-0.0], [0.0], [-0.0]], np.float16), bits, group)
+    assert z.view(np.uint16)[0, 0] == 0x0000 and s.view(np.uint16)[0, 0] == 0x0000 and not q.any()
+
+
 def test_quantizer_codes_match_numpy_single_precision_steps():
     """Same steps taken with numpy's IEEE float32 ufuncs (a different engine)."""
     bits, group, qmax = 4, 128, 15
