@@ -15,7 +15,8 @@
  *   Every pointer is a DEVICE pointer unless its name ends in _host.
  *   `stream` is a cudaStream_t passed as void* (NULL = the legacy default
  *   stream).  All calls are asynchronous on that stream and never synchronise
- *   the device, except the *_host entry point, which says so.
+ *   the device, except the *_host entry point and spqt_workspace_status, which
+ *   say so.
  *   The caller owns every buffer; the library allocates nothing, frees nothing
  *   and keeps no pointer after a call returns.
  *
@@ -26,15 +27,16 @@
  *           3-bit block: G/4 bytes of a 2-bit plane, byte j = sum_{u<4}
  *           (code[j + u*G/4] & 3) << 2u, then G/8 bytes of a 1-bit plane,
  *           byte j = sum_{u<8} (code[j + u*G/8] >> 2) << u.
- *   scales, zeros : fp16 arrays of R*n entries, entry (r,k) at index r*n + k.
- *           A weight is What[r*G+i][k] = scales[r,k] * code_i + zeros[r,k]
+ *   scale_zero : R*n pairs of fp16 in the same block order: the pair of block
+ *           (r,k) is at fp16 index 2*(r*n + k): first the scale, then the zero.
+ *           A weight is What[r*G+i][k] = scale[r,k] * code_i + zero[r,k]
  *           ("zero" is the additive offset of the block, its minimum).
  *
  * Errors
  *   Every entry point returns a spqt_status.  Arguments that can be checked on
- *   the host are checked before anything is launched; a failed check launches
- *   nothing.  The contents of idx/count are trusted (indices in [0,n), no
- *   duplicates, count <= n).
+ *   the host are checked before anything is put on the stream; a failed check
+ *   launches nothing.  The contents of idx/count are trusted (indices in [0,n),
+ *   no duplicates, count <= n) unless checked mode is on.
  */
 #ifndef SPQT_H
 #define SPQT_H
@@ -48,11 +50,12 @@ extern "C" {
 
 typedef enum {
     SPQT_OK = 0,
-    SPQT_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, ldw < n                 */
-    SPQT_ERR_UNSUPPORTED = 2, /* bits not in {3,4}, group not in {64,128}, m % group != 0 */
-    SPQT_ERR_ALIGNMENT = 3,   /* a pointer is not aligned as documented                   */
-    SPQT_ERR_WORKSPACE = 4,   /* workspace smaller than spqt_packed_sizes reports         */
-    SPQT_ERR_CUDA = 5         /* the CUDA runtime reported an error (launch, copy, query) */
+    SPQT_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, ldw < n; a bad index list (checked mode) */
+    SPQT_ERR_UNSUPPORTED = 2, /* bits not in {3,4}, group not in {64,128}, m % group != 0, n too large     */
+    SPQT_ERR_ALIGNMENT = 3,   /* a pointer is not aligned as documented                                    */
+    SPQT_ERR_WORKSPACE = 4,   /* workspace smaller than spqt_packed_sizes reports                          */
+    SPQT_ERR_CUDA = 5,        /* the CUDA runtime reported an error (launch, copy, query)                  */
+    SPQT_ERR_TIMEOUT = 6      /* a bounded wait inside a kernel expired (seen through spqt_workspace_status) */
 } spqt_status;
 
 /* Human-readable name of a status code; never NULL. */
@@ -62,35 +65,39 @@ const char* spqt_status_string(int status);
 int spqt_version(void);
 
 /*
- * Sizes in bytes of the buffers a problem needs.  Any out-pointer may be NULL.
- * Needs no GPU.  gemv_workspace_bytes covers both GEMV entry points.
+ * Sizes in bytes of the buffers a problem needs (layout of paper Sec. 4.1.2: R*n
+ * blocks; one scale and one offset per block, Sec. 4.1.1).  Any out-pointer may
+ * be NULL.  Needs no GPU.  gemv_workspace_bytes covers every GEMV entry point.
  */
 spqt_status spqt_packed_sizes(int m, int n, int bits, int group,
-                              size_t* codes_bytes, size_t* scales_bytes, size_t* zeros_bytes,
+                              size_t* codes_bytes, size_t* scale_zero_bytes,
                               size_t* gemv_workspace_bytes);
 
 /*
  * Offline conversion: quantize W group by group and write it in zigzag order
- * (paper Sec. 3.2 "first quantized into the zigzag weight layout", Sec. 4.1.2).
+ * (paper Sec. 3.2, Sec. 4.1.2; run once per model, Sec. 5).
  * Per block: zero = min of the G weights; scale = fp16((max - zero) / (2^b - 1)),
  * the subtraction and division each one IEEE fp32 operation; code_i =
  * clamp(rint((w_i - zero) / scale), 0, 2^b - 1) with ties to even, all zero when
- * scale == 0.  Results are bit-reproducible.
- *   W      : fp16, row-major [m][ldw], ldw >= n, 2-byte aligned.
- *   codes  : R*n*B bytes, 16-byte aligned.   scales, zeros : R*n fp16, 16-byte aligned.
+ * scale == 0.  A minimum or maximum that is zero counts as +0.0 whatever the
+ * signs of the zeros in the group.  Results are bit-reproducible.
+ *   W          : fp16, row-major [m][ldw], ldw >= n, 2-byte aligned.
+ *   codes      : R*n*B bytes, 16-byte aligned.
+ *   scale_zero : 2*R*n fp16, 16-byte aligned.
  */
 spqt_status spqt_pack(const void* W, int m, int n, int ldw, int bits, int group,
-                      void* codes, void* scales, void* zeros, void* stream);
+                      void* codes, void* scale_zero, void* stream);
 
 /*
- * Inverse of the layout step of spqt_pack (a checking aid): natural-order codes,
- * one byte each, q_u8[j*n + k] = code of row j, column k.
+ * Inverse of the layout step of spqt_pack (a checking aid for the layout of
+ * paper Sec. 4.1.2): natural-order codes, one byte each, q_u8[j*n + k] = code
+ * of row j, column k.
  */
 spqt_status spqt_unpack(const void* codes, int m, int n, int bits, int group,
                         void* q_u8, void* stream);
 
 /*
- * Sparse index collection (paper Sec. 4.2.3, "Sparse index collecting kernel"):
+ * Sparse index collection (paper Sec. 4.2.3, the index-collecting kernel):
  * idx[0:*count] = every k with |x_k| > t, in ascending order; *count = how many.
  * The comparison is strict and exact (fp16 widened); NaN entries are never
  * active.  idx must hold n entries.  x: fp16[n], 2-byte aligned.  idx, count:
@@ -106,15 +113,15 @@ spqt_status spqt_sparsify(const void* x, int n, float t,
  * evenly over the workers of that block-row; partial sums are accumulated in
  * fp32 and combined in a fixed order, so a call is bit-reproducible.  idx may be
  * in any order.  *count == 0 gives y = 0.
- *   codes/scales/zeros : as written by spqt_pack, 16-byte aligned.
- *   x : fp16[n], 4-byte aligned.  idx : int32[>= *count].  count : int32 on the device.
+ *   codes, scale_zero : as written by spqt_pack, 16-byte aligned.
+ *   x : fp16[n], 2-byte aligned.  idx : int32[>= *count].  count : int32 on the device.
  *   y : fp16[m], 2-byte aligned.
  *   workspace : gemv_workspace_bytes of device memory, 16-byte aligned, zeroed
  *       ONCE by the caller before its first use; every call leaves it ready for
  *       the next.  Two calls that may overlap on the GPU need two workspaces.
- * Supported: bits 4 or 3 with group 64 or 128.
+ * Supported: bits 4 or 3 with group 64 or 128; n <= 65535 (column numbers travel as 16 bits).
  */
-spqt_status spqt_sparse_gemv(const void* codes, const void* scales, const void* zeros,
+spqt_status spqt_sparse_gemv(const void* codes, const void* scale_zero,
                              int m, int n, int bits, int group,
                              const void* x, const int32_t* idx, const int32_t* count,
                              void* y, void* workspace, size_t workspace_bytes, void* stream);
@@ -124,19 +131,22 @@ spqt_status spqt_sparse_gemv(const void* codes, const void* scales, const void* 
  * a kernel of its own before every GEMV, Sec. 4.2.3; on this GPU a separate launch plus the
  * count -> idx -> blocks chain of dependent reads costs more than a small GEMV itself).  Results
  * are identical to the two calls: idx[0:*count] ascending, *count, and the same y bits.  idx (n
- * entries) and count are written; the other arguments are those of spqt_sparse_gemv.  For
- * n > 32768 the two kernels are launched one after the other instead.
+ * entries) and count are written; the other arguments are those of spqt_sparse_gemv.  When x is too
+ * long for the in-kernel scan (n above about 30000) the two kernels are launched one after the
+ * other instead.
  */
-spqt_status spqt_sparsify_gemv(const void* codes, const void* scales, const void* zeros,
+spqt_status spqt_sparsify_gemv(const void* codes, const void* scale_zero,
                                int m, int n, int bits, int group,
                                const void* x, float t, int32_t* idx, int32_t* count,
                                void* y, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * The same kernel over all n columns with no index list: the dense GEMV on the
- * zigzag layout (paper Sec. 4.2.2), the sparsity-free comparison.
+ * zigzag layout (paper Sec. 4.2.2), the sparsity-free comparison.  Any n when n is a multiple of 8
+ * and x is 16-byte aligned (whole chunks of a block-row are then fetched by bulk copies); otherwise
+ * n <= 65535.
  */
-spqt_status spqt_dense_gemv(const void* codes, const void* scales, const void* zeros,
+spqt_status spqt_dense_gemv(const void* codes, const void* scale_zero,
                             int m, int n, int bits, int group, const void* x,
                             void* y, void* workspace, size_t workspace_bytes, void* stream);
 
@@ -154,18 +164,28 @@ spqt_status spqt_dense_gemv(const void* codes, const void* scales, const void* z
  *   - Problems whose workspace (spqt_packed_sizes: gemv_workspace_bytes) exceeds 1 MiB are refused
  *     with SPQT_ERR_WORKSPACE; every Llama-shaped layer used in this repository fits.
  *   - The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
- *     that device current) and keeps it; make that first call before any stream capture begins.
+ *     that device current) and keeps it; make that first call before any stream capture begins, and
+ *     from one host thread (the look-up is not guarded against two threads making it at once).
  *   - All calls on a device share the one array, which still holds the previous call's contents; the
  *     part that must start at zero (arrival counters, status word, the tagged words that carry partial
- *     sums between thread blocks: up to about 0.9 MiB) is cleared on `stream` before the kernel.  Two calls that may overlap on the GPU (different streams, no ordering) race on it:
- *     order them, or use spqt_sparse_gemv with separate workspaces.
- *   - Because the status word is cleared per call, spqt_workspace_status does not apply here.
+ *     sums between thread blocks: up to about 0.9 MiB) is cleared on `stream` before the kernel, after
+ *     every argument check has passed.  Two calls that may overlap on the GPU (different streams, no
+ *     ordering) race on it: order them, or use spqt_sparse_gemv with separate workspaces.
+ *   - Because the status word is cleared per call, it describes the last call only: read it with
+ *     spqt_static_status after that call.
  * Other arguments, alignment rules and error codes are those of spqt_sparse_gemv.
  */
-spqt_status spqt_sparse_gemv_static(const void* codes, const void* scales, const void* zeros,
+spqt_status spqt_sparse_gemv_static(const void* codes, const void* scale_zero,
                                     int m, int n, int bits, int group,
                                     const void* x, const int32_t* idx, const int32_t* count,
                                     void* y, void* stream);
+
+/*
+ * Status word of the built-in scratch after the last spqt_sparse_gemv_static call on this device
+ * and stream (same meaning and return value as spqt_workspace_status; waits for the stream).
+ * m and group are those of that call.
+ */
+spqt_status spqt_static_status(int m, int group, int* status_host, void* stream);
 
 /*
  * One decode-time linear layer from HOST activations (paper Sec. 3.2: hidden
@@ -176,9 +196,9 @@ spqt_status spqt_sparse_gemv_static(const void* codes, const void* scales, const
  * should be pinned for the copies to be asynchronous (the kernel then writes y
  * straight into y_host and the copy back is skipped); x_dev (fp16[n]), idx_dev
  * (int32[n]), count_dev (int32[1]) and y_dev (fp16[m]) are caller-provided
- * device staging buffers.  This is the only entry point that synchronises.
+ * device staging buffers.  This entry point synchronises.
  */
-spqt_status spqt_sparse_linear_host(const void* codes, const void* scales, const void* zeros,
+spqt_status spqt_sparse_linear_host(const void* codes, const void* scale_zero,
                                     int m, int n, int bits, int group,
                                     const void* x_host, float t, void* y_host,
                                     void* x_dev, int32_t* idx_dev, int32_t* count_dev, void* y_dev,
@@ -201,18 +221,20 @@ spqt_status spqt_set_tuning(int gemv_ctas, int no_overlap);
  * normal path).  With on != 0, spqt_sparse_gemv and spqt_sparse_gemv_static first check the list on
  * the device: *count in [0, n], every index in [0, n), and, for n <= 1048576, no index twice.  A bad
  * list sets the workspace's status word to 2 and the product is computed with a count of 0 (y = 0)
- * instead of reading wherever the indices point.  Costs two small extra launches per call; the check
- * keeps its state per device, so checked calls on one device must not overlap.  Process-wide, not
- * thread-safe.
+ * instead of reading wherever the indices point.  The verdict is per call: a later call with a good
+ * list on the same workspace computes its product normally, although the status word stays set until
+ * the caller zeroes the workspace.  Costs two small extra launches per call; the check keeps its
+ * state per device, so checked calls on one device must not overlap.  Process-wide, not thread-safe.
  */
 spqt_status spqt_set_debug(int on);
 
 /*
  * Reads the workspace's status word into *status_host (a host int) and waits for
  * the stream: 0 = every GEMV that used this workspace ran to completion;
- * 1 = a bounded wait expired inside a GEMV kernel (which then drained its copies
- * and returned early, leaving y unspecified); 2 = checked mode found a bad index
- * list.  The word is sticky until the caller zeroes the workspace again.
+ * 1 = a bounded wait expired inside a GEMV kernel (which then returned early,
+ * leaving y unspecified); 2 = checked mode found a bad index list.  The word is
+ * sticky until the caller zeroes the workspace again.  Returns SPQT_OK for 0,
+ * SPQT_ERR_TIMEOUT for 1 and SPQT_ERR_INVALID_ARG for 2 (after writing *status_host).
  */
 spqt_status spqt_workspace_status(const void* workspace, int m, int group, int* status_host, void* stream);
 

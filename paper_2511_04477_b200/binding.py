@@ -19,8 +19,8 @@ LIB_PATH = os.path.join(_HERE, "libspqt.so")
 
 EXPORTS = (
     "spqt_status_string", "spqt_version", "spqt_packed_sizes", "spqt_pack", "spqt_unpack",
-    "spqt_sparsify", "spqt_sparse_gemv", "spqt_sparse_gemv_static", "spqt_sparsify_gemv", "spqt_dense_gemv", "spqt_sparse_linear_host",
-    "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_launch_count",
+    "spqt_sparsify", "spqt_sparse_gemv", "spqt_sparse_gemv_static", "spqt_static_status", "spqt_sparsify_gemv", "spqt_dense_gemv",
+    "spqt_sparse_linear_host", "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_launch_count",
 )
 
 _lib = None
@@ -45,17 +45,19 @@ def lib() -> ctypes.CDLL:
         L.spqt_status_string.restype = ctypes.c_char_p
         L.spqt_status_string.argtypes = [i32]
         L.spqt_version.restype = i32
-        L.spqt_packed_sizes.argtypes = [i32, i32, i32, i32] + [ctypes.POINTER(sz)] * 4
-        L.spqt_pack.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp, vp]
+        L.spqt_packed_sizes.argtypes = [i32, i32, i32, i32] + [ctypes.POINTER(sz)] * 3
+        L.spqt_pack.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp]
         L.spqt_unpack.argtypes = [vp, i32, i32, i32, i32, vp, vp]
         L.spqt_sparsify.argtypes = [vp, i32, ctypes.c_float, vp, vp, vp]
-        L.spqt_sparse_gemv.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
-        L.spqt_sparse_gemv_static.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp]
+        L.spqt_sparse_gemv.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
+        L.spqt_sparse_gemv_static.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp]
         L.spqt_sparse_gemv_static.restype = i32
-        L.spqt_sparsify_gemv.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, vp, vp, vp, vp, sz, vp]
+        L.spqt_static_status.argtypes = [i32, i32, ctypes.POINTER(i32), vp]
+        L.spqt_static_status.restype = i32
+        L.spqt_sparsify_gemv.argtypes = [vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, vp, vp, vp, vp, sz, vp]
         L.spqt_sparsify_gemv.restype = i32
-        L.spqt_dense_gemv.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, sz, vp]
-        L.spqt_sparse_linear_host.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, vp,
+        L.spqt_dense_gemv.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, sz, vp]
+        L.spqt_sparse_linear_host.argtypes = [vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, vp,
                                               vp, vp, vp, vp, vp, sz, vp]
         L.spqt_set_tuning.argtypes = [i32, i32]
         L.spqt_set_debug.argtypes = [i32]
@@ -97,13 +99,12 @@ def _dev(t: torch.Tensor, dtype, name: str) -> int:
 @dataclass
 class PackedSizes:
     codes_bytes: int
-    scales_bytes: int
-    zeros_bytes: int
+    scale_zero_bytes: int
     gemv_workspace_bytes: int
 
 
 def spqt_packed_sizes(m: int, n: int, bits: int = 4, group: int = 128) -> PackedSizes:
-    out = [ctypes.c_size_t(0) for _ in range(4)]
+    out = [ctypes.c_size_t(0) for _ in range(3)]
     _ok(lib().spqt_packed_sizes(m, n, bits, group, *[ctypes.byref(o) for o in out]), "spqt_packed_sizes")
     return PackedSizes(*[int(o.value) for o in out])
 
@@ -111,17 +112,26 @@ def spqt_packed_sizes(m: int, n: int, bits: int = 4, group: int = 128) -> Packed
 @dataclass
 class Packed:
     """Device buffers written by :func:`spqt_pack` (zigzag layout)."""
-    codes: torch.Tensor    # uint8[R*n*B]
-    scales: torch.Tensor   # float16[R*n]
-    zeros: torch.Tensor    # float16[R*n]
+    codes: torch.Tensor        # uint8[R*n*B]
+    scale_zero: torch.Tensor   # float16[2*R*n]: (scale, zero) of block (r,k) at 2*(r*n+k)
     m: int
     n: int
     bits: int
     group: int
 
     @property
+    def scales(self) -> torch.Tensor:
+        """float16[R*n], a strided view of scale_zero."""
+        return self.scale_zero[0::2]
+
+    @property
+    def zeros(self) -> torch.Tensor:
+        """float16[R*n], a strided view of scale_zero."""
+        return self.scale_zero[1::2]
+
+    @property
     def nbytes(self) -> int:
-        return self.codes.numel() + 2 * self.scales.numel() + 2 * self.zeros.numel()
+        return self.codes.numel() + 2 * self.scale_zero.numel()
 
 
 def new_workspace(m: int, n: int, bits: int = 4, group: int = 128, device=None) -> torch.Tensor:
@@ -138,11 +148,10 @@ def spqt_pack(W: torch.Tensor, bits: int = 4, group: int = 128, stream=None) -> 
     m, n = W.shape
     sz = spqt_packed_sizes(m, n, bits, group)
     codes = torch.empty(sz.codes_bytes, dtype=torch.uint8, device=W.device)
-    scales = torch.empty(sz.scales_bytes // 2, dtype=torch.float16, device=W.device)
-    zeros = torch.empty(sz.zeros_bytes // 2, dtype=torch.float16, device=W.device)
+    scale_zero = torch.empty(sz.scale_zero_bytes // 2, dtype=torch.float16, device=W.device)
     _ok(lib().spqt_pack(W.data_ptr(), m, n, W.stride(0), bits, group, codes.data_ptr(),
-                        scales.data_ptr(), zeros.data_ptr(), _stream(stream)), "spqt_pack")
-    return Packed(codes, scales, zeros, m, n, bits, group)
+                        scale_zero.data_ptr(), _stream(stream)), "spqt_pack")
+    return Packed(codes, scale_zero, m, n, bits, group)
 
 
 def spqt_unpack(p: Packed, stream=None) -> torch.Tensor:
@@ -174,8 +183,8 @@ def spqt_sparse_gemv(p: Packed, x: torch.Tensor, idx: torch.Tensor, count: torch
     if x.numel() != p.n or y.numel() != p.m:
         raise ValueError("x must have n entries and y m entries")
     _ok(lib().spqt_sparse_gemv(
-        _dev(p.codes, torch.uint8, "codes"), _dev(p.scales, torch.float16, "scales"),
-        _dev(p.zeros, torch.float16, "zeros"), p.m, p.n, p.bits, p.group,
+        _dev(p.codes, torch.uint8, "codes"), _dev(p.scale_zero, torch.float16, "scale_zero"),
+        p.m, p.n, p.bits, p.group,
         _dev(x, torch.float16, "x"), _dev(idx, torch.int32, "idx"), _dev(count, torch.int32, "count"),
         _dev(y, torch.float16, "y"), _dev(workspace, torch.uint8, "workspace"), workspace.numel(),
         _stream(stream)), "spqt_sparse_gemv")
@@ -190,8 +199,8 @@ def spqt_sparse_gemv_static(p: Packed, x: torch.Tensor, idx: torch.Tensor, count
     if x.numel() != p.n or y.numel() != p.m:
         raise ValueError("x must have n entries and y m entries")
     _ok(lib().spqt_sparse_gemv_static(
-        _dev(p.codes, torch.uint8, "codes"), _dev(p.scales, torch.float16, "scales"),
-        _dev(p.zeros, torch.float16, "zeros"), p.m, p.n, p.bits, p.group,
+        _dev(p.codes, torch.uint8, "codes"), _dev(p.scale_zero, torch.float16, "scale_zero"),
+        p.m, p.n, p.bits, p.group,
         _dev(x, torch.float16, "x"), _dev(idx, torch.int32, "idx"), _dev(count, torch.int32, "count"),
         _dev(y, torch.float16, "y"), _stream(stream)), "spqt_sparse_gemv_static")
     return y
@@ -209,8 +218,8 @@ def spqt_sparsify_gemv(p: Packed, x: torch.Tensor, t: float, workspace: torch.Te
     if x.numel() != p.n or y.numel() != p.m or idx.numel() < p.n:
         raise ValueError("x and idx must have n entries and y m entries")
     _ok(lib().spqt_sparsify_gemv(
-        _dev(p.codes, torch.uint8, "codes"), _dev(p.scales, torch.float16, "scales"),
-        _dev(p.zeros, torch.float16, "zeros"), p.m, p.n, p.bits, p.group,
+        _dev(p.codes, torch.uint8, "codes"), _dev(p.scale_zero, torch.float16, "scale_zero"),
+        p.m, p.n, p.bits, p.group,
         _dev(x, torch.float16, "x"), float(t), _dev(idx, torch.int32, "idx"), _dev(count, torch.int32, "count"),
         _dev(y, torch.float16, "y"), _dev(workspace, torch.uint8, "workspace"), workspace.numel(),
         _stream(stream)), "spqt_sparsify_gemv")
@@ -224,8 +233,8 @@ def spqt_dense_gemv(p: Packed, x: torch.Tensor, workspace: torch.Tensor, y: torc
     if x.numel() != p.n or y.numel() != p.m:
         raise ValueError("x must have n entries and y m entries")
     _ok(lib().spqt_dense_gemv(
-        _dev(p.codes, torch.uint8, "codes"), _dev(p.scales, torch.float16, "scales"),
-        _dev(p.zeros, torch.float16, "zeros"), p.m, p.n, p.bits, p.group,
+        _dev(p.codes, torch.uint8, "codes"), _dev(p.scale_zero, torch.float16, "scale_zero"),
+        p.m, p.n, p.bits, p.group,
         _dev(x, torch.float16, "x"), _dev(y, torch.float16, "y"),
         _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)), "spqt_dense_gemv")
     return y
@@ -251,7 +260,7 @@ def spqt_sparse_linear_host(h: HostLinear, t: float, stream=None) -> torch.Tenso
     """x in ``h.x_host`` -> y in ``h.y_host`` (copies, index collection, sparse GEMV, sync)."""
     p = h.p
     _ok(lib().spqt_sparse_linear_host(
-        p.codes.data_ptr(), p.scales.data_ptr(), p.zeros.data_ptr(), p.m, p.n, p.bits, p.group,
+        p.codes.data_ptr(), p.scale_zero.data_ptr(), p.m, p.n, p.bits, p.group,
         h.x_host.data_ptr(), float(t), h.y_host.data_ptr(), h.x_dev.data_ptr(), h.idx.data_ptr(),
         h.count.data_ptr(), h.y_dev.data_ptr(), h.workspace.data_ptr(), h.workspace.numel(),
         _stream(stream)), "spqt_sparse_linear_host")
@@ -274,12 +283,27 @@ def spqt_set_tuning(gemv_ctas: int = 0, no_overlap: int = 0) -> None:
     _ok(lib().spqt_set_tuning(int(gemv_ctas), int(no_overlap)), "spqt_set_tuning")
 
 
-def spqt_workspace_status(workspace: torch.Tensor, m: int, group: int = 128, stream=None) -> int:
-    """0 unless a bounded on-chip wait expired in a GEMV that used this workspace (synchronises)."""
-    out = ctypes.c_int(-1)
-    _ok(lib().spqt_workspace_status(_dev(workspace, torch.uint8, "workspace"), m, group,
-                                    ctypes.byref(out), _stream(stream)), "spqt_workspace_status")
+def _status_word(rc: int, out: ctypes.c_int, where: str) -> int:
+    # the call returns SPQT_ERR_TIMEOUT (6) / SPQT_ERR_INVALID_ARG (1) for a non-zero word it has read
+    if out.value == -1 or rc not in (0, 1, 6):
+        raise SpqtError(rc, where)
     return int(out.value)
+
+
+def spqt_workspace_status(workspace: torch.Tensor, m: int, group: int = 128, stream=None) -> int:
+    """The workspace's status word: 0, 1 (a bounded on-chip wait expired in a GEMV that used this workspace)
+    or 2 (checked mode refused an index list).  Synchronises."""
+    out = ctypes.c_int(-1)
+    rc = lib().spqt_workspace_status(_dev(workspace, torch.uint8, "workspace"), m, group,
+                                     ctypes.byref(out), _stream(stream))
+    return _status_word(rc, out, "spqt_workspace_status")
+
+
+def spqt_static_status(m: int, group: int = 128, stream=None) -> int:
+    """Status word of the built-in scratch after the last spqt_sparse_gemv_static call (synchronises)."""
+    out = ctypes.c_int(-1)
+    rc = lib().spqt_static_status(m, group, ctypes.byref(out), _stream(stream))
+    return _status_word(rc, out, "spqt_static_status")
 
 
 def spqt_launch_count() -> int:

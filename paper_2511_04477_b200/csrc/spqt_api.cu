@@ -35,29 +35,29 @@ const char* spqt_status_string(int s)
         case SPQT_ERR_ALIGNMENT: return "SPQT_ERR_ALIGNMENT";
         case SPQT_ERR_WORKSPACE: return "SPQT_ERR_WORKSPACE";
         case SPQT_ERR_CUDA: return "SPQT_ERR_CUDA";
+        case SPQT_ERR_TIMEOUT: return "SPQT_ERR_TIMEOUT";
         default: return "SPQT_ERR_UNKNOWN";
     }
 }
 
-int spqt_version(void) { return 1000; }
+int spqt_version(void) { return 2000; }
 
 spqt_status spqt_packed_sizes(int m, int n, int bits, int group,
-                              size_t* codes_bytes, size_t* scales_bytes, size_t* zeros_bytes,
+                              size_t* codes_bytes, size_t* scale_zero_bytes,
                               size_t* gemv_workspace_bytes)
 {
     spqt::Format f;
     spqt_status st = spqt::make_format(m, n, bits, group, &f);
     if (st != SPQT_OK) return st;
     if (codes_bytes) *codes_bytes = f.blocks * (size_t)f.B;
-    if (scales_bytes) *scales_bytes = f.blocks * 2;
-    if (zeros_bytes) *zeros_bytes = f.blocks * 2;
+    if (scale_zero_bytes) *scale_zero_bytes = f.blocks * 4;
     if (gemv_workspace_bytes) *gemv_workspace_bytes = spqt::workspace_bytes(f);
     return SPQT_OK;
 }
 
 unsigned long long spqt_launch_count(void) { return spqt::g_launches.load(std::memory_order_relaxed); }
 
-spqt_status spqt_sparse_linear_host(const void* codes, const void* scales, const void* zeros,
+spqt_status spqt_sparse_linear_host(const void* codes, const void* scale_zero,
                                     int m, int n, int bits, int group,
                                     const void* x_host, float t, void* y_host,
                                     void* x_dev, int32_t* idx_dev, int32_t* count_dev, void* y_dev,
@@ -80,7 +80,7 @@ spqt_status spqt_sparse_linear_host(const void* codes, const void* scales, const
     else
         (void)cudaGetLastError();  // pageable memory is not an error here
     // index collection and product in one launch (two for very long x: the call decides)
-    st = spqt_sparsify_gemv(codes, scales, zeros, m, n, bits, group, x_dev, t, idx_dev, count_dev,
+    st = spqt_sparsify_gemv(codes, scale_zero, m, n, bits, group, x_dev, t, idx_dev, count_dev,
                             y_target, workspace, workspace_bytes, stream);
     if (st != SPQT_OK) return st;
     if (y_target == y_dev &&

@@ -16,27 +16,36 @@
 // (when the device can hold all of them at once) and the partial sums go through
 // the shared memory of the cluster's first CTA instead of global memory.
 //
-// Inside a CTA, kWorkers warps each run their own copy pipeline over chunks of
-// 32 list entries (64 with groups of 64 rows: 2 KB of 4-bit codes either way;
-// chunks are dealt round-robin to the warps); nothing is shared
-// between the warps until the end of a segment.  Per chunk, three stages, all
-// cp.async into the warp's private shared-memory ring, one commit group per
-// iteration:
-//   A  the chunk's column numbers (one 4-byte copy per lane and entry);
-//   B  once A has landed: the code blocks (16 bytes per lane, the lanes of a
-//      block adjacent so that every 32-byte sector crosses once, fetched with
-//      64-byte L2 granularity so that an inactive neighbour block is not dragged
-//      in) and the 4-byte words holding x_k, scale_rk and zero_rk of the lane's
-//      own entry;
-//   C  once B has landed: lane l turns its words into a = x_k*scale_rk (exact in
-//      fp32) and x_k*zero_rk, the multipliers are dealt out with shuffles, and
-//      the warp does the dequantize-FMA work.
-// A runs 2*kDepth chunks ahead of C and B kDepth chunks ahead, so kDepth chunks
-// (2 KB each) per warp are in flight.  Two more warps, the writers (one per
-// hand-over buffer), add the workers' sums at the end of a segment, publish the
-// partial and, if this CTA is the last contributor of the block-row, produce y;
-// their waits on shared-memory barriers are bounded in wall time (on expiry the
-// workspace's status word is set and the kernel returns).
+// The list a CTA works from lives in shared memory as one 32-bit word per active
+// entry: the column number in the low half, the fp16 bits of x_k in the high half.
+// The prologue builds it: from idx and x (sparse call), by scanning x itself (the
+// call that collects the indices in the same launch: every CTA scans x, counts the
+// active entries of every 256-entry piece and expands only the pieces that overlap
+// the list positions its own slices cover), or not at all (dense call).  When the
+// part of the list a CTA needs exceeds the shared-memory window, the window is
+// rebuilt between spans of the slice.
+//
+// Inside a CTA, every worker warp owns a contiguous part of each slice and runs its
+// own copy pipeline over chunks of 32 list entries (64 with groups of 64 rows: 2 KB
+// of 4-bit codes either way), kDepth chunks in flight; nothing is shared between
+// the warps until the end of a segment.  Per chunk:
+//   issue    lane e reads the word of entry e, copies the 4-byte (scale, zero) pair
+//            of block (r, k_e) and keeps the entry word with the chunk; the code
+//            blocks are copied 16 bytes per lane, the lanes of a block adjacent so
+//            that every 32-byte sector crosses once, with 64-byte L2 granularity so
+//            that an inactive neighbour block is not dragged in (cp.async).  The
+//            dense call instead fetches the chunk's codes, pairs and x values with
+//            three bulk copies issued by one lane (they are contiguous).
+//   consume  lane e turns its pair into a = x_k*scale (exact in fp32) and
+//            x_k*zero, writes the two packed multiplier pairs of its entry to
+//            shared memory; then every lane does the dequantize-FMA work on its 16
+//            bytes of each block, reading the block's multipliers back.
+// Entries past the end of a part are clamped to its last entry with weight 0, and
+// the 512-byte steps of a chunk that hold no entry are skipped.  Two more warps,
+// the writers (one per hand-over buffer), add the workers' sums at the end of a
+// segment, publish the partial and, if this CTA is the last contributor of the
+// block-row, produce y; their waits on shared-memory barriers are bounded in wall
+// time (on expiry the workspace's status word is set and the kernel returns).
 //
 // Arithmetic:  y[j] = sum_k a_k * code_jk + sum_k x_k * zero_rk.  A 4-bit code
 // becomes an fp32 operand with no conversion: the nibble masked in place at bit
@@ -50,39 +59,36 @@
 
 namespace spqt {
 
-// 12 workers + 2 writers = 14 warps leave 128 registers per thread: measured faster than 18 + 2 at 96
-// registers (which spilled) on every shape, and than 10, 11, 13 or 14 workers.
 #ifndef SPQT_WORKERS
-#define SPQT_WORKERS 12
+#define SPQT_WORKERS 16
 #endif
 #ifndef SPQT_DEPTH
 #define SPQT_DEPTH 3
 #endif
-constexpr int kWorkers = SPQT_WORKERS;   // compute warps
-#ifndef SPQT_WRITERS
-#define SPQT_WRITERS 2
+#ifndef SPQT_CAP
+#define SPQT_CAP 12288
 #endif
-constexpr int kWriters = SPQT_WRITERS;     // 1 or 2 writer warps; segment sg goes to writer sg % kWriters
-constexpr int kWriterWarp = kWorkers;      // the first of them
-constexpr int kGemvThreads = (kWorkers + kWriters) * 32;
+constexpr int kWorkers = SPQT_WORKERS;   // compute warps
+constexpr int kWriters = 2;              // writer warps; segment sg goes to writer sg % kWriters
+constexpr int kWriterWarp = kWorkers;    // the first of them
+constexpr int kWarps = kWorkers + kWriters;
+constexpr int kGemvThreads = kWarps * 32;
 // list entries per chunk: 2 KB of 4-bit code blocks for either group size (32 blocks of 128 rows, 64 of 64)
 __host__ __device__ constexpr int chunk_entries(int group) { return 32 * (128 / group); }
 constexpr int kDepth = SPQT_DEPTH;       // chunks in flight per warp
 constexpr unsigned long long kWaitNs = 1000000000ull;  // bound on every mbarrier wait: one second
 constexpr int kMaxCluster = 8;           // largest thread-block cluster (CTAs of one block-row) used
-constexpr int kMaxFusedN = 32768;        // largest n whose index collection can run inside the GEMV
-constexpr int kFusedCols = 16384;        // list entries (16-bit column numbers) a CTA keeps in shared memory in that case
+constexpr int kCap = SPQT_CAP;              // list entries a CTA keeps in shared memory at a time
+constexpr int kMaxListN = 65535;         // column numbers travel as 16 bits
+constexpr int kMaxFusedN = 32768;        // longest x the in-kernel scan handles (128 pieces of 256 entries)
+constexpr int kMaxPieces = kMaxFusedN / 256;
+
+enum : int { kModeList = 0, kModeFused = 1, kModeDense = 2 };
+enum : int { kFlagIdentity = 1, kFlagXs = 2 };
 
 static int g_tune_ctas = 0;  // 0 = one CTA per SM
 int g_no_pdl = 0;            // 1 = plain stream-ordered launches (also read by the index-collection launch)
 static int g_no_cluster = 0; // 1 = never launch thread-block clusters
-
-#ifdef SPQT_TRACE
-__device__ long long* g_trace;  // time stamps of CTA 0 (debug builds only)
-#define SPQT_TRACE_EVENT(cond, slot) do { if ((cond) && blockIdx.x == 0 && spqt_tr && (slot) < 4096) spqt_tr[(slot)] = clock64(); } while (0)
-#else
-#define SPQT_TRACE_EVENT(cond, slot) do { } while (0)
-#endif
 
 }  // namespace spqt
 
@@ -99,224 +105,286 @@ struct GemvSmem {
     static constexpr int CH = chunk_entries(G);
     struct Stage {
         alignas(16) unsigned char codes[CH * B];  // block e of the chunk at e*B
-        unsigned meta[3][CH];                     // words holding x_k, scale_rk, zero_rk of entry e
+        alignas(16) unsigned meta[CH];            // (scale, zero) pair of entry e
+        alignas(16) unsigned xc[CH];              // list calls: the entry word; dense call: CH fp16 values of x
     };
-    Stage stage[kWorkers][kDepth];
-    alignas(16) int cols[kWorkers][2 * kDepth][CH];  // column numbers of the chunks ahead
-    alignas(16) float red[2][kWorkers][G];               // per-warp partial sums of a finished segment
-    float red_z[2][kWorkers];                            // and their offset terms
+    Stage stage[kWorkers][kDepth];                 // (the prologue borrows this area for its copy of x and its masks)
+    alignas(16) float mult[kWorkers][CH][4];       // packed multiplier pairs of the chunk in work
+    alignas(16) float red[2][kWorkers][G];         // per-warp partial sums of a finished segment
+    float red_z[2][kWorkers];                      // and their offset terms
+    alignas(8) uint64_t full[kWorkers][kDepth];    // dense call: completion of a stage's bulk copies
     uint64_t red_full[2], red_empty[2];
     // thread-block clusters only: partial sums the other CTAs of the cluster store here (CTA rank 0)
     alignas(16) float xred[kMaxCluster][G + 4];
-    uint64_t xbar;                                       // counts their arrivals
-    // fused index collection only
-    alignas(16) int load_tot[kMaxFusedN / 256];  // active entries of every 256 entries of x
-    unsigned short fused_cols[kFusedCols];       // the part of the index list this CTA reads, when it fits (n <= 32768)
+    uint64_t xbar;                                 // counts their arrivals
+    alignas(16) int tot[kMaxPieces];               // in-kernel scan: active entries of every 256 entries of x
+    alignas(16) unsigned ent[kCap];                // the resident part of the list: x bits << 16 | column
 };
 
-// FUSED: the index collection runs in the kernel's prologue.  Every CTA copies x to shared memory and
-// scans it (each lane tests 8 entries in fp16; popc and warp reductions give the number of active
-// entries of every 256-entry piece), then expands only the pieces that overlap the list positions its
-// own slices cover: into shared memory, or, when that part is too long, into idx_out, from where it
-// reads them back like a list collected by a separate launch.  The CTAs that work on block-row 0
-// cover the whole list between them and write idx_out; CTA 0 writes the count.
-template <int G, int BITS, bool DENSE, bool ODD_N, bool FUSED, bool CLUSTER>
+struct GemvArgs {
+    const uint8_t* codes;
+    const unsigned* meta;       // (scale, zero) pairs
+    int R, n;
+    const __half* x;
+    const int32_t* idx;
+    const int32_t* count;
+    __half* y;
+    int* counters;
+    int* status;
+    unsigned long long* words;
+    float* partials;
+    float* zpartials;
+    int max_slots;
+    unsigned magic_p, magic_r;
+    int cluster_k;
+    float thr;
+    int32_t* idx_out;
+    int32_t* count_out;
+    int flags;
+};
+
+template <int G, int BITS, int MODE, bool CLUSTER>
 __global__ void __launch_bounds__(kGemvThreads, 1)
-gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales,
-                 const __half* __restrict__ zeros, int R, int n,
-                 const __half* __restrict__ x, const int32_t* idx_in,
-                 const int32_t* count_ptr, __half* __restrict__ y,
-                 int* __restrict__ counters, int* __restrict__ status,
-                 unsigned long long* __restrict__ words, float* __restrict__ partials,
-                 float* __restrict__ zpartials, int max_slots, unsigned magic_p, unsigned magic_r,
-                 int cluster_k, float thr, int32_t* idx_out, int32_t* count_out)
+gemv_kernel(const GemvArgs a)
 {
     constexpr int B = G * BITS / 8;
-    constexpr int LPB = G / 32;       // lanes that share one block (each owns 32 of its rows)
+    constexpr int LPB = G / 32;       // copies: lanes per 4-bit block (16 bytes each)
     constexpr int CB = (B % 16 == 0) ? 16 : 8;   // bytes per copy: 3-bit blocks of 64 rows are only 8-byte aligned
     static_assert(BITS == 3 || BITS == 4, "3- or 4-bit codes");
-    constexpr int SLOTS = 32 / LPB;   // blocks per 512-byte warp load
-    constexpr int KEEP = 32 / SLOTS;  // values per lane after the in-warp reduce-scatter
+    constexpr int SLOTS = 32 / LPB;   // copies: 4-bit blocks per 512-byte round
     constexpr int CH = chunk_entries(G);  // list entries per chunk
     constexpr int EPL = CH / 32;          // entries whose metadata a lane holds
-    constexpr int SUBS = CH / SLOTS;      // 512-byte loads per chunk
+    constexpr int SUBS = CH / SLOTS;      // copies: rounds per chunk
+    // arithmetic: LM lanes share a block, each owns 16 of its rows (16 accumulators per lane: half the
+    // registers of a 32-row share, which is what lets twice the warps stay resident)
+    constexpr int LM = G / 16;
+    constexpr int SLM = 32 / LM;          // blocks per step
+    constexpr int MSUBS = CH / SLM;       // steps per chunk
+    constexpr int KEEP = 16 / SLM;        // values per lane after the in-warp reduce-scatter
     constexpr int D = kDepth;
+    constexpr bool DENSE = MODE == kModeDense;
+    constexpr bool FUSED = MODE == kModeFused;
+    using Smem = GemvSmem<G, BITS>;
+    using Stage = typename Smem::Stage;
 
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    GemvSmem<G, BITS>& sm = *reinterpret_cast<GemvSmem<G, BITS>*>(smem_raw);
+    Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
 
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int tid = threadIdx.x, lane = tid & 31;
+    // the warp number through a shuffle: the compiler then knows it is the same in every lane and keeps
+    // everything derived from it (the work map, the stage addresses) in uniform registers
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
     const int P = gridDim.x, c = blockIdx.x;
-#ifdef SPQT_TRACE
-    long long* const spqt_tr = g_trace;  // one load: an event is then a clock read and a store
-#endif
-    SPQT_TRACE_EVENT(tid == 0, 3990);
-#ifdef SPQT_TRACE
-    if (tid == 0 && g_trace && c < 200) g_trace[2000 + c] = (long long)global_ns();
-#endif
-
+    const int n = a.n, R = a.R;
     if (tid == 0) {
         for (int b = 0; b < 2; ++b) {
             mbar_init(&sm.red_full[b], kWorkers);
             mbar_init(&sm.red_empty[b], 1);
         }
-        if (CLUSTER) mbar_init(&sm.xbar, cluster_k - 1);
-        if (CLUSTER) asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (DENSE) {
+            for (int w = 0; w < kWorkers; ++w)
+                for (int s = 0; s < D; ++s) mbar_init(&sm.full[w][s], 1);
+        }
+        if (CLUSTER) mbar_init(&sm.xbar, a.cluster_k - 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
     // Cluster launch (cluster_k CTAs work on one block-row and CTA rank 0 collects their sums): nobody
     // may touch another CTA's barrier before it is initialised.  Arrive now, wait much later.
     if (CLUSTER) cluster_arrive();
 
+    Piece pc;
+    pc.init_rows(R, P, c, a.magic_p, a.magic_r);
+
     // Programmatic dependent launch: this grid may have been started while the previous kernel of
-    // the stream was still draining.  Nothing above touches global memory; everything below waits
-    // for that kernel to complete, and lets the next kernel of the stream start early in turn.
+    // the stream was still draining.  Nothing above touches memory another kernel writes; everything
+    // below waits for that kernel to complete, and lets the next kernel of the stream start early in turn.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-    int count = 0;
-    if (!FUSED) count = DENSE ? n : *count_ptr;  // in flight while the row range is worked out
-    Piece pc;
-    pc.init_rows(R, P, c, magic_p, magic_r);
-    const int32_t* idx = idx_in;
-    const unsigned short* xb0 = reinterpret_cast<const unsigned short*>(x);
-    int need_lo = 0;          // FUSED: first list position held in sm.fused_cols
-    bool cols_local = false;  // FUSED: the pipeline reads its column numbers from sm.fused_cols
-    if (FUSED) {
-        // Three short loops over the 256-entry pieces of x (piece li belongs to warp li % kWarps, lane l
-        // holds entries 8l..8l+7): (1) activity mask of the lane's entries and the piece totals, four
-        // pieces per warp and round so that their loads share one round trip, (2) every warp sums the
-        // totals below its own pieces, (3) the pieces that overlap the list positions this CTA needs are
-        // expanded into column numbers.  The per-lane masks wait in shared memory that the pipeline
-        // only uses afterwards.
-        constexpr int kWarps = kGemvThreads / 32;
-        constexpr int kPiecesPerRound = 4;
-        unsigned char* pm = reinterpret_cast<unsigned char*>(smem_raw);  // per (piece, lane): activity of its 8 entries
-        using Smem = GemvSmem<G, BITS>;
-        static_assert(offsetof(Smem, red_z) >= kMaxFusedN / 8,
-                      "the prologue's scratch must fit in the part of shared memory it borrows");
-        const int nv = (n + 255) / 256;
-        for (int i = nv + tid; i < kMaxFusedN / 256; i += kGemvThreads) sm.load_tot[i] = 0;
-        const bool vec_ok = (reinterpret_cast<uintptr_t>(x) & 15) == 0;
+    // ------------------------------------------------------------ prologue: the list in shared memory
+    // Scratch borrowed from the stage area until the pipeline starts: a copy of x (16-bit words,
+    // padded to whole 256-entry pieces) and, for the in-kernel scan, one activity byte per lane and piece.
+    const int nv = (n + 255) >> 8;
+    const unsigned xs_addr = smem_u32(&sm.stage[0][0]);
+    unsigned char* const pm = reinterpret_cast<unsigned char*>(&sm.stage[0][0]) + (size_t)nv * 512;
+    const unsigned short* const xg = reinterpret_cast<const unsigned short*>(a.x);
+    const bool vec_ok = (reinterpret_cast<uintptr_t>(a.x) & 15) == 0;
+    const bool has_xs = FUSED || (a.flags & kFlagXs) != 0;
+    const unsigned ent_base = smem_u32(&sm.ent[0]);
+
+    // piece li of x (entries 256 li + 8 lane .. + 7) from global memory, zero past the end
+    auto load_piece = [&](int li) -> uint4 {
+        const int k0 = li * 256 + lane * 8;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (vec_ok && k0 + 8 <= n) {
+            v = __ldg(reinterpret_cast<const uint4*>(a.x + k0));
+        } else if (k0 < n) {
+            unsigned short hv[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) hv[e] = (k0 + e < n) ? __ldg(xg + k0 + e) : (unsigned short)0;
+            v.x = hv[0] | ((unsigned)hv[1] << 16);
+            v.y = hv[2] | ((unsigned)hv[3] << 16);
+            v.z = hv[4] | ((unsigned)hv[5] << 16);
+            v.w = hv[6] | ((unsigned)hv[7] << 16);
+        }
+        return v;
+    };
+
+    // Copy x to shared memory; the in-kernel scan also records which entries are active and how many
+    // per piece.  Run by the warps gw = 0..NW-1 of a group; the caller synchronises the group afterwards.
+    auto stage_x = [&](int gw, int NW) {
+        constexpr int kPiecesPerRound = 4;   // loads of one round share a round trip
         // the largest fp16 value not above t (any negative value if t < 0: everything but NaN is
         // active; +inf if t is NaN or +inf: nothing is)
+        const float thr = a.thr;
         const __half thr_h = (thr != thr) ? __ushort_as_half((unsigned short)0x7c00)
                                           : (thr < 0.0f ? __float2half_rn(-1.0f) : __float2half_rd(thr));
         const __half2 thr_h2 = __half2half2(thr_h);
-        SPQT_TRACE_EVENT(tid == 0, 3991);
+        if (FUSED) {
+            for (int i = nv + gw * 32 + lane; i < kMaxPieces; i += NW * 32) sm.tot[i] = 0;
+        }
 #pragma unroll 1
-        for (int l0 = warp; l0 < nv; l0 += kPiecesPerRound * kWarps) {
+        for (int l0 = gw; l0 < nv; l0 += kPiecesPerRound * NW) {
             uint4 xv[kPiecesPerRound];
 #pragma unroll
             for (int j = 0; j < kPiecesPerRound; ++j) {
-                const int li = l0 + j * kWarps, k0 = li * 256 + lane * 8;
+                const int li = l0 + j * NW;
                 xv[j] = make_uint4(0u, 0u, 0u, 0u);
-                if (li < nv) {  // uniform across the warp
-                    if (vec_ok && k0 + 8 <= n) {
-                        xv[j] = __ldg(reinterpret_cast<const uint4*>(x + k0));
-                    } else {
-                        unsigned short hv[8];
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) hv[e] = (k0 + e < n) ? __ldg(xb0 + k0 + e) : (unsigned short)0;
-                        xv[j].x = hv[0] | ((unsigned)hv[1] << 16);
-                        xv[j].y = hv[2] | ((unsigned)hv[3] << 16);
-                        xv[j].z = hv[4] | ((unsigned)hv[5] << 16);
-                        xv[j].w = hv[6] | ((unsigned)hv[7] << 16);
-                    }
-                }
+                if (li < nv) xv[j] = load_piece(li);  // uniform across the warp
             }
 #pragma unroll
             for (int j = 0; j < kPiecesPerRound; ++j) {
-                const int li = l0 + j * kWarps, k0 = li * 256 + lane * 8;
+                const int li = l0 + j * NW, k0 = li * 256 + lane * 8;
                 if (li < nv) {
-                    const unsigned wds[4] = {xv[j].x, xv[j].y, xv[j].z, xv[j].w};
-                    unsigned m8 = 0;
+                    sts_v4(xs_addr + (unsigned)li * 512u + (unsigned)lane * 16u, xv[j]);
+                    if (FUSED) {
+                        const unsigned wds[4] = {xv[j].x, xv[j].y, xv[j].z, xv[j].w};
+                        unsigned m8 = 0;
 #pragma unroll
-                    for (int e2 = 0; e2 < 4; ++e2) {
-                        // |x| > t  <=>  |x| > (largest fp16 value <= t): two entries per compare, in fp16,
-                        // exact; the ordered compare is false for NaN
-                        const unsigned ab = wds[e2] & 0x7fff7fffu;
-                        const unsigned gt = __hgt2_mask(*reinterpret_cast<const __half2*>(&ab), thr_h2);
-                        m8 |= (gt & (1u << (2 * e2))) | (gt & (0x20000u << (2 * e2))) >> 16;
+                        for (int e2 = 0; e2 < 4; ++e2) {
+                            // |x| > t  <=>  |x| > (largest fp16 value <= t): two entries per compare, in fp16,
+                            // exact; the ordered compare is false for NaN
+                            const unsigned ab = wds[e2] & 0x7fff7fffu;
+                            const unsigned gt = __hgt2_mask(*reinterpret_cast<const __half2*>(&ab), thr_h2);
+                            m8 |= (gt & (1u << (2 * e2))) | (gt & (0x20000u << (2 * e2))) >> 16;
+                        }
+                        const int left = n - k0;  // entries of this lane that exist
+                        if (left < 8) m8 &= (left <= 0) ? 0u : ((1u << left) - 1u);
+                        pm[li * 32 + lane] = (unsigned char)m8;
+                        const unsigned tot = __reduce_add_sync(0xffffffffu, (unsigned)__popc(m8));
+                        if (lane == 0) sm.tot[li] = (int)tot;
                     }
-                    const int left = n - k0;  // entries of this lane that exist
-                    if (left < 8) m8 &= (left <= 0) ? 0u : ((1u << left) - 1u);
-                    pm[li * 32 + lane] = (unsigned char)m8;
-                    const unsigned tot = __reduce_add_sync(0xffffffffu, (unsigned)__popc(m8));
-                    if (lane == 0) sm.load_tot[li] = (int)tot;
                 }
             }
         }
-        __syncthreads();
-        SPQT_TRACE_EVENT(tid == 0, 3992);
-        // (2) every warp for itself: lane l holds the totals of pieces 4l..4l+3; sums over the pieces
-        // below a given one come from one warp reduction each
-        int tot4[4];
-        {
-            const int4 t4 = *reinterpret_cast<const int4*>(&sm.load_tot[lane * 4]);  // zero past nv (cleared below)
-            tot4[0] = t4.x; tot4[1] = t4.y; tot4[2] = t4.z; tot4[3] = t4.w;
-        }
-        count = (int)__reduce_add_sync(0xffffffffu, (unsigned)(tot4[0] + tot4[1] + tot4[2] + tot4[3]));
-        SPQT_TRACE_EVENT(tid == 0, 3993);
-        pc.set_count(count);
-        if (c == 0 && tid == 0) *count_out = count;
-        // list positions this CTA will read: the union of its slices.  If that part fits in shared
-        // memory the pipeline takes its column numbers from there (no round trip through global
-        // memory); otherwise they go to idx_out and come back like a list collected by a separate launch.
-        // (A piece that spans several block-rows ends the first one and begins the last one: its slices
-        // cover the whole list between them.)
-        need_lo = 0;
-        int need_hi = count;
-        if (pc.r_first == pc.r_last) pc.slice(pc.r_first, &need_lo, &need_hi);
-        cols_local = (need_hi - need_lo) <= kFusedCols;
-        const unsigned need_len = (unsigned)max(need_hi - need_lo, 0);
-        const unsigned fc0 = smem_u32(&sm.fused_cols[0]);
-        SPQT_TRACE_EVENT(tid == 0, 3994);
-        // (3) the pieces that overlap [need_lo, need_hi): prefix sums over the lanes, then one
-        // predicated store per entry (a divergent branch per entry would cost far more than the store)
+    };
+
+    // The window [lo, hi) of the list into sm.ent, by the threads gt = 0..NT-1 (warps gw = 0..NW-1) of
+    // a group.  The in-kernel scan also writes the list positions [olo, ohi) of the index list the
+    // call returns.  The caller synchronises the group before (x staged) and afterwards.
+    auto build_window = [&](int lo, int hi, int olo, int ohi, int gw, int NW) {
+        if (FUSED) {
+            // lane l holds the totals of pieces 4l..4l+3; sums over the pieces below a given one come
+            // from one warp reduction each
+            int tot4[4];
+            {
+                const int4 t4 = *reinterpret_cast<const int4*>(&sm.tot[lane * 4]);
+                tot4[0] = t4.x; tot4[1] = t4.y; tot4[2] = t4.z; tot4[3] = t4.w;
+            }
+            const unsigned len = (unsigned)max(hi - lo, 0), olen = (unsigned)max(ohi - olo, 0);
 #pragma unroll 1
-        for (int li = warp; li < nv; li += kWarps) {
-            unsigned below = 0;  // active entries of this lane's pieces that come before piece li
+            for (int li = gw; li < nv; li += NW) {
+                unsigned below = 0;  // active entries of this lane's pieces that come before piece li
 #pragma unroll
-            for (int q = 0; q < 4; ++q) below += (lane * 4 + q < li) ? (unsigned)tot4[q] : 0u;
-            const int base = (int)__reduce_add_sync(0xffffffffu, below);
-            const int q = li & 3;
-            const int tsel = q == 0 ? tot4[0] : q == 1 ? tot4[1] : q == 2 ? tot4[2] : tot4[3];
-            const int end = base + __shfl_sync(0xffffffffu, tsel, li >> 2);
-            if (end <= need_lo || base >= need_hi) continue;  // uniform across the warp
-            const unsigned m8 = pm[li * 32 + lane];
-            const int c8 = __popc(m8);
-            int incl = c8;
+                for (int q = 0; q < 4; ++q) below += (lane * 4 + q < li) ? (unsigned)tot4[q] : 0u;
+                const int base = (int)__reduce_add_sync(0xffffffffu, below);
+                const int q = li & 3;
+                const int tsel = q == 0 ? tot4[0] : q == 1 ? tot4[1] : q == 2 ? tot4[2] : tot4[3];
+                const int end = base + __shfl_sync(0xffffffffu, tsel, li >> 2);
+                const bool in_win = end > lo && base < hi, in_out = end > olo && base < ohi;
+                if (!in_win && !in_out) continue;  // uniform across the warp
+                const unsigned m8 = pm[li * 32 + lane];
+                const uint4 xv = lds_v4(xs_addr + (unsigned)li * 512u + (unsigned)lane * 16u);
+                const unsigned xw[4] = {xv.x, xv.y, xv.z, xv.w};
+                const int c8 = __popc(m8);
+                int incl = c8;
 #pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int up = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += up;
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int up = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += up;
+                }
+                int pos = base + incl - c8;
+                const int col0 = li * 256 + lane * 8;
+                // one predicated store per entry (a divergent branch per entry would cost far more)
+                if (in_win) {
+                    int p2 = pos;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const unsigned on = (m8 >> e) & 1u, d = (unsigned)(p2 - lo);
+                        const unsigned xb = (e & 1) ? (xw[e >> 1] & 0xffff0000u) : (xw[e >> 1] << 16);
+                        st_shared_u32_if(on & (d < len ? 1u : 0u), ent_base + 4u * d, xb | (unsigned)(col0 + e));
+                        p2 += (int)on;
+                    }
+                }
+                if (in_out) {
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const unsigned on = (m8 >> e) & 1u, d = (unsigned)(pos - olo);
+                        st_global_if(on & (d < olen ? 1u : 0u), a.idx_out + pos, col0 + e);
+                        pos += (int)on;
+                    }
+                }
             }
-            int pos = base + incl - c8;
-            const int col0 = li * 256 + lane * 8;
-            if (cols_local) {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const unsigned on = (m8 >> e) & 1u, d = (unsigned)(pos - need_lo);
-                    st_shared_u16_if(on & (d < need_len ? 1u : 0u), fc0 + 2u * d, col0 + e);
-                    pos += (int)on;
-                }
-            } else {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const unsigned on = (m8 >> e) & 1u, d = (unsigned)(pos - need_lo);
-                    st_global_if(on & (d < need_len ? 1u : 0u), idx_out + pos, col0 + e);
-                    pos += (int)on;
-                }
+        } else if (!DENSE) {
+            const bool identity = (a.flags & kFlagIdentity) != 0;
+            const int NT = NW * 32, gt = gw * 32 + lane;
+#pragma unroll 4
+            for (int i = gt; i < hi - lo; i += NT) {
+                const unsigned col = identity ? (unsigned)(lo + i) : (unsigned)__ldg(a.idx + lo + i);
+                const unsigned xb = has_xs ? lds_u16(xs_addr + 2u * col) : (unsigned)__ldg(xg + col);
+                sm.ent[i] = (xb << 16) | col;
             }
         }
-        SPQT_TRACE_EVENT(lane == 0, 3960 + warp);
-        __syncthreads();  // the CTA's own writes (shared or global) are visible to its pipeline
-        idx = idx_out;
+    };
+
+    int count = 0;
+    bool resident = true;
+    int win_lo = 0;  // list position of sm.ent[0]
+    if (DENSE) {
+        count = n;
+        pc.set_count(n, 8);
     } else {
+        if (!FUSED) count = (a.flags & kFlagIdentity) ? n : __ldg(a.count);  // in flight while x is staged
+        if (has_xs) stage_x(warp, kWarps);
+        __syncthreads();
+        if (FUSED) {
+            const int4 t4 = *reinterpret_cast<const int4*>(&sm.tot[lane * 4]);
+            count = (int)__reduce_add_sync(0xffffffffu, (unsigned)(t4.x + t4.y + t4.z + t4.w));
+            if (c == 0 && tid == 0) *a.count_out = count;
+        }
         pc.set_count(count);
+        // list positions this CTA will read: the union of its slices.  (A piece that spans several
+        // block-rows ends the first one and begins the last one: its slices cover the whole list
+        // between them.)
+        int need_lo = 0, need_hi = count;
+        if (pc.r_first == pc.r_last) pc.slice(pc.r_first, &need_lo, &need_hi);
+        resident = (need_hi - need_lo) <= kCap;
+        int olo = 0, ohi = 0;  // the part of the returned index list this CTA writes: its slice of block-row 0
+        if (FUSED && pc.r_first == 0) pc.slice(0, &olo, &ohi);
+        if (resident) {
+            win_lo = need_lo;
+            build_window(need_lo, need_hi, olo, ohi, warp, kWarps);
+        } else {
+            // the window of the first span; the workers rebuild it for every later span
+            int p0, p1;
+            pc.slice(pc.r_first, &p0, &p1);
+            win_lo = p0;
+            const int whi = min(p1, p0 + kCap);
+            build_window(p0, whi, max(olo, p0), min(ohi, whi), warp, kWarps);
+        }
+        __syncthreads();  // the list is in place; the stage area is free for the pipeline
     }
-    SPQT_TRACE_EVENT(tid == 0, 4000);
     if (CLUSTER) cluster_wait();  // every CTA of the cluster has initialised its barriers by now
 
     if (warp >= kWriterWarp) {
@@ -326,19 +394,15 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
         constexpr int RPL = G / 32;  // rows per lane
         constexpr int kStride = G + 2;  // words per contributing CTA: G sums, the offset term, one of padding
         const int wr = warp - kWriterWarp;
+        __half* const y = a.y;
+        int* const counters = a.counters;
         bool ok = true;
-        if (FUSED && cols_local && pc.r_first == 0) {
-            // this CTA's slice of block-row 0 is its part of the index list the call returns
-            int p0, p1;
-            pc.slice(0, &p0, &p1);
-            for (int i = p0 + wr * 32 + lane; i < p1; i += 32 * kWriters) idx_out[i] = sm.fused_cols[i - need_lo];
-        }
         for (int r = pc.r_first + wr, sg = wr; r <= pc.r_last; r += kWriters, sg += kWriters) {
             const int b = sg & 1;  // hand-over buffer of this segment
             int first, nslots;
             pc.contributors(r, &first, &nslots);
             const int mine = c - first;
-            unsigned long long* const row_words = words + (size_t)r * kTagSlots * kStride;
+            unsigned long long* const row_words = a.words + (size_t)r * kTagSlots * kStride;
             // A block-row that is not the CTA's first is shared with CTAs that work on it first and are
             // done long before this one.  While the workers are still computing, watch for their words
             // (one word per CTA as a cheap hint, at a low rate).  Once all of them are there, this CTA
@@ -373,9 +437,9 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
                         if (spec) break;
                     }
                     if (mbar_test(&sm.red_full[b], (sg >> 1) & 1)) break;  // own sums are ready: stop watching
-                    if (it == 64) t0 = global_ns();
-                    if (it > 64 && global_ns() - t0 > kWaitNs) break;
-                    __nanosleep(100);
+                    if (it == 0) t0 = global_ns();
+                    else if (global_ns() - t0 > kWaitNs) break;
+                    __nanosleep(400);   // a look every fraction of a microsecond: the watching must not take issue slots from the workers
                 }
                 if (spec) {
 #pragma unroll
@@ -423,7 +487,7 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
 #pragma unroll
                 for (int i = 0; i < RPL; ++i) t[i] += v[i];
                 zsum += zpart;
-                for (int s = 1; s < cluster_k; ++s) {
+                for (int s = 1; s < a.cluster_k; ++s) {
 #pragma unroll
                     for (int i = 0; i < RPL; ++i) t[i] += sm.xred[s][lane * RPL + i];
                     zsum += sm.xred[s][G];
@@ -497,10 +561,10 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
             } else {
                 // many contributors: plain fp32 partials in a region of their own, a fence, and the
                 // counter; the last to arrive reads eight slots at a time
-                const size_t pslot = (size_t)r * max_slots + mine;
+                const size_t pslot = (size_t)r * a.max_slots + mine;
 #pragma unroll
-                for (int i = 0; i < RPL; ++i) __stcg(partials + pslot * G + lane * RPL + i, v[i]);
-                if (lane == 0) __stcg(zpartials + pslot, zpart);
+                for (int i = 0; i < RPL; ++i) __stcg(a.partials + pslot * G + lane * RPL + i, v[i]);
+                if (lane == 0) __stcg(a.zpartials + pslot, zpart);
                 __threadfence();
                 __syncwarp();
                 int prev = 0;
@@ -508,8 +572,8 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
                 prev = __shfl_sync(0xffffffffu, prev, 0);
                 if (prev != nslots - 1) continue;
                 __threadfence();
-                const float* p = partials + (size_t)r * max_slots * G + lane * RPL;
-                const float* zp = zpartials + (size_t)r * max_slots;
+                const float* p = a.partials + (size_t)r * a.max_slots * G + lane * RPL;
+                const float* zp = a.zpartials + (size_t)r * a.max_slots;
                 for (int s0 = 0; s0 < nslots; s0 += 8) {
                     float pv[8][RPL], pz[8];
 #pragma unroll
@@ -548,283 +612,270 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
                 else counters[r] = 0;
             }
         }
-        SPQT_TRACE_EVENT(lane == 0, 4002);
-#ifdef SPQT_TRACE
-        if (lane == 0 && g_trace && c < 200) g_trace[2200 + c] = (long long)global_ns();
-#endif
-        if (!ok && lane == 0) atomicExch(status, 1);
+        if (!ok && lane == 0) atomicExch(a.status, 1);
         return;
     }
 
     // ---------------------------------------------------------------- workers
     // Everything the loop touches in shared memory is addressed with 32-bit shared addresses kept in
-    // registers (ring positions are byte offsets that wrap), and entries past the end of a slice are
-    // handled by clamping the entry number (they re-read the slice's last entry and get weight 0)
-    // rather than by branches: the loop is bound by instruction issue.
-    using Stage = typename GemvSmem<G, BITS>::Stage;
+    // registers, and the control around a chunk is kept to a handful of instructions: the loop is
+    // bound by instruction issue and by the half-rate integer pipe, so every instruction outside the
+    // arithmetic counts.  Per chunk k of a warp: ISSUE(k) the copies; once they have landed PREP(k),
+    // the multipliers of its entries; MATH(k); then ISSUE(k+D) into the stage MATH(k) has freed.
     constexpr unsigned kStageBytes = (unsigned)sizeof(Stage);
-    constexpr unsigned kMetaOff = (unsigned)(CH * B);     // offset of Stage::meta
-    constexpr unsigned kColsBytes = CH * 4;               // one chunk of column numbers
-    static_assert(offsetof(Stage, meta) == kMetaOff, "stage layout");
-    const int slot = lane / LPB, h = lane % LPB;
-    const unsigned short* xb = reinterpret_cast<const unsigned short*>(x);
+    constexpr unsigned kMetaOff = (unsigned)offsetof(Stage, meta);
+    constexpr unsigned kXcOff = (unsigned)offsetof(Stage, xc);
+    const int slot = lane / LPB, h = lane % LPB;   // copies
+    const int mslot = lane / LM, mh = lane % LM;   // arithmetic
     const unsigned stage_base = smem_u32(&sm.stage[warp][0]);
-    const unsigned cols_base = smem_u32(&sm.cols[warp][0][0]);
-    const unsigned fused_base = smem_u32(&sm.fused_cols[0]) - 2u * (unsigned)need_lo;  // + 2 * list position
-    const bool use_list = !DENSE && !(FUSED && cols_local);  // column numbers come through stage A
+    const unsigned mult_base = smem_u32(&sm.mult[warp][0][0]);
+    const unsigned full_base = smem_u32(&sm.full[warp][0]);
+    const unsigned lane0 = lane == 0 ? 1u : 0u;
 
-    // column number of entry e of a chunk: 32-bit entries in the stage-A ring, 16-bit ones in the list
-    // the fused prologue keeps
-    auto col_at = [&](unsigned chunk_addr, int e) -> unsigned {
-        if (!FUSED || use_list) return lds_u32(chunk_addr + 4u * e);
-        return lds_u16(chunk_addr + 2u * e);
+    // block-row constants of the issue side, refreshed when it enters a new block-row
+    const uint8_t* b_codes = nullptr;   // codes of the block-row (list calls: this lane's 16-byte part)
+    const unsigned* b_meta = nullptr;   // (scale, zero) pairs of the block-row
+    auto enter_row = [&](int r) {
+        const size_t row_base = (size_t)r * (size_t)n;
+        b_codes = a.codes + row_base * B + ((!DENSE && BITS == 4) ? 16 * h : 0);
+        b_meta = a.meta + row_base;
     };
 
-    Cursor ca, cb;  // stage A / stage B cursors (the consume side walks the segments itself)
-    ca.init(pc, warp, CH);
-    cb = ca;
-    // Ring positions (byte offsets) of the chunk stage C works on: rc_s in the ring of D stages, rc_c
-    // in the ring of 2*D chunks of column numbers, rb_c = D chunks further in that ring.  Stage B
-    // refills the stage slot C has just read and takes its columns from rb_c; stage A refills rc_c.
-    unsigned rc_s = 0, rc_c = 0, rb_c = D * kColsBytes;
-    auto wrap = [](unsigned& v, unsigned step, unsigned len) { v = (v + step == len) ? 0u : v + step; };
-
-    // block-row constants of stage B, refreshed when its cursor enters a new block-row
-    int b_row = -1;
-    unsigned b_par = 0;                       // parity of r*n: which half of a word holds element (r,k)
-    const uint8_t* b_codes = nullptr;         // codes of the block-row, this lane's 16-byte part
-    const unsigned short* b_scales = nullptr; // scales / zeros of the block-row
-    const unsigned short* b_zeros = nullptr;
-
-    // stage A: column numbers of the warp's next chunk
-    auto issue_a = [&](unsigned ring_c) {
-        if (use_list && ca.valid(pc)) {
+    // the list words of the entries a lane handles in the chunk at list position pos (FULL: all CH
+    // entries exist; else the entries past the end of the part read the part's last entry again)
+    auto load_entries = [&](int pos, int valid, bool full, unsigned* ev) {
+        const unsigned ent_addr = ent_base + 4u * (unsigned)(pos - win_lo);
 #pragma unroll
-            for (int q = 0; q < EPL; ++q) {
-                const int e = lane + 32 * q;
-                if (ca.pos + e < ca.p1) cp_async_4(cols_base + ring_c + 4u * e, idx + ca.pos + e);
-            }
-            ca.advance(pc, warp);
-        }
-    };
-    // stage B: code blocks and metadata words of the next chunk (its column numbers have landed)
-    // (pre: column numbers of the copies and of the lane's metadata entry, read ahead of time by prep_b,
-    // or nullptr to read them here)
-    auto issue_b = [&](unsigned ring_s, unsigned ring_c, const unsigned* pre) {
-        if (cb.valid(pc)) {
-            if (cb.r != b_row) {
-                b_row = cb.r;
-                const size_t row_base = (size_t)b_row * (size_t)n;
-                b_par = ODD_N ? (unsigned)(row_base & 1) : 0u;  // n even: every block-row starts on a word
-                b_codes = codes + row_base * B + (BITS == 4 ? 16 * h : 0);
-                b_scales = reinterpret_cast<const unsigned short*>(scales) + row_base;
-                b_zeros = reinterpret_cast<const unsigned short*>(zeros) + row_base;
-            }
-            const int vm1 = min(cb.p1 - cb.pos, CH) - 1;  // last entry of this chunk that exists
-            // address of the chunk's first column number (unused when DENSE)
-            const unsigned cols_addr = use_list ? cols_base + ring_c : fused_base + 2u * (unsigned)cb.pos;
-            const unsigned st_addr = stage_base + ring_s;
-            if (BITS == 4) {
-#pragma unroll
-                for (int u = 0; u < SUBS; ++u) {
-                    const int e = min(u * SLOTS + slot, vm1);
-                    const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : (pre ? pre[u] : col_at(cols_addr, e));
-                    if (DENSE) cp_async_16(st_addr + lane * 16 + u * 512, b_codes + (size_t)kk * B);
-                    else cp_async_16_l2_64(st_addr + lane * 16 + u * 512, b_codes + (size_t)kk * B);
-                }
-            } else {
-                // 3-bit blocks (48 or 24 bytes): the chunk's bytes in copies of CB bytes, lane after lane
-                constexpr int NC = CH * B / CB / 32;
-#pragma unroll
-                for (int q = 0; q < NC; ++q) {
-                    const int off = (q * 32 + lane) * CB;    // byte offset inside the chunk's stage
-                    const int e = min(off / B, vm1), part = off % B;
-                    const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : col_at(cols_addr, e);
-                    const uint8_t* src = b_codes + (size_t)kk * B + part;
-                    if (CB == 16) {
-                        if (DENSE) cp_async_16(st_addr + off, src);
-                        else cp_async_16_l2_64(st_addr + off, src);
-                    } else {
-                        cp_async_8(st_addr + off, src);
-                    }
-                }
-            }
-#pragma unroll
-            for (int q = 0; q < EPL; ++q) {
-                // the aligned 4-byte word that holds each fp16 value (index rounded down to even)
-                const int e = min(lane + 32 * q, vm1);
-                const unsigned kk = DENSE ? (unsigned)(cb.pos + e) : ((pre && BITS == 4) ? pre[SUBS + q] : col_at(cols_addr, e));
-                const unsigned mdst = st_addr + kMetaOff + 4u * (lane + 32 * q);
-                const int mo = (int)kk - (int)((kk ^ b_par) & 1u);  // may be -1 only when r*n is odd: still inside the array
-                if (!ODD_N || kk != (unsigned)(n - 1)) {
-                    cp_async_4_ca(mdst, xb + (kk & ~1u));
-                    cp_async_4(mdst + CH * 4, b_scales + mo);
-                    cp_async_4(mdst + 2 * CH * 4, b_zeros + mo);
-                } else {
-                    // n odd: the word of the last column may reach past the end of an array; fetch directly
-                    sts_u32(mdst, (unsigned)__ldg(xb + kk) << ((kk & 1u) * 16));
-                    sts_u32(mdst + CH * 4, (unsigned)__ldg(b_scales + kk) << (((kk ^ b_par) & 1u) * 16));
-                    sts_u32(mdst + 2 * CH * 4, (unsigned)__ldg(b_zeros + kk) << (((kk ^ b_par) & 1u) * 16));
-                }
-            }
-            cb.advance(pc, warp);
+        for (int q = 0; q < EPL; ++q) {
+            const int e = lane + 32 * q;
+            ev[q] = lds_u32(ent_addr + 4u * (unsigned)(full ? e : min(e, valid - 1)));
         }
     };
 
-    // The column numbers stage B will need at the end of this iteration, read before the arithmetic so
-    // that the shared-memory latency hides under it (4-bit sparse path only).
-    auto prep_b = [&](unsigned ring_c, unsigned* pre) {
-        if (!DENSE && BITS == 4 && cb.valid(pc)) {
-            const int vm1 = min(cb.p1 - cb.pos, CH) - 1;
-            const unsigned cols_addr = use_list ? cols_base + ring_c : fused_base + 2u * (unsigned)cb.pos;
-#pragma unroll
-            for (int u = 0; u < SUBS; ++u) pre[u] = col_at(cols_addr, min(u * SLOTS + slot, vm1));
-#pragma unroll
-            for (int q = 0; q < EPL; ++q) pre[SUBS + q] = col_at(cols_addr, min(lane + 32 * q, vm1));
+    // ISSUE: the copies of one chunk (entries pos .. pos+valid-1 of the current block-row's list) into a stage
+    auto issue = [&](int pos, int valid, bool full, unsigned st_addr, unsigned bar_addr) {
+        if (DENSE) {
+            // the chunk's blocks, pairs and x values are contiguous: three bulk copies by one lane
+            mbar_expect_tx_if(lane0, bar_addr, (unsigned)valid * (B + 6));
+            bulk_copy_if(lane0, st_addr, b_codes + (size_t)pos * B, (unsigned)valid * B, bar_addr);
+            bulk_copy_if(lane0, st_addr + kMetaOff, b_meta + pos, (unsigned)valid * 4, bar_addr);
+            bulk_copy_if(lane0, st_addr + kXcOff, a.x + pos, (unsigned)valid * 2, bar_addr);
+            return;
         }
-    };
-
-    // fill the pipeline: D chunks of columns, then D chunks of blocks (each needs its columns)
-#pragma unroll 1
-    for (int s = 0; s < D; ++s) {
-        issue_a(s * kColsBytes);
-        cp_async_commit();
-    }
-#pragma unroll 1
-    for (int s = 0; s < D; ++s) {
-        cp_async_wait<D - 1>();
-        __syncwarp();
-        issue_b(s * kStageBytes, s * kColsBytes, nullptr);
-        issue_a((D + s) * kColsBytes);
-        cp_async_commit();
-    }
-
-    unsigned long long acc[16];  // 32 fp32 sums, two per register
+        unsigned col[EPL];
+        load_entries(pos, valid, full, col);
 #pragma unroll
-    for (int i = 0; i < 16; ++i) acc[i] = 0ull;
-    bool ok = true;
-#ifdef SPQT_TRACE
-    long long tr_wait = 0, tr_issue = 0, tr_math = 0, tr_n = 0;
-    SPQT_TRACE_EVENT(lane == 0, 3900 + warp);
-#endif
-
-    for (int r = pc.r_first, sg = 0; r <= pc.r_last; ++r, ++sg) {
-        int p0, p1;
-        pc.slice(r, &p0, &p1);
-        const unsigned c_par = ODD_N ? (unsigned)(((size_t)r * (size_t)n) & 1) : 0u;
-        float zl = 0.0f;  // this lane's share of sum x_k * zero_rk
-        for (int pos = p0 + warp * CH; pos < p1; pos += kWorkers * CH) {
-            // ---- stage C of the oldest chunk: everything it needs is in commit groups that wait<D-1> covers
-#ifdef SPQT_TRACE
-            const long long tc0 = clock64();
-#endif
-            cp_async_wait<D - 1>();
-            __syncwarp();
-#ifdef SPQT_TRACE
-            const long long tc1 = clock64();
-#endif
-            unsigned pre[SUBS + EPL];
-            prep_b(rb_c, pre);
-            const unsigned st_addr = stage_base + rc_s;
-#ifdef SPQT_TRACE
-            const long long tc2 = clock64();
-#endif
-            float a[EPL];  // x_k * scale_rk of the entries this lane holds (entry lane + 32 q)
-#pragma unroll
-            for (int q = 0; q < EPL; ++q) {
-                const unsigned xw = lds_u32(st_addr + kMetaOff + 4u * (lane + 32 * q));
-                const unsigned sw = lds_u32(st_addr + kMetaOff + 4u * (lane + 32 * q) + CH * 4);
-                const unsigned zw = lds_u32(st_addr + kMetaOff + 4u * (lane + 32 * q) + 2 * CH * 4);
-                const int e = min(lane + 32 * q, p1 - pos - 1);  // the entry whose metadata this lane holds
-                unsigned kk;
-                if (DENSE) kk = (unsigned)(pos + e);
-                else kk = col_at(use_list ? cols_base + rc_c : fused_base + 2u * (unsigned)pos, e);
-                const unsigned xs = (kk & 1u) * 16, ms = ((kk ^ c_par) & 1u) * 16;
-                const float xf = __half2float(__ushort_as_half((unsigned short)(xw >> xs)));
-                const float sf = __half2float(__ushort_as_half((unsigned short)(sw >> ms)));
-                const float zf = __half2float(__ushort_as_half((unsigned short)(zw >> ms)));
-                const float xin = (e == lane + 32 * q) ? xf : 0.0f;  // 0 past the end of the slice
-                a[q] = xin * sf;                                      // exact
-                zl = fmaf(xin, zf, zl);
-            }
+        for (int q = 0; q < EPL; ++q) {
+            col[q] &= 0xffffu;
+            cp_async_4(st_addr + kMetaOff + 4u * (lane + 32 * q), b_meta + col[q]);
+        }
+        if (BITS == 4) {
+            // (steps past the end of the part copy the part's last block again: an L2 hit, and no branch)
 #pragma unroll
             for (int u = 0; u < SUBS; ++u) {
-                const float au = __shfl_sync(0xffffffffu, a[(u * SLOTS) / 32], (u * SLOTS + slot) & 31);
-                if (BITS == 4) {
-                    const uint4 wv = lds_v4(st_addr + lane * 16 + u * 512);
-                    fma_block16(acc, wv, au);
-                } else {
-                    // lane h of a block: words h and h+LPB of the 2-bit plane, word h of the 1-bit plane
-                    const unsigned blk = st_addr + (u * SLOTS + slot) * B + 4u * h;
-                    fma_block3(acc, lds_u32(blk), lds_u32(blk + 4u * LPB), lds_u32(blk + 8u * LPB), au);
-                }
+                const unsigned cu = __shfl_sync(0xffffffffu, col[(u * SLOTS) / 32], (u * SLOTS + slot) & 31);
+                cp_async_16_l2_64(st_addr + lane * 16 + u * 512, b_codes + (size_t)cu * B);
             }
-            __syncwarp();  // every lane has read its part of the slots that B and A now refill
-            issue_b(rc_s, rb_c, (!DENSE && BITS == 4) ? pre : nullptr);
-            issue_a(rc_c);
-            cp_async_commit();
-            wrap(rc_s, kStageBytes, D * kStageBytes);
-            wrap(rc_c, kColsBytes, 2 * D * kColsBytes);
-            wrap(rb_c, kColsBytes, 2 * D * kColsBytes);
-#ifdef SPQT_TRACE
-            tr_wait += tc1 - tc0; tr_issue += 0; tr_math += clock64() - tc2; ++tr_n;
-#endif
-        }
-
-        // ---- end of the segment: in-warp reduce-scatter over the column slots, then hand the
-        // per-warp sums to the writer warp
-        const int b = sg & 1;
-        if (sg >= 2) {
-            ok = mbar_wait(&sm.red_empty[b], ((sg >> 1) - 1) & 1);
-            if (!ok) break;
-        }
-        float accf[32];
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            unpack2(acc[i], accf[2 * i], accf[2 * i + 1]);
-            acc[i] = 0ull;
-        }
-        float t16[16], t8[8], t4[4], keep[4];
-        halve<32>(accf, t16, lane, 16);
-        halve<16>(t16, t8, lane, 8);
-        halve<8>(t8, t4, lane, 4);
-        int a_base;
-        if (LPB == 4) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) keep[i] = t4[i];
-            a_base = lane & 0x1c;
         } else {
-            float t2[2];
-            halve<4>(t4, t2, lane, 2);
-            keep[0] = t2[0];
-            keep[1] = t2[1];
-            a_base = lane & 0x1e;
-        }
+            // 3-bit blocks (48 or 24 bytes): the chunk's bytes in copies of CB bytes, lane after lane
+            constexpr int NC = CH * B / CB / 32;
 #pragma unroll
-        for (int i = 0; i < KEEP; ++i) {
-            const int ai = a_base + i;  // accumulator index = word*8 + nibble
-            const int cw = ai >> 3, e2 = ai & 7;
-            const int row = (BITS == 4)
-                                ? 16 * h + 4 * cw + (e2 >> 1) + (e2 & 1) * (G / 2)
-                                : 4 * h + (e2 >> 1) + (G / 8) * (cw >> 1) + (G / 4) * ((cw & 1) + 2 * (e2 & 1));
-            sm.red[b][warp][row] = keep[i] * 0x1p56f;  // undo the 2^-56 of the subnormal trick
+            for (int q = 0; q < NC; ++q) {
+                const int off = (q * 32 + lane) * CB;    // byte offset inside the chunk's stage
+                const int e = off / B, part = off % B;
+                const unsigned cu = __shfl_sync(0xffffffffu, col[(q * 32 * CB / B) / 32], e & 31);
+                const uint8_t* src = b_codes + (size_t)cu * B + part;
+                if (CB == 16) cp_async_16_l2_64(st_addr + off, src);
+                else cp_async_8(st_addr + off, src);
+            }
         }
+    };
+
+    unsigned long long acc[8];  // 16 fp32 sums, two per register
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) zl += __shfl_xor_sync(0xffffffffu, zl, o);
-        if (lane == 0) sm.red_z[b][warp] = zl;
-        __syncwarp();
-        SPQT_TRACE_EVENT(tid == 0, 3950 + sg);
-        if (lane == 0) mbar_arrive(&sm.red_full[b]);
+    for (int i = 0; i < 8; ++i) acc[i] = 0ull;
+    float zl = 0.0f;     // this lane's share of sum x_k * zero_rk of the current segment
+
+    // PREP: lane e turns the pair of its entry into a = x_k*scale (exact in fp32), written as two packed
+    // multiplier pairs, and adds x_k*zero to its share of the offset term
+    auto prep = [&](unsigned st_addr, int pos, int valid, bool full) {
+        unsigned ev[EPL];
+        if (!DENSE) load_entries(pos, valid, full, ev);
+#pragma unroll
+        for (int q = 0; q < EPL; ++q) {
+            const int e = lane + 32 * q;
+            const unsigned mz = lds_u32(st_addr + kMetaOff + 4u * e);
+            const unsigned xb = DENSE ? lds_u16(st_addr + kXcOff + 2u * e) : (ev[q] >> 16);
+            const float xf = __half2float(__ushort_as_half((unsigned short)xb));
+            const float sf = __half2float(__ushort_as_half((unsigned short)(mz & 0xffffu)));
+            const float zf = __half2float(__ushort_as_half((unsigned short)(mz >> 16)));
+            float am = xf * sf;   // exact
+            float zt = xf * zf;   // exact
+            if (!full) {          // an entry past the end of the part: weight 0
+                am = e < valid ? am : 0.0f;
+                zt = e < valid ? zt : 0.0f;
+            }
+            zl += zt;
+            const unsigned long long aa = pack2(am, am);
+            sts_pairs(mult_base + 16u * e, fmul2(aa, pack2(0x1p93f, 0x1p89f)), fmul2(aa, pack2(0x1p85f, 0x1p81f)));
+        }
+    };
+
+    // MATH: one step of a chunk: SLM blocks, each lane 16 codes of one of them
+    auto step = [&](unsigned st_addr, int u) {
+        unsigned long long m01, m23;
+        lds_pairs(mult_base + 16u * (u * SLM + mslot), m01, m23);
+        if (BITS == 4) {
+            const uint2 wv = lds_v2(st_addr + lane * 8 + u * 256);
+            fma_block8(acc, wv, m01, m23);
+        } else {
+            // lane t of a block: word t of the 2-bit plane (G/16 words); its top bits are the even
+            // (t < LM/2) or odd bits of word t mod LM/2 of the 1-bit plane
+            const unsigned blk = st_addr + (u * SLM + mslot) * B;
+            const unsigned w2 = lds_u32(blk + 4u * mh);
+            const unsigned w1 = lds_u32(blk + (G / 4) + 4u * (mh % (LM / 2))) >> (mh / (LM / 2));
+            fma_block3(acc, w2, w1, m01, m23);
+        }
+    };
+
+    // Stage ring: chunk number k of this warp (in issue order = consume order) uses stage k mod D, so
+    // ISSUE(k+D) refills the stage MATH(k) has just read.  wi: where the issue side stands in the
+    // warp's sequence of chunks (it runs ahead of the arithmetic, across block-rows); wc: the arithmetic.
+    unsigned rc = 0;   // byte offset of the arithmetic's stage
+    unsigned bc = 0;   // dense call: byte offset of that stage's barrier, and its phase parity
+    unsigned par = 0;
+    Walker wi, wc;
+    wc.first(pc, warp, resident);
+    wi = wc;
+    bool ok = true;
+    // moves the issue side to its next non-empty part (within the current span only when the window is
+    // rebuilt between spans); false when there is none
+    auto seek_issue = [&]() -> bool {
+        if (resident) {
+            while (wi.valid(pc) && !wi.has_chunk()) wi.next_span(pc, warp, true);
+        }
+        const bool more = wi.valid(pc) && wi.has_chunk();
+        if (more) enter_row(wi.r);
+        return more;
+    };
+    bool more_i = seek_issue();
+    // ISSUE of the warp's next chunk, if there is one, into the stage at byte offset rs; one commit
+    // group per call either way
+    auto issue_next = [&](unsigned rs, unsigned bs) {
+        if (more_i) {
+            const int left = wi.end - wi.pos;
+            if (left >= CH) issue(wi.pos, CH, true, stage_base + rs, full_base + bs);
+            else issue(wi.pos, left, false, stage_base + rs, full_base + bs);
+            wi.pos += CH;
+            if (wi.pos >= wi.end) more_i = seek_issue();
+        }
+        if (!DENSE) cp_async_commit();
+    };
+    // fills the pipeline, starting with the stage the arithmetic will read next
+    auto prime = [&]() {
+        unsigned rs = rc, bs = bc;
+#pragma unroll 1
+        for (int s = 0; s < D; ++s) {
+            issue_next(rs, bs);
+            rs = (rs + kStageBytes == D * kStageBytes) ? 0u : rs + kStageBytes;
+            bs = (bs + 8u == D * 8u) ? 0u : bs + 8u;
+        }
+    };
+    prime();
+
+    int sg = 0;
+    while (wc.valid(pc)) {
+#pragma unroll 1
+        for (int pos = wc.pos; pos < wc.end; pos += CH) {
+            const int left = wc.end - pos;
+            if (DENSE) {
+                if (ok) ok = mbar_wait_addr(full_base + bc, par);
+            } else {
+                cp_async_wait<D - 1>();
+                __syncwarp();
+            }
+            const unsigned st_addr = stage_base + rc;
+            if (left >= CH) {
+                prep(st_addr, pos, CH, true);
+                __syncwarp();
+                // a full chunk: straight-line code (branches between the steps made the compiler shuffle
+                // the accumulators around them, half as many instructions again)
+#pragma unroll
+                for (int u = 0; u < MSUBS; ++u) step(st_addr, u);
+            } else {
+                prep(st_addr, pos, left, false);
+                __syncwarp();
+                // the last chunk of a part: only the steps that hold entries
+                const int nsub = (left + SLM - 1) / SLM;
+#pragma unroll 1
+                for (int u = 0; u < nsub; ++u) step(st_addr, u);
+            }
+            __syncwarp();  // every lane is done with this chunk's stage and multipliers
+            issue_next(rc, bc);
+            if (rc + kStageBytes == D * kStageBytes) { rc = 0u; bc = 0u; par ^= 1u; } else { rc += kStageBytes; bc += 8u; }
+        }
+        if (wc.last_of_segment()) {
+            // ---- end of the segment: in-warp reduce-scatter over the column slots, then hand the
+            // per-warp sums to the writer warp
+            const int b = sg & 1;
+            if (sg >= 2 && ok) ok = mbar_wait(&sm.red_empty[b], ((sg >> 1) - 1) & 1);
+            float accf[16];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                unpack2(acc[i], accf[2 * i], accf[2 * i + 1]);
+                acc[i] = 0ull;
+            }
+            // lanes that differ in the bits above log2(LM) hold sums of the same rows
+            float t8[8], t4[4], keep[4];
+            halve<16>(accf, t8, lane, 16);
+            halve<8>(t8, t4, lane, 8);
+            if (LM == 8) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) keep[i] = t4[i];
+            } else {
+                float t2[2];
+                halve<4>(t4, t2, lane, 4);
+                keep[0] = t2[0];
+                keep[1] = t2[1];
+            }
+            const int a_base = mslot * KEEP;
+#pragma unroll
+            for (int i = 0; i < KEEP; ++i) {
+                const int ai = a_base + i;  // accumulator index = word*8 + nibble
+                const int cw = ai >> 3, e2 = ai & 7;
+                const int row = (BITS == 4)
+                                    ? 8 * mh + 4 * cw + (e2 >> 1) + (e2 & 1) * (G / 2)
+                                    : 4 * mh + (e2 >> 1) + (G / 4) * (2 * (e2 & 1) + cw);
+                sm.red[b][warp][row] = keep[i] * 0x1p56f;  // undo the 2^-56 of the subnormal trick
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) zl += __shfl_xor_sync(0xffffffffu, zl, o);
+            if (lane == 0) sm.red_z[b][warp] = zl;
+            zl = 0.0f;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.red_full[b]);
+            ++sg;
+        }
+        wc.next_span(pc, warp, resident);
+        if (!DENSE && !resident && wc.valid(pc)) {
+            // The next span needs another part of the list: every worker has drained its pipeline (the
+            // span's chunks are consumed), so the stage area and the window can be rebuilt.
+            cp_async_wait<0>();
+            worker_barrier(kWorkers * 32);
+            if (has_xs) stage_x(warp, kWorkers);
+            worker_barrier(kWorkers * 32);
+            int olo = 0, ohi = 0;
+            if (FUSED && wc.r == 0) { olo = wc.lo; ohi = wc.hi; }
+            win_lo = wc.lo;
+            build_window(wc.lo, wc.hi, olo, ohi, warp, kWorkers);
+            worker_barrier(kWorkers * 32);
+            wi = wc;
+            more_i = seek_issue();
+            prime();
+        }
     }
-    cp_async_wait<0>();
-    SPQT_TRACE_EVENT(tid == 0, 4001);
-#ifdef SPQT_TRACE
-    if (blockIdx.x == 0 && lane == 0 && g_trace) {
-        g_trace[3000 + warp * 4 + 0] = tr_wait; g_trace[3000 + warp * 4 + 1] = tr_issue;
-        g_trace[3000 + warp * 4 + 2] = tr_math; g_trace[3000 + warp * 4 + 3] = tr_n;
-    }
-#endif
-    if (!ok && lane == 0) atomicExch(status, 1);
+    if (!DENSE) cp_async_wait<0>();
+    if (!ok && lane == 0) atomicExch(a.status, 1);
 }
 
 // ---------------------------------------------------------------- host side
@@ -837,6 +888,7 @@ gemv_kernel(const uint8_t* __restrict__ codes, const __half* __restrict__ scales
 constexpr int kDebugBits = 1 << 20;
 static __device__ unsigned g_debug_bitmap[kDebugBits / 32];  // all zero between calls
 static __device__ int g_debug_count;                         // the count the GEMV is given
+static __device__ int g_debug_bad;                           // verdict of the call being checked
 static int g_debug = 0;
 
 __global__ void debug_mark_kernel(const int32_t* __restrict__ idx, const int32_t* __restrict__ count, int n,
@@ -854,11 +906,13 @@ __global__ void debug_mark_kernel(const int32_t* __restrict__ idx, const int32_t
             if (atomicOr(&g_debug_bitmap[k >> 5], bit) & bit) bad = true;  // seen before
         }
     }
-    if (bad) atomicExch(status, 2);
+    if (bad) {
+        atomicExch(status, 2);       // sticky, for the caller
+        atomicExch(&g_debug_bad, 1); // this call's verdict
+    }
 }
 
-__global__ void debug_clear_kernel(const int32_t* __restrict__ idx, const int32_t* __restrict__ count, int n,
-                                   const int* __restrict__ status)
+__global__ void debug_clear_kernel(const int32_t* __restrict__ idx, const int32_t* __restrict__ count, int n)
 {
     const int c = *count;
     const int lim = c < 0 ? 0 : (c > n ? n : c);
@@ -866,7 +920,10 @@ __global__ void debug_clear_kernel(const int32_t* __restrict__ idx, const int32_
         const int k = idx[i];
         if (k >= 0 && k < n && n <= kDebugBits) g_debug_bitmap[k >> 5] = 0u;
     }
-    if (blockIdx.x == 0 && threadIdx.x == 0) g_debug_count = (*status != 0) ? 0 : c;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        g_debug_count = g_debug_bad ? 0 : c;
+        g_debug_bad = 0;  // ready for the next checked call
+    }
 }
 
 // Launches the two kernels; returns the device address of the count the GEMV must use.
@@ -883,7 +940,7 @@ static spqt_status debug_check(const int32_t* idx, const int32_t* count, int n, 
     }
     const int blocks = n < 256 * 64 ? (n + 255) / 256 : 64;
     debug_mark_kernel<<<blocks, 256, 0, s>>>(idx, count, n, status);
-    debug_clear_kernel<<<blocks, 256, 0, s>>>(idx, count, n, status);
+    debug_clear_kernel<<<1, 256, 0, s>>>(idx, count, n);
     if (cudaGetLastError() != cudaSuccess) return SPQT_ERR_CUDA;
     count_launch(2);
     *checked_count = count_addr[dev];
@@ -896,14 +953,21 @@ struct FusedArgs {
     int32_t* count_out;
 };
 
-template <int G, int BITS, bool DENSE, bool ODD_N, bool FUSED>
-static spqt_status launch_gemv(const Format& f, const void* codes, const void* scales,
-                               const void* zeros, const void* x, const int32_t* idx,
-                               const int32_t* count, void* y, void* workspace, cudaStream_t s,
-                               FusedArgs fa)
+// Bytes of the stage area the prologue may borrow, and what it needs for an x of n entries.
+template <int G, int BITS>
+constexpr size_t stage_area_bytes() { return sizeof(GemvSmem<G, BITS>::stage); }
+inline size_t scratch_bytes(int n, bool fused) { return (size_t)((n + 255) / 256) * (fused ? 544 : 512); }
+
+template <int G, int BITS>
+static bool fused_fits(int n) { return n <= kMaxFusedN && scratch_bytes(n, true) <= stage_area_bytes<G, BITS>(); }
+
+template <int G, int BITS, int MODE>
+static spqt_status launch_gemv(const Format& f, const void* codes, const void* meta, const void* x,
+                               const int32_t* idx, const int32_t* count, void* y, void* workspace,
+                               cudaStream_t s, FusedArgs fa, int flags)
 {
-    auto kernel = gemv_kernel<G, BITS, DENSE, ODD_N, FUSED, false>;
-    auto kernel_c = gemv_kernel<G, BITS, DENSE, ODD_N, FUSED, true>;  // the thread-block-cluster variant
+    auto kernel = gemv_kernel<G, BITS, MODE, false>;
+    auto kernel_c = gemv_kernel<G, BITS, MODE, true>;  // the thread-block-cluster variant
     static bool configured[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPQT_ERR_CUDA;
@@ -926,11 +990,28 @@ static spqt_status launch_gemv(const Format& f, const void* codes, const void* s
     if (P > kMaxCtas) P = kMaxCtas;
     if (P < 1) P = 1;
     const int slots = max_slots(f.R);
-    int* counters = static_cast<int*>(workspace);
-    int* status = counters + f.R;
-    unsigned long long* words = reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) + header_bytes(f.R));
-    float* partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + header_bytes(f.R) + tagged_bytes(f));
-    float* zpartials = partials + (size_t)f.R * slots * G;
+    GemvArgs ga;
+    ga.codes = static_cast<const uint8_t*>(codes);
+    ga.meta = static_cast<const unsigned*>(meta);
+    ga.R = f.R;
+    ga.n = f.n;
+    ga.x = static_cast<const __half*>(x);
+    ga.idx = idx;
+    ga.count = count;
+    ga.y = static_cast<__half*>(y);
+    ga.counters = static_cast<int*>(workspace);
+    ga.status = ga.counters + f.R;
+    ga.words = reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) + header_bytes(f.R));
+    ga.partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + header_bytes(f.R) + tagged_bytes(f));
+    ga.zpartials = ga.partials + (size_t)f.R * slots * G;
+    ga.max_slots = slots;
+    ga.magic_p = magic_of((unsigned)P);
+    ga.magic_r = magic_of((unsigned)f.R);
+    ga.thr = fa.t;
+    ga.idx_out = fa.idx_out;
+    ga.count_out = fa.count_out;
+    ga.flags = flags;
+    if (MODE == kModeList && scratch_bytes(f.n, false) <= stage_area_bytes<G, BITS>()) ga.flags |= kFlagXs;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(P);
     cfg.blockDim = dim3(kGemvThreads);
@@ -966,50 +1047,62 @@ static spqt_status launch_gemv(const Format& f, const void* codes, const void* s
             if (known == 1) { cluster_k = k; ++nattr; }
         }
     }
+    ga.cluster_k = cluster_k;
     cfg.attrs = attr;
     cfg.numAttrs = nattr;
-    const cudaError_t err = cudaLaunchKernelEx(
-        &cfg, cluster_k ? kernel_c : kernel, static_cast<const uint8_t*>(codes), static_cast<const __half*>(scales),
-        static_cast<const __half*>(zeros), f.R, f.n, static_cast<const __half*>(x), idx, count,
-        static_cast<__half*>(y), counters, status, words, partials, zpartials, slots,
-        magic_of((unsigned)P), magic_of((unsigned)f.R), cluster_k, fa.t, fa.idx_out, fa.count_out);
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, cluster_k ? kernel_c : kernel, ga);
     count_launch();
     return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SPQT_OK : SPQT_ERR_CUDA;
 }
 
-template <bool DENSE, bool FUSED = false>
-static spqt_status gemv_entry(const void* codes, const void* scales, const void* zeros,
-                              int m, int n, int bits, int group, const void* x,
-                              const int32_t* idx, const int32_t* count, void* y,
-                              void* workspace, size_t ws_bytes, void* stream,
-                              FusedArgs fa = FusedArgs{0.0f, nullptr, nullptr})
+// Everything that can be checked on the host, in the order the header documents; nothing is put on
+// the stream before all of it has passed.
+static spqt_status check_gemv_args(const void* codes, const void* meta, int m, int n, int bits, int group,
+                                   const void* x, const int32_t* idx, const int32_t* count, bool dense, void* y,
+                                   void* workspace, size_t ws_bytes, Format* f)
 {
-    if (!codes || !scales || !zeros || !x || !y || !workspace) return SPQT_ERR_INVALID_ARG;
-    if (!DENSE && (!idx || !count)) return SPQT_ERR_INVALID_ARG;
-    if (FUSED && n > kMaxFusedN) return SPQT_ERR_UNSUPPORTED;
-    Format f;
-    spqt_status st = make_format(m, n, bits, group, &f);
+    if (!codes || !meta || !x || !y || !workspace) return SPQT_ERR_INVALID_ARG;
+    if (!dense && (!idx || !count)) return SPQT_ERR_INVALID_ARG;
+    spqt_status st = make_format(m, n, bits, group, f);
     if (st != SPQT_OK) return st;
-    if (!aligned(codes, 16) || !aligned(scales, 16) || !aligned(zeros, 16) || !aligned(x, 4) ||
-        !aligned(y, 2) || !aligned(workspace, 16) || (!DENSE && (!aligned(idx, 4) || !aligned(count, 4))))
+    if (!aligned(codes, 16) || !aligned(meta, 16) || !aligned(x, 2) || !aligned(y, 2) || !aligned(workspace, 16) ||
+        (!dense && (!aligned(idx, 4) || !aligned(count, 4))))
         return SPQT_ERR_ALIGNMENT;
-    if (ws_bytes < workspace_bytes(f)) return SPQT_ERR_WORKSPACE;
-    if ((long long)f.R * kMaxCtas >= (1ll << 31)) return SPQT_ERR_UNSUPPORTED;  // the work map is 32-bit
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (!DENSE && !FUSED && g_debug) {
-        st = debug_check(idx, count, n, static_cast<int*>(workspace) + f.R, s, &count);
+    if (ws_bytes < workspace_bytes(*f)) return SPQT_ERR_WORKSPACE;
+    if ((long long)f->R * kMaxCtas >= (1ll << 31)) return SPQT_ERR_UNSUPPORTED;  // the work map is 32-bit
+    return SPQT_OK;
+}
+
+template <int MODE>
+static spqt_status gemv_dispatch(const Format& f, const void* codes, const void* meta, const void* x,
+                                 const int32_t* idx, const int32_t* count, void* y, void* workspace,
+                                 cudaStream_t s, FusedArgs fa, int flags)
+{
+    if (f.bits == 4 && f.group == 128) return launch_gemv<128, 4, MODE>(f, codes, meta, x, idx, count, y, workspace, s, fa, flags);
+    if (f.bits == 4 && f.group == 64) return launch_gemv<64, 4, MODE>(f, codes, meta, x, idx, count, y, workspace, s, fa, flags);
+    if (f.bits == 3 && f.group == 128) return launch_gemv<128, 3, MODE>(f, codes, meta, x, idx, count, y, workspace, s, fa, flags);
+    if (f.bits == 3 && f.group == 64) return launch_gemv<64, 3, MODE>(f, codes, meta, x, idx, count, y, workspace, s, fa, flags);
+    return SPQT_ERR_UNSUPPORTED;
+}
+
+static bool fused_fits_format(const Format& f)
+{
+    if (f.bits == 4 && f.group == 128) return fused_fits<128, 4>(f.n);
+    if (f.bits == 4 && f.group == 64) return fused_fits<64, 4>(f.n);
+    if (f.bits == 3 && f.group == 128) return fused_fits<128, 3>(f.n);
+    return fused_fits<64, 3>(f.n);
+}
+
+// The sparse call after its arguments have been checked.
+static spqt_status sparse_checked(const Format& f, const void* codes, const void* meta, const void* x,
+                                  const int32_t* idx, const int32_t* count, void* y, void* workspace, cudaStream_t s)
+{
+    if (f.n > kMaxListN) return SPQT_ERR_UNSUPPORTED;
+    if (g_debug) {
+        spqt_status st = debug_check(idx, count, f.n, static_cast<int*>(workspace) + f.R, s, &count);
         if (st != SPQT_OK) return st;
     }
-    const bool odd = (n & 1) != 0;
-#define SPQT_DISPATCH(GG, BB)                                                                                      \
-    return odd ? launch_gemv<GG, BB, DENSE, true, FUSED>(f, codes, scales, zeros, x, idx, count, y, workspace, s, fa) \
-               : launch_gemv<GG, BB, DENSE, false, FUSED>(f, codes, scales, zeros, x, idx, count, y, workspace, s, fa)
-    if (bits == 4 && group == 128) { SPQT_DISPATCH(128, 4); }
-    if (bits == 4 && group == 64) { SPQT_DISPATCH(64, 4); }
-    if (bits == 3 && group == 128) { SPQT_DISPATCH(128, 3); }
-    if (bits == 3 && group == 64) { SPQT_DISPATCH(64, 3); }
-#undef SPQT_DISPATCH
-    return SPQT_ERR_UNSUPPORTED;
+    return gemv_dispatch<kModeList>(f, codes, meta, x, idx, count, y, workspace, s, FusedArgs{0.0f, nullptr, nullptr}, 0);
 }
 
 }  // namespace spqt
@@ -1019,47 +1112,80 @@ static spqt_status gemv_entry(const void* codes, const void* scales, const void*
 constexpr size_t kStaticScratchBytes = size_t(1) << 20;
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
-#ifdef SPQT_TRACE
-extern "C" int spqt_debug_set_trace(void* buf) { return (int)cudaMemcpyToSymbol(spqt::g_trace, &buf, sizeof(buf)); }
-#endif
+// Device address of the scratch on the current device (looked up once per device); nullptr on error.
+static void* static_scratch_address()
+{
+    // In host code the array's name is only a handle; the device address has to be asked for,
+    // once per device, with that device current.
+    static void* scratch_addr[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (scratch_addr[dev] == nullptr) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return nullptr;
+        scratch_addr[dev] = p;
+    }
+    return scratch_addr[dev];
+}
 
 extern "C" {
 
-spqt_status spqt_sparse_gemv(const void* codes, const void* scales, const void* zeros,
+spqt_status spqt_sparse_gemv(const void* codes, const void* scale_zero,
                              int m, int n, int bits, int group,
                              const void* x, const int32_t* idx, const int32_t* count,
                              void* y, void* workspace, size_t workspace_bytes, void* stream)
 {
-    return spqt::gemv_entry<false>(codes, scales, zeros, m, n, bits, group, x, idx, count, y,
-                                   workspace, workspace_bytes, stream);
+    using namespace spqt;
+    Format f;
+    spqt_status st = check_gemv_args(codes, scale_zero, m, n, bits, group, x, idx, count, false, y, workspace,
+                                     workspace_bytes, &f);
+    if (st != SPQT_OK) return st;
+    return sparse_checked(f, codes, scale_zero, x, idx, count, y, workspace, static_cast<cudaStream_t>(stream));
 }
 
-spqt_status spqt_sparsify_gemv(const void* codes, const void* scales, const void* zeros,
+spqt_status spqt_sparsify_gemv(const void* codes, const void* scale_zero,
                                int m, int n, int bits, int group,
                                const void* x, float t, int32_t* idx, int32_t* count,
                                void* y, void* workspace, size_t workspace_bytes, void* stream)
 {
-    if (n > spqt::kMaxFusedN) {
+    using namespace spqt;
+    Format f;
+    spqt_status st = check_gemv_args(codes, scale_zero, m, n, bits, group, x, idx, count, false, y, workspace,
+                                     workspace_bytes, &f);
+    if (st != SPQT_OK) return st;
+    if (n > kMaxListN) return SPQT_ERR_UNSUPPORTED;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (!fused_fits_format(f)) {
         // too long for the in-kernel scan: the same result from the two separate launches
-        spqt_status st = spqt_sparsify(x, n, t, idx, count, stream);
+        st = spqt_sparsify(x, n, t, idx, count, stream);
         if (st != SPQT_OK) return st;
-        return spqt_sparse_gemv(codes, scales, zeros, m, n, bits, group, x, idx, count, y, workspace,
-                                workspace_bytes, stream);
+        return gemv_dispatch<kModeList>(f, codes, scale_zero, x, idx, count, y, workspace, s,
+                                        FusedArgs{0.0f, nullptr, nullptr}, 0);
     }
-    return spqt::gemv_entry<false, true>(codes, scales, zeros, m, n, bits, group, x, idx, count, y,
-                                         workspace, workspace_bytes, stream,
-                                         spqt::FusedArgs{t, idx, count});
+    return gemv_dispatch<kModeFused>(f, codes, scale_zero, x, nullptr, nullptr, y, workspace, s,
+                                     FusedArgs{t, idx, count}, 0);
 }
 
-spqt_status spqt_dense_gemv(const void* codes, const void* scales, const void* zeros,
+spqt_status spqt_dense_gemv(const void* codes, const void* scale_zero,
                             int m, int n, int bits, int group, const void* x,
                             void* y, void* workspace, size_t workspace_bytes, void* stream)
 {
-    return spqt::gemv_entry<true>(codes, scales, zeros, m, n, bits, group, x, nullptr, nullptr, y,
-                                  workspace, workspace_bytes, stream);
+    using namespace spqt;
+    Format f;
+    spqt_status st = check_gemv_args(codes, scale_zero, m, n, bits, group, x, nullptr, nullptr, true, y, workspace,
+                                     workspace_bytes, &f);
+    if (st != SPQT_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const FusedArgs none{0.0f, nullptr, nullptr};
+    // whole chunks of a block-row by bulk copies when every chunk starts on a 16-byte boundary
+    if ((n & 7) == 0 && aligned(x, 16))
+        return gemv_dispatch<kModeDense>(f, codes, scale_zero, x, nullptr, nullptr, y, workspace, s, none, 0);
+    if (n > kMaxListN) return SPQT_ERR_UNSUPPORTED;
+    // otherwise the list path over the identity list
+    return gemv_dispatch<kModeList>(f, codes, scale_zero, x, nullptr, nullptr, y, workspace, s, none, kFlagIdentity);
 }
 
-spqt_status spqt_sparse_gemv_static(const void* codes, const void* scales, const void* zeros,
+spqt_status spqt_sparse_gemv_static(const void* codes, const void* scale_zero,
                                     int m, int n, int bits, int group,
                                     const void* x, const int32_t* idx, const int32_t* count,
                                     void* y, void* stream)
@@ -1069,22 +1195,32 @@ spqt_status spqt_sparse_gemv_static(const void* codes, const void* scales, const
     spqt_status st = make_format(m, n, bits, group, &f);
     if (st != SPQT_OK) return st;
     if (workspace_bytes(f) > kStaticScratchBytes) return SPQT_ERR_WORKSPACE;  // problem too large for the built-in scratch
-    // In host code the array's name is only a handle; the device address has to be asked for,
-    // once per device, with that device current.
-    static void* scratch_addr[64] = {};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPQT_ERR_CUDA;
-    if (scratch_addr[dev] == nullptr) {
-        void* p = nullptr;
-        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || p == nullptr) return SPQT_ERR_CUDA;
-        scratch_addr[dev] = p;
-    }
+    void* const scratch = static_scratch_address();
+    if (scratch == nullptr) return SPQT_ERR_CUDA;
+    st = check_gemv_args(codes, scale_zero, m, n, bits, group, x, idx, count, false, y, scratch, kStaticScratchBytes, &f);
+    if (st != SPQT_OK) return st;
+    if (n > kMaxListN) return SPQT_ERR_UNSUPPORTED;
     // The scratch keeps whatever the previous call (or an interrupted one, or one of another shape)
     // left: the arrival counters, the status word and the tagged words must start at zero.
-    if (cudaMemsetAsync(scratch_addr[dev], 0, header_bytes(f.R) + tagged_bytes(f), static_cast<cudaStream_t>(stream)) != cudaSuccess)
-        return SPQT_ERR_CUDA;
-    return gemv_entry<false>(codes, scales, zeros, m, n, bits, group, x, idx, count, y,
-                             scratch_addr[dev], kStaticScratchBytes, stream);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemsetAsync(scratch, 0, header_bytes(f.R) + tagged_bytes(f), s) != cudaSuccess) return SPQT_ERR_CUDA;
+    return sparse_checked(f, codes, scale_zero, x, idx, count, y, scratch, s);
+}
+
+// Reads a status word (device) into *status_host, waits, and maps it to a return value.
+static spqt_status read_status_word(const int* word, int* status_host, cudaStream_t s)
+{
+    if (cudaMemcpyAsync(status_host, word, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return SPQT_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return SPQT_ERR_CUDA;
+    return *status_host == 0 ? SPQT_OK : (*status_host == 1 ? SPQT_ERR_TIMEOUT : SPQT_ERR_INVALID_ARG);
+}
+
+spqt_status spqt_static_status(int m, int group, int* status_host, void* stream)
+{
+    if (!status_host || m <= 0 || (group != 64 && group != 128) || m % group) return SPQT_ERR_INVALID_ARG;
+    void* const scratch = static_scratch_address();
+    if (scratch == nullptr) return SPQT_ERR_CUDA;
+    return read_status_word(static_cast<const int*>(scratch) + m / group, status_host, static_cast<cudaStream_t>(stream));
 }
 
 spqt_status spqt_set_debug(int on)
@@ -1105,11 +1241,7 @@ spqt_status spqt_set_tuning(int gemv_ctas, int reserved)
 spqt_status spqt_workspace_status(const void* workspace, int m, int group, int* status_host, void* stream)
 {
     if (!workspace || !status_host || m <= 0 || (group != 64 && group != 128) || m % group) return SPQT_ERR_INVALID_ARG;
-    const int* word = static_cast<const int*>(workspace) + m / group;
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (cudaMemcpyAsync(status_host, word, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return SPQT_ERR_CUDA;
-    if (cudaStreamSynchronize(s) != cudaSuccess) return SPQT_ERR_CUDA;
-    return SPQT_OK;
+    return read_status_word(static_cast<const int*>(workspace) + m / group, status_host, static_cast<cudaStream_t>(stream));
 }
 
 }  // extern "C"

@@ -1,7 +1,7 @@
 // Device-side building blocks of the GEMV kernel: PTX wrappers (mbarriers with bounded waits,
-// cp.async, tagged 64-bit words, shared-memory accesses by 32-bit address, thread-block-cluster
-// primitives, predicated stores) and the packed-FMA dequantization arithmetic.  Included by
-// spqt_gemv.cu only, after its compile-time constants.
+// cp.async, bulk copies, tagged 64-bit words, shared-memory accesses by 32-bit address,
+// thread-block-cluster primitives, predicated stores) and the packed-FMA dequantization arithmetic.
+// Included by spqt_gemv.cu only, after its compile-time constants.
 #pragma once
 
 namespace spqt {
@@ -46,27 +46,64 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, unsigned parity)
 }
 
 // Bounded wait for the phase with the given parity; false when the bound
-// (wall time, so that a logic error can never hold the GPU) expires.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity)
+// (wall time, so that a logic error can never hold the GPU) expires.  The wait itself
+// is the hardware's: try_wait with a time hint suspends the warp until the phase
+// completes or the hint runs out, so a waiting warp issues next to no instructions
+// (a software spin on a short try_wait was measured to take more issue slots than
+// the arithmetic of the warps it shares a scheduler with).
+constexpr unsigned kSuspendNs = 100000u;  // one suspension: 0.1 ms at most
+__device__ __forceinline__ bool mbar_wait_addr(unsigned addr, unsigned parity)
 {
-    const unsigned addr = smem_u32(bar);
     unsigned long long t0 = 0;
     for (unsigned it = 0;; ++it) {
         unsigned done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(done)
-            : "r"(addr), "r"(parity)
+            : "r"(addr), "r"(parity), "r"(kSuspendNs)
             : "memory");
         if (done) return true;
-        if (it == 16) t0 = global_ns();
-        if (it > 16) {
-            __nanosleep(64);
-            if (global_ns() - t0 > kWaitNs) return false;
-        }
+        if (it == 0) t0 = global_ns();
+        else if (global_ns() - t0 > kWaitNs) return false;
     }
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity) { return mbar_wait_addr(smem_u32(bar), parity); }
+
+// Bulk copies (the dense path: whole chunks of a block-row are contiguous).  The copy completes on
+// the mbarrier by the number of bytes it moved; one thread first announces the total with expect_tx.
+// Source, destination and size are multiples of 16 bytes.  This GPU's own memory only, no multicast.
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar_addr, unsigned bytes)
+{
+    asm volatile("{\n\t.reg .b64 st;\n\tmbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n\t}" ::"r"(bar_addr), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_copy(unsigned smem_dst, const void* gmem_src, unsigned bytes, unsigned bar_addr)
+{
+    asm volatile("cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_dst),
+                 "l"(gmem_src), "r"(bytes), "r"(bar_addr)
+                 : "memory");
+}
+// the same under a predicate (no branch: one lane of a warp issues for all)
+__device__ __forceinline__ void mbar_expect_tx_if(unsigned cond, unsigned bar_addr, unsigned bytes)
+{
+    asm volatile("{\n\t.reg .pred p;\n\t.reg .b64 st;\n\tsetp.ne.u32 p, %0, 0;\n\t"
+                 "@p mbarrier.arrive.expect_tx.shared::cta.b64 st, [%1], %2;\n\t}" ::"r"(cond), "r"(bar_addr), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_copy_if(unsigned cond, unsigned smem_dst, const void* gmem_src, unsigned bytes,
+                                             unsigned bar_addr)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %0, 0;\n\t"
+                 "@p cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%1], [%2], %3, [%4];\n\t}" ::"r"(cond),
+                 "r"(smem_dst), "l"(gmem_src), "r"(bytes), "r"(bar_addr)
+                 : "memory");
+}
+// barrier among the worker warps only (id 1); every worker warp must reach it
+__device__ __forceinline__ void worker_barrier(int threads)
+{
+    asm volatile("bar.sync 1, %0;" ::"r"(threads) : "memory");
 }
 
 __device__ __forceinline__ void cp_async_16(unsigned smem_dst, const void* gmem_src)
@@ -124,9 +161,32 @@ __device__ __forceinline__ uint4 lds_v4(unsigned addr)
     asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
     return v;
 }
+__device__ __forceinline__ uint2 lds_v2(unsigned addr)
+{
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr) : "memory");
+    return v;
+}
 __device__ __forceinline__ void sts_u32(unsigned addr, unsigned v)
 {
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+__device__ __forceinline__ void sts_v4(unsigned addr, const uint4& v)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+// two packed multiplier pairs (four fp32 values) of one list entry
+__device__ __forceinline__ void lds_pairs(unsigned addr, unsigned long long& a, unsigned long long& b)
+{
+    asm volatile("ld.shared.v2.u64 {%0, %1}, [%2];" : "=l"(a), "=l"(b) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void sts_pairs(unsigned addr, unsigned long long a, unsigned long long b)
+{
+    asm volatile("st.shared.v2.u64 [%0], {%1, %2};" ::"r"(addr), "l"(a), "l"(b) : "memory");
+}
+__device__ __forceinline__ void st_shared_u32_if(unsigned cond, unsigned smem_dst, unsigned v)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %0, 0;\n\t@p st.shared.u32 [%1], %2;\n\t}" ::"r"(cond), "r"(smem_dst), "r"(v) : "memory");
 }
 
 // ---- thread-block clusters: the CTAs of one block-row hand their sums to CTA rank 0 through its
@@ -164,17 +224,14 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, unsigned parity
         unsigned done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+            "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2, %3;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
             : "=r"(done)
-            : "r"(addr), "r"(parity)
+            : "r"(addr), "r"(parity), "r"(kSuspendNs)
             : "memory");
         if (done) return true;
-        if (it == 16) t0 = global_ns();
-        if (it > 16) {
-            __nanosleep(64);
-            if (global_ns() - t0 > kWaitNs) return false;
-        }
+        if (it == 0) t0 = global_ns();
+        else if (global_ns() - t0 > kWaitNs) return false;
     }
 }
 
@@ -232,28 +289,25 @@ __device__ __forceinline__ unsigned long long fmul2(unsigned long long a, unsign
     return d;
 }
 
-// acc (32 fp32 sums in 16 registers) += the 32 codes of a lane's 16 bytes, each times a (scaled by 2^-56).
-__device__ __forceinline__ void fma_block16(unsigned long long* acc, const uint4& w, float a)
+// acc (16 fp32 sums in 8 registers) += the 16 codes of a lane's 8 bytes, each times a (scaled by
+// 2^-56), given the multiplier pairs m01 = a*(2^93, 2^89) and m23 = a*(2^85, 2^81).
+__device__ __forceinline__ void fma_block8(unsigned long long* acc, const uint2& w, unsigned long long m01,
+                                           unsigned long long m23)
 {
-    const unsigned long long aa = pack2(a, a);
-    const unsigned long long m01 = fmul2(aa, pack2(0x1p93f, 0x1p89f)), m23 = fmul2(aa, pack2(0x1p85f, 0x1p81f));
     fma_word(acc + 0, w.x, m01, m23);
     fma_word(acc + 4, w.y, m01, m23);
-    fma_word(acc + 8, w.z, m01, m23);
-    fma_word(acc + 12, w.w, m01, m23);
 }
 
-// 3-bit codes: w2a, w2b are words of the 2-bit plane (byte i, field v = bits 2v..2v+1), w1 the word
-// of the 1-bit plane whose byte i, bit u carries the top bit of the code in w2a (u = 2v) or w2b
-// (u = 2v+1).  The fields are first widened to four words of eight 4-bit codes, then treated like
-// 4-bit codes: word 0/1 = w2a fields v = {0,2} / {1,3}, word 2/3 = the same of w2b (low nibble first).
-__device__ __forceinline__ void fma_block3(unsigned long long* acc, unsigned w2a, unsigned w2b, unsigned w1, float a)
+// 3-bit codes: w2 is a word of the 2-bit plane (byte i, field v = bits 2v..2v+1), w1 the matching word
+// of the 1-bit plane, already shifted so that bit 2v of byte i is the top bit of the code in field v.
+// The fields are first widened to two words of eight 4-bit codes (fields v = {0,2}, then {1,3}; low
+// nibble first), then treated like 4-bit codes.
+__device__ __forceinline__ void fma_block3(unsigned long long* acc, unsigned w2, unsigned w1, unsigned long long m01,
+                                           unsigned long long m23)
 {
-    const unsigned c0 = (w2a & 0x33333333u) | ((w1 << 2) & 0x44444444u);
-    const unsigned c1 = ((w2a >> 2) & 0x33333333u) | (w1 & 0x44444444u);
-    const unsigned c2 = (w2b & 0x33333333u) | ((w1 << 1) & 0x44444444u);
-    const unsigned c3 = ((w2b >> 2) & 0x33333333u) | ((w1 >> 1) & 0x44444444u);
-    fma_block16(acc, make_uint4(c0, c1, c2, c3), a);
+    const unsigned c0 = (w2 & 0x33333333u) | ((w1 << 2) & 0x44444444u);
+    const unsigned c1 = ((w2 >> 2) & 0x33333333u) | (w1 & 0x44444444u);
+    fma_block8(acc, make_uint2(c0, c1), m01, m23);
 }
 
 // One step of a butterfly reduce-scatter: lanes that differ in bit `bit` hold

@@ -1,14 +1,9 @@
 // The work map of the GEMV kernel: which block-rows, and which slices of the active index list,
 // belong to which CTA and warp (32-bit arithmetic, divisions by multiply-high).  Included by
-// spqt_gemv.cu only, after its compile-time constants (kWorkers).
+// spqt_gemv.cu only, after its compile-time constants (kWorkers, kCap).
 #pragma once
 
 namespace spqt {
-
-// ---------------------------------------------------------------- work map
-
-// The piece of CTA c: block-rows r_first..r_last, and of each the slice of the
-// active list that belongs to this CTA.  Uniform across the CTA.
 
 // floor(v / d) for any 32-bit v from the multiplier m = floor((2^32 - 1) / d): the high product is
 // the quotient or one less (the multiplier falls short of 2^32 / d by at most 1), one compare fixes it.
@@ -19,8 +14,13 @@ __device__ __forceinline__ unsigned magic_div(unsigned v, unsigned d, unsigned m
     return q + ((v - q * d >= d) ? 1u : 0u);
 }
 
+// The piece of CTA c: block-rows r_first..r_last, and of each the slice of the active list that
+// belongs to this CTA.  The R block-rows are laid end to end and cut into P equal pieces; the
+// fraction [u0,u1) of a block-row is the slice [u0*count/P, u1*count/P) of the list.  Uniform across
+// the CTA.  `unit` scales the slices: the dense path counts in groups of 8 columns so that every
+// slice starts on a 16-byte boundary of x.
 struct Piece {
-    int R, P, c, count, r_first, r_last;
+    int R, P, c, count, unit, r_first, r_last;
     unsigned mP, mR;  // multipliers of magic_div for P and R, computed by the host
     unsigned qc, rc;  // count = qc * P + rc: keeps the slice arithmetic in 32 bits (the host checks R * P < 2^31)
 
@@ -30,27 +30,29 @@ struct Piece {
         R = R_; P = P_; c = c_;
         mP = mP_;
         mR = mR_;
+        unit = 1;
         const unsigned lo = (unsigned)c * (unsigned)R, hi = lo + (unsigned)R;
         r_first = (int)magic_div(lo, (unsigned)P, mP);
         r_last = (int)magic_div(hi - 1u, (unsigned)P, mP);
     }
-    __device__ __forceinline__ void set_count(int count_)
+    // count_ list entries, in units of unit_ entries (count_ a multiple of unit_)
+    __device__ __forceinline__ void set_count(int count_, int unit_ = 1)
     {
-        count = count_;
+        unit = unit_;
+        count = count_ / unit_;
         qc = magic_div((unsigned)count, (unsigned)P, mP);
         rc = (unsigned)count - qc * (unsigned)P;
     }
     // floor(u * count / P) for 0 <= u <= P
     __device__ __forceinline__ int scaled(unsigned u) const { return (int)(u * qc + magic_div(u * rc, (unsigned)P, mP)); }
-    __device__ __forceinline__ void slice_compute(int row, int* a, int* b) const
+    __device__ __forceinline__ void slice(int row, int* a, int* b) const
     {
         const unsigned lo = (unsigned)c * (unsigned)R, hi = lo + (unsigned)R, base = (unsigned)row * (unsigned)P;
         const unsigned u0 = (lo > base ? lo : base) - base;
         const unsigned u1 = (hi < base + (unsigned)P ? hi : base + (unsigned)P) - base;
-        *a = scaled(u0);
-        *b = scaled(u1);
+        *a = scaled(u0) * unit;
+        *b = scaled(u1) * unit;
     }
-    __device__ __forceinline__ void slice(int row, int* a, int* b) const { slice_compute(row, a, b); }
     // contributors to block-row `row`: CTAs first .. first+n-1
     __device__ __forceinline__ void contributors(int row, int* first, int* n) const
     {
@@ -61,37 +63,53 @@ struct Piece {
     }
 };
 
-// A warp's position in its sequence of chunks: list position `pos` of the
-// chunk's first entry inside block-row r (whose slice ends at p1).
-struct Cursor {
-    int r, pos, p1;
-    int chunk;  // list entries per chunk (32 or 64, by format)
-    __device__ __forceinline__ void settle(const Piece& pc, int warp)
+// The part [a,b) of the span [lo,hi) that worker warp `warp` processes: the span is cut into
+// kWorkers contiguous parts whose boundaries are multiples of 8 entries from lo.
+__device__ __forceinline__ void warp_part(int lo, int hi, int warp, int* a, int* b)
+{
+    const int q = (hi - lo + 7) >> 3;
+    const int ua = (warp * q) / kWorkers, ub = ((warp + 1) * q) / kWorkers;
+    *a = lo + 8 * ua;
+    *b = min(lo + 8 * ub, hi);
+}
+
+// A warp's walk over its work.  The CTA's slice of a block-row (a segment) is processed as one span
+// when the list entries the CTA needs are all resident in shared memory, else as consecutive spans
+// of at most kCap entries (the shared-memory window is rebuilt between them).  Within a span the
+// warp owns the part [pos, end).
+struct Walker {
+    int r, lo, hi, seg_hi;
+    int pos, end;
+    __device__ __forceinline__ bool valid(const Piece& pc) const { return r <= pc.r_last; }
+    __device__ __forceinline__ void open_segment(const Piece& pc, int warp, bool resident)
     {
-        while (r <= pc.r_last && pos >= p1) {
-            ++r;
-            if (r <= pc.r_last) {
-                int p0;
-                pc.slice(r, &p0, &p1);
-                pos = p0 + warp * chunk;
-            }
+        if (r <= pc.r_last) {
+            int p0, p1;
+            pc.slice(r, &p0, &p1);
+            seg_hi = p1;
+            lo = p0;
+            hi = resident ? p1 : min(p1, p0 + kCap);
+            warp_part(lo, hi, warp, &pos, &end);
         }
     }
-    __device__ __forceinline__ void init(const Piece& pc, int warp, int chunk_)
+    __device__ __forceinline__ void first(const Piece& pc, int warp, bool resident)
     {
-        chunk = chunk_;
         r = pc.r_first;
-        int p0;
-        pc.slice(r, &p0, &p1);
-        pos = p0 + warp * chunk;
-        settle(pc, warp);
+        open_segment(pc, warp, resident);
     }
-    __device__ __forceinline__ bool valid(const Piece& pc) const { return r <= pc.r_last; }
-    __device__ __forceinline__ void advance(const Piece& pc, int warp)
+    __device__ __forceinline__ bool last_of_segment() const { return hi >= seg_hi; }
+    __device__ __forceinline__ void next_span(const Piece& pc, int warp, bool resident)
     {
-        pos += kWorkers * chunk;
-        if (pos >= p1) settle(pc, warp);
+        if (hi < seg_hi) {
+            lo = hi;
+            hi = min(seg_hi, lo + kCap);
+            warp_part(lo, hi, warp, &pos, &end);
+        } else {
+            ++r;
+            open_segment(pc, warp, resident);
+        }
     }
+    __device__ __forceinline__ bool has_chunk() const { return pos < end; }
 };
 
 }  // namespace spqt

@@ -14,7 +14,7 @@ constexpr int kPackThreads = 256; // 8 warps, 4 columns each
 template <int G, int BITS>
 __global__ void __launch_bounds__(kPackThreads)
 pack_kernel(const __half* __restrict__ W, int n, int ldw,
-            uint8_t* __restrict__ codes, __half* __restrict__ scales, __half* __restrict__ zeros)
+            uint8_t* __restrict__ codes, __half2* __restrict__ scale_zero)
 {
     constexpr int B = G * BITS / 8;
     constexpr int QMAX = (1 << BITS) - 1;
@@ -64,6 +64,9 @@ pack_kernel(const __half* __restrict__ W, int n, int ldw,
             lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
             hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
         }
+        // a zero extreme of either sign counts as +0.0 (x + (+0.0) is x, except that -0.0 becomes +0.0)
+        lo = __fadd_rn(lo, 0.0f);
+        hi = __fadd_rn(hi, 0.0f);
         // scale = fp16((max - min) / qmax): one IEEE subtract, one IEEE divide, RN-even
         const float s32 = __fdiv_rn(__fsub_rn(hi, lo), (float)QMAX);
         const __half sh = __float2half_rn(s32);
@@ -98,10 +101,7 @@ pack_kernel(const __half* __restrict__ W, int n, int ldw,
                 out[b] = (uint8_t)v;
             }
         }
-        if (lane == 0) {
-            scales[blk] = sh;
-            zeros[blk] = __float2half_rn(lo);  // exact: lo is an fp16 value
-        }
+        if (lane == 0) scale_zero[blk] = __halves2half2(sh, __float2half_rn(lo));  // exact: lo is an fp16 value
         __syncwarp();
     }
 }
@@ -116,7 +116,7 @@ constexpr int kPack4Cols = 128;
 template <int G>
 __global__ void __launch_bounds__(kPack4Cols)
 pack4_kernel(const __half* __restrict__ W, int n, int ldw,
-             uint8_t* __restrict__ codes, __half* __restrict__ scales, __half* __restrict__ zeros)
+             uint8_t* __restrict__ codes, __half2* __restrict__ scale_zero)
 {
     constexpr int B = G / 2;
     constexpr int QMAX = 15;
@@ -146,7 +146,8 @@ pack4_kernel(const __half* __restrict__ W, int n, int ldw,
         lo_h = __hmin(lo_h, v);
         hi_h = __hmax(hi_h, v);
     }
-    const float lo = __half2float(lo_h), hi = __half2float(hi_h);
+    // a zero extreme of either sign counts as +0.0
+    const float lo = __fadd_rn(__half2float(lo_h), 0.0f), hi = __fadd_rn(__half2float(hi_h), 0.0f);
     // scale = fp16((max - min) / qmax): one IEEE subtract, one IEEE divide, RN-even
     const __half sh = __float2half_rn(__fdiv_rn(__fsub_rn(hi, lo), (float)QMAX));
     const float sf = __half2float(sh);
@@ -170,8 +171,7 @@ pack4_kernel(const __half* __restrict__ W, int n, int ldw,
         }
         out[q] = make_uint4(wds[0], wds[1], wds[2], wds[3]);
     }
-    scales[blk] = sh;
-    zeros[blk] = lo_h;
+    scale_zero[blk] = __halves2half2(sh, __float2half_rn(lo));
 }
 
 // One thread per weight: read its code out of the zigzag buffer.
@@ -196,8 +196,8 @@ __global__ void unpack_kernel(const uint8_t* __restrict__ codes, int m, int n, u
 }
 
 template <int G, int BITS>
-static spqt_status launch_pack(const Format& f, const void* W, int ldw, void* codes, void* scales,
-                               void* zeros, cudaStream_t s)
+static spqt_status launch_pack(const Format& f, const void* W, int ldw, void* codes, void* scale_zero,
+                               cudaStream_t s)
 {
     // (with G = 128 its 34 KB tile per 128 threads leaves too few warps per SM to hide the division
     // chains, and the warp-per-column kernel below is faster)
@@ -205,14 +205,14 @@ static spqt_status launch_pack(const Format& f, const void* W, int ldw, void* co
         dim3 grid4((f.n + kPack4Cols - 1) / kPack4Cols, f.R);
         pack4_kernel<G><<<grid4, kPack4Cols, 0, s>>>(
             static_cast<const __half*>(W), f.n, ldw, static_cast<uint8_t*>(codes),
-            static_cast<__half*>(scales), static_cast<__half*>(zeros));
+            static_cast<__half2*>(scale_zero));
         count_launch();
         return cudaGetLastError() == cudaSuccess ? SPQT_OK : SPQT_ERR_CUDA;
     }
     dim3 grid((f.n + kPackCols - 1) / kPackCols, f.R);
     pack_kernel<G, BITS><<<grid, kPackThreads, 0, s>>>(
         static_cast<const __half*>(W), f.n, ldw, static_cast<uint8_t*>(codes),
-        static_cast<__half*>(scales), static_cast<__half*>(zeros));
+        static_cast<__half2*>(scale_zero));
     count_launch();
     return cudaGetLastError() == cudaSuccess ? SPQT_OK : SPQT_ERR_CUDA;
 }
@@ -233,22 +233,22 @@ static spqt_status launch_unpack(const Format& f, const void* codes, void* q, cu
 extern "C" {
 
 spqt_status spqt_pack(const void* W, int m, int n, int ldw, int bits, int group,
-                      void* codes, void* scales, void* zeros, void* stream)
+                      void* codes, void* scale_zero, void* stream)
 {
     using namespace spqt;
-    if (!W || !codes || !scales || !zeros) return SPQT_ERR_INVALID_ARG;
+    if (!W || !codes || !scale_zero) return SPQT_ERR_INVALID_ARG;
     Format f;
     spqt_status st = make_format(m, n, bits, group, &f);
     if (st != SPQT_OK) return st;
     if (ldw < n) return SPQT_ERR_INVALID_ARG;
     if (f.R > 65535) return SPQT_ERR_UNSUPPORTED;
-    if (!aligned(W, 2) || !aligned(codes, 16) || !aligned(scales, 16) || !aligned(zeros, 16))
+    if (!aligned(W, 2) || !aligned(codes, 16) || !aligned(scale_zero, 16))
         return SPQT_ERR_ALIGNMENT;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (bits == 4 && group == 128) return launch_pack<128, 4>(f, W, ldw, codes, scales, zeros, s);
-    if (bits == 4 && group == 64) return launch_pack<64, 4>(f, W, ldw, codes, scales, zeros, s);
-    if (bits == 3 && group == 128) return launch_pack<128, 3>(f, W, ldw, codes, scales, zeros, s);
-    return launch_pack<64, 3>(f, W, ldw, codes, scales, zeros, s);
+    if (bits == 4 && group == 128) return launch_pack<128, 4>(f, W, ldw, codes, scale_zero, s);
+    if (bits == 4 && group == 64) return launch_pack<64, 4>(f, W, ldw, codes, scale_zero, s);
+    if (bits == 3 && group == 128) return launch_pack<128, 3>(f, W, ldw, codes, scale_zero, s);
+    return launch_pack<64, 3>(f, W, ldw, codes, scale_zero, s);
 }
 
 spqt_status spqt_unpack(const void* codes, int m, int n, int bits, int group, void* q_u8, void* stream)

@@ -190,7 +190,7 @@ def run_stack(layers=32, tokens=100, peak=None):
            "needed_gbs": needed / ms_token * 1e-6, "pct_of_measured_peak": 100 * needed / ms_token * 1e-6 / (peak or _peak()),
            "thresholds": thr,
            "realised_sparsity": {k: {"mean": float(np.mean(v)), "min": float(np.min(v)), "max": float(np.max(v))} for k, v in sp.items()},
-           "packed_gb": sum(p.codes.numel() + 2 * p.scales.numel() + 2 * p.zeros.numel() for row in packs for p in row.values()) * 1e-9,
+           "packed_gb": sum(p.nbytes for row in packs for p in row.values()) * 1e-9,
            "device_status": status}
     return out
 

@@ -34,8 +34,9 @@ def test_every_declared_symbol_is_exported(L):
 def test_status_strings(L):
     assert binding.status_string(0) == "SPQT_OK"
     assert binding.status_string(2) == "SPQT_ERR_UNSUPPORTED"
+    assert binding.status_string(6) == "SPQT_ERR_TIMEOUT"
     assert binding.status_string(99) == "SPQT_ERR_UNKNOWN"
-    assert L.spqt_version() >= 1000
+    assert L.spqt_version() >= 2000
 
 
 @pytest.mark.parametrize("m,n,bits,group,B", [(4096, 4096, 4, 128, 64), (14336, 4096, 4, 64, 32),
@@ -44,7 +45,7 @@ def test_packed_sizes(L, m, n, bits, group, B):
     s = binding.spqt_packed_sizes(m, n, bits, group)
     R = m // group
     assert s.codes_bytes == R * n * B
-    assert s.scales_bytes == R * n * 2 and s.zeros_bytes == R * n * 2
+    assert s.scale_zero_bytes == R * n * 4
     assert s.gemv_workspace_bytes >= R * 4 + 4 * (m + R)      # counters + one worker's partials
     assert s.gemv_workspace_bytes < 64 << 20
 
@@ -66,23 +67,29 @@ def test_bad_arguments_launch_nothing(L):
     a16 = (base + 15) // 16 * 16            # 16-byte aligned fake "device" address; never dereferenced
     ws = binding.spqt_packed_sizes(128, 8, 4, 128).gemv_workspace_bytes
     # null pointers
-    assert L.spqt_pack(None, 128, 8, 8, 4, 128, a16, a16, a16, None) == 1
+    assert L.spqt_pack(None, 128, 8, 8, 4, 128, a16, a16, None) == 1
     assert L.spqt_sparsify(None, 8, 0.5, a16, a16, None) == 1
-    assert L.spqt_sparse_gemv(a16, a16, a16, 128, 8, 4, 128, a16, None, a16, a16, a16, ws, None) == 1
-    assert L.spqt_dense_gemv(a16, a16, None, 128, 8, 4, 128, a16, a16, a16, ws, None) == 1
+    assert L.spqt_sparse_gemv(a16, a16, 128, 8, 4, 128, a16, None, a16, a16, a16, ws, None) == 1
+    assert L.spqt_dense_gemv(a16, None, 128, 8, 4, 128, a16, a16, a16, ws, None) == 1
+    assert L.spqt_sparsify_gemv(a16, a16, 128, 8, 4, 128, a16, 0.5, a16, None, a16, a16, ws, None) == 1
     # ldw < n, negative n
-    assert L.spqt_pack(a16, 128, 8, 4, 4, 128, a16, a16, a16, None) == 1
+    assert L.spqt_pack(a16, 128, 8, 4, 4, 128, a16, a16, None) == 1
     assert L.spqt_sparsify(a16, -1, 0.5, a16, a16, None) == 1
-    # unsupported format
-    assert L.spqt_pack(a16, 100, 8, 8, 4, 128, a16, a16, a16, None) == 2
-    assert L.spqt_sparse_gemv(a16, a16, a16, 128, 8, 8, 128, a16, a16, a16, a16, a16, ws, None) == 2
+    # unsupported format; more columns than the 16-bit column numbers of the list reach
+    assert L.spqt_pack(a16, 100, 8, 8, 4, 128, a16, a16, None) == 2
+    assert L.spqt_sparse_gemv(a16, a16, 128, 8, 8, 128, a16, a16, a16, a16, a16, ws, None) == 2
+    big = binding.spqt_packed_sizes(128, 70000, 4, 128).gemv_workspace_bytes
+    assert L.spqt_sparse_gemv(a16, a16, 128, 70000, 4, 128, a16, a16, a16, a16, a16, big, None) == 2
     # misaligned
-    assert L.spqt_pack(a16, 128, 8, 8, 4, 128, a16 + 4, a16, a16, None) == 3
-    assert L.spqt_sparse_gemv(a16 + 8, a16, a16, 128, 8, 4, 128, a16, a16, a16, a16, a16, ws, None) == 3
+    assert L.spqt_pack(a16, 128, 8, 8, 4, 128, a16 + 4, a16, None) == 3
+    assert L.spqt_sparse_gemv(a16 + 8, a16, 128, 8, 4, 128, a16, a16, a16, a16, a16, ws, None) == 3
+    assert L.spqt_sparse_gemv(a16, a16, 128, 8, 4, 128, a16 + 1, a16, a16, a16, a16, ws, None) == 3
     assert L.spqt_sparsify(a16 + 1, 8, 0.5, a16, a16, None) == 3
     # workspace too small
-    assert L.spqt_sparse_gemv(a16, a16, a16, 128, 8, 4, 128, a16, a16, a16, a16, a16, ws - 1, None) == 4
-    assert L.spqt_dense_gemv(a16, a16, a16, 128, 8, 4, 128, a16, a16, a16, 16, None) == 4
+    assert L.spqt_sparse_gemv(a16, a16, 128, 8, 4, 128, a16, a16, a16, a16, a16, ws - 1, None) == 4
+    assert L.spqt_dense_gemv(a16, a16, 128, 8, 4, 128, a16, a16, a16, 16, None) == 4
     assert L.spqt_set_tuning(-1, 0) == 1
+    assert L.spqt_set_tuning(0, 4) == 1
     assert L.spqt_workspace_status(None, 128, 128, None, None) == 1
+    assert L.spqt_static_status(100, 128, None, None) == 1
     assert binding.spqt_launch_count() == before

@@ -49,7 +49,7 @@ def test_static_scratch_entry_point_refuses_what_does_not_fit_or_is_malformed():
     L = binding.lib()
     p, xd, idx, cnt = _case(128, 64, 128, 3, 0.5)
     y = torch.empty(128, dtype=torch.float16, device="cuda")
-    args = lambda m, n, bits, group: (p.codes.data_ptr(), p.scales.data_ptr(), p.zeros.data_ptr(), m, n, bits, group,
+    args = lambda m, n, bits, group: (p.codes.data_ptr(), p.scale_zero.data_ptr(), m, n, bits, group,
                                       xd.data_ptr(), idx.data_ptr(), cnt.data_ptr(), y.data_ptr(), None)
     before = binding.spqt_launch_count()
     assert L.spqt_sparse_gemv_static(*args(128, 64, 5, 128)) == 2          # unsupported format
