@@ -91,14 +91,15 @@ def realised_sparsity(x: np.ndarray, t: float) -> float:
     return float(np.count_nonzero(~(a > np.float32(t)))) / max(1, x.size)
 
 
-def lossless_weights(m: int, n: int, a: int = 5, b: int = 3) -> np.ndarray:
-    """W[j][k] = ((a*j + b*k) mod 16) / 16 with a odd: every run of >= 16
-    consecutive rows of a column holds both 0 and 15/16, so a 4-bit min/max
-    quantizer reproduces the matrix exactly (scale 1/16, offset 0)."""
-    assert a % 2 == 1
+def lossless_weights(m: int, n: int, a: int = 5, b: int = 3, levels: int = 16) -> np.ndarray:
+    """W[j][k] = ((a*j + b*k) mod levels) / levels with a odd and levels a power of two (16 for
+    4-bit codes, 8 for 3-bit ones): every run of >= levels consecutive rows of a column holds both 0
+    and (levels-1)/levels, so a min/max quantizer with that many levels reproduces the matrix exactly
+    (scale 1/levels, offset 0)."""
+    assert a % 2 == 1 and levels in (8, 16)
     j = np.arange(m, dtype=np.int64)[:, None]
     k = np.arange(n, dtype=np.int64)[None, :]
-    return (((a * j + b * k) % 16).astype(np.float32) / 16.0).astype(np.float16)
+    return (((a * j + b * k) % levels).astype(np.float32) / float(levels)).astype(np.float16)
 
 
 def small_rational_activations(n: int, seed: int) -> np.ndarray:

@@ -155,21 +155,29 @@ def test_one_hot_probes_return_the_dequantized_column(bits, group):
         assert np.all(np.abs(y.astype(np.float64) - y_ref) <= (2.0**-11 + 2.0**-20) * np.abs(y_ref) + 2.0**-25)
 
 
-@pytest.mark.parametrize("group", [64, 128])
-def test_lossless_family_is_bit_exact(group):
-    # (4-bit only: the family needs 16 levels)
+@pytest.mark.parametrize("bits,group", GEMV_FORMATS)
+def test_lossless_family_is_bit_exact(bits, group):
+    """W = ((5j + 3k) mod 2^bits) / 2^bits quantizes without loss, x in {+-1, +-2, +-1/2}: every partial sum
+    is exact in fp32, so the sparse, fused and dense results must equal the oracle's bit for bit."""
     m, n = 4 * group, 700
-    W = inputs.lossless_weights(m, n)
+    W = inputs.lossless_weights(m, n, levels=1 << bits)
     x = inputs.small_rational_activations(n, seed=12)
-    p = pack_on_gpu(W, 4, group)
+    p = pack_on_gpu(W, bits, group)
     codes, s, z = packed_to_host(p)
-    ws = binding.new_workspace(m, n, 4, group)
+    ws = binding.new_workspace(m, n, bits, group)
     for t in (0.25, 0.75, 1.5):
         y, idx, cnt = run_sparse(p, x, t, ws)
-        y_ref, _ = oracle.sparse_gemv(codes, s, z, m, n, x, idx, 4, group)
+        y_ref, _ = oracle.sparse_gemv(codes, s, z, m, n, x, idx, bits, group)
         assert np.array_equal(y.astype(np.float64), y_ref.astype(np.float16).astype(np.float64))
         y2, _, _ = run_sparse(p, x, t, ws, shuffle_seed=3)       # any index order
         assert np.array_equal(y2, y)
+        yf, _, _ = binding.spqt_sparsify_gemv(p, dev(x), t, ws)
+        torch.cuda.synchronize()
+        assert np.array_equal(yf.cpu().numpy(), y)
+    yd = binding.spqt_dense_gemv(p, dev(x), ws)
+    torch.cuda.synchronize()
+    yd_ref, _ = oracle.dense_gemv(codes, s, z, m, n, x, bits, group)
+    assert np.array_equal(yd.cpu().numpy().astype(np.float64), yd_ref.astype(np.float16).astype(np.float64))
 
 
 def test_index_order_does_not_matter_beyond_rounding_and_calls_are_reproducible():
@@ -277,6 +285,19 @@ def test_checked_mode_refuses_bad_index_lists():
     # and the next well-formed call on a fresh workspace is untouched by all that
     y, status = run_checked(idx, c)
     assert status == 0 and np.array_equal(y.view(np.uint16), y_plain.view(np.uint16))
+    # the verdict is per call: after a refusal the same workspace serves a well-formed list normally,
+    # while its status word stays set until the caller zeroes the workspace
+    ws = binding.new_workspace(m, n, bits, group)
+    try:
+        binding.spqt_set_debug(True)
+        bad_idx = idx.clone(); bad_idx[0] = n
+        y_bad = binding.spqt_sparse_gemv(p, xd, bad_idx, cnt, ws).cpu().numpy()
+        y_good = binding.spqt_sparse_gemv(p, xd, idx, cnt, ws).cpu().numpy()
+    finally:
+        binding.spqt_set_debug(False)
+    assert not y_bad.any()
+    assert np.array_equal(y_good.view(np.uint16), y_plain.view(np.uint16))
+    assert binding.spqt_workspace_status(ws, m, group) == 2
 
 
 @pytest.mark.parametrize("m,group", [(4096, 128), (8192, 128), (2048, 64)])
@@ -442,7 +463,7 @@ def test_config_single_gemv_4096x4096_seed0_every_row():
 @pytest.mark.parametrize("name,m,n,dist", [l for l in inputs.LLAMA3_8B_LINEARS if l[0] in ("q", "k", "gate", "down")])
 def test_llama3_8b_shapes_on_sampled_rows(name, m, n, dist):
     bits, group = 4, 128
-    W = inputs.weights(m, n, seed=hash(name) % 1000)
+    W = inputs.weights(m, n, seed={"q": 401, "k": 402, "gate": 403, "down": 404}[name])
     x = inputs.activations(n, seed=7, dist=dist)
     p = pack_on_gpu(W, bits, group)
     codes, s, z = packed_to_host(p)
@@ -555,3 +576,109 @@ def test_kernels_are_counted():
     x = dev(inputs.activations(256, seed=1))
     binding.spqt_sparsify(x, 0.5)
     assert binding.spqt_launch_count() == before + 1
+
+
+# ------------------------------------------------------------------ a1: zeros of both signs in a group
+
+@pytest.mark.parametrize("bits,group", FORMATS)
+def test_pack_of_groups_with_zeros_of_both_signs_is_byte_identical(bits, group):
+    """Pruned weights: groups whose minimum (or maximum) is zero with -0.0 and +0.0 both present, in either
+    order, and all-zero groups of either sign.  The stored offset is +0.0 whatever the order."""
+    m, n = 2 * group, 136                      # 136 columns: the 4-bit G=64 kernel's vector path too
+    W = np.abs(inputs.weights(m, n, seed=5))
+    W[::3] = np.float16(0.0)
+    W[1::7] = np.float16(-0.0)
+    W[:, 5] = -W[:, 5]                         # maximum zero
+    W[:group, 9] = np.float16(-0.0)            # a whole group of -0.0
+    W[group:, 9] = np.float16(0.0)
+    W[0, 11], W[1, 11] = np.float16(0.0), np.float16(-0.0)
+    W[0, 12], W[1, 12] = np.float16(-0.0), np.float16(0.0)
+    codes, s, z = oracle.pack(W, bits, group)
+    assert not z[:, [0, 9, 11, 12]].view(np.uint16).any()          # +0.0 offsets
+    gc, gs, gz = packed_to_host(pack_on_gpu(W, bits, group))
+    assert np.array_equal(gs.view(np.uint16), s.view(np.uint16))
+    assert np.array_equal(gz.view(np.uint16), z.view(np.uint16))
+    assert np.array_equal(gc, codes)
+
+
+# ------------------------------------------------------------------ lists longer than the shared-memory window
+
+@pytest.mark.parametrize("bits,group", [(4, 128), (3, 64)])
+@pytest.mark.parametrize("m_blocks,n", [(300, 20000), (2, 20000), (5, 32768), (160, 32768)])
+def test_lists_longer_than_the_shared_memory_window(bits, group, m_blocks, n):
+    """A CTA keeps 12288 list entries in shared memory at a time; with more active entries than that in
+    its slices the window is rebuilt between spans -- in the sparse call, in the call that collects the
+    indices itself (which then also writes the returned list span by span) and in the dense call over an
+    odd number of columns.  Index list bit-exact, y on sampled rows against the oracle, and the one-launch
+    and two-launch routes agree bit for bit."""
+    m = m_blocks * group
+    nn = n - 1 if n == 20000 else n            # 19999 columns: the dense call takes the list path as well
+    W = inputs.weights(m, nn, seed=m_blocks + n)
+    x = inputs.activations(nn, seed=77 + n)
+    p = pack_on_gpu(W, bits, group)
+    codes, s, z = packed_to_host(p)
+    ws = binding.new_workspace(m, nn, bits, group)
+    rows = np.unique(np.concatenate([np.random.Generator(np.random.PCG64(3)).integers(0, m, size=64),
+                                     [0, group - 1, group, m - group, m - 1]])).astype(np.int32)
+    xd = dev(x)
+    for sp in (0.0, 0.1):
+        t = inputs.threshold_for_sparsity(x, sp)
+        ref_idx, ref_cnt = oracle.sparsify(x, t)
+        assert ref_cnt > 12288
+        y, idx, cnt = run_sparse(p, x, t, ws)
+        assert cnt == ref_cnt and np.array_equal(idx, ref_idx)
+        y_ref, bound = oracle.sparse_gemv(codes, s, z, m, nn, x, ref_idx, bits, group, rows=rows)
+        check_y(y[rows], y_ref, bound, "sparse, long list, sparsity %.1f" % sp)
+        idx_t = torch.full((nn,), -7, dtype=torch.int32, device="cuda")
+        cnt_t = torch.full((1,), -7, dtype=torch.int32, device="cuda")
+        yf, _, _ = binding.spqt_sparsify_gemv(p, xd, t, ws, idx_t, cnt_t)
+        torch.cuda.synchronize()
+        got = idx_t.cpu().numpy()
+        assert int(cnt_t.item()) == ref_cnt
+        assert np.array_equal(got[:ref_cnt], ref_idx) and np.all(got[ref_cnt:] == -7)
+        assert np.array_equal(yf.cpu().numpy().view(np.uint16), y.view(np.uint16))
+    yd = binding.spqt_dense_gemv(p, xd, ws)
+    torch.cuda.synchronize()
+    yd_ref, dbound = oracle.dense_gemv(codes, s, z, m, nn, x, bits, group, rows=rows)
+    check_y(yd.cpu().numpy()[rows], yd_ref, dbound, "dense, long x")
+    assert binding.spqt_workspace_status(ws, m, group) == 0
+
+
+# ------------------------------------------------------------------ Llama-2-70B-shaped linears at full size
+
+@pytest.mark.parametrize("bits,group", FORMATS)
+@pytest.mark.parametrize("name,m,n", [("up", 28672, 8192), ("down", 8192, 28672)])
+def test_llama2_70b_mlp_shapes_at_full_size_on_sampled_rows(bits, group, name, m, n):
+    """8192 -> 28672 and 28672 -> 8192 in every format, x ~ Laplace with 1 % of the entries multiplied by 20,
+    50 % sparsity, in the launch configuration the benchmark times: sparse, index collection in the same
+    launch, and dense, on sampled rows; packed bytes of two block-rows against the oracle's pack."""
+    W = inputs.weights(m, n, seed=900 + bits + group + (0 if name == "up" else 1))
+    x = inputs.activations(n, seed=901, outlier_frac=0.01, outlier_scale=20.0)
+    p = pack_on_gpu(W, bits, group)
+    codes, s, z = packed_to_host(p)
+    B = oracle.block_bytes(bits, group)
+    for r in (0, m // group - 1):
+        c_ref, s_ref, z_ref = oracle.pack(np.ascontiguousarray(W[r * group:(r + 1) * group]), bits, group)
+        assert np.array_equal(codes[r * n * B:(r + 1) * n * B], c_ref)
+        assert np.array_equal(s[r], s_ref[0]) and np.array_equal(z[r], z_ref[0])
+    del W
+    ws = binding.new_workspace(m, n, bits, group)
+    rows = np.unique(np.concatenate([np.random.Generator(np.random.PCG64(8)).integers(0, m, size=96),
+                                     [0, group - 1, group, m - group, m - 1]])).astype(np.int32)
+    t = inputs.threshold_for_sparsity(x, 0.5)
+    y, idx, cnt = run_sparse(p, x, t, ws)
+    ref_idx, ref_cnt = oracle.sparsify(x, t)
+    assert cnt == ref_cnt and np.array_equal(idx, ref_idx)
+    y_ref, bound = oracle.sparse_gemv(codes, s, z, m, n, x, ref_idx, bits, group, rows=rows)
+    check_y(y[rows], y_ref, bound, "%s sparse" % name)
+    idx_t = torch.full((n,), -7, dtype=torch.int32, device="cuda")
+    cnt_t = torch.full((1,), -7, dtype=torch.int32, device="cuda")
+    yf, _, _ = binding.spqt_sparsify_gemv(p, dev(x), t, ws, idx_t, cnt_t)
+    torch.cuda.synchronize()
+    assert int(cnt_t.item()) == ref_cnt and np.array_equal(idx_t.cpu().numpy()[:ref_cnt], ref_idx)
+    assert np.array_equal(yf.cpu().numpy().view(np.uint16), y.view(np.uint16))
+    yd = binding.spqt_dense_gemv(p, dev(x), ws)
+    torch.cuda.synchronize()
+    yd_ref, dbound = oracle.dense_gemv(codes, s, z, m, n, x, bits, group, rows=rows)
+    check_y(yd.cpu().numpy()[rows], yd_ref, dbound, "%s dense" % name)
+    assert binding.spqt_workspace_status(ws, m, group) == 0

@@ -270,21 +270,23 @@ def test_one_hot_probe_returns_the_column():
         assert np.array_equal(b, 1.5 * np.abs(col))
 
 
-def test_lossless_family_gemv_equals_integer_arithmetic():
-    m, n = 256, 300
-    W = inputs.lossless_weights(m, n)
+@pytest.mark.parametrize("bits,group", [(4, 128), (4, 64), (3, 128), (3, 64)])
+def test_lossless_family_gemv_equals_integer_arithmetic(bits, group):
+    m, n, levels = 256, 300, 1 << bits
+    W = inputs.lossless_weights(m, n, levels=levels)
     x = inputs.small_rational_activations(n, seed=4)
-    codes, s, z = oracle.pack(W, 4, 128)
+    codes, s, z = oracle.pack(W, bits, group)
+    assert np.all(s.astype(np.float64) == 1.0 / levels) and not z.any()
     t = 0.75                                               # drops the +-0.5 entries
     idx, cnt = oracle.sparsify(x, t)
     keep = np.abs(x.astype(np.float64)) > t
     assert np.array_equal(idx, np.nonzero(keep)[0])
     j = np.arange(m)[:, None]
     k = np.arange(n)[None, :]
-    num = ((5 * j + 3 * k) % 16).astype(np.int64)          # 16 * W, integers
+    num = ((5 * j + 3 * k) % levels).astype(np.int64)      # levels * W, integers
     x2 = np.rint(x.astype(np.float64) * 2).astype(np.int64)  # 2 * x, integers
-    ref = (num[:, keep] @ x2[keep]) / 32.0                 # exact
-    y, _ = oracle.sparse_gemv(codes, s, z, m, n, x, idx, 4, 128)
+    ref = (num[:, keep] @ x2[keep]) / (2.0 * levels)       # exact
+    y, _ = oracle.sparse_gemv(codes, s, z, m, n, x, idx, bits, group)
     assert np.array_equal(y, ref)
 
 
