@@ -84,11 +84,13 @@ constexpr int kMaxFusedN = 32768;        // longest x the in-kernel scan handles
 constexpr int kMaxPieces = kMaxFusedN / 256;
 
 enum : int { kModeList = 0, kModeFused = 1, kModeDense = 2 };
-enum : int { kFlagIdentity = 1, kFlagXs = 2 };
+enum : int { kFlagIdentity = 1, kFlagXs = 2, kFlagStatic = 4 };
+constexpr int kMaxStaticSeg = 8;         // block-rows per CTA the static-partition ablation handles
 
 static int g_tune_ctas = 0;  // 0 = one CTA per SM
 int g_no_pdl = 0;            // 1 = plain stream-ordered launches (also read by the index-collection launch)
 static int g_no_cluster = 0; // 1 = never launch thread-block clusters
+static int g_static_partition = 0;  // 1 = ablation: static partition of the matrix columns instead of the list
 
 }  // namespace spqt
 
@@ -118,6 +120,7 @@ struct GemvSmem {
     alignas(16) float xred[kMaxCluster][G + 4];
     uint64_t xbar;                                 // counts their arrivals
     alignas(16) int tot[kMaxPieces];               // in-kernel scan: active entries of every 256 entries of x
+    int static_table[kMaxStaticSeg][kWorkers + 1]; // ablation: list positions of a static column partition
     alignas(16) unsigned ent[kCap];                // the resident part of the list: x bits << 16 | column
 };
 
@@ -364,12 +367,58 @@ gemv_kernel(const GemvArgs a)
             if (c == 0 && tid == 0) *a.count_out = count;
         }
         pc.set_count(count);
+        if (FUSED && (a.flags & kFlagStatic) && pc.r_last - pc.r_first < kMaxStaticSeg) {
+            // Ablation, the paper's "sparse without load balancing": every CTA, and inside it every warp,
+            // takes a fixed range of the matrix COLUMNS of its block-row and works on whatever active
+            // entries fall into it.  Boundary j of the CTA's column range in a block-row becomes the list
+            // position "active entries below that column", read off the scan: the totals of the pieces
+            // below, plus the activity bits below the column inside its piece.
+            const int nseg = pc.r_last - pc.r_first + 1;
+            int tot4[4];
+            {
+                const int4 t4 = *reinterpret_cast<const int4*>(&sm.tot[lane * 4]);
+                tot4[0] = t4.x; tot4[1] = t4.y; tot4[2] = t4.z; tot4[3] = t4.w;
+            }
+#pragma unroll 1
+            for (int q = warp; q < nseg * (kWorkers + 1); q += kWarps) {
+                const int sgi = q / (kWorkers + 1), j = q % (kWorkers + 1);
+                unsigned u0, u1;
+                pc.fraction(pc.r_first + sgi, &u0, &u1);
+                const int k0 = (int)((u0 * (unsigned)n) / (unsigned)P), k1 = (int)((u1 * (unsigned)n) / (unsigned)P);
+                const int kb = k0 + (int)(((long long)(k1 - k0) * j) / kWorkers);
+                const int piece = kb >> 8, lane_of = (kb & 255) >> 3, bit = kb & 7;
+                unsigned below = 0;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) below += (lane * 4 + i < piece) ? (unsigned)tot4[i] : 0u;
+                const unsigned m8 = piece < nv ? pm[piece * 32 + lane] : 0u;
+                below += lane < lane_of ? (unsigned)__popc(m8) : (lane == lane_of ? (unsigned)__popc(m8 & ((1u << bit) - 1u)) : 0u);
+                const int posk = (int)__reduce_add_sync(0xffffffffu, below);
+                if (lane == 0) sm.static_table[sgi][j] = posk;
+            }
+            __syncthreads();
+            pc.table = &sm.static_table[0][0];
+        }
         // list positions this CTA will read: the union of its slices.  (A piece that spans several
         // block-rows ends the first one and begins the last one: its slices cover the whole list
         // between them.)
         int need_lo = 0, need_hi = count;
         if (pc.r_first == pc.r_last) pc.slice(pc.r_first, &need_lo, &need_hi);
+        if (pc.table != nullptr && pc.r_first != pc.r_last) {
+            // a static partition: the CTA's column ranges in its first and last block-row, and whole rows between
+            int a0, b0, a1, b1;
+            pc.slice(pc.r_first, &a0, &b0);
+            pc.slice(pc.r_last, &a1, &b1);
+            need_lo = pc.r_last - pc.r_first > 1 ? 0 : min(a0, a1);
+            need_hi = pc.r_last - pc.r_first > 1 ? count : max(b0, b1);
+        }
         resident = (need_hi - need_lo) <= kCap;
+        if (!resident && pc.table != nullptr) {
+            // (the ablation does not rebuild windows: long lists take the balanced partition)
+            pc.table = nullptr;
+            need_lo = 0;
+            need_hi = count;
+            if (pc.r_first == pc.r_last) pc.slice(pc.r_first, &need_lo, &need_hi);
+        }
         int olo = 0, ohi = 0;  // the part of the returned index list this CTA writes: its slice of block-row 0
         if (FUSED && pc.r_first == 0) pc.slice(0, &olo, &ohi);
         if (resident) {
@@ -1012,6 +1061,7 @@ static spqt_status launch_gemv(const Format& f, const void* codes, const void* m
     ga.count_out = fa.count_out;
     ga.flags = flags;
     if (MODE == kModeList && scratch_bytes(f.n, false) <= stage_area_bytes<G, BITS>()) ga.flags |= kFlagXs;
+    if (MODE == kModeFused && g_static_partition) ga.flags |= kFlagStatic;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(P);
     cfg.blockDim = dim3(kGemvThreads);
@@ -1231,10 +1281,11 @@ spqt_status spqt_set_debug(int on)
 
 spqt_status spqt_set_tuning(int gemv_ctas, int reserved)
 {
-    if (gemv_ctas < 0 || reserved < 0 || reserved > 3) return SPQT_ERR_INVALID_ARG;
+    if (gemv_ctas < 0 || reserved < 0 || reserved > 7) return SPQT_ERR_INVALID_ARG;
     spqt::g_tune_ctas = gemv_ctas;
     spqt::g_no_pdl = reserved & 1;
     spqt::g_no_cluster = (reserved >> 1) & 1;
+    spqt::g_static_partition = (reserved >> 2) & 1;
     return SPQT_OK;
 }
 

@@ -23,6 +23,9 @@ struct Piece {
     int R, P, c, count, unit, r_first, r_last;
     unsigned mP, mR;  // multipliers of magic_div for P and R, computed by the host
     unsigned qc, rc;  // count = qc * P + rc: keeps the slice arithmetic in 32 bits (the host checks R * P < 2^31)
+    // Ablation (no load balancing): list positions of the boundaries of a static partition of the matrix
+    // COLUMNS, [segment][kWorkers + 1] in shared memory; nullptr = the balanced partition of the list.
+    const int* table;
 
     // the block-rows of the piece do not depend on the count: computed while the count is being fetched
     __device__ __forceinline__ void init_rows(int R_, int P_, int c_, unsigned mP_, unsigned mR_)
@@ -31,6 +34,7 @@ struct Piece {
         mP = mP_;
         mR = mR_;
         unit = 1;
+        table = nullptr;
         const unsigned lo = (unsigned)c * (unsigned)R, hi = lo + (unsigned)R;
         r_first = (int)magic_div(lo, (unsigned)P, mP);
         r_last = (int)magic_div(hi - 1u, (unsigned)P, mP);
@@ -45,8 +49,21 @@ struct Piece {
     }
     // floor(u * count / P) for 0 <= u <= P
     __device__ __forceinline__ int scaled(unsigned u) const { return (int)(u * qc + magic_div(u * rc, (unsigned)P, mP)); }
+    // the fraction [u0, u1) / P of block-row `row` that belongs to this CTA
+    __device__ __forceinline__ void fraction(int row, unsigned* u0, unsigned* u1) const
+    {
+        const unsigned lo = (unsigned)c * (unsigned)R, hi = lo + (unsigned)R, base = (unsigned)row * (unsigned)P;
+        *u0 = (lo > base ? lo : base) - base;
+        *u1 = (hi < base + (unsigned)P ? hi : base + (unsigned)P) - base;
+    }
     __device__ __forceinline__ void slice(int row, int* a, int* b) const
     {
+        if (table != nullptr) {
+            const int* t = table + (row - r_first) * (kWorkers + 1);
+            *a = t[0];
+            *b = t[kWorkers];
+            return;
+        }
         const unsigned lo = (unsigned)c * (unsigned)R, hi = lo + (unsigned)R, base = (unsigned)row * (unsigned)P;
         const unsigned u0 = (lo > base ? lo : base) - base;
         const unsigned u1 = (hi < base + (unsigned)P ? hi : base + (unsigned)P) - base;
@@ -65,8 +82,14 @@ struct Piece {
 
 // The part [a,b) of the span [lo,hi) that worker warp `warp` processes: the span is cut into
 // kWorkers contiguous parts whose boundaries are multiples of 8 entries from lo.
-__device__ __forceinline__ void warp_part(int lo, int hi, int warp, int* a, int* b)
+__device__ __forceinline__ void warp_part(const Piece& pc, int r, int lo, int hi, int warp, int* a, int* b)
 {
+    if (pc.table != nullptr) {  // static column partition: the warp's column range, as list positions
+        const int* t = pc.table + (r - pc.r_first) * (kWorkers + 1);
+        *a = t[warp];
+        *b = t[warp + 1];
+        return;
+    }
     const int q = (hi - lo + 7) >> 3;
     const int ua = (warp * q) / kWorkers, ub = ((warp + 1) * q) / kWorkers;
     *a = lo + 8 * ua;
@@ -89,7 +112,7 @@ struct Walker {
             seg_hi = p1;
             lo = p0;
             hi = resident ? p1 : min(p1, p0 + kCap);
-            warp_part(lo, hi, warp, &pos, &end);
+            warp_part(pc, r, lo, hi, warp, &pos, &end);
         }
     }
     __device__ __forceinline__ void first(const Piece& pc, int warp, bool resident)
@@ -103,7 +126,7 @@ struct Walker {
         if (hi < seg_hi) {
             lo = hi;
             hi = min(seg_hi, lo + kCap);
-            warp_part(lo, hi, warp, &pos, &end);
+            warp_part(pc, r, lo, hi, warp, &pos, &end);
         } else {
             ++r;
             open_segment(pc, warp, resident);

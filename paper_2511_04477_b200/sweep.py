@@ -1,21 +1,16 @@
-"""Sparsity and format sweeps of the sparse GEMV against the same-layout dense GEMV.
+"""The benchmark's other workloads: sparsity sweep, format sweep, dense shape sweep and the 32-layer stack.
 
-    python -m paper_2511_04477_b200.sweep sparsity      # 0-90 % on 4096x14336 and 14336x4096, int4 g128
-    python -m paper_2511_04477_b200.sweep formats       # Llama-2-70B-shaped linears x {int4,int3} x {g64,g128}, 50 %
-    python -m paper_2511_04477_b200.sweep stack         # 32-layer Llama-3-8B-shaped stack, thresholds calibrated for 40 %
-
+Used by ``bench.py --config sweep|formats|dense|stack`` (and, in reduced form, by its default line).
 Each case packs several distinct weight copies (together well above the 126 MB L2), visits them
-round-robin inside one CUDA graph and times graph replays with CUDA events.  Printed per case: device
-microseconds per call, effective GB/s over the bytes the method needs, percent of the measured HBM
-peak, speed-up over the dense GEMV on the same packed buffers, and the ideal 1/(1 - sparsity).
-Weights are random-init on the device; x and thresholds come from the seeded input module.
+round-robin inside one CUDA graph and times graph replays with CUDA events on the launching stream.
+Weights are random-init on the device (their values do not affect timing); x and thresholds come
+from the seeded input module.
 """
 from __future__ import annotations
 
 import json
 import math
 import os
-import sys
 
 import numpy as np
 import torch
@@ -23,23 +18,26 @@ import torch
 from . import binding, inputs
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+L2_BYTES = 126e6
 
 
-def _peak():
+def hbm_peak():
+    """(GB/s, "measured" | "fallback"): the measured copy bandwidth of this machine's B200s."""
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
-            return float(json.load(f)["hbm_gbs"])
+            return float(json.load(f)["hbm_gbs"]), "measured"
     except Exception:
-        return 6650.0
+        return 6650.0, "fallback"
 
 
 def needed_bytes(m, n, count, bits, group):
+    """Algorithmic bytes of one GEMV: the active blocks with their scale and zero, x, the list, y."""
     R, B = m // group, group * bits // 8
     return count * R * (B + 4) + 2 * n + 4 * count + 4 + 2 * m
 
 
 def graph_us(fn, calls, replays=20):
-    """Median device time per call of `calls` calls captured in one graph."""
+    """(median, min) device microseconds per call of `calls` calls captured in one graph."""
     s = torch.cuda.Stream()
     with torch.cuda.stream(s):
         for i in range(min(calls, 4)):
@@ -59,21 +57,29 @@ def graph_us(fn, calls, replays=20):
             e1.record(s)
             e1.synchronize()
             ts.append(e0.elapsed_time(e1) * 1e3 / calls)
-    return float(np.median(ts))
+    return float(np.median(ts)), float(np.min(ts))
 
 
-def make_copies(m, n, bits, group, copies):
+def make_copies(m, n, bits, group, copies, seed0=0):
     g = torch.Generator(device="cuda")
     out = []
     for c in range(copies):
-        g.manual_seed(c)
+        g.manual_seed(seed0 + c)
         W = torch.empty((m, n), dtype=torch.float32, device="cuda").normal_(0.0, 0.02, generator=g).half()
         out.append(binding.spqt_pack(W, bits, group))
         del W
     return out
 
 
-def run_case(m, n, bits, group, sparsities, x, copies, peak):
+def copies_for(m, n, bits, group, at_least=4, at_most=160):
+    """Distinct packed copies so that the bytes between two visits of a copy exceed twice the L2."""
+    size = (m // group) * n * (group * bits // 8 + 4)
+    return int(min(at_most, max(at_least, math.ceil(2.4 * L2_BYTES / size))))
+
+
+def run_case(m, n, bits, group, sparsities, x, copies, peak, unbalanced=False):
+    """Sparse (given list), fused (list collected in the same launch) and dense GEMV on `copies` rotated
+    packed matrices, for every sparsity."""
     packs = make_copies(m, n, bits, group, copies)
     xd = torch.from_numpy(x).cuda()
     ws = binding.new_workspace(m, n, bits, group)
@@ -81,38 +87,92 @@ def run_case(m, n, bits, group, sparsities, x, copies, peak):
     idx = torch.empty(n, dtype=torch.int32, device="cuda")
     cnt = torch.zeros(1, dtype=torch.int32, device="cuda")
     calls = max(copies, 16)
-    t_dense = graph_us(lambda i, s: binding.spqt_dense_gemv(packs[i % copies], xd, ws, y, stream=s), calls)
+    t_dense, _ = graph_us(lambda i, s: binding.spqt_dense_gemv(packs[i % copies], xd, ws, y, stream=s), calls)
     rows = []
     for sp in sparsities:
         t = inputs.threshold_for_sparsity(x, sp)
         binding.spqt_sparsify(xd, t, idx, cnt)
         torch.cuda.synchronize()
         count = int(cnt.item())
-        t_sparse = graph_us(lambda i, s: binding.spqt_sparse_gemv(packs[i % copies], xd, idx, cnt, ws, y, stream=s), calls)
-        t_fused = graph_us(lambda i, s: binding.spqt_sparsify_gemv(packs[i % copies], xd, t, ws, idx, cnt, y, stream=s), calls)
+        t_sparse, _ = graph_us(lambda i, s: binding.spqt_sparse_gemv(packs[i % copies], xd, idx, cnt, ws, y, stream=s), calls)
+        t_fused, _ = graph_us(lambda i, s: binding.spqt_sparsify_gemv(packs[i % copies], xd, t, ws, idx, cnt, y, stream=s), calls)
         nb = needed_bytes(m, n, count, bits, group)
-        rows.append({"m": m, "n": n, "bits": bits, "group": group, "sparsity": 1.0 - count / n, "count": count,
-                     "sparse_us": t_sparse, "fused_us": t_fused, "dense_us": t_dense,
-                     "sparse_gbs": nb / t_sparse * 1e-3, "pct_of_measured_peak": 100 * nb / t_sparse * 1e-3 / peak,
-                     "dense_gbs": needed_bytes(m, n, n, bits, group) / t_dense * 1e-3,
-                     "speedup_vs_dense": t_dense / t_sparse, "ideal": 1.0 / max(1e-9, count / n)})
+        row = {"m": m, "n": n, "bits": bits, "group": group, "sparsity": 1.0 - count / n, "count": count,
+               "copies": copies, "sparse_us": t_sparse, "fused_us": t_fused, "dense_us": t_dense,
+               "sparse_gbs": nb / t_sparse * 1e-3, "frac_of_peak": nb / t_sparse * 1e-3 / peak,
+               "fused_gbs": (nb + 2 * n + 4 * count + 4) / t_fused * 1e-3,
+               "fused_frac_of_peak": (nb + 2 * n + 4 * count + 4) / t_fused * 1e-3 / peak,
+               "dense_gbs": needed_bytes(m, n, n, bits, group) / t_dense * 1e-3,
+               "dense_frac_of_peak": needed_bytes(m, n, n, bits, group) / t_dense * 1e-3 / peak,
+               "speedup_vs_dense": t_dense / t_sparse, "fused_speedup_vs_dense": t_dense / t_fused,
+               "ideal": 1.0 / max(1e-9, count / n)}
+        if unbalanced:
+            try:
+                binding.spqt_set_tuning(0, 4)   # static column partition, no load balancing
+                t_unb, _ = graph_us(lambda i, s: binding.spqt_sparsify_gemv(packs[i % copies], xd, t, ws, idx, cnt, y, stream=s), calls)
+            finally:
+                binding.spqt_set_tuning(0, 0)
+            row["unbalanced_us"] = t_unb
+            row["unbalanced_speedup_vs_dense"] = t_dense / t_unb
+        rows.append(row)
+    status = binding.spqt_workspace_status(ws, m, group)
+    for r in rows:
+        r["device_status"] = status
     del packs
     torch.cuda.empty_cache()
     return rows
 
 
-def show(rows):
-    print("| m x n | fmt | sparsity | sparse us | +idx us | dense us | GB/s needed | % peak | x dense | ideal |")
-    print("|---|---|---|---|---|---|---|---|---|---|")
-    for r in rows:
-        print("| %dx%d | int%d g%d | %.1f%% | %.2f | %.2f | %.2f | %.0f | %.1f | %.2f | %.2f |" % (
-            r["m"], r["n"], r["bits"], r["group"], 100 * r["sparsity"], r["sparse_us"], r["fused_us"], r["dense_us"],
-            r["sparse_gbs"], r["pct_of_measured_peak"], r["speedup_vs_dense"], r["ideal"]), flush=True)
+def sparsity_sweep(peak, sparsities=None, copies=64, unbalanced=False):
+    """0-90 % on a 14336 -> 4096 down-projection and a 4096 -> 14336 up-projection, int4 g128, 64 rotated copies."""
+    sps = sparsities if sparsities is not None else [i / 10 for i in range(10)]
+    out = []
+    for (m, n, dist) in [(4096, 14336, "gauss"), (14336, 4096, "laplace")]:
+        x = inputs.activations(n, seed=3, dist=dist)
+        out += run_case(m, n, 4, 128, sps, x, copies, peak, unbalanced=unbalanced)
+    return out
 
 
-def copies_for(m, n, bits, group):
-    size = (m // group) * n * (group * bits // 8 + 4)
-    return int(min(64, max(4, math.ceil(512e6 / size))))
+def format_sweep(peak, shapes=None, formats=None):
+    """Llama-2-70B-shaped linears x {int4, int3} x {g128, g64} at 50 %, x with 1 % outliers x20."""
+    out = []
+    for (name, m, n, dist) in (shapes if shapes is not None else inputs.LLAMA2_70B_LINEARS):
+        x = inputs.activations(n, seed=5, dist=dist, outlier_frac=0.01, outlier_scale=20.0)
+        for (bits, group) in (formats if formats is not None else [(4, 128), (4, 64), (3, 128), (3, 64)]):
+            out += run_case(m, n, bits, group, [0.5], x, copies_for(m, n, bits, group, at_least=4, at_most=16), peak)
+    return out
+
+
+def dense_shape_sweep(peak):
+    """The dense zigzag GEMV on the paper's 15 shapes m in {2048, 4096, 8192} x k in {1024 ... 16384}
+    (its hyper-parameter study, Sec. 6), int4 g128, over the CTA counts the autotuner would try."""
+    out = []
+    for m in (2048, 4096, 8192):
+        for n in (1024, 2048, 4096, 8192, 16384):
+            copies = copies_for(m, n, 4, 128)
+            packs = make_copies(m, n, 4, 128, copies)
+            xd = torch.from_numpy(inputs.activations(n, seed=11)).cuda()
+            ws = binding.new_workspace(m, n, 4, 128)
+            y = torch.empty(m, dtype=torch.float16, device="cuda")
+            calls = max(copies, 16)
+            row = {"m": m, "n": n, "copies": copies}
+            best = None
+            for ctas in (0, 64, 96, 128, 148):
+                try:
+                    binding.spqt_set_tuning(ctas, 0)
+                    us, _ = graph_us(lambda i, s: binding.spqt_dense_gemv(packs[i % copies], xd, ws, y, stream=s), calls, replays=10)
+                finally:
+                    binding.spqt_set_tuning(0, 0)
+                row["us_ctas_%d" % ctas] = us
+                if best is None or us < best[1]:
+                    best = (ctas, us)
+            row["best_ctas"], row["best_us"] = best
+            row["dense_gbs"] = needed_bytes(m, n, n, 4, 128) / best[1] * 1e-3
+            row["frac_of_peak"] = row["dense_gbs"] / peak
+            out.append(row)
+            del packs
+            torch.cuda.empty_cache()
+    return out
 
 
 STACK_SITES = [  # (site, stacked matrix rows, n, distribution of the site's input)
@@ -147,6 +207,7 @@ def build_stack(layers, tokens, sparsity=0.4, calib_vectors=64):
 def run_stack(layers=32, tokens=100, peak=None):
     """Per-token pass over the linear layers of the whole stack: 4 launches per layer (index collection
     inside the GEMV), one CUDA graph per token, device-timed; tokens/s of the linear layers."""
+    peak = peak or hbm_peak()[0]
     packs, thr, xs = build_stack(layers, tokens)
     ws = {site: binding.new_workspace(m, n, 4, 128) for (site, m, n, _) in STACK_SITES}
     y = {site: torch.empty(m, dtype=torch.float16, device="cuda") for (site, m, n, _) in STACK_SITES}
@@ -187,44 +248,11 @@ def run_stack(layers=32, tokens=100, peak=None):
     status = max(binding.spqt_workspace_status(ws[site], m, 128) for (site, m, n, _) in STACK_SITES)
     out = {"layers": layers, "tokens": tokens, "ms_per_token": ms_token, "tokens_per_s": 1e3 / ms_token,
            "launches_per_token": 4 * layers, "needed_gb_per_token": needed * 1e-9,
-           "needed_gbs": needed / ms_token * 1e-6, "pct_of_measured_peak": 100 * needed / ms_token * 1e-6 / (peak or _peak()),
+           "needed_gbs": needed / ms_token * 1e-6, "frac_of_peak": needed / ms_token * 1e-6 / peak,
            "thresholds": thr,
            "realised_sparsity": {k: {"mean": float(np.mean(v)), "min": float(np.min(v)), "max": float(np.max(v))} for k, v in sp.items()},
            "packed_gb": sum(p.nbytes for row in packs for p in row.values()) * 1e-9,
            "device_status": status}
+    del packs, graphs
+    torch.cuda.empty_cache()
     return out
-
-
-def main(argv):
-    which = argv[0] if argv else "sparsity"
-    peak = _peak()
-    binding.lib()
-    out = []
-    if which == "sparsity":
-        for (m, n, dist) in [(4096, 14336, "gauss"), (14336, 4096, "laplace")]:
-            x = inputs.activations(n, seed=3, dist=dist)
-            sps = [i / 10 for i in range(10)]
-            out += run_case(m, n, 4, 128, sps, x, copies_for(m, n, 4, 128), peak)
-    elif which == "formats":
-        for (name, m, n, dist) in inputs.LLAMA2_70B_LINEARS:
-            x = inputs.activations(n, seed=5, dist=dist, outlier_frac=0.01, outlier_scale=20.0)
-            for bits in (4, 3):
-                for group in (128, 64):
-                    out += run_case(m, n, bits, group, [0.5], x, copies_for(m, n, bits, group), peak)
-    elif which == "stack":
-        res = run_stack(peak=peak)
-        print("32-layer stack: %.3f ms per token over the linear layers, %.0f tokens/s, %d launches per token, "
-              "%.2f GB needed per token (%.0f GB/s, %.1f %% of the measured HBM peak); realised sparsity %s" % (
-                  res["ms_per_token"], res["tokens_per_s"], res["launches_per_token"], res["needed_gb_per_token"],
-                  res["needed_gbs"], res["pct_of_measured_peak"],
-                  {k: "%.3f (%.3f-%.3f)" % (v["mean"], v["min"], v["max"]) for k, v in res["realised_sparsity"].items()}))
-        print(json.dumps({"sweep": which, "hbm_peak_gbs": peak, "result": res}))
-        return
-    else:
-        raise SystemExit("usage: python -m paper_2511_04477_b200.sweep [sparsity|formats|stack]")
-    show(out)
-    print(json.dumps({"sweep": which, "hbm_peak_gbs": peak, "rows": out}))
-
-
-if __name__ == "__main__":
-    main(sys.argv[1:])

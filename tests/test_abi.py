@@ -89,7 +89,7 @@ def test_bad_arguments_launch_nothing(L):
     assert L.spqt_sparse_gemv(a16, a16, 128, 8, 4, 128, a16, a16, a16, a16, a16, ws - 1, None) == 4
     assert L.spqt_dense_gemv(a16, a16, 128, 8, 4, 128, a16, a16, a16, 16, None) == 4
     assert L.spqt_set_tuning(-1, 0) == 1
-    assert L.spqt_set_tuning(0, 4) == 1
+    assert L.spqt_set_tuning(0, 8) == 1
     assert L.spqt_workspace_status(None, 128, 128, None, None) == 1
     assert L.spqt_static_status(100, 128, None, None) == 1
     assert binding.spqt_launch_count() == before

@@ -682,3 +682,38 @@ def test_llama2_70b_mlp_shapes_at_full_size_on_sampled_rows(bits, group, name, m
     yd_ref, dbound = oracle.dense_gemv(codes, s, z, m, n, x, bits, group, rows=rows)
     check_y(yd.cpu().numpy()[rows], yd_ref, dbound, "%s dense" % name)
     assert binding.spqt_workspace_status(ws, m, group) == 0
+
+
+# ------------------------------------------------------------------ ablation: no load balancing
+
+@pytest.mark.parametrize("bits,group", [(4, 128), (3, 64)])
+@pytest.mark.parametrize("m_blocks,n", [(2, 300), (32, 4096), (48, 4096), (224, 4096), (3, 1111)])
+def test_static_column_partition_ablation_matches_the_oracle(bits, group, m_blocks, n):
+    """The paper's "sparse without load balancing": CTAs and warps take fixed ranges of the matrix columns.
+    Same index list and, up to the order of the partial sums, the same y -- also when the active entries
+    are all in one part of x (the case the static partition balances worst)."""
+    m = m_blocks * group
+    W = inputs.weights(m, n, seed=m + n + 11)
+    p = pack_on_gpu(W, bits, group)
+    codes, s, z = packed_to_host(p)
+    ws = binding.new_workspace(m, n, bits, group)
+    spread = inputs.activations(n, seed=13 + n)
+    clustered = spread.copy()
+    clustered[n // 3:] = (clustered[n // 3:].astype(np.float32) * 1e-3).astype(np.float16)   # active entries in the first third
+    for x, sp in ((spread, 0.5), (spread, 0.0), (clustered, 0.7)):
+        t = inputs.threshold_for_sparsity(x, sp)
+        ref_idx, ref_cnt = oracle.sparsify(x, t)
+        y_ref, bound = oracle.sparse_gemv(codes, s, z, m, n, x, ref_idx, bits, group)
+        idx = torch.full((n,), -7, dtype=torch.int32, device="cuda")
+        cnt = torch.full((1,), -7, dtype=torch.int32, device="cuda")
+        try:
+            binding.spqt_set_tuning(0, 4)
+            y, _, _ = binding.spqt_sparsify_gemv(p, dev(x), t, ws, idx, cnt)
+            torch.cuda.synchronize()
+        finally:
+            binding.spqt_set_tuning(0, 0)
+        got = idx.cpu().numpy()
+        assert int(cnt.item()) == ref_cnt
+        assert np.array_equal(got[:ref_cnt], ref_idx) and np.all(got[ref_cnt:] == -7)
+        check_y(y.cpu().numpy(), y_ref, bound, "static partition, sparsity %.1f" % sp)
+    assert binding.spqt_workspace_status(ws, m, group) == 0
