@@ -1,29 +1,37 @@
 #!/usr/bin/env python
 """Benchmark of the SpQt hot path on B200: one line of JSON on stdout.
 
-Workload (the configuration the metric is quoted on): the seven linear layers of
-one Llama-3-8B-shaped decoder layer at batch 1 -- q, k, v, o (4096->4096,
-4096->1024 x2, 4096->4096), gate/up (4096->14336), down (14336->4096) -- INT4
-codes, group 128, fp16 scale and zero, zigzag layout, 50 % activation sparsity.
-A *step* is one pass over those seven matrices: four index collections
-(attention input shared by q,k,v; attention output for o; MLP input shared by
-gate,up; MLP hidden for down) and the products with all seven matrices -- in
-four launches: matrices that share an input are packed as one (q|k|v, gate|up),
-and each launch collects its indices in its own prologue (spqt_sparsify_gemv).
-The seven matrices kept apart (7 launches, and 4 + 7 launches) are timed as well.  Eight distinct layer
-copies (about 0.93 GB of packed weights, far larger than the 126 MB L2) are
-visited round-robin so that weights really come from HBM.
+    python bench.py [--gpus N] [--steps K] [--warmup W]            the headline line (config "layer")
+    python bench.py --config sweep | formats | dense | stack       the other workloads, one JSON line each
+    python bench.py --impl reference                               the fp64 CPU oracle on a bounded sample
+
+Workload of the headline line (the configuration the metric is quoted on): the seven linear layers of
+one Llama-3-8B-shaped decoder layer at batch 1 -- q, k, v, o (4096->4096, 4096->1024 x2, 4096->4096),
+gate/up (4096->14336), down (14336->4096) -- INT4 codes, group 128, fp16 scale and zero, zigzag layout,
+50 % activation sparsity.  A *step* is one pass over those seven matrices: four index collections
+(attention input shared by q,k,v; attention output for o; MLP input shared by gate,up; MLP hidden for
+down) and the products with all seven matrices -- in four launches: matrices that share an input are
+packed as one (q|k|v, gate|up), and each launch collects its indices in its own prologue
+(spqt_sparsify_gemv).  Eight distinct layer copies (about 1.5 GB of packed weights, far larger than the
+126 MB L2) are visited round-robin so that weights really come from HBM.
 
 value  = effective GB/s over the bytes the method needs
-         (sum over GEMVs of count*R*(B+4) + 2n + 4count + 4 + 2m, plus 2n + 4count + 4
-         per index collection), whole job, inputs resident in HBM.
+         (sum over GEMVs of count*R*(B+4) + 2n + 4count + 4 + 2m, plus 2n + 4count + 4 per index
+         collection), whole job, inputs resident in HBM.  The K-step region is timed with CUDA events
+         on the launching stream and repeated until a quarter of a second of device time has been
+         timed; the value is that of the median region, the minimum is reported beside it.
 e2e    = the same metric through spqt_sparse_linear_host: x copied from pinned host memory,
          y written into pinned host memory by the kernel, the copy and the final wait of every
          call inside the timed region.
-roofline.achieved = algorithmic bytes per sparse-GEMV launch / its mean duration
-         (device events over a region that launches only the GEMVs of the same steps).
+roofline.achieved = algorithmic bytes per launch of the dominant kernel (gemv_kernel, index collection
+         inside: all four launches of a step are that kernel) / its mean duration in the timed region.
 
-`--impl reference` times the fp64 CPU oracle on a bounded sample of the same workload.
+The other workloads: `sweep` = sparsity 0-90 % on the 14336->4096 and 4096->14336 projections against the
+same-layout dense GEMV, 64 rotated weight copies, with the no-load-balancing ablation beside it;
+`formats` = Llama-2-70B-shaped linears x {int4, int3} x {g128, g64} at 50 % with outlier activations;
+`dense` = the dense zigzag GEMV on the paper's 15 shapes over several grid sizes; `stack` = a per-token
+pass over a 32-layer Llama-3-8B-shaped stack with thresholds calibrated once for 40 % (tokens/s of the
+linear layers).  The default line carries a short summary of each.
 """
 from __future__ import annotations
 
@@ -45,12 +53,11 @@ BITS, GROUP = 4, 128
 SPARSITY = 0.5
 LAYER_COPIES = 8
 X_POOL = 4            # distinct hidden states per site, rotated
-FALLBACK_HBM_GBS = 6650.0
+MIN_TIMED_S = 0.25    # device time to accumulate over repeated K-step regions
 METRIC = "sparse int4 GEMV effective HBM GB/s at 50% sparsity (Llama-3-8B-shaped decode-layer linears, batch 1)"
 
-# ncu (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes of one sparse-GEMV launch, from the
-# capture summarised in profiles/gemv_int4_g128_28672x8192_full.md (a 117 MB matrix; traffic grows in
-# proportion to the active blocks; 1.06 on the bench-sized 28672x4096 case, 1.12 on the 117 MB one).
+# ncu (dram__bytes_read.sum + dram__bytes_write.sum) / algorithmic bytes of one launch of the fused kernel on the
+# benchmark's stacked gate|up matrix (28672 x 4096, 50 %): traffic grows in proportion to the active blocks.
 NCU_TRAFFIC_RATIO = 1.06
 
 
@@ -61,15 +68,6 @@ def needed_bytes_gemv(m, n, count, bits=BITS, group=GROUP):
 
 def needed_bytes_sparsify(n, count):
     return 2 * n + 4 * count + 4
-
-
-def measured_peak():
-    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
-    try:
-        with open(p) as f:
-            return float(json.load(f)["hbm_gbs"]), "measured"
-    except Exception:
-        return FALLBACK_HBM_GBS, "fallback"
 
 
 class ClockSampler:
@@ -97,7 +95,7 @@ class ClockSampler:
 
     def __exit__(self, *a):
         if self.proc is not None:
-            time.sleep(0.15)
+            time.sleep(0.1)
             self.proc.terminate()
             try:
                 self.proc.wait(timeout=2)
@@ -192,12 +190,84 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+# --------------------------------------------------------------------------- the other workloads
+
+def roofline_obj(achieved, peak, peak_kind, bytes_per_launch, us_per_launch, kernel, traffic_ratio=NCU_TRAFFIC_RATIO):
+    return {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+            "traffic": traffic_ratio * bytes_per_launch if traffic_ratio else None, "peak_kind": "of " + peak_kind,
+            "kernel": kernel, "algorithmic_bytes_per_launch": bytes_per_launch, "avg_launch_us": us_per_launch}
+
+
+def other_config_line(which, local, quick=False):
+    """One of the other workloads as a dict in the same format as the headline line."""
+    import torch
+    from paper_2511_04477_b200 import sweep
+    peak, kind = sweep.hbm_peak()
+    base = {"n_gpus": 1, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int4/int3 codes, f32 accumulate, f16 in/out", "data": "synthetic", "unit": "GB/s"}
+    with ClockSampler(local) as clk:
+        if which == "sweep":
+            rows = sweep.sparsity_sweep(peak, sparsities=[0.5] if quick else None, copies=64, unbalanced=True)
+            at50 = [r for r in rows if abs(r["sparsity"] - 0.5) < 0.03]
+            r0 = at50[0]
+            nb = sweep.needed_bytes(r0["m"], r0["n"], r0["count"], 4, 128) + needed_bytes_sparsify(r0["n"], r0["count"])
+            line = dict(base, metric="sparse int4 GEMV effective HBM GB/s at 50% sparsity on the 14336->4096 projection "
+                                     "(sparsity sweep, 64 rotated weight copies)",
+                        value=r0["fused_gbs"], ms_per_step=r0["fused_us"] * 1e-3, steps=20, warmup=4,
+                        config={"workload": "sparsity sweep 0-90% on 4096x14336 and 14336x4096, int4 g128, sparse / index collection in "
+                                            "the same launch / dense on the same packed buffers; 64 distinct weight copies rotated (2 GB, L2 is 126 MB)"},
+                        roofline=roofline_obj(r0["fused_gbs"], peak, kind, nb, r0["fused_us"], "gemv_kernel<128,4,fused>"),
+                        speedup_vs_dense_at_50pct={"%dx%d" % (r["m"], r["n"]): {"given_list": r["speedup_vs_dense"], "index_collection_inside": r["fused_speedup_vs_dense"],
+                                                                                 "no_load_balancing": r.get("unbalanced_speedup_vs_dense")} for r in at50},
+                        rows=rows)
+        elif which == "formats":
+            shapes = [s for s in __import__("paper_2511_04477_b200.inputs", fromlist=["x"]).LLAMA2_70B_LINEARS if (not quick or s[0] == "up")]
+            rows = sweep.format_sweep(peak, shapes=shapes)
+            r0 = [r for r in rows if r["m"] == 28672 and r["bits"] == 4 and r["group"] == 128][0]
+            nb = sweep.needed_bytes(r0["m"], r0["n"], r0["count"], 4, 128) + needed_bytes_sparsify(r0["n"], r0["count"])
+            line = dict(base, metric="sparse GEMV effective HBM GB/s at 50% sparsity on the 8192->28672 projection, int4 g128 "
+                                     "(Llama-2-70B-shaped format sweep)",
+                        value=r0["fused_gbs"], ms_per_step=r0["fused_us"] * 1e-3, steps=20, warmup=4,
+                        config={"workload": "Llama-2-70B-shaped linears (8192x8192, 28672x8192, 8192x28672) x {int4,int3} x {g128,g64}, 50% sparsity, "
+                                            "x ~ Laplace with 1% of entries x20; >= 4 rotated weight copies (> 2x L2)"},
+                        roofline=roofline_obj(r0["fused_gbs"], peak, kind, nb, r0["fused_us"], "gemv_kernel<128,4,fused>", 1.13),
+                        frac_of_peak={"%dx%d int%d g%d" % (r["m"], r["n"], r["bits"], r["group"]): {
+                            "sparse": r["frac_of_peak"], "index_collection_inside": r["fused_frac_of_peak"], "dense": r["dense_frac_of_peak"],
+                            "speedup_vs_dense": r["fused_speedup_vs_dense"]} for r in rows},
+                        rows=rows)
+        elif which == "dense":
+            rows = sweep.dense_shape_sweep(peak)
+            best = max(rows, key=lambda r: r["frac_of_peak"])
+            nb = sweep.needed_bytes(best["m"], best["n"], best["n"], 4, 128)
+            line = dict(base, metric="dense zigzag int4 GEMV effective HBM GB/s, best of the 15 shapes of the paper's hyper-parameter study",
+                        value=best["dense_gbs"], ms_per_step=best["best_us"] * 1e-3, steps=10, warmup=4,
+                        config={"workload": "dense same-layout GEMV, m in {2048,4096,8192} x n in {1024..16384}, int4 g128, grids of 64/96/128/148 CTAs "
+                                            "and the built-in rule; rotated weight copies > 2x L2"},
+                        roofline=roofline_obj(best["dense_gbs"], peak, kind, nb, best["best_us"], "gemv_kernel<128,4,dense>", 1.0),
+                        rows=rows)
+        elif which == "stack":
+            res = sweep.run_stack(layers=32, tokens=40 if quick else 100, peak=peak)
+            nb = res["needed_gb_per_token"] * 1e9 / res["launches_per_token"]
+            line = dict(base, metric="tokens/s of the linear layers, 32-layer Llama-3-8B-shaped stack, int4 g128, thresholds calibrated for 40% sparsity",
+                        unit="tokens/s", value=res["tokens_per_s"], ms_per_step=res["ms_per_token"], steps=res["tokens"], warmup=3,
+                        config={"workload": "32 layers x (q|k|v, o, gate|up, down), 3.7 GB packed; per-site thresholds calibrated once on 64 pooled vectors; "
+                                            "fresh x per token; one CUDA graph per token (128 launches, index collection inside)"},
+                        roofline=roofline_obj(res["needed_gbs"], peak, kind, nb, res["ms_per_token"] * 1e3 / res["launches_per_token"],
+                                              "gemv_kernel<128,4,fused>"),
+                        result=res)
+        else:
+            raise SystemExit("unknown --config %r" % which)
+    line["clocks"] = clk.summary()
+    torch.cuda.empty_cache()
+    return line
+
+
 # --------------------------------------------------------------------------- our arm
 
 def run_ours(args):
     import torch
     import torch.distributed as dist
-    from paper_2511_04477_b200 import binding, inputs
+    from paper_2511_04477_b200 import binding, inputs, sweep
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -209,6 +279,13 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
     binding.lib()
+
+    if args.config != "layer":
+        if rank == 0:
+            print(json.dumps(other_config_line(args.config, local, quick=args.quick)), flush=True)
+        if world > 1:
+            dist.destroy_process_group()
+        return
 
     linears = inputs.LLAMA3_8B_LINEARS
     sites = {"attn_in": ("laplace", 4096, ["q", "k", "v"]), "attn_out": ("laplace", 4096, ["o"]),
@@ -261,20 +338,6 @@ def run_ours(args):
         for s, nm in stacked.items():
             binding.spqt_sparsify_gemv(L[nm], xd[s][j], ts[s][j], ws[nm], idx[s], cnt[s], ys[nm], stream=stream)
 
-    def seven_launch_step(i):
-        """The seven matrices kept apart: per site one launch collects the indices and multiplies the
-        first matrix; the site's other matrices reuse the index list."""
-        L = layers[i % LAYER_COPIES]
-        j = i % X_POOL
-        for s in sites:
-            first = True
-            for nm in sites[s][2]:
-                if first:
-                    binding.spqt_sparsify_gemv(L[nm], xd[s][j], ts[s][j], ws[nm], idx[s], cnt[s], ys[nm], stream=stream)
-                    first = False
-                else:
-                    binding.spqt_sparse_gemv(L[nm], xd[s][j], idx[s], cnt[s], ws[nm], ys[nm], stream=stream)
-
     def step(i, with_sparsify=True, gemv=True, dense=False, names=None):
         L = layers[i % LAYER_COPIES]
         j = i % X_POOL if with_sparsify else 0   # kernel-only regions keep the index lists of pool entry 0
@@ -305,7 +368,7 @@ def run_ours(args):
             b += needed_bytes_gemv(shape[nm][0], shape[nm][1], c[s])
         return b
 
-    def gemv_bytes(i, dense=False):
+    def gemv_bytes(dense=False):
         c = counts[0]
         return sum(needed_bytes_gemv(shape[nm][0], shape[nm][1], shape[nm][1] if dense else c[site_of[nm]])
                    for nm in stacked.values())
@@ -319,10 +382,11 @@ def run_ours(args):
         """Steps captured per CUDA graph: the largest divisor of K not above 64 (so that exactly K run)."""
         return max(d for d in range(1, min(K, 64) + 1) if K % d == 0)
 
-    def timed(fn, K, W):
-        """W warm-up steps, then EXACTLY K steps between two events on the launching stream, launched as
-        replays of a captured CUDA graph (so that the device, not the Python launch path, is timed);
-        max over ranks (ms)."""
+    def timed(fn, K, W, min_s=0.0, max_regions=4000):
+        """W warm-up steps, then regions of EXACTLY K steps each between two events on the launching stream,
+        launched as replays of a captured CUDA graph (so that the device, not the Python launch path, is
+        timed), barrier + synchronize on both sides of every region; regions are repeated until min_s of
+        device time has been timed.  Returns the list of region times (ms, max over ranks)."""
         g = graph_len(K)
         with torch.cuda.stream(stream):
             for i in range(W):
@@ -336,61 +400,77 @@ def run_ours(args):
             graph.replay()          # one untimed replay: graph upload, instruction caches
         barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        with torch.cuda.stream(stream):
-            e0.record(stream)
-            for _ in range(K // g):
-                graph.replay()
-            e1.record(stream)
-        barrier()
-        return max_over_ranks(e0.elapsed_time(e1), dev)
+        regions, total = [], 0.0
+        while True:
+            with torch.cuda.stream(stream):
+                e0.record(stream)
+                for _ in range(K // g):
+                    graph.replay()
+                e1.record(stream)
+            barrier()
+            ms = max_over_ranks(e0.elapsed_time(e1), dev)
+            regions.append(ms)
+            total += ms * 1e-3
+            if total >= min_s or len(regions) >= max_regions:
+                break
+        return regions
 
     K, W = args.steps, max(args.warmup, 3)
+    med = lambda v: float(np.median(v))
 
     # ---- main timed region (whole hot path), with clocks sampled during it
     l0 = binding.spqt_launch_count()
     with ClockSampler(local) as clk:
-        ms = timed(hot_path_step, K, W)
+        regions = timed(hot_path_step, K, W, min_s=MIN_TIMED_S)
     launches = binding.spqt_launch_count() - l0
+    ms, ms_min = med(regions), float(np.min(regions))
     g_len = graph_len(K)
     launches_timed = 4 * K
-    ms_seven = timed(seven_launch_step, K, W)      # the seven matrices kept apart, 7 launches
-    ms_separate = timed(lambda i: step(i), K, W)   # and as 4 + 7 separate launches
-    total_bytes = (K // g_len) * sum(step_bytes(i) for i in range(W, W + g_len))
-    value = world * total_bytes / (ms * 1e-3) / 1e9
+    bytes_K = (K // g_len) * sum(step_bytes(i) for i in range(W, W + g_len))
+    value = world * bytes_K / (ms * 1e-3) / 1e9
+    peak, peak_kind = sweep.hbm_peak()
+    avg_launch_bytes = bytes_K / launches_timed
+    avg_launch_us = ms * 1e3 / launches_timed
+    achieved = avg_launch_bytes / avg_launch_us * 1e-3
 
-    # ---- kernel-only regions for the roofline and the dense comparison (index lists of pool entry 0)
+    # ---- kernel-only regions: index lists given (pool entry 0), the dense comparison, index collection alone
     with torch.cuda.stream(stream):
         for s in sites:
             binding.spqt_sparsify(xd[s][0], ts[s][0], idx[s], cnt[s], stream=stream)
-    ms_gemv = timed(lambda i: step(i, with_sparsify=False, names="stacked"), K, W)
-    ms_dense = timed(lambda i: step(i, with_sparsify=False, dense=True, names="stacked"), K, W)
-    ms_sparsify = timed(lambda i: step(i, gemv=False), K, W)
+    ms_gemv = med(timed(lambda i: step(i, with_sparsify=False, names="stacked"), K, W, min_s=0.05))
+    ms_dense = med(timed(lambda i: step(i, with_sparsify=False, dense=True, names="stacked"), K, W, min_s=0.05))
+    ms_sparsify = med(timed(lambda i: step(i, gemv=False), K, W, min_s=0.02))
+    ms_separate = med(timed(lambda i: step(i, names="stacked"), K, W, min_s=0.05))     # 4 index collections + 4 GEMVs
     with torch.cuda.stream(stream):
         for s in sites:
             binding.spqt_sparsify(xd[s][0], ts[s][0], idx[s], cnt[s], stream=stream)
-    gb = K * gemv_bytes(0)
-    gb_dense = K * gemv_bytes(0, dense=True)
-    n_gemv = 4 * K
-    achieved = gb / (ms_gemv * 1e-3) / 1e9
-    peak, peak_kind = measured_peak()
+    gb = K * gemv_bytes()
+    gb_dense = K * gemv_bytes(dense=True)
 
-    # per-shape device time, rotating the same layer copies (gemv only)
+    # ---- per shape, cold: enough distinct copies of every matrix that a copy has left L2 before its next visit
     per_shape = {}
     for nm in order + ["qkv", "gateup"]:
         s = site_of[nm]
-
-        reps = 8 * LAYER_COPIES
-        t_sp = timed(lambda i, nm=nm, s=s: binding.spqt_sparse_gemv(
-            layers[i % LAYER_COPIES][nm], xd[s][0], idx[s], cnt[s], ws[nm], ys[nm], stream=stream), reps, 3)
-        t_de = timed(lambda i, nm=nm, s=s: binding.spqt_dense_gemv(
-            layers[i % LAYER_COPIES][nm], xd[s][0], ws[nm], ys[nm], stream=stream), reps, 3)
         m, n = shape[nm]
+        ncopy = sweep.copies_for(m, n, BITS, GROUP)
+        packs = sweep.make_copies(m, n, BITS, GROUP, ncopy, seed0=500)
+        reps = max(ncopy, 32)
+        t_sp = med(timed(lambda i, nm=nm, s=s: binding.spqt_sparse_gemv(
+            packs[i % ncopy], xd[s][0], idx[s], cnt[s], ws[nm], ys[nm], stream=stream), reps, 3, min_s=0.02))
+        t_fu = med(timed(lambda i, nm=nm, s=s: binding.spqt_sparsify_gemv(
+            packs[i % ncopy], xd[s][0], ts[s][0], ws[nm], idx[s], cnt[s], ys[nm], stream=stream), reps, 3, min_s=0.02))
+        t_de = med(timed(lambda i, nm=nm, s=s: binding.spqt_dense_gemv(
+            packs[i % ncopy], xd[s][0], ws[nm], ys[nm], stream=stream), reps, 3, min_s=0.02))
         c0 = counts[0][s]
-        per_shape[nm] = {"m": m, "n": n, "count": c0,
-                         "sparse_us": t_sp * 1e3 / reps, "dense_us": t_de * 1e3 / reps,
+        per_shape[nm] = {"m": m, "n": n, "count": c0, "copies": ncopy, "cold": True,
+                         "sparse_us": t_sp * 1e3 / reps, "fused_us": t_fu * 1e3 / reps, "dense_us": t_de * 1e3 / reps,
                          "sparse_gbs": needed_bytes_gemv(m, n, c0) / (t_sp * 1e-3 / reps) / 1e9,
+                         "fused_gbs": (needed_bytes_gemv(m, n, c0) + needed_bytes_sparsify(n, c0)) / (t_fu * 1e-3 / reps) / 1e9,
                          "dense_gbs": needed_bytes_gemv(m, n, n) / (t_de * 1e-3 / reps) / 1e9,
-                         "speedup_vs_dense": t_de / t_sp}
+                         "speedup_vs_dense": t_de / t_sp, "fused_speedup_vs_dense": t_de / t_fu}
+        per_shape[nm]["fused_frac_of_peak"] = per_shape[nm]["fused_gbs"] / peak
+        del packs
+        torch.cuda.empty_cache()
 
     # ---- achievable read and gather rates of this GPU with the GEMV's copy instruction (rank 0 only)
     probes = None
@@ -440,47 +520,63 @@ def run_ours(args):
 
     status = max(binding.spqt_workspace_status(ws[nm], shape[nm][0], GROUP) for nm in shape)
 
+    # ---- short forms of the other workloads (rank 0), so that one run covers them
+    others = None
+    if rank == 0 and not args.no_extra:
+        del layers, hosts
+        torch.cuda.empty_cache()
+        others = {}
+        sw = other_config_line("sweep", local, quick=True)
+        others["sparsity_sweep_at_50pct"] = sw["speedup_vs_dense_at_50pct"]
+        fm = other_config_line("formats", local, quick=True)
+        others["formats_28672x8192_frac_of_peak"] = fm["frac_of_peak"]
+        st = other_config_line("stack", local, quick=True)
+        others["stack_32_layers"] = {k: st["result"][k] for k in ("tokens_per_s", "ms_per_token", "needed_gb_per_token", "needed_gbs",
+                                                                    "frac_of_peak", "tokens", "device_status")}
+
     if rank == 0:
         cpu = oracle_sample(3, 1) if world >= 1 else None
         cpu_all = cpu["cores"]
         cpu1 = oracle_sample(1, 0, threads=1)      # the same sample on one core
         import oracle as _oracle
         _oracle.set_threads(cpu_all)
-        avg_launch_bytes = gb / n_gemv
-        traffic = NCU_TRAFFIC_RATIO * avg_launch_bytes
+        clocks = clk.summary()
         line = {
             "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": K, "warmup": W,
-            "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": ms / K, "ms_per_step_min": ms_min / K, "regions_timed": len(regions),
+            "device_seconds_timed": float(np.sum(regions)) * 1e-3,
+            "us_x_mhz_per_step": (ms / K * 1e3) * clocks["sm_mhz"] if clocks["sm_mhz"] else None,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "int4 codes, f32 accumulate, f16 in/out", "data": "synthetic",
             "config": {"workload": "llama3-8b decode-layer linears q,k,v,o,gate,up,down; int4 g128 zigzag; batch 1; "
                                    "50%% sparsity; q|k|v and gate|up packed as one matrix each (they share x and idx); per step "
                                    "4 launches, each collecting its indices and multiplying, one stream, "
                                    "replayed from a CUDA graph of %d steps" % g_len,
-                       "l2_defeat": "%d distinct layer copies rotated, %.2f GB of packed weights (> 126 MB L2)" % (
-                           LAYER_COPIES, weight_bytes / 1e9),
+                       "l2_defeat": "%d distinct layer copies rotated, %.2f GB of packed weights (> 126 MB L2); per-shape numbers use "
+                                    "enough copies of each matrix that the bytes between two visits exceed twice the L2" % (
+                                        LAYER_COPIES, weight_bytes / 1e9),
                        "parallelism": "replicas only" if world > 1 else "single GPU"},
-            "us_per_gemv": ms_gemv * 1e3 / n_gemv,
-            "us_per_step": {"hot_path": ms * 1e3 / K, "gemv_only": ms_gemv * 1e3 / K,
+            "us_per_launch": avg_launch_us,
+            "us_per_step": {"hot_path": ms * 1e3 / K, "gemv_only_given_lists": ms_gemv * 1e3 / K,
                             "dense_gemv_only": ms_dense * 1e3 / K, "sparsify_only": ms_sparsify * 1e3 / K,
-                            "seven_matrices_7_launches": ms_seven * 1e3 / K,
-                            "seven_matrices_4_sparsify_7_gemv_launches": ms_separate * 1e3 / K},
-            "speedup_vs_dense_same_layout": ms_dense / ms_gemv,
+                            "four_sparsify_plus_four_gemv_launches": ms_separate * 1e3 / K},
+            "speedup_vs_dense_same_layout": ms_dense / ms,
+            "speedup_vs_dense_same_layout_given_lists": ms_dense / ms_gemv,
             "dense_gbs": gb_dense / (ms_dense * 1e-3) / 1e9,
+            "gemv_only_gbs": gb / (ms_gemv * 1e-3) / 1e9,
             "pct_of_peak": {"of_measured_%.0f" % peak: 100 * achieved / peak, "of_nominal_8000": 100 * achieved / 8000,
                             "of_probed_gather": 100 * achieved / probes["gather_64B_half_of_lines_gbs"]},
             "probed_rooflines": probes,
             "per_shape": per_shape,
-            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": traffic, "peak_kind": "of " + peak_kind,
-                         "kernel": "gemv_kernel<128,sparse>", "algorithmic_bytes_per_launch": avg_launch_bytes,
-                         "avg_launch_us": ms_gemv * 1e3 / n_gemv},
+            "roofline": roofline_obj(achieved, peak, peak_kind, avg_launch_bytes, avg_launch_us, "gemv_kernel<128,4,fused>"),
             "cpu_baseline": {"value": cpu["value"], "unit": "GB/s", "cores": cpu["cores"], "kind": "oracle",
                              "sample": cpu["sample"], "single_thread_value": cpu1["value"]},
             "e2e": {"value": world * e2e_bytes / e2e_s / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s / e2e_K * 1e3},
-            "gpu_launches": launches_timed, "launches_counted_incl_warmup_and_capture": launches,
-            "clocks": clk.summary(),
+            "gpu_launches": launches_timed, "launches_counted_incl_warmup_capture_and_repeats": launches,
+            "clocks": clocks,
             "device_status": status,
+            "other_configs": others,
             "paper_context": "paper reports up to 1.55x end-to-end decode speedup and up to 1.78x sparse-GEMV "
                              "speedup at 50% sparsity on Apple GPUs (Q4_K); other hardware, context only",
         }
@@ -495,6 +591,9 @@ def main():
     ap.add_argument("--steps", type=int, default=1024)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="layer", choices=["layer", "sweep", "formats", "dense", "stack"])
+    ap.add_argument("--quick", action="store_true", help="reduced form of --config sweep/formats/stack")
+    ap.add_argument("--no-extra", action="store_true", help="headline line without the summaries of the other workloads")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

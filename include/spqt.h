@@ -221,6 +221,26 @@ spqt_status spqt_sparse_linear_host(const void* codes, const void* scale_zero,
 spqt_status spqt_set_tuning(int gemv_ctas, int no_overlap);
 
 /*
+ * Per-shape profiling (paper Sec. 3.2: GEMV shapes are profiled per platform to pick the kernel's
+ * hyper-parameters; Sec. 6, hyper-parameter study).  Times the call that collects the indices and
+ * multiplies (spqt_sparsify_gemv with threshold t on x) and the dense call on this problem for a set
+ * of grid sizes -- one CTA per SM, and every whole number 1..8 of CTAs per block-row that fits the
+ * device -- and remembers the fastest of each for this (m, n, bits, group): later calls of
+ * spqt_sparsify_gemv / spqt_sparse_gemv and of spqt_dense_gemv with the same shape use them
+ * (spqt_set_tuning with a non-zero grid size still overrides).  Results of those calls do not change
+ * beyond the order of partial sums.  Arguments are those of spqt_sparsify_gemv; idx, count and y are
+ * overwritten.  If `flush` is not NULL its flush_bytes bytes are rewritten before every timed launch, so
+ * that a buffer larger than L2 makes the weights come from HBM as in steady-state decoding.
+ * ctas_sparse / ctas_dense (host, may be NULL) receive the choices.  Synchronises the stream many
+ * times; call it once per shape at start-up, outside any stream capture.  The table holds 256 shapes,
+ * is process-wide and not thread-safe.
+ */
+spqt_status spqt_autotune(const void* codes, const void* scale_zero, int m, int n, int bits, int group,
+                          const void* x, float t, int32_t* idx, int32_t* count, void* y,
+                          void* workspace, size_t workspace_bytes, void* flush, size_t flush_bytes,
+                          int* ctas_sparse, int* ctas_dense, void* stream);
+
+/*
  * Checked mode (off by default; paper Sec. 4.2.3 assumes a well-formed index list and so does the
  * normal path).  With on != 0, spqt_sparse_gemv and spqt_sparse_gemv_static first check the list on
  * the device: *count in [0, n], every index in [0, n), and, for n <= 1048576, no index twice.  A bad

@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libspqt.so")
 EXPORTS = (
     "spqt_status_string", "spqt_version", "spqt_packed_sizes", "spqt_pack", "spqt_unpack",
     "spqt_sparsify", "spqt_sparse_gemv", "spqt_sparse_gemv_static", "spqt_static_status", "spqt_sparsify_gemv", "spqt_dense_gemv",
-    "spqt_sparse_linear_host", "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_launch_count",
+    "spqt_sparse_linear_host", "spqt_autotune", "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_launch_count",
 )
 
 _lib = None
@@ -59,6 +59,9 @@ def lib() -> ctypes.CDLL:
         L.spqt_dense_gemv.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, sz, vp]
         L.spqt_sparse_linear_host.argtypes = [vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, vp,
                                               vp, vp, vp, vp, vp, sz, vp]
+        L.spqt_autotune.argtypes = [vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, vp, vp, vp, vp, sz, vp, sz,
+                                    ctypes.POINTER(i32), ctypes.POINTER(i32), vp]
+        L.spqt_autotune.restype = i32
         L.spqt_set_tuning.argtypes = [i32, i32]
         L.spqt_set_debug.argtypes = [i32]
         L.spqt_probe_read.argtypes = [vp, sz, i32, vp, vp]
@@ -277,6 +280,22 @@ def spqt_probe_read(buf: torch.Tensor, pattern: int, moved: torch.Tensor, stream
 def spqt_set_debug(on: bool) -> None:
     """Checked mode: validate idx/count on the device before every sparse GEMV (off by default)."""
     _ok(lib().spqt_set_debug(1 if on else 0), "spqt_set_debug")
+
+
+def spqt_autotune(p: Packed, x: torch.Tensor, t: float, workspace: torch.Tensor, flush: torch.Tensor = None, stream=None):
+    """Profile grid sizes for this shape and keep the fastest -> (ctas for the sparse calls, ctas for the dense call).
+    ``flush``: an optional uint8 buffer larger than L2, rewritten before every timed launch.  Synchronises."""
+    idx = torch.empty(p.n, dtype=torch.int32, device=x.device)
+    count = torch.empty(1, dtype=torch.int32, device=x.device)
+    y = torch.empty(p.m, dtype=torch.float16, device=x.device)
+    a, b = ctypes.c_int(0), ctypes.c_int(0)
+    _ok(lib().spqt_autotune(
+        _dev(p.codes, torch.uint8, "codes"), _dev(p.scale_zero, torch.float16, "scale_zero"), p.m, p.n, p.bits, p.group,
+        _dev(x, torch.float16, "x"), float(t), idx.data_ptr(), count.data_ptr(), y.data_ptr(),
+        _dev(workspace, torch.uint8, "workspace"), workspace.numel(),
+        flush.data_ptr() if flush is not None else None, flush.numel() if flush is not None else 0,
+        ctypes.byref(a), ctypes.byref(b), _stream(stream)), "spqt_autotune")
+    return int(a.value), int(b.value)
 
 
 def spqt_set_tuning(gemv_ctas: int = 0, no_overlap: int = 0) -> None:

@@ -1002,6 +1002,36 @@ struct FusedArgs {
     int32_t* count_out;
 };
 
+// Grid sizes found by spqt_autotune, per (shape, format, kind of call).  Process-wide, small, searched
+// linearly; not thread-safe (like spqt_set_tuning).
+struct TunedEntry {
+    int m, n, bits, group, mode, ctas;
+};
+constexpr int kMaxTuned = 256;
+static TunedEntry g_tuned[kMaxTuned];
+static int g_tuned_count = 0;
+
+static int tuned_ctas(const Format& f, int mode)
+{
+    for (int i = 0; i < g_tuned_count; ++i) {
+        const TunedEntry& e = g_tuned[i];
+        if (e.m == f.m && e.n == f.n && e.bits == f.bits && e.group == f.group && e.mode == mode) return e.ctas;
+    }
+    return 0;
+}
+
+static void store_tuned(const Format& f, int mode, int ctas)
+{
+    for (int i = 0; i < g_tuned_count; ++i) {
+        TunedEntry& e = g_tuned[i];
+        if (e.m == f.m && e.n == f.n && e.bits == f.bits && e.group == f.group && e.mode == mode) {
+            e.ctas = ctas;
+            return;
+        }
+    }
+    if (g_tuned_count < kMaxTuned) g_tuned[g_tuned_count++] = TunedEntry{f.m, f.n, f.bits, f.group, mode, ctas};
+}
+
 // Bytes of the stage area the prologue may borrow, and what it needs for an x of n entries.
 template <int G, int BITS>
 constexpr size_t stage_area_bytes() { return sizeof(GemvSmem<G, BITS>::stage); }
@@ -1029,10 +1059,20 @@ static spqt_status launch_gemv(const Format& f, const void* codes, const void* m
     }
     const int sms = sm_count();
     if (sms <= 0) return SPQT_ERR_CUDA;
-    int P = g_tune_ctas > 0 ? g_tune_ctas : sms;
-    // With few block-rows, a whole number of CTAs per block-row (if that keeps >= 85 % of the SMs
-    // busy) gives every CTA a single segment: no CTA then carries two aggregation chains.
-    if (g_tune_ctas == 0 && f.R <= P && (P / f.R) * f.R * 100 >= 85 * P) P = (P / f.R) * f.R;
+    const int tuned = g_tune_ctas > 0 ? g_tune_ctas : tuned_ctas(f, MODE);
+    int P = tuned > 0 ? tuned : sms;
+    if (tuned == 0 && f.R <= P) {
+        // With few block-rows, a whole number of CTAs per block-row (if that keeps >= 85 % of the SMs
+        // busy) gives every CTA a single segment: no CTA then carries two aggregation chains.
+        int k = P / f.R;
+        // A small matrix gains nothing from more than four CTAs per block-row: the combination of many
+        // partial sums then costs more than the extra CTAs save (measured: 1024 x 4096 takes 6.8 us on 144
+        // CTAs, 4.9 us on 32).  "Small": under 256 KB of blocks per CTA at four CTAs per block-row.
+        const size_t row_bytes = (size_t)f.n * (size_t)(f.B + 4);
+        const bool small = k > 4 && row_bytes / 4 < (size_t(256) << 10);
+        if (small) k = 4;
+        if (small || k * f.R * 100 >= 85 * P) P = k * f.R;
+    }
     // no more CTAs than pieces of at least 64 columns of one block-row
     const long long pieces = (long long)f.R * ((f.n + 63) / 64);
     if (P > pieces) P = (int)pieces;
@@ -1271,6 +1311,66 @@ spqt_status spqt_static_status(int m, int group, int* status_host, void* stream)
     void* const scratch = static_scratch_address();
     if (scratch == nullptr) return SPQT_ERR_CUDA;
     return read_status_word(static_cast<const int*>(scratch) + m / group, status_host, static_cast<cudaStream_t>(stream));
+}
+
+spqt_status spqt_autotune(const void* codes, const void* scale_zero, int m, int n, int bits, int group,
+                          const void* x, float t, int32_t* idx, int32_t* count, void* y,
+                          void* workspace, size_t workspace_bytes, void* flush, size_t flush_bytes,
+                          int* ctas_sparse, int* ctas_dense, void* stream)
+{
+    using namespace spqt;
+    Format f;
+    spqt_status st = check_gemv_args(codes, scale_zero, m, n, bits, group, x, idx, count, false, y, workspace,
+                                     workspace_bytes, &f);
+    if (st != SPQT_OK) return st;
+    if (n > kMaxListN) return SPQT_ERR_UNSUPPORTED;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const int sms = sm_count();
+    if (sms <= 0) return SPQT_ERR_CUDA;
+    // candidates: one CTA per SM, and every whole number (1..8) of CTAs per block-row that fits
+    int cand[10], ncand = 0;
+    cand[ncand++] = sms;
+    for (int k = 1; k <= kMaxCluster; ++k)
+        if ((long long)k * f.R <= sms && k * f.R != sms) cand[ncand++] = k * f.R;
+    cudaEvent_t e0, e1;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return SPQT_ERR_CUDA;
+    const int saved = g_tune_ctas;
+    const bool fused_ok = fused_fits_format(f);
+    int best[2] = {0, 0};
+    st = SPQT_OK;
+    for (int kind = 0; kind < 2 && st == SPQT_OK; ++kind) {   // 0: index collection + sparse product, 1: dense product
+        float best_ms = 0.0f;
+        for (int ci = 0; ci < ncand && st == SPQT_OK; ++ci) {
+            g_tune_ctas = cand[ci];
+            float ms_min = 0.0f;
+            for (int rep = 0; rep < 6 && st == SPQT_OK; ++rep) {   // the first repetition warms up
+                if (flush && flush_bytes && cudaMemsetAsync(flush, rep, flush_bytes, s) != cudaSuccess) st = SPQT_ERR_CUDA;
+                if (cudaEventRecord(e0, s) != cudaSuccess) st = SPQT_ERR_CUDA;
+                if (st == SPQT_OK) {
+                    if (kind == 0) st = spqt_sparsify_gemv(codes, scale_zero, m, n, bits, group, x, t, idx, count, y, workspace, workspace_bytes, stream);
+                    else st = spqt_dense_gemv(codes, scale_zero, m, n, bits, group, x, y, workspace, workspace_bytes, stream);
+                }
+                if (cudaEventRecord(e1, s) != cudaSuccess || cudaEventSynchronize(e1) != cudaSuccess) st = SPQT_ERR_CUDA;
+                float ms = 0.0f;
+                if (st == SPQT_OK && cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) st = SPQT_ERR_CUDA;
+                if (rep > 0 && (ms_min == 0.0f || ms < ms_min)) ms_min = ms;
+            }
+            if (st == SPQT_OK && (best[kind] == 0 || ms_min < best_ms)) {
+                best[kind] = cand[ci];
+                best_ms = ms_min;
+            }
+        }
+    }
+    g_tune_ctas = saved;
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (st != SPQT_OK) return st;
+    store_tuned(f, fused_ok ? kModeFused : kModeList, best[0]);
+    if (fused_ok) store_tuned(f, kModeList, best[0]);
+    store_tuned(f, (n & 7) == 0 && aligned(x, 16) ? kModeDense : kModeList, best[1]);
+    if (ctas_sparse) *ctas_sparse = best[0];
+    if (ctas_dense) *ctas_dense = best[1];
+    return SPQT_OK;
 }
 
 spqt_status spqt_set_debug(int on)

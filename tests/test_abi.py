@@ -88,6 +88,8 @@ def test_bad_arguments_launch_nothing(L):
     # workspace too small
     assert L.spqt_sparse_gemv(a16, a16, 128, 8, 4, 128, a16, a16, a16, a16, a16, ws - 1, None) == 4
     assert L.spqt_dense_gemv(a16, a16, 128, 8, 4, 128, a16, a16, a16, 16, None) == 4
+    assert L.spqt_autotune(a16, a16, 128, 8, 4, 128, None, 0.5, a16, a16, a16, a16, ws, None, 0, None, None, None) == 1
+    assert L.spqt_autotune(a16, a16, 128, 8, 4, 128, a16, 0.5, a16, a16, a16, a16, ws - 1, None, 0, None, None, None) == 4
     assert L.spqt_set_tuning(-1, 0) == 1
     assert L.spqt_set_tuning(0, 8) == 1
     assert L.spqt_workspace_status(None, 128, 128, None, None) == 1

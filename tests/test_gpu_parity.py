@@ -717,3 +717,36 @@ def test_static_column_partition_ablation_matches_the_oracle(bits, group, m_bloc
         assert np.array_equal(got[:ref_cnt], ref_idx) and np.all(got[ref_cnt:] == -7)
         check_y(y.cpu().numpy(), y_ref, bound, "static partition, sparsity %.1f" % sp)
     assert binding.spqt_workspace_status(ws, m, group) == 0
+
+
+# ------------------------------------------------------------------ per-shape profiling
+
+def test_autotune_picks_a_grid_and_results_stay_right():
+    """spqt_autotune times the candidate grids for a shape and later calls use its choice; the results
+    still match the oracle, and a small matrix is not spread over every SM."""
+    m, n, bits, group = 1024, 4096, 4, 128
+    W = inputs.weights(m, n, seed=301)
+    x = inputs.activations(n, seed=302)
+    p = pack_on_gpu(W, bits, group)
+    codes, s, z = packed_to_host(p)
+    ws = binding.new_workspace(m, n, bits, group)
+    t = inputs.threshold_for_sparsity(x, 0.5)
+    flush = torch.empty(192 << 20, dtype=torch.uint8, device="cuda")
+    before = binding.spqt_launch_count()
+    ctas_sparse, ctas_dense = binding.spqt_autotune(p, dev(x), t, ws, flush)
+    assert binding.spqt_launch_count() > before + 20          # it really timed launches
+    R = m // group
+    valid = {148} | {k * R for k in range(1, 9)}
+    assert ctas_sparse in valid and ctas_dense in valid
+    y, idx, cnt = run_sparse(p, x, t, ws)
+    ref_idx, ref_cnt = oracle.sparsify(x, t)
+    assert cnt == ref_cnt and np.array_equal(idx, ref_idx)
+    y_ref, bound = oracle.sparse_gemv(codes, s, z, m, n, x, ref_idx, bits, group)
+    check_y(y, y_ref, bound, "after autotune, sparse")
+    yf, _, _ = binding.spqt_sparsify_gemv(p, dev(x), t, ws)
+    yd = binding.spqt_dense_gemv(p, dev(x), ws)
+    torch.cuda.synchronize()
+    check_y(yf.cpu().numpy(), y_ref, bound, "after autotune, fused")
+    yd_ref, dbound = oracle.dense_gemv(codes, s, z, m, n, x, bits, group)
+    check_y(yd.cpu().numpy(), yd_ref, dbound, "after autotune, dense")
+    assert binding.spqt_workspace_status(ws, m, group) == 0
