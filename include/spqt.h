@@ -221,6 +221,23 @@ spqt_status spqt_sparse_linear_host(const void* codes, const void* scale_zero,
 spqt_status spqt_set_tuning(int gemv_ctas, int no_overlap);
 
 /*
+ * Threshold calibration (paper Sec. 5, the calibration threshold tool; Sec. 3.2: thresholds are
+ * computed once per sparsity level from calibration activations).  *threshold (a device float) =
+ * the nearest-rank order statistic of |x| over the pool x[0:count] of fp16 calibration activations:
+ * the ceil(sparsity * N)-th smallest magnitude (1-based; N = the entries that are not NaN), so that at
+ * least that fraction of the pool is inactive under "active <=> |x| > threshold".  sparsity <= 0, or an
+ * empty pool, gives -1 (nothing dropped).  Exact: a histogram over the 2^15 fp16 magnitudes.
+ *   x : fp16[count], 2-byte aligned; the activations of one site (or of all the matrices that share an
+ *       input), over as many calibration tokens as wanted, concatenated.
+ *   workspace : 131072 bytes, 4-byte aligned, zeroed ONCE by the caller; every call leaves it zeroed.
+ * The two modes of the paper's tool sit on top of this call in paper_2511_04477_b200/calibrate.py:
+ * one global sparsity for every site, or per-matrix sparsities averaged over the matrices that share an
+ * input ({q,k,v}, {gate,up}) so that they share one threshold and one index collection.
+ */
+spqt_status spqt_calibrate_threshold(const void* x, size_t count, double sparsity, float* threshold,
+                                     void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Per-shape profiling (paper Sec. 3.2: GEMV shapes are profiled per platform to pick the kernel's
  * hyper-parameters; Sec. 6, hyper-parameter study).  Times the call that collects the indices and
  * multiplies (spqt_sparsify_gemv with threshold t on x) and the dense call on this problem for a set

@@ -13,6 +13,8 @@ import os
 import subprocess
 import threading
 
+import math
+
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -177,3 +179,21 @@ def threads() -> int:
 
 def set_threads(t: int) -> None:
     _load().spqt_oracle_set_threads(int(t))
+
+
+def calibrate_threshold(pool, sparsity: float) -> float:
+    """Nearest-rank threshold of |x| over a pool of fp16 calibration activations (calibration threshold tool,
+    Sec. 5): the ceil(sparsity * N)-th smallest magnitude, N = the entries that are not NaN; -1 when nothing
+    is to be dropped.  Written out with a full sort."""
+    a = np.abs(np.asarray(pool, dtype=np.float16).ravel().astype(np.float64))
+    a = np.sort(a[~np.isnan(a)])
+    if a.size == 0 or not (sparsity > 0.0):
+        return -1.0
+    rank = int(min(a.size, max(1, math.ceil(sparsity * a.size - 1e-9))))
+    return float(a[rank - 1])
+
+
+def group_sparsity(levels) -> float:
+    """Sparsity shared by the matrices that read one input: the mean of their levels (customized mode, Sec. 5)."""
+    levels = [float(v) for v in levels]
+    return sum(levels) / len(levels)

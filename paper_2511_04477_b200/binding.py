@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libspqt.so")
 EXPORTS = (
     "spqt_status_string", "spqt_version", "spqt_packed_sizes", "spqt_pack", "spqt_unpack",
     "spqt_sparsify", "spqt_sparse_gemv", "spqt_sparse_gemv_static", "spqt_static_status", "spqt_sparsify_gemv", "spqt_dense_gemv",
-    "spqt_sparse_linear_host", "spqt_autotune", "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_launch_count",
+    "spqt_sparse_linear_host", "spqt_autotune", "spqt_calibrate_threshold", "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_launch_count",
 )
 
 _lib = None
@@ -62,6 +62,8 @@ def lib() -> ctypes.CDLL:
         L.spqt_autotune.argtypes = [vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, vp, vp, vp, vp, sz, vp, sz,
                                     ctypes.POINTER(i32), ctypes.POINTER(i32), vp]
         L.spqt_autotune.restype = i32
+        L.spqt_calibrate_threshold.argtypes = [vp, sz, ctypes.c_double, vp, vp, sz, vp]
+        L.spqt_calibrate_threshold.restype = i32
         L.spqt_set_tuning.argtypes = [i32, i32]
         L.spqt_set_debug.argtypes = [i32]
         L.spqt_probe_read.argtypes = [vp, sz, i32, vp, vp]
@@ -296,6 +298,25 @@ def spqt_autotune(p: Packed, x: torch.Tensor, t: float, workspace: torch.Tensor,
         flush.data_ptr() if flush is not None else None, flush.numel() if flush is not None else 0,
         ctypes.byref(a), ctypes.byref(b), _stream(stream)), "spqt_autotune")
     return int(a.value), int(b.value)
+
+
+def new_calibration_workspace(device=None) -> torch.Tensor:
+    """Zeroed histogram workspace of spqt_calibrate_threshold (zeroed once; every call leaves it zeroed)."""
+    return torch.zeros(32768, dtype=torch.int32, device=device or "cuda")
+
+
+def spqt_calibrate_threshold(x: torch.Tensor, sparsity: float, workspace: torch.Tensor = None,
+                             threshold: torch.Tensor = None, stream=None) -> torch.Tensor:
+    """Nearest-rank threshold of |x| over a pool of fp16 calibration activations -> float32[1] on the device."""
+    if workspace is None:
+        workspace = new_calibration_workspace(x.device)
+    if threshold is None:
+        threshold = torch.empty(1, dtype=torch.float32, device=x.device)
+    _ok(lib().spqt_calibrate_threshold(
+        _dev(x, torch.float16, "x") if x.numel() else None, x.numel(), float(sparsity),
+        _dev(threshold, torch.float32, "threshold"), _dev(workspace, torch.int32, "workspace"), workspace.numel() * 4,
+        _stream(stream)), "spqt_calibrate_threshold")
+    return threshold
 
 
 def spqt_set_tuning(gemv_ctas: int = 0, no_overlap: int = 0) -> None:

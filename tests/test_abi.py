@@ -90,6 +90,9 @@ def test_bad_arguments_launch_nothing(L):
     assert L.spqt_dense_gemv(a16, a16, 128, 8, 4, 128, a16, a16, a16, 16, None) == 4
     assert L.spqt_autotune(a16, a16, 128, 8, 4, 128, None, 0.5, a16, a16, a16, a16, ws, None, 0, None, None, None) == 1
     assert L.spqt_autotune(a16, a16, 128, 8, 4, 128, a16, 0.5, a16, a16, a16, a16, ws - 1, None, 0, None, None, None) == 4
+    assert L.spqt_calibrate_threshold(None, 8, 0.5, a16, a16, 131072, None) == 1
+    assert L.spqt_calibrate_threshold(a16, 8, 1.5, a16, a16, 131072, None) == 1
+    assert L.spqt_calibrate_threshold(a16, 8, 0.5, a16, a16, 131071, None) == 4
     assert L.spqt_set_tuning(-1, 0) == 1
     assert L.spqt_set_tuning(0, 8) == 1
     assert L.spqt_workspace_status(None, 128, 128, None, None) == 1

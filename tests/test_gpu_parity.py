@@ -750,3 +750,32 @@ def test_autotune_picks_a_grid_and_results_stay_right():
     yd_ref, dbound = oracle.dense_gemv(codes, s, z, m, n, x, bits, group)
     check_y(yd.cpu().numpy(), yd_ref, dbound, "after autotune, dense")
     assert binding.spqt_workspace_status(ws, m, group) == 0
+
+
+# ------------------------------------------------------------------ threshold calibration
+
+def test_calibration_threshold_is_the_exact_order_statistic():
+    from paper_2511_04477_b200 import calibrate
+    g = np.random.Generator(np.random.PCG64(9))
+    pools = {"laplace": g.laplace(0.0, 1.0, size=64 * 4096).astype(np.float16),
+             "gauss": g.standard_normal(32 * 14336).astype(np.float16),
+             "ties": (g.integers(0, 5, size=1000) * 0.25).astype(np.float16),
+             "one": np.array([-3.0], np.float16)}
+    pools["laplace"][:7] = [np.nan, np.inf, -np.inf, 0.0, -0.0, 65504.0, 6e-8]
+    ws = binding.new_calibration_workspace()
+    for name, pool in pools.items():
+        for sp in (0.0, 1e-6, 0.25, 0.4, 0.5, 0.9, 1.0):
+            t = float(binding.spqt_calibrate_threshold(dev(pool), sp, ws).item())
+            assert t == oracle.calibrate_threshold(pool, sp), (name, sp)
+        assert not ws.any()                                       # the histogram is left zeroed
+    assert float(binding.spqt_calibrate_threshold(torch.empty(0, dtype=torch.float16, device="cuda"), 0.5, ws).item()) == -1.0
+    # the two modes of the tool: one global level; per-matrix levels averaged over the matrices that share an input
+    sites = {"attn_in": dev(pools["laplace"]), "attn_out": dev(pools["laplace"][::2].copy()),
+             "mlp_in": dev(pools["laplace"][1::2].copy()), "mlp_mid": dev(pools["gauss"])}
+    host = {k: v.cpu().numpy() for k, v in sites.items()}
+    uni = calibrate.unified(sites, 0.4)
+    assert uni == {k: oracle.calibrate_threshold(host[k], 0.4) for k in sites}
+    levels = {"q": 0.3, "k": 0.5, "v": 0.4, "o": 0.25, "gate": 0.6, "up": 0.5, "down": 0.45}
+    grp = calibrate.grouped(sites, levels)
+    for site, names in calibrate.LLAMA_GROUPS.items():
+        assert grp[site] == oracle.calibrate_threshold(host[site], oracle.group_sparsity([levels[nm] for nm in names]))

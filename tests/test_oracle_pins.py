@@ -368,3 +368,34 @@ def test_outlier_recipe():
     changed = np.nonzero(x0 != x1)[0]
     assert 70 <= changed.size <= 82
     assert np.allclose(x1[changed].astype(np.float32), 20 * x0[changed].astype(np.float32), rtol=2e-3)
+
+
+# ------------------------------------------------------------------ threshold calibration
+
+def test_calibration_threshold_hand_example_and_rank_property():
+    pool = np.array([0.5, -2.0, 1.0, 0.25, np.nan, -0.25], np.float16)     # N = 5 entries that are not NaN
+    assert oracle.calibrate_threshold(pool, 0.5) == 0.5                      # rank ceil(2.5) = 3 of .25 .25 .5 1 2
+    assert oracle.calibrate_threshold(pool, 0.4) == 0.25                     # rank 2
+    assert oracle.calibrate_threshold(pool, 1.0) == 2.0
+    assert oracle.calibrate_threshold(pool, 0.0) == -1.0
+    assert oracle.calibrate_threshold(np.zeros(0, np.float16), 0.5) == -1.0
+    g = np.random.Generator(np.random.PCG64(5))
+    x = g.standard_normal(5000).astype(np.float16)
+    a = np.abs(x.astype(np.float64))
+    for s in (0.1, 0.25, 0.5, 0.9, 0.999):
+        t = oracle.calibrate_threshold(x, s)
+        rank = math.ceil(s * x.size - 1e-9)
+        assert np.count_nonzero(a <= t) >= rank > np.count_nonzero(a < t)   # t is the rank-th smallest magnitude
+        idx, cnt = oracle.sparsify(x, t)
+        assert x.size - cnt >= rank                                          # at least that many entries are dropped
+
+
+def test_calibration_threshold_matches_closed_forms_and_group_mean():
+    g = np.random.Generator(np.random.PCG64(6))
+    lap = g.laplace(0.0, 1.0, size=400_000).astype(np.float16)
+    assert abs(oracle.calibrate_threshold(lap, 0.5) - math.log(2.0)) < 0.01
+    assert abs(oracle.calibrate_threshold(lap, 0.25) - 0.2877) < 0.01
+    gau = g.standard_normal(400_000).astype(np.float16)
+    assert abs(oracle.calibrate_threshold(gau, 0.5) - 0.6745) < 0.01
+    assert oracle.group_sparsity([0.3, 0.5, 0.4]) == pytest.approx(0.4, abs=1e-15)
+    assert oracle.group_sparsity([0.5]) == 0.5
