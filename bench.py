@@ -421,7 +421,7 @@ def run_ours(args):
     # ---- main timed region (whole hot path), with clocks sampled during it
     l0 = binding.spqt_launch_count()
     with ClockSampler(local) as clk:
-        regions = timed(hot_path_step, K, W, min_s=MIN_TIMED_S)
+        regions = timed(hot_path_step, K, W, min_s=args.min_seconds)
     launches = binding.spqt_launch_count() - l0
     ms, ms_min = med(regions), float(np.min(regions))
     g_len = graph_len(K)
@@ -592,6 +592,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="layer", choices=["layer", "sweep", "formats", "dense", "stack"])
+    ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_S,
+                    help="device time to accumulate over repeated K-step regions of the headline measurement")
     ap.add_argument("--quick", action="store_true", help="reduced form of --config sweep/formats/stack")
     ap.add_argument("--no-extra", action="store_true", help="headline line without the summaries of the other workloads")
     args = ap.parse_args()

@@ -359,8 +359,33 @@ gemv_kernel(const GemvArgs a)
         pc.set_count(n, 8);
     } else {
         if (!FUSED) count = (a.flags & kFlagIdentity) ? n : __ldg(a.count);  // in flight while x is staged
+        // A given list that fits the window whole is copied whole, whatever the count turns out to be
+        // (idx holds n entries): its first entries are then loaded beside x and the count, in the same
+        // round trip, instead of after them.  Entries past the count are never used.
+        constexpr int kEarly = 8;
+        const bool whole_list = !FUSED && !(a.flags & kFlagIdentity) && has_xs && n <= kCap;
+        int early[kEarly];
+        if (whole_list) {
+#pragma unroll
+            for (int j = 0; j < kEarly; ++j) {
+                const int i = tid + j * kGemvThreads;
+                early[j] = i < n ? __ldg(a.idx + i) : 0;
+            }
+        }
         if (has_xs) stage_x(warp, kWarps);
         __syncthreads();
+        if (whole_list) {
+#pragma unroll
+            for (int j = 0; j < kEarly; ++j) {
+                const int i = tid + j * kGemvThreads;
+                const unsigned col = min((unsigned)early[j], (unsigned)(n - 1));   // past the count: anything, but in range
+                if (i < n) sm.ent[i] = (lds_u16(xs_addr + 2u * col) << 16) | col;
+            }
+            for (int i = tid + kEarly * kGemvThreads; i < n; i += kGemvThreads) {
+                const unsigned col = min((unsigned)__ldg(a.idx + i), (unsigned)(n - 1));
+                sm.ent[i] = (lds_u16(xs_addr + 2u * col) << 16) | col;
+            }
+        }
         if (FUSED) {
             const int4 t4 = *reinterpret_cast<const int4*>(&sm.tot[lane * 4]);
             count = (int)__reduce_add_sync(0xffffffffu, (unsigned)(t4.x + t4.y + t4.z + t4.w));
@@ -421,7 +446,10 @@ gemv_kernel(const GemvArgs a)
         }
         int olo = 0, ohi = 0;  // the part of the returned index list this CTA writes: its slice of block-row 0
         if (FUSED && pc.r_first == 0) pc.slice(0, &olo, &ohi);
-        if (resident) {
+        if (whole_list) {
+            win_lo = 0;          // the whole list is in place already
+            resident = true;
+        } else if (resident) {
             win_lo = need_lo;
             build_window(need_lo, need_hi, olo, ohi, warp, kWarps);
         } else {
@@ -684,10 +712,18 @@ gemv_kernel(const GemvArgs a)
     // block-row constants of the issue side, refreshed when it enters a new block-row
     const uint8_t* b_codes = nullptr;   // codes of the block-row (list calls: this lane's 16-byte part)
     const unsigned* b_meta = nullptr;   // (scale, zero) pairs of the block-row
-    auto enter_row = [&](int r) {
+    const uint8_t* d_codes = nullptr;   // dense call: where the issue side's next chunk starts in the three arrays
+    const unsigned* d_meta = nullptr;
+    const __half* d_x = nullptr;
+    auto enter_row = [&](int r, int pos) {
         const size_t row_base = (size_t)r * (size_t)n;
         b_codes = a.codes + row_base * B + ((!DENSE && BITS == 4) ? 16 * h : 0);
         b_meta = a.meta + row_base;
+        if (DENSE) {
+            d_codes = b_codes + (size_t)pos * B;
+            d_meta = b_meta + pos;
+            d_x = a.x + pos;
+        }
     };
 
     // the list words of the entries a lane handles in the chunk at list position pos (FULL: all CH
@@ -704,11 +740,23 @@ gemv_kernel(const GemvArgs a)
     // ISSUE: the copies of one chunk (entries pos .. pos+valid-1 of the current block-row's list) into a stage
     auto issue = [&](int pos, int valid, bool full, unsigned st_addr, unsigned bar_addr) {
         if (DENSE) {
-            // the chunk's blocks, pairs and x values are contiguous: three bulk copies by one lane
-            mbar_expect_tx_if(lane0, bar_addr, (unsigned)valid * (B + 6));
-            bulk_copy_if(lane0, st_addr, b_codes + (size_t)pos * B, (unsigned)valid * B, bar_addr);
-            bulk_copy_if(lane0, st_addr + kMetaOff, b_meta + pos, (unsigned)valid * 4, bar_addr);
-            bulk_copy_if(lane0, st_addr + kXcOff, a.x + pos, (unsigned)valid * 2, bar_addr);
+            // the chunk's blocks, pairs and x values are contiguous: three bulk copies by one lane, from
+            // three pointers that simply advance (computing the addresses afresh for every chunk took
+            // five times the instructions)
+            if (full) {
+                mbar_expect_tx_if(lane0, bar_addr, (unsigned)CH * (B + 6));
+                bulk_copy_if(lane0, st_addr, d_codes, (unsigned)CH * B, bar_addr);
+                bulk_copy_if(lane0, st_addr + kMetaOff, d_meta, (unsigned)CH * 4, bar_addr);
+                bulk_copy_if(lane0, st_addr + kXcOff, d_x, (unsigned)CH * 2, bar_addr);
+            } else {
+                mbar_expect_tx_if(lane0, bar_addr, (unsigned)valid * (B + 6));
+                bulk_copy_if(lane0, st_addr, d_codes, (unsigned)valid * B, bar_addr);
+                bulk_copy_if(lane0, st_addr + kMetaOff, d_meta, (unsigned)valid * 4, bar_addr);
+                bulk_copy_if(lane0, st_addr + kXcOff, d_x, (unsigned)valid * 2, bar_addr);
+            }
+            d_codes += CH * B;
+            d_meta += CH;
+            d_x += CH;
             return;
         }
         unsigned col[EPL];
@@ -804,7 +852,7 @@ gemv_kernel(const GemvArgs a)
             while (wi.valid(pc) && !wi.has_chunk()) wi.next_span(pc, warp, true);
         }
         const bool more = wi.valid(pc) && wi.has_chunk();
-        if (more) enter_row(wi.r);
+        if (more) enter_row(wi.r, wi.pos);
         return more;
     };
     bool more_i = seek_issue();

@@ -15,7 +15,7 @@ import os
 import numpy as np
 import torch
 
-from . import binding, inputs
+from . import binding, calibrate, inputs
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 L2_BYTES = 126e6
@@ -196,11 +196,13 @@ def build_stack(layers, tokens, sparsity=0.4, calib_vectors=64):
             row[site] = binding.spqt_pack(W, 4, 128)
             del W
         packs.append(row)
+    pools = {}
     for i, (site, m, n, dist) in enumerate(STACK_SITES):
-        calib = [inputs.activations(n, seed=9000 + 100 * i + c, dist=dist) for c in range(calib_vectors)]
-        thr[site] = inputs.pooled_threshold(calib, sparsity)
+        calib = np.concatenate([inputs.activations(n, seed=9000 + 100 * i + c, dist=dist) for c in range(calib_vectors)])
+        pools[site] = torch.from_numpy(calib).cuda()
         host = np.stack([inputs.activations(n, seed=20000 + 1000 * i + t, dist=dist) for t in range(tokens)])
         xs[site] = (host, torch.from_numpy(host).cuda())
+    thr = calibrate.unified(pools, sparsity)     # one global level: every site's threshold from its own pool
     return packs, thr, xs
 
 
