@@ -197,3 +197,29 @@ def group_sparsity(levels) -> float:
     """Sparsity shared by the matrices that read one input: the mean of their levels (customized mode, Sec. 5)."""
     levels = [float(v) for v in levels]
     return sum(levels) / len(levels)
+
+
+def union_sparsify(X, t: float):
+    """Small batch (several decode rows at once, Sec. 3.2 / Sec. 4.1.3 on beams): the columns that are active
+    in at least one row, k with |X[b][k]| > t for some b, ascending, and their number."""
+    X = np.ascontiguousarray(X, dtype=np.float16)
+    active = set()
+    for b in range(X.shape[0]):
+        idx, cnt = sparsify(X[b], t)
+        active.update(int(k) for k in idx[:cnt])
+    out = np.array(sorted(active), dtype=np.int32)
+    return out, int(out.size)
+
+
+def sparse_gemm_small(codes, scales, zeros, m, n, X, idx, bits=4, group=128, rows=None):
+    """Y[b][j] = sum over the union list of What[j][k] * X[b][k]: every row of the batch is multiplied over
+    the same columns (the union of the rows' active sets), each with its own values -- also those at or
+    below the threshold in that row: the block is read for the batch anyway.  Returns (Y, bound), both
+    float64 [B][rows]; bound[b][j] = sum |What[j][k]| |X[b][k]| over the list."""
+    X = np.ascontiguousarray(X, dtype=np.float16)
+    ys, bs = [], []
+    for b in range(X.shape[0]):
+        y, bound = sparse_gemv(codes, scales, zeros, m, n, X[b], idx, bits, group, rows=rows)
+        ys.append(y)
+        bs.append(bound)
+    return np.stack(ys), np.stack(bs)

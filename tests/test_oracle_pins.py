@@ -399,3 +399,47 @@ def test_calibration_threshold_matches_closed_forms_and_group_mean():
     assert abs(oracle.calibrate_threshold(gau, 0.5) - 0.6745) < 0.01
     assert oracle.group_sparsity([0.3, 0.5, 0.4]) == pytest.approx(0.4, abs=1e-15)
     assert oracle.group_sparsity([0.5]) == 0.5
+
+
+# ------------------------------------------------------------------ small batch over the union of active sets
+
+def test_union_of_active_sets_matches_a_brute_force_scan():
+    g = np.random.Generator(np.random.PCG64(21))
+    X = g.standard_normal((5, 300)).astype(np.float16)
+    X[:, 7] = np.float16(0.1)                  # column 7: below the threshold in every row, NaN in one
+    X[1, 7] = np.float16(np.nan)
+    X[:, 9] = np.float16(0.0)                  # column 9: active through one row only
+    X[0, 9] = np.float16(-np.inf)
+    t = 1.2
+    idx, cnt = oracle.union_sparsify(X, t)
+    brute = [k for k in range(300) if any(abs(float(X[b, k])) > t for b in range(5))]   # NaN compares false
+    assert cnt == len(brute) and idx.tolist() == brute
+    assert 9 in brute and 7 not in brute
+    one, c1 = oracle.union_sparsify(X[:1], t)
+    ref, c2 = oracle.sparsify(X[0], t)
+    assert c1 == c2 and np.array_equal(one, ref)            # a batch of one is the plain index collection
+
+
+def test_small_batch_rows_are_products_over_the_union_in_exact_rationals():
+    m, n, bits, group, B = 8, 6, 4, 4, 3
+    g = np.random.Generator(np.random.PCG64(22))
+    W = (g.integers(-8, 8, size=(m, n)) / 8.0).astype(np.float16)
+    X = (g.integers(-4, 5, size=(B, n)) / 2.0).astype(np.float16)
+    codes, s, z = oracle.pack(W, bits, group)
+    What = oracle.dequantize(codes, s, z, m, n, bits, group)
+    t = 0.75
+    idx, cnt = oracle.union_sparsify(X, t)
+    Y, bound = oracle.sparse_gemm_small(codes, s, z, m, n, X, idx, bits, group)
+    for b in range(B):
+        for j in range(m):
+            ref = sum(Fraction(float(What[j, k])) * Fraction(float(X[b, k])) for k in idx)
+            assert Fraction(float(Y[b, j])) == ref
+            assert Fraction(float(bound[b, j])) == sum(abs(Fraction(float(What[j, k])) * Fraction(float(X[b, k]))) for k in idx)
+    # rows that are all the same give the single-row product in every row
+    Xs = np.repeat(X[:1], 4, axis=0)
+    i1, c1 = oracle.sparsify(X[0], t)
+    iu, cu = oracle.union_sparsify(Xs, t)
+    assert np.array_equal(i1, iu)
+    y1, _ = oracle.sparse_gemv(codes, s, z, m, n, X[0], i1, bits, group)
+    Ys, _ = oracle.sparse_gemm_small(codes, s, z, m, n, Xs, iu, bits, group)
+    assert all(np.array_equal(Ys[b], y1) for b in range(4))
