@@ -221,6 +221,33 @@ spqt_status spqt_sparse_linear_host(const void* codes, const void* scale_zero,
 spqt_status spqt_set_tuning(int gemv_ctas, int no_overlap);
 
 /*
+ * Small batch: B = 1..8 decode rows at once (paper Sec. 3.3 and Sec. 4.1.3 expect beam search with
+ * small beams on the same layout; Sec. 5: with more than one token the system dispatches dense kernels).
+ * The sparse call multiplies every row over the UNION of the rows' active sets:
+ *   idx[0:*count] = every k with |X[b][k]| > t for at least one row b, ascending;
+ *   Y[b][j] = sum_{i < *count} What[j][idx[i]] * X[b][idx[i]]   for every row b
+ * (a row's entries at or below the threshold in columns of the union are used with their values: the
+ * block is read for the batch anyway, so this is never less accurate than thresholding row by row).
+ * Every active block is fetched once for the whole batch.  The dense call is the same over all n
+ * columns.  Dispatch rule: with one row use spqt_sparsify_gemv; with 2..8 rows the sparse call here
+ * as long as the union keeps some sparsity (the union of B sets that are each 50 % sparse is
+ * 1 - 2^-B dense), the dense call otherwise and for prompts; rows beyond 8 in further calls.
+ *   X : fp16 [batch][ldx], ldx >= n, 2-byte aligned.   Y : fp16 [batch][ldy], ldy >= m.
+ *   idx : int32[n], count : int32, both on the device, written by the sparse call.
+ *   workspace : spqt_gemm_small_workspace bytes, 16-byte aligned, zeroed ONCE by the caller; every call
+ *       leaves it ready for the next.  Sums are added in a fixed order: calls are bit-reproducible.
+ * Batches of 5..8 rows run as two passes of four rows over the same list.  Two launches (three for
+ * more than four rows) per sparse call; asynchronous on `stream`.
+ */
+spqt_status spqt_gemm_small_workspace(int m, int n, int bits, int group, size_t* workspace_bytes);
+spqt_status spqt_sparse_gemm_small(const void* codes, const void* scale_zero, int m, int n, int bits, int group,
+                                   const void* X, int ldx, int batch, float t, int32_t* idx, int32_t* count,
+                                   void* Y, int ldy, void* workspace, size_t workspace_bytes, void* stream);
+spqt_status spqt_dense_gemm_small(const void* codes, const void* scale_zero, int m, int n, int bits, int group,
+                                  const void* X, int ldx, int batch, void* Y, int ldy,
+                                  void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Threshold calibration (paper Sec. 5, the calibration threshold tool; Sec. 3.2: thresholds are
  * computed once per sparsity level from calibration activations).  *threshold (a device float) =
  * the nearest-rank order statistic of |x| over the pool x[0:count] of fp16 calibration activations:

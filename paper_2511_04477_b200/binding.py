@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libspqt.so")
 EXPORTS = (
     "spqt_status_string", "spqt_version", "spqt_packed_sizes", "spqt_pack", "spqt_unpack",
     "spqt_sparsify", "spqt_sparse_gemv", "spqt_sparse_gemv_static", "spqt_static_status", "spqt_sparsify_gemv", "spqt_dense_gemv",
-    "spqt_sparse_linear_host", "spqt_autotune", "spqt_calibrate_threshold", "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_launch_count",
+    "spqt_sparse_linear_host", "spqt_gemm_small_workspace", "spqt_sparse_gemm_small", "spqt_dense_gemm_small", "spqt_autotune", "spqt_calibrate_threshold", "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_launch_count",
 )
 
 _lib = None
@@ -59,6 +59,12 @@ def lib() -> ctypes.CDLL:
         L.spqt_dense_gemv.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, sz, vp]
         L.spqt_sparse_linear_host.argtypes = [vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, vp,
                                               vp, vp, vp, vp, vp, sz, vp]
+        L.spqt_gemm_small_workspace.argtypes = [i32, i32, i32, i32, ctypes.POINTER(sz)]
+        L.spqt_gemm_small_workspace.restype = i32
+        L.spqt_sparse_gemm_small.argtypes = [vp, vp, i32, i32, i32, i32, vp, i32, i32, ctypes.c_float, vp, vp, vp, i32, vp, sz, vp]
+        L.spqt_sparse_gemm_small.restype = i32
+        L.spqt_dense_gemm_small.argtypes = [vp, vp, i32, i32, i32, i32, vp, i32, i32, vp, i32, vp, sz, vp]
+        L.spqt_dense_gemm_small.restype = i32
         L.spqt_autotune.argtypes = [vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, vp, vp, vp, vp, sz, vp, sz,
                                     ctypes.POINTER(i32), ctypes.POINTER(i32), vp]
         L.spqt_autotune.restype = i32
@@ -282,6 +288,50 @@ def spqt_probe_read(buf: torch.Tensor, pattern: int, moved: torch.Tensor, stream
 def spqt_set_debug(on: bool) -> None:
     """Checked mode: validate idx/count on the device before every sparse GEMV (off by default)."""
     _ok(lib().spqt_set_debug(1 if on else 0), "spqt_set_debug")
+
+
+def new_gemm_small_workspace(p: Packed) -> torch.Tensor:
+    """Zeroed workspace of the small-batch calls (zeroed once; every call leaves it ready for the next)."""
+    out = ctypes.c_size_t(0)
+    _ok(lib().spqt_gemm_small_workspace(p.m, p.n, p.bits, p.group, ctypes.byref(out)), "spqt_gemm_small_workspace")
+    return torch.zeros(int(out.value), dtype=torch.uint8, device=p.codes.device)
+
+
+def _batch(p: Packed, X: torch.Tensor, Y: torch.Tensor):
+    if X.dim() != 2 or X.stride(1) != 1 or X.shape[1] != p.n or not (1 <= X.shape[0] <= 8):
+        raise ValueError("X must be [batch <= 8][n] with unit column stride")
+    if Y is None:
+        Y = torch.empty((X.shape[0], p.m), dtype=torch.float16, device=X.device)
+    if Y.dtype != torch.float16 or X.dtype != torch.float16 or not X.is_cuda or not Y.is_cuda:
+        raise TypeError("X and Y must be CUDA float16 tensors")
+    if Y.shape != (X.shape[0], p.m) or Y.stride(1) != 1:
+        raise ValueError("Y must be [batch][m] with unit column stride")
+    return Y
+
+
+def spqt_sparse_gemm_small(p: Packed, X: torch.Tensor, t: float, workspace: torch.Tensor, idx: torch.Tensor = None,
+                           count: torch.Tensor = None, Y: torch.Tensor = None, stream=None):
+    """2..8 decode rows over the union of their active sets -> (Y [batch][m], idx, count)."""
+    Y = _batch(p, X, Y)
+    if idx is None:
+        idx = torch.empty(p.n, dtype=torch.int32, device=X.device)
+    if count is None:
+        count = torch.empty(1, dtype=torch.int32, device=X.device)
+    _ok(lib().spqt_sparse_gemm_small(
+        _dev(p.codes, torch.uint8, "codes"), _dev(p.scale_zero, torch.float16, "scale_zero"), p.m, p.n, p.bits, p.group,
+        X.data_ptr(), X.stride(0), X.shape[0], float(t), _dev(idx, torch.int32, "idx"), _dev(count, torch.int32, "count"),
+        Y.data_ptr(), Y.stride(0), _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)),
+        "spqt_sparse_gemm_small")
+    return Y, idx, count
+
+
+def spqt_dense_gemm_small(p: Packed, X: torch.Tensor, workspace: torch.Tensor, Y: torch.Tensor = None, stream=None):
+    Y = _batch(p, X, Y)
+    _ok(lib().spqt_dense_gemm_small(
+        _dev(p.codes, torch.uint8, "codes"), _dev(p.scale_zero, torch.float16, "scale_zero"), p.m, p.n, p.bits, p.group,
+        X.data_ptr(), X.stride(0), X.shape[0], Y.data_ptr(), Y.stride(0),
+        _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)), "spqt_dense_gemm_small")
+    return Y
 
 
 def spqt_autotune(p: Packed, x: torch.Tensor, t: float, workspace: torch.Tensor, flush: torch.Tensor = None, stream=None):

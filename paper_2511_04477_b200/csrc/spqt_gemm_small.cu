@@ -1,0 +1,405 @@
+// Small batch (2..8 decode rows at once: beams, speculative tokens): the sparse product over the UNION
+// of the rows' active sets, and its dense twin.  Every active block is fetched once for the whole
+// batch and its codes are extracted once; only the FMAs are repeated per row, so the byte and the
+// integer-instruction cost per row falls with the batch size.
+//
+//   union_sparsify_kernel   one CTA, ballot/popc compaction like the batch-1 index collection, with
+//                           "active" = |X[b][k]| > t in at least one row b.
+//   gemm_small_kernel       grid (S, R): CTA (s, r) takes the s-th of S equal slices of the union list
+//                           for block-row r; its 8 warps take the slice's chunks of 32 entries in turn,
+//                           each with two code buffers (the next chunk's copies fly during the
+//                           arithmetic).  Lane e of a chunk holds entry e: it loads the entry's column,
+//                           its (scale, zero) pair and the batch's x values and writes the packed
+//                           multiplier pairs of every row; then the warp does the dequantize-FMA work,
+//                           four rows per pass.  Partial sums go warp -> CTA (shared memory) -> block-row
+//                           (fp32 partials in the workspace, arrive-only counter, the last CTA adds them
+//                           in slice order: bit-reproducible).
+// Batches of 5..8 rows run as two passes of up to four rows over the same union list.
+#include <cstddef>
+
+#include "spqt_common.cuh"
+
+namespace spqt {
+constexpr unsigned long long kWaitNs = 1000000000ull;
+}
+#include "spqt_gemv_device.cuh"
+
+namespace spqt {
+
+constexpr int kSmallWarps = 8;
+constexpr int kSmallThreads = kSmallWarps * 32;
+constexpr int kSmallRows = 4;      // batch rows per pass
+constexpr int kSmallMaxSplit = 8;  // slices per block-row at most
+constexpr int kSmallChunk = 32;    // list entries per chunk
+
+__global__ void __launch_bounds__(1024)
+union_sparsify_kernel(const __half* __restrict__ X, int ldx, int batch, int n, float t,
+                      int32_t* __restrict__ idx, int32_t* __restrict__ count)
+{
+    __shared__ int warp_total[32];
+    __shared__ int warp_base[32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int seg = ((n + 32 * 32 - 1) / (32 * 32)) * 32;
+    const int begin = min(warp * seg, n), end = min(begin + seg, n);
+    auto active = [&](int k) -> bool {
+        bool on = false;
+        for (int b = 0; b < batch; ++b) on = on || (fabsf(__half2float(X[(size_t)b * ldx + k])) > t);  // NaN: false
+        return on;
+    };
+    int total = 0;
+    for (int k0 = begin; k0 < end; k0 += 32) {
+        const int k = k0 + lane;
+        total += __popc(__ballot_sync(0xffffffffu, (k < end) && active(k)));
+    }
+    if (lane == 0) warp_total[warp] = total;
+    __syncthreads();
+    if (warp == 0) {
+        int v = warp_total[lane], incl = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            int up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        warp_base[lane] = incl - v;
+        if (lane == 31) *count = incl;
+    }
+    __syncthreads();
+    int base = warp_base[warp];
+    for (int k0 = begin; k0 < end; k0 += 32) {
+        const int k = k0 + lane;
+        const bool p = (k < end) && active(k);
+        const unsigned mask = __ballot_sync(0xffffffffu, p);
+        if (p) idx[base + __popc(mask & ((1u << lane) - 1u))] = k;
+        base += __popc(mask);
+    }
+}
+
+template <int G, int BITS>
+struct SmallSmem {
+    static constexpr int B = G * BITS / 8;
+    alignas(16) unsigned char codes[kSmallWarps][2][kSmallChunk * B];
+    alignas(16) float mult[kSmallWarps][kSmallChunk][kSmallRows][4];
+    alignas(16) float red[kSmallWarps][kSmallRows][G];
+    float red_z[kSmallWarps][kSmallRows];
+    int last;
+};
+
+// idx == nullptr: the dense product (the list is 0, 1, .., n-1 and count is n).
+template <int G, int BITS>
+__global__ void __launch_bounds__(kSmallThreads)
+gemm_small_kernel(const uint8_t* __restrict__ codes, const unsigned* __restrict__ meta, int n,
+                  const __half* __restrict__ X, int ldx, int batch,
+                  const int32_t* __restrict__ idx, const int32_t* __restrict__ count_ptr,
+                  __half* __restrict__ Y, int ldy, float* __restrict__ partials, int* __restrict__ counters)
+{
+    constexpr int B = G * BITS / 8;
+    constexpr int CH = kSmallChunk;
+    constexpr int CB = (B % 16 == 0) ? 16 : 8;        // bytes per copy
+    constexpr int NC = CH * B / CB / 32;              // copies per lane and chunk
+    constexpr int LM = G / 16;                        // arithmetic: lanes per block, 16 codes each
+    constexpr int SLM = 32 / LM;                      // blocks per step
+    constexpr int MSUBS = CH / SLM;                   // steps per chunk
+    constexpr int KEEP = 16 / SLM;
+    constexpr int ROWS = kSmallRows;
+    extern __shared__ __align__(16) unsigned char small_raw[];
+    SmallSmem<G, BITS>& sm = *reinterpret_cast<SmallSmem<G, BITS>*>(small_raw);
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
+    const int s = blockIdx.x, S = gridDim.x, r = blockIdx.y;
+    const int mslot = lane / LM, mh = lane % LM;
+
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
+    const int count = idx ? __ldg(count_ptr) : n;
+    const int lo = (int)(((long long)s * count) / S), hi = (int)(((long long)(s + 1) * count) / S);
+    const size_t row_base = (size_t)r * (size_t)n;
+    const uint8_t* row_codes = codes + row_base * B;
+    const unsigned* row_meta = meta + row_base;
+    const unsigned cbuf = smem_u32(&sm.codes[warp][0][0]);
+    const unsigned mbuf = smem_u32(&sm.mult[warp][0][0][0]);
+    constexpr unsigned kBufBytes = CH * B;
+
+    unsigned long long acc[ROWS][8];
+    float zl[ROWS];
+#pragma unroll
+    for (int b = 0; b < ROWS; ++b) {
+        zl[b] = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[b][i] = 0ull;
+    }
+
+    // column of the entry this lane holds in the chunk at list position pos (past the end: the last entry again)
+    auto column_at = [&](int pos) -> int {
+        const int e = min(pos + lane, hi - 1);
+        return idx ? __ldg(idx + e) : e;
+    };
+    // the chunk's code blocks into one of the warp's two buffers, lane after lane
+    auto copy_codes = [&](int col, unsigned dst) {
+#pragma unroll
+        for (int q = 0; q < NC; ++q) {
+            const int off = (q * 32 + lane) * CB;
+            const int e = off / B, part = off % B;
+            const int cu = __shfl_sync(0xffffffffu, col, e);
+            const uint8_t* src = row_codes + (size_t)cu * B + part;
+            if (CB == 16) cp_async_16_l2_64(dst + off, src);
+            else cp_async_8(dst + off, src);
+        }
+        cp_async_commit();
+    };
+
+    const int first = lo + warp * CH, stride = kSmallWarps * CH;
+    if (first < hi) {
+        int col = column_at(first);
+        copy_codes(col, cbuf);
+        int col_next = first + stride < hi ? column_at(first + stride) : 0;
+        unsigned cur = 0;
+        for (int pos = first; pos < hi; pos += stride) {
+            const bool more = pos + stride < hi;
+            if (more) copy_codes(col_next, cbuf + (cur == 0u ? kBufBytes : 0u));
+            else cp_async_commit();
+            const int col_after = pos + 2 * stride < hi ? column_at(pos + 2 * stride) : 0;
+            // lane e: the pair and the batch's x values of its entry -> multiplier pairs of every row
+            const bool on = pos + lane < hi;
+            const unsigned mz = __ldg(row_meta + col);
+            const float sf = __half2float(__ushort_as_half((unsigned short)(mz & 0xffffu)));
+            const float zf = __half2float(__ushort_as_half((unsigned short)(mz >> 16)));
+#pragma unroll
+            for (int b = 0; b < ROWS; ++b) {
+                float xf = 0.0f;
+                if (on && b < batch) xf = __half2float(__ldg(X + (size_t)b * ldx + col));
+                const float am = xf * sf;       // exact
+                zl[b] += xf * zf;               // exact product
+                const unsigned long long aa = pack2(am, am);
+                sts_pairs(mbuf + 16u * (lane * ROWS + b), fmul2(aa, pack2(0x1p93f, 0x1p89f)), fmul2(aa, pack2(0x1p85f, 0x1p81f)));
+            }
+            cp_async_wait<1>();   // this chunk's copies have landed (the next chunk's may still fly)
+            __syncwarp();
+            const int valid = min(CH, hi - pos);
+            const int nsub = (valid + SLM - 1) / SLM;
+#pragma unroll 1
+            for (int u = 0; u < nsub; ++u) {
+                const unsigned ent = (unsigned)(u * SLM + mslot);
+                if (BITS == 4) {
+                    const uint2 wv = lds_v2(cbuf + cur + lane * 8 + u * 256);
+#pragma unroll
+                    for (int b = 0; b < ROWS; ++b) {
+                        unsigned long long m01, m23;
+                        lds_pairs(mbuf + 16u * (ent * ROWS + b), m01, m23);
+                        fma_block8(acc[b], wv, m01, m23);
+                    }
+                } else {
+                    const unsigned blk = cbuf + cur + ent * B;
+                    const unsigned w2 = lds_u32(blk + 4u * mh);
+                    const unsigned w1 = lds_u32(blk + (G / 4) + 4u * (mh % (LM / 2))) >> (mh / (LM / 2));
+#pragma unroll
+                    for (int b = 0; b < ROWS; ++b) {
+                        unsigned long long m01, m23;
+                        lds_pairs(mbuf + 16u * (ent * ROWS + b), m01, m23);
+                        fma_block3(acc[b], w2, w1, m01, m23);
+                    }
+                }
+            }
+            __syncwarp();
+            cur = (cur == 0u) ? kBufBytes : 0u;
+            col = col_next;
+            col_next = col_after;
+        }
+    }
+    cp_async_wait<0>();
+
+    // warp -> CTA: reduce-scatter over the block slots, per batch row
+#pragma unroll
+    for (int b = 0; b < ROWS; ++b) {
+        float accf[16];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) unpack2(acc[b][i], accf[2 * i], accf[2 * i + 1]);
+        float t8[8], t4[4], keep[4];
+        halve<16>(accf, t8, lane, 16);
+        halve<8>(t8, t4, lane, 8);
+        if (LM == 8) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) keep[i] = t4[i];
+        } else {
+            float t2[2];
+            halve<4>(t4, t2, lane, 4);
+            keep[0] = t2[0];
+            keep[1] = t2[1];
+        }
+#pragma unroll
+        for (int i = 0; i < KEEP; ++i) {
+            const int ai = mslot * KEEP + i;  // accumulator index = word*8 + nibble
+            const int cw = ai >> 3, e2 = ai & 7;
+            const int row = (BITS == 4) ? 8 * mh + 4 * cw + (e2 >> 1) + (e2 & 1) * (G / 2)
+                                        : 4 * mh + (e2 >> 1) + (G / 4) * (2 * (e2 & 1) + cw);
+            sm.red[warp][b][row] = keep[i] * 0x1p56f;
+        }
+        float z = zl[b];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) z += __shfl_xor_sync(0xffffffffu, z, o);
+        if (lane == 0) sm.red_z[warp][b] = z;
+    }
+    __syncthreads();
+
+    // CTA -> block-row
+    float* mine = partials + ((size_t)r * kSmallMaxSplit + s) * ROWS * (G + 1);
+    for (int i = tid; i < ROWS * (G + 1); i += kSmallThreads) {
+        const int b = i / (G + 1), j = i % (G + 1);
+        float v = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kSmallWarps; ++w) v += (j < G) ? sm.red[w][b][j] : sm.red_z[w][b];
+        if (S == 1) {
+            // the only CTA of its block-row: keep the sums in place (warp 0's slot; every element has one writer)
+            if (j < G) sm.red[0][b][j] = v;
+            else sm.red_z[0][b] = v;
+        } else {
+            __stcg(mine + i, v);
+        }
+    }
+    if (S == 1) {
+        __syncthreads();
+        for (int i = tid; i < batch * G; i += kSmallThreads) {
+            const int b = i / G, j = i % G;
+            Y[(size_t)b * ldy + (size_t)r * G + j] = __float2half_rn(sm.red[0][b][j] + sm.red_z[0][b]);
+        }
+        return;
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) sm.last = (atomicAdd(counters + r, 1) == S - 1) ? 1 : 0;
+    __syncthreads();
+    if (!sm.last) return;
+    __threadfence();
+    const float* rowp = partials + (size_t)r * kSmallMaxSplit * ROWS * (G + 1);
+    for (int i = tid; i < batch * G; i += kSmallThreads) {
+        const int b = i / G, j = i % G;
+        float v = 0.0f, z = 0.0f;
+        for (int q = 0; q < S; ++q) {
+            v += __ldcg(rowp + ((size_t)q * ROWS + b) * (G + 1) + j);
+            z += __ldcg(rowp + ((size_t)q * ROWS + b) * (G + 1) + G);
+        }
+        Y[(size_t)b * ldy + (size_t)r * G + j] = __float2half_rn(v + z);
+    }
+    if (tid == 0) counters[r] = 0;   // ready for the next call
+}
+
+inline size_t small_header_bytes(int R) { return (((size_t)R * 4 + 255) / 256) * 256; }
+inline size_t small_workspace_bytes(const Format& f)
+{
+    return small_header_bytes(f.R) + (size_t)f.R * kSmallMaxSplit * kSmallRows * (size_t)(f.group + 1) * sizeof(float);
+}
+
+template <int G, int BITS>
+static spqt_status launch_small(const Format& f, const void* codes, const void* meta, const __half* X, int ldx,
+                                int batch, const int32_t* idx, const int32_t* count, __half* Y, int ldy,
+                                void* workspace, cudaStream_t s)
+{
+    auto kernel = gemm_small_kernel<G, BITS>;
+    static bool configured[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPQT_ERR_CUDA;
+    const int smem = (int)sizeof(SmallSmem<G, BITS>);
+    if (!configured[dev]) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return SPQT_ERR_CUDA;
+        configured[dev] = true;
+    }
+    const int sms = sm_count();
+    if (sms <= 0) return SPQT_ERR_CUDA;
+    int S = (3 * sms + f.R - 1) / f.R;   // about three CTAs per SM
+    if (S > kSmallMaxSplit) S = kSmallMaxSplit;
+    if (S < 1) S = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(S, f.R);
+    cfg.blockDim = dim3(kSmallThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_no_pdl ? 0 : 1;
+    int* counters = static_cast<int*>(workspace);
+    float* partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + small_header_bytes(f.R));
+    for (int b0 = 0; b0 < batch; b0 += kSmallRows) {
+        const int nb = batch - b0 < kSmallRows ? batch - b0 : kSmallRows;
+        const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, static_cast<const uint8_t*>(codes),
+                                                   static_cast<const unsigned*>(meta), f.n, X + (size_t)b0 * ldx, ldx, nb, idx, count,
+                                                   Y + (size_t)b0 * ldy, ldy, partials, counters);
+        count_launch();
+        if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SPQT_ERR_CUDA;
+    }
+    return SPQT_OK;
+}
+
+static spqt_status small_entry(const void* codes, const void* meta, int m, int n, int bits, int group,
+                               const void* X, int ldx, int batch, bool dense, float t, int32_t* idx, int32_t* count,
+                               void* Y, int ldy, void* workspace, size_t ws_bytes, void* stream)
+{
+    if (!codes || !meta || !X || !Y || !workspace) return SPQT_ERR_INVALID_ARG;
+    if (!dense && (!idx || !count)) return SPQT_ERR_INVALID_ARG;
+    if (batch < 1 || batch > 8 || ldx < n || ldy < m) return SPQT_ERR_INVALID_ARG;
+    Format f;
+    spqt_status st = make_format(m, n, bits, group, &f);
+    if (st != SPQT_OK) return st;
+    if (!aligned(codes, 16) || !aligned(meta, 16) || !aligned(X, 2) || !aligned(Y, 2) || !aligned(workspace, 16) ||
+        (!dense && (!aligned(idx, 4) || !aligned(count, 4))))
+        return SPQT_ERR_ALIGNMENT;
+    if (ws_bytes < small_workspace_bytes(f)) return SPQT_ERR_WORKSPACE;
+    if (f.R > 65535) return SPQT_ERR_UNSUPPORTED;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const __half* Xh = static_cast<const __half*>(X);
+    if (!dense) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(1);
+        cfg.blockDim = dim3(1024);
+        cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = g_no_pdl ? 0 : 1;
+        const cudaError_t err = cudaLaunchKernelEx(&cfg, union_sparsify_kernel, Xh, ldx, batch, n, t, idx, count);
+        count_launch();
+        if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SPQT_ERR_CUDA;
+    }
+    const int32_t* li = dense ? nullptr : idx;
+    const int32_t* lc = dense ? nullptr : count;
+    __half* Yh = static_cast<__half*>(Y);
+    if (bits == 4 && group == 128) return launch_small<128, 4>(f, codes, meta, Xh, ldx, batch, li, lc, Yh, ldy, workspace, s);
+    if (bits == 4 && group == 64) return launch_small<64, 4>(f, codes, meta, Xh, ldx, batch, li, lc, Yh, ldy, workspace, s);
+    if (bits == 3 && group == 128) return launch_small<128, 3>(f, codes, meta, Xh, ldx, batch, li, lc, Yh, ldy, workspace, s);
+    return launch_small<64, 3>(f, codes, meta, Xh, ldx, batch, li, lc, Yh, ldy, workspace, s);
+}
+
+}  // namespace spqt
+
+extern "C" {
+
+spqt_status spqt_gemm_small_workspace(int m, int n, int bits, int group, size_t* workspace_bytes)
+{
+    spqt::Format f;
+    spqt_status st = spqt::make_format(m, n, bits, group, &f);
+    if (st != SPQT_OK) return st;
+    if (workspace_bytes) *workspace_bytes = spqt::small_workspace_bytes(f);
+    return SPQT_OK;
+}
+
+spqt_status spqt_sparse_gemm_small(const void* codes, const void* scale_zero, int m, int n, int bits, int group,
+                                   const void* X, int ldx, int batch, float t, int32_t* idx, int32_t* count,
+                                   void* Y, int ldy, void* workspace, size_t workspace_bytes, void* stream)
+{
+    return spqt::small_entry(codes, scale_zero, m, n, bits, group, X, ldx, batch, false, t, idx, count, Y, ldy,
+                             workspace, workspace_bytes, stream);
+}
+
+spqt_status spqt_dense_gemm_small(const void* codes, const void* scale_zero, int m, int n, int bits, int group,
+                                  const void* X, int ldx, int batch, void* Y, int ldy,
+                                  void* workspace, size_t workspace_bytes, void* stream)
+{
+    return spqt::small_entry(codes, scale_zero, m, n, bits, group, X, ldx, batch, true, 0.0f, nullptr, nullptr, Y, ldy,
+                             workspace, workspace_bytes, stream);
+}
+
+}  // extern "C"

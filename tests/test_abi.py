@@ -93,6 +93,12 @@ def test_bad_arguments_launch_nothing(L):
     assert L.spqt_calibrate_threshold(None, 8, 0.5, a16, a16, 131072, None) == 1
     assert L.spqt_calibrate_threshold(a16, 8, 1.5, a16, a16, 131072, None) == 1
     assert L.spqt_calibrate_threshold(a16, 8, 0.5, a16, a16, 131071, None) == 4
+    sws = ctypes.c_size_t(0)
+    assert L.spqt_gemm_small_workspace(128, 8, 4, 128, ctypes.byref(sws)) == 0 and sws.value >= 8 * 4 * 129 * 4
+    assert L.spqt_gemm_small_workspace(100, 8, 4, 128, ctypes.byref(sws)) == 2
+    assert L.spqt_sparse_gemm_small(a16, a16, 128, 8, 4, 128, a16, 8, 9, 0.5, a16, a16, a16, 128, a16, sws.value, None) == 1   # batch > 8
+    assert L.spqt_sparse_gemm_small(a16, a16, 128, 8, 4, 128, a16, 4, 2, 0.5, a16, a16, a16, 128, a16, sws.value, None) == 1   # ldx < n
+    assert L.spqt_dense_gemm_small(a16, a16, 128, 8, 4, 128, a16, 8, 2, a16, 128, a16, sws.value - 1, None) == 4
     assert L.spqt_set_tuning(-1, 0) == 1
     assert L.spqt_set_tuning(0, 8) == 1
     assert L.spqt_workspace_status(None, 128, 128, None, None) == 1

@@ -779,3 +779,74 @@ def test_calibration_threshold_is_the_exact_order_statistic():
     grp = calibrate.grouped(sites, levels)
     for site, names in calibrate.LLAMA_GROUPS.items():
         assert grp[site] == oracle.calibrate_threshold(host[site], oracle.group_sparsity([levels[nm] for nm in names]))
+
+
+# ------------------------------------------------------------------ small batch over the union of active sets
+
+@pytest.mark.parametrize("bits,group", GEMV_FORMATS)
+@pytest.mark.parametrize("m_blocks,n,batch", [(2, 300, 2), (8, 4096, 4), (3, 1111, 3), (32, 4096, 8), (1, 1, 1), (224, 1024, 5)])
+def test_small_batch_over_the_union_matches_the_oracle(bits, group, m_blocks, n, batch):
+    m = m_blocks * group
+    W = inputs.weights(m, n, seed=m + n + batch)
+    X = np.stack([inputs.activations(n, seed=500 + 10 * batch + b, dist="laplace" if b % 2 == 0 else "gauss") for b in range(batch)])
+    if n > 100:
+        X[0, 3] = np.float16(np.nan)
+        X[batch - 1, 4] = np.float16(-np.inf)
+    p = pack_on_gpu(W, bits, group)
+    codes, s, z = packed_to_host(p)
+    ws = binding.new_gemm_small_workspace(p)
+    big = torch.full((batch, n + 8), 7.0, dtype=torch.float16, device="cuda")        # rows with a leading dimension
+    big[:, :n] = dev(X)
+    Xd = big[:, :n]
+    rows = None if m <= 4096 else np.unique(np.random.Generator(np.random.PCG64(4)).integers(0, m, size=128)).astype(np.int32)
+    for sp in (0.5, 0.9, 0.0, None):
+        t = float("inf") if sp is None else inputs.threshold_for_sparsity(X[0], sp)
+        idx = torch.full((n,), -7, dtype=torch.int32, device="cuda")
+        cnt = torch.full((1,), -7, dtype=torch.int32, device="cuda")
+        Y = torch.full((batch, m), float("nan"), dtype=torch.float16, device="cuda")
+        binding.spqt_sparse_gemm_small(p, Xd, t, ws, idx, cnt, Y)
+        torch.cuda.synchronize()
+        ref_idx, ref_cnt = oracle.union_sparsify(X, t)
+        got = idx.cpu().numpy()
+        assert int(cnt.item()) == ref_cnt
+        assert np.array_equal(got[:ref_cnt], ref_idx) and np.all(got[ref_cnt:] == -7)
+        Y_ref, bound = oracle.sparse_gemm_small(codes, s, z, m, n, X, ref_idx, bits, group, rows=rows)
+        Yh = Y.cpu().numpy()
+        for b in range(batch):
+            if n > 100 and b == 0 and 3 in ref_idx:
+                continue                                         # the NaN entry is in the union through another row
+            check_y(Yh[b] if rows is None else Yh[b][rows], Y_ref[b], bound[b], "batch row %d, sparsity %r" % (b, sp))
+        Y2 = torch.empty_like(Y)
+        binding.spqt_sparse_gemm_small(p, Xd, t, ws, idx, cnt, Y2)
+        torch.cuda.synchronize()
+        assert torch.equal(Y.view(torch.int16), Y2.view(torch.int16))        # fixed order of sums
+    Xc = X.copy()
+    if n > 100:
+        Xc[0, 3] = np.float16(0.5)
+        Xc[batch - 1, 4] = np.float16(-0.5)
+    Yd = binding.spqt_dense_gemm_small(p, dev(Xc), ws)
+    torch.cuda.synchronize()
+    for b in range(batch):
+        yd_ref, dbound = oracle.dense_gemv(codes, s, z, m, n, Xc[b], bits, group, rows=rows)
+        yb = Yd.cpu().numpy()[b]
+        check_y(yb if rows is None else yb[rows], yd_ref, dbound, "dense batch row %d" % b)
+    assert not ws[: 4 * (m // group)].any()                      # arrival counters back at zero
+
+
+def test_small_batch_of_identical_rows_equals_the_single_row_call():
+    m, n, bits, group = 1024, 4096, 4, 128
+    W = inputs.weights(m, n, seed=44)
+    x = inputs.activations(n, seed=45)
+    p = pack_on_gpu(W, bits, group)
+    t = inputs.threshold_for_sparsity(x, 0.5)
+    y1, idx1, cnt1 = run_sparse(p, x, t, binding.new_workspace(m, n, bits, group))
+    X = np.repeat(x[None, :], 6, axis=0)
+    Y, idx, cnt = binding.spqt_sparse_gemm_small(p, dev(X), t, binding.new_gemm_small_workspace(p))
+    torch.cuda.synchronize()
+    assert int(cnt.item()) == cnt1 and np.array_equal(idx.cpu().numpy()[:cnt1], idx1)
+    Yh = Y.cpu().numpy().astype(np.float64)
+    codes, s, z = packed_to_host(p)
+    y_ref, bound = oracle.sparse_gemv(codes, s, z, m, n, x, idx1, bits, group)
+    for b in range(6):
+        check_y(Y.cpu().numpy()[b], y_ref, bound, "row %d" % b)
+        assert np.array_equal(Yh[b], Yh[0])
