@@ -2,7 +2,7 @@
 """Benchmark of the SpQt hot path on B200: one line of JSON on stdout.
 
     python bench.py [--gpus N] [--steps K] [--warmup W]            the headline line (config "layer")
-    python bench.py --config sweep | formats | dense | stack       the other workloads, one JSON line each
+    python bench.py --config sweep | formats | dense | batch | stack   the other workloads, one JSON line each
     python bench.py --impl reference                               the fp64 CPU oracle on a bounded sample
 
 Workload of the headline line (the configuration the metric is quoted on): the seven linear layers of
@@ -29,7 +29,8 @@ roofline.achieved = algorithmic bytes per launch of the dominant kernel (gemv_ke
 The other workloads: `sweep` = sparsity 0-90 % on the 14336->4096 and 4096->14336 projections against the
 same-layout dense GEMV, 64 rotated weight copies, with the no-load-balancing ablation beside it;
 `formats` = Llama-2-70B-shaped linears x {int4, int3} x {g128, g64} at 50 % with outlier activations;
-`dense` = the dense zigzag GEMV on the paper's 15 shapes over several grid sizes; `stack` = a per-token
+`dense` = the dense zigzag GEMV on the paper's 15 shapes over several grid sizes; `batch` = 1, 2, 4, 8 rows
+over the union of their active sets; `stack` = a per-token
 pass over a 32-layer Llama-3-8B-shaped stack with thresholds calibrated once for 40 % (tokens/s of the
 linear layers).  The default line carries a short summary of each.
 """
@@ -244,6 +245,17 @@ def other_config_line(which, local, quick=False):
                         config={"workload": "dense same-layout GEMV, m in {2048,4096,8192} x n in {1024..16384}, int4 g128, grids of 64/96/128/148 CTAs "
                                             "and the built-in rule; rotated weight copies > 2x L2"},
                         roofline=roofline_obj(best["dense_gbs"], peak, kind, nb, best["best_us"], "gemv_kernel<128,4,dense>", 1.0),
+                        rows=rows)
+        elif which == "batch":
+            rows = sweep.batch_sweep(peak)
+            r0 = [r for r in rows if r["m"] == 28672 and r["rows"] == "beam-like" and r["batch"] == 4][0]
+            nb = r0["sparse_gbs"] * r0["sparse_us"] * 1e3
+            line = dict(base, metric="sparse int4 GEMM effective HBM GB/s, 4 beam-like rows over the union of their active sets, "
+                                     "stacked gate|up matrix 28672x4096",
+                        value=r0["sparse_gbs"], ms_per_step=r0["sparse_us"] * 1e-3, steps=20, warmup=4,
+                        config={"workload": "1, 2, 4, 8 rows on 28672x4096 and 4096x14336, int4 g128, threshold for 50% on the first row; rows independent "
+                                            "or beam-like (a common hidden state plus 20% individual noise); union index collection + product, and dense"},
+                        roofline=roofline_obj(r0["sparse_gbs"], peak, kind, nb, r0["sparse_us"], "gemm_small_kernel<128,4>", None),
                         rows=rows)
         elif which == "stack":
             res = sweep.run_stack(layers=32, tokens=40 if quick else 100, peak=peak)
@@ -591,7 +603,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1024)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="layer", choices=["layer", "sweep", "formats", "dense", "stack"])
+    ap.add_argument("--config", default="layer", choices=["layer", "sweep", "formats", "dense", "batch", "stack"])
     ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_S,
                     help="device time to accumulate over repeated K-step regions of the headline measurement")
     ap.add_argument("--quick", action="store_true", help="reduced form of --config sweep/formats/stack")

@@ -237,7 +237,8 @@ spqt_status spqt_set_tuning(int gemv_ctas, int no_overlap);
  *   workspace : spqt_gemm_small_workspace bytes, 16-byte aligned, zeroed ONCE by the caller; every call
  *       leaves it ready for the next.  Sums are added in a fixed order: calls are bit-reproducible.
  * Batches of 5..8 rows run as two passes of four rows over the same list.  Two launches (three for
- * more than four rows) per sparse call; asynchronous on `stream`.
+ * more than four rows) per sparse call; asynchronous on `stream`.  The sparse call needs n <= 65535
+ * (SPQT_ERR_UNSUPPORTED beyond).
  */
 spqt_status spqt_gemm_small_workspace(int m, int n, int bits, int group, size_t* workspace_bytes);
 spqt_status spqt_sparse_gemm_small(const void* codes, const void* scale_zero, int m, int n, int bits, int group,

@@ -28,7 +28,7 @@ namespace spqt {
 
 constexpr int kSmallWarps = 8;
 constexpr int kSmallThreads = kSmallWarps * 32;
-constexpr int kSmallRows = 4;      // batch rows per pass
+constexpr int kSmallRows = 4;      // batch rows per pass at most (a pass of one or two rows keeps two sets of sums)
 constexpr int kSmallMaxSplit = 8;  // slices per block-row at most
 constexpr int kSmallChunk = 32;    // list entries per chunk
 
@@ -48,11 +48,18 @@ union_sparsify_kernel(const __half* __restrict__ X, int ldx, int batch, int n, f
         for (int b = 0; b < batch; ++b) on = on || (fabsf(__half2float(X[(size_t)b * ldx + k])) > t);  // NaN: false
         return on;
     };
-    int total = 0;
-    for (int k0 = begin; k0 < end; k0 += 32) {
-        const int k = k0 + lane;
-        total += __popc(__ballot_sync(0xffffffffu, (k < end) && active(k)));
+    // one pass over X: bit `it` of `flags` = this lane's column of the warp's it-th group of 32 is active
+    // (at most 64 groups per warp: n < 2^16); the loads of different groups do not depend on one another
+    unsigned long long flags = 0;
+    const int groups = (end - begin + 31) >> 5;
+#pragma unroll 4
+    for (int it = 0; it < groups; ++it) {
+        const int k = begin + it * 32 + lane;
+        if (k < end && active(k)) flags |= 1ull << it;
     }
+    int total = __popcll(flags);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
     if (lane == 0) warp_total[warp] = total;
     __syncthreads();
     if (warp == 0) {
@@ -67,28 +74,30 @@ union_sparsify_kernel(const __half* __restrict__ X, int ldx, int batch, int n, f
     }
     __syncthreads();
     int base = warp_base[warp];
-    for (int k0 = begin; k0 < end; k0 += 32) {
-        const int k = k0 + lane;
-        const bool p = (k < end) && active(k);
+    for (int it = 0; it < groups; ++it) {
+        const bool p = (flags >> it) & 1ull;
         const unsigned mask = __ballot_sync(0xffffffffu, p);
-        if (p) idx[base + __popc(mask & ((1u << lane) - 1u))] = k;
+        if (p) idx[base + __popc(mask & ((1u << lane) - 1u))] = begin + it * 32 + lane;
         base += __popc(mask);
     }
 }
 
-template <int G, int BITS>
+template <int G, int BITS, int ROWS>
 struct SmallSmem {
     static constexpr int B = G * BITS / 8;
     alignas(16) unsigned char codes[kSmallWarps][2][kSmallChunk * B];
-    alignas(16) float mult[kSmallWarps][kSmallChunk][kSmallRows][4];
-    alignas(16) float red[kSmallWarps][kSmallRows][G];
-    float red_z[kSmallWarps][kSmallRows];
+    alignas(16) float mult[kSmallWarps][kSmallChunk][ROWS][4];
+    alignas(16) float red[kSmallWarps][ROWS][G];
+    float red_z[kSmallWarps][ROWS];
     int last;
 };
 
 // idx == nullptr: the dense product (the list is 0, 1, .., n-1 and count is n).
-template <int G, int BITS>
-__global__ void __launch_bounds__(kSmallThreads)
+// CTAs resident per SM: the sums of four rows take 64 registers of a thread, which leaves room for two CTAs.
+constexpr int small_ctas_per_sm(int rows) { return rows <= 2 ? 3 : 2; }
+
+template <int G, int BITS, int ROWS>
+__global__ void __launch_bounds__(kSmallThreads, small_ctas_per_sm(ROWS))
 gemm_small_kernel(const uint8_t* __restrict__ codes, const unsigned* __restrict__ meta, int n,
                   const __half* __restrict__ X, int ldx, int batch,
                   const int32_t* __restrict__ idx, const int32_t* __restrict__ count_ptr,
@@ -102,9 +111,8 @@ gemm_small_kernel(const uint8_t* __restrict__ codes, const unsigned* __restrict_
     constexpr int SLM = 32 / LM;                      // blocks per step
     constexpr int MSUBS = CH / SLM;                   // steps per chunk
     constexpr int KEEP = 16 / SLM;
-    constexpr int ROWS = kSmallRows;
     extern __shared__ __align__(16) unsigned char small_raw[];
-    SmallSmem<G, BITS>& sm = *reinterpret_cast<SmallSmem<G, BITS>*>(small_raw);
+    SmallSmem<G, BITS, ROWS>& sm = *reinterpret_cast<SmallSmem<G, BITS, ROWS>*>(small_raw);
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
     const int s = blockIdx.x, S = gridDim.x, r = blockIdx.y;
@@ -150,26 +158,63 @@ gemm_small_kernel(const uint8_t* __restrict__ codes, const unsigned* __restrict_
         cp_async_commit();
     };
 
+    // lane e's entry of a chunk: its (scale, zero) pair and the batch's x values (0 past the end of the slice)
+    auto load_entry = [&](int pos, int col, unsigned& mz, unsigned short* xb) {
+        const bool on = pos + lane < hi;
+        mz = __ldg(row_meta + col);
+#pragma unroll
+        for (int b = 0; b < ROWS; ++b)
+            xb[b] = (on && b < batch) ? __ldg(reinterpret_cast<const unsigned short*>(X) + (size_t)b * ldx + col) : (unsigned short)0;
+    };
+    auto step = [&](unsigned cb, int u) {
+        const unsigned ent = (unsigned)(u * SLM + mslot);
+        if (BITS == 4) {
+            const uint2 wv = lds_v2(cb + lane * 8 + u * 256);
+#pragma unroll
+            for (int b = 0; b < ROWS; ++b) {
+                unsigned long long m01, m23;
+                lds_pairs(mbuf + 16u * (ent * ROWS + b), m01, m23);
+                fma_block8(acc[b], wv, m01, m23);
+            }
+        } else {
+            const unsigned blk = cb + ent * B;
+            const unsigned w2 = lds_u32(blk + 4u * mh);
+            const unsigned w1 = lds_u32(blk + (G / 4) + 4u * (mh % (LM / 2))) >> (mh / (LM / 2));
+#pragma unroll
+            for (int b = 0; b < ROWS; ++b) {
+                unsigned long long m01, m23;
+                lds_pairs(mbuf + 16u * (ent * ROWS + b), m01, m23);
+                fma_block3(acc[b], w2, w1, m01, m23);
+            }
+        }
+    };
+
     const int first = lo + warp * CH, stride = kSmallWarps * CH;
     if (first < hi) {
         int col = column_at(first);
         copy_codes(col, cbuf);
         int col_next = first + stride < hi ? column_at(first + stride) : 0;
+        unsigned mz;
+        unsigned short xb[ROWS];
+        load_entry(first, col, mz, xb);
         unsigned cur = 0;
         for (int pos = first; pos < hi; pos += stride) {
             const bool more = pos + stride < hi;
             if (more) copy_codes(col_next, cbuf + (cur == 0u ? kBufBytes : 0u));
             else cp_async_commit();
+            // the loads of the chunks to come, ahead of this chunk's arithmetic
             const int col_after = pos + 2 * stride < hi ? column_at(pos + 2 * stride) : 0;
-            // lane e: the pair and the batch's x values of its entry -> multiplier pairs of every row
-            const bool on = pos + lane < hi;
-            const unsigned mz = __ldg(row_meta + col);
+            unsigned mz_next = 0;
+            unsigned short xb_next[ROWS];
+#pragma unroll
+            for (int b = 0; b < ROWS; ++b) xb_next[b] = 0;
+            if (more) load_entry(pos + stride, col_next, mz_next, xb_next);
+            // lane e: multiplier pairs of every row for its entry
             const float sf = __half2float(__ushort_as_half((unsigned short)(mz & 0xffffu)));
             const float zf = __half2float(__ushort_as_half((unsigned short)(mz >> 16)));
 #pragma unroll
             for (int b = 0; b < ROWS; ++b) {
-                float xf = 0.0f;
-                if (on && b < batch) xf = __half2float(__ldg(X + (size_t)b * ldx + col));
+                const float xf = __half2float(__ushort_as_half(xb[b]));
                 const float am = xf * sf;       // exact
                 zl[b] += xf * zf;               // exact product
                 const unsigned long long aa = pack2(am, am);
@@ -178,34 +223,21 @@ gemm_small_kernel(const uint8_t* __restrict__ codes, const unsigned* __restrict_
             cp_async_wait<1>();   // this chunk's copies have landed (the next chunk's may still fly)
             __syncwarp();
             const int valid = min(CH, hi - pos);
-            const int nsub = (valid + SLM - 1) / SLM;
+            if (valid == CH) {
+#pragma unroll
+                for (int u = 0; u < MSUBS; ++u) step(cbuf + cur, u);
+            } else {
+                const int nsub = (valid + SLM - 1) / SLM;
 #pragma unroll 1
-            for (int u = 0; u < nsub; ++u) {
-                const unsigned ent = (unsigned)(u * SLM + mslot);
-                if (BITS == 4) {
-                    const uint2 wv = lds_v2(cbuf + cur + lane * 8 + u * 256);
-#pragma unroll
-                    for (int b = 0; b < ROWS; ++b) {
-                        unsigned long long m01, m23;
-                        lds_pairs(mbuf + 16u * (ent * ROWS + b), m01, m23);
-                        fma_block8(acc[b], wv, m01, m23);
-                    }
-                } else {
-                    const unsigned blk = cbuf + cur + ent * B;
-                    const unsigned w2 = lds_u32(blk + 4u * mh);
-                    const unsigned w1 = lds_u32(blk + (G / 4) + 4u * (mh % (LM / 2))) >> (mh / (LM / 2));
-#pragma unroll
-                    for (int b = 0; b < ROWS; ++b) {
-                        unsigned long long m01, m23;
-                        lds_pairs(mbuf + 16u * (ent * ROWS + b), m01, m23);
-                        fma_block3(acc[b], w2, w1, m01, m23);
-                    }
-                }
+                for (int u = 0; u < nsub; ++u) step(cbuf + cur, u);
             }
             __syncwarp();
             cur = (cur == 0u) ? kBufBytes : 0u;
             col = col_next;
             col_next = col_after;
+            mz = mz_next;
+#pragma unroll
+            for (int b = 0; b < ROWS; ++b) xb[b] = xb_next[b];
         }
     }
     cp_async_wait<0>();
@@ -244,7 +276,7 @@ gemm_small_kernel(const uint8_t* __restrict__ codes, const unsigned* __restrict_
     __syncthreads();
 
     // CTA -> block-row
-    float* mine = partials + ((size_t)r * kSmallMaxSplit + s) * ROWS * (G + 1);
+    float* mine = partials + ((size_t)r * kSmallMaxSplit + s) * kSmallRows * (G + 1);
     for (int i = tid; i < ROWS * (G + 1); i += kSmallThreads) {
         const int b = i / (G + 1), j = i % (G + 1);
         float v = 0.0f;
@@ -272,13 +304,13 @@ gemm_small_kernel(const uint8_t* __restrict__ codes, const unsigned* __restrict_
     __syncthreads();
     if (!sm.last) return;
     __threadfence();
-    const float* rowp = partials + (size_t)r * kSmallMaxSplit * ROWS * (G + 1);
+    const float* rowp = partials + (size_t)r * kSmallMaxSplit * kSmallRows * (G + 1);
     for (int i = tid; i < batch * G; i += kSmallThreads) {
         const int b = i / G, j = i % G;
         float v = 0.0f, z = 0.0f;
         for (int q = 0; q < S; ++q) {
-            v += __ldcg(rowp + ((size_t)q * ROWS + b) * (G + 1) + j);
-            z += __ldcg(rowp + ((size_t)q * ROWS + b) * (G + 1) + G);
+            v += __ldcg(rowp + ((size_t)q * kSmallRows + b) * (G + 1) + j);
+            z += __ldcg(rowp + ((size_t)q * kSmallRows + b) * (G + 1) + G);
         }
         Y[(size_t)b * ldy + (size_t)r * G + j] = __float2half_rn(v + z);
     }
@@ -291,27 +323,43 @@ inline size_t small_workspace_bytes(const Format& f)
     return small_header_bytes(f.R) + (size_t)f.R * kSmallMaxSplit * kSmallRows * (size_t)(f.group + 1) * sizeof(float);
 }
 
-template <int G, int BITS>
-static spqt_status launch_small(const Format& f, const void* codes, const void* meta, const __half* X, int ldx,
-                                int batch, const int32_t* idx, const int32_t* count, __half* Y, int ldy,
-                                void* workspace, cudaStream_t s)
+// Slices per block-row: the grid runs in waves of `per_sm` CTAs per SM; a CTA costs a fixed part (set-up,
+// reduction, the exchange of partial sums) plus its share of the list.  Pick the split with the lowest
+// estimate; ties go to the smaller one.
+static int small_split(int R, int n, int sms, int per_sm)
 {
-    auto kernel = gemm_small_kernel<G, BITS>;
+    const double slots = (double)per_sm * sms;
+    int best = 1;
+    double best_t = 0.0;
+    for (int S = 1; S <= kSmallMaxSplit; ++S) {
+        const double waves = (double)((long long)((R * (double)S + slots - 1) / slots));
+        const double t = waves * (4.0 + 1.5 * (double)n / (256.0 * S));
+        if (S == 1 || t < best_t - 1e-9) {
+            best = S;
+            best_t = t;
+        }
+    }
+    return best;
+}
+
+template <int G, int BITS, int ROWS>
+static spqt_status launch_small_rows(const Format& f, const void* codes, const void* meta, const __half* X, int ldx,
+                                     int nb, const int32_t* idx, const int32_t* count, __half* Y, int ldy,
+                                     void* workspace, cudaStream_t s)
+{
+    auto kernel = gemm_small_kernel<G, BITS, ROWS>;
     static bool configured[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPQT_ERR_CUDA;
-    const int smem = (int)sizeof(SmallSmem<G, BITS>);
+    const int smem = (int)sizeof(SmallSmem<G, BITS, ROWS>);
     if (!configured[dev]) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return SPQT_ERR_CUDA;
         configured[dev] = true;
     }
     const int sms = sm_count();
     if (sms <= 0) return SPQT_ERR_CUDA;
-    int S = (3 * sms + f.R - 1) / f.R;   // about three CTAs per SM
-    if (S > kSmallMaxSplit) S = kSmallMaxSplit;
-    if (S < 1) S = 1;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(S, f.R);
+    cfg.gridDim = dim3(small_split(f.R, f.n, sms, small_ctas_per_sm(ROWS)), f.R);
     cfg.blockDim = dim3(kSmallThreads);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = s;
@@ -322,13 +370,24 @@ static spqt_status launch_small(const Format& f, const void* codes, const void* 
     cfg.numAttrs = g_no_pdl ? 0 : 1;
     int* counters = static_cast<int*>(workspace);
     float* partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + small_header_bytes(f.R));
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, static_cast<const uint8_t*>(codes),
+                                               static_cast<const unsigned*>(meta), f.n, X, ldx, nb, idx, count,
+                                               Y, ldy, partials, counters);
+    count_launch();
+    return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SPQT_OK : SPQT_ERR_CUDA;
+}
+
+template <int G, int BITS>
+static spqt_status launch_small(const Format& f, const void* codes, const void* meta, const __half* X, int ldx,
+                                int batch, const int32_t* idx, const int32_t* count, __half* Y, int ldy,
+                                void* workspace, cudaStream_t s)
+{
     for (int b0 = 0; b0 < batch; b0 += kSmallRows) {
         const int nb = batch - b0 < kSmallRows ? batch - b0 : kSmallRows;
-        const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, static_cast<const uint8_t*>(codes),
-                                                   static_cast<const unsigned*>(meta), f.n, X + (size_t)b0 * ldx, ldx, nb, idx, count,
-                                                   Y + (size_t)b0 * ldy, ldy, partials, counters);
-        count_launch();
-        if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SPQT_ERR_CUDA;
+        const spqt_status st =
+            nb <= 2 ? launch_small_rows<G, BITS, 2>(f, codes, meta, X + (size_t)b0 * ldx, ldx, nb, idx, count, Y + (size_t)b0 * ldy, ldy, workspace, s)
+                    : launch_small_rows<G, BITS, 4>(f, codes, meta, X + (size_t)b0 * ldx, ldx, nb, idx, count, Y + (size_t)b0 * ldy, ldy, workspace, s);
+        if (st != SPQT_OK) return st;
     }
     return SPQT_OK;
 }
@@ -348,6 +407,7 @@ static spqt_status small_entry(const void* codes, const void* meta, int m, int n
         return SPQT_ERR_ALIGNMENT;
     if (ws_bytes < small_workspace_bytes(f)) return SPQT_ERR_WORKSPACE;
     if (f.R > 65535) return SPQT_ERR_UNSUPPORTED;
+    if (!dense && n > 65535) return SPQT_ERR_UNSUPPORTED;  // the index collection keeps 64 flag bits per lane
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const __half* Xh = static_cast<const __half*>(X);
     if (!dense) {

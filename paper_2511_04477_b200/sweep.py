@@ -175,6 +175,48 @@ def dense_shape_sweep(peak):
     return out
 
 
+def batch_sweep(peak):
+    """Small batches (1, 2, 4, 8 rows) on the stacked gate|up matrix and the down projection, int4 g128: rows that
+    are independent draws (their union is 1 - 2^-B dense at 50 % each) and rows that share most of their
+    hidden state, as beams do (a common vector plus 20 % individual noise).  Sparse over the union, and dense."""
+    out = []
+    for (m, n, dist) in [(28672, 4096, "laplace"), (4096, 14336, "gauss")]:
+        copies = copies_for(m, n, 4, 128)
+        packs = make_copies(m, n, 4, 128, copies)
+        calls = max(copies, 16)
+        ws1 = binding.new_workspace(m, n, 4, 128)
+        wsb = binding.new_gemm_small_workspace(packs[0])
+        idx = torch.empty(n, dtype=torch.int32, device="cuda")
+        cnt = torch.zeros(1, dtype=torch.int32, device="cuda")
+        base = inputs.activations(n, seed=31, dist=dist).astype(np.float32)
+        for kind in ("independent", "beam-like"):
+            for batch in (1, 2, 4, 8):
+                if kind == "independent":
+                    X = np.stack([inputs.activations(n, seed=40 + b, dist=dist) for b in range(batch)])
+                else:
+                    X = np.stack([(base + 0.2 * inputs.activations(n, seed=60 + b, dist=dist).astype(np.float32)).astype(np.float16)
+                                  for b in range(batch)])
+                t = inputs.threshold_for_sparsity(X[0], 0.5)
+                Xd = torch.from_numpy(X).cuda()
+                Y = torch.empty((batch, m), dtype=torch.float16, device="cuda")
+                if batch == 1:
+                    us, _ = graph_us(lambda i, s: binding.spqt_sparsify_gemv(packs[i % copies], Xd[0], t, ws1, idx, cnt, Y[0], stream=s), calls)
+                    us_d, _ = graph_us(lambda i, s: binding.spqt_dense_gemv(packs[i % copies], Xd[0], ws1, Y[0], stream=s), calls)
+                else:
+                    us, _ = graph_us(lambda i, s: binding.spqt_sparse_gemm_small(packs[i % copies], Xd, t, wsb, idx, cnt, Y, stream=s), calls)
+                    us_d, _ = graph_us(lambda i, s: binding.spqt_dense_gemm_small(packs[i % copies], Xd, wsb, Y, stream=s), calls)
+                torch.cuda.synchronize()
+                count = int(cnt.item())
+                nb = needed_bytes(m, n, count, 4, 128) + (batch - 1) * (2 * n + 2 * m)
+                out.append({"m": m, "n": n, "rows": kind, "batch": batch, "union_count": count, "union_sparsity": 1.0 - count / n,
+                            "sparse_us": us, "sparse_us_per_row": us / batch, "dense_us": us_d, "dense_us_per_row": us_d / batch,
+                            "sparse_gbs": nb / us * 1e-3, "frac_of_peak": nb / us * 1e-3 / peak,
+                            "speedup_vs_dense": us_d / us})
+        del packs
+        torch.cuda.empty_cache()
+    return out
+
+
 STACK_SITES = [  # (site, stacked matrix rows, n, distribution of the site's input)
     ("attn_in", 6144, 4096, "laplace"),    # q | k | v share x and idx
     ("attn_out", 4096, 4096, "laplace"),   # o
