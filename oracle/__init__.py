@@ -223,3 +223,33 @@ def sparse_gemm_small(codes, scales, zeros, m, n, X, idx, bits=4, group=128, row
         ys.append(y)
         bs.append(bound)
     return np.stack(ys), np.stack(bs)
+
+
+def rowwise_quantize(W, bits: int = 4, group: int = 128):
+    """The conventional layout the paper contrasts the zigzag layout with (Sec. 2, Sec. 4.1.1): a quantization
+    group is `group` consecutive COLUMNS of one row.  Same quantizer as `quantize` (min/max, round to nearest),
+    applied along the other axis: the groups of W along its rows are the groups of W^T down its columns.
+    fp16 W[m][n] -> (q uint8[m][n], scales fp16[m][n/group], zeros fp16[m][n/group])."""
+    Wt = np.ascontiguousarray(np.asarray(W, dtype=np.float16).T)
+    q, s, z = quantize(Wt, bits, group)
+    return np.ascontiguousarray(q.T), np.ascontiguousarray(s.T), np.ascontiguousarray(z.T)
+
+
+def rowwise_pack_codes(q, bits: int = 4, group: int = 128) -> np.ndarray:
+    """Row-wise block order: block (j, g) = the codes of columns g*group .. g*group+group-1 of row j, stored at
+    block index j*(n/group) + g; inside a block the bytes follow the same rule as a zigzag block."""
+    q = np.ascontiguousarray(q, dtype=np.uint8)
+    m, n = q.shape
+    B = block_bytes(bits, group)
+    by_group_then_row = pack_codes(np.ascontiguousarray(q.T), bits, group).reshape(n // group, m, B)
+    return np.ascontiguousarray(by_group_then_row.transpose(1, 0, 2)).reshape(-1)
+
+
+def rowwise_dense_gemv(q, scales, zeros, x, group: int = 128):
+    """y[j] = sum_k (scale[j][k/group] * q[j][k] + zero[j][k/group]) * x[k] in float64, and
+    bound[j] = sum_k |What[j][k]| |x[k]|."""
+    s = np.repeat(np.asarray(scales, dtype=np.float16).astype(np.float64), group, axis=1)
+    z = np.repeat(np.asarray(zeros, dtype=np.float16).astype(np.float64), group, axis=1)
+    What = s * np.asarray(q, dtype=np.float64) + z
+    xv = np.asarray(x, dtype=np.float16).astype(np.float64)
+    return What @ xv, np.abs(What) @ np.abs(xv)

@@ -443,3 +443,64 @@ def test_small_batch_rows_are_products_over_the_union_in_exact_rationals():
     y1, _ = oracle.sparse_gemv(codes, s, z, m, n, X[0], i1, bits, group)
     Ys, _ = oracle.sparse_gemm_small(codes, s, z, m, n, Xs, iu, bits, group)
     assert all(np.array_equal(Ys[b], y1) for b in range(4))
+
+
+# ---------------------------------------------------------------- row-wise baseline layout (Sec. 2, Sec. 4.1.1)
+
+def test_rowwise_hand_example():
+    # The two groups of the hand-worked example (tests/golden/hand_example.txt, columns 0 and 2 of
+    # block-row 0), laid along rows instead of down columns: same scales, offsets and codes.
+    W = np.array([[0.0, 0.25, 0.5, 3.75], [1.0, 2.0, 3.0, 4.0]], dtype=np.float16)
+    q, s, z = oracle.rowwise_quantize(W, 4, 4)
+    assert q.tolist() == [[0, 1, 2, 15], [0, 5, 10, 15]]
+    assert s.shape == (2, 1) and z.shape == (2, 1)
+    assert float(s[0, 0]) == 0.25 and float(z[0, 0]) == 0.0
+    assert s.view(np.uint16)[1, 0] == 0x3266 and float(z[1, 0]) == 1.0
+    # bytes of a block: byte i = code i | code i+2 << 4 (group of 4)
+    assert oracle.rowwise_pack_codes(q, 4, 4).tolist() == [0x20, 0xF1, 0xA0, 0xF5]
+    x = np.array([1.0, -2.0, 0.5, 1.0], dtype=np.float16)
+    y, bound = oracle.rowwise_dense_gemv(q, s, z, x, 4)
+    assert y[0] == 0.0 - 0.5 + 0.25 + 3.75
+    s1 = 0.199951171875
+    assert y[1] == (1 + 0 * s1) * 1 + (1 + 5 * s1) * -2 + (1 + 10 * s1) * 0.5 + (1 + 15 * s1) * 1
+    assert bound[0] == 0.5 + 0.25 + 3.75
+
+
+def test_rowwise_quantizer_brute_force():
+    # per row and per group of consecutive columns, the quantizer's steps in numpy float32
+    rng = np.random.default_rng(11)
+    m, n, G = 5, 24, 8
+    W = (rng.standard_normal((m, n)) * 0.05).astype(np.float16)
+    q, s, z = oracle.rowwise_quantize(W, 4, G)
+    for j in range(m):
+        for g in range(n // G):
+            w = W[j, g * G:(g + 1) * G].astype(np.float32)
+            lo, hi = np.float32(w.min()), np.float32(w.max())
+            sc = np.float16(np.float32(hi - lo) / np.float32(15))
+            assert s[j, g] == sc and z[j, g] == np.float16(lo)
+            sf = np.float32(sc)
+            codes = np.clip(np.rint((w - lo) / sf), 0, 15).astype(np.uint8) if sf != 0 else np.zeros(G, np.uint8)
+            assert q[j, g * G:(g + 1) * G].tolist() == codes.tolist()
+
+
+def test_rowwise_layout_and_product_exact():
+    from fractions import Fraction
+    rng = np.random.default_rng(12)
+    m, n, G = 3, 16, 8
+    W = (rng.standard_normal((m, n)) * 0.1).astype(np.float16)
+    x = rng.choice(np.array([1.0, -2.0, 0.5, 0.0, 3.0], dtype=np.float16), n)
+    q, s, z = oracle.rowwise_quantize(W, 4, G)
+    codes = oracle.rowwise_pack_codes(q, 4, G)
+    B = G // 2
+    assert codes.size == m * (n // G) * B
+    for j in range(m):
+        for g in range(n // G):
+            blk = codes[(j * (n // G) + g) * B:(j * (n // G) + g + 1) * B]
+            for i in range(B):
+                assert blk[i] == (q[j, g * G + i] | (q[j, g * G + i + B] << 4))
+    y, _ = oracle.rowwise_dense_gemv(q, s, z, x, G)
+    for j in range(m):
+        acc = Fraction(0)
+        for k in range(n):
+            acc += (Fraction(float(s[j, k // G])) * int(q[j, k]) + Fraction(float(z[j, k // G]))) * Fraction(float(x[k]))
+        assert abs(float(acc) - y[j]) <= 1e-12 * max(1.0, abs(float(acc)))
