@@ -249,6 +249,32 @@ spqt_status spqt_dense_gemm_small(const void* codes, const void* scale_zero, int
                                   void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Comparison baseline, not part of the method: the conventional ROW-WISE grouping the paper contrasts
+ * its layout with (paper Sec. 2 and Sec. 4.1.1: groups of consecutive weights of one row suit a
+ * row-parallel GEMV but conflict with column sparsity; Sec. 6 compares the dense kernel over the zigzag
+ * layout with the stock row-wise one on 15 shapes).  Same quantizer as spqt_pack, 4-bit only:
+ *   block (j, g) = the codes of columns g*group .. g*group+group-1 of row j, at byte
+ *                  (j*(n/group) + g) * group/2; byte i of a block = code i | code (i + group/2) << 4;
+ *   scale_zero   = fp16 pairs (scale, zero) in the same block order.
+ * n must be a multiple of group (SPQT_ERR_UNSUPPORTED otherwise; any m >= 1); bits must be 4.
+ *   spqt_rowwise_packed_sizes : bytes of codes (m*n/2) and of scale_zero (4*m*n/group); host only.
+ *   spqt_rowwise_pack         : W fp16 row-major [m][ldw >= n] (2-byte aligned) -> codes, scale_zero
+ *                               (both 16-byte aligned, caller-allocated).
+ *   spqt_rowwise_dense_gemv   : y[j] = sum_k What[j][k] * x[k] over all n columns; x fp16[n], y fp16[m]
+ *                               (2-byte aligned); n <= 16384 (SPQT_ERR_UNSUPPORTED beyond: a row must fit
+ *                               the 16 warps of a CTA).  Needs no workspace: every row is summed inside one
+ *                               CTA, in a fixed order (bit-reproducible).
+ * All device pointers; asynchronous on `stream`; nothing is allocated or retained.
+ */
+spqt_status spqt_rowwise_packed_sizes(int m, int n, int bits, int group,
+                                      size_t* codes_bytes, size_t* scale_zero_bytes);
+spqt_status spqt_rowwise_pack(const void* W, int m, int n, int ldw, int bits, int group,
+                              void* codes, void* scale_zero, void* stream);
+spqt_status spqt_rowwise_dense_gemv(const void* codes, const void* scale_zero,
+                                    int m, int n, int bits, int group,
+                                    const void* x, void* y, void* stream);
+
+/*
  * Threshold calibration (paper Sec. 5, the calibration threshold tool; Sec. 3.2: thresholds are
  * computed once per sparsity level from calibration activations).  *threshold (a device float) =
  * the nearest-rank order statistic of |x| over the pool x[0:count] of fp16 calibration activations:

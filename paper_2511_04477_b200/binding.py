@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libspqt.so")
 EXPORTS = (
     "spqt_status_string", "spqt_version", "spqt_packed_sizes", "spqt_pack", "spqt_unpack",
     "spqt_sparsify", "spqt_sparse_gemv", "spqt_sparse_gemv_static", "spqt_static_status", "spqt_sparsify_gemv", "spqt_dense_gemv",
-    "spqt_sparse_linear_host", "spqt_gemm_small_workspace", "spqt_sparse_gemm_small", "spqt_dense_gemm_small", "spqt_autotune", "spqt_calibrate_threshold", "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_launch_count",
+    "spqt_sparse_linear_host", "spqt_gemm_small_workspace", "spqt_sparse_gemm_small", "spqt_dense_gemm_small", "spqt_rowwise_packed_sizes", "spqt_rowwise_pack", "spqt_rowwise_dense_gemv", "spqt_autotune", "spqt_calibrate_threshold", "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_launch_count",
 )
 
 _lib = None
@@ -57,6 +57,9 @@ def lib() -> ctypes.CDLL:
         L.spqt_sparsify_gemv.argtypes = [vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, vp, vp, vp, vp, sz, vp]
         L.spqt_sparsify_gemv.restype = i32
         L.spqt_dense_gemv.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, sz, vp]
+        L.spqt_rowwise_packed_sizes.argtypes = [i32, i32, i32, i32] + [ctypes.POINTER(sz)] * 2
+        L.spqt_rowwise_pack.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp]
+        L.spqt_rowwise_dense_gemv.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp]
         L.spqt_sparse_linear_host.argtypes = [vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, vp,
                                               vp, vp, vp, vp, vp, sz, vp]
         L.spqt_gemm_small_workspace.argtypes = [i32, i32, i32, i32, ctypes.POINTER(sz)]
@@ -332,6 +335,54 @@ def spqt_dense_gemm_small(p: Packed, X: torch.Tensor, workspace: torch.Tensor, Y
         X.data_ptr(), X.stride(0), X.shape[0], Y.data_ptr(), Y.stride(0),
         _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)), "spqt_dense_gemm_small")
     return Y
+
+
+@dataclass
+class RowwisePacked:
+    """Device buffers written by :func:`spqt_rowwise_pack` (the row-wise comparison layout)."""
+    codes: torch.Tensor        # uint8[m*n/2]
+    scale_zero: torch.Tensor   # float16[2*m*n/group]
+    m: int
+    n: int
+    bits: int
+    group: int
+
+    @property
+    def scales(self) -> torch.Tensor:
+        return self.scale_zero[0::2]
+
+    @property
+    def zeros(self) -> torch.Tensor:
+        return self.scale_zero[1::2]
+
+
+def spqt_rowwise_packed_sizes(m: int, n: int, bits: int = 4, group: int = 128):
+    out = [ctypes.c_size_t(0) for _ in range(2)]
+    _ok(lib().spqt_rowwise_packed_sizes(m, n, bits, group, *[ctypes.byref(o) for o in out]), "spqt_rowwise_packed_sizes")
+    return int(out[0].value), int(out[1].value)
+
+
+def spqt_rowwise_pack(W: torch.Tensor, bits: int = 4, group: int = 128, stream=None) -> RowwisePacked:
+    if W.dim() != 2 or W.stride(1) != 1:
+        raise ValueError("W must be 2-D with unit column stride")
+    if not W.is_cuda or W.dtype != torch.float16:
+        raise TypeError("W must be a CUDA float16 tensor")
+    m, n = W.shape
+    cb, sb = spqt_rowwise_packed_sizes(m, n, bits, group)
+    codes = torch.empty(cb, dtype=torch.uint8, device=W.device)
+    scale_zero = torch.empty(sb // 2, dtype=torch.float16, device=W.device)
+    _ok(lib().spqt_rowwise_pack(W.data_ptr(), m, n, W.stride(0), bits, group, codes.data_ptr(),
+                                scale_zero.data_ptr(), _stream(stream)), "spqt_rowwise_pack")
+    return RowwisePacked(codes, scale_zero, m, n, bits, group)
+
+
+def spqt_rowwise_dense_gemv(p: RowwisePacked, x: torch.Tensor, y: torch.Tensor = None, stream=None) -> torch.Tensor:
+    if y is None:
+        y = torch.empty(p.m, dtype=torch.float16, device=x.device)
+    _ok(lib().spqt_rowwise_dense_gemv(
+        _dev(p.codes, torch.uint8, "codes"), _dev(p.scale_zero, torch.float16, "scale_zero"), p.m, p.n, p.bits, p.group,
+        _dev(x, torch.float16, "x"), _dev(y, torch.float16, "y"), _stream(stream)), "spqt_rowwise_dense_gemv")
+    return y
 
 
 def spqt_autotune(p: Packed, x: torch.Tensor, t: float, workspace: torch.Tensor, flush: torch.Tensor = None, stream=None):

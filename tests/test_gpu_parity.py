@@ -850,3 +850,55 @@ def test_small_batch_of_identical_rows_equals_the_single_row_call():
     for b in range(6):
         check_y(Y.cpu().numpy()[b], y_ref, bound, "row %d" % b)
         assert np.array_equal(Yh[b], Yh[0])
+
+
+# ---------------------------------------------------------------- row-wise comparison baseline
+
+@pytest.mark.parametrize("group", [128, 64])
+@pytest.mark.parametrize("m,n", [(8, 128), (1000, 1152), (333, 1024), (1024, 4096), (4096, 4096), (2051, 14336), (64, 16384), (5000, 2048)])
+def test_rowwise_baseline_pack_and_dense_gemv_match_the_oracle(group, m, n):
+    W = inputs.weights(m, n, seed=3 * m + n + group)
+    W[0, :group] = np.float16(0.25)                      # a constant group: scale 0
+    W[m - 1, n - group:n - group + 2] = np.array([0.0, -0.0], dtype=np.float16)
+    x = inputs.activations(n, seed=m + 7, dist="gauss" if n > 8192 else "laplace")
+    q, s, z = oracle.rowwise_quantize(W, 4, group)
+    p = binding.spqt_rowwise_pack(dev(W), 4, group)
+    torch.cuda.synchronize()
+    assert np.array_equal(p.codes.cpu().numpy(), oracle.rowwise_pack_codes(q, 4, group))
+    assert np.array_equal(p.scales.cpu().numpy().view(np.uint16).reshape(m, n // group), s.view(np.uint16))
+    assert np.array_equal(p.zeros.cpu().numpy().view(np.uint16).reshape(m, n // group), z.view(np.uint16))
+    y = torch.full((m,), float("nan"), dtype=torch.float16, device="cuda")
+    binding.spqt_rowwise_dense_gemv(p, dev(x), y)
+    torch.cuda.synchronize()
+    y_ref, bound = oracle.rowwise_dense_gemv(q, s, z, x, group)
+    check_y(y.cpu().numpy(), y_ref, bound, "row-wise dense %dx%d g%d" % (m, n, group))
+    y2 = binding.spqt_rowwise_dense_gemv(p, dev(x))
+    torch.cuda.synchronize()
+    assert torch.equal(y.view(torch.int16), y2.view(torch.int16))             # fixed order of sums
+
+
+@pytest.mark.parametrize("group", [128, 64])
+def test_rowwise_baseline_is_exact_on_lossless_weights(group):
+    # codes along a row take every value 0..15 inside every group (the column coefficient is odd), so
+    # scale = 1/16 and zero = 0: the product is an exact small rational
+    m, n = 515, 3072
+    j, k = np.meshgrid(np.arange(m), np.arange(n), indexing="ij")
+    W = (((3 * j + 5 * k) % 16) / 16.0).astype(np.float16)
+    x = np.random.Generator(np.random.PCG64(8)).choice(np.array([1, -1, 2, -2, 0.5, -0.5], dtype=np.float16), n)
+    p = binding.spqt_rowwise_pack(dev(W), 4, group)
+    y = binding.spqt_rowwise_dense_gemv(p, dev(x))
+    torch.cuda.synchronize()
+    exact = W.astype(np.float64) @ x.astype(np.float64)
+    assert np.array_equal(y.cpu().numpy(), exact.astype(np.float16))
+    assert np.array_equal(exact.astype(np.float16).astype(np.float64), exact)   # the exact result is an fp16 value
+
+
+def test_rowwise_baseline_refuses_what_it_does_not_cover():
+    L = binding.lib()
+    buf = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    a = buf.data_ptr()
+    assert L.spqt_rowwise_pack(a, 8, 100, 100, 4, 128, a, a, None) == 2          # n not a multiple of the group
+    assert L.spqt_rowwise_pack(a, 8, 128, 128, 3, 128, a, a, None) == 2          # 4-bit only
+    assert L.spqt_rowwise_dense_gemv(a, a, 8, 16384 + 128, 4, 128, a, a, None) == 2
+    assert L.spqt_rowwise_dense_gemv(a, a, 8, 128, 4, 128, None, a, None) == 1
+    assert L.spqt_rowwise_dense_gemv(a + 4, a, 8, 128, 4, 128, a, a, None) == 3
