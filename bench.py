@@ -243,8 +243,9 @@ def other_config_line(which, local, quick=False):
             line = dict(base, metric="dense zigzag int4 GEMV effective HBM GB/s, best of the 15 shapes of the paper's hyper-parameter study",
                         value=best["dense_gbs"], ms_per_step=best["best_us"] * 1e-3, steps=10, warmup=4,
                         config={"workload": "dense same-layout GEMV, m in {2048,4096,8192} x n in {1024..16384}, int4 g128, grids of 64/96/128/148 CTAs "
-                                            "and the built-in rule; rotated weight copies > 2x L2"},
+                                            "and the built-in rule; beside it the row-wise-layout baseline (spqt_rowwise_dense_gemv) on the same shapes; rotated weight copies > 2x L2"},
                         roofline=roofline_obj(best["dense_gbs"], peak, kind, nb, best["best_us"], "gemv_kernel<128,4,dense>", 1.0),
+                        zigzag_dense_vs_rowwise={"%dx%d" % (r["m"], r["n"]): r["zigzag_dense_vs_rowwise"] for r in rows},
                         rows=rows)
         elif which == "batch":
             rows = sweep.batch_sweep(peak)

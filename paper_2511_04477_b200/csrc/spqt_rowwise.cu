@@ -14,7 +14,8 @@
 // group walks over chunks of ROWS rows: the chunk's codes and (scale, zero) pairs arrive through a
 // three-stage cp.async ring per warp; per row a lane forms sum(code * x) of its 32 codes, applies its
 // group's scale and adds zero * sum(x); the ROWS values are reduced across the warp by a butterfly
-// reduce-scatter, across the row group's warps through shared memory (fixed order: bit-reproducible).
+// reduce-scatter, across the row group's warps through a ring of shared-memory buffers guarded by
+// mbarriers (bounded waits), added by the group's first warp in warp order: bit-reproducible.
 #include <cstddef>
 
 #include "spqt_common.cuh"
@@ -31,6 +32,7 @@ constexpr int kRwThreads = kRwWarps * 32;
 constexpr int kRwDepth = 3;          // chunks in flight per warp
 constexpr int kRwStep = 512;         // bytes of one row's codes a warp covers (1024 columns)
 constexpr int kRwMaxN = kRwWarps * 1024;
+constexpr int kRwParts = 4;          // chunks whose per-warp sums may wait to be added
 
 // ---------------------------------------------------------------- conversion
 
@@ -91,13 +93,10 @@ struct RwSmem {
         alignas(16) unsigned meta[ROWS][NG];
     };
     Stage stage[kRwWarps][kRwDepth];
-    float part[2][kRwWarps][ROWS];  // per-warp sums of a chunk's rows, double-buffered
+    float part[kRwParts][kRwWarps][ROWS];   // per-warp sums of a chunk's rows: a ring of kRwParts chunks
+    uint64_t full[kRwWarps][kRwParts];      // per row group: every warp of the group has written its sums
+    uint64_t empty[kRwWarps][kRwParts];     // per row group: the summing warp has read them
 };
-
-__device__ __forceinline__ void group_barrier(int id, int threads)
-{
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
-}
 
 // Sums of ROWS values per lane -> one row's sum over the warp in the lanes with (lane & (32/ROWS - 1)) == 0;
 // `row` = which row that lane holds.
@@ -147,7 +146,13 @@ rowwise_gemv_kernel(const uint8_t* __restrict__ codes, const unsigned* __restric
     Smem& sm = *reinterpret_cast<Smem*>(rw_raw);
     const int lane = threadIdx.x & 31;
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
-    if (warp >= Wc * Rg) return;  // (the named barriers below only count the warps of a row group)
+    if (threadIdx.x < kRwWarps * kRwParts) {
+        mbar_init(&sm.full[0][0] + threadIdx.x, (unsigned)Wc);
+        mbar_init(&sm.empty[0][0] + threadIdx.x, 1u);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncthreads();
+    if (warp >= Wc * Rg) return;
     const int rg = warp / Wc, cw = warp - rg * Wc;
 
     asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -160,17 +165,6 @@ rowwise_gemv_kernel(const uint8_t* __restrict__ codes, const unsigned* __restric
     const int blk = (16 * lane) / B, i0 = (16 * lane) % B;
     const int c_lo = cw * 1024 + blk * G + i0;
     const bool live = c_lo < n;  // n is a multiple of G: a lane's block lies wholly inside or outside the row
-    unsigned long long xm[16];
-    float xs = 0.0f;
-#pragma unroll
-    for (int t = 0; t < 16; ++t) {
-        const float xl = live ? __half2float(x[c_lo + t]) : 0.0f;
-        const float xh = live ? __half2float(x[c_lo + t + G / 2]) : 0.0f;
-        xs += xl + xh;
-        // nibble positions of byte t inside its 32-bit word (after the shift by 16 for bytes 2 and 3):
-        // bits 0 and 4 (even byte) or 8 and 12 (odd byte); multiplier = x * 2^(93 - position)
-        xm[t] = (t & 1) ? pack2(xl * 0x1p85f, xh * 0x1p81f) : pack2(xl * 0x1p93f, xh * 0x1p89f);
-    }
     // where this lane copies from (lanes outside the row copy their slice's first bytes and multiply by 0)
     const size_t code_off = (size_t)cw * kRwStep + (live ? (size_t)lane * 16 : 0);
     const int meta_g = (lane < NG && cw * NG + lane < ng) ? cw * NG + lane : cw * NG;
@@ -197,7 +191,46 @@ rowwise_gemv_kernel(const uint8_t* __restrict__ codes, const unsigned* __restric
     int t = (int)blockIdx.x * Rg + rg;
 #pragma unroll
     for (int d = 0; d < D; ++d) issue(t + d * stride, d);
-    int st = 0, buf = 0;
+    // the lane's 32 values of x, as multipliers (the first chunks are on their way meanwhile)
+    unsigned long long xm[16];
+    float xs = 0.0f;
+    {
+        unsigned short xl[16], xh[16];
+        if (live && (reinterpret_cast<uintptr_t>(x) & 15) == 0) {
+            const uint4* pl = reinterpret_cast<const uint4*>(x + c_lo);
+            const uint4* ph = reinterpret_cast<const uint4*>(x + c_lo + G / 2);
+            const uint4 v[4] = {__ldg(pl), __ldg(pl + 1), __ldg(ph), __ldg(ph + 1)};
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const unsigned wl[4] = {v[h].x, v[h].y, v[h].z, v[h].w};
+                const unsigned wh[4] = {v[2 + h].x, v[2 + h].y, v[2 + h].z, v[2 + h].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    xl[8 * h + 2 * e] = (unsigned short)(wl[e] & 0xffffu);
+                    xl[8 * h + 2 * e + 1] = (unsigned short)(wl[e] >> 16);
+                    xh[8 * h + 2 * e] = (unsigned short)(wh[e] & 0xffffu);
+                    xh[8 * h + 2 * e + 1] = (unsigned short)(wh[e] >> 16);
+                }
+            }
+        } else {
+            const unsigned short* xb = reinterpret_cast<const unsigned short*>(x);
+#pragma unroll
+            for (int t = 0; t < 16; ++t) {
+                xl[t] = live ? __ldg(xb + c_lo + t) : (unsigned short)0;
+                xh[t] = live ? __ldg(xb + c_lo + t + G / 2) : (unsigned short)0;
+            }
+        }
+#pragma unroll
+        for (int t = 0; t < 16; ++t) {
+            const float fl = __half2float(__ushort_as_half(xl[t])), fh = __half2float(__ushort_as_half(xh[t]));
+            xs += fl + fh;
+            // nibble positions of byte t inside its 32-bit word (after the shift by 16 for bytes 2 and 3):
+            // bits 0 and 4 (even byte) or 8 and 12 (odd byte); multiplier = x * 2^(93 - position)
+            xm[t] = (t & 1) ? pack2(fl * 0x1p85f, fh * 0x1p81f) : pack2(fl * 0x1p93f, fh * 0x1p89f);
+        }
+    }
+    int st = 0;
+    unsigned k = 0;  // chunks this row group has finished
     for (; t < chunks; t += stride) {
         cp_async_wait<D - 1>();
         __syncwarp();
@@ -231,16 +264,31 @@ rowwise_gemv_kernel(const uint8_t* __restrict__ codes, const unsigned* __restric
 
         int row_in_chunk;
         const float r = reduce_rows<ROWS>(val, lane, &row_in_chunk);
-        if ((lane & (32 / ROWS - 1)) == 0) sm.part[buf][warp][row_in_chunk] = r;
-        if (Wc > 1) group_barrier(1 + rg, Wc * 32);
-        else __syncwarp();
-        if (cw == 0 && lane < ROWS) {
-            float s = 0.0f;
-            for (int w = 0; w < Wc; ++w) s += sm.part[buf][rg * Wc + w][lane];
-            const int row = t * ROWS + lane;
-            if (row < m) y[row] = __float2half_rn(s);
+        const bool holder = (lane & (32 / ROWS - 1)) == 0;
+        if (Wc == 1) {
+            const int row = t * ROWS + row_in_chunk;
+            if (holder && row < m) y[row] = __float2half_rn(r);
+            continue;
         }
-        buf ^= 1;
+        // hand the warp's sums to the row group's first warp through a ring of kRwParts chunks: nobody
+        // waits for the slowest warp of a chunk except the one that adds them up
+        const unsigned b = k % kRwParts, ph = (k / kRwParts) & 1u;
+        if (k >= kRwParts && !mbar_wait(&sm.empty[rg][b], ph ^ 1u)) break;  // (bounded: never hangs)
+        if (holder) sm.part[b][warp][row_in_chunk] = r;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sm.full[rg][b]);
+        if (cw == 0) {
+            if (!mbar_wait(&sm.full[rg][b], ph)) break;
+            if (lane < ROWS) {
+                float s = 0.0f;
+                for (int w = 0; w < Wc; ++w) s += sm.part[b][rg * Wc + w][lane];
+                const int row = t * ROWS + lane;
+                if (row < m) y[row] = __float2half_rn(s);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.empty[rg][b]);
+        }
+        ++k;
     }
     cp_async_wait<0>();
 }

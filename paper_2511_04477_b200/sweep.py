@@ -145,7 +145,8 @@ def format_sweep(peak, shapes=None, formats=None):
 
 def dense_shape_sweep(peak):
     """The dense zigzag GEMV on the paper's 15 shapes m in {2048, 4096, 8192} x k in {1024 ... 16384}
-    (its hyper-parameter study, Sec. 6), int4 g128, over the CTA counts the autotuner would try."""
+    (its hyper-parameter study, Sec. 6), int4 g128, over the CTA counts the autotuner would try, and the
+    row-wise-layout baseline on the same shapes (the comparison the paper makes there)."""
     out = []
     for m in (2048, 4096, 8192):
         for n in (1024, 2048, 4096, 8192, 16384):
@@ -169,8 +170,22 @@ def dense_shape_sweep(peak):
             row["best_ctas"], row["best_us"] = best
             row["dense_gbs"] = needed_bytes(m, n, n, 4, 128) / best[1] * 1e-3
             row["frac_of_peak"] = row["dense_gbs"] / peak
-            out.append(row)
             del packs
+            # the comparison baseline: the same weights' distribution in the row-wise layout, row-parallel kernel
+            g = torch.Generator(device="cuda")
+            rw = []
+            for c in range(copies):
+                g.manual_seed(c)
+                W = torch.empty((m, n), dtype=torch.float32, device="cuda").normal_(0.0, 0.02, generator=g).half()
+                rw.append(binding.spqt_rowwise_pack(W, 4, 128))
+                del W
+            us_rw, _ = graph_us(lambda i, s: binding.spqt_rowwise_dense_gemv(rw[i % copies], xd, y, stream=s), calls, replays=10)
+            row["rowwise_us"] = us_rw
+            row["rowwise_gbs"] = needed_bytes(m, n, n, 4, 128) / us_rw * 1e-3
+            row["rowwise_frac_of_peak"] = row["rowwise_gbs"] / peak
+            row["zigzag_dense_vs_rowwise"] = us_rw / row["us_ctas_0"]
+            out.append(row)
+            del rw
             torch.cuda.empty_cache()
     return out
 
