@@ -253,3 +253,95 @@ def rowwise_dense_gemv(q, scales, zeros, x, group: int = 128):
     What = s * np.asarray(q, dtype=np.float64) + z
     xv = np.asarray(x, dtype=np.float16).astype(np.float64)
     return What @ xv, np.abs(What) @ np.abs(xv)
+
+
+# ---------------------------------------------------------------- two-level ("K-quant"-style) format
+#
+# The format the paper's implementation builds on (Sec. 2): superblocks of 256 weights split into eight
+# blocks of 32, 4-bit codes, a 6-bit scale and a 6-bit minimum per block, a 16-bit scale and a 16-bit
+# minimum per superblock; here in the zigzag arrangement (a superblock = 256 consecutive ROWS of one
+# column, superblocks stored row-major over (block-row, column), Sec. 4.1.2).  The paper fixes neither the
+# rounding rule nor the bit arrangement inside a superblock; the reading taken (both sides implement it):
+#   per block i of a superblock:  lo_i = min(min_j w_j, 0),  range_i = max_j w_j - lo_i,
+#                                 step_i = range_i / 15,      neg_i = -lo_i                      (fp32)
+#   per superblock:               d = fp16(max_i step_i / 63),  dmin = fp16(max_i neg_i / 63)
+#                                 sc_i = min(rint(step_i / d), 63),  m_i = min(rint(neg_i / dmin), 63)
+#   weight:                       q_j = clamp(rint((w_j + dmin*m_i) / (d*sc_i)), 0, 15)   (0 if d*sc_i == 0)
+#   dequantized:                  What_j = d*sc_i*q_j - dmin*m_i
+# every operation a single IEEE fp32 operation (rint = round to nearest even), so that another
+# implementation of the same steps produces the same bytes.
+# Record of a superblock (G = sub*nsub weights): G/2 bytes of codes (byte i = q_i | q_{i+G/2} << 4), then the
+# 2*nsub six-bit fields sc_0.., m_0.. as a little-endian bit string (field f at bits 6f..6f+5) padded to whole
+# bytes, then d and dmin as little-endian fp16: 128 + 12 + 4 = 144 bytes for sub = 32, nsub = 8.
+
+def kq_record_bytes(sub: int = 32, nsub: int = 8) -> int:
+    return sub * nsub // 2 + (12 * nsub + 7) // 8 + 4
+
+
+def kq_quantize(W, sub: int = 32, nsub: int = 8):
+    """fp16 W[m][n] -> (q uint8[m][n], sc uint8[R][nsub][n], mn uint8[R][nsub][n], d fp16[R][n], dmin fp16[R][n])."""
+    W = np.ascontiguousarray(W, dtype=np.float16)
+    m, n = W.shape
+    G = sub * nsub
+    assert m % G == 0
+    R = m // G
+    f32 = np.float32
+    w = W.astype(f32).reshape(R, nsub, sub, n)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        lo = np.minimum(w.min(axis=2), f32(0)) + f32(0)            # (a zero of either sign counts as +0.0)
+        step = ((w.max(axis=2) - lo).astype(f32) / f32(15)).astype(f32)
+        neg = (-lo).astype(f32)
+        d = (step.max(axis=1) / f32(63)).astype(f32).astype(np.float16)
+        dmin = (neg.max(axis=1) / f32(63)).astype(f32).astype(np.float16)
+        df, dminf = d.astype(f32)[:, None, :], dmin.astype(f32)[:, None, :]
+        sc = np.where(df != 0, np.minimum(np.rint((step / df).astype(f32)), f32(63)), f32(0)).astype(np.uint8)
+        mn = np.where(dminf != 0, np.minimum(np.rint((neg / dminf).astype(f32)), f32(63)), f32(0)).astype(np.uint8)
+        s_eff = (df * sc.astype(f32)).astype(f32)[:, :, None, :]
+        o_eff = (dminf * mn.astype(f32)).astype(f32)[:, :, None, :]
+        quo = ((w + o_eff).astype(f32) / s_eff).astype(f32)
+        q = np.where(s_eff != 0, np.clip(np.rint(quo), f32(0), f32(15)), f32(0)).astype(np.uint8)
+    return q.reshape(m, n), sc, mn, d, dmin
+
+
+def kq_pack(q, sc, mn, d, dmin, sub: int = 32, nsub: int = 8) -> np.ndarray:
+    """The records, uint8[R][n][record bytes] flattened (superblock (r, k) at record index r*n + k)."""
+    G = sub * nsub
+    m, n = q.shape
+    R = m // G
+    nf = (12 * nsub + 7) // 8
+    rec = np.zeros((R, n, kq_record_bytes(sub, nsub)), np.uint8)
+    qb = q.reshape(R, G, n)
+    rec[:, :, :G // 2] = (qb[:, :G // 2, :] | (qb[:, G // 2:, :] << 4)).transpose(0, 2, 1)
+    fields = np.concatenate([sc, mn], axis=1).astype(np.uint64)        # [R][2*nsub][n]
+    bits = np.zeros((R, n), dtype=object)
+    for f in range(2 * nsub):
+        bits = bits + (fields[:, f, :].astype(object) << (6 * f))
+    for b in range(nf):
+        rec[:, :, G // 2 + b] = ((bits >> (8 * b)) & 0xFF).astype(np.uint8)
+    du, mu = np.asarray(d, np.float16).view(np.uint16), np.asarray(dmin, np.float16).view(np.uint16)
+    o = G // 2 + nf
+    rec[:, :, o], rec[:, :, o + 1] = (du & 0xFF).astype(np.uint8), (du >> 8).astype(np.uint8)
+    rec[:, :, o + 2], rec[:, :, o + 3] = (mu & 0xFF).astype(np.uint8), (mu >> 8).astype(np.uint8)
+    return rec.reshape(-1)
+
+
+def kq_dequantize_rows(q, sc, mn, d, dmin, rows, sub: int = 32, nsub: int = 8) -> np.ndarray:
+    """What[rows][n] in float64: d*sc_i*q - dmin*m_i with i the block of the row inside its superblock."""
+    G = sub * nsub
+    rows = np.asarray(rows, dtype=np.int64)
+    r, i = rows // G, (rows % G) // sub
+    s = d.astype(np.float64)[r, :] * sc[r, i, :].astype(np.float64)
+    o = dmin.astype(np.float64)[r, :] * mn[r, i, :].astype(np.float64)
+    return s * q[rows, :].astype(np.float64) - o
+
+
+def kq_gemv(q, sc, mn, d, dmin, x, idx=None, rows=None, sub: int = 32, nsub: int = 8):
+    """y[j] = sum over idx (all columns if None) of What[j][k] * x[k], float64; and the bound sum |What||x|."""
+    m, n = q.shape
+    rows = np.arange(m) if rows is None else np.asarray(rows)
+    What = kq_dequantize_rows(q, sc, mn, d, dmin, rows, sub, nsub)
+    xv = np.asarray(x, dtype=np.float16).astype(np.float64)
+    if idx is not None:
+        idx = np.asarray(idx, dtype=np.int64)
+        What, xv = What[:, idx], xv[idx]
+    return What @ xv, np.abs(What) @ np.abs(xv)

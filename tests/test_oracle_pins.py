@@ -2,6 +2,7 @@
 other than itself -- a hand-worked example, a closed form, a library routine,
 exact integer/rational arithmetic, or an invariant the mathematics fixes."""
 import math
+import os
 from fractions import Fraction
 
 import numpy as np
@@ -504,3 +505,115 @@ def test_rowwise_layout_and_product_exact():
         for k in range(n):
             acc += (Fraction(float(s[j, k // G])) * int(q[j, k]) + Fraction(float(z[j, k // G]))) * Fraction(float(x[k]))
         assert abs(float(acc) - y[j]) <= 1e-12 * max(1.0, abs(float(acc)))
+
+
+# ---------------------------------------------------------------- two-level format (Sec. 2: 6-bit block scales/minimums)
+
+def _golden_kq():
+    out = {}
+    with open(os.path.join(os.path.dirname(__file__), "golden", "kq_superblock.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            key, *vals = line.split()
+            out[key] = vals
+    return out
+
+
+def test_kq_hand_worked_superblock():
+    g = _golden_kq()
+    W = np.array([float(v) for v in g["w"]], dtype=np.float16).reshape(8, 1)
+    q, sc, mn, d, dmin = oracle.kq_quantize(W, 4, 2)
+    assert q.ravel().tolist() == [int(v) for v in g["q"]]
+    assert sc.ravel().tolist() == [int(v) for v in g["sc"]] and mn.ravel().tolist() == [int(v) for v in g["m"]]
+    assert int(d.view(np.uint16)[0, 0]) == int(g["d_bits"][0], 16) and int(dmin.view(np.uint16)[0, 0]) == int(g["dmin_bits"][0], 16)
+    assert oracle.kq_pack(q, sc, mn, d, dmin, 4, 2).tolist() == [int(v, 16) for v in g["record"]]
+    assert oracle.kq_record_bytes(4, 2) == 11 and oracle.kq_record_bytes() == 144
+    What = oracle.kq_dequantize_rows(q, sc, mn, d, dmin, np.arange(8), 4, 2).ravel()
+    assert What.tolist() == [float(v) for v in g["dequantized"]]
+    y, bound = oracle.kq_gemv(q, sc, mn, d, dmin, np.array([2.0], np.float16), sub=4, nsub=2)
+    assert y.tolist() == [2 * float(v) for v in g["dequantized"]] and bound.tolist() == [2 * abs(float(v)) for v in g["dequantized"]]
+
+
+def test_kq_quantizer_against_a_scalar_restatement():
+    f32 = np.float32
+    rng = np.random.default_rng(21)
+    sub, nsub, n = 4, 3, 7
+    W = (rng.standard_normal((2 * sub * nsub, n)) * 0.3).astype(np.float16)
+    W[:sub, 0] = np.float16(0.25)                  # a constant positive block: minimum field 0
+    W[:, 1] = np.float16(0.0)                      # an all-zero superblock column (both superblocks)
+    W[sub:2 * sub, 2] = -np.abs(W[sub:2 * sub, 2])  # an all-negative block
+    q, sc, mn, d, dmin = oracle.kq_quantize(W, sub, nsub)
+    G = sub * nsub
+    for r in range(2):
+        for k in range(n):
+            blocks = [W[r * G + i * sub: r * G + (i + 1) * sub, k].astype(f32) for i in range(nsub)]
+            lo = [min(f32(b.min()), f32(0)) for b in blocks]
+            step = [f32(f32(b.max()) - l) / f32(15) for b, l in zip(blocks, lo)]
+            neg = [f32(-l) for l in lo]
+            dd = np.float16(f32(max(step)) / f32(63))
+            dm = np.float16(f32(max(neg)) / f32(63))
+            assert d[r, k] == dd and dmin[r, k] == dm
+            for i in range(nsub):
+                s_i = int(min(np.rint(step[i] / f32(dd)), 63)) if f32(dd) != 0 else 0
+                m_i = int(min(np.rint(neg[i] / f32(dm)), 63)) if f32(dm) != 0 else 0
+                assert sc[r, i, k] == s_i and mn[r, i, k] == m_i
+                se, oe = f32(dd) * f32(s_i), f32(dm) * f32(m_i)
+                for j in range(sub):
+                    want = int(np.clip(np.rint(f32(blocks[i][j] + oe) / se), 0, 15)) if se != 0 else 0
+                    assert q[r * G + i * sub + j, k] == want
+    assert not q[:, 1].any() and not sc[:, :, 1].any() and float(d[0, 1]) == 0.0
+    assert mn[0, 0, 0] == 0 and mn[0, 1, 2] > 0
+
+
+def test_kq_error_bound_scaling_and_fields():
+    rng = np.random.default_rng(22)
+    m, n = 512, 40
+    W = (rng.standard_normal((m, n)) * 0.02).astype(np.float16)
+    q, sc, mn, d, dmin = oracle.kq_quantize(W)
+    assert q.max() <= 15 and sc.max() <= 63 and mn.max() <= 63 and sc.max() == 63 and mn.max() == 63
+    What = oracle.kq_dequantize_rows(q, sc, mn, d, dmin, np.arange(m))
+    w = W.astype(np.float64).reshape(2, 8, 32, n)
+    lo = np.minimum(w.min(axis=2), 0.0)
+    rng_i = w.max(axis=2) - lo
+    s_eff = d.astype(np.float64)[:, None, :] * sc
+    o_eff = dmin.astype(np.float64)[:, None, :] * mn
+    # half a step, plus what the 6-bit rounding of the step and of the minimum can add at the ends of the range
+    lim = s_eff / 2 + np.abs(rng_i - 15 * s_eff) + np.abs(o_eff + lo) + 1e-7
+    err = np.abs(What.reshape(2, 8, 32, n) - w)
+    assert np.all(err <= lim[:, :, None, :])
+    assert np.median(err / np.maximum(s_eff[:, :, None, :], 1e-12)) < 0.3
+    # scaling W by a power of two scales d and dmin and leaves every integer field alone
+    q2, sc2, mn2, d2, dmin2 = oracle.kq_quantize((W.astype(np.float32) * 4).astype(np.float16))
+    assert np.array_equal(q, q2) and np.array_equal(sc, sc2) and np.array_equal(mn, mn2)
+    assert np.array_equal(d2.astype(np.float32), d.astype(np.float32) * 4) and np.array_equal(dmin2.astype(np.float32), dmin.astype(np.float32) * 4)
+    # the record: codes, then the sixteen 6-bit fields as a little-endian bit string, then d and dmin
+    rec = oracle.kq_pack(q, sc, mn, d, dmin).reshape(2, n, 144)
+    for (r, k) in [(0, 0), (1, 17), (1, 39)]:
+        b = rec[r, k]
+        for i in range(128):
+            assert b[i] == (q[r * 256 + i, k] | (q[r * 256 + 128 + i, k] << 4))
+        bits = int.from_bytes(bytes(b[128:140].tolist()), "little")
+        assert [(bits >> (6 * f)) & 63 for f in range(16)] == sc[r, :, k].tolist() + mn[r, :, k].tolist()
+        assert int.from_bytes(bytes(b[140:142].tolist()), "little") == int(d.view(np.uint16)[r, k])
+        assert int.from_bytes(bytes(b[142:144].tolist()), "little") == int(dmin.view(np.uint16)[r, k])
+
+
+def test_kq_product_in_exact_rationals_and_over_a_list():
+    from fractions import Fraction
+    rng = np.random.default_rng(23)
+    sub, nsub, n = 4, 2, 9
+    W = (rng.standard_normal((16, n)) * 0.2).astype(np.float16)
+    x = (rng.standard_normal(n)).astype(np.float16)
+    q, sc, mn, d, dmin = oracle.kq_quantize(W, sub, nsub)
+    idx = np.array([7, 0, 3], dtype=np.int32)
+    y, bound = oracle.kq_gemv(q, sc, mn, d, dmin, x, idx, sub=sub, nsub=nsub)
+    yd, _ = oracle.kq_gemv(q, sc, mn, d, dmin, x, sub=sub, nsub=nsub)
+    for j in range(16):
+        r, i = j // 8, (j % 8) // sub
+        def wh(k):
+            return Fraction(float(d[r, k])) * int(sc[r, i, k]) * int(q[j, k]) - Fraction(float(dmin[r, k])) * int(mn[r, i, k])
+        acc = sum((wh(int(k)) * Fraction(float(x[k])) for k in idx), Fraction(0))
+        accd = sum((wh(k) * Fraction(float(x[k])) for k in range(n)), Fraction(0))
+        ab = sum((abs(wh(int(k))) * abs(Fraction(float(x[k]))) for k in idx), Fraction(0))
+        assert abs(float(acc) - y[j]) <= 1e-12 and abs(float(accd) - yd[j]) <= 1e-12 and abs(float(ab) - bound[j]) <= 1e-12
