@@ -275,6 +275,42 @@ spqt_status spqt_rowwise_dense_gemv(const void* codes, const void* scale_zero,
                                     const void* x, void* y, void* stream);
 
 /*
+ * The two-level format the paper's implementation builds on (paper Sec. 2: superblocks of 256 weights
+ * split into eight blocks of 32, 4-bit codes, a 6-bit scale and a 6-bit minimum per block, a 16-bit scale
+ * and minimum per superblock), in the zigzag arrangement of Sec. 4.1.2: a superblock is 256 consecutive
+ * ROWS of one column; superblock (r, k) is record r*n + k.  A record is 144 bytes:
+ *   bytes 0..127   codes, byte i = q_i | q_{i+128} << 4            (rows r*256 + i and r*256 + 128 + i)
+ *   bytes 128..139 the sixteen 6-bit fields sc_0..sc_7, m_0..m_7 as a little-endian bit string
+ *                  (field f at bits 6f..6f+5)
+ *   bytes 140..143 d, dmin: fp16, little-endian
+ * and row j of block i (rows 32i..32i+31 of the superblock) dequantizes to  d*sc_i*q_j - dmin*m_i.
+ * The paper states neither the rounding rule nor the bit arrangement; the rule implemented (every step
+ * one IEEE fp32 operation, rint = round to nearest even, zeros of either sign count as +0.0):
+ *   lo_i = min(min_j w_j, 0), step_i = (max_j w_j - lo_i)/15, neg_i = 0 - lo_i;
+ *   d = fp16(max_i step_i/63), dmin = fp16(max_i neg_i/63);
+ *   sc_i = min(rint(step_i/d), 63), m_i = min(rint(neg_i/dmin), 63)   (0 when the divisor is 0);
+ *   q_j = clamp(rint((w_j + dmin*m_i)/(d*sc_i)), 0, 15)                 (0 when d*sc_i is 0).
+ * m must be a multiple of 256 (SPQT_ERR_UNSUPPORTED otherwise); any n >= 1.
+ *   spqt_kq_packed_sizes : bytes of the records (144*n*m/256) and of the GEMV workspace; host only.
+ *   spqt_kq_pack         : W fp16 row-major [m][ldw >= n] (2-byte aligned) -> records (16-byte aligned).
+ *   spqt_kq_sparse_gemv  : y[j] = sum_{i < *count} What[j][idx[i]] * x[idx[i]]; idx, count as written by
+ *                          spqt_sparsify (any order of distinct in-range columns; trusted); x fp16[n],
+ *                          y fp16[m] (2-byte aligned).
+ *   spqt_kq_dense_gemv   : the same over all n columns.
+ *   workspace : workspace_bytes of device memory, 16-byte aligned, zeroed ONCE by the caller; every call
+ *               leaves it ready for the next (SPQT_ERR_WORKSPACE if too small).  Sums are added in a fixed
+ *               order: calls are bit-reproducible.
+ * All device pointers; asynchronous on `stream`; nothing is allocated or retained.
+ */
+spqt_status spqt_kq_packed_sizes(int m, int n, size_t* records_bytes, size_t* workspace_bytes);
+spqt_status spqt_kq_pack(const void* W, int m, int n, int ldw, void* records, void* stream);
+spqt_status spqt_kq_sparse_gemv(const void* records, int m, int n, const void* x,
+                                const int32_t* idx, const int32_t* count, void* y,
+                                void* workspace, size_t workspace_bytes, void* stream);
+spqt_status spqt_kq_dense_gemv(const void* records, int m, int n, const void* x, void* y,
+                               void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Threshold calibration (paper Sec. 5, the calibration threshold tool; Sec. 3.2: thresholds are
  * computed once per sparsity level from calibration activations).  *threshold (a device float) =
  * the nearest-rank order statistic of |x| over the pool x[0:count] of fp16 calibration activations:

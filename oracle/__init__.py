@@ -263,7 +263,8 @@ def rowwise_dense_gemv(q, scales, zeros, x, group: int = 128):
 # column, superblocks stored row-major over (block-row, column), Sec. 4.1.2).  The paper fixes neither the
 # rounding rule nor the bit arrangement inside a superblock; the reading taken (both sides implement it):
 #   per block i of a superblock:  lo_i = min(min_j w_j, 0),  range_i = max_j w_j - lo_i,
-#                                 step_i = range_i / 15,      neg_i = -lo_i                      (fp32)
+#                                 step_i = range_i / 15,      neg_i = 0 - lo_i                   (fp32;
+#                                 zeros of either sign count as +0.0)
 #   per superblock:               d = fp16(max_i step_i / 63),  dmin = fp16(max_i neg_i / 63)
 #                                 sc_i = min(rint(step_i / d), 63),  m_i = min(rint(neg_i / dmin), 63)
 #   weight:                       q_j = clamp(rint((w_j + dmin*m_i) / (d*sc_i)), 0, 15)   (0 if d*sc_i == 0)
@@ -289,8 +290,9 @@ def kq_quantize(W, sub: int = 32, nsub: int = 8):
     w = W.astype(f32).reshape(R, nsub, sub, n)
     with np.errstate(divide="ignore", invalid="ignore"):
         lo = np.minimum(w.min(axis=2), f32(0)) + f32(0)            # (a zero of either sign counts as +0.0)
-        step = ((w.max(axis=2) - lo).astype(f32) / f32(15)).astype(f32)
-        neg = (-lo).astype(f32)
+        hi = w.max(axis=2) + f32(0)
+        step = ((hi - lo).astype(f32) / f32(15)).astype(f32)
+        neg = (f32(0) - lo).astype(f32)                            # (0 - 0 is +0.0)
         d = (step.max(axis=1) / f32(63)).astype(f32).astype(np.float16)
         dmin = (neg.max(axis=1) / f32(63)).astype(f32).astype(np.float16)
         df, dminf = d.astype(f32)[:, None, :], dmin.astype(f32)[:, None, :]

@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libspqt.so")
 EXPORTS = (
     "spqt_status_string", "spqt_version", "spqt_packed_sizes", "spqt_pack", "spqt_unpack",
     "spqt_sparsify", "spqt_sparse_gemv", "spqt_sparse_gemv_static", "spqt_static_status", "spqt_sparsify_gemv", "spqt_dense_gemv",
-    "spqt_sparse_linear_host", "spqt_gemm_small_workspace", "spqt_sparse_gemm_small", "spqt_dense_gemm_small", "spqt_rowwise_packed_sizes", "spqt_rowwise_pack", "spqt_rowwise_dense_gemv", "spqt_autotune", "spqt_calibrate_threshold", "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_launch_count",
+    "spqt_sparse_linear_host", "spqt_gemm_small_workspace", "spqt_sparse_gemm_small", "spqt_dense_gemm_small", "spqt_rowwise_packed_sizes", "spqt_rowwise_pack", "spqt_rowwise_dense_gemv", "spqt_kq_packed_sizes", "spqt_kq_pack", "spqt_kq_sparse_gemv", "spqt_kq_dense_gemv", "spqt_autotune", "spqt_calibrate_threshold", "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_launch_count",
 )
 
 _lib = None
@@ -60,6 +60,10 @@ def lib() -> ctypes.CDLL:
         L.spqt_rowwise_packed_sizes.argtypes = [i32, i32, i32, i32] + [ctypes.POINTER(sz)] * 2
         L.spqt_rowwise_pack.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp]
         L.spqt_rowwise_dense_gemv.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp]
+        L.spqt_kq_packed_sizes.argtypes = [i32, i32] + [ctypes.POINTER(sz)] * 2
+        L.spqt_kq_pack.argtypes = [vp, i32, i32, i32, vp, vp]
+        L.spqt_kq_sparse_gemv.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, sz, vp]
+        L.spqt_kq_dense_gemv.argtypes = [vp, i32, i32, vp, vp, vp, sz, vp]
         L.spqt_sparse_linear_host.argtypes = [vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, vp,
                                               vp, vp, vp, vp, vp, sz, vp]
         L.spqt_gemm_small_workspace.argtypes = [i32, i32, i32, i32, ctypes.POINTER(sz)]
@@ -382,6 +386,58 @@ def spqt_rowwise_dense_gemv(p: RowwisePacked, x: torch.Tensor, y: torch.Tensor =
     _ok(lib().spqt_rowwise_dense_gemv(
         _dev(p.codes, torch.uint8, "codes"), _dev(p.scale_zero, torch.float16, "scale_zero"), p.m, p.n, p.bits, p.group,
         _dev(x, torch.float16, "x"), _dev(y, torch.float16, "y"), _stream(stream)), "spqt_rowwise_dense_gemv")
+    return y
+
+
+@dataclass
+class KqPacked:
+    """Device buffer written by :func:`spqt_kq_pack` (144-byte records of the two-level format, zigzag order)."""
+    records: torch.Tensor      # uint8[(m/256)*n*144]
+    m: int
+    n: int
+
+
+def spqt_kq_packed_sizes(m: int, n: int):
+    out = [ctypes.c_size_t(0) for _ in range(2)]
+    _ok(lib().spqt_kq_packed_sizes(m, n, *[ctypes.byref(o) for o in out]), "spqt_kq_packed_sizes")
+    return int(out[0].value), int(out[1].value)
+
+
+def spqt_kq_pack(W: torch.Tensor, stream=None) -> KqPacked:
+    if W.dim() != 2 or W.stride(1) != 1:
+        raise ValueError("W must be 2-D with unit column stride")
+    if not W.is_cuda or W.dtype != torch.float16:
+        raise TypeError("W must be a CUDA float16 tensor")
+    m, n = W.shape
+    rb, _ = spqt_kq_packed_sizes(m, n)
+    records = torch.empty(rb, dtype=torch.uint8, device=W.device)
+    _ok(lib().spqt_kq_pack(W.data_ptr(), m, n, W.stride(0), records.data_ptr(), _stream(stream)), "spqt_kq_pack")
+    return KqPacked(records, m, n)
+
+
+def new_kq_workspace(p: KqPacked) -> torch.Tensor:
+    """Zeroed GEMV workspace for the two-level format (zeroed once; every call leaves it ready for the next)."""
+    _, wb = spqt_kq_packed_sizes(p.m, p.n)
+    return torch.zeros(wb, dtype=torch.uint8, device=p.records.device)
+
+
+def spqt_kq_sparse_gemv(p: KqPacked, x: torch.Tensor, idx: torch.Tensor, count: torch.Tensor, workspace: torch.Tensor,
+                        y: torch.Tensor = None, stream=None) -> torch.Tensor:
+    if y is None:
+        y = torch.empty(p.m, dtype=torch.float16, device=x.device)
+    _ok(lib().spqt_kq_sparse_gemv(
+        _dev(p.records, torch.uint8, "records"), p.m, p.n, _dev(x, torch.float16, "x"), _dev(idx, torch.int32, "idx"),
+        _dev(count, torch.int32, "count"), _dev(y, torch.float16, "y"), _dev(workspace, torch.uint8, "workspace"),
+        workspace.numel(), _stream(stream)), "spqt_kq_sparse_gemv")
+    return y
+
+
+def spqt_kq_dense_gemv(p: KqPacked, x: torch.Tensor, workspace: torch.Tensor, y: torch.Tensor = None, stream=None) -> torch.Tensor:
+    if y is None:
+        y = torch.empty(p.m, dtype=torch.float16, device=x.device)
+    _ok(lib().spqt_kq_dense_gemv(
+        _dev(p.records, torch.uint8, "records"), p.m, p.n, _dev(x, torch.float16, "x"), _dev(y, torch.float16, "y"),
+        _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)), "spqt_kq_dense_gemv")
     return y
 
 

@@ -902,3 +902,73 @@ def test_rowwise_baseline_refuses_what_it_does_not_cover():
     assert L.spqt_rowwise_dense_gemv(a, a, 8, 16384 + 128, 4, 128, a, a, None) == 2
     assert L.spqt_rowwise_dense_gemv(a, a, 8, 128, 4, 128, None, a, None) == 1
     assert L.spqt_rowwise_dense_gemv(a + 4, a, 8, 128, 4, 128, a, a, None) == 3
+
+
+# ---------------------------------------------------------------- two-level format (6-bit block scales and minimums)
+
+@pytest.mark.parametrize("m_blocks,n", [(1, 1), (1, 300), (2, 1111), (16, 4096), (4, 14336), (56, 1024)])
+def test_kq_pack_bytes_and_products_match_the_oracle(m_blocks, n):
+    m = 256 * m_blocks
+    W = inputs.weights(m, n, seed=9 * m_blocks + n)
+    if n >= 300:
+        W[:32, 0] = np.abs(W[:32, 0])                     # a block without negative weights: minimum field 0
+        W[:256, 1] = np.float16(0.0)                      # an all-zero superblock
+        W[:256, 2] = np.float16(-0.0)
+        W[32:64, 3] = np.float16(0.125)                   # a constant block
+    x = inputs.activations(n, seed=m_blocks + 70, dist="gauss" if n > 8192 else "laplace")
+    q, sc, mn, d, dmin = oracle.kq_quantize(W)
+    p = binding.spqt_kq_pack(dev(W))
+    torch.cuda.synchronize()
+    got = p.records.cpu().numpy()
+    want = oracle.kq_pack(q, sc, mn, d, dmin)
+    assert np.array_equal(got, want), "first differing byte %d" % int(np.nonzero(got != want)[0][0])
+    ws = binding.new_kq_workspace(p)
+    xd = dev(x)
+    for sp in (0.5, 0.9, 0.0, None):
+        t = float("inf") if sp is None else inputs.threshold_for_sparsity(x, sp)
+        idx, cnt = binding.spqt_sparsify(xd, t)
+        y = torch.full((m,), float("nan"), dtype=torch.float16, device="cuda")
+        binding.spqt_kq_sparse_gemv(p, xd, idx, cnt, ws, y)
+        torch.cuda.synchronize()
+        c = int(cnt.item())
+        y_ref, bound = oracle.kq_gemv(q, sc, mn, d, dmin, x, idx.cpu().numpy()[:c])
+        check_y(y.cpu().numpy(), y_ref, bound, "two-level sparse, sparsity %r" % sp)
+        y2 = binding.spqt_kq_sparse_gemv(p, xd, idx, cnt, ws)
+        torch.cuda.synchronize()
+        assert torch.equal(y.view(torch.int16), y2.view(torch.int16))           # fixed order of sums
+    yd = binding.spqt_kq_dense_gemv(p, xd, ws)
+    torch.cuda.synchronize()
+    y_ref, bound = oracle.kq_gemv(q, sc, mn, d, dmin, x)
+    check_y(yd.cpu().numpy(), y_ref, bound, "two-level dense")
+    assert not ws[: 4 * m_blocks].any()                                        # arrival counters back at zero
+
+
+def test_kq_llama_shape_on_sampled_rows_and_a_shuffled_list():
+    m, n = 14336, 4096
+    W = inputs.weights(m, n, seed=77)
+    x = inputs.activations(n, seed=78)
+    q, sc, mn, d, dmin = oracle.kq_quantize(W)
+    p = binding.spqt_kq_pack(dev(W))
+    ws = binding.new_kq_workspace(p)
+    t = inputs.threshold_for_sparsity(x, 0.5)
+    xd = dev(x)
+    idx, cnt = binding.spqt_sparsify(xd, t)
+    torch.cuda.synchronize()
+    c = int(cnt.item())
+    perm = np.random.Generator(np.random.PCG64(5)).permutation(c)
+    idx[:c] = idx[:c][torch.from_numpy(perm).cuda()]
+    y = binding.spqt_kq_sparse_gemv(p, xd, idx, cnt, ws)
+    torch.cuda.synchronize()
+    rows = np.unique(np.random.Generator(np.random.PCG64(6)).integers(0, m, size=256))
+    y_ref, bound = oracle.kq_gemv(q, sc, mn, d, dmin, x, idx.cpu().numpy()[:c], rows=rows)
+    check_y(y.cpu().numpy()[rows], y_ref, bound, "two-level 14336x4096")
+
+
+def test_kq_refuses_what_it_does_not_cover():
+    L = binding.lib()
+    buf = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    a = buf.data_ptr()
+    assert L.spqt_kq_pack(a, 128, 8, 8, a, None) == 2                        # m not a multiple of 256
+    assert L.spqt_kq_dense_gemv(a, 256, 8, a, a, a, 16, None) == 4           # workspace too small
+    assert L.spqt_kq_sparse_gemv(a, 256, 8, a, None, a, a, a, 1 << 16, None) == 1
+    assert L.spqt_kq_dense_gemv(a + 8, 256, 8, a, a, a, 1 << 16, None) == 3
