@@ -2,7 +2,7 @@
 """Benchmark of the SpQt hot path on B200: one line of JSON on stdout.
 
     python bench.py [--gpus N] [--steps K] [--warmup W]            the headline line (config "layer")
-    python bench.py --config sweep | formats | dense | batch | stack   the other workloads, one JSON line each
+    python bench.py --config sweep | formats | dense | batch | kquant | stack   the other workloads, one JSON line each
     python bench.py --impl reference                               the fp64 CPU oracle on a bounded sample
 
 Workload of the headline line (the configuration the metric is quoted on): the seven linear layers of
@@ -246,6 +246,16 @@ def other_config_line(which, local, quick=False):
                                             "and the built-in rule; beside it the row-wise-layout baseline (spqt_rowwise_dense_gemv) on the same shapes; rotated weight copies > 2x L2"},
                         roofline=roofline_obj(best["dense_gbs"], peak, kind, nb, best["best_us"], "gemv_kernel<128,4,dense>", 1.0),
                         zigzag_dense_vs_rowwise={"%dx%d" % (r["m"], r["n"]): r["zigzag_dense_vs_rowwise"] for r in rows},
+                        rows=rows)
+        elif which == "kquant":
+            rows = sweep.kq_sweep(peak)
+            r0 = [r for r in rows if r["m"] == 28672 and r["n"] == 8192][0]
+            nb = r0["sparse_gbs"] * r0["sparse_us"] * 1e3
+            line = dict(base, metric="sparse GEMV over the two-level format (256-row superblocks, 6-bit block scales and minimums), effective HBM GB/s at 50% sparsity, 28672x8192",
+                        value=r0["sparse_gbs"], ms_per_step=r0["sparse_us"] * 1e-3, steps=20, warmup=4,
+                        config={"workload": "two-level format in the zigzag arrangement, 144-byte records; index list given (and, beside it, collected by a launch of its own); "
+                                            "50% sparsity; Llama-3-8B-shaped linears and 28672x8192; rotated weight copies > 2x L2"},
+                        roofline=roofline_obj(r0["sparse_gbs"], peak, kind, nb, r0["sparse_us"], "kq_gemv_kernel", None),
                         rows=rows)
         elif which == "batch":
             rows = sweep.batch_sweep(peak)
@@ -604,7 +614,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1024)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="layer", choices=["layer", "sweep", "formats", "dense", "batch", "stack"])
+    ap.add_argument("--config", default="layer", choices=["layer", "sweep", "formats", "dense", "batch", "kquant", "stack"])
     ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_S,
                     help="device time to accumulate over repeated K-step regions of the headline measurement")
     ap.add_argument("--quick", action="store_true", help="reduced form of --config sweep/formats/stack")

@@ -214,15 +214,21 @@ kq_gemv_kernel(const uint8_t* __restrict__ records, int n, const __half* __restr
             }
             __syncwarp();
             const int valid = min(CH, hi - pos);
-            const int nsub = (valid + 1) >> 1;
             const unsigned cb = rbuf + cur;
-#pragma unroll 1
-            for (int u = 0; u < nsub; ++u) {
+            auto step = [&](int u) {
                 const unsigned e = (unsigned)(2 * u + half);
                 const uint2 wv = lds_v2(cb + e * kKqRec + (unsigned)t * 8u);
                 unsigned long long m01, m23;
                 lds_pairs(mbuf + 16u * (e * 4u + (unsigned)(t >> 2)), m01, m23);
                 fma_block8(acc, wv, m01, m23);
+            };
+            if (valid == CH) {
+#pragma unroll
+                for (int u = 0; u < CH / 2; ++u) step(u);   // a full chunk: straight-line code
+            } else {
+                const int nsub = (valid + 1) >> 1;
+#pragma unroll 1
+                for (int u = 0; u < nsub; ++u) step(u);
             }
             __syncwarp();
             cur = (cur == 0u) ? kBufBytes : 0u;

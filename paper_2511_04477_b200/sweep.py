@@ -190,6 +190,48 @@ def dense_shape_sweep(peak):
     return out
 
 
+def kq_sweep(peak):
+    """The two-level format (144-byte records of 256 rows of a column): the index collection followed by the
+    sparse product over the list at 50 %, the product alone, and the dense product, on Llama-3-8B-shaped linears
+    and one Llama-2-70B-shaped one.  Needed bytes per active superblock: 144."""
+    out = []
+    for (m, n, dist) in [(4096, 4096, "laplace"), (6144, 4096, "laplace"), (28672, 4096, "laplace"), (4096, 14336, "gauss"),
+                         (28672, 8192, "laplace")]:
+        R = m // 256
+        copies = int(min(64, max(4, math.ceil(2.4 * L2_BYTES / (R * n * 144)))))
+        g = torch.Generator(device="cuda")
+        packs = []
+        for c in range(copies):
+            g.manual_seed(c)
+            W = torch.empty((m, n), dtype=torch.float32, device="cuda").normal_(0.0, 0.02, generator=g).half()
+            packs.append(binding.spqt_kq_pack(W))
+            del W
+        x = inputs.activations(n, seed=21, dist=dist)
+        t = inputs.threshold_for_sparsity(x, 0.5)
+        xd = torch.from_numpy(x).cuda()
+        ws = binding.new_kq_workspace(packs[0])
+        idx, cnt = binding.spqt_sparsify(xd, t)
+        torch.cuda.synchronize()
+        count = int(cnt.item())
+        y = torch.empty(m, dtype=torch.float16, device="cuda")
+        calls = max(copies, 16)
+
+        def both(i, s):
+            binding.spqt_sparsify(xd, t, idx, cnt, stream=s)
+            binding.spqt_kq_sparse_gemv(packs[i % copies], xd, idx, cnt, ws, y, stream=s)
+        us_both, _ = graph_us(both, calls)
+        us_sp, _ = graph_us(lambda i, s: binding.spqt_kq_sparse_gemv(packs[i % copies], xd, idx, cnt, ws, y, stream=s), calls)
+        us_de, _ = graph_us(lambda i, s: binding.spqt_kq_dense_gemv(packs[i % copies], xd, ws, y, stream=s), calls)
+        nb = lambda c: c * R * 144 + 2 * n + 4 * c + 4 + 2 * m
+        out.append({"m": m, "n": n, "count": count, "copies": copies, "sparsify_plus_sparse_us": us_both, "sparse_us": us_sp,
+                    "dense_us": us_de, "sparse_gbs": nb(count) / us_sp * 1e-3, "frac_of_peak": nb(count) / us_sp * 1e-3 / peak,
+                    "dense_gbs": nb(n) / us_de * 1e-3, "dense_frac_of_peak": nb(n) / us_de * 1e-3 / peak,
+                    "speedup_vs_dense": us_de / us_sp, "speedup_vs_dense_with_index_collection": us_de / us_both})
+        del packs
+        torch.cuda.empty_cache()
+    return out
+
+
 def batch_sweep(peak):
     """Small batches (1, 2, 4, 8 rows) on the stacked gate|up matrix and the down projection, int4 g128: rows that
     are independent draws (their union is 1 - 2^-B dense at 50 % each) and rows that share most of their
