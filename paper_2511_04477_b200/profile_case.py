@@ -1,10 +1,12 @@
 """Run one sparse and one dense GEMV a few times on a single packed matrix, with L2 flushed
 before every call -- a small, self-terminating case for `ncu` captures.
 
-    python -m paper_2511_04477_b200.profile_case M N SPARSITY [GROUP] [REPEATS] [fused|pack|sparsify]
+    python -m paper_2511_04477_b200.profile_case M N SPARSITY [GROUP] [REPEATS] [fused|pack|sparsify|rowwise|kq|batch4]
 
 With `fused` the sparse call is the one that collects the indices in the same launch; with `pack` only the
-offline conversion is repeated, with `sparsify` only the index collection (L2 flushed before each as well).
+offline conversion is repeated, with `sparsify` only the index collection (L2 flushed before each as well);
+`rowwise` = the row-wise baseline's dense GEMV, `kq` = the two-level format's sparse and dense GEMV, `batch4` = four
+beam-like rows over the union of their active sets and the dense batch call.
 
 Weights are random-init on the device (values do not affect timing); x and the threshold come
 from the seeded input module.  Prints the active count and the workspace status word.
@@ -26,7 +28,49 @@ def main(argv):
     fused = mode == "fused"
     torch.manual_seed(0)
     W = (torch.randn(m, n, device="cuda", dtype=torch.float32) * 0.02).half()
+    if mode in ("rowwise", "kq"):
+        x = inputs.activations(n, seed=1)
+        xd = torch.from_numpy(x).cuda()
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        if mode == "rowwise":
+            p = binding.spqt_rowwise_pack(W, 4, group)
+            del W
+            for _ in range(repeats):
+                flush.zero_()
+                binding.spqt_rowwise_dense_gemv(p, xd)
+            torch.cuda.synchronize()
+            print("ok rowwise")
+            return
+        p = binding.spqt_kq_pack(W)
+        del W
+        ws = binding.new_kq_workspace(p)
+        idx, cnt = binding.spqt_sparsify(xd, inputs.threshold_for_sparsity(x, sp))
+        for _ in range(repeats):
+            flush.zero_()
+            binding.spqt_kq_sparse_gemv(p, xd, idx, cnt, ws)
+            flush.zero_()
+            binding.spqt_kq_dense_gemv(p, xd, ws)
+        torch.cuda.synchronize()
+        print("ok kq count=%d" % int(cnt.item()))
+        return
     p = binding.spqt_pack(W, 4, group)
+    if mode == "batch4":
+        import numpy as np
+        del W
+        base = inputs.activations(n, seed=31).astype(np.float32)
+        X = np.stack([(base + 0.2 * inputs.activations(n, seed=60 + b).astype(np.float32)).astype(np.float16) for b in range(4)])
+        Xd = torch.from_numpy(X).cuda()
+        t = inputs.threshold_for_sparsity(X[0], sp)
+        ws = binding.new_gemm_small_workspace(p)
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        for _ in range(repeats):
+            flush.zero_()
+            Y, idx, cnt = binding.spqt_sparse_gemm_small(p, Xd, t, ws)
+            flush.zero_()
+            binding.spqt_dense_gemm_small(p, Xd, ws)
+        torch.cuda.synchronize()
+        print("ok batch4 union count=%d" % int(cnt.item()))
+        return
     if mode == "pack":
         flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
         for _ in range(repeats):
