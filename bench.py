@@ -556,6 +556,17 @@ def run_ours(args):
         st = other_config_line("stack", local, quick=True)
         others["stack_32_layers"] = {k: st["result"][k] for k in ("tokens_per_s", "ms_per_token", "needed_gb_per_token", "needed_gbs",
                                                                     "frac_of_peak", "tokens", "device_status")}
+        de = other_config_line("dense", local)
+        others["rowwise_baseline_us_over_zigzag_dense_us"] = de["zigzag_dense_vs_rowwise"]
+        ba = other_config_line("batch", local)
+        others["small_batch_beam_like_28672x4096"] = {
+            "B=%d" % r["batch"]: {"union_sparsity": r["union_sparsity"], "sparse_us_per_row": r["sparse_us_per_row"],
+                                  "dense_us_per_row": r["dense_us_per_row"], "speedup_vs_dense": r["speedup_vs_dense"]}
+            for r in ba["rows"] if r["m"] == 28672 and r["rows"] == "beam-like"}
+        kq = other_config_line("kquant", local)
+        others["two_level_format_at_50pct"] = {
+            "%dx%d" % (r["m"], r["n"]): {"sparse_frac_of_peak": r["frac_of_peak"], "dense_frac_of_peak": r["dense_frac_of_peak"],
+                                         "speedup_vs_dense": r["speedup_vs_dense"]} for r in kq["rows"]}
 
     if rank == 0:
         cpu = oracle_sample(3, 1) if world >= 1 else None
