@@ -62,7 +62,7 @@ def test_group_sizes_outside_64_and_128_are_refused(hand_example):
 
 # ------------------------------------------------------------------ a2: index collection
 
-@pytest.mark.parametrize("n", [1, 2, 31, 32, 33, 1023, 1024, 1025, 4096, 8192, 14336, 28672, 40000])
+@pytest.mark.parametrize("n", [1, 2, 31, 32, 33, 1023, 1024, 1025, 4096, 8192, 14336, 28672, 40000, 65536, 65537, 100000])
 def test_index_list_is_bit_exact(n):
     x = inputs.activations(n, seed=1000 + n, dist="laplace" if n % 2 == 0 else "gauss")
     if n > 100:
