@@ -104,3 +104,22 @@ def test_bad_arguments_launch_nothing(L):
     assert L.spqt_workspace_status(None, 128, 128, None, None) == 1
     assert L.spqt_static_status(100, 128, None, None) == 1
     assert binding.spqt_launch_count() == before
+
+
+def test_sizes_and_refusals_of_the_rowwise_and_two_level_entries(L):
+    assert binding.spqt_rowwise_packed_sizes(4096, 4096, 4, 128) == (4096 * 4096 // 2, 4096 * 32 * 4)
+    assert binding.spqt_rowwise_packed_sizes(3, 64, 4, 64) == (96, 12)
+    sz = ctypes.c_size_t(0)
+    assert L.spqt_rowwise_packed_sizes(8, 100, 4, 128, ctypes.byref(sz), None) == 2      # n not a multiple of the group
+    assert L.spqt_rowwise_packed_sizes(8, 128, 3, 128, ctypes.byref(sz), None) == 2      # 4-bit only
+    assert L.spqt_rowwise_packed_sizes(0, 128, 4, 128, ctypes.byref(sz), None) == 1
+    rec, ws = binding.spqt_kq_packed_sizes(14336, 4096)
+    assert rec == (14336 // 256) * 4096 * 144 and ws >= 56 * 4 and ws % 16 == 0
+    assert L.spqt_kq_packed_sizes(128, 8, ctypes.byref(sz), None) == 2                   # m not a multiple of 256
+    assert L.spqt_kq_packed_sizes(256, 0, ctypes.byref(sz), None) == 1
+    # null pointers are refused before any launch (no GPU needed to say so)
+    assert L.spqt_rowwise_pack(None, 8, 128, 128, 4, 128, None, None, None) == 1
+    assert L.spqt_rowwise_dense_gemv(None, None, 8, 128, 4, 128, None, None, None) == 1
+    assert L.spqt_kq_pack(None, 256, 8, 8, None, None) == 1
+    assert L.spqt_kq_dense_gemv(None, 256, 8, None, None, None, 0, None) == 1
+    assert L.spqt_kq_sparse_gemv(None, 256, 8, None, None, None, None, None, 0, None) == 1
