@@ -69,4 +69,8 @@ extern int g_no_pdl;          // 1 = launch strictly stream-ordered (spqt_set_tu
 int sm_count();               // SMs of the current device (cached per device); <= 0 on error
 void count_launch(int k = 1); // bump the process-wide launch counter
 
+// Index collection over `batch` rows of X (columns active in at least one row, ascending; n < 2^16), one launch.
+spqt_status launch_sparsify_rows(const __half* X, int ldx, int batch, int n, float t, int32_t* idx, int32_t* count,
+                                 cudaStream_t stream);
+
 }  // namespace spqt

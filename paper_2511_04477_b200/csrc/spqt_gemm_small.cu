@@ -3,8 +3,7 @@
 // batch and its codes are extracted once; only the FMAs are repeated per row, so the byte and the
 // integer-instruction cost per row falls with the batch size.
 //
-//   union_sparsify_kernel   one CTA, ballot/popc compaction like the batch-1 index collection, with
-//                           "active" = |X[b][k]| > t in at least one row b.
+//   sparsify_rows_kernel    (spqt_sparsify.cu) one CTA; "active" = |X[b][k]| > t in at least one row b.
 //   gemm_small_kernel       grid (S, R): CTA (s, r) takes the s-th of S equal slices of the union list
 //                           for block-row r; its 8 warps take the slice's chunks of 32 entries in turn,
 //                           each with two code buffers (the next chunk's copies fly during the
@@ -32,61 +31,12 @@ constexpr int kSmallRows = 4;      // batch rows per pass at most (a pass of one
 constexpr int kSmallMaxSplit = 8;  // slices per block-row at most
 constexpr int kSmallChunk = 32;    // list entries per chunk
 
-__global__ void __launch_bounds__(1024)
-union_sparsify_kernel(const __half* __restrict__ X, int ldx, int batch, int n, float t,
-                      int32_t* __restrict__ idx, int32_t* __restrict__ count)
-{
-    __shared__ int warp_total[32];
-    __shared__ int warp_base[32];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const int seg = ((n + 32 * 32 - 1) / (32 * 32)) * 32;
-    const int begin = min(warp * seg, n), end = min(begin + seg, n);
-    auto active = [&](int k) -> bool {
-        bool on = false;
-        for (int b = 0; b < batch; ++b) on = on || (fabsf(__half2float(X[(size_t)b * ldx + k])) > t);  // NaN: false
-        return on;
-    };
-    // one pass over X: bit `it` of `flags` = this lane's column of the warp's it-th group of 32 is active
-    // (at most 64 groups per warp: n < 2^16); the loads of different groups do not depend on one another
-    unsigned long long flags = 0;
-    const int groups = (end - begin + 31) >> 5;
-#pragma unroll 4
-    for (int it = 0; it < groups; ++it) {
-        const int k = begin + it * 32 + lane;
-        if (k < end && active(k)) flags |= 1ull << it;
-    }
-    int total = __popcll(flags);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
-    if (lane == 0) warp_total[warp] = total;
-    __syncthreads();
-    if (warp == 0) {
-        int v = warp_total[lane], incl = v;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            int up = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += up;
-        }
-        warp_base[lane] = incl - v;
-        if (lane == 31) *count = incl;
-    }
-    __syncthreads();
-    int base = warp_base[warp];
-    for (int it = 0; it < groups; ++it) {
-        const bool p = (flags >> it) & 1ull;
-        const unsigned mask = __ballot_sync(0xffffffffu, p);
-        if (p) idx[base + __popc(mask & ((1u << lane) - 1u))] = begin + it * 32 + lane;
-        base += __popc(mask);
-    }
-}
-
 template <int G, int BITS, int ROWS>
 struct SmallSmem {
     static constexpr int B = G * BITS / 8;
     alignas(16) unsigned char codes[kSmallWarps][2][kSmallChunk * B];
     alignas(16) float mult[kSmallWarps][kSmallChunk][ROWS][4];
+    alignas(16) unsigned ent[kSmallWarps][2][kSmallChunk][ROWS + 1];  // per entry: its (scale, zero) pair and the words holding the rows' x values
     alignas(16) float red[kSmallWarps][ROWS][G];
     float red_z[kSmallWarps][ROWS];
     int last;
@@ -158,14 +108,6 @@ gemm_small_kernel(const uint8_t* __restrict__ codes, const unsigned* __restrict_
         cp_async_commit();
     };
 
-    // lane e's entry of a chunk: its (scale, zero) pair and the batch's x values (0 past the end of the slice)
-    auto load_entry = [&](int pos, int col, unsigned& mz, unsigned short* xb) {
-        const bool on = pos + lane < hi;
-        mz = __ldg(row_meta + col);
-#pragma unroll
-        for (int b = 0; b < ROWS; ++b)
-            xb[b] = (on && b < batch) ? __ldg(reinterpret_cast<const unsigned short*>(X) + (size_t)b * ldx + col) : (unsigned short)0;
-    };
     auto step = [&](unsigned cb, int u) {
         const unsigned ent = (unsigned)(u * SLM + mslot);
         if (BITS == 4) {
@@ -189,55 +131,77 @@ gemm_small_kernel(const uint8_t* __restrict__ codes, const unsigned* __restrict_
         }
     };
 
+    // The (scale, zero) pair and the x values of an entry travel like its codes: asynchronous copies into
+    // shared memory, one chunk ahead (held in registers across a chunk's arithmetic they made the compiler
+    // move the loads next to their use, and every chunk then waited for a round of gathers).  x is fetched as
+    // the aligned 4-byte word that holds the value; without that alignment the values are loaded directly.
+    const bool xw_ok = (reinterpret_cast<uintptr_t>(X) & 3) == 0 && (ldx & 1) == 0;
+    const unsigned ebuf = smem_u32(&sm.ent[warp][0][0][0]);
+    constexpr unsigned kEntBytes = CH * (ROWS + 1) * 4;
+    auto issue_chunk = [&](int col, unsigned which) {
+        const unsigned ed = ebuf + which * kEntBytes + (unsigned)lane * (ROWS + 1) * 4u;
+        cp_async_4(ed, row_meta + col);
+        if (xw_ok) {
+#pragma unroll
+            for (int b = 0; b < ROWS; ++b)
+                if (b < batch) cp_async_4(ed + 4u * (1 + b), reinterpret_cast<const unsigned*>(X + (size_t)b * ldx + (col & ~1)));
+        }
+        copy_codes(col, cbuf + which * kBufBytes);   // (commits the group)
+    };
+
     const int first = lo + warp * CH, stride = kSmallWarps * CH;
     if (first < hi) {
         int col = column_at(first);
-        copy_codes(col, cbuf);
+        issue_chunk(col, 0u);
         int col_next = first + stride < hi ? column_at(first + stride) : 0;
-        unsigned mz;
-        unsigned short xb[ROWS];
-        load_entry(first, col, mz, xb);
         unsigned cur = 0;
         for (int pos = first; pos < hi; pos += stride) {
             const bool more = pos + stride < hi;
-            if (more) copy_codes(col_next, cbuf + (cur == 0u ? kBufBytes : 0u));
+            if (more) issue_chunk(col_next, cur ^ 1u);
             else cp_async_commit();
-            // the loads of the chunks to come, ahead of this chunk's arithmetic
             const int col_after = pos + 2 * stride < hi ? column_at(pos + 2 * stride) : 0;
-            unsigned mz_next = 0;
-            unsigned short xb_next[ROWS];
-#pragma unroll
-            for (int b = 0; b < ROWS; ++b) xb_next[b] = 0;
-            if (more) load_entry(pos + stride, col_next, mz_next, xb_next);
-            // lane e: multiplier pairs of every row for its entry
-            const float sf = __half2float(__ushort_as_half((unsigned short)(mz & 0xffffu)));
-            const float zf = __half2float(__ushort_as_half((unsigned short)(mz >> 16)));
-#pragma unroll
-            for (int b = 0; b < ROWS; ++b) {
-                const float xf = __half2float(__ushort_as_half(xb[b]));
-                const float am = xf * sf;       // exact
-                zl[b] += xf * zf;               // exact product
-                const unsigned long long aa = pack2(am, am);
-                sts_pairs(mbuf + 16u * (lane * ROWS + b), fmul2(aa, pack2(0x1p93f, 0x1p89f)), fmul2(aa, pack2(0x1p85f, 0x1p81f)));
-            }
             cp_async_wait<1>();   // this chunk's copies have landed (the next chunk's may still fly)
             __syncwarp();
+            // lane e: multiplier pairs of every row for its entry
+            {
+                const bool on = pos + lane < hi;
+                const unsigned ea = ebuf + cur * kEntBytes + (unsigned)lane * (ROWS + 1) * 4u;
+                const unsigned mz = lds_u32(ea);
+                const float sf = __half2float(__ushort_as_half((unsigned short)(mz & 0xffffu)));
+                const float zf = __half2float(__ushort_as_half((unsigned short)(mz >> 16)));
+#pragma unroll
+                for (int b = 0; b < ROWS; ++b) {
+                    unsigned short xb = 0;
+                    if (on && b < batch) {
+                        if (xw_ok) {
+                            const unsigned w = lds_u32(ea + 4u * (1 + b));
+                            xb = (unsigned short)((col & 1) ? (w >> 16) : (w & 0xffffu));
+                        } else {
+                            xb = __ldg(reinterpret_cast<const unsigned short*>(X) + (size_t)b * ldx + col);
+                        }
+                    }
+                    const float xf = __half2float(__ushort_as_half(xb));
+                    const float am = xf * sf;       // exact
+                    zl[b] += xf * zf;               // exact product
+                    const unsigned long long aa = pack2(am, am);
+                    sts_pairs(mbuf + 16u * (lane * ROWS + b), fmul2(aa, pack2(0x1p93f, 0x1p89f)), fmul2(aa, pack2(0x1p85f, 0x1p81f)));
+                }
+            }
+            __syncwarp();
+            const unsigned cb = cbuf + cur * kBufBytes;
             const int valid = min(CH, hi - pos);
             if (valid == CH) {
 #pragma unroll
-                for (int u = 0; u < MSUBS; ++u) step(cbuf + cur, u);
+                for (int u = 0; u < MSUBS; ++u) step(cb, u);
             } else {
                 const int nsub = (valid + SLM - 1) / SLM;
 #pragma unroll 1
-                for (int u = 0; u < nsub; ++u) step(cbuf + cur, u);
+                for (int u = 0; u < nsub; ++u) step(cb, u);
             }
             __syncwarp();
-            cur = (cur == 0u) ? kBufBytes : 0u;
+            cur ^= 1u;
             col = col_next;
             col_next = col_after;
-            mz = mz_next;
-#pragma unroll
-            for (int b = 0; b < ROWS; ++b) xb[b] = xb_next[b];
         }
     }
     cp_async_wait<0>();
@@ -411,18 +375,8 @@ static spqt_status small_entry(const void* codes, const void* meta, int m, int n
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const __half* Xh = static_cast<const __half*>(X);
     if (!dense) {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(1);
-        cfg.blockDim = dim3(1024);
-        cfg.stream = s;
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = g_no_pdl ? 0 : 1;
-        const cudaError_t err = cudaLaunchKernelEx(&cfg, union_sparsify_kernel, Xh, ldx, batch, n, t, idx, count);
-        count_launch();
-        if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return SPQT_ERR_CUDA;
+        const spqt_status st2 = launch_sparsify_rows(Xh, ldx, batch, n, t, idx, count, s);
+        if (st2 != SPQT_OK) return st2;
     }
     const int32_t* li = dense ? nullptr : idx;
     const int32_t* lc = dense ? nullptr : count;
