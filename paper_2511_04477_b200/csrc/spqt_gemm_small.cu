@@ -6,7 +6,7 @@
 //   sparsify_rows_kernel    (spqt_sparsify.cu) one CTA; "active" = |X[b][k]| > t in at least one row b.
 //   gemm_small_kernel       grid (S, R): CTA (s, r) takes the s-th of S equal slices of the union list
 //                           for block-row r; its 8 warps take the slice's chunks of 32 entries in turn,
-//                           each with two code buffers (the next chunk's copies fly during the
+//                           each with three chunk buffers (the next chunks' copies fly during the
 //                           arithmetic).  Lane e of a chunk holds entry e: it loads the entry's column,
 //                           its (scale, zero) pair and the batch's x values and writes the packed
 //                           multiplier pairs of every row; then the warp does the dequantize-FMA work,
@@ -30,13 +30,17 @@ constexpr int kSmallThreads = kSmallWarps * 32;
 constexpr int kSmallRows = 4;      // batch rows per pass at most (a pass of one or two rows keeps two sets of sums)
 constexpr int kSmallMaxSplit = 8;  // slices per block-row at most
 constexpr int kSmallChunk = 32;    // list entries per chunk
+#ifndef SPQT_SMALL_DEPTH
+#define SPQT_SMALL_DEPTH 3
+#endif
+constexpr int kSmallDepth = SPQT_SMALL_DEPTH;     // chunk buffers per warp
 
 template <int G, int BITS, int ROWS>
 struct SmallSmem {
     static constexpr int B = G * BITS / 8;
-    alignas(16) unsigned char codes[kSmallWarps][2][kSmallChunk * B];
+    alignas(16) unsigned char codes[kSmallWarps][kSmallDepth][kSmallChunk * B];
     alignas(16) float mult[kSmallWarps][kSmallChunk][ROWS][4];
-    alignas(16) unsigned ent[kSmallWarps][2][kSmallChunk][ROWS + 1];  // per entry: its (scale, zero) pair and the words holding the rows' x values
+    alignas(16) unsigned ent[kSmallWarps][kSmallDepth][kSmallChunk][ROWS + 1];  // per entry: its (scale, zero) pair and the words holding the rows' x values
     alignas(16) float red[kSmallWarps][ROWS][G];
     float red_z[kSmallWarps][ROWS];
     int last;
@@ -94,7 +98,7 @@ gemm_small_kernel(const uint8_t* __restrict__ codes, const unsigned* __restrict_
         const int e = min(pos + lane, hi - 1);
         return idx ? __ldg(idx + e) : e;
     };
-    // the chunk's code blocks into one of the warp's two buffers, lane after lane
+    // the chunk's code blocks into one of the warp's buffers, lane after lane
     auto copy_codes = [&](int col, unsigned dst) {
 #pragma unroll
         for (int q = 0; q < NC; ++q) {
@@ -108,26 +112,38 @@ gemm_small_kernel(const uint8_t* __restrict__ codes, const unsigned* __restrict_
         cp_async_commit();
     };
 
+    // One step: the lane's 16 codes become eight packed operand pairs ONCE (masks and shifts), then every
+    // row of the batch multiplies them with its own multiplier pairs.
     auto step = [&](unsigned cb, int u) {
         const unsigned ent = (unsigned)(u * SLM + mslot);
+        uint2 wv;
         if (BITS == 4) {
-            const uint2 wv = lds_v2(cb + lane * 8 + u * 256);
-#pragma unroll
-            for (int b = 0; b < ROWS; ++b) {
-                unsigned long long m01, m23;
-                lds_pairs(mbuf + 16u * (ent * ROWS + b), m01, m23);
-                fma_block8(acc[b], wv, m01, m23);
-            }
+            wv = lds_v2(cb + lane * 8 + u * 256);
         } else {
             const unsigned blk = cb + ent * B;
             const unsigned w2 = lds_u32(blk + 4u * mh);
             const unsigned w1 = lds_u32(blk + (G / 4) + 4u * (mh % (LM / 2))) >> (mh / (LM / 2));
+            wv.x = (w2 & 0x33333333u) | ((w1 << 2) & 0x44444444u);     // the two planes widened to nibble codes
+            wv.y = ((w2 >> 2) & 0x33333333u) | (w1 & 0x44444444u);
+        }
+        unsigned long long op[8];
+        {
+            const unsigned w = wv.x, v = wv.x >> 16, w2b = wv.y, v2 = wv.y >> 16;
+            op[0] = pack2(__uint_as_float(w & 0x0000000fu), __uint_as_float(w & 0x000000f0u));
+            op[1] = pack2(__uint_as_float(w & 0x00000f00u), __uint_as_float(w & 0x0000f000u));
+            op[2] = pack2(__uint_as_float(v & 0x0000000fu), __uint_as_float(v & 0x000000f0u));
+            op[3] = pack2(__uint_as_float(v & 0x00000f00u), __uint_as_float(v & 0x0000f000u));
+            op[4] = pack2(__uint_as_float(w2b & 0x0000000fu), __uint_as_float(w2b & 0x000000f0u));
+            op[5] = pack2(__uint_as_float(w2b & 0x00000f00u), __uint_as_float(w2b & 0x0000f000u));
+            op[6] = pack2(__uint_as_float(v2 & 0x0000000fu), __uint_as_float(v2 & 0x000000f0u));
+            op[7] = pack2(__uint_as_float(v2 & 0x00000f00u), __uint_as_float(v2 & 0x0000f000u));
+        }
 #pragma unroll
-            for (int b = 0; b < ROWS; ++b) {
-                unsigned long long m01, m23;
-                lds_pairs(mbuf + 16u * (ent * ROWS + b), m01, m23);
-                fma_block3(acc[b], w2, w1, m01, m23);
-            }
+        for (int b = 0; b < ROWS; ++b) {
+            unsigned long long m01, m23;
+            lds_pairs(mbuf + 16u * (ent * ROWS + b), m01, m23);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) ffma2(acc[b][i], op[i], (i & 1) ? m23 : m01);
         }
     };
 
@@ -149,18 +165,26 @@ gemm_small_kernel(const uint8_t* __restrict__ codes, const unsigned* __restrict_
         copy_codes(col, cbuf + which * kBufBytes);   // (commits the group)
     };
 
+    // kSmallDepth buffers per warp: the copies of the next kSmallDepth - 1 chunks fly during a chunk's arithmetic
     const int first = lo + warp * CH, stride = kSmallWarps * CH;
     if (first < hi) {
-        int col = column_at(first);
-        issue_chunk(col, 0u);
-        int col_next = first + stride < hi ? column_at(first + stride) : 0;
+        constexpr int D = kSmallDepth;
+        int cols[D];   // columns of this lane's entry in the chunks at pos, pos + stride, ..
+#pragma unroll
+        for (int d = 0; d < D; ++d) cols[d] = first + d * stride < hi ? column_at(first + d * stride) : 0;
+#pragma unroll
+        for (int d = 0; d < D - 1; ++d) {
+            if (first + d * stride < hi) issue_chunk(cols[d], (unsigned)d);
+            else cp_async_commit();
+        }
         unsigned cur = 0;
         for (int pos = first; pos < hi; pos += stride) {
-            const bool more = pos + stride < hi;
-            if (more) issue_chunk(col_next, cur ^ 1u);
+            const unsigned nxt = cur + (D - 1) >= (unsigned)D ? cur + (D - 1) - D : cur + (D - 1);
+            if (pos + (D - 1) * stride < hi) issue_chunk(cols[D - 1], nxt);
             else cp_async_commit();
-            const int col_after = pos + 2 * stride < hi ? column_at(pos + 2 * stride) : 0;
-            cp_async_wait<1>();   // this chunk's copies have landed (the next chunk's may still fly)
+            const int col_after = pos + D * stride < hi ? column_at(pos + D * stride) : 0;
+            const int col = cols[0];
+            cp_async_wait<D - 1>();   // this chunk's copies have landed (the later chunks' may still fly)
             __syncwarp();
             // lane e: multiplier pairs of every row for its entry
             {
@@ -199,9 +223,10 @@ gemm_small_kernel(const uint8_t* __restrict__ codes, const unsigned* __restrict_
                 for (int u = 0; u < nsub; ++u) step(cb, u);
             }
             __syncwarp();
-            cur ^= 1u;
-            col = col_next;
-            col_next = col_after;
+            cur = cur + 1 == (unsigned)D ? 0u : cur + 1;
+#pragma unroll
+            for (int d = 0; d + 1 < D; ++d) cols[d] = cols[d + 1];
+            cols[D - 1] = col_after;
         }
     }
     cp_async_wait<0>();
