@@ -1,8 +1,8 @@
 // Sparse index collection: hidden state x and a threshold t -> the ascending
 // list of the entries with |x_k| > t and its length.  Two kernels, one CTA each:
 //   sparsify_kernel (one row, any n): each warp owns a contiguous segment of x, counts its active entries
-//     with __ballot_sync/__popc, the 32 warp totals are scanned in shared memory, and each warp then
-//     writes its indices at its base offset.
+//     with __ballot_sync/__popc (the loads of eight groups of 32 entries in flight together), the 32 warp
+//     totals are scanned in shared memory, and each warp then writes its indices at its base offset.
 //   sparsify_rows_kernel (the small batch, n < 2^16: "active in at least one of B rows"): 16-byte loads,
 //     all of a piece's loads in flight together (with B rows, loads that wait for one another cost a round
 //     trip each); compaction by warp scans.  For a single row it measured no faster than the kernel above
@@ -35,11 +35,27 @@ sparsify_kernel(const __half* __restrict__ x, int n, float t,
     const int seg = ((n + 32 * 32 - 1) / (32 * 32)) * 32;
     const int begin = min(warp * seg, n), end = min(begin + seg, n);
 
+    // Eight groups of 32 entries at a time: their loads are issued together (addresses clamped into x instead
+    // of guarded, so that nothing makes one load wait for another), then one ballot per group.  Up to 64
+    // groups per warp (n <= 65536) the lane's activity bits stay in a register for the writing phase.
+    const int groups = (end - begin + 31) >> 5;
+    const bool in_regs = groups <= 64;
+    unsigned long long flags = 0ull;
     int total = 0;
-    for (int k0 = begin; k0 < end; k0 += 32) {
-        const int k = k0 + lane;
-        const bool p = (k < end) && is_active(x[k], t);
-        total += __popc(__ballot_sync(0xffffffffu, p));
+    for (int g0 = 0; g0 < groups; g0 += 8) {
+        __half v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            if (g0 + j < groups) v[j] = x[min(begin + (g0 + j) * 32 + lane, n - 1)];   // (uniform condition)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (g0 + j < groups) {
+                const int k = begin + (g0 + j) * 32 + lane;
+                const bool p = (k < end) && is_active(v[j], t);
+                total += __popc(__ballot_sync(0xffffffffu, p));
+                if (p) flags |= 1ull << ((g0 + j) & 63);
+            }
+        }
     }
     if (lane == 0) warp_total[warp] = total;
     __syncthreads();
@@ -55,6 +71,15 @@ sparsify_kernel(const __half* __restrict__ x, int n, float t,
     }
     __syncthreads();
     int base = warp_base[warp];
+    if (in_regs) {
+        for (int g = 0; g < groups; ++g) {
+            const bool p = (flags >> g) & 1ull;
+            const unsigned mask = __ballot_sync(0xffffffffu, p);
+            if (p) idx[base + __popc(mask & ((1u << lane) - 1u))] = begin + g * 32 + lane;
+            base += __popc(mask);
+        }
+        return;
+    }
     for (int k0 = begin; k0 < end; k0 += 32) {
         const int k = k0 + lane;
         const bool p = (k < end) && is_active(x[k], t);
