@@ -1,5 +1,8 @@
 // Sparse index collection: hidden state x and a threshold t -> the ascending
-// list of the entries with |x_k| > t and its length.  Two kernels, one CTA each:
+// list of the entries with |x_k| > t and its length.  Three kernels:
+//   sparsify_cluster_kernel (one row, 6144 < n <= 65536): the compaction below spread over a thread-block
+//     cluster of 8 CTAs, warp totals exchanged through distributed shared memory (3.4 against 4.9 us at
+//     n = 14336; no gain at n = 4096, where the single CTA stays).
 //   sparsify_kernel (one row, any n): each warp owns a contiguous segment of x, counts its active entries
 //     with __ballot_sync/__popc (the loads of eight groups of 32 entries in flight together), the 32 warp
 //     totals are scanned in shared memory, and each warp then writes its indices at its base offset.
@@ -87,6 +90,80 @@ sparsify_kernel(const __half* __restrict__ x, int n, float t,
         if (p) idx[base + __popc(mask & ((1u << lane) - 1u))] = k;
         base += __popc(mask);
     }
+}
+
+// The same compaction spread over a thread-block cluster of 8 CTAs of 8 warps (n <= 65536): one SM's
+// instruction rate is what a single CTA spends most of its time on once n reaches several thousand.  The 64
+// warps own consecutive segments of x; every CTA leaves its warps' totals in its own shared memory, the
+// cluster synchronises, and each warp adds up the totals of the warps before it, reading the other CTAs'
+// tables through distributed shared memory.  A second cluster barrier keeps every CTA's table alive until
+// all have read it.  (Hardware barriers that every CTA reaches unconditionally: nothing to time out.)
+constexpr int kClusterCtas = 8;
+constexpr int kClusterWarps = 8;
+
+__global__ void __launch_bounds__(kClusterWarps * 32)
+sparsify_cluster_kernel(const __half* __restrict__ x, int n, float t, int32_t* __restrict__ idx, int32_t* __restrict__ count)
+{
+    __shared__ int warp_total[kClusterWarps];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    unsigned rank;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+    const int gw = (int)rank * kClusterWarps + warp;      // this warp among the cluster's 64
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    constexpr int kAll = kClusterCtas * kClusterWarps;
+    const int seg = ((n + kAll * 32 - 1) / (kAll * 32)) * 32;   // at most 1024 entries: 32 groups
+    const int begin = min(gw * seg, n), end = min(begin + seg, n);
+    const int groups = (end - begin + 31) >> 5;
+    unsigned flags = 0u;
+    int total = 0;
+    for (int g0 = 0; g0 < groups; g0 += 8) {
+        __half v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j)
+            if (g0 + j < groups) v[j] = x[min(begin + (g0 + j) * 32 + lane, n - 1)];   // (uniform condition)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            if (g0 + j < groups) {
+                const int k = begin + (g0 + j) * 32 + lane;
+                const bool p = (k < end) && is_active(v[j], t);
+                total += __popc(__ballot_sync(0xffffffffu, p));
+                if (p) flags |= 1u << (g0 + j);
+            }
+        }
+    }
+    if (lane == 0) warp_total[warp] = total;
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    // lane l looks up the totals of warps l and l + 32 of the cluster
+    int below = 0, all = 0;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        const int w = lane + 32 * h;
+        unsigned remote;
+        const unsigned local = static_cast<unsigned>(__cvta_generic_to_shared(&warp_total[w % kClusterWarps]));
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"((unsigned)(w / kClusterWarps)));
+        int v;
+        asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(v) : "r"(remote) : "memory");
+        below += (w < gw) ? v : 0;
+        all += v;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        below += __shfl_xor_sync(0xffffffffu, below, o);
+        all += __shfl_xor_sync(0xffffffffu, all, o);
+    }
+    if (gw == 0 && lane == 0) *count = all;
+    int base = below;
+    for (int g = 0; g < groups; ++g) {
+        const bool p = (flags >> g) & 1u;
+        const unsigned mask = __ballot_sync(0xffffffffu, p);
+        if (p) idx[base + __popc(mask & ((1u << lane) - 1u))] = begin + g * 32 + lane;
+        base += __popc(mask);
+    }
+    // nobody leaves while another CTA may still be reading its table
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
 // Lane l of a warp holds the 8 columns 256*piece + 8*l .. + 7 of each of the warp's pieces (a warp owns up
@@ -226,6 +303,28 @@ extern "C" spqt_status spqt_sparsify(const void* x, int n, float t,
     using namespace spqt;
     if (n < 0 || !count || (n > 0 && (!x || !idx))) return SPQT_ERR_INVALID_ARG;
     if (!aligned(x, 2) || !aligned(idx, 4) || !aligned(count, 4)) return SPQT_ERR_ALIGNMENT;
+    // from a few thousand entries on, the compaction spread over a cluster of 8 CTAs (falls back to the
+    // single CTA below if the cluster cannot be launched)
+    if (n > 6144 && n <= 65536) {
+        cudaLaunchConfig_t cc = {};
+        cc.gridDim = dim3(kClusterCtas);
+        cc.blockDim = dim3(kClusterWarps * 32);
+        cc.stream = static_cast<cudaStream_t>(stream);
+        cudaLaunchAttribute ca[2];
+        ca[0].id = cudaLaunchAttributeClusterDimension;
+        ca[0].val.clusterDim.x = kClusterCtas;
+        ca[0].val.clusterDim.y = 1;
+        ca[0].val.clusterDim.z = 1;
+        ca[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        ca[1].val.programmaticStreamSerializationAllowed = 1;
+        cc.attrs = ca;
+        cc.numAttrs = g_no_pdl ? 1 : 2;
+        if (cudaLaunchKernelEx(&cc, sparsify_cluster_kernel, static_cast<const __half*>(x), n, t, idx, count) == cudaSuccess) {
+            count_launch();
+            return cudaGetLastError() == cudaSuccess ? SPQT_OK : SPQT_ERR_CUDA;
+        }
+        (void)cudaGetLastError();
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(1);
     cfg.blockDim = dim3(kSparsifyThreads);
