@@ -205,6 +205,18 @@ spqt_status spqt_sparse_linear_host(const void* codes, const void* scale_zero,
                                     void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The same without the wait at the end: everything is enqueued on `stream` and the call returns; y_host
+ * is valid once the caller has synchronised the stream (several linears of a token step can be enqueued
+ * one after the other, each with its own staging buffers and workspace, and waited for once).  x_host
+ * must stay unchanged until then; pageable x_host / y_host make the copies synchronous, not wrong.
+ */
+spqt_status spqt_sparse_linear_host_async(const void* codes, const void* scale_zero,
+                                          int m, int n, int bits, int group,
+                                          const void* x_host, float t, void* y_host,
+                                          void* x_dev, int32_t* idx_dev, int32_t* count_dev, void* y_dev,
+                                          void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Tuning aid: number of CTAs of the GEMV grid (0 restores the built-in rule, one
  * persistent CTA per SM; values above 512 are clamped).  `no_overlap` is a set of bits, 0 by
  * default: bit 0 launches the GEMV kernels strictly stream-ordered instead of letting a GEMV start

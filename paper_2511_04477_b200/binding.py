@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libspqt.so")
 EXPORTS = (
     "spqt_status_string", "spqt_version", "spqt_packed_sizes", "spqt_pack", "spqt_unpack",
     "spqt_sparsify", "spqt_sparse_gemv", "spqt_sparse_gemv_static", "spqt_static_status", "spqt_sparsify_gemv", "spqt_dense_gemv",
-    "spqt_sparse_linear_host", "spqt_gemm_small_workspace", "spqt_sparse_gemm_small", "spqt_dense_gemm_small", "spqt_rowwise_packed_sizes", "spqt_rowwise_pack", "spqt_rowwise_dense_gemv", "spqt_kq_packed_sizes", "spqt_kq_pack", "spqt_kq_sparse_gemv", "spqt_kq_dense_gemv", "spqt_autotune", "spqt_calibrate_threshold", "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_launch_count",
+    "spqt_sparse_linear_host", "spqt_sparse_linear_host_async", "spqt_gemm_small_workspace", "spqt_sparse_gemm_small", "spqt_dense_gemm_small", "spqt_rowwise_packed_sizes", "spqt_rowwise_pack", "spqt_rowwise_dense_gemv", "spqt_kq_packed_sizes", "spqt_kq_pack", "spqt_kq_sparse_gemv", "spqt_kq_dense_gemv", "spqt_autotune", "spqt_calibrate_threshold", "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_launch_count",
 )
 
 _lib = None
@@ -66,6 +66,7 @@ def lib() -> ctypes.CDLL:
         L.spqt_kq_dense_gemv.argtypes = [vp, i32, i32, vp, vp, vp, sz, vp]
         L.spqt_sparse_linear_host.argtypes = [vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, vp,
                                               vp, vp, vp, vp, vp, sz, vp]
+        L.spqt_sparse_linear_host_async.argtypes = L.spqt_sparse_linear_host.argtypes
         L.spqt_gemm_small_workspace.argtypes = [i32, i32, i32, i32, ctypes.POINTER(sz)]
         L.spqt_gemm_small_workspace.restype = i32
         L.spqt_sparse_gemm_small.argtypes = [vp, vp, i32, i32, i32, i32, vp, i32, i32, ctypes.c_float, vp, vp, vp, i32, vp, sz, vp]
@@ -274,10 +275,12 @@ class HostLinear:
         self.workspace = workspace if workspace is not None else new_workspace(p.m, p.n, p.bits, p.group, dev)
 
 
-def spqt_sparse_linear_host(h: HostLinear, t: float, stream=None) -> torch.Tensor:
-    """x in ``h.x_host`` -> y in ``h.y_host`` (copies, index collection, sparse GEMV, sync)."""
+def spqt_sparse_linear_host(h: HostLinear, t: float, stream=None, wait: bool = True) -> torch.Tensor:
+    """x in ``h.x_host`` -> y in ``h.y_host`` (copies, index collection, sparse GEMV; with ``wait`` the call
+    returns when y is there, otherwise once everything is enqueued and the caller synchronises the stream)."""
     p = h.p
-    _ok(lib().spqt_sparse_linear_host(
+    fn = lib().spqt_sparse_linear_host if wait else lib().spqt_sparse_linear_host_async
+    _ok(fn(
         p.codes.data_ptr(), p.scale_zero.data_ptr(), p.m, p.n, p.bits, p.group,
         h.x_host.data_ptr(), float(t), h.y_host.data_ptr(), h.x_dev.data_ptr(), h.idx.data_ptr(),
         h.count.data_ptr(), h.y_dev.data_ptr(), h.workspace.data_ptr(), h.workspace.numel(),

@@ -57,11 +57,10 @@ spqt_status spqt_packed_sizes(int m, int n, int bits, int group,
 
 unsigned long long spqt_launch_count(void) { return spqt::g_launches.load(std::memory_order_relaxed); }
 
-spqt_status spqt_sparse_linear_host(const void* codes, const void* scale_zero,
-                                    int m, int n, int bits, int group,
-                                    const void* x_host, float t, void* y_host,
-                                    void* x_dev, int32_t* idx_dev, int32_t* count_dev, void* y_dev,
-                                    void* workspace, size_t workspace_bytes, void* stream)
+static spqt_status linear_host(const void* codes, const void* scale_zero, int m, int n, int bits, int group,
+                               const void* x_host, float t, void* y_host,
+                               void* x_dev, int32_t* idx_dev, int32_t* count_dev, void* y_dev,
+                               void* workspace, size_t workspace_bytes, void* stream, bool wait)
 {
     if (!x_host || !y_host || !x_dev || !y_dev) return SPQT_ERR_INVALID_ARG;
     spqt::Format f;
@@ -86,8 +85,28 @@ spqt_status spqt_sparse_linear_host(const void* codes, const void* scale_zero,
     if (y_target == y_dev &&
         cudaMemcpyAsync(y_host, y_dev, (size_t)m * 2, cudaMemcpyDeviceToHost, s) != cudaSuccess)
         return SPQT_ERR_CUDA;
-    if (cudaStreamSynchronize(s) != cudaSuccess) return SPQT_ERR_CUDA;
+    if (wait && cudaStreamSynchronize(s) != cudaSuccess) return SPQT_ERR_CUDA;
     return SPQT_OK;
+}
+
+spqt_status spqt_sparse_linear_host(const void* codes, const void* scale_zero,
+                                    int m, int n, int bits, int group,
+                                    const void* x_host, float t, void* y_host,
+                                    void* x_dev, int32_t* idx_dev, int32_t* count_dev, void* y_dev,
+                                    void* workspace, size_t workspace_bytes, void* stream)
+{
+    return linear_host(codes, scale_zero, m, n, bits, group, x_host, t, y_host, x_dev, idx_dev, count_dev, y_dev,
+                       workspace, workspace_bytes, stream, true);
+}
+
+spqt_status spqt_sparse_linear_host_async(const void* codes, const void* scale_zero,
+                                          int m, int n, int bits, int group,
+                                          const void* x_host, float t, void* y_host,
+                                          void* x_dev, int32_t* idx_dev, int32_t* count_dev, void* y_dev,
+                                          void* workspace, size_t workspace_bytes, void* stream)
+{
+    return linear_host(codes, scale_zero, m, n, bits, group, x_host, t, y_host, x_dev, idx_dev, count_dev, y_dev,
+                       workspace, workspace_bytes, stream, false);
 }
 
 }  // extern "C"

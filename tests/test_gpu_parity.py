@@ -555,6 +555,18 @@ def test_host_entry_point_matches_the_device_path():
     y_dev, idx, cnt = run_sparse(p, x, t, binding.new_workspace(m, n, bits, group))
     assert np.array_equal(y_host.view(np.uint16), y_dev.view(np.uint16))
     assert int(h.count.item()) == cnt
+    # the variant that does not wait: two linears enqueued one after the other, one synchronisation
+    h2 = binding.HostLinear(p)
+    x2 = inputs.activations(n, seed=73)
+    h.y_host.zero_()
+    h2.x_host.copy_(torch.from_numpy(x2))
+    s = torch.cuda.Stream()
+    binding.spqt_sparse_linear_host(h, t, stream=s, wait=False)
+    binding.spqt_sparse_linear_host(h2, t, stream=s, wait=False)
+    s.synchronize()
+    assert np.array_equal(h.y_host.numpy().view(np.uint16), y_dev.view(np.uint16))
+    y2, _, _ = run_sparse(p, x2, t, binding.new_workspace(m, n, bits, group))
+    assert np.array_equal(h2.y_host.numpy().view(np.uint16), y2.view(np.uint16))
 
 
 def test_read_and_gather_probes_fetch_what_they_report():
