@@ -173,7 +173,7 @@ sparsify_cluster_kernel(const __half* __restrict__ x, int n, float t, int32_t* _
 // over the warps, and every lane writes its own active columns behind those of the lanes before it.
 __global__ void __launch_bounds__(1024)
 sparsify_rows_kernel(const __half* __restrict__ X, int ldx, int batch, int n, float t,
-                      int32_t* __restrict__ idx, int32_t* __restrict__ count)
+                     int32_t* __restrict__ idx, int32_t* __restrict__ count)
 {
     __shared__ int warp_total[32];
     __shared__ int warp_base[32];
@@ -192,49 +192,43 @@ sparsify_rows_kernel(const __half* __restrict__ X, int ldx, int batch, int n, fl
 
     unsigned long long flags = 0ull;                   // byte j: activity bits of the lane's 8 columns of piece j
 #pragma unroll 1
-    for (int j0 = 0; j0 < pp; ++j0) {
-        uint4 v[1][8];
+    for (int j = 0; j < pp; ++j) {
+        const int k0 = (warp * pp + j) * 256 + lane * 8;
+        const bool have = k0 < n;
+        uint4 v[8];
 #pragma unroll
-        for (int j = 0; j < 1; ++j) {
-            const int piece = warp * pp + j0 + j, k0 = piece * 256 + lane * 8;
-            const bool have = k0 < n;
+        for (int b = 0; b < 8; ++b) {
+            v[b] = make_uint4(0u, 0u, 0u, 0u);
+            if (have && b < batch) {
+                const size_t off = (size_t)b * ldx + k0;
+                if (vec_ok && k0 + 8 <= n) {
+                    v[b] = __ldg(reinterpret_cast<const uint4*>(Xs + off));
+                } else {
+                    unsigned short h[8];
 #pragma unroll
-            for (int b = 0; b < 8; ++b) {
-                v[j][b] = make_uint4(0u, 0u, 0u, 0u);
-                if (have && b < batch) {
-                    const size_t off = (size_t)b * ldx + k0;
-                    if (vec_ok && k0 + 8 <= n) {
-                        v[j][b] = __ldg(reinterpret_cast<const uint4*>(Xs + off));
-                    } else {
-                        unsigned short h[8];
-#pragma unroll
-                        for (int e = 0; e < 8; ++e) h[e] = (k0 + e < n) ? __ldg(Xs + off + e) : (unsigned short)0;
-                        v[j][b] = make_uint4(h[0] | ((unsigned)h[1] << 16), h[2] | ((unsigned)h[3] << 16),
-                                             h[4] | ((unsigned)h[5] << 16), h[6] | ((unsigned)h[7] << 16));
-                    }
+                    for (int e = 0; e < 8; ++e) h[e] = (k0 + e < n) ? __ldg(Xs + off + e) : (unsigned short)0;
+                    v[b] = make_uint4(h[0] | ((unsigned)h[1] << 16), h[2] | ((unsigned)h[3] << 16),
+                                      h[4] | ((unsigned)h[5] << 16), h[6] | ((unsigned)h[7] << 16));
                 }
             }
         }
+        unsigned m8 = 0;
 #pragma unroll
-        for (int j = 0; j < 1; ++j) {
-            unsigned m8 = 0;
+        for (int b = 0; b < 8; ++b) {
+            if (b < batch) {   // (uniform)
+                const unsigned wds[4] = {v[b].x, v[b].y, v[b].z, v[b].w};
 #pragma unroll
-            for (int b = 0; b < 8; ++b) {
-                if (b < batch) {   // (uniform)
-                    const unsigned wds[4] = {v[j][b].x, v[j][b].y, v[j][b].z, v[j][b].w};
-#pragma unroll
-                    for (int e2 = 0; e2 < 4; ++e2) {
-                        const unsigned ab = wds[e2] & 0x7fff7fffu;
-                        const unsigned gt = __hgt2_mask(*reinterpret_cast<const __half2*>(&ab), thr_h2);   // false for NaN
-                        m8 |= ((gt & 1u) | ((gt >> 15) & 2u)) << (2 * e2);
-                    }
+                for (int e2 = 0; e2 < 4; ++e2) {
+                    const unsigned ab = wds[e2] & 0x7fff7fffu;
+                    const unsigned gt = __hgt2_mask(*reinterpret_cast<const __half2*>(&ab), thr_h2);   // false for NaN
+                    m8 |= ((gt & 1u) | ((gt >> 15) & 2u)) << (2 * e2);
                 }
             }
-            // columns past n do not exist (with a negative threshold their zeros would count)
-            const int left = n - ((warp * pp + j0 + j) * 256 + lane * 8);
-            if (left < 8) m8 &= (left <= 0) ? 0u : ((1u << left) - 1u);
-            flags |= (unsigned long long)m8 << (8 * (j0 + j));
         }
+        // columns past n do not exist (with a negative threshold their zeros would count)
+        const int left = n - k0;
+        if (left < 8) m8 &= (left <= 0) ? 0u : ((1u << left) - 1u);
+        flags |= (unsigned long long)m8 << (8 * j);
     }
     int total = __popcll(flags);
 #pragma unroll
