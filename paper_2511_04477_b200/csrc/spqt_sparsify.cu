@@ -6,7 +6,8 @@
 //   sparsify_kernel (one row, any n): each warp owns a contiguous segment of x, counts its active entries
 //     with __ballot_sync/__popc (the loads of eight groups of 32 entries in flight together), the 32 warp
 //     totals are scanned in shared memory, and each warp then writes its indices at its base offset.
-//   sparsify_rows_kernel (the small batch, n < 2^16: "active in at least one of B rows"): 16-byte loads,
+//   sparsify_rows_kernel (the small batch, n < 2^16: "active in at least one of B rows"; one CTA, or a
+//     cluster of 8 CTAs from n = 6144 up): 16-byte loads,
 //     all of a piece's loads in flight together (with B rows, loads that wait for one another cost a round
 //     trip each); compaction by warp scans.  For a single row it measured no faster than the kernel above
 //     (2.7 against 2.3 us at n = 4096, 5.9 against 5.2 us at n = 14336), which therefore keeps that job.
@@ -171,17 +172,24 @@ sparsify_cluster_kernel(const __half* __restrict__ x, int n, float t, int32_t* _
 // 2-byte loads at a ragged end or when X is not aligned for it), and a piece's loads are all issued before
 // the first compare, so that they share one round trip.  Then the usual compaction: totals per warp, a scan
 // over the warps, and every lane writes its own active columns behind those of the lanes before it.
-__global__ void __launch_bounds__(1024)
+// CLUSTER: the same on a thread-block cluster of 8 CTAs of 8 warps (the 64 warps own consecutive runs of
+// pieces; warp totals are exchanged through distributed shared memory as in sparsify_cluster_kernel).
+template <bool CLUSTER>
+__global__ void __launch_bounds__(CLUSTER ? kClusterWarps * 32 : 1024)
 sparsify_rows_kernel(const __half* __restrict__ X, int ldx, int batch, int n, float t,
                      int32_t* __restrict__ idx, int32_t* __restrict__ count)
 {
     __shared__ int warp_total[32];
     __shared__ int warp_base[32];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31, cta_warp = threadIdx.x >> 5;
+    unsigned rank = 0;
+    if (CLUSTER) asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+    const int warp = CLUSTER ? (int)rank * kClusterWarps + cta_warp : cta_warp;   // among all the warps at work
+    constexpr int kAllWarps = CLUSTER ? kClusterCtas * kClusterWarps : 32;
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int pieces = (n + 255) >> 8;
-    const int pp = (pieces + 31) >> 5;                 // pieces per warp, at most 8
+    const int pp = (pieces + kAllWarps - 1) / kAllWarps;   // pieces per warp, at most 8
     const bool vec_ok = (reinterpret_cast<uintptr_t>(X) & 15) == 0 && (ldx & 7) == 0;
     const unsigned short* Xs = reinterpret_cast<const unsigned short*>(X);
     // the largest fp16 value not above t (any negative value if t < 0: everything but NaN is active; +inf if t
@@ -233,20 +241,46 @@ sparsify_rows_kernel(const __half* __restrict__ X, int ldx, int batch, int n, fl
     int total = __popcll(flags);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) total += __shfl_xor_sync(0xffffffffu, total, o);
-    if (lane == 0) warp_total[warp] = total;
-    __syncthreads();
-    if (warp == 0) {
-        int v = warp_total[lane], incl = v;
+    int base;
+    if (CLUSTER) {
+        if (lane == 0) warp_total[cta_warp] = total;
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+        int below = 0, all = 0;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            int up = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += up;
+        for (int h = 0; h < 2; ++h) {
+            const int w = lane + 32 * h;   // lane l looks up the totals of warps l and l + 32 of the cluster
+            unsigned remote;
+            const unsigned local = static_cast<unsigned>(__cvta_generic_to_shared(&warp_total[w % kClusterWarps]));
+            asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"((unsigned)(w / kClusterWarps)));
+            int v;
+            asm volatile("ld.shared::cluster.s32 %0, [%1];" : "=r"(v) : "r"(remote) : "memory");
+            below += (w < warp) ? v : 0;
+            all += v;
         }
-        warp_base[lane] = incl - v;
-        if (lane == 31) *count = incl;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            below += __shfl_xor_sync(0xffffffffu, below, o);
+            all += __shfl_xor_sync(0xffffffffu, all, o);
+        }
+        if (warp == 0 && lane == 0) *count = all;
+        base = below;
+    } else {
+        if (lane == 0) warp_total[warp] = total;
+        __syncthreads();
+        if (warp == 0) {
+            int v = warp_total[lane], incl = v;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                int up = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += up;
+            }
+            warp_base[lane] = incl - v;
+            if (lane == 31) *count = incl;
+        }
+        __syncthreads();
+        base = warp_base[warp];
     }
-    __syncthreads();
-    int base = warp_base[warp];
     for (int j = 0; j < pp; ++j) {
         const unsigned m8 = (unsigned)(flags >> (8 * j)) & 0xffu;
         const int c8 = __popc(m8);
@@ -268,6 +302,10 @@ sparsify_rows_kernel(const __half* __restrict__ X, int ldx, int batch, int n, fl
         }
         base += __shfl_sync(0xffffffffu, incl, 31);
     }
+    if (CLUSTER) {   // nobody leaves while another CTA may still be reading its table
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    }
 }
 
 
@@ -275,16 +313,32 @@ sparsify_rows_kernel(const __half* __restrict__ X, int ldx, int batch, int n, fl
 spqt_status launch_sparsify_rows(const __half* X, int ldx, int batch, int n, float t, int32_t* idx, int32_t* count,
                                  cudaStream_t stream)
 {
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(1);
-    cfg.blockDim = dim3(1024);
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = kClusterCtas;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.stream = stream;
+    // from a few thousand columns on, the cluster of 8 CTAs (falls back to the single CTA if it cannot be launched)
+    if (n > 6144) {
+        cfg.gridDim = dim3(kClusterCtas);
+        cfg.blockDim = dim3(kClusterWarps * 32);
+        cfg.attrs = g_no_pdl ? attr + 1 : attr;
+        cfg.numAttrs = g_no_pdl ? 1 : 2;
+        if (cudaLaunchKernelEx(&cfg, sparsify_rows_kernel<true>, X, ldx, batch, n, t, idx, count) == cudaSuccess) {
+            count_launch();
+            return cudaGetLastError() == cudaSuccess ? SPQT_OK : SPQT_ERR_CUDA;
+        }
+        (void)cudaGetLastError();
+    }
+    cfg.gridDim = dim3(1);
+    cfg.blockDim = dim3(1024);
     cfg.attrs = attr;
     cfg.numAttrs = g_no_pdl ? 0 : 1;
-    const cudaError_t err = cudaLaunchKernelEx(&cfg, sparsify_rows_kernel, X, ldx, batch, n, t, idx, count);
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, sparsify_rows_kernel<false>, X, ldx, batch, n, t, idx, count);
     count_launch();
     return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SPQT_OK : SPQT_ERR_CUDA;
 }

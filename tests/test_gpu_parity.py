@@ -796,7 +796,8 @@ def test_calibration_threshold_is_the_exact_order_statistic():
 # ------------------------------------------------------------------ small batch over the union of active sets
 
 @pytest.mark.parametrize("bits,group", GEMV_FORMATS)
-@pytest.mark.parametrize("m_blocks,n,batch", [(2, 300, 2), (8, 4096, 4), (3, 1111, 3), (32, 4096, 8), (1, 1, 1), (224, 1024, 5)])
+@pytest.mark.parametrize("m_blocks,n,batch", [(2, 300, 2), (8, 4096, 4), (3, 1111, 3), (32, 4096, 8), (1, 1, 1), (224, 1024, 5),
+                                                  (4, 14336, 4), (2, 20001, 3), (1, 65535, 2)])
 def test_small_batch_over_the_union_matches_the_oracle(bits, group, m_blocks, n, batch):
     m = m_blocks * group
     W = inputs.weights(m, n, seed=m + n + batch)
