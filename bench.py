@@ -2,7 +2,7 @@
 """Benchmark of the SpQt hot path on B200: one line of JSON on stdout.
 
     python bench.py [--gpus N] [--steps K] [--warmup W]            the headline line (config "layer")
-    python bench.py --config sweep | formats | dense | batch | kquant | stack   the other workloads, one JSON line each
+    python bench.py --config sweep | formats | dense | batch | kquant | models | stack   the other workloads, one JSON line each
     python bench.py --impl reference                               the fp64 CPU oracle on a bounded sample
 
 Workload of the headline line (the configuration the metric is quoted on): the seven linear layers of
@@ -30,7 +30,7 @@ roofline.achieved = algorithmic bytes per launch of the dominant kernel (gemv_ke
 The other workloads: `sweep` = sparsity 0-90 % on the 14336->4096 and 4096->14336 projections against the
 same-layout dense GEMV, 64 rotated weight copies, with the no-load-balancing ablation beside it;
 `formats` = Llama-2-70B-shaped linears x {int4, int3} x {g128, g64} at 50 % with outlier activations;
-`dense` = the dense zigzag GEMV on the paper's 15 shapes over several grid sizes; `batch` = 1, 2, 4, 8 rows
+`models` = the GEMV shapes of three model sizes at 25, 40 and 50 %; `dense` = the dense zigzag GEMV on the paper's 15 shapes over several grid sizes; `batch` = 1, 2, 4, 8 rows
 over the union of their active sets; `stack` = a per-token
 pass over a 32-layer Llama-3-8B-shaped stack with thresholds calibrated once for 40 % (tokens/s of the
 linear layers).  The default line carries a short summary of each.
@@ -247,6 +247,18 @@ def other_config_line(which, local, quick=False):
                                             "and the built-in rule; beside it the row-wise-layout baseline (spqt_rowwise_dense_gemv) on the same shapes; rotated weight copies > 2x L2"},
                         roofline=roofline_obj(best["dense_gbs"], peak, kind, nb, best["best_us"], "gemv_kernel<128,4,dense>", 1.0),
                         zigzag_dense_vs_rowwise={"%dx%d" % (r["m"], r["n"]): r["zigzag_dense_vs_rowwise"] for r in rows},
+                        rows=rows)
+        elif which == "models":
+            rows = sweep.model_shapes_sweep(peak)
+            r0 = [r for r in rows if r["shape"] == "70b gate,up" and abs(r["sparsity"] - 0.5) < 0.03][0]
+            nb = sweep.needed_bytes(r0["m"], r0["n"], r0["count"], 4, 128)
+            line = dict(base, metric="sparse int4 GEMV effective HBM GB/s at 50% sparsity, 28672x8192 (GEMV shapes of three model sizes at 25/40/50%)",
+                        value=r0["sparse_gbs"], ms_per_step=r0["sparse_us"] * 1e-3, steps=20, warmup=4,
+                        config={"workload": "Llama-3-8B-, Llama-2-13B- and Llama-2-70B-shaped linears, int4 g128, sparsity 25/40/50%, given list / index "
+                                            "collection inside / dense; rotated weight copies > 2x L2"},
+                        roofline=roofline_obj(r0["sparse_gbs"], peak, kind, nb, r0["sparse_us"], "gemv_kernel<128,4,list>"),
+                        speedup_vs_dense={"%s @%d%%" % (r["shape"], round(100 * r["sparsity"])): {"given_list": r["speedup_vs_dense"],
+                                                                                                 "index_collection_inside": r["fused_speedup_vs_dense"]} for r in rows},
                         rows=rows)
         elif which == "kquant":
             rows = sweep.kq_sweep(peak)
@@ -636,7 +648,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1024)
     ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", default="layer", choices=["layer", "sweep", "formats", "dense", "batch", "kquant", "stack"])
+    ap.add_argument("--config", default="layer", choices=["layer", "sweep", "formats", "dense", "batch", "kquant", "models", "stack"])
     ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_S,
                     help="device time to accumulate over repeated K-step regions of the headline measurement")
     ap.add_argument("--quick", action="store_true", help="reduced form of --config sweep/formats/stack")

@@ -143,6 +143,22 @@ def format_sweep(peak, shapes=None, formats=None):
     return out
 
 
+def model_shapes_sweep(peak):
+    """The GEMV shapes of three model sizes at the paper's three sparsity levels (its GEMV-level experiment,
+    Sec. 6): Llama-3-8B-, Llama-2-13B- and Llama-2-70B-shaped linears, int4 g128, 25 / 40 / 50 %."""
+    shapes = [("8b q,o", 4096, 4096, "laplace"), ("8b gate,up", 14336, 4096, "laplace"), ("8b down", 4096, 14336, "gauss"),
+              ("13b q,k,v,o", 5120, 5120, "laplace"), ("13b gate,up", 13824, 5120, "laplace"), ("13b down", 5120, 13824, "gauss"),
+              ("70b q,o", 8192, 8192, "laplace"), ("70b gate,up", 28672, 8192, "laplace"), ("70b down", 8192, 28672, "gauss")]
+    out = []
+    for (name, m, n, dist) in shapes:
+        x = inputs.activations(n, seed=7, dist=dist)
+        rows = run_case(m, n, 4, 128, [0.25, 0.4, 0.5], x, copies_for(m, n, 4, 128, at_least=4, at_most=40), peak)
+        for r in rows:
+            r["shape"] = name
+        out += rows
+    return out
+
+
 def dense_shape_sweep(peak):
     """The dense zigzag GEMV on the paper's 15 shapes m in {2048, 4096, 8192} x k in {1024 ... 16384}
     (its hyper-parameter study, Sec. 6), int4 g128, over the CTA counts the autotuner would try, and the
