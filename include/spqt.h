@@ -221,8 +221,8 @@ spqt_status spqt_sparse_linear_host_async(const void* codes, const void* scale_z
  * persistent CTA per SM; values above 512 are clamped).  `no_overlap` is a set of bits, 0 by
  * default: bit 0 launches the GEMV kernels strictly stream-ordered instead of letting a GEMV start
  * (and wait inside the kernel) while the previous kernel of the stream drains; bit 1 never launches
- * thread-block clusters (otherwise the 2..8 CTAs that share a block-row combine their sums through
- * shared memory when the device can hold all the clusters at once); bit 2 is an ablation, the paper's
+ * thread-block clusters (otherwise, in spqt_sparse_gemv and spqt_dense_gemv, the 2..8 CTAs that share a
+ * block-row combine their sums through shared memory when the device can hold all the clusters at once); bit 2 is an ablation, the paper's
  * "sparse without load balancing" (Sec. 6): spqt_sparsify_gemv then gives every CTA, and inside it every
  * warp, a fixed range of the matrix columns of its block-row instead of an even share of the active
  * list (same results up to the order of partial sums; lists longer than the shared-memory window and

@@ -1183,7 +1183,12 @@ static spqt_status launch_gemv(const Format& f, const void* codes, const void* m
     // A whole number (2..8) of CTAs per block-row: launch them as one thread-block cluster each, if the
     // device can hold all the clusters at once (asked once per kernel, cluster size and device).
     int cluster_k = 0;
-    if (!g_no_cluster && f.R <= P && P % f.R == 0 && P / f.R >= 2 && P / f.R <= kMaxCluster) {
+    // Not for the call that collects the indices inside: alone, or behind launches of its own kind, it gains
+    // 0.3-0.45 us from a cluster like the others, but in a stream that alternates it with launches that fill
+    // every SM (the stacked gate|up matrix of a decoder layer) every such pair of launches was measured 1.4-1.8 us
+    // slower than the sum of its parts (0.2-0.6 us for the other kinds of call): a layer's four launches take
+    // 37.1 us without these clusters and 38.7 us with them.  The CTAs of a cluster can only start together.
+    if (!g_no_cluster && MODE != kModeFused && f.R <= P && P % f.R == 0 && P / f.R >= 2 && P / f.R <= kMaxCluster) {
         const int k = P / f.R;
         static signed char fits[64][kMaxCluster + 1][149] = {};  // [device][k][clusters]: 0 unknown, 1 yes, -1 no
         const int nclusters = P / k;
