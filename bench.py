@@ -20,8 +20,9 @@ value  = effective GB/s over the bytes the method needs
          collection), whole job, inputs resident in HBM.  The K-step region is timed with CUDA events
          on the launching stream and repeated until a quarter of a second of device time has been
          timed; the value is that of the median region, the minimum is reported beside it.
-e2e    = the same metric through spqt_sparse_linear_host_async (four calls and one wait per step; a wait after
-         every call is reported beside it): x copied from pinned host memory,
+e2e    = the same metric through spqt_host_step_launch (the step's four host-buffer linears recorded once and
+         replayed with one call, one wait per step; four asynchronous calls, and a wait after every call, are
+         reported beside it): x copied from pinned host memory,
          y written into pinned host memory by the kernel, the copy and the final wait of every
          call inside the timed region.
 roofline.achieved = algorithmic bytes per launch of the dominant kernel (gemv_kernel, index collection
@@ -547,26 +548,37 @@ def run_ours(args):
         for nm in e2e_names:
             hosts[L][nm].x_host.copy_(torch.from_numpy(xs[site_of[nm]][0]))
 
-    def e2e_step(i, wait_per_call):
+    steps_rec = [binding.HostStep([hosts[L][nm] for nm in e2e_names], [ts[site_of[nm]][0] for nm in e2e_names])
+                 for L in range(LAYER_COPIES)]
+
+    def e2e_step(i, how):
+        if how == "recorded":
+            # the step's four linears recorded once (spqt_host_step_create), replayed with one call; one wait
+            steps_rec[i % LAYER_COPIES].launch(stream=stream)
+            stream.synchronize()
+            return
         for nm in e2e_names:
-            binding.spqt_sparse_linear_host(hosts[i % LAYER_COPIES][nm], ts[site_of[nm]][0], stream=stream, wait=wait_per_call)
-        if not wait_per_call:
+            binding.spqt_sparse_linear_host(hosts[i % LAYER_COPIES][nm], ts[site_of[nm]][0], stream=stream, wait=(how == "wait_per_call"))
+        if how == "async_calls":
             stream.synchronize()       # one wait per step: the step's four results are then in pinned host memory
 
     e2e_K = min(K, 64)
 
-    def e2e_time(wait_per_call):
+    def e2e_time(how):
         for i in range(3):
-            e2e_step(i, wait_per_call)
+            e2e_step(i, how)
         barrier()
         t0 = time.perf_counter()
         for i in range(3, 3 + e2e_K):
-            e2e_step(i, wait_per_call)
+            e2e_step(i, how)
         torch.cuda.synchronize()
         return max_over_ranks(time.perf_counter() - t0, dev)
 
-    e2e_s_per_call = e2e_time(True)
-    e2e_s = e2e_time(False)
+    e2e_s_per_call = e2e_time("wait_per_call")
+    e2e_s_async = e2e_time("async_calls")
+    e2e_s = e2e_time("recorded")
+    for r in steps_rec:
+        r.close()
     e2e_bytes = e2e_K * sum(needed_bytes_gemv(shape[nm][0], shape[nm][1], counts[0][site_of[nm]])
                             + needed_bytes_sparsify(shape[nm][1], counts[0][site_of[nm]]) for nm in e2e_names)
     h2d = sum(shape[nm][1] * 2 for nm in e2e_names)
@@ -638,8 +650,10 @@ def run_ours(args):
                              "sample": cpu["sample"], "single_thread_value": cpu1["value"]},
             "e2e": {"value": world * e2e_bytes / e2e_s / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": e2e_s / e2e_K * 1e3,
-                    "calls": "4 spqt_sparse_linear_host_async calls per step (each: copy in, one launch, result written to pinned host "
-                             "memory) and one stream synchronisation",
+                    "calls": "one spqt_host_step_launch per step (the step's four linears recorded once: per linear the copy of x from "
+                             "pinned host memory, one launch, y written into pinned host memory) and one stream synchronisation",
+                    "ms_per_step_four_async_calls_one_wait": e2e_s_async / e2e_K * 1e3,
+                    "value_four_async_calls_one_wait": world * e2e_bytes / e2e_s_async / 1e9,
                     "ms_per_step_waiting_after_every_call": e2e_s_per_call / e2e_K * 1e3,
                     "value_waiting_after_every_call": world * e2e_bytes / e2e_s_per_call / 1e9},
             "gpu_launches": launches_timed, "launches_counted_incl_warmup_capture_and_repeats": launches,

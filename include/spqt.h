@@ -193,8 +193,9 @@ spqt_status spqt_static_status(int m, int group, int* status_host, void* stream)
  * copies x_host (fp16[n]) to x_dev, runs spqt_sparsify_gemv (same results as
  * spqt_sparsify followed by spqt_sparse_gemv), copies y (fp16[m]) to y_host and
  * waits for the stream.  x_host / y_host
- * should be pinned for the copies to be asynchronous (the kernel then writes y
- * straight into y_host and the copy back is skipped); x_dev (fp16[n]), idx_dev
+ * should be pinned (then a one-CTA kernel fetches x over the bus instead of the copy
+ * engine, whose start-up latency is several times the transfer of a few KB, and the
+ * GEMV kernel writes y straight into y_host: no copy back); x_dev (fp16[n]), idx_dev
  * (int32[n]), count_dev (int32[1]) and y_dev (fp16[m]) are caller-provided
  * device staging buffers.  This entry point synchronises.
  */
@@ -215,6 +216,42 @@ spqt_status spqt_sparse_linear_host_async(const void* codes, const void* scale_z
                                           const void* x_host, float t, void* y_host,
                                           void* x_dev, int32_t* idx_dev, int32_t* count_dev, void* y_dev,
                                           void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * A token step recorded once and replayed: the host-buffer linears of a step (each described like the
+ * arguments of spqt_sparse_linear_host_async: same meaning and alignment of every field) are captured,
+ * in order, into one CUDA graph -- the transfer of every x from its x_host (all of them at the head of the
+ * step), per linear the launch that collects the indices and multiplies, and the way y reaches y_host -- so
+ * that a step costs the host one launch call.
+ *   spqt_host_step_create  : builds the graph (allocates host-side CUDA objects; not a hot-path call;
+ *                            nothing runs on the device).  The pointers, shapes and thresholds are fixed
+ *                            from here on; the CONTENTS of the x_host buffers are read at every launch.
+ *                            The linears must not share staging buffers or workspaces.  Returns a handle
+ *                            in *step; SPQT_ERR_CUDA if the capture fails, the failing linear's status if
+ *                            one of them is refused.
+ *   spqt_host_step_launch  : enqueues one replay on `stream`; asynchronous; the y_host buffers are valid
+ *                            once the caller has synchronised the stream.  One replay at a time per handle.
+ *   spqt_host_step_destroy : frees the handle (after its last replay has finished).
+ * Not thread-safe per handle.  No counterpart in the paper (its linears live inside llama.cpp's graph).
+ */
+typedef struct {
+    const void* codes;
+    const void* scale_zero;
+    int m, n, bits, group;
+    const void* x_host;
+    float t;
+    void* y_host;
+    void* x_dev;
+    int32_t* idx_dev;
+    int32_t* count_dev;
+    void* y_dev;
+    void* workspace;
+    size_t workspace_bytes;
+} spqt_host_linear;
+
+spqt_status spqt_host_step_create(const spqt_host_linear* linears, int count, void** step);
+spqt_status spqt_host_step_launch(void* step, void* stream);
+spqt_status spqt_host_step_destroy(void* step);
 
 /*
  * Tuning aid: number of CTAs of the GEMV grid (0 restores the built-in rule, one

@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libspqt.so")
 EXPORTS = (
     "spqt_status_string", "spqt_version", "spqt_packed_sizes", "spqt_pack", "spqt_unpack",
     "spqt_sparsify", "spqt_sparse_gemv", "spqt_sparse_gemv_static", "spqt_static_status", "spqt_sparsify_gemv", "spqt_dense_gemv",
-    "spqt_sparse_linear_host", "spqt_sparse_linear_host_async", "spqt_gemm_small_workspace", "spqt_sparse_gemm_small", "spqt_dense_gemm_small", "spqt_rowwise_packed_sizes", "spqt_rowwise_pack", "spqt_rowwise_dense_gemv", "spqt_kq_packed_sizes", "spqt_kq_pack", "spqt_kq_sparse_gemv", "spqt_kq_dense_gemv", "spqt_autotune", "spqt_calibrate_threshold", "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_launch_count",
+    "spqt_sparse_linear_host", "spqt_sparse_linear_host_async", "spqt_host_step_create", "spqt_host_step_launch", "spqt_host_step_destroy", "spqt_gemm_small_workspace", "spqt_sparse_gemm_small", "spqt_dense_gemm_small", "spqt_rowwise_packed_sizes", "spqt_rowwise_pack", "spqt_rowwise_dense_gemv", "spqt_kq_packed_sizes", "spqt_kq_pack", "spqt_kq_sparse_gemv", "spqt_kq_dense_gemv", "spqt_autotune", "spqt_calibrate_threshold", "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_launch_count",
 )
 
 _lib = None
@@ -67,6 +67,9 @@ def lib() -> ctypes.CDLL:
         L.spqt_sparse_linear_host.argtypes = [vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, vp,
                                               vp, vp, vp, vp, vp, sz, vp]
         L.spqt_sparse_linear_host_async.argtypes = L.spqt_sparse_linear_host.argtypes
+        L.spqt_host_step_create.argtypes = [vp, i32, ctypes.POINTER(vp)]
+        L.spqt_host_step_launch.argtypes = [vp, vp]
+        L.spqt_host_step_destroy.argtypes = [vp]
         L.spqt_gemm_small_workspace.argtypes = [i32, i32, i32, i32, ctypes.POINTER(sz)]
         L.spqt_gemm_small_workspace.restype = i32
         L.spqt_sparse_gemm_small.argtypes = [vp, vp, i32, i32, i32, i32, vp, i32, i32, ctypes.c_float, vp, vp, vp, i32, vp, sz, vp]
@@ -286,6 +289,46 @@ def spqt_sparse_linear_host(h: HostLinear, t: float, stream=None, wait: bool = T
         h.count.data_ptr(), h.y_dev.data_ptr(), h.workspace.data_ptr(), h.workspace.numel(),
         _stream(stream)), "spqt_sparse_linear_host")
     return h.y_host
+
+
+class _HostLinearDesc(ctypes.Structure):
+    _fields_ = [("codes", ctypes.c_void_p), ("scale_zero", ctypes.c_void_p), ("m", ctypes.c_int), ("n", ctypes.c_int),
+                ("bits", ctypes.c_int), ("group", ctypes.c_int), ("x_host", ctypes.c_void_p), ("t", ctypes.c_float),
+                ("y_host", ctypes.c_void_p), ("x_dev", ctypes.c_void_p), ("idx_dev", ctypes.c_void_p),
+                ("count_dev", ctypes.c_void_p), ("y_dev", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
+                ("workspace_bytes", ctypes.c_size_t)]
+
+
+class HostStep:
+    """The host-buffer linears of a token step (``HostLinear`` objects and their thresholds) recorded once by
+    spqt_host_step_create; :meth:`launch` replays them with one call (asynchronous: synchronise the stream before
+    reading the ``y_host`` buffers).  Keeps the ``HostLinear`` objects alive."""
+
+    def __init__(self, hs, ts):
+        self.hs = list(hs)
+        arr = (_HostLinearDesc * len(self.hs))()
+        for d, h, t in zip(arr, self.hs, ts):
+            p = h.p
+            d.codes, d.scale_zero, d.m, d.n, d.bits, d.group = p.codes.data_ptr(), p.scale_zero.data_ptr(), p.m, p.n, p.bits, p.group
+            d.x_host, d.t, d.y_host = h.x_host.data_ptr(), float(t), h.y_host.data_ptr()
+            d.x_dev, d.idx_dev, d.count_dev, d.y_dev = h.x_dev.data_ptr(), h.idx.data_ptr(), h.count.data_ptr(), h.y_dev.data_ptr()
+            d.workspace, d.workspace_bytes = h.workspace.data_ptr(), h.workspace.numel()
+        self.handle = ctypes.c_void_p(None)
+        _ok(lib().spqt_host_step_create(ctypes.cast(arr, ctypes.c_void_p), len(self.hs), ctypes.byref(self.handle)), "spqt_host_step_create")
+
+    def launch(self, stream=None) -> None:
+        _ok(lib().spqt_host_step_launch(self.handle, _stream(stream)), "spqt_host_step_launch")
+
+    def close(self) -> None:
+        if self.handle:
+            lib().spqt_host_step_destroy(self.handle)
+            self.handle = ctypes.c_void_p(None)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
 
 
 def spqt_probe_read(buf: torch.Tensor, pattern: int, moved: torch.Tensor, stream=None) -> None:

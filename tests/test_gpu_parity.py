@@ -567,6 +567,18 @@ def test_host_entry_point_matches_the_device_path():
     assert np.array_equal(h.y_host.numpy().view(np.uint16), y_dev.view(np.uint16))
     y2, _, _ = run_sparse(p, x2, t, binding.new_workspace(m, n, bits, group))
     assert np.array_equal(h2.y_host.numpy().view(np.uint16), y2.view(np.uint16))
+    # and both recorded once as a step, replayed twice with different contents of the x buffers
+    step = binding.HostStep([h, h2], [t, t])
+    for (xa, xb, ya, yb) in ((x, x2, y_dev, y2), (x2, x, y2, y_dev)):
+        h.x_host.copy_(torch.from_numpy(xa))
+        h2.x_host.copy_(torch.from_numpy(xb))
+        h.y_host.zero_()
+        h2.y_host.zero_()
+        step.launch(stream=s)
+        s.synchronize()
+        assert np.array_equal(h.y_host.numpy().view(np.uint16), ya.view(np.uint16))
+        assert np.array_equal(h2.y_host.numpy().view(np.uint16), yb.view(np.uint16))
+    step.close()
 
 
 def test_read_and_gather_probes_fetch_what_they_report():
