@@ -22,40 +22,7 @@ int sm_count()
     return cached[dev];
 }
 
-}  // namespace spqt
-
-extern "C" {
-
-const char* spqt_status_string(int s)
-{
-    switch (s) {
-        case SPQT_OK: return "SPQT_OK";
-        case SPQT_ERR_INVALID_ARG: return "SPQT_ERR_INVALID_ARG";
-        case SPQT_ERR_UNSUPPORTED: return "SPQT_ERR_UNSUPPORTED";
-        case SPQT_ERR_ALIGNMENT: return "SPQT_ERR_ALIGNMENT";
-        case SPQT_ERR_WORKSPACE: return "SPQT_ERR_WORKSPACE";
-        case SPQT_ERR_CUDA: return "SPQT_ERR_CUDA";
-        case SPQT_ERR_TIMEOUT: return "SPQT_ERR_TIMEOUT";
-        default: return "SPQT_ERR_UNKNOWN";
-    }
-}
-
-int spqt_version(void) { return 2000; }
-
-spqt_status spqt_packed_sizes(int m, int n, int bits, int group,
-                              size_t* codes_bytes, size_t* scale_zero_bytes,
-                              size_t* gemv_workspace_bytes)
-{
-    spqt::Format f;
-    spqt_status st = spqt::make_format(m, n, bits, group, &f);
-    if (st != SPQT_OK) return st;
-    if (codes_bytes) *codes_bytes = f.blocks * (size_t)f.B;
-    if (scale_zero_bytes) *scale_zero_bytes = f.blocks * 4;
-    if (gemv_workspace_bytes) *gemv_workspace_bytes = spqt::workspace_bytes(f);
-    return SPQT_OK;
-}
-
-unsigned long long spqt_launch_count(void) { return spqt::g_launches.load(std::memory_order_relaxed); }
+// ---------------------------------------------------------------- host-buffer path
 
 // x from pinned host memory into its device staging buffer by a kernel (one CTA): for the few KB of a hidden
 // state the copy engine's start-up latency is several times the transfer, while a kernel's loads over the bus
@@ -118,9 +85,9 @@ static spqt_status launch_fetch(const FetchList& fl, int count, cudaStream_t s)
     la[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     la[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = la;
-    cfg.numAttrs = spqt::g_no_pdl ? 0 : 1;
+    cfg.numAttrs = g_no_pdl ? 0 : 1;
     if (cudaLaunchKernelEx(&cfg, fetch_x_kernel, fl) != cudaSuccess) return SPQT_ERR_CUDA;
-    spqt::count_launch();
+    count_launch();
     return SPQT_OK;
 }
 
@@ -130,8 +97,8 @@ static spqt_status linear_host(const void* codes, const void* scale_zero, int m,
                                void* workspace, size_t workspace_bytes, void* stream, bool wait, bool x_in_place = false)
 {
     if (!x_host || !y_host || !x_dev || !y_dev) return SPQT_ERR_INVALID_ARG;
-    spqt::Format f;
-    spqt_status st = spqt::make_format(m, n, bits, group, &f);
+    Format f;
+    spqt_status st = make_format(m, n, bits, group, &f);
     if (st != SPQT_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // x: fetched by a small kernel if x_host is pinned memory the device can address, by a copy otherwise
@@ -162,13 +129,53 @@ static spqt_status linear_host(const void* codes, const void* scale_zero, int m,
     return SPQT_OK;
 }
 
+struct HostStep {
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t exec = nullptr;
+};
+
+}  // namespace spqt
+
+extern "C" {
+
+const char* spqt_status_string(int s)
+{
+    switch (s) {
+        case SPQT_OK: return "SPQT_OK";
+        case SPQT_ERR_INVALID_ARG: return "SPQT_ERR_INVALID_ARG";
+        case SPQT_ERR_UNSUPPORTED: return "SPQT_ERR_UNSUPPORTED";
+        case SPQT_ERR_ALIGNMENT: return "SPQT_ERR_ALIGNMENT";
+        case SPQT_ERR_WORKSPACE: return "SPQT_ERR_WORKSPACE";
+        case SPQT_ERR_CUDA: return "SPQT_ERR_CUDA";
+        case SPQT_ERR_TIMEOUT: return "SPQT_ERR_TIMEOUT";
+        default: return "SPQT_ERR_UNKNOWN";
+    }
+}
+
+int spqt_version(void) { return 2000; }
+
+spqt_status spqt_packed_sizes(int m, int n, int bits, int group,
+                              size_t* codes_bytes, size_t* scale_zero_bytes,
+                              size_t* gemv_workspace_bytes)
+{
+    spqt::Format f;
+    spqt_status st = spqt::make_format(m, n, bits, group, &f);
+    if (st != SPQT_OK) return st;
+    if (codes_bytes) *codes_bytes = f.blocks * (size_t)f.B;
+    if (scale_zero_bytes) *scale_zero_bytes = f.blocks * 4;
+    if (gemv_workspace_bytes) *gemv_workspace_bytes = spqt::workspace_bytes(f);
+    return SPQT_OK;
+}
+
+unsigned long long spqt_launch_count(void) { return spqt::g_launches.load(std::memory_order_relaxed); }
+
 spqt_status spqt_sparse_linear_host(const void* codes, const void* scale_zero,
                                     int m, int n, int bits, int group,
                                     const void* x_host, float t, void* y_host,
                                     void* x_dev, int32_t* idx_dev, int32_t* count_dev, void* y_dev,
                                     void* workspace, size_t workspace_bytes, void* stream)
 {
-    return linear_host(codes, scale_zero, m, n, bits, group, x_host, t, y_host, x_dev, idx_dev, count_dev, y_dev,
+    return spqt::linear_host(codes, scale_zero, m, n, bits, group, x_host, t, y_host, x_dev, idx_dev, count_dev, y_dev,
                        workspace, workspace_bytes, stream, true);
 }
 
@@ -178,16 +185,10 @@ spqt_status spqt_sparse_linear_host_async(const void* codes, const void* scale_z
                                           void* x_dev, int32_t* idx_dev, int32_t* count_dev, void* y_dev,
                                           void* workspace, size_t workspace_bytes, void* stream)
 {
-    return linear_host(codes, scale_zero, m, n, bits, group, x_host, t, y_host, x_dev, idx_dev, count_dev, y_dev,
+    return spqt::linear_host(codes, scale_zero, m, n, bits, group, x_host, t, y_host, x_dev, idx_dev, count_dev, y_dev,
                        workspace, workspace_bytes, stream, false);
 }
 
-namespace {
-struct HostStep {
-    cudaGraph_t graph = nullptr;
-    cudaGraphExec_t exec = nullptr;
-};
-}  // namespace
 
 spqt_status spqt_host_step_create(const spqt_host_linear* linears, int count, void** step)
 {
@@ -196,18 +197,18 @@ spqt_status spqt_host_step_create(const spqt_host_linear* linears, int count, vo
     cudaStream_t s = nullptr;
     if (cudaStreamCreateWithFlags(&s, cudaStreamNonBlocking) != cudaSuccess) return SPQT_ERR_CUDA;
     spqt_status st = SPQT_OK;
-    HostStep* h = new HostStep();
+    spqt::HostStep* h = new spqt::HostStep();
     if (cudaStreamBeginCapture(s, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
         st = SPQT_ERR_CUDA;
     } else {
         // every x the device can reach is fetched at the head of the step (one CTA per vector), so that the
         // linears then follow one another without a transfer in between
         bool* fetched = new bool[count]();
-        FetchList fl = {};
+        spqt::FetchList fl = {};
         int k = 0;
         for (int i = 0; i < count && st == SPQT_OK; ++i) {
             const spqt_host_linear& l = linears[i];
-            void* xv = (l.x_host && l.x_dev && l.n > 0) ? device_view(l.x_host) : nullptr;
+            void* xv = (l.x_host && l.x_dev && l.n > 0) ? spqt::device_view(l.x_host) : nullptr;
             if (xv) {
                 fl.src[k] = static_cast<const unsigned short*>(xv);
                 fl.dst[k] = static_cast<unsigned short*>(l.x_dev);
@@ -215,14 +216,14 @@ spqt_status spqt_host_step_create(const spqt_host_linear* linears, int count, vo
                 fetched[i] = true;
                 ++k;
             }
-            if (k == kFetchMax || (i == count - 1 && k > 0)) {
-                st = launch_fetch(fl, k, s);
+            if (k == spqt::kFetchMax || (i == count - 1 && k > 0)) {
+                st = spqt::launch_fetch(fl, k, s);
                 k = 0;
             }
         }
         for (int i = 0; i < count && st == SPQT_OK; ++i) {
             const spqt_host_linear& l = linears[i];
-            st = linear_host(l.codes, l.scale_zero, l.m, l.n, l.bits, l.group, l.x_host, l.t, l.y_host, l.x_dev, l.idx_dev,
+            st = spqt::linear_host(l.codes, l.scale_zero, l.m, l.n, l.bits, l.group, l.x_host, l.t, l.y_host, l.x_dev, l.idx_dev,
                              l.count_dev, l.y_dev, l.workspace, l.workspace_bytes, s, false, fetched[i]);
         }
         delete[] fetched;
@@ -246,14 +247,14 @@ spqt_status spqt_host_step_create(const spqt_host_linear* linears, int count, vo
 spqt_status spqt_host_step_launch(void* step, void* stream)
 {
     if (!step) return SPQT_ERR_INVALID_ARG;
-    HostStep* h = static_cast<HostStep*>(step);
+    spqt::HostStep* h = static_cast<spqt::HostStep*>(step);
     return cudaGraphLaunch(h->exec, static_cast<cudaStream_t>(stream)) == cudaSuccess ? SPQT_OK : SPQT_ERR_CUDA;
 }
 
 spqt_status spqt_host_step_destroy(void* step)
 {
     if (!step) return SPQT_ERR_INVALID_ARG;
-    HostStep* h = static_cast<HostStep*>(step);
+    spqt::HostStep* h = static_cast<spqt::HostStep*>(step);
     (void)cudaGraphExecDestroy(h->exec);
     (void)cudaGraphDestroy(h->graph);
     delete h;
