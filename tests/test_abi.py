@@ -123,3 +123,12 @@ def test_sizes_and_refusals_of_the_rowwise_and_two_level_entries(L):
     assert L.spqt_kq_pack(None, 256, 8, 8, None, None) == 1
     assert L.spqt_kq_dense_gemv(None, 256, 8, None, None, None, 0, None) == 1
     assert L.spqt_kq_sparse_gemv(None, 256, 8, None, None, None, None, None, 0, None) == 1
+
+
+def test_host_step_refuses_bad_arguments_without_touching_the_device(L):
+    handle = ctypes.c_void_p(None)
+    assert L.spqt_host_step_create(None, 1, ctypes.byref(handle)) == 1
+    assert L.spqt_host_step_create(ctypes.c_void_p(16), 0, ctypes.byref(handle)) == 1
+    assert L.spqt_host_step_create(ctypes.c_void_p(16), 1, None) == 1
+    assert L.spqt_host_step_launch(None, None) == 1
+    assert L.spqt_host_step_destroy(None) == 1
