@@ -255,6 +255,14 @@ def rowwise_dense_gemv(q, scales, zeros, x, group: int = 128):
     return What @ xv, np.abs(What) @ np.abs(xv)
 
 
+def rowwise_thresholded_gemv(q, scales, zeros, x, t: float, group: int = 128):
+    """The row-wise product over the active entries only: |x[k]| > t (NaN never active); the others count as zero."""
+    xv = np.asarray(x, dtype=np.float16).astype(np.float64)
+    with np.errstate(invalid="ignore"):
+        active = np.abs(xv) > float(t)
+    return rowwise_dense_gemv(q, scales, zeros, np.where(active, xv, 0.0).astype(np.float16), group)
+
+
 # ---------------------------------------------------------------- two-level ("K-quant"-style) format
 #
 # The format the paper's implementation builds on (Sec. 2): superblocks of 256 weights split into eight

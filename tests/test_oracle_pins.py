@@ -467,6 +467,19 @@ def test_rowwise_hand_example():
     assert bound[0] == 0.5 + 0.25 + 3.75
 
 
+def test_rowwise_thresholded_product_drops_exactly_the_inactive_entries():
+    W = np.array([[0.0, 0.25, 0.5, 3.75], [1.0, 2.0, 3.0, 4.0]], dtype=np.float16)
+    q, s, z = oracle.rowwise_quantize(W, 4, 4)
+    x = np.array([1.0, -2.0, 0.5, np.nan], dtype=np.float16)
+    y, bound = oracle.rowwise_thresholded_gemv(q, s, z, x, 0.75, 4)          # active: columns 0 and 1
+    assert y[0] == 0.0 * 1 + 0.25 * -2 and bound[0] == 0.5
+    s1 = 0.199951171875
+    assert y[1] == (1 + 0 * s1) * 1 + (1 + 5 * s1) * -2
+    y0, _ = oracle.rowwise_thresholded_gemv(q, s, z, np.array([1.0, -2.0, 0.5, 0.0], np.float16), -1.0, 4)
+    yd, _ = oracle.rowwise_dense_gemv(q, s, z, np.array([1.0, -2.0, 0.5, 0.0], np.float16), 4)
+    assert np.array_equal(y0, yd)
+
+
 def test_rowwise_quantizer_brute_force():
     # per row and per group of consecutive columns, the quantizer's steps in numpy float32
     rng = np.random.default_rng(11)
