@@ -322,6 +322,15 @@ spqt_status spqt_rowwise_pack(const void* W, int m, int n, int ldw, int bits, in
 spqt_status spqt_rowwise_dense_gemv(const void* codes, const void* scale_zero,
                                     int m, int n, int bits, int group,
                                     const void* x, void* y, void* stream);
+/*
+ * The same product with the entries at or below the threshold treated as zero (|x[k]| > t is active, as in
+ * spqt_sparsify; NaN is never active): what activation sparsity can do on the row-wise layout, where a
+ * sparse column is scattered over a group of every row (paper Sec. 2, Sec. 4.1.1) -- no block can be
+ * skipped, every byte is still read, only the contributions vanish.  Same arguments and limits.
+ */
+spqt_status spqt_rowwise_thresholded_gemv(const void* codes, const void* scale_zero,
+                                          int m, int n, int bits, int group,
+                                          const void* x, float t, void* y, void* stream);
 
 /*
  * The two-level format the paper's implementation builds on (paper Sec. 2: superblocks of 256 weights

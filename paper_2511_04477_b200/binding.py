@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libspqt.so")
 EXPORTS = (
     "spqt_status_string", "spqt_version", "spqt_packed_sizes", "spqt_pack", "spqt_unpack",
     "spqt_sparsify", "spqt_sparse_gemv", "spqt_sparse_gemv_static", "spqt_static_status", "spqt_sparsify_gemv", "spqt_dense_gemv",
-    "spqt_sparse_linear_host", "spqt_sparse_linear_host_async", "spqt_host_step_create", "spqt_host_step_launch", "spqt_host_step_destroy", "spqt_gemm_small_workspace", "spqt_sparse_gemm_small", "spqt_dense_gemm_small", "spqt_rowwise_packed_sizes", "spqt_rowwise_pack", "spqt_rowwise_dense_gemv", "spqt_kq_packed_sizes", "spqt_kq_pack", "spqt_kq_sparse_gemv", "spqt_kq_dense_gemv", "spqt_autotune", "spqt_calibrate_threshold", "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_launch_count",
+    "spqt_sparse_linear_host", "spqt_sparse_linear_host_async", "spqt_host_step_create", "spqt_host_step_launch", "spqt_host_step_destroy", "spqt_gemm_small_workspace", "spqt_sparse_gemm_small", "spqt_dense_gemm_small", "spqt_rowwise_packed_sizes", "spqt_rowwise_pack", "spqt_rowwise_dense_gemv", "spqt_rowwise_thresholded_gemv", "spqt_kq_packed_sizes", "spqt_kq_pack", "spqt_kq_sparse_gemv", "spqt_kq_dense_gemv", "spqt_autotune", "spqt_calibrate_threshold", "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_launch_count",
 )
 
 _lib = None
@@ -60,6 +60,7 @@ def lib() -> ctypes.CDLL:
         L.spqt_rowwise_packed_sizes.argtypes = [i32, i32, i32, i32] + [ctypes.POINTER(sz)] * 2
         L.spqt_rowwise_pack.argtypes = [vp, i32, i32, i32, i32, i32, vp, vp, vp]
         L.spqt_rowwise_dense_gemv.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp]
+        L.spqt_rowwise_thresholded_gemv.argtypes = [vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, vp, vp]
         L.spqt_kq_packed_sizes.argtypes = [i32, i32] + [ctypes.POINTER(sz)] * 2
         L.spqt_kq_pack.argtypes = [vp, i32, i32, i32, vp, vp]
         L.spqt_kq_sparse_gemv.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, sz, vp]
@@ -484,6 +485,15 @@ def spqt_kq_dense_gemv(p: KqPacked, x: torch.Tensor, workspace: torch.Tensor, y:
     _ok(lib().spqt_kq_dense_gemv(
         _dev(p.records, torch.uint8, "records"), p.m, p.n, _dev(x, torch.float16, "x"), _dev(y, torch.float16, "y"),
         _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)), "spqt_kq_dense_gemv")
+    return y
+
+
+def spqt_rowwise_thresholded_gemv(p: RowwisePacked, x: torch.Tensor, t: float, y: torch.Tensor = None, stream=None) -> torch.Tensor:
+    if y is None:
+        y = torch.empty(p.m, dtype=torch.float16, device=x.device)
+    _ok(lib().spqt_rowwise_thresholded_gemv(
+        _dev(p.codes, torch.uint8, "codes"), _dev(p.scale_zero, torch.float16, "scale_zero"), p.m, p.n, p.bits, p.group,
+        _dev(x, torch.float16, "x"), float(t), _dev(y, torch.float16, "y"), _stream(stream)), "spqt_rowwise_thresholded_gemv")
     return y
 
 

@@ -138,7 +138,7 @@ __device__ __forceinline__ float reduce_rows(const float* v, int lane, int* row)
 template <int G, int ROWS>
 __global__ void __launch_bounds__(kRwThreads, 1)
 rowwise_gemv_kernel(const uint8_t* __restrict__ codes, const unsigned* __restrict__ meta, int m, int n,
-                    const __half* __restrict__ x, __half* __restrict__ y, int Wc, int Rg)
+                    const __half* __restrict__ x, __half* __restrict__ y, int Wc, int Rg, int sparse, float thr)
 {
     using Smem = RwSmem<G, ROWS>;
     constexpr int B = G / 2, NG = Smem::NG, D = kRwDepth;
@@ -222,7 +222,13 @@ rowwise_gemv_kernel(const uint8_t* __restrict__ codes, const unsigned* __restric
         }
 #pragma unroll
         for (int t = 0; t < 16; ++t) {
-            const float fl = __half2float(__ushort_as_half(xl[t])), fh = __half2float(__ushort_as_half(xh[t]));
+            // the thresholded call: entries with |x| <= threshold (and NaN) count as zero -- the row-wise
+            // layout cannot skip their bytes, only their contribution
+            float fl = __half2float(__ushort_as_half(xl[t])), fh = __half2float(__ushort_as_half(xh[t]));
+            if (sparse) {
+                fl = fabsf(fl) > thr ? fl : 0.0f;
+                fh = fabsf(fh) > thr ? fh : 0.0f;
+            }
             xs += fl + fh;
             // nibble positions of byte t inside its 32-bit word (after the shift by 16 for bytes 2 and 3):
             // bits 0 and 4 (even byte) or 8 and 12 (odd byte); multiplier = x * 2^(93 - position)
@@ -306,7 +312,7 @@ static spqt_status rowwise_format(int m, int n, int bits, int group)
 
 template <int G, int ROWS>
 static spqt_status launch_rowwise(const void* codes, const void* meta, int m, int n, const void* x, void* y,
-                                  int Wc, int Rg, int sms, cudaStream_t s)
+                                  int Wc, int Rg, int sms, int sparse, float thr, cudaStream_t s)
 {
     auto kernel = rowwise_gemv_kernel<G, ROWS>;
     static bool configured[64] = {};
@@ -331,13 +337,14 @@ static spqt_status launch_rowwise(const void* codes, const void* meta, int m, in
     cfg.attrs = attr;
     cfg.numAttrs = g_no_pdl ? 0 : 1;
     const cudaError_t err = cudaLaunchKernelEx(&cfg, kernel, static_cast<const uint8_t*>(codes), static_cast<const unsigned*>(meta),
-                                               m, n, static_cast<const __half*>(x), static_cast<__half*>(y), Wc, Rg);
+                                               m, n, static_cast<const __half*>(x), static_cast<__half*>(y), Wc, Rg, sparse, thr);
     count_launch();
     return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SPQT_OK : SPQT_ERR_CUDA;
 }
 
 template <int G>
-static spqt_status dispatch_rowwise(const void* codes, const void* meta, int m, int n, const void* x, void* y, cudaStream_t s)
+static spqt_status dispatch_rowwise(const void* codes, const void* meta, int m, int n, const void* x, void* y, int sparse, float thr,
+                                    cudaStream_t s)
 {
     const int sms = sm_count();
     if (sms <= 0) return SPQT_ERR_CUDA;
@@ -346,9 +353,9 @@ static spqt_status dispatch_rowwise(const void* codes, const void* meta, int m, 
     if (Wc > 1 && Rg > 8) Rg = 8;
     // the largest chunk of rows that still gives every row group of a full grid a chunk
     const long long groups = (long long)sms * Rg;
-    if ((m + 7) / 8 >= groups) return launch_rowwise<G, 8>(codes, meta, m, n, x, y, Wc, Rg, sms, s);
-    if ((m + 3) / 4 >= groups) return launch_rowwise<G, 4>(codes, meta, m, n, x, y, Wc, Rg, sms, s);
-    return launch_rowwise<G, 2>(codes, meta, m, n, x, y, Wc, Rg, sms, s);
+    if ((m + 7) / 8 >= groups) return launch_rowwise<G, 8>(codes, meta, m, n, x, y, Wc, Rg, sms, sparse, thr, s);
+    if ((m + 3) / 4 >= groups) return launch_rowwise<G, 4>(codes, meta, m, n, x, y, Wc, Rg, sms, sparse, thr, s);
+    return launch_rowwise<G, 2>(codes, meta, m, n, x, y, Wc, Rg, sms, sparse, thr, s);
 }
 
 }  // namespace spqt
@@ -386,8 +393,8 @@ spqt_status spqt_rowwise_pack(const void* W, int m, int n, int ldw, int bits, in
     return cudaGetLastError() == cudaSuccess ? SPQT_OK : SPQT_ERR_CUDA;
 }
 
-spqt_status spqt_rowwise_dense_gemv(const void* codes, const void* scale_zero, int m, int n, int bits, int group,
-                                    const void* x, void* y, void* stream)
+static spqt_status rowwise_entry(const void* codes, const void* scale_zero, int m, int n, int bits, int group,
+                                 const void* x, void* y, int sparse, float t, void* stream)
 {
     if (!codes || !scale_zero || !x || !y) return SPQT_ERR_INVALID_ARG;
     const spqt_status st = spqt::rowwise_format(m, n, bits, group);
@@ -396,8 +403,20 @@ spqt_status spqt_rowwise_dense_gemv(const void* codes, const void* scale_zero, i
     if (!spqt::aligned(codes, 16) || !spqt::aligned(scale_zero, 16) || !spqt::aligned(x, 2) || !spqt::aligned(y, 2))
         return SPQT_ERR_ALIGNMENT;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    return group == 128 ? spqt::dispatch_rowwise<128>(codes, scale_zero, m, n, x, y, s)
-                        : spqt::dispatch_rowwise<64>(codes, scale_zero, m, n, x, y, s);
+    return group == 128 ? spqt::dispatch_rowwise<128>(codes, scale_zero, m, n, x, y, sparse, t, s)
+                        : spqt::dispatch_rowwise<64>(codes, scale_zero, m, n, x, y, sparse, t, s);
+}
+
+spqt_status spqt_rowwise_dense_gemv(const void* codes, const void* scale_zero, int m, int n, int bits, int group,
+                                    const void* x, void* y, void* stream)
+{
+    return rowwise_entry(codes, scale_zero, m, n, bits, group, x, y, 0, 0.0f, stream);
+}
+
+spqt_status spqt_rowwise_thresholded_gemv(const void* codes, const void* scale_zero, int m, int n, int bits, int group,
+                                          const void* x, float t, void* y, void* stream)
+{
+    return rowwise_entry(codes, scale_zero, m, n, bits, group, x, y, 1, t, stream);
 }
 
 }  // extern "C"

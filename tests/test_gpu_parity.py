@@ -900,6 +900,16 @@ def test_rowwise_baseline_pack_and_dense_gemv_match_the_oracle(group, m, n):
     y2 = binding.spqt_rowwise_dense_gemv(p, dev(x))
     torch.cuda.synchronize()
     assert torch.equal(y.view(torch.int16), y2.view(torch.int16))             # fixed order of sums
+    # thresholded: the inactive entries (and a NaN) contribute nothing
+    xs = x.copy()
+    if n > 100:
+        xs[5] = np.float16(np.nan)
+    for sp in (0.5, 0.0):
+        t = inputs.threshold_for_sparsity(x, sp)
+        yt = binding.spqt_rowwise_thresholded_gemv(p, dev(xs), t)
+        torch.cuda.synchronize()
+        yt_ref, tb = oracle.rowwise_thresholded_gemv(q, s, z, xs, t, group)
+        check_y(yt.cpu().numpy(), yt_ref, tb, "row-wise thresholded %dx%d g%d sparsity %r" % (m, n, group, sp))
 
 
 @pytest.mark.parametrize("group", [128, 64])
