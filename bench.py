@@ -260,6 +260,8 @@ def other_config_line(which, local, quick=False):
                                             "and the built-in rule; beside it the row-wise-layout baseline (spqt_rowwise_dense_gemv) on the same shapes; rotated weight copies > 2x L2"},
                         roofline=roofline_obj(best["dense_gbs"], peak, kind, nb, best["best_us"], "gemv_kernel<128,4,dense>", 1.0),
                         zigzag_dense_vs_rowwise={"%dx%d" % (r["m"], r["n"]): r["zigzag_dense_vs_rowwise"] for r in rows},
+                        speedup_from_50pct_sparsity={"%dx%d" % (r["m"], r["n"]): {"rowwise_layout": r["rowwise_sparse_speedup_over_its_dense"],
+                                                                                    "zigzag_layout": r["zigzag_sparse_speedup_over_its_dense"]} for r in rows},
                         rows=rows)
         elif which == "models":
             rows = sweep.model_shapes_sweep(peak)

@@ -200,6 +200,20 @@ def dense_shape_sweep(peak):
             row["rowwise_gbs"] = needed_bytes(m, n, n, 4, 128) / us_rw * 1e-3
             row["rowwise_frac_of_peak"] = row["rowwise_gbs"] / peak
             row["zigzag_dense_vs_rowwise"] = us_rw / row["us_ctas_0"]
+            # activation sparsity on each layout at 50 %: the row-wise kernel with the inactive entries zeroed
+            # (it reads every byte), the zigzag kernel over the list (collected in the same launch)
+            x50 = inputs.activations(n, seed=11)
+            t50 = inputs.threshold_for_sparsity(x50, 0.5)
+            us_rw_t, _ = graph_us(lambda i, s: binding.spqt_rowwise_thresholded_gemv(rw[i % copies], xd, t50, y, stream=s), calls, replays=10)
+            zz = make_copies(m, n, 4, 128, copies)
+            idx = torch.empty(n, dtype=torch.int32, device="cuda")
+            cnt = torch.zeros(1, dtype=torch.int32, device="cuda")
+            us_zz_s, _ = graph_us(lambda i, s: binding.spqt_sparsify_gemv(zz[i % copies], xd, t50, ws, idx, cnt, y, stream=s), calls, replays=10)
+            del zz
+            row["rowwise_thresholded_us"] = us_rw_t
+            row["rowwise_sparse_speedup_over_its_dense"] = us_rw / us_rw_t
+            row["zigzag_sparse_us"] = us_zz_s
+            row["zigzag_sparse_speedup_over_its_dense"] = row["us_ctas_0"] / us_zz_s
             out.append(row)
             del rw
             torch.cuda.empty_cache()
