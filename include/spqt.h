@@ -226,7 +226,9 @@ spqt_status spqt_sparse_linear_host_async(const void* codes, const void* scale_z
  *   spqt_host_step_create  : builds the graph (allocates host-side CUDA objects; not a hot-path call;
  *                            nothing runs on the device).  The pointers, shapes and thresholds are fixed
  *                            from here on; the CONTENTS of the x_host buffers are read at every launch.
- *                            The linears must not share staging buffers or workspaces.  Returns a handle
+ *                            The linears must not share staging buffers or workspaces; x_host and y_host
+ *                            must be pinned memory (a copy from pageable memory cannot be recorded:
+ *                            SPQT_ERR_CUDA).  Returns a handle
  *                            in *step; SPQT_ERR_CUDA if the capture fails, the failing linear's status if
  *                            one of them is refused.
  *   spqt_host_step_launch  : enqueues one replay on `stream`; asynchronous; the y_host buffers are valid
