@@ -37,22 +37,26 @@
 //            dense call instead fetches the chunk's codes, pairs and x values with
 //            three bulk copies issued by one lane (they are contiguous).
 //   consume  lane e turns its pair into a = x_k*scale (exact in fp32) and
-//            x_k*zero, writes the two packed multiplier pairs of its entry to
+//            x_k*zero, writes the packed multiplier pair of its entry to
 //            shared memory; then every lane does the dequantize-FMA work on its 16
-//            bytes of each block, reading the block's multipliers back.
+//            codes of each block, reading the block's multiplier back.
 // Entries past the end of a part are clamped to its last entry with weight 0, and
 // the 512-byte steps of a chunk that hold no entry are skipped.  Two more warps,
 // the writers (one per hand-over buffer), add the workers' sums at the end of a
 // segment, publish the partial and, if this CTA is the last contributor of the
-// block-row, produce y; their waits on shared-memory barriers are bounded in wall
-// time (on expiry the workspace's status word is set and the kernel returns).
+// block-row, produce y; they wait for the workers at a hardware barrier and for
+// other CTAs with waits bounded in wall time (on expiry the workspace's status word
+// is set and the kernel returns).
 //
 // Arithmetic:  y[j] = sum_k a_k * code_jk + sum_k x_k * zero_rk.  A 4-bit code
-// becomes an fp32 operand with no conversion: the nibble masked in place at bit
-// p of an otherwise zero word IS the fp32 subnormal code*2^(p-149); the matching
-// multiplier a*2^(93-p) is an exact power-of-two rescale, so each product is
-// a*code*2^-56 up to the single rounding of the FMA.  One logic op and one FMA
-// per weight; two FMAs are issued as one packed fma.rn.f32x2.
+// becomes an fp32 operand with no conversion: a word whose bits above bit 22 are
+// zero IS an fp32 subnormal, its integer value times 2^-149, and the multiplier
+// a*2^93 is an exact power-of-two rescale, so each product is a*value*2^-56 up to
+// the single rounding of the FMA.  Per 16-bit half-word the operands are its low
+// 4, 8, 12 and 16 bits (u_j = q_0 + 16 q_1 + ... + 16^j q_j: three masks, the last
+// needs none); the sums over the list are linear in them, so the per-code sums
+// come back at the end of a segment as (U_j - U_{j-1}) / 16^j.  Under one logic op
+// and one FMA per weight; two FMAs are issued as one packed fma.rn.f32x2.
 #include <cstddef>
 
 #include "spqt_common.cuh"
@@ -111,7 +115,7 @@ struct GemvSmem {
         alignas(16) unsigned xc[CH];              // list calls: the entry word; dense call: CH fp16 values of x
     };
     Stage stage[kWorkers][kDepth];                 // (the prologue borrows this area for its copy of x and its masks)
-    alignas(16) float mult[kWorkers][CH][4];       // packed multiplier pairs of the chunk in work
+    alignas(16) float mult[kWorkers][CH][2];       // packed multiplier pair (a, a) * 2^93 of every entry of the chunk in work
     alignas(16) float red[2][kWorkers][G];         // per-warp partial sums of a finished segment
     float red_z[2][kWorkers];                      // and their offset terms
     alignas(8) uint64_t full[kWorkers][kDepth];    // dense call: completion of a stage's bulk copies
@@ -536,8 +540,7 @@ gemv_kernel(const GemvArgs a)
                     for (int j = 0; j < kSpec; ++j) oz[j] = __shfl_sync(0xffffffffu, oz[j], 0);
                 }
             }
-            ok = mbar_wait(&sm.red_full[b], (sg >> 1) & 1);
-            if (!ok) break;
+            handover_wait(b, (kWorkers + 1) * 32);
             float v[RPL];
 #pragma unroll
             for (int i = 0; i < RPL; ++i) v[i] = 0.0f;
@@ -806,8 +809,8 @@ gemv_kernel(const GemvArgs a)
     for (int i = 0; i < 8; ++i) acc[i] = 0ull;
     float zl = 0.0f;     // this lane's share of sum x_k * zero_rk of the current segment
 
-    // PREP: lane e turns the pair of its entry into a = x_k*scale (exact in fp32), written as two packed
-    // multiplier pairs, and adds x_k*zero to its share of the offset term
+    // PREP: lane e turns the pair of its entry into a = x_k*scale (exact in fp32), written as the packed
+    // multiplier pair (a, a) * 2^93, and adds x_k*zero to its share of the offset term
     auto prep = [&](unsigned st_addr, int pos, int valid, bool full) {
         unsigned ev[EPL];
         if (!DENSE) load_entries(pos, valid, full, ev);
@@ -827,24 +830,23 @@ gemv_kernel(const GemvArgs a)
             }
             zl += zt;
             const unsigned long long aa = pack2(am, am);
-            sts_pairs(mult_base + 16u * e, fmul2(aa, pack2(0x1p93f, 0x1p89f)), fmul2(aa, pack2(0x1p85f, 0x1p81f)));
+            sts_u64(mult_base + 8u * e, fmul2(aa, pack2(0x1p93f, 0x1p93f)));
         }
     };
 
     // MATH: one step of a chunk: SLM blocks, each lane 16 codes of one of them
     auto step = [&](unsigned st_addr, int u) {
-        unsigned long long m01, m23;
-        lds_pairs(mult_base + 16u * (u * SLM + mslot), m01, m23);
+        const unsigned long long mm = lds_u64(mult_base + 8u * (u * SLM + mslot));
         if (BITS == 4) {
             const uint2 wv = lds_v2(st_addr + lane * 8 + u * 256);
-            fma_block8(acc, wv, m01, m23);
+            fma_block8_cum(acc, wv, mm);
         } else {
             // lane t of a block: word t of the 2-bit plane (G/16 words); its top bits are the even
             // (t < LM/2) or odd bits of word t mod LM/2 of the 1-bit plane
             const unsigned blk = st_addr + (u * SLM + mslot) * B;
             const unsigned w2 = lds_u32(blk + 4u * mh);
             const unsigned w1 = lds_u32(blk + (G / 4) + 4u * (mh % (LM / 2))) >> (mh / (LM / 2));
-            fma_block3(acc, w2, w1, m01, m23);
+            fma_block3_cum(acc, w2, w1, mm);
         }
     };
 
@@ -939,6 +941,7 @@ gemv_kernel(const GemvArgs a)
             float t8[8], t4[4], keep[4];
             halve<16>(accf, t8, lane, 16);
             halve<8>(t8, t4, lane, 8);
+            uncumulate(t4);   // the four values are the cumulative sums of one half-word
             if (LM == 8) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i) keep[i] = t4[i];
@@ -963,7 +966,8 @@ gemv_kernel(const GemvArgs a)
             if (lane == 0) sm.red_z[b][warp] = zl;
             zl = 0.0f;
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.red_full[b]);
+            if (lane == 0) mbar_arrive(&sm.red_full[b]);   // what the watching writer tests
+            handover_arrive(b, (kWorkers + 1) * 32);       // what it finally waits on
             ++sg;
         }
         wc.next_span(pc, warp, resident);

@@ -106,6 +106,22 @@ __device__ __forceinline__ void worker_barrier(int threads)
     asm volatile("bar.sync 1, %0;" ::"r"(threads) : "memory");
 }
 
+// Hand-over of a finished segment from the worker warps to its writer warp (hardware barriers 2 and
+// 3, one per hand-over buffer): the workers arrive without waiting, the writer waits.  A warp waiting
+// at a hardware barrier issues nothing, whereas a warp in mbarrier.try_wait re-tests the barrier
+// about every 60 ns (a dozen instructions each time, measured from the instruction mix) on the
+// scheduler it shares with four worker warps.  Like __syncthreads it cannot time out: every worker warp
+// passes every segment end, whatever its bounded waits returned.
+// (threads = all worker threads plus the writer's 32)
+__device__ __forceinline__ void handover_arrive(int b, int threads)
+{
+    asm volatile("bar.arrive %0, %1;" ::"r"(2 + b), "r"(threads) : "memory");
+}
+__device__ __forceinline__ void handover_wait(int b, int threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(2 + b), "r"(threads) : "memory");
+}
+
 __device__ __forceinline__ void cp_async_16(unsigned smem_dst, const void* gmem_src)
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
@@ -308,6 +324,52 @@ __device__ __forceinline__ void fma_block3(unsigned long long* acc, unsigned w2,
     const unsigned c0 = (w2 & 0x33333333u) | ((w1 << 2) & 0x44444444u);
     const unsigned c1 = ((w2 >> 2) & 0x33333333u) | (w1 & 0x44444444u);
     fma_block8(acc, make_uint2(c0, c1), m01, m23);
+}
+
+// The cumulative form of the same arithmetic, for blocks whose codes all share one multiplier a
+// (mm = (a, a) * 2^93).  Instead of the four codes q0..q3 of a 16-bit half-word, the four sums
+// u_j = q0 + 16 q1 + ... + 16^j q_j (the half-word masked to its low 4(j+1) bits, a subnormal like the
+// single codes) are accumulated: the top one needs no mask, so a word costs seven masks and a shift
+// instead of eight and a shift, and one multiplier pair instead of two.  The sums are linear in the
+// codes, so the sum over the list of a*q_j is recovered once per segment as (U_j - U_{j-1}) / 16^j;
+// every U_j is dominated by its own top code, which keeps the rounding error of that difference at
+// the level of a direct sum (a factor 1 + 1/16 + ... above it at most).
+__device__ __forceinline__ void fma_word_cum(unsigned long long* acc, unsigned w, unsigned long long mm)
+{
+    const unsigned v = w >> 16;
+    ffma2(acc[0], pack2(__uint_as_float(w & 0x0000000fu), __uint_as_float(w & 0x000000ffu)), mm);
+    ffma2(acc[1], pack2(__uint_as_float(w & 0x00000fffu), __uint_as_float(w & 0x0000ffffu)), mm);
+    ffma2(acc[2], pack2(__uint_as_float(v & 0x0000000fu), __uint_as_float(v & 0x000000ffu)), mm);
+    ffma2(acc[3], pack2(__uint_as_float(v & 0x00000fffu), __uint_as_float(v)), mm);
+}
+__device__ __forceinline__ void fma_block8_cum(unsigned long long* acc, const uint2& w, unsigned long long mm)
+{
+    fma_word_cum(acc + 0, w.x, mm);
+    fma_word_cum(acc + 4, w.y, mm);
+}
+__device__ __forceinline__ void fma_block3_cum(unsigned long long* acc, unsigned w2, unsigned w1, unsigned long long mm)
+{
+    const unsigned c0 = (w2 & 0x33333333u) | ((w1 << 2) & 0x44444444u);
+    const unsigned c1 = ((w2 >> 2) & 0x33333333u) | (w1 & 0x44444444u);
+    fma_block8_cum(acc, make_uint2(c0, c1), mm);
+}
+// u[0..3] = the four cumulative sums of one half-word -> the four code sums, each still times 2^-56
+__device__ __forceinline__ void uncumulate(float* u)
+{
+    const float s1 = (u[1] - u[0]) * 0x1p-4f, s2 = (u[2] - u[1]) * 0x1p-8f, s3 = (u[3] - u[2]) * 0x1p-12f;
+    u[1] = s1;
+    u[2] = s2;
+    u[3] = s3;
+}
+__device__ __forceinline__ unsigned long long lds_u64(unsigned addr)
+{
+    unsigned long long v;
+    asm volatile("ld.shared.u64 %0, [%1];" : "=l"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sts_u64(unsigned addr, unsigned long long v)
+{
+    asm volatile("st.shared.u64 [%0], %1;" ::"r"(addr), "l"(v) : "memory");
 }
 
 // One step of a butterfly reduce-scatter: lanes that differ in bit `bit` hold
