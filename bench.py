@@ -542,6 +542,19 @@ def run_ours(args):
                 best = max(best, float(moved.item()) / (e0.elapsed_time(e1) * 1e-3) / 1e9)
             probes[key] = best
         del buf
+        # the loop's arithmetic alone, operands in shared memory: the rate at which instruction issue saturates,
+        # expressed as the bytes per second the same number of 2 KB chunks (2176 bytes with metadata) stands for
+        sink = torch.empty(512 * torch.cuda.get_device_properties(dev).multi_processor_count, dtype=torch.float32,
+                           device=dev)
+        best = 0.0
+        for _ in range(3):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            chunks = binding.spqt_probe_arith(4000, sink)
+            e1.record()
+            e1.synchronize()
+            best = max(best, chunks * 2176.0 / (e0.elapsed_time(e1) * 1e-3) / 1e9)
+        probes["arithmetic_only_int4_g128_gbs_equivalent"] = best
 
     # ---- end to end from host buffers through the C ABI (copies + sync inside the timed region)
     e2e_names = list(stacked.values())

@@ -440,6 +440,18 @@ spqt_status spqt_workspace_status(const void* workspace, int m, int group, int* 
 spqt_status spqt_probe_read(const void* buf, size_t bytes, int pattern,
                             unsigned long long* moved, void* stream);
 
+/*
+ * Measurement aid, not part of the method: the dequantize-FMA arithmetic of the GEMV loop alone.  One
+ * CTA of 16 warps per SM; every warp runs `chunks_per_warp` (>= 1) full 2 KB chunks of 4-bit codes with
+ * groups of 128 rows (eight 512-byte steps each) on operands that already sit in shared memory: no
+ * copies, no list handling, no reduction.  `sink` (device, sink_floats >= 512 per SM or
+ * SPQT_ERR_INVALID_ARG; written so that the arithmetic is kept) receives meaningless sums; *chunks_total (host) receives the number of chunks
+ * the launch processes.  Time it with events on `stream`: chunks per second times the bytes a chunk
+ * stands for (2176 with its metadata) is the bandwidth at which instruction issue alone saturates.
+ */
+spqt_status spqt_probe_arith(int chunks_per_warp, float* sink, size_t sink_floats,
+                             unsigned long long* chunks_total, void* stream);
+
 /* Number of kernels the library has launched in this process (a counter for
  * benchmarks; not synchronised with the device). */
 unsigned long long spqt_launch_count(void);

@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libspqt.so")
 EXPORTS = (
     "spqt_status_string", "spqt_version", "spqt_packed_sizes", "spqt_pack", "spqt_unpack",
     "spqt_sparsify", "spqt_sparse_gemv", "spqt_sparse_gemv_static", "spqt_static_status", "spqt_sparsify_gemv", "spqt_dense_gemv",
-    "spqt_sparse_linear_host", "spqt_sparse_linear_host_async", "spqt_host_step_create", "spqt_host_step_launch", "spqt_host_step_destroy", "spqt_gemm_small_workspace", "spqt_sparse_gemm_small", "spqt_dense_gemm_small", "spqt_rowwise_packed_sizes", "spqt_rowwise_pack", "spqt_rowwise_dense_gemv", "spqt_rowwise_thresholded_gemv", "spqt_kq_packed_sizes", "spqt_kq_pack", "spqt_kq_sparse_gemv", "spqt_kq_dense_gemv", "spqt_autotune", "spqt_calibrate_threshold", "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_launch_count",
+    "spqt_sparse_linear_host", "spqt_sparse_linear_host_async", "spqt_host_step_create", "spqt_host_step_launch", "spqt_host_step_destroy", "spqt_gemm_small_workspace", "spqt_sparse_gemm_small", "spqt_dense_gemm_small", "spqt_rowwise_packed_sizes", "spqt_rowwise_pack", "spqt_rowwise_dense_gemv", "spqt_rowwise_thresholded_gemv", "spqt_kq_packed_sizes", "spqt_kq_pack", "spqt_kq_sparse_gemv", "spqt_kq_dense_gemv", "spqt_autotune", "spqt_calibrate_threshold", "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_probe_arith", "spqt_launch_count",
 )
 
 _lib = None
@@ -85,6 +85,8 @@ def lib() -> ctypes.CDLL:
         L.spqt_set_tuning.argtypes = [i32, i32]
         L.spqt_set_debug.argtypes = [i32]
         L.spqt_probe_read.argtypes = [vp, sz, i32, vp, vp]
+        L.spqt_probe_arith.argtypes = [i32, vp, sz, ctypes.POINTER(ctypes.c_ulonglong), vp]
+        L.spqt_probe_arith.restype = i32
         L.spqt_workspace_status.argtypes = [vp, i32, i32, ctypes.POINTER(i32), vp]
         L.spqt_launch_count.restype = ctypes.c_ulonglong
         for name in ("spqt_packed_sizes", "spqt_pack", "spqt_unpack", "spqt_sparsify",
@@ -337,6 +339,15 @@ def spqt_probe_read(buf: torch.Tensor, pattern: int, moved: torch.Tensor, stream
     half of every 128-byte line); adds the bytes fetched to `moved` (int64[1] on the device)."""
     _ok(lib().spqt_probe_read(_dev(buf, torch.uint8, "buf"), buf.numel(), int(pattern),
                               _dev(moved, torch.int64, "moved"), _stream(stream)), "spqt_probe_read")
+
+
+def spqt_probe_arith(chunks_per_warp: int, sink: torch.Tensor, stream=None) -> int:
+    """Measurement aid: the GEMV loop's arithmetic alone on shared-memory operands (16 warps per SM, `chunks_per_warp`
+    2 KB chunks each); `sink` is float32 on the device, at least 512 values per SM.  Returns the chunks processed."""
+    total = ctypes.c_ulonglong(0)
+    _ok(lib().spqt_probe_arith(int(chunks_per_warp), _dev(sink, torch.float32, "sink"), sink.numel(), ctypes.byref(total),
+                               _stream(stream)), "spqt_probe_arith")
+    return int(total.value)
 
 
 def spqt_set_debug(on: bool) -> None:

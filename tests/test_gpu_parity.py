@@ -595,6 +595,23 @@ def test_read_and_gather_probes_fetch_what_they_report():
     assert abs(int(moved.item()) - all_blocks // 2) <= all_blocks // 100
 
 
+def test_arithmetic_probe_does_the_work_it_reports():
+    """The arithmetic-only probe: chunk count as documented, sums that grow with the chunks (the arithmetic is not
+    optimised away), and a sink that is too small is refused."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    sink = torch.zeros(512 * sms, dtype=torch.float32, device="cuda")
+    assert binding.spqt_probe_arith(30, sink) == sms * 16 * 30
+    torch.cuda.synchronize()
+    a = sink.double().cpu().numpy().copy()
+    assert binding.spqt_probe_arith(60, sink) == sms * 16 * 60
+    torch.cuda.synchronize()
+    b = sink.double().cpu().numpy()
+    assert np.all(np.isfinite(a)) and np.all(a > 0)
+    assert np.allclose(b, 2 * a, rtol=1e-4)       # whole rounds of the three stages: twice the sums
+    with pytest.raises(binding.SpqtError):
+        binding.spqt_probe_arith(30, sink[: 512 * sms - 1])
+
+
 def test_kernels_are_counted():
     before = binding.spqt_launch_count()
     x = dev(inputs.activations(256, seed=1))
