@@ -46,12 +46,12 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, unsigned parity)
 }
 
 // Bounded wait for the phase with the given parity; false when the bound
-// (wall time, so that a logic error can never hold the GPU) expires.  The wait itself
-// is the hardware's: try_wait with a time hint suspends the warp until the phase
-// completes or the hint runs out, so a waiting warp issues next to no instructions
-// (a software spin on a short try_wait was measured to take more issue slots than
-// the arithmetic of the warps it shares a scheduler with).
-constexpr unsigned kSuspendNs = 100000u;  // one suspension: 0.1 ms at most
+// (wall time, so that a logic error can never hold the GPU) expires.  One try_wait
+// blocks for up to about 4 us on this GPU (with or without the time hint), re-testing
+// the barrier about every 60 ns while it does, a dozen instructions each time: far
+// fewer than a software spin on test_wait, but not nothing -- which is why the long
+// wait of the writer warps is a hardware barrier instead (handover_wait below).
+constexpr unsigned kSuspendNs = 100000u;  // the time hint of one try_wait
 __device__ __forceinline__ bool mbar_wait_addr(unsigned addr, unsigned parity)
 {
     unsigned long long t0 = 0;
