@@ -39,7 +39,7 @@ template <int G, int BITS, int ROWS>
 struct SmallSmem {
     static constexpr int B = G * BITS / 8;
     alignas(16) unsigned char codes[kSmallWarps][kSmallDepth][kSmallChunk * B];
-    alignas(16) float mult[kSmallWarps][kSmallChunk][ROWS][4];
+    alignas(16) float mult[kSmallWarps][kSmallChunk][ROWS][2];   // (a, a) * 2^93 per entry and batch row
     alignas(16) unsigned ent[kSmallWarps][kSmallDepth][kSmallChunk][ROWS + 1];  // per entry: its (scale, zero) pair and the words holding the rows' x values
     alignas(16) float red[kSmallWarps][ROWS][G];
     float red_z[kSmallWarps][ROWS];
@@ -113,7 +113,7 @@ gemm_small_kernel(const uint8_t* __restrict__ codes, const unsigned* __restrict_
     };
 
     // One step: the lane's 16 codes become eight packed operand pairs ONCE (masks and shifts), then every
-    // row of the batch multiplies them with its own multiplier pairs.
+    // row of the batch multiplies them with its own multiplier pair.
     auto step = [&](unsigned cb, int u) {
         const unsigned ent = (unsigned)(u * SLM + mslot);
         uint2 wv;
@@ -129,21 +129,21 @@ gemm_small_kernel(const uint8_t* __restrict__ codes, const unsigned* __restrict_
         unsigned long long op[8];
         {
             const unsigned w = wv.x, v = wv.x >> 16, w2b = wv.y, v2 = wv.y >> 16;
-            op[0] = pack2(__uint_as_float(w & 0x0000000fu), __uint_as_float(w & 0x000000f0u));
-            op[1] = pack2(__uint_as_float(w & 0x00000f00u), __uint_as_float(w & 0x0000f000u));
-            op[2] = pack2(__uint_as_float(v & 0x0000000fu), __uint_as_float(v & 0x000000f0u));
-            op[3] = pack2(__uint_as_float(v & 0x00000f00u), __uint_as_float(v & 0x0000f000u));
-            op[4] = pack2(__uint_as_float(w2b & 0x0000000fu), __uint_as_float(w2b & 0x000000f0u));
-            op[5] = pack2(__uint_as_float(w2b & 0x00000f00u), __uint_as_float(w2b & 0x0000f000u));
-            op[6] = pack2(__uint_as_float(v2 & 0x0000000fu), __uint_as_float(v2 & 0x000000f0u));
-            op[7] = pack2(__uint_as_float(v2 & 0x00000f00u), __uint_as_float(v2 & 0x0000f000u));
+            // the cumulative values of every half-word (its low 4, 8, 12 and 16 bits), as in the batch-1 kernel
+            op[0] = pack2(__uint_as_float(w & 0x0000000fu), __uint_as_float(w & 0x000000ffu));
+            op[1] = pack2(__uint_as_float(w & 0x00000fffu), __uint_as_float(w & 0x0000ffffu));
+            op[2] = pack2(__uint_as_float(v & 0x0000000fu), __uint_as_float(v & 0x000000ffu));
+            op[3] = pack2(__uint_as_float(v & 0x00000fffu), __uint_as_float(v));
+            op[4] = pack2(__uint_as_float(w2b & 0x0000000fu), __uint_as_float(w2b & 0x000000ffu));
+            op[5] = pack2(__uint_as_float(w2b & 0x00000fffu), __uint_as_float(w2b & 0x0000ffffu));
+            op[6] = pack2(__uint_as_float(v2 & 0x0000000fu), __uint_as_float(v2 & 0x000000ffu));
+            op[7] = pack2(__uint_as_float(v2 & 0x00000fffu), __uint_as_float(v2));
         }
 #pragma unroll
         for (int b = 0; b < ROWS; ++b) {
-            unsigned long long m01, m23;
-            lds_pairs(mbuf + 16u * (ent * ROWS + b), m01, m23);
+            const unsigned long long mm = lds_u64(mbuf + 8u * (ent * ROWS + b));
 #pragma unroll
-            for (int i = 0; i < 8; ++i) ffma2(acc[b][i], op[i], (i & 1) ? m23 : m01);
+            for (int i = 0; i < 8; ++i) ffma2(acc[b][i], op[i], mm);
         }
     };
 
@@ -186,7 +186,7 @@ gemm_small_kernel(const uint8_t* __restrict__ codes, const unsigned* __restrict_
             const int col = cols[0];
             cp_async_wait<D - 1>();   // this chunk's copies have landed (the later chunks' may still fly)
             __syncwarp();
-            // lane e: multiplier pairs of every row for its entry
+            // lane e: the multiplier pair of every row for its entry
             {
                 const bool on = pos + lane < hi;
                 const unsigned ea = ebuf + cur * kEntBytes + (unsigned)lane * (ROWS + 1) * 4u;
@@ -208,7 +208,7 @@ gemm_small_kernel(const uint8_t* __restrict__ codes, const unsigned* __restrict_
                     const float am = xf * sf;       // exact
                     zl[b] += xf * zf;               // exact product
                     const unsigned long long aa = pack2(am, am);
-                    sts_pairs(mbuf + 16u * (lane * ROWS + b), fmul2(aa, pack2(0x1p93f, 0x1p89f)), fmul2(aa, pack2(0x1p85f, 0x1p81f)));
+                    sts_u64(mbuf + 8u * (lane * ROWS + b), fmul2(aa, pack2(0x1p93f, 0x1p93f)));
                 }
             }
             __syncwarp();
@@ -240,6 +240,7 @@ gemm_small_kernel(const uint8_t* __restrict__ codes, const unsigned* __restrict_
         float t8[8], t4[4], keep[4];
         halve<16>(accf, t8, lane, 16);
         halve<8>(t8, t4, lane, 8);
+        uncumulate(t4);
         if (LM == 8) {
 #pragma unroll
             for (int i = 0; i < 4; ++i) keep[i] = t4[i];
