@@ -282,13 +282,20 @@ def rowwise_thresholded_gemv(q, scales, zeros, x, t: float, group: int = 128):
 # Record of a superblock (G = sub*nsub weights): G/2 bytes of codes (byte i = q_i | q_{i+G/2} << 4), then the
 # 2*nsub six-bit fields sc_0.., m_0.. as a little-endian bit string (field f at bits 6f..6f+5) padded to whole
 # bytes, then d and dmin as little-endian fp16: 128 + 12 + 4 = 144 bytes for sub = 32, nsub = 8.
+# Other code widths (Sec. 4.1.3: any width from 2 to 8 bits): bits = 2 or 8 puts 2^bits - 1 in the place of 15
+# and changes the code bytes only -- 8 bits: byte i = q_i (G bytes); 2 bits: byte i = q_i | q_{i+G/4} << 2 |
+# q_{i+G/2} << 4 | q_{i+3G/4} << 6 (G/4 bytes); records of 272 and 80 bytes.  Pinned by hand-worked superblocks
+# (tests/golden/kq_superblock_2bit.txt, _8bit.txt), the scalar restatement, the error bound and the layout check.
 
-def kq_record_bytes(sub: int = 32, nsub: int = 8) -> int:
-    return sub * nsub // 2 + (12 * nsub + 7) // 8 + 4
+def kq_record_bytes(sub: int = 32, nsub: int = 8, bits: int = 4) -> int:
+    return sub * nsub * bits // 8 + (12 * nsub + 7) // 8 + 4
 
 
-def kq_quantize(W, sub: int = 32, nsub: int = 8):
-    """fp16 W[m][n] -> (q uint8[m][n], sc uint8[R][nsub][n], mn uint8[R][nsub][n], d fp16[R][n], dmin fp16[R][n])."""
+def kq_quantize(W, sub: int = 32, nsub: int = 8, bits: int = 4):
+    """fp16 W[m][n] -> (q uint8[m][n], sc uint8[R][nsub][n], mn uint8[R][nsub][n], d fp16[R][n], dmin fp16[R][n]).
+    bits = width of a code (2, 4 or 8): the codes run from 0 to 2^bits - 1, everything else is the same rule."""
+    assert bits in (2, 4, 8)
+    top = np.float32((1 << bits) - 1)
     W = np.ascontiguousarray(W, dtype=np.float16)
     m, n = W.shape
     G = sub * nsub
@@ -299,7 +306,7 @@ def kq_quantize(W, sub: int = 32, nsub: int = 8):
     with np.errstate(divide="ignore", invalid="ignore"):
         lo = np.minimum(w.min(axis=2), f32(0)) + f32(0)            # (a zero of either sign counts as +0.0)
         hi = w.max(axis=2) + f32(0)
-        step = ((hi - lo).astype(f32) / f32(15)).astype(f32)
+        step = ((hi - lo).astype(f32) / top).astype(f32)
         neg = (f32(0) - lo).astype(f32)                            # (0 - 0 is +0.0)
         d = (step.max(axis=1) / f32(63)).astype(f32).astype(np.float16)
         dmin = (neg.max(axis=1) / f32(63)).astype(f32).astype(np.float16)
@@ -309,27 +316,35 @@ def kq_quantize(W, sub: int = 32, nsub: int = 8):
         s_eff = (df * sc.astype(f32)).astype(f32)[:, :, None, :]
         o_eff = (dminf * mn.astype(f32)).astype(f32)[:, :, None, :]
         quo = ((w + o_eff).astype(f32) / s_eff).astype(f32)
-        q = np.where(s_eff != 0, np.clip(np.rint(quo), f32(0), f32(15)), f32(0)).astype(np.uint8)
+        q = np.where(s_eff != 0, np.clip(np.rint(quo), f32(0), top), f32(0)).astype(np.uint8)
     return q.reshape(m, n), sc, mn, d, dmin
 
 
-def kq_pack(q, sc, mn, d, dmin, sub: int = 32, nsub: int = 8) -> np.ndarray:
-    """The records, uint8[R][n][record bytes] flattened (superblock (r, k) at record index r*n + k)."""
+def kq_pack(q, sc, mn, d, dmin, sub: int = 32, nsub: int = 8, bits: int = 4) -> np.ndarray:
+    """The records, uint8[R][n][record bytes] flattened (superblock (r, k) at record index r*n + k).  Codes of a
+    superblock's G rows: 4 bits, byte i = q_i | q_{i+G/2} << 4; 8 bits, byte i = q_i; 2 bits, byte i =
+    q_i | q_{i+G/4} << 2 | q_{i+G/2} << 4 | q_{i+3G/4} << 6."""
+    assert bits in (2, 4, 8)
     G = sub * nsub
     m, n = q.shape
     R = m // G
     nf = (12 * nsub + 7) // 8
-    rec = np.zeros((R, n, kq_record_bytes(sub, nsub)), np.uint8)
+    nc = G * bits // 8
+    rec = np.zeros((R, n, kq_record_bytes(sub, nsub, bits)), np.uint8)
     qb = q.reshape(R, G, n)
-    rec[:, :, :G // 2] = (qb[:, :G // 2, :] | (qb[:, G // 2:, :] << 4)).transpose(0, 2, 1)
+    per = 8 // bits                                   # codes per byte
+    codes = np.zeros((R, nc, n), np.uint8)
+    for f in range(per):
+        codes |= (qb[:, f * nc:(f + 1) * nc, :] << (bits * f)).astype(np.uint8)
+    rec[:, :, :nc] = codes.transpose(0, 2, 1)
     fields = np.concatenate([sc, mn], axis=1).astype(np.uint64)        # [R][2*nsub][n]
-    bits = np.zeros((R, n), dtype=object)
+    fbits = np.zeros((R, n), dtype=object)
     for f in range(2 * nsub):
-        bits = bits + (fields[:, f, :].astype(object) << (6 * f))
+        fbits = fbits + (fields[:, f, :].astype(object) << (6 * f))
     for b in range(nf):
-        rec[:, :, G // 2 + b] = ((bits >> (8 * b)) & 0xFF).astype(np.uint8)
+        rec[:, :, nc + b] = ((fbits >> (8 * b)) & 0xFF).astype(np.uint8)
     du, mu = np.asarray(d, np.float16).view(np.uint16), np.asarray(dmin, np.float16).view(np.uint16)
-    o = G // 2 + nf
+    o = nc + nf
     rec[:, :, o], rec[:, :, o + 1] = (du & 0xFF).astype(np.uint8), (du >> 8).astype(np.uint8)
     rec[:, :, o + 2], rec[:, :, o + 3] = (mu & 0xFF).astype(np.uint8), (mu >> 8).astype(np.uint8)
     return rec.reshape(-1)

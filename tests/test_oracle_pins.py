@@ -522,9 +522,9 @@ def test_rowwise_layout_and_product_exact():
 
 # ---------------------------------------------------------------- two-level format (Sec. 2: 6-bit block scales/minimums)
 
-def _golden_kq():
+def _golden_kq(name="kq_superblock.txt"):
     out = {}
-    with open(os.path.join(os.path.dirname(__file__), "golden", "kq_superblock.txt")) as f:
+    with open(os.path.join(os.path.dirname(__file__), "golden", name)) as f:
         for line in f:
             if line.startswith("#") or not line.strip():
                 continue
@@ -548,21 +548,38 @@ def test_kq_hand_worked_superblock():
     assert y.tolist() == [2 * float(v) for v in g["dequantized"]] and bound.tolist() == [2 * abs(float(v)) for v in g["dequantized"]]
 
 
-def test_kq_quantizer_against_a_scalar_restatement():
+@pytest.mark.parametrize("bits,name", [(2, "kq_superblock_2bit.txt"), (8, "kq_superblock_8bit.txt")])
+def test_kq_hand_worked_superblock_other_widths(bits, name):
+    g = _golden_kq(name)
+    W = np.array([float(v) for v in g["w"]], dtype=np.float16).reshape(8, 1)
+    q, sc, mn, d, dmin = oracle.kq_quantize(W, 4, 2, bits)
+    assert q.ravel().tolist() == [int(v) for v in g["q"]]
+    assert sc.ravel().tolist() == [int(v) for v in g["sc"]] and mn.ravel().tolist() == [int(v) for v in g["m"]]
+    assert int(d.view(np.uint16)[0, 0]) == int(g["d_bits"][0], 16) and int(dmin.view(np.uint16)[0, 0]) == int(g["dmin_bits"][0], 16)
+    assert oracle.kq_pack(q, sc, mn, d, dmin, 4, 2, bits).tolist() == [int(v, 16) for v in g["record"]]
+    assert oracle.kq_record_bytes(4, 2, bits) == len(g["record"])
+    assert oracle.kq_record_bytes(bits=2) == 80 and oracle.kq_record_bytes(bits=8) == 272
+    What = oracle.kq_dequantize_rows(q, sc, mn, d, dmin, np.arange(8), 4, 2).ravel()
+    assert What.tolist() == [float(v) for v in g["dequantized"]]
+
+
+@pytest.mark.parametrize("bits", [4, 2, 8])
+def test_kq_quantizer_against_a_scalar_restatement(bits):
     f32 = np.float32
+    top = (1 << bits) - 1
     rng = np.random.default_rng(21)
     sub, nsub, n = 4, 3, 7
     W = (rng.standard_normal((2 * sub * nsub, n)) * 0.3).astype(np.float16)
     W[:sub, 0] = np.float16(0.25)                  # a constant positive block: minimum field 0
     W[:, 1] = np.float16(0.0)                      # an all-zero superblock column (both superblocks)
     W[sub:2 * sub, 2] = -np.abs(W[sub:2 * sub, 2])  # an all-negative block
-    q, sc, mn, d, dmin = oracle.kq_quantize(W, sub, nsub)
+    q, sc, mn, d, dmin = oracle.kq_quantize(W, sub, nsub, bits)
     G = sub * nsub
     for r in range(2):
         for k in range(n):
             blocks = [W[r * G + i * sub: r * G + (i + 1) * sub, k].astype(f32) for i in range(nsub)]
             lo = [min(f32(b.min()), f32(0)) for b in blocks]
-            step = [f32(f32(b.max()) - l) / f32(15) for b, l in zip(blocks, lo)]
+            step = [f32(f32(b.max()) - l) / f32(top) for b, l in zip(blocks, lo)]
             neg = [f32(-l) for l in lo]
             dd = np.float16(f32(max(step)) / f32(63))
             dm = np.float16(f32(max(neg)) / f32(63))
@@ -573,10 +590,46 @@ def test_kq_quantizer_against_a_scalar_restatement():
                 assert sc[r, i, k] == s_i and mn[r, i, k] == m_i
                 se, oe = f32(dd) * f32(s_i), f32(dm) * f32(m_i)
                 for j in range(sub):
-                    want = int(np.clip(np.rint(f32(blocks[i][j] + oe) / se), 0, 15)) if se != 0 else 0
+                    want = int(np.clip(np.rint(f32(blocks[i][j] + oe) / se), 0, top)) if se != 0 else 0
                     assert q[r * G + i * sub + j, k] == want
     assert not q[:, 1].any() and not sc[:, :, 1].any() and float(d[0, 1]) == 0.0
     assert mn[0, 0, 0] == 0 and mn[0, 1, 2] > 0
+
+
+@pytest.mark.parametrize("bits", [2, 8])
+def test_kq_error_bound_and_code_layout_other_widths(bits):
+    rng = np.random.default_rng(24)
+    m, n, top = 512, 24, (1 << bits) - 1
+    W = (rng.standard_normal((m, n)) * 0.02).astype(np.float16)
+    q, sc, mn, d, dmin = oracle.kq_quantize(W, bits=bits)
+    assert q.max() == top and sc.max() == 63 and mn.max() == 63
+    What = oracle.kq_dequantize_rows(q, sc, mn, d, dmin, np.arange(m))
+    w = W.astype(np.float64).reshape(2, 8, 32, n)
+    lo = np.minimum(w.min(axis=2), 0.0)
+    s_eff = d.astype(np.float64)[:, None, :] * sc
+    o_eff = dmin.astype(np.float64)[:, None, :] * mn
+    lim = s_eff / 2 + np.abs(w.max(axis=2) - lo - top * s_eff) + np.abs(o_eff + lo) + 1e-7
+    err = np.abs(What.reshape(2, 8, 32, n) - w)
+    assert np.all(err <= lim[:, :, None, :])
+    # finer codes, smaller error: 8-bit steps are 17 times finer than 4-bit ones, 2-bit steps 5 times coarser
+    q4, sc4, mn4, d4, dmin4 = oracle.kq_quantize(W)
+    err4 = np.abs(oracle.kq_dequantize_rows(q4, sc4, mn4, d4, dmin4, np.arange(m)) - W.astype(np.float64))
+    ratio = np.mean(err) / np.mean(err4)
+    assert (3.0 < ratio < 7.0) if bits == 2 else (ratio < 0.25)
+    # the record: codes (2 bits: four quarter-planes per byte; 8 bits: one per byte), fields, d, dmin
+    nc = 256 * bits // 8
+    rec = oracle.kq_pack(q, sc, mn, d, dmin, bits=bits).reshape(2, n, nc + 16)
+    for (r, k) in [(0, 0), (1, 11), (1, 23)]:
+        b = rec[r, k]
+        for i in range(nc):
+            if bits == 8:
+                assert b[i] == q[r * 256 + i, k]
+            else:
+                assert b[i] == (q[r * 256 + i, k] | (q[r * 256 + 64 + i, k] << 2) | (q[r * 256 + 128 + i, k] << 4) | (q[r * 256 + 192 + i, k] << 6))
+        fb = int.from_bytes(bytes(b[nc:nc + 12].tolist()), "little")
+        assert [(fb >> (6 * f)) & 63 for f in range(16)] == sc[r, :, k].tolist() + mn[r, :, k].tolist()
+        assert int.from_bytes(bytes(b[nc + 12:nc + 14].tolist()), "little") == int(d.view(np.uint16)[r, k])
+        assert int.from_bytes(bytes(b[nc + 14:nc + 16].tolist()), "little") == int(dmin.view(np.uint16)[r, k])
 
 
 def test_kq_error_bound_scaling_and_fields():
