@@ -371,6 +371,24 @@ spqt_status spqt_kq_dense_gemv(const void* records, int m, int n, const void* x,
                                void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The same format with other code widths (paper Sec. 4.1.3: the grouping works for any code width from
+ * 2 to 8 bits).  bits = 2, 4 or 8 (SPQT_ERR_UNSUPPORTED otherwise); bits = 4 is exactly the format above.
+ * 2^bits - 1 takes the place of 15 in the rule, and only the code bytes of a record change:
+ *   bits = 8 : bytes 0..255, byte i = q_i; record of 272 bytes (fields at 256, d and dmin at 268)
+ *   bits = 2 : bytes 0..63,  byte i = q_i | q_{i+64} << 2 | q_{i+128} << 4 | q_{i+192} << 6;
+ *              record of 80 bytes (fields at 64, d and dmin at 76)
+ * Arguments, workspace, alignment and error behaviour as for the spqt_kq_* calls; the workspace does not
+ * depend on the width.
+ */
+spqt_status spqt_kqw_packed_sizes(int m, int n, int bits, size_t* records_bytes, size_t* workspace_bytes);
+spqt_status spqt_kqw_pack(const void* W, int m, int n, int ldw, int bits, void* records, void* stream);
+spqt_status spqt_kqw_sparse_gemv(const void* records, int m, int n, int bits, const void* x,
+                                 const int32_t* idx, const int32_t* count, void* y,
+                                 void* workspace, size_t workspace_bytes, void* stream);
+spqt_status spqt_kqw_dense_gemv(const void* records, int m, int n, int bits, const void* x, void* y,
+                                void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Threshold calibration (paper Sec. 5, the calibration threshold tool; Sec. 3.2: thresholds are
  * computed once per sparsity level from calibration activations).  *threshold (a device float) =
  * the nearest-rank order statistic of |x| over the pool x[0:count] of fp16 calibration activations:

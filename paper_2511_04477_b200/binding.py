@@ -20,7 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libspqt.so")
 EXPORTS = (
     "spqt_status_string", "spqt_version", "spqt_packed_sizes", "spqt_pack", "spqt_unpack",
     "spqt_sparsify", "spqt_sparse_gemv", "spqt_sparse_gemv_static", "spqt_static_status", "spqt_sparsify_gemv", "spqt_dense_gemv",
-    "spqt_sparse_linear_host", "spqt_sparse_linear_host_async", "spqt_host_step_create", "spqt_host_step_launch", "spqt_host_step_destroy", "spqt_gemm_small_workspace", "spqt_sparse_gemm_small", "spqt_dense_gemm_small", "spqt_rowwise_packed_sizes", "spqt_rowwise_pack", "spqt_rowwise_dense_gemv", "spqt_rowwise_thresholded_gemv", "spqt_kq_packed_sizes", "spqt_kq_pack", "spqt_kq_sparse_gemv", "spqt_kq_dense_gemv", "spqt_autotune", "spqt_calibrate_threshold", "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_probe_arith", "spqt_launch_count",
+    "spqt_sparse_linear_host", "spqt_sparse_linear_host_async", "spqt_host_step_create", "spqt_host_step_launch", "spqt_host_step_destroy", "spqt_gemm_small_workspace", "spqt_sparse_gemm_small", "spqt_dense_gemm_small", "spqt_rowwise_packed_sizes", "spqt_rowwise_pack", "spqt_rowwise_dense_gemv", "spqt_rowwise_thresholded_gemv", "spqt_kq_packed_sizes", "spqt_kq_pack", "spqt_kq_sparse_gemv", "spqt_kq_dense_gemv", "spqt_kqw_packed_sizes", "spqt_kqw_pack", "spqt_kqw_sparse_gemv", "spqt_kqw_dense_gemv", "spqt_autotune", "spqt_calibrate_threshold", "spqt_set_tuning", "spqt_set_debug", "spqt_workspace_status", "spqt_probe_read", "spqt_probe_arith", "spqt_launch_count",
 )
 
 _lib = None
@@ -65,6 +65,12 @@ def lib() -> ctypes.CDLL:
         L.spqt_kq_pack.argtypes = [vp, i32, i32, i32, vp, vp]
         L.spqt_kq_sparse_gemv.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, sz, vp]
         L.spqt_kq_dense_gemv.argtypes = [vp, i32, i32, vp, vp, vp, sz, vp]
+        L.spqt_kqw_packed_sizes.argtypes = [i32, i32, i32] + [ctypes.POINTER(sz)] * 2
+        L.spqt_kqw_pack.argtypes = [vp, i32, i32, i32, i32, vp, vp]
+        L.spqt_kqw_sparse_gemv.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
+        L.spqt_kqw_dense_gemv.argtypes = [vp, i32, i32, i32, vp, vp, vp, sz, vp]
+        for name in ("spqt_kqw_packed_sizes", "spqt_kqw_pack", "spqt_kqw_sparse_gemv", "spqt_kqw_dense_gemv"):
+            getattr(L, name).restype = i32
         L.spqt_sparse_linear_host.argtypes = [vp, vp, i32, i32, i32, i32, vp, ctypes.c_float, vp,
                                               vp, vp, vp, vp, vp, sz, vp]
         L.spqt_sparse_linear_host_async.argtypes = L.spqt_sparse_linear_host.argtypes
@@ -450,9 +456,10 @@ def spqt_rowwise_dense_gemv(p: RowwisePacked, x: torch.Tensor, y: torch.Tensor =
 @dataclass
 class KqPacked:
     """Device buffer written by :func:`spqt_kq_pack` (144-byte records of the two-level format, zigzag order)."""
-    records: torch.Tensor      # uint8[(m/256)*n*144]
+    records: torch.Tensor      # uint8[(m/256)*n*144]  (80 or 272 bytes per record with 2- or 8-bit codes)
     m: int
     n: int
+    bits: int = 4
 
 
 def spqt_kq_packed_sizes(m: int, n: int):
@@ -471,6 +478,45 @@ def spqt_kq_pack(W: torch.Tensor, stream=None) -> KqPacked:
     records = torch.empty(rb, dtype=torch.uint8, device=W.device)
     _ok(lib().spqt_kq_pack(W.data_ptr(), m, n, W.stride(0), records.data_ptr(), _stream(stream)), "spqt_kq_pack")
     return KqPacked(records, m, n)
+
+
+def spqt_kqw_packed_sizes(m: int, n: int, bits: int):
+    out = [ctypes.c_size_t(0) for _ in range(2)]
+    _ok(lib().spqt_kqw_packed_sizes(m, n, bits, *[ctypes.byref(o) for o in out]), "spqt_kqw_packed_sizes")
+    return int(out[0].value), int(out[1].value)
+
+
+def spqt_kqw_pack(W: torch.Tensor, bits: int, stream=None) -> KqPacked:
+    """The two-level format with 2-, 4- or 8-bit codes."""
+    if W.dim() != 2 or W.stride(1) != 1:
+        raise ValueError("W must be 2-D with unit column stride")
+    if not W.is_cuda or W.dtype != torch.float16:
+        raise TypeError("W must be a CUDA float16 tensor")
+    m, n = W.shape
+    rb, _ = spqt_kqw_packed_sizes(m, n, bits)
+    records = torch.empty(rb, dtype=torch.uint8, device=W.device)
+    _ok(lib().spqt_kqw_pack(W.data_ptr(), m, n, W.stride(0), bits, records.data_ptr(), _stream(stream)), "spqt_kqw_pack")
+    return KqPacked(records, m, n, bits)
+
+
+def spqt_kqw_sparse_gemv(p: KqPacked, x: torch.Tensor, idx: torch.Tensor, count: torch.Tensor, workspace: torch.Tensor,
+                         y: torch.Tensor = None, stream=None) -> torch.Tensor:
+    if y is None:
+        y = torch.empty(p.m, dtype=torch.float16, device=x.device)
+    _ok(lib().spqt_kqw_sparse_gemv(
+        _dev(p.records, torch.uint8, "records"), p.m, p.n, p.bits, _dev(x, torch.float16, "x"),
+        _dev(idx, torch.int32, "idx"), _dev(count, torch.int32, "count"), _dev(y, torch.float16, "y"),
+        _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)), "spqt_kqw_sparse_gemv")
+    return y
+
+
+def spqt_kqw_dense_gemv(p: KqPacked, x: torch.Tensor, workspace: torch.Tensor, y: torch.Tensor = None, stream=None) -> torch.Tensor:
+    if y is None:
+        y = torch.empty(p.m, dtype=torch.float16, device=x.device)
+    _ok(lib().spqt_kqw_dense_gemv(
+        _dev(p.records, torch.uint8, "records"), p.m, p.n, p.bits, _dev(x, torch.float16, "x"), _dev(y, torch.float16, "y"),
+        _dev(workspace, torch.uint8, "workspace"), workspace.numel(), _stream(stream)), "spqt_kqw_dense_gemv")
+    return y
 
 
 def new_kq_workspace(p: KqPacked) -> torch.Tensor:

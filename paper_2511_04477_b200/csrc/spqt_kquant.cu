@@ -6,6 +6,11 @@
 // m_0..7 as a little-endian bit string (12 bytes), d and dmin as fp16.  Dequantized weight of row j of
 // block i:  d*sc_i*q_j - dmin*m_i.  The paper fixes neither the rounding rule nor the bit arrangement;
 // the rule implemented is stated at kq_pack_kernel, every step a single IEEE fp32 operation.
+// Other code widths (Sec. 4.1.3: any width from 2 to 8 bits): the kernels are templates over BITS = 2, 4, 8;
+// 2^BITS - 1 replaces 15 in the rule and only the code bytes of a record change -- 8 bits: byte i = q_i (256
+// bytes, records of 272); 2 bits: byte i = q_i | q_{i+64} << 2 | q_{i+128} << 4 | q_{i+192} << 6 (64 bytes,
+// records of 80).  Their arithmetic sums, per 16-bit half-word, the value of its low byte and of both bytes
+// (the cumulative form of the main kernel) and takes the difference at the end.
 //
 //   kq_pack_kernel   a CTA stages a 256 x 32 tile of W; a warp quantizes four columns, lane l owning rows
 //                    l, l+32, .. (one row of every block).
@@ -30,7 +35,9 @@ constexpr unsigned long long kWaitNs = 1000000000ull;
 namespace spqt {
 
 constexpr int kKqG = 256;           // rows of a superblock
-constexpr int kKqRec = 144;         // bytes of a record
+__host__ __device__ constexpr int kq_code_bytes(int bits) { return kKqG * bits / 8; }
+__host__ __device__ constexpr int kq_rec_bytes(int bits) { return kq_code_bytes(bits) + 16; }
+__host__ __device__ constexpr int kq_ctas_per_sm(int bits) { return bits == 8 ? 2 : 3; }   // (shared memory: two record buffers per warp)
 constexpr int kKqWarps = 8;
 constexpr int kKqThreads = kKqWarps * 32;
 constexpr int kKqChunk = 16;        // list entries per chunk
@@ -43,9 +50,12 @@ constexpr int kKqPackCols = 32;
 //   per superblock:   d = fp16(max_i step_i / 63),  dmin = fp16(max_i neg_i / 63)
 //                     sc_i = min(rint(step_i / d), 63),  m_i = min(rint(neg_i / dmin), 63)   (0 if the divisor is 0)
 //   per weight:       q_j = clamp(rint((w_j + dmin*m_i) / (d*sc_i)), 0, 15)                   (0 if d*sc_i == 0)
+// (15 = 2^BITS - 1 for 4-bit codes; 3 and 255 for the other widths)
+template <int BITS>
 __global__ void __launch_bounds__(256)
 kq_pack_kernel(const __half* __restrict__ W, int n, int ldw, uint8_t* __restrict__ records)
 {
+    constexpr int kTop = (1 << BITS) - 1, NCB = kq_code_bytes(BITS), REC = kq_rec_bytes(BITS);
     __shared__ __align__(16) __half tile[kKqG][kKqPackCols + 2];
     const int r = blockIdx.y, k0 = blockIdx.x * kKqPackCols, tid = threadIdx.x;
     for (int e = tid; e < kKqG * kKqPackCols; e += 256) {
@@ -70,7 +80,7 @@ kq_pack_kernel(const __half* __restrict__ W, int n, int ldw, uint8_t* __restrict
             }
             lo = __fadd_rn(fminf(lo, 0.0f), 0.0f);  // a zero of either sign counts as +0.0
             hi = __fadd_rn(hi, 0.0f);
-            step[u] = __fdiv_rn(__fsub_rn(hi, lo), 15.0f);
+            step[u] = __fdiv_rn(__fsub_rn(hi, lo), (float)kTop);
             neg[u] = __fsub_rn(0.0f, lo);           // (0 - 0 is +0.0)
             step_max = fmaxf(step_max, step[u]);
             neg_max = fmaxf(neg_max, neg[u]);
@@ -85,12 +95,20 @@ kq_pack_kernel(const __half* __restrict__ W, int n, int ldw, uint8_t* __restrict
             sc[u] = (df != 0.0f) ? (unsigned)min(__float2int_rn(__fdiv_rn(step[u], df)), 63) : 0u;
             mn[u] = (dminf != 0.0f) ? (unsigned)min(__float2int_rn(__fdiv_rn(neg[u], dminf)), 63) : 0u;
             const float se = __fmul_rn(df, (float)sc[u]), oe = __fmul_rn(dminf, (float)mn[u]);
-            q[u] = (se != 0.0f) ? max(0, min(__float2int_rn(__fdiv_rn(__fadd_rn(w[u], oe), se)), 15)) : 0;
+            q[u] = (se != 0.0f) ? max(0, min(__float2int_rn(__fdiv_rn(__fadd_rn(w[u], oe), se)), kTop)) : 0;
         }
-        uint8_t* rec = records + ((size_t)r * n + k) * kKqRec;
-        // byte i = code of row i | code of row i + 128 << 4; this lane holds rows lane + 32u
+        uint8_t* rec = records + ((size_t)r * n + k) * REC;
+        // this lane holds the codes of rows lane + 32u
+        if (BITS == 4) {            // byte i = code of row i | code of row i + 128 << 4
 #pragma unroll
-        for (int u = 0; u < 4; ++u) rec[lane + 32 * u] = (uint8_t)(q[u] | (q[u + 4] << 4));
+            for (int u = 0; u < 4; ++u) rec[lane + 32 * u] = (uint8_t)(q[u] | (q[u + 4] << 4));
+        } else if (BITS == 8) {     // byte i = code of row i
+#pragma unroll
+            for (int u = 0; u < 8; ++u) rec[lane + 32 * u] = (uint8_t)q[u];
+        } else {                    // byte i = codes of rows i, i + 64, i + 128, i + 192, two bits each
+#pragma unroll
+            for (int u = 0; u < 2; ++u) rec[lane + 32 * u] = (uint8_t)(q[u] | (q[u + 2] << 2) | (q[u + 4] << 4) | (q[u + 6] << 6));
+        }
         if (lane == 0) {
             unsigned long long lo64 = 0ull;  // fields 0..9 and the low 4 bits of field 10
             unsigned hi32 = 0u;              // bits 64..95
@@ -101,7 +119,7 @@ kq_pack_kernel(const __half* __restrict__ W, int n, int ldw, uint8_t* __restrict
                 if (b < 64) lo64 |= v << b;
                 if (b + 6 > 64) hi32 |= (b >= 64) ? (unsigned)(v << (b - 64)) : (unsigned)(v >> (64 - b));
             }
-            unsigned* tail = reinterpret_cast<unsigned*>(rec + 128);  // records start on 16-byte boundaries
+            unsigned* tail = reinterpret_cast<unsigned*>(rec + NCB);  // records start on 16-byte boundaries
             tail[0] = (unsigned)lo64;
             tail[1] = (unsigned)(lo64 >> 32);
             tail[2] = hi32;
@@ -112,8 +130,9 @@ kq_pack_kernel(const __half* __restrict__ W, int n, int ldw, uint8_t* __restrict
 
 // ---------------------------------------------------------------- GEMV
 
+template <int BITS>
 struct KqSmem {
-    alignas(16) unsigned char rec[kKqWarps][2][kKqChunk * kKqRec];  // two record buffers per warp
+    alignas(16) unsigned char rec[kKqWarps][2][kKqChunk * kq_rec_bytes(BITS)];  // two record buffers per warp
     alignas(16) float mult[kKqWarps][kKqChunk][4][4];               // per entry and lane group: two packed multiplier pairs
     alignas(16) float red[kKqWarps][kKqG];
     float red_z[kKqWarps][8];
@@ -130,16 +149,18 @@ __device__ __forceinline__ unsigned kq_field(unsigned w0, unsigned w1, unsigned 
 }
 
 // idx == nullptr: the dense product (the list is 0, 1, .., n-1 and count is n).
-__global__ void __launch_bounds__(kKqThreads, 3)
+template <int BITS>
+__global__ void __launch_bounds__(kKqThreads, kq_ctas_per_sm(BITS))
 kq_gemv_kernel(const uint8_t* __restrict__ records, int n, const __half* __restrict__ x,
                const int32_t* __restrict__ idx, const int32_t* __restrict__ count_ptr,
                __half* __restrict__ y, float* __restrict__ partials, int* __restrict__ counters)
 {
     constexpr int CH = kKqChunk, G = kKqG;
-    constexpr int NP = CH * kKqRec / 16;         // 16-byte pieces of a chunk
+    constexpr int REC = kq_rec_bytes(BITS), NCB = kq_code_bytes(BITS), PPR = REC / 16;
+    constexpr int NP = CH * REC / 16;            // 16-byte pieces of a chunk
     constexpr int NC = (NP + 31) / 32;           // copies per lane and chunk
     extern __shared__ __align__(16) unsigned char kq_raw[];
-    KqSmem& sm = *reinterpret_cast<KqSmem*>(kq_raw);
+    KqSmem<BITS>& sm = *reinterpret_cast<KqSmem<BITS>*>(kq_raw);
     const int tid = threadIdx.x, lane = tid & 31;
     const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
     const int s = blockIdx.x, S = gridDim.x, r = blockIdx.y;
@@ -150,10 +171,10 @@ kq_gemv_kernel(const uint8_t* __restrict__ records, int n, const __half* __restr
 
     const int count = idx ? __ldg(count_ptr) : n;
     const int lo = (int)(((long long)s * count) / S), hi = (int)(((long long)(s + 1) * count) / S);
-    const uint8_t* row_rec = records + (size_t)r * (size_t)n * kKqRec;
+    const uint8_t* row_rec = records + (size_t)r * (size_t)n * REC;
     const unsigned rbuf = smem_u32(&sm.rec[warp][0][0]);
     const unsigned mbuf = smem_u32(&sm.mult[warp][0][0][0]);
-    constexpr unsigned kBufBytes = CH * kKqRec;
+    constexpr unsigned kBufBytes = CH * REC;
     const unsigned short* xb = reinterpret_cast<const unsigned short*>(x);
 
     unsigned long long acc[8];
@@ -170,9 +191,9 @@ kq_gemv_kernel(const uint8_t* __restrict__ records, int n, const __half* __restr
 #pragma unroll
         for (int q = 0; q < NC; ++q) {
             const int p = q * 32 + lane;
-            const int e = p / 9, part = p - 9 * e;
+            const int e = p / PPR, part = p - PPR * e;
             const int cu = __shfl_sync(0xffffffffu, col, e & 15);
-            if (p < NP) cp_async_16_l2_64(dst + (unsigned)(e * kKqRec + part * 16), row_rec + (size_t)cu * kKqRec + part * 16);
+            if (p < NP) cp_async_16_l2_64(dst + (unsigned)(e * REC + part * 16), row_rec + (size_t)cu * REC + part * 16);
         }
         cp_async_commit();
     };
@@ -195,7 +216,7 @@ kq_gemv_kernel(const uint8_t* __restrict__ records, int n, const __half* __restr
             // lanes e and e+16: the fields of entry e -> multiplier pairs of lane groups 2*half, 2*half+1 and
             // the offset terms of blocks 4*half .. 4*half+3
             {
-                const unsigned ra = rbuf + cur + (unsigned)(t * kKqRec) + 128u;
+                const unsigned ra = rbuf + cur + (unsigned)(t * REC) + (unsigned)NCB;
                 const uint4 tail = lds_v4(ra);
                 const float xf = __half2float(__ushort_as_half(xv));
                 const float df = __half2float(__ushort_as_half((unsigned short)(tail.w & 0xffffu)));
@@ -205,8 +226,11 @@ kq_gemv_kernel(const uint8_t* __restrict__ records, int n, const __half* __restr
                     const int sb = 2 * half + g2;   // lane group: rows of blocks sb (low nibbles) and sb + 4 (high nibbles)
                     const float a_lo = xf * (df * (float)kq_field(tail.x, tail.y, tail.z, sb));       // d*sc is exact
                     const float a_hi = xf * (df * (float)kq_field(tail.x, tail.y, tail.z, sb + 4));
-                    sts_pairs(mbuf + 16u * (unsigned)(t * 4 + sb), pack2(a_lo * 0x1p93f, a_hi * 0x1p89f),
-                              pack2(a_lo * 0x1p85f, a_hi * 0x1p81f));
+                    if (BITS == 4)
+                        sts_pairs(mbuf + 16u * (unsigned)(t * 4 + sb), pack2(a_lo * 0x1p93f, a_hi * 0x1p89f),
+                                  pack2(a_lo * 0x1p85f, a_hi * 0x1p81f));
+                    else   // one pair: the high rows' codes sit in the same bytes (2 bits, four bits up) or in bytes of their own (8 bits)
+                        sts_u64(mbuf + 16u * (unsigned)(t * 4 + sb), pack2(a_lo * 0x1p93f, a_hi * (BITS == 2 ? 0x1p89f : 0x1p93f)));
                 }
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
@@ -217,10 +241,41 @@ kq_gemv_kernel(const uint8_t* __restrict__ records, int n, const __half* __restr
             const unsigned cb = rbuf + cur;
             auto step = [&](int u) {
                 const unsigned e = (unsigned)(2 * u + half);
-                const uint2 wv = lds_v2(cb + e * kKqRec + (unsigned)t * 8u);
-                unsigned long long m01, m23;
-                lds_pairs(mbuf + 16u * (e * 4u + (unsigned)(t >> 2)), m01, m23);
-                fma_block8(acc, wv, m01, m23);
+                if (BITS == 4) {
+                    const uint2 wv = lds_v2(cb + e * REC + (unsigned)t * 8u);
+                    unsigned long long m01, m23;
+                    lds_pairs(mbuf + 16u * (e * 4u + (unsigned)(t >> 2)), m01, m23);
+                    fma_block8(acc, wv, m01, m23);
+                    return;
+                }
+                // 2 and 8 bits: per 16-bit half-word the value of its first byte's code and the value of both
+                // codes together (second code times 256) are summed; the second code's sum is their difference
+                const unsigned long long mm = lds_u64(mbuf + 16u * (e * 4u + (unsigned)(t >> 2)));
+                if (BITS == 8) {
+                    const uint2 lw = lds_v2(cb + e * REC + (unsigned)t * 8u);           // rows 8t .. 8t+7
+                    const uint2 hw = lds_v2(cb + e * REC + 128u + (unsigned)t * 8u);    // rows 128+8t ..
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+                        const unsigned l = k ? lw.y : lw.x, h = k ? hw.y : hw.x, lv = l >> 16, hv = h >> 16;
+                        ffma2(acc[4 * k + 0], pack2(__uint_as_float(l & 0xffu), __uint_as_float(h & 0xffu)), mm);
+                        ffma2(acc[4 * k + 1], pack2(__uint_as_float(l & 0xffffu), __uint_as_float(h & 0xffffu)), mm);
+                        ffma2(acc[4 * k + 2], pack2(__uint_as_float(lv & 0xffu), __uint_as_float(hv & 0xffu)), mm);
+                        ffma2(acc[4 * k + 3], pack2(__uint_as_float(lv), __uint_as_float(hv)), mm);
+                    }
+                } else {
+                    // byte i holds rows i, i+64, i+128, i+192: lanes 0..7 use fields 0 and 2 of bytes 8t.., lanes
+                    // 8..15 fields 1 and 3 of bytes 8(t-8)..
+                    const uint2 wv = lds_v2(cb + e * REC + (unsigned)(t & 7) * 8u);
+                    const int sh = 2 * (t >> 3);
+#pragma unroll
+                    for (int k = 0; k < 2; ++k) {
+                        const unsigned w = (k ? wv.y : wv.x) >> sh, v = w >> 16;
+                        ffma2(acc[4 * k + 0], pack2(__uint_as_float(w & 0x03u), __uint_as_float(w & 0x30u)), mm);
+                        ffma2(acc[4 * k + 1], pack2(__uint_as_float(w & 0x0303u), __uint_as_float(w & 0x3030u)), mm);
+                        ffma2(acc[4 * k + 2], pack2(__uint_as_float(v & 0x03u), __uint_as_float(v & 0x30u)), mm);
+                        ffma2(acc[4 * k + 3], pack2(__uint_as_float(v & 0x0303u), __uint_as_float(v & 0x3030u)), mm);
+                    }
+                }
             };
             if (valid == CH) {
 #pragma unroll
@@ -247,6 +302,13 @@ kq_gemv_kernel(const uint8_t* __restrict__ records, int n, const __half* __restr
             unpack2(acc[b], lo_rows[b], hi_rows[b]);
             lo_rows[b] += __shfl_xor_sync(0xffffffffu, lo_rows[b], 16);
             hi_rows[b] += __shfl_xor_sync(0xffffffffu, hi_rows[b], 16);
+        }
+        if (BITS != 4) {   // odd positions hold (first code + 256 * second code) of a half-word
+#pragma unroll
+            for (int b = 1; b < 8; b += 2) {
+                lo_rows[b] = (lo_rows[b] - lo_rows[b - 1]) * 0x1p-8f;
+                hi_rows[b] = (hi_rows[b] - hi_rows[b - 1]) * 0x1p-8f;
+            }
         }
         if (half == 0) {
 #pragma unroll
@@ -314,6 +376,7 @@ static spqt_status kq_shape(int m, int n)
     return SPQT_OK;
 }
 
+template <int BITS>
 static spqt_status kq_launch(const void* records, int m, int n, const void* x, const int32_t* idx, const int32_t* count,
                              void* y, void* workspace, size_t ws_bytes, void* stream)
 {
@@ -328,15 +391,15 @@ static spqt_status kq_launch(const void* records, int m, int n, const void* x, c
     static bool configured[64] = {};
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return SPQT_ERR_CUDA;
-    const int smem = (int)sizeof(KqSmem);
+    const int smem = (int)sizeof(KqSmem<BITS>);
     if (!configured[dev]) {
-        if (cudaFuncSetAttribute(kq_gemv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return SPQT_ERR_CUDA;
+        if (cudaFuncSetAttribute(kq_gemv_kernel<BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return SPQT_ERR_CUDA;
         configured[dev] = true;
     }
     const int sms = sm_count();
     if (sms <= 0) return SPQT_ERR_CUDA;
-    // slices per block-row: fill the three CTAs per SM once; never less than a chunk per warp
-    int S = (3 * sms) / R;
+    // slices per block-row: fill the resident CTAs of every SM once; never less than a chunk per warp
+    int S = (kq_ctas_per_sm(BITS) * sms) / R;
     const int by_work = n / (kKqChunk * kKqWarps);
     if (S > by_work) S = by_work;
     if (S > kKqMaxSplit) S = kKqMaxSplit;
@@ -353,7 +416,7 @@ static spqt_status kq_launch(const void* records, int m, int n, const void* x, c
     cfg.numAttrs = g_no_pdl ? 0 : 1;
     int* counters = static_cast<int*>(workspace);
     float* partials = reinterpret_cast<float*>(static_cast<char*>(workspace) + kq_header_bytes(R));
-    const cudaError_t err = cudaLaunchKernelEx(&cfg, kq_gemv_kernel, static_cast<const uint8_t*>(records), n,
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, kq_gemv_kernel<BITS>, static_cast<const uint8_t*>(records), n,
                                                static_cast<const __half*>(x), idx, count, static_cast<__half*>(y), partials, counters);
     count_launch();
     return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SPQT_OK : SPQT_ERR_CUDA;
@@ -363,40 +426,79 @@ static spqt_status kq_launch(const void* records, int m, int n, const void* x, c
 
 extern "C" {
 
-spqt_status spqt_kq_packed_sizes(int m, int n, size_t* records_bytes, size_t* workspace_bytes)
+static bool kq_bits_ok(int bits) { return bits == 2 || bits == 4 || bits == 8; }
+
+spqt_status spqt_kqw_packed_sizes(int m, int n, int bits, size_t* records_bytes, size_t* workspace_bytes)
 {
     const spqt_status st = spqt::kq_shape(m, n);
     if (st != SPQT_OK) return st;
-    if (records_bytes) *records_bytes = (size_t)(m / spqt::kKqG) * (size_t)n * spqt::kKqRec;
+    if (!kq_bits_ok(bits)) return SPQT_ERR_UNSUPPORTED;
+    if (records_bytes) *records_bytes = (size_t)(m / spqt::kKqG) * (size_t)n * spqt::kq_rec_bytes(bits);
     if (workspace_bytes) *workspace_bytes = spqt::kq_workspace_bytes(m / spqt::kKqG);
     return SPQT_OK;
 }
 
-spqt_status spqt_kq_pack(const void* W, int m, int n, int ldw, void* records, void* stream)
+spqt_status spqt_kqw_pack(const void* W, int m, int n, int ldw, int bits, void* records, void* stream)
 {
     if (!W || !records) return SPQT_ERR_INVALID_ARG;
     const spqt_status st = spqt::kq_shape(m, n);
     if (st != SPQT_OK) return st;
+    if (!kq_bits_ok(bits)) return SPQT_ERR_UNSUPPORTED;
     if (ldw < n) return SPQT_ERR_INVALID_ARG;
     if (!spqt::aligned(W, 2) || !spqt::aligned(records, 16)) return SPQT_ERR_ALIGNMENT;
     const dim3 grid((n + spqt::kKqPackCols - 1) / spqt::kKqPackCols, m / spqt::kKqG);
-    spqt::kq_pack_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(static_cast<const __half*>(W), n, ldw,
-                                                                               static_cast<uint8_t*>(records));
+    const cudaStream_t st_ = static_cast<cudaStream_t>(stream);
+    const __half* w = static_cast<const __half*>(W);
+    uint8_t* rec = static_cast<uint8_t*>(records);
+    if (bits == 2) spqt::kq_pack_kernel<2><<<grid, 256, 0, st_>>>(w, n, ldw, rec);
+    else if (bits == 4) spqt::kq_pack_kernel<4><<<grid, 256, 0, st_>>>(w, n, ldw, rec);
+    else spqt::kq_pack_kernel<8><<<grid, 256, 0, st_>>>(w, n, ldw, rec);
     spqt::count_launch();
     return cudaGetLastError() == cudaSuccess ? SPQT_OK : SPQT_ERR_CUDA;
+}
+
+static spqt_status kq_launch_bits(int bits, const void* records, int m, int n, const void* x, const int32_t* idx,
+                                  const int32_t* count, void* y, void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (bits == 2) return spqt::kq_launch<2>(records, m, n, x, idx, count, y, workspace, workspace_bytes, stream);
+    if (bits == 4) return spqt::kq_launch<4>(records, m, n, x, idx, count, y, workspace, workspace_bytes, stream);
+    if (bits == 8) return spqt::kq_launch<8>(records, m, n, x, idx, count, y, workspace, workspace_bytes, stream);
+    return SPQT_ERR_UNSUPPORTED;
+}
+
+spqt_status spqt_kqw_sparse_gemv(const void* records, int m, int n, int bits, const void* x, const int32_t* idx,
+                                 const int32_t* count, void* y, void* workspace, size_t workspace_bytes, void* stream)
+{
+    if (!idx || !count) return SPQT_ERR_INVALID_ARG;
+    return kq_launch_bits(bits, records, m, n, x, idx, count, y, workspace, workspace_bytes, stream);
+}
+
+spqt_status spqt_kqw_dense_gemv(const void* records, int m, int n, int bits, const void* x, void* y, void* workspace,
+                                size_t workspace_bytes, void* stream)
+{
+    return kq_launch_bits(bits, records, m, n, x, nullptr, nullptr, y, workspace, workspace_bytes, stream);
+}
+
+spqt_status spqt_kq_packed_sizes(int m, int n, size_t* records_bytes, size_t* workspace_bytes)
+{
+    return spqt_kqw_packed_sizes(m, n, 4, records_bytes, workspace_bytes);
+}
+
+spqt_status spqt_kq_pack(const void* W, int m, int n, int ldw, void* records, void* stream)
+{
+    return spqt_kqw_pack(W, m, n, ldw, 4, records, stream);
 }
 
 spqt_status spqt_kq_sparse_gemv(const void* records, int m, int n, const void* x, const int32_t* idx, const int32_t* count,
                                 void* y, void* workspace, size_t workspace_bytes, void* stream)
 {
-    if (!idx || !count) return SPQT_ERR_INVALID_ARG;
-    return spqt::kq_launch(records, m, n, x, idx, count, y, workspace, workspace_bytes, stream);
+    return spqt_kqw_sparse_gemv(records, m, n, 4, x, idx, count, y, workspace, workspace_bytes, stream);
 }
 
 spqt_status spqt_kq_dense_gemv(const void* records, int m, int n, const void* x, void* y, void* workspace,
                                size_t workspace_bytes, void* stream)
 {
-    return spqt::kq_launch(records, m, n, x, nullptr, nullptr, y, workspace, workspace_bytes, stream);
+    return spqt_kqw_dense_gemv(records, m, n, 4, x, y, workspace, workspace_bytes, stream);
 }
 
 }  // extern "C"

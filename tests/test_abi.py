@@ -123,6 +123,14 @@ def test_sizes_and_refusals_of_the_rowwise_and_two_level_entries(L):
     assert L.spqt_kq_pack(None, 256, 8, 8, None, None) == 1
     assert L.spqt_kq_dense_gemv(None, 256, 8, None, None, None, 0, None) == 1
     assert L.spqt_kq_sparse_gemv(None, 256, 8, None, None, None, None, None, 0, None) == 1
+    # other code widths of the same format: sizes per width, unsupported widths, null pointers
+    assert binding.spqt_kqw_packed_sizes(14336, 4096, 4) == (rec, ws)
+    assert binding.spqt_kqw_packed_sizes(14336, 4096, 2)[0] == 56 * 4096 * 80
+    assert binding.spqt_kqw_packed_sizes(14336, 4096, 8) == (56 * 4096 * 272, ws)
+    assert L.spqt_kqw_packed_sizes(256, 8, 3, ctypes.byref(sz), None) == 2
+    assert L.spqt_kqw_pack(None, 256, 8, 8, 8, None, None) == 1
+    assert L.spqt_kqw_dense_gemv(None, 256, 8, 2, None, None, None, 0, None) == 1
+    assert L.spqt_kqw_sparse_gemv(None, 256, 8, 8, None, None, None, None, None, 0, None) == 1
 
 
 def test_host_step_refuses_bad_arguments_without_touching_the_device(L):

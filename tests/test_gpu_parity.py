@@ -1049,3 +1049,60 @@ def test_kq_refuses_what_it_does_not_cover():
     assert L.spqt_kq_dense_gemv(a, 256, 8, a, a, a, 16, None) == 4           # workspace too small
     assert L.spqt_kq_sparse_gemv(a, 256, 8, a, None, a, a, a, 1 << 16, None) == 1
     assert L.spqt_kq_dense_gemv(a + 8, 256, 8, a, a, a, 1 << 16, None) == 3
+
+
+@pytest.mark.parametrize("bits", [2, 8])
+@pytest.mark.parametrize("m_blocks,n", [(1, 1), (2, 1111), (16, 4096), (4, 14336)])
+def test_kq_other_code_widths_match_the_oracle(bits, m_blocks, n):
+    """The two-level format with 2- and 8-bit codes: record bytes identical to the oracle's, sparse and dense
+    products within the tolerance, repeated calls bit-identical."""
+    m = 256 * m_blocks
+    W = inputs.weights(m, n, seed=5 * m_blocks + n + bits)
+    if n >= 300:
+        W[:32, 0] = np.abs(W[:32, 0])
+        W[:256, 1] = np.float16(0.0)
+        W[:256, 2] = np.float16(-0.0)
+        W[32:64, 3] = np.float16(0.125)
+    x = inputs.activations(n, seed=m_blocks + 90, dist="gauss" if n > 8192 else "laplace")
+    q, sc, mn, d, dmin = oracle.kq_quantize(W, bits=bits)
+    p = binding.spqt_kqw_pack(dev(W), bits)
+    torch.cuda.synchronize()
+    got = p.records.cpu().numpy()
+    want = oracle.kq_pack(q, sc, mn, d, dmin, bits=bits)
+    assert got.size == want.size == m_blocks * n * oracle.kq_record_bytes(bits=bits)
+    assert np.array_equal(got, want), "first differing byte %d" % int(np.nonzero(got != want)[0][0])
+    ws = binding.new_kq_workspace(p)
+    xd = dev(x)
+    for sp in (0.5, 0.9, 0.0, None):
+        t = float("inf") if sp is None else inputs.threshold_for_sparsity(x, sp)
+        idx, cnt = binding.spqt_sparsify(xd, t)
+        y = torch.full((m,), float("nan"), dtype=torch.float16, device="cuda")
+        binding.spqt_kqw_sparse_gemv(p, xd, idx, cnt, ws, y)
+        torch.cuda.synchronize()
+        c = int(cnt.item())
+        y_ref, bound = oracle.kq_gemv(q, sc, mn, d, dmin, x, idx.cpu().numpy()[:c])
+        check_y(y.cpu().numpy(), y_ref, bound, "two-level %d-bit sparse, sparsity %r" % (bits, sp))
+        y2 = binding.spqt_kqw_sparse_gemv(p, xd, idx, cnt, ws)
+        torch.cuda.synchronize()
+        assert torch.equal(y.view(torch.int16), y2.view(torch.int16))
+    yd = binding.spqt_kqw_dense_gemv(p, xd, ws)
+    torch.cuda.synchronize()
+    y_ref, bound = oracle.kq_gemv(q, sc, mn, d, dmin, x)
+    check_y(yd.cpu().numpy(), y_ref, bound, "two-level %d-bit dense" % bits)
+    assert not ws[: 4 * m_blocks].any()
+
+
+def test_kq_width_four_is_the_plain_format_and_other_widths_are_refused():
+    W = inputs.weights(512, 300, seed=3)
+    a = binding.spqt_kq_pack(dev(W))
+    b = binding.spqt_kqw_pack(dev(W), 4)
+    torch.cuda.synchronize()
+    assert torch.equal(a.records, b.records)
+    L = binding.lib()
+    buf = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    p = buf.data_ptr()
+    for bits in (1, 3, 5, 6, 7, 16):
+        assert L.spqt_kqw_pack(p, 256, 8, 8, bits, p, None) == 2
+        assert L.spqt_kqw_dense_gemv(p, 256, 8, bits, p, p, p, 1 << 16, None) == 2
+    assert binding.spqt_kqw_packed_sizes(512, 10, 2)[0] == 2 * 10 * 80
+    assert binding.spqt_kqw_packed_sizes(512, 10, 8)[0] == 2 * 10 * 272
