@@ -277,12 +277,13 @@ def other_config_line(which, local, quick=False):
                         rows=rows)
         elif which == "kquant":
             rows = sweep.kq_sweep(peak)
-            r0 = [r for r in rows if r["m"] == 28672 and r["n"] == 8192][0]
+            r0 = [r for r in rows if r["m"] == 28672 and r["n"] == 8192 and r["bits"] == 4][0]
             nb = r0["sparse_gbs"] * r0["sparse_us"] * 1e3
             line = dict(base, metric="sparse GEMV over the two-level format (256-row superblocks, 6-bit block scales and minimums), effective HBM GB/s at 50% sparsity, 28672x8192",
                         value=r0["sparse_gbs"], ms_per_step=r0["sparse_us"] * 1e-3, steps=20, warmup=4,
                         config={"workload": "two-level format in the zigzag arrangement, 144-byte records; index list given (and, beside it, collected by a launch of its own); "
-                                            "50% sparsity; Llama-3-8B-shaped linears and 28672x8192; rotated weight copies > 2x L2"},
+                                            "50% sparsity; Llama-3-8B-shaped linears and 28672x8192 with 4-bit codes, 28672x4096 and 28672x8192 also with 2- and 8-bit codes "
+                                            "(80- and 272-byte records); rotated weight copies > 2x L2"},
                         roofline=roofline_obj(r0["sparse_gbs"], peak, kind, nb, r0["sparse_us"], "kq_gemv_kernel", None),
                         rows=rows)
         elif which == "batch":
@@ -623,8 +624,9 @@ def run_ours(args):
             for r in ba["rows"] if r["m"] == 28672 and r["rows"] == "beam-like"}
         kq = other_config_line("kquant", local)
         others["two_level_format_at_50pct"] = {
-            "%dx%d" % (r["m"], r["n"]): {"sparse_frac_of_peak": r["frac_of_peak"], "dense_frac_of_peak": r["dense_frac_of_peak"],
-                                         "speedup_vs_dense": r["speedup_vs_dense"]} for r in kq["rows"]}
+            "%dx%d%s" % (r["m"], r["n"], "" if r["bits"] == 4 else " %d-bit codes" % r["bits"]):
+                {"sparse_frac_of_peak": r["frac_of_peak"], "dense_frac_of_peak": r["dense_frac_of_peak"],
+                 "speedup_vs_dense": r["speedup_vs_dense"]} for r in kq["rows"]}
 
     if rank == 0:
         cpu = oracle_sample(3, 1) if world >= 1 else None

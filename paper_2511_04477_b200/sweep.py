@@ -221,20 +221,25 @@ def dense_shape_sweep(peak):
 
 
 def kq_sweep(peak):
-    """The two-level format (144-byte records of 256 rows of a column): the index collection followed by the
-    sparse product over the list at 50 %, the product alone, and the dense product, on Llama-3-8B-shaped linears
-    and one Llama-2-70B-shaped one.  Needed bytes per active superblock: 144."""
+    """The two-level format (one record per 256 rows of a column): the index collection followed by the sparse
+    product over the list at 50 %, the product alone, and the dense product, on Llama-3-8B-shaped linears and one
+    Llama-2-70B-shaped one with 4-bit codes, and with 2- and 8-bit codes on the two largest.  Needed bytes per
+    active superblock: the record, 144 bytes (80 and 272 with 2- and 8-bit codes)."""
     out = []
-    for (m, n, dist) in [(4096, 4096, "laplace"), (6144, 4096, "laplace"), (28672, 4096, "laplace"), (4096, 14336, "gauss"),
-                         (28672, 8192, "laplace")]:
+    cases = [(4096, 4096, "laplace", 4), (6144, 4096, "laplace", 4), (28672, 4096, "laplace", 4), (4096, 14336, "gauss", 4),
+             (28672, 8192, "laplace", 4),
+             # the other code widths, on the two large shapes
+             (28672, 4096, "laplace", 2), (28672, 4096, "laplace", 8), (28672, 8192, "laplace", 2), (28672, 8192, "laplace", 8)]
+    for (m, n, dist, bits) in cases:
         R = m // 256
-        copies = int(min(64, max(4, math.ceil(2.4 * L2_BYTES / (R * n * 144)))))
+        rec = 256 * bits // 8 + 16
+        copies = int(min(64, max(4, math.ceil(2.4 * L2_BYTES / (R * n * rec)))))
         g = torch.Generator(device="cuda")
         packs = []
         for c in range(copies):
             g.manual_seed(c)
             W = torch.empty((m, n), dtype=torch.float32, device="cuda").normal_(0.0, 0.02, generator=g).half()
-            packs.append(binding.spqt_kq_pack(W))
+            packs.append(binding.spqt_kqw_pack(W, bits))
             del W
         x = inputs.activations(n, seed=21, dist=dist)
         t = inputs.threshold_for_sparsity(x, 0.5)
@@ -248,12 +253,12 @@ def kq_sweep(peak):
 
         def both(i, s):
             binding.spqt_sparsify(xd, t, idx, cnt, stream=s)
-            binding.spqt_kq_sparse_gemv(packs[i % copies], xd, idx, cnt, ws, y, stream=s)
+            binding.spqt_kqw_sparse_gemv(packs[i % copies], xd, idx, cnt, ws, y, stream=s)
         us_both, _ = graph_us(both, calls)
-        us_sp, _ = graph_us(lambda i, s: binding.spqt_kq_sparse_gemv(packs[i % copies], xd, idx, cnt, ws, y, stream=s), calls)
-        us_de, _ = graph_us(lambda i, s: binding.spqt_kq_dense_gemv(packs[i % copies], xd, ws, y, stream=s), calls)
-        nb = lambda c: c * R * 144 + 2 * n + 4 * c + 4 + 2 * m
-        out.append({"m": m, "n": n, "count": count, "copies": copies, "sparsify_plus_sparse_us": us_both, "sparse_us": us_sp,
+        us_sp, _ = graph_us(lambda i, s: binding.spqt_kqw_sparse_gemv(packs[i % copies], xd, idx, cnt, ws, y, stream=s), calls)
+        us_de, _ = graph_us(lambda i, s: binding.spqt_kqw_dense_gemv(packs[i % copies], xd, ws, y, stream=s), calls)
+        nb = lambda c: c * R * rec + 2 * n + 4 * c + 4 + 2 * m
+        out.append({"m": m, "n": n, "bits": bits, "count": count, "copies": copies, "sparsify_plus_sparse_us": us_both, "sparse_us": us_sp,
                     "dense_us": us_de, "sparse_gbs": nb(count) / us_sp * 1e-3, "frac_of_peak": nb(count) / us_sp * 1e-3 / peak,
                     "dense_gbs": nb(n) / us_de * 1e-3, "dense_frac_of_peak": nb(n) / us_de * 1e-3 / peak,
                     "speedup_vs_dense": us_de / us_sp, "speedup_vs_dense_with_index_collection": us_de / us_both})
