@@ -282,10 +282,12 @@ def rowwise_thresholded_gemv(q, scales, zeros, x, t: float, group: int = 128):
 # Record of a superblock (G = sub*nsub weights): G/2 bytes of codes (byte i = q_i | q_{i+G/2} << 4), then the
 # 2*nsub six-bit fields sc_0.., m_0.. as a little-endian bit string (field f at bits 6f..6f+5) padded to whole
 # bytes, then d and dmin as little-endian fp16: 128 + 12 + 4 = 144 bytes for sub = 32, nsub = 8.
-# Other code widths (Sec. 4.1.3: any width from 2 to 8 bits): bits = 2 or 8 puts 2^bits - 1 in the place of 15
-# and changes the code bytes only -- 8 bits: byte i = q_i (G bytes); 2 bits: byte i = q_i | q_{i+G/4} << 2 |
-# q_{i+G/2} << 4 | q_{i+3G/4} << 6 (G/4 bytes); records of 272 and 80 bytes.  Pinned by hand-worked superblocks
-# (tests/golden/kq_superblock_2bit.txt, _8bit.txt), the scalar restatement, the error bound and the layout check.
+# Other code widths (Sec. 4.1.3: any width from 2 to 8 bits): bits = 2, 5, 6 or 8 puts 2^bits - 1 in the place
+# of 15 and changes the code bytes only -- 8 bits: byte i = q_i (G bytes); 2 bits: byte i = q_i | q_{i+G/4} << 2 |
+# q_{i+G/2} << 4 | q_{i+3G/4} << 6 (G/4 bytes); 5 and 6 bits: the low four bits of every code as for 4 bits, then
+# the high bits q >> 4, one per row (bit j%8 of byte j/8) or two per row arranged like 2-bit codes; records of
+# 80, 176, 208 and 272 bytes.  Pinned by hand-worked superblocks (tests/golden/kq_superblock_2bit.txt, _5bit,
+# _6bit, _8bit), the scalar restatement, the error bound and the layout check.
 
 def kq_record_bytes(sub: int = 32, nsub: int = 8, bits: int = 4) -> int:
     return sub * nsub * bits // 8 + (12 * nsub + 7) // 8 + 4
@@ -293,8 +295,8 @@ def kq_record_bytes(sub: int = 32, nsub: int = 8, bits: int = 4) -> int:
 
 def kq_quantize(W, sub: int = 32, nsub: int = 8, bits: int = 4):
     """fp16 W[m][n] -> (q uint8[m][n], sc uint8[R][nsub][n], mn uint8[R][nsub][n], d fp16[R][n], dmin fp16[R][n]).
-    bits = width of a code (2, 4 or 8): the codes run from 0 to 2^bits - 1, everything else is the same rule."""
-    assert bits in (2, 4, 8)
+    bits = width of a code (2, 4, 5, 6 or 8): the codes run from 0 to 2^bits - 1, everything else is the same rule."""
+    assert bits in (2, 4, 5, 6, 8)
     top = np.float32((1 << bits) - 1)
     W = np.ascontiguousarray(W, dtype=np.float16)
     m, n = W.shape
@@ -323,8 +325,10 @@ def kq_quantize(W, sub: int = 32, nsub: int = 8, bits: int = 4):
 def kq_pack(q, sc, mn, d, dmin, sub: int = 32, nsub: int = 8, bits: int = 4) -> np.ndarray:
     """The records, uint8[R][n][record bytes] flattened (superblock (r, k) at record index r*n + k).  Codes of a
     superblock's G rows: 4 bits, byte i = q_i | q_{i+G/2} << 4; 8 bits, byte i = q_i; 2 bits, byte i =
-    q_i | q_{i+G/4} << 2 | q_{i+G/2} << 4 | q_{i+3G/4} << 6."""
-    assert bits in (2, 4, 8)
+    q_i | q_{i+G/4} << 2 | q_{i+G/2} << 4 | q_{i+3G/4} << 6; 5 and 6 bits, the low four bits of every code as
+    for 4 bits (G/2 bytes), then the high bits h = q >> 4: one bit per row, bit j%8 of byte j/8 (5 bits), or
+    two bits per row arranged like 2-bit codes (6 bits)."""
+    assert bits in (2, 4, 5, 6, 8)
     G = sub * nsub
     m, n = q.shape
     R = m // G
@@ -332,10 +336,23 @@ def kq_pack(q, sc, mn, d, dmin, sub: int = 32, nsub: int = 8, bits: int = 4) -> 
     nc = G * bits // 8
     rec = np.zeros((R, n, kq_record_bytes(sub, nsub, bits)), np.uint8)
     qb = q.reshape(R, G, n)
-    per = 8 // bits                                   # codes per byte
-    codes = np.zeros((R, nc, n), np.uint8)
-    for f in range(per):
-        codes |= (qb[:, f * nc:(f + 1) * nc, :] << (bits * f)).astype(np.uint8)
+    def plane(v, width):                              # G values of `width` bits -> G*width/8 bytes, 8/width per byte
+        nb, per = G * width // 8, 8 // width
+        out = np.zeros((R, nb, n), np.uint8)
+        for f in range(per):
+            out |= (v[:, f * nb:(f + 1) * nb, :] << (width * f)).astype(np.uint8)
+        return out
+    if bits in (2, 4, 8):
+        codes = plane(qb, bits)
+    else:
+        h = qb >> 4
+        if bits == 5:                                 # bit j % 8 of byte j / 8
+            high = np.zeros((R, G // 8, n), np.uint8)
+            for e in range(8):
+                high |= (h[:, e::8, :] << e).astype(np.uint8)
+        else:
+            high = plane(h, 2)
+        codes = np.concatenate([plane(qb & 15, 4), high], axis=1)
     rec[:, :, :nc] = codes.transpose(0, 2, 1)
     fields = np.concatenate([sc, mn], axis=1).astype(np.uint64)        # [R][2*nsub][n]
     fbits = np.zeros((R, n), dtype=object)

@@ -548,7 +548,8 @@ def test_kq_hand_worked_superblock():
     assert y.tolist() == [2 * float(v) for v in g["dequantized"]] and bound.tolist() == [2 * abs(float(v)) for v in g["dequantized"]]
 
 
-@pytest.mark.parametrize("bits,name", [(2, "kq_superblock_2bit.txt"), (8, "kq_superblock_8bit.txt")])
+@pytest.mark.parametrize("bits,name", [(2, "kq_superblock_2bit.txt"), (5, "kq_superblock_5bit.txt"),
+                                       (6, "kq_superblock_6bit.txt"), (8, "kq_superblock_8bit.txt")])
 def test_kq_hand_worked_superblock_other_widths(bits, name):
     g = _golden_kq(name)
     W = np.array([float(v) for v in g["w"]], dtype=np.float16).reshape(8, 1)
@@ -558,12 +559,12 @@ def test_kq_hand_worked_superblock_other_widths(bits, name):
     assert int(d.view(np.uint16)[0, 0]) == int(g["d_bits"][0], 16) and int(dmin.view(np.uint16)[0, 0]) == int(g["dmin_bits"][0], 16)
     assert oracle.kq_pack(q, sc, mn, d, dmin, 4, 2, bits).tolist() == [int(v, 16) for v in g["record"]]
     assert oracle.kq_record_bytes(4, 2, bits) == len(g["record"])
-    assert oracle.kq_record_bytes(bits=2) == 80 and oracle.kq_record_bytes(bits=8) == 272
+    assert [oracle.kq_record_bytes(bits=b) for b in (2, 5, 6, 8)] == [80, 176, 208, 272]
     What = oracle.kq_dequantize_rows(q, sc, mn, d, dmin, np.arange(8), 4, 2).ravel()
     assert What.tolist() == [float(v) for v in g["dequantized"]]
 
 
-@pytest.mark.parametrize("bits", [4, 2, 8])
+@pytest.mark.parametrize("bits", [4, 2, 5, 6, 8])
 def test_kq_quantizer_against_a_scalar_restatement(bits):
     f32 = np.float32
     top = (1 << bits) - 1
@@ -596,7 +597,7 @@ def test_kq_quantizer_against_a_scalar_restatement(bits):
     assert mn[0, 0, 0] == 0 and mn[0, 1, 2] > 0
 
 
-@pytest.mark.parametrize("bits", [2, 8])
+@pytest.mark.parametrize("bits", [2, 5, 6, 8])
 def test_kq_error_bound_and_code_layout_other_widths(bits):
     rng = np.random.default_rng(24)
     m, n, top = 512, 24, (1 << bits) - 1
@@ -615,17 +616,26 @@ def test_kq_error_bound_and_code_layout_other_widths(bits):
     q4, sc4, mn4, d4, dmin4 = oracle.kq_quantize(W)
     err4 = np.abs(oracle.kq_dequantize_rows(q4, sc4, mn4, d4, dmin4, np.arange(m)) - W.astype(np.float64))
     ratio = np.mean(err) / np.mean(err4)
-    assert (3.0 < ratio < 7.0) if bits == 2 else (ratio < 0.25)
+    # mean error against the 4-bit format's: about 15 / (2^bits - 1)
+    assert {2: 3.0, 5: 0.35, 6: 0.17, 8: 0.03}[bits] < ratio < {2: 7.0, 5: 0.65, 6: 0.35, 8: 0.25}[bits]
     # the record: codes (2 bits: four quarter-planes per byte; 8 bits: one per byte), fields, d, dmin
     nc = 256 * bits // 8
     rec = oracle.kq_pack(q, sc, mn, d, dmin, bits=bits).reshape(2, n, nc + 16)
     for (r, k) in [(0, 0), (1, 11), (1, 23)]:
         b = rec[r, k]
+        col = q[r * 256:(r + 1) * 256, k].astype(int)
+        quarters = lambda v, i: v[i] | (v[64 + i] << 2) | (v[128 + i] << 4) | (v[192 + i] << 6)
         for i in range(nc):
             if bits == 8:
-                assert b[i] == q[r * 256 + i, k]
-            else:
-                assert b[i] == (q[r * 256 + i, k] | (q[r * 256 + 64 + i, k] << 2) | (q[r * 256 + 128 + i, k] << 4) | (q[r * 256 + 192 + i, k] << 6))
+                assert b[i] == col[i]
+            elif bits == 2:
+                assert b[i] == quarters(col, i)
+            elif i < 128:                               # 5 and 6 bits: the low four bits like 4-bit codes
+                assert b[i] == ((col[i] & 15) | ((col[128 + i] & 15) << 4))
+            elif bits == 5:                             # then one high bit per row
+                assert b[i] == sum(((col[8 * (i - 128) + e] >> 4) & 1) << e for e in range(8))
+            else:                                       # or two, arranged like 2-bit codes
+                assert b[i] == quarters(col >> 4, i - 128)
         fb = int.from_bytes(bytes(b[nc:nc + 12].tolist()), "little")
         assert [(fb >> (6 * f)) & 63 for f in range(16)] == sc[r, :, k].tolist() + mn[r, :, k].tolist()
         assert int.from_bytes(bytes(b[nc + 12:nc + 14].tolist()), "little") == int(d.view(np.uint16)[r, k])
