@@ -372,11 +372,16 @@ spqt_status spqt_kq_dense_gemv(const void* records, int m, int n, const void* x,
 
 /*
  * The same format with other code widths (paper Sec. 4.1.3: the grouping works for any code width from
- * 2 to 8 bits).  bits = 2, 4 or 8 (SPQT_ERR_UNSUPPORTED otherwise); bits = 4 is exactly the format above.
- * 2^bits - 1 takes the place of 15 in the rule, and only the code bytes of a record change:
+ * 2 to 8 bits).  bits = 2, 4, 5, 6 or 8 (SPQT_ERR_UNSUPPORTED otherwise); bits = 4 is exactly the format
+ * above.  2^bits - 1 takes the place of 15 in the rule, and only the code bytes of a record change:
  *   bits = 8 : bytes 0..255, byte i = q_i; record of 272 bytes (fields at 256, d and dmin at 268)
  *   bits = 2 : bytes 0..63,  byte i = q_i | q_{i+64} << 2 | q_{i+128} << 4 | q_{i+192} << 6;
  *              record of 80 bytes (fields at 64, d and dmin at 76)
+ *   bits = 5 : bytes 0..127 the low four bits, byte i = (q_i & 15) | (q_{i+128} & 15) << 4; bytes 128..159
+ *              the fifth bit of every row, bit j%8 of byte 128 + j/8; record of 176 bytes
+ *   bits = 6 : bytes 0..127 as for 5; bytes 128..191 the high two bits h = q >> 4, byte 128 + i =
+ *              h_i | h_{i+64} << 2 | h_{i+128} << 4 | h_{i+192} << 6; record of 208 bytes
+ * (the fields follow the code bytes, then d and dmin).
  * Arguments, workspace, alignment and error behaviour as for the spqt_kq_* calls; the workspace does not
  * depend on the width.
  */

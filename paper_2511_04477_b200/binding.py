@@ -456,7 +456,7 @@ def spqt_rowwise_dense_gemv(p: RowwisePacked, x: torch.Tensor, y: torch.Tensor =
 @dataclass
 class KqPacked:
     """Device buffer written by :func:`spqt_kq_pack` (144-byte records of the two-level format, zigzag order)."""
-    records: torch.Tensor      # uint8[(m/256)*n*144]  (80 or 272 bytes per record with 2- or 8-bit codes)
+    records: torch.Tensor      # uint8[(m/256)*n*144]  (80, 176, 208 or 272 bytes per record with 2-, 5-, 6- or 8-bit codes)
     m: int
     n: int
     bits: int = 4
@@ -487,7 +487,7 @@ def spqt_kqw_packed_sizes(m: int, n: int, bits: int):
 
 
 def spqt_kqw_pack(W: torch.Tensor, bits: int, stream=None) -> KqPacked:
-    """The two-level format with 2-, 4- or 8-bit codes."""
+    """The two-level format with 2-, 4-, 5-, 6- or 8-bit codes."""
     if W.dim() != 2 or W.stride(1) != 1:
         raise ValueError("W must be 2-D with unit column stride")
     if not W.is_cuda or W.dtype != torch.float16:

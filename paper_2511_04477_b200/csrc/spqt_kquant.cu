@@ -6,11 +6,14 @@
 // m_0..7 as a little-endian bit string (12 bytes), d and dmin as fp16.  Dequantized weight of row j of
 // block i:  d*sc_i*q_j - dmin*m_i.  The paper fixes neither the rounding rule nor the bit arrangement;
 // the rule implemented is stated at kq_pack_kernel, every step a single IEEE fp32 operation.
-// Other code widths (Sec. 4.1.3: any width from 2 to 8 bits): the kernels are templates over BITS = 2, 4, 8;
-// 2^BITS - 1 replaces 15 in the rule and only the code bytes of a record change -- 8 bits: byte i = q_i (256
+// Other code widths (Sec. 4.1.3: any width from 2 to 8 bits): the kernels are templates over BITS = 2, 4, 5, 6,
+// 8; 2^BITS - 1 replaces 15 in the rule and only the code bytes of a record change -- 8 bits: byte i = q_i (256
 // bytes, records of 272); 2 bits: byte i = q_i | q_{i+64} << 2 | q_{i+128} << 4 | q_{i+192} << 6 (64 bytes,
-// records of 80).  Their arithmetic sums, per 16-bit half-word, the value of its low byte and of both bytes
-// (the cumulative form of the main kernel) and takes the difference at the end.
+// records of 80); 5 and 6 bits: the low four bits as 4-bit codes, then a plane of the high bits q >> 4, one per
+// row (bit j%8 of byte j/8) or two per row arranged like 2-bit codes (records of 176 and 208).  The arithmetic of
+// the 2- and 8-bit codes and of the high planes sums cumulative values (per 16-bit half-word the value of its
+// first code and of both codes together; per byte of single bits its low 1, 2, .. 8 bits: the cumulative form of
+// the main kernel) and takes the differences at the end.
 //
 //   kq_pack_kernel   a CTA stages a 256 x 32 tile of W; a warp quantizes four columns, lane l owning rows
 //                    l, l+32, .. (one row of every block).
@@ -37,7 +40,7 @@ namespace spqt {
 constexpr int kKqG = 256;           // rows of a superblock
 __host__ __device__ constexpr int kq_code_bytes(int bits) { return kKqG * bits / 8; }
 __host__ __device__ constexpr int kq_rec_bytes(int bits) { return kq_code_bytes(bits) + 16; }
-__host__ __device__ constexpr int kq_ctas_per_sm(int bits) { return bits == 8 ? 2 : 3; }   // (shared memory: two record buffers per warp)
+__host__ __device__ constexpr int kq_ctas_per_sm(int bits) { return bits >= 5 ? 2 : 3; }   // (registers of a second accumulator set; shared memory of the record buffers)
 constexpr int kKqWarps = 8;
 constexpr int kKqThreads = kKqWarps * 32;
 constexpr int kKqChunk = 16;        // list entries per chunk
@@ -105,6 +108,22 @@ kq_pack_kernel(const __half* __restrict__ W, int n, int ldw, uint8_t* __restrict
         } else if (BITS == 8) {     // byte i = code of row i
 #pragma unroll
             for (int u = 0; u < 8; ++u) rec[lane + 32 * u] = (uint8_t)q[u];
+        } else if (BITS == 5 || BITS == 6) {
+            // the low four bits like 4-bit codes, then the high bits: one per row, bit j % 8 of byte j / 8 (the
+            // 32 rows lane + 32u of all lanes are one 32-bit word), or two per row arranged like 2-bit codes
+#pragma unroll
+            for (int u = 0; u < 4; ++u) rec[lane + 32 * u] = (uint8_t)((q[u] & 15) | ((q[u + 4] & 15) << 4));
+            if (BITS == 5) {
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const unsigned bal = __ballot_sync(0xffffffffu, (q[u] >> 4) & 1);
+                    if (lane == 0) reinterpret_cast<unsigned*>(rec + 128)[u] = bal;
+                }
+            } else {
+#pragma unroll
+                for (int u = 0; u < 2; ++u)
+                    rec[128 + lane + 32 * u] = (uint8_t)((q[u] >> 4) | ((q[u + 2] >> 4) << 2) | ((q[u + 4] >> 4) << 4) | ((q[u + 6] >> 4) << 6));
+            }
         } else {                    // byte i = codes of rows i, i + 64, i + 128, i + 192, two bits each
 #pragma unroll
             for (int u = 0; u < 2; ++u) rec[lane + 32 * u] = (uint8_t)(q[u] | (q[u + 2] << 2) | (q[u + 4] << 4) | (q[u + 6] << 6));
@@ -180,6 +199,10 @@ kq_gemv_kernel(const uint8_t* __restrict__ records, int n, const __half* __restr
     unsigned long long acc[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc[i] = 0ull;
+    constexpr bool kHigh = BITS == 5 || BITS == 6;   // a second plane with the bits above the low four
+    unsigned long long acch[kHigh ? 8 : 1];          // its sums (cumulative, see the step), same rows as acc
+#pragma unroll
+    for (int i = 0; i < (kHigh ? 8 : 1); ++i) acch[i] = 0ull;
     float zl[4] = {0.0f, 0.0f, 0.0f, 0.0f};      // x*dmin*m of blocks 4*half .. 4*half+3
 
     // column of the entry lanes e and e+16 hold in the chunk at list position pos (past the end: the last entry again)
@@ -226,7 +249,7 @@ kq_gemv_kernel(const uint8_t* __restrict__ records, int n, const __half* __restr
                     const int sb = 2 * half + g2;   // lane group: rows of blocks sb (low nibbles) and sb + 4 (high nibbles)
                     const float a_lo = xf * (df * (float)kq_field(tail.x, tail.y, tail.z, sb));       // d*sc is exact
                     const float a_hi = xf * (df * (float)kq_field(tail.x, tail.y, tail.z, sb + 4));
-                    if (BITS == 4)
+                    if (BITS == 4 || kHigh)
                         sts_pairs(mbuf + 16u * (unsigned)(t * 4 + sb), pack2(a_lo * 0x1p93f, a_hi * 0x1p89f),
                                   pack2(a_lo * 0x1p85f, a_hi * 0x1p81f));
                     else   // one pair: the high rows' codes sit in the same bytes (2 bits, four bits up) or in bytes of their own (8 bits)
@@ -241,11 +264,36 @@ kq_gemv_kernel(const uint8_t* __restrict__ records, int n, const __half* __restr
             const unsigned cb = rbuf + cur;
             auto step = [&](int u) {
                 const unsigned e = (unsigned)(2 * u + half);
-                if (BITS == 4) {
+                if (BITS == 4 || kHigh) {
                     const uint2 wv = lds_v2(cb + e * REC + (unsigned)t * 8u);
                     unsigned long long m01, m23;
                     lds_pairs(mbuf + 16u * (e * 4u + (unsigned)(t >> 2)), m01, m23);
-                    fma_block8(acc, wv, m01, m23);
+                    fma_block8(acc, wv, m01, m23);     // the low four bits of every code
+                    if (BITS == 6) {
+                        // the high two bits, 16 times the weight: a plane laid out like 2-bit codes, summed the same way
+                        const unsigned long long mh = fmul2(m01, pack2(16.0f, 16.0f));
+                        const uint2 hv = lds_v2(cb + e * REC + 128u + (unsigned)(t & 7) * 8u);
+                        const int sh = 2 * (t >> 3);
+#pragma unroll
+                        for (int k = 0; k < 2; ++k) {
+                            const unsigned w = (k ? hv.y : hv.x) >> sh, v = w >> 16;
+                            ffma2(acch[4 * k + 0], pack2(__uint_as_float(w & 0x03u), __uint_as_float(w & 0x30u)), mh);
+                            ffma2(acch[4 * k + 1], pack2(__uint_as_float(w & 0x0303u), __uint_as_float(w & 0x3030u)), mh);
+                            ffma2(acch[4 * k + 2], pack2(__uint_as_float(v & 0x03u), __uint_as_float(v & 0x30u)), mh);
+                            ffma2(acch[4 * k + 3], pack2(__uint_as_float(v & 0x0303u), __uint_as_float(v & 0x3030u)), mh);
+                        }
+                    } else if (BITS == 5) {
+                        // the fifth bit of rows 8t.. and 128+8t..: one byte each; position b sums the byte's low b+1 bits
+                        const unsigned long long mh = fmul2(m01, pack2(16.0f, 256.0f));   // (a_lo, a_hi) * 16 * 2^93
+                        unsigned lb, hb;
+                        asm volatile("ld.shared.u8 %0, [%1];" : "=r"(lb) : "r"(cb + e * REC + 128u + (unsigned)t) : "memory");
+                        asm volatile("ld.shared.u8 %0, [%1];" : "=r"(hb) : "r"(cb + e * REC + 144u + (unsigned)t) : "memory");
+#pragma unroll
+                        for (int b = 0; b < 8; ++b) {
+                            const unsigned mk = (2u << b) - 1u;
+                            ffma2(acch[b], pack2(__uint_as_float(lb & mk), __uint_as_float(hb & mk)), mh);
+                        }
+                    }
                     return;
                 }
                 // 2 and 8 bits: per 16-bit half-word the value of its first byte's code and the value of both
@@ -303,7 +351,33 @@ kq_gemv_kernel(const uint8_t* __restrict__ records, int n, const __half* __restr
             lo_rows[b] += __shfl_xor_sync(0xffffffffu, lo_rows[b], 16);
             hi_rows[b] += __shfl_xor_sync(0xffffffffu, hi_rows[b], 16);
         }
-        if (BITS != 4) {   // odd positions hold (first code + 256 * second code) of a half-word
+        if (kHigh) {
+            float lh[8], hh[8];
+#pragma unroll
+            for (int b = 0; b < 8; ++b) {
+                unpack2(acch[b], lh[b], hh[b]);
+                lh[b] += __shfl_xor_sync(0xffffffffu, lh[b], 16);
+                hh[b] += __shfl_xor_sync(0xffffffffu, hh[b], 16);
+            }
+            if (BITS == 6) {      // pairs, as for 2-bit codes
+#pragma unroll
+                for (int b = 1; b < 8; b += 2) {
+                    lh[b] = (lh[b] - lh[b - 1]) * 0x1p-8f;
+                    hh[b] = (hh[b] - hh[b - 1]) * 0x1p-8f;
+                }
+            } else {              // a chain over the eight bits of a byte
+#pragma unroll
+                for (int b = 7; b > 0; --b) {
+                    lh[b] = (lh[b] - lh[b - 1]) * (1.0f / (float)(1 << b));
+                    hh[b] = (hh[b] - hh[b - 1]) * (1.0f / (float)(1 << b));
+                }
+            }
+#pragma unroll
+            for (int b = 0; b < 8; ++b) {
+                lo_rows[b] += lh[b];
+                hi_rows[b] += hh[b];
+            }
+        } else if (BITS != 4) {   // odd positions hold (first code + 256 * second code) of a half-word
 #pragma unroll
             for (int b = 1; b < 8; b += 2) {
                 lo_rows[b] = (lo_rows[b] - lo_rows[b - 1]) * 0x1p-8f;
@@ -426,7 +500,7 @@ static spqt_status kq_launch(const void* records, int m, int n, const void* x, c
 
 extern "C" {
 
-static bool kq_bits_ok(int bits) { return bits == 2 || bits == 4 || bits == 8; }
+static bool kq_bits_ok(int bits) { return bits == 2 || bits == 4 || bits == 5 || bits == 6 || bits == 8; }
 
 spqt_status spqt_kqw_packed_sizes(int m, int n, int bits, size_t* records_bytes, size_t* workspace_bytes)
 {
@@ -452,6 +526,8 @@ spqt_status spqt_kqw_pack(const void* W, int m, int n, int ldw, int bits, void* 
     uint8_t* rec = static_cast<uint8_t*>(records);
     if (bits == 2) spqt::kq_pack_kernel<2><<<grid, 256, 0, st_>>>(w, n, ldw, rec);
     else if (bits == 4) spqt::kq_pack_kernel<4><<<grid, 256, 0, st_>>>(w, n, ldw, rec);
+    else if (bits == 5) spqt::kq_pack_kernel<5><<<grid, 256, 0, st_>>>(w, n, ldw, rec);
+    else if (bits == 6) spqt::kq_pack_kernel<6><<<grid, 256, 0, st_>>>(w, n, ldw, rec);
     else spqt::kq_pack_kernel<8><<<grid, 256, 0, st_>>>(w, n, ldw, rec);
     spqt::count_launch();
     return cudaGetLastError() == cudaSuccess ? SPQT_OK : SPQT_ERR_CUDA;
@@ -462,6 +538,8 @@ static spqt_status kq_launch_bits(int bits, const void* records, int m, int n, c
 {
     if (bits == 2) return spqt::kq_launch<2>(records, m, n, x, idx, count, y, workspace, workspace_bytes, stream);
     if (bits == 4) return spqt::kq_launch<4>(records, m, n, x, idx, count, y, workspace, workspace_bytes, stream);
+    if (bits == 5) return spqt::kq_launch<5>(records, m, n, x, idx, count, y, workspace, workspace_bytes, stream);
+    if (bits == 6) return spqt::kq_launch<6>(records, m, n, x, idx, count, y, workspace, workspace_bytes, stream);
     if (bits == 8) return spqt::kq_launch<8>(records, m, n, x, idx, count, y, workspace, workspace_bytes, stream);
     return SPQT_ERR_UNSUPPORTED;
 }

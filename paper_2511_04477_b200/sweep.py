@@ -224,12 +224,13 @@ def kq_sweep(peak):
     """The two-level format (one record per 256 rows of a column): the index collection followed by the sparse
     product over the list at 50 %, the product alone, and the dense product, on Llama-3-8B-shaped linears and one
     Llama-2-70B-shaped one with 4-bit codes, and with 2- and 8-bit codes on the two largest.  Needed bytes per
-    active superblock: the record, 144 bytes (80 and 272 with 2- and 8-bit codes)."""
+    active superblock: the record, 144 bytes (80, 176, 208 and 272 with 2-, 5-, 6- and 8-bit codes)."""
     out = []
     cases = [(4096, 4096, "laplace", 4), (6144, 4096, "laplace", 4), (28672, 4096, "laplace", 4), (4096, 14336, "gauss", 4),
              (28672, 8192, "laplace", 4),
              # the other code widths, on the two large shapes
-             (28672, 4096, "laplace", 2), (28672, 4096, "laplace", 8), (28672, 8192, "laplace", 2), (28672, 8192, "laplace", 8)]
+             (28672, 4096, "laplace", 2), (28672, 4096, "laplace", 8), (28672, 8192, "laplace", 2), (28672, 8192, "laplace", 5),
+             (28672, 8192, "laplace", 6), (28672, 8192, "laplace", 8)]
     for (m, n, dist, bits) in cases:
         R = m // 256
         rec = 256 * bits // 8 + 16

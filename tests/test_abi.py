@@ -127,6 +127,8 @@ def test_sizes_and_refusals_of_the_rowwise_and_two_level_entries(L):
     assert binding.spqt_kqw_packed_sizes(14336, 4096, 4) == (rec, ws)
     assert binding.spqt_kqw_packed_sizes(14336, 4096, 2)[0] == 56 * 4096 * 80
     assert binding.spqt_kqw_packed_sizes(14336, 4096, 8) == (56 * 4096 * 272, ws)
+    assert binding.spqt_kqw_packed_sizes(14336, 4096, 5)[0] == 56 * 4096 * 176
+    assert binding.spqt_kqw_packed_sizes(14336, 4096, 6)[0] == 56 * 4096 * 208
     assert L.spqt_kqw_packed_sizes(256, 8, 3, ctypes.byref(sz), None) == 2
     assert L.spqt_kqw_pack(None, 256, 8, 8, 8, None, None) == 1
     assert L.spqt_kqw_dense_gemv(None, 256, 8, 2, None, None, None, 0, None) == 1

@@ -1051,10 +1051,10 @@ def test_kq_refuses_what_it_does_not_cover():
     assert L.spqt_kq_dense_gemv(a + 8, 256, 8, a, a, a, 1 << 16, None) == 3
 
 
-@pytest.mark.parametrize("bits", [2, 8])
+@pytest.mark.parametrize("bits", [2, 5, 6, 8])
 @pytest.mark.parametrize("m_blocks,n", [(1, 1), (2, 1111), (16, 4096), (4, 14336)])
 def test_kq_other_code_widths_match_the_oracle(bits, m_blocks, n):
-    """The two-level format with 2- and 8-bit codes: record bytes identical to the oracle's, sparse and dense
+    """The two-level format with 2-, 5-, 6- and 8-bit codes: record bytes identical to the oracle's, sparse and dense
     products within the tolerance, repeated calls bit-identical."""
     m = 256 * m_blocks
     W = inputs.weights(m, n, seed=5 * m_blocks + n + bits)
@@ -1101,8 +1101,10 @@ def test_kq_width_four_is_the_plain_format_and_other_widths_are_refused():
     L = binding.lib()
     buf = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
     p = buf.data_ptr()
-    for bits in (1, 3, 5, 6, 7, 16):
+    for bits in (1, 3, 7, 16):
         assert L.spqt_kqw_pack(p, 256, 8, 8, bits, p, None) == 2
         assert L.spqt_kqw_dense_gemv(p, 256, 8, bits, p, p, p, 1 << 16, None) == 2
     assert binding.spqt_kqw_packed_sizes(512, 10, 2)[0] == 2 * 10 * 80
     assert binding.spqt_kqw_packed_sizes(512, 10, 8)[0] == 2 * 10 * 272
+    assert binding.spqt_kqw_packed_sizes(512, 10, 5)[0] == 2 * 10 * 176
+    assert binding.spqt_kqw_packed_sizes(512, 10, 6)[0] == 2 * 10 * 208
