@@ -1,11 +1,11 @@
 """Run one sparse and one dense GEMV a few times on a single packed matrix, with L2 flushed
 before every call -- a small, self-terminating case for `ncu` captures.
 
-    python -m paper_2511_04477_b200.profile_case M N SPARSITY [GROUP] [REPEATS] [fused|pack|sparsify|rowwise|kq|batch4]
+    python -m paper_2511_04477_b200.profile_case M N SPARSITY [GROUP] [REPEATS] [fused|pack|sparsify|rowwise|kq|kq2|kq5|kq6|kq8|batch4]
 
 With `fused` the sparse call is the one that collects the indices in the same launch; with `pack` only the
 offline conversion is repeated, with `sparsify` only the index collection (L2 flushed before each as well);
-`rowwise` = the row-wise baseline's dense GEMV, `kq` = the two-level format's sparse and dense GEMV, `batch4` = four
+`rowwise` = the row-wise baseline's dense GEMV, `kq` = the two-level format's sparse and dense GEMV (`kq2`, `kq5`, `kq6`, `kq8`: with codes of that width), `batch4` = four
 beam-like rows over the union of their active sets and the dense batch call.
 
 Weights are random-init on the device (values do not affect timing); x and the threshold come
@@ -28,7 +28,7 @@ def main(argv):
     fused = mode == "fused"
     torch.manual_seed(0)
     W = (torch.randn(m, n, device="cuda", dtype=torch.float32) * 0.02).half()
-    if mode in ("rowwise", "kq"):
+    if mode == "rowwise" or mode.startswith("kq"):
         x = inputs.activations(n, seed=1)
         xd = torch.from_numpy(x).cuda()
         flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
@@ -41,15 +41,15 @@ def main(argv):
             torch.cuda.synchronize()
             print("ok rowwise")
             return
-        p = binding.spqt_kq_pack(W)
+        p = binding.spqt_kqw_pack(W, int(mode[2:] or 4))
         del W
         ws = binding.new_kq_workspace(p)
         idx, cnt = binding.spqt_sparsify(xd, inputs.threshold_for_sparsity(x, sp))
         for _ in range(repeats):
             flush.zero_()
-            binding.spqt_kq_sparse_gemv(p, xd, idx, cnt, ws)
+            binding.spqt_kqw_sparse_gemv(p, xd, idx, cnt, ws)
             flush.zero_()
-            binding.spqt_kq_dense_gemv(p, xd, ws)
+            binding.spqt_kqw_dense_gemv(p, xd, ws)
         torch.cuda.synchronize()
         print("ok kq count=%d" % int(cnt.item()))
         return
