@@ -1140,8 +1140,14 @@ static spqt_status launch_gemv(const Format& f, const void* codes, const void* m
         // While a CTA's share stays under half a megabyte the launch is latency-bound, and leaving up to a
         // quarter of the SMs idle costs less than partial sums that cross CTAs in a ragged pattern
         // (measured: 14336 x 4096 on 112 CTAs, one block-row each, 8.9 us against 9.7 us on 148).
-        const bool light = (size_t)f.R * row_bytes / (size_t)P < (size_t(512) << 10);
-        if (small || k * f.R * 100 >= (light ? 75 : 85) * P) P = k * f.R;
+        const size_t share = (size_t)f.R * row_bytes / (size_t)P;
+        const bool light = share < (size_t(512) << 10);
+        // The dense call streams every block: from about a third of a megabyte per CTA the idle SMs cost more than
+        // the ragged pieces (measured, 64 block-rows: 8192 x 28672 takes 28.5 us on 148 CTAs against 31.1 us on
+        // 128, 8192 x 16384 18.3 against 19.3 us, 8192 x 8192 11.7 against 11.2 us; the sparse calls, with half
+        // the bytes, stay better off on 128).
+        const bool heavy_dense = MODE == kModeDense && share >= (size_t(320) << 10);
+        if (small || (!heavy_dense && k * f.R * 100 >= (light ? 75 : 85) * P)) P = k * f.R;
     }
     // no more CTAs than pieces of at least 64 columns of one block-row
     const long long pieces = (long long)f.R * ((f.n + 63) / 64);
