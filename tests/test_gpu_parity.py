@@ -1108,3 +1108,47 @@ def test_kq_width_four_is_the_plain_format_and_other_widths_are_refused():
     assert binding.spqt_kqw_packed_sizes(512, 10, 8)[0] == 2 * 10 * 272
     assert binding.spqt_kqw_packed_sizes(512, 10, 5)[0] == 2 * 10 * 176
     assert binding.spqt_kqw_packed_sizes(512, 10, 6)[0] == 2 * 10 * 208
+
+
+@pytest.mark.parametrize("seed", [1, 2])
+def test_random_shapes_across_the_partition_regimes(seed):
+    """Seeded random cases over the regimes of the work map -- block-rows far below, near and above the SM count,
+    lists that fit the shared-memory window and lists that do not, every format, thresholds from 0 to 99 % -- through
+    the given-list, index-collecting and dense calls: lists bit-exact, the two sparse routes bit-identical, sampled
+    rows against the oracle."""
+    rng = np.random.default_rng(seed)
+    for it in range(12):
+        bits, group = GEMV_FORMATS[it % 4]
+        R = int(rng.choice([1, 2, 7, 31, 74, 147, 148, 149, 160, 223, 296, 300, 451, 1000]))
+        n = int(rng.choice([64, 777, 4096, 5000, 12288, 12289, 20001, 32768]))
+        if R * group * n > 3e8:
+            n = 4096
+        m = R * group
+        sp = float(rng.choice([0.0, 0.1, 0.5, 0.9, 0.99]))
+        torch.manual_seed(100 * seed + it)
+        Wd = (torch.randn(m, n, device="cuda") * 0.02).half()
+        x = inputs.activations(n, seed=1000 * seed + it)
+        t = inputs.threshold_for_sparsity(x, sp)
+        p = binding.spqt_pack(Wd, bits, group)
+        del Wd
+        ws = binding.new_workspace(m, n, bits, group)
+        xd = dev(x)
+        idx, cnt = binding.spqt_sparsify(xd, t)
+        y = binding.spqt_sparse_gemv(p, xd, idx, cnt, ws)
+        yf, idx2, cnt2 = binding.spqt_sparsify_gemv(p, xd, t, ws)
+        yd = binding.spqt_dense_gemv(p, xd, ws)
+        torch.cuda.synchronize()
+        what = "int%d g%d R=%d n=%d sparsity %.2f" % (bits, group, R, n, sp)
+        ref_idx, ref_cnt = oracle.sparsify(x, t)
+        assert int(cnt.item()) == ref_cnt and int(cnt2.item()) == ref_cnt, what
+        assert np.array_equal(idx.cpu().numpy()[:ref_cnt], ref_idx) and np.array_equal(idx2.cpu().numpy()[:ref_cnt], ref_idx), what
+        assert torch.equal(y.view(torch.int16), yf.view(torch.int16)), what
+        rows = np.unique(rng.integers(0, m, size=64))
+        codes, s, z = packed_to_host(p)
+        y_ref, bound = oracle.sparse_gemv(codes, s, z, m, n, x, ref_idx, bits, group, rows=rows)
+        check_y(y.cpu().numpy()[rows], y_ref, bound, what)
+        y_ref, bound = oracle.dense_gemv(codes, s, z, m, n, x, bits, group, rows=rows)
+        check_y(yd.cpu().numpy()[rows], y_ref, bound, what + " dense")
+        assert binding.spqt_workspace_status(ws, m, group) == 0, what
+        del p, ws
+        torch.cuda.empty_cache()
