@@ -1128,7 +1128,7 @@ static spqt_status launch_gemv(const Format& f, const void* codes, const void* m
     int P = tuned > 0 ? tuned : sms;
     if (tuned == 0 && f.R <= P) {
         // With few block-rows, a whole number of CTAs per block-row (if that keeps >= 85 % of the SMs
-        // busy; 75 % for light launches, below) gives every CTA a single segment: no CTA then carries two
+        // busy; 70 % for light launches, below) gives every CTA a single segment: no CTA then carries two
         // aggregation chains.
         int k = P / f.R;
         // A small matrix gains nothing from more than four CTAs per block-row: the combination of many
@@ -1137,9 +1137,10 @@ static spqt_status launch_gemv(const Format& f, const void* codes, const void* m
         const size_t row_bytes = (size_t)f.n * (size_t)(f.B + 4);
         const bool small = k > 4 && row_bytes / 4 < (size_t(256) << 10);
         if (small) k = 4;
-        // While a CTA's share stays under half a megabyte the launch is latency-bound, and leaving up to a
-        // quarter of the SMs idle costs less than partial sums that cross CTAs in a ragged pattern
-        // (measured: 14336 x 4096 on 112 CTAs, one block-row each, 8.9 us against 9.7 us on 148).
+        // While a CTA's share stays under half a megabyte the launch is latency-bound, and leaving up to 30 %
+        // of the SMs idle costs less than partial sums that cross CTAs in a ragged pattern
+        // (measured: 14336 x 4096 on 112 CTAs, one block-row each, 8.9 us against 9.7 us on 148; 13824 x 5120
+        // on 108 CTAs 8.7 against 9.6 us).
         const size_t share = (size_t)f.R * row_bytes / (size_t)P;
         const bool light = share < (size_t(512) << 10);
         // The dense call streams every block: from about a third of a megabyte per CTA the idle SMs cost more than
@@ -1147,7 +1148,7 @@ static spqt_status launch_gemv(const Format& f, const void* codes, const void* m
         // 128, 8192 x 16384 18.3 against 19.3 us, 8192 x 8192 11.7 against 11.2 us; the sparse calls, with half
         // the bytes, stay better off on 128).
         const bool heavy_dense = MODE == kModeDense && share >= (size_t(320) << 10);
-        if (small || (!heavy_dense && k * f.R * 100 >= (light ? 75 : 85) * P)) P = k * f.R;
+        if (small || (!heavy_dense && k * f.R * 100 >= (light ? 70 : 85) * P)) P = k * f.R;
     }
     // no more CTAs than pieces of at least 64 columns of one block-row
     const long long pieces = (long long)f.R * ((f.n + 63) / 64);
