@@ -1135,8 +1135,15 @@ static spqt_status launch_gemv(const Format& f, const void* codes, const void* m
         // partial sums then costs more than the extra CTAs save (measured: 1024 x 4096 takes 6.8 us on 144
         // CTAs, 4.9 us on 32).  "Small": under 256 KB of blocks per CTA at four CTAs per block-row.
         const size_t row_bytes = (size_t)f.n * (size_t)(f.B + 4);
-        const bool small = k > 4 && row_bytes / 4 < (size_t(256) << 10);
+        bool small = k > 4 && row_bytes / 4 < (size_t(256) << 10);
         if (small) k = 4;
+        // A block-row of under 96 KB is not worth cutting at all once there are 32 of them (measured:
+        // 4096 x 1024 takes 4.0 / 4.5 / 3.8 us -- given list, index collection inside, dense -- on 32 CTAs
+        // against 4.5 / 5.5 / 3.8 on 128; 8192 x 1024 4.1 / 4.6 / 3.8 on 64 against 4.8 / 5.5 / 4.2 on 128).
+        if (k > 1 && f.R >= 32 && row_bytes < (size_t(96) << 10)) {
+            k = 1;
+            small = true;
+        }
         // While a CTA's share stays under half a megabyte the launch is latency-bound, and leaving up to 30 %
         // of the SMs idle costs less than partial sums that cross CTAs in a ragged pattern
         // (measured: 14336 x 4096 on 112 CTAs, one block-row each, 8.9 us against 9.7 us on 148; 13824 x 5120
